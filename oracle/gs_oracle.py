@@ -1,0 +1,277 @@
+"""ctypes front end of the CPU oracle (``gs_oracle.cpp``).
+
+TEST INFRASTRUCTURE ONLY: imported by ``tests/``, by the smoke check and by the benchmark's
+``cpu_baseline`` / ``--impl reference`` legs.  The product path never imports it, and this
+module imports nothing from the CUDA package.
+
+Scenes and cameras are duck-typed: any object with the attributes ``means, log_scales, quats,
+opacity_logits, base_color, app, active_degree, sh_rest | features + mlp_weights`` and
+``width, height, fx, fy, cx, cy, w2c, near_plane, far_plane, background``.  All floating-point
+inputs are widened to float64 exactly (fp16 and fp32 are subsets of fp64).
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from types import SimpleNamespace
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "gs_oracle.cpp")
+_LIB = os.path.join(_HERE, "libgs_oracle.so")
+_lib = None
+
+TILE = 16
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with g++ (-O2, no FMA contraction, OpenMP)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["g++", "-std=c++17", "-O2", "-ffp-contract=off", "-fopenmp", "-fPIC", "-shared",
+               "-o", _LIB, _SRC]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def _p(a, t):
+    return a.ctypes.data_as(C.POINTER(t)) if a is not None else None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        build()
+        _lib = C.CDLL(_LIB)
+        _lib.gso_tile_rects_f32.restype = C.c_int64
+        _lib.gso_tile_rects_from_px.restype = C.c_int64
+        _lib.gso_num_mlp_weights.restype = C.c_int
+        _lib.gso_mlp_macs.restype = C.c_int
+    return _lib
+
+
+def num_threads() -> int:
+    """Threads the OpenMP loops use (all host cores unless OMP_NUM_THREADS says otherwise)."""
+    env = os.environ.get("OMP_NUM_THREADS")
+    return int(env) if env else (os.cpu_count() or 1)
+
+
+def _f64(a):
+    return None if a is None else np.ascontiguousarray(np.asarray(a), dtype=np.float64)
+
+
+def _dp(a):
+    return _p(a, C.c_double)
+
+
+def cam_array(cam) -> np.ndarray:
+    c = np.zeros(23, np.float64)
+    c[0], c[1] = cam.width, cam.height
+    c[2:6] = cam.fx, cam.fy, cam.cx, cam.cy
+    c[6:18] = np.asarray(cam.w2c, np.float64).reshape(12)
+    c[18], c[19] = cam.near_plane, cam.far_plane
+    c[20:23] = cam.background
+    return c
+
+
+# ------------------------------------------------------------------------------------------
+# thin wrappers, one per exported function
+# ------------------------------------------------------------------------------------------
+
+def sh_basis(d):
+    d = _f64(d); Y = np.zeros(16)
+    lib().gso_sh_basis(_dp(d), _dp(Y))
+    return Y
+
+
+def sh_basis_grad(d):
+    d = _f64(d); G = np.zeros((16, 3))
+    lib().gso_sh_basis_grad(_dp(d), _dp(G))
+    return G
+
+
+def quat_to_rot(q):
+    q = _f64(q); R = np.zeros((3, 3))
+    lib().gso_quat_to_rot(_dp(q), _dp(R))
+    return R
+
+
+def mlp_macs(fold: bool) -> int:
+    return lib().gso_mlp_macs(int(fold))
+
+
+def num_mlp_weights() -> int:
+    return lib().gso_num_mlp_weights()
+
+
+def preprocess(means, log_scales, quats, opacity_logits, cam):
+    means, log_scales, quats, logits = _f64(means), _f64(log_scales), _f64(quats), _f64(opacity_logits)
+    n = means.shape[0]
+    o = SimpleNamespace(
+        mean2d=np.zeros((n, 2)), cov2d=np.zeros((n, 3)), conic=np.zeros((n, 3)), opacity=np.zeros(n),
+        extent=np.zeros((n, 2)), depth32=np.zeros(n, np.float32), dir=np.zeros((n, 3)),
+        valid=np.zeros(n, np.uint8), visible=np.zeros(n, np.uint8), rect_px=np.zeros((n, 4), np.int32))
+    cam_a = cam_array(cam)
+    lib().gso_preprocess(C.c_int64(n), _dp(means), _dp(log_scales), _dp(quats), _dp(logits), _dp(cam_a),
+                         _dp(o.mean2d), _dp(o.cov2d), _dp(o.conic), _dp(o.opacity), _dp(o.extent),
+                         _p(o.depth32, C.c_float), _dp(o.dir), _p(o.valid, C.c_uint8),
+                         _p(o.visible, C.c_uint8), _p(o.rect_px, C.c_int32))
+    o.depth_bits = o.depth32.view(np.uint32)
+    return o
+
+
+def _app_args(scene):
+    sh = _f64(scene.sh_rest) if scene.app == 0 else None
+    ft = _f64(scene.features) if scene.app == 1 else None
+    wt = _f64(scene.mlp_weights) if scene.app == 1 else None
+    return _f64(scene.base_color), sh, ft, wt
+
+
+def appearance_forward(scene, dirs, mask=None, deg=None):
+    base, sh, ft, wt = _app_args(scene)
+    dirs = _f64(dirs); n = dirs.shape[0]
+    color, resid = np.zeros((n, 3)), np.zeros((n, 3))
+    deg = scene.active_degree if deg is None else deg
+    m = None if mask is None else np.ascontiguousarray(mask, np.uint8)
+    lib().gso_appearance_forward(C.c_int64(n), C.c_int(scene.app), C.c_int(deg), _dp(base), _dp(sh),
+                                 _dp(ft), _dp(wt), _dp(dirs), _p(m, C.c_uint8), _dp(color), _dp(resid))
+    return color, resid
+
+
+def appearance_backward(scene, dirs, g_color, mask=None, deg=None):
+    base, sh, ft, wt = _app_args(scene)
+    dirs, g_color = _f64(dirs), _f64(g_color); n = dirs.shape[0]
+    deg = scene.active_degree if deg is None else deg
+    m = None if mask is None else np.ascontiguousarray(mask, np.uint8)
+    o = SimpleNamespace(base_color=np.zeros((n, 3)), dirs=np.zeros((n, 3)), sh_rest=None,
+                        features=None, mlp_weights=None)
+    if scene.app == 0:
+        o.sh_rest = np.zeros((n, 15, 3))
+    else:
+        o.features = np.zeros((n, 8)); o.mlp_weights = np.zeros(num_mlp_weights())
+    lib().gso_appearance_backward(C.c_int64(n), C.c_int(scene.app), C.c_int(deg), _dp(base), _dp(sh),
+                                  _dp(ft), _dp(wt), _dp(dirs), _p(m, C.c_uint8), _dp(g_color),
+                                  _dp(o.base_color), _dp(o.sh_rest), _dp(o.features),
+                                  _dp(o.mlp_weights), _dp(o.dirs))
+    return o
+
+
+def tile_rects_f32(valid, mean2d_f32, extent_f32, width, height):
+    """Integer stage on fp32 per-Gaussian values (from either side)."""
+    valid = np.ascontiguousarray(valid, np.uint8)
+    m = np.ascontiguousarray(mean2d_f32, np.float32); e = np.ascontiguousarray(extent_f32, np.float32)
+    n = valid.shape[0]
+    rect = np.zeros((n, 4), np.int32); tt = np.zeros(n, np.uint32)
+    P = lib().gso_tile_rects_f32(C.c_int64(n), _p(valid, C.c_uint8), _p(m, C.c_float), _p(e, C.c_float),
+                                 C.c_int(width), C.c_int(height), _p(rect, C.c_int32), _p(tt, C.c_uint32))
+    return rect, tt, int(P)
+
+
+def tile_rects_from_px(visible, rect_px):
+    visible = np.ascontiguousarray(visible, np.uint8); rect_px = np.ascontiguousarray(rect_px, np.int32)
+    n = visible.shape[0]
+    rect = np.zeros((n, 4), np.int32); tt = np.zeros(n, np.uint32)
+    P = lib().gso_tile_rects_from_px(C.c_int64(n), _p(visible, C.c_uint8), _p(rect_px, C.c_int32),
+                                     _p(rect, C.c_int32), _p(tt, C.c_uint32))
+    return rect, tt, int(P)
+
+
+def sorted_instances(rect, depth_bits, width, height, P):
+    rect = np.ascontiguousarray(rect, np.int32); db = np.ascontiguousarray(depth_bits, np.uint32)
+    gx, gy = (width + TILE - 1) // TILE, (height + TILE - 1) // TILE
+    keys = np.zeros(P, np.uint64); vals = np.zeros(P, np.uint32)
+    ranges = np.zeros((gx * gy, 2), np.uint32)
+    lib().gso_sorted_instances(C.c_int64(rect.shape[0]), _p(rect, C.c_int32), _p(db, C.c_uint32),
+                               C.c_int(gx), C.c_int64(P), _p(keys, C.c_uint64), _p(vals, C.c_uint32))
+    lib().gso_tile_ranges(C.c_int64(P), _p(keys, C.c_uint64), C.c_int(gx * gy), _p(ranges, C.c_uint32))
+    return keys, vals, ranges
+
+
+def blend_forward(cam, vals, ranges, mean2d, conic, opacity, color):
+    W, H = cam.width, cam.height
+    bg = _f64(cam.background)
+    o = SimpleNamespace(image=np.zeros((3, H, W)), final_T=np.zeros((H, W)),
+                        n_contrib=np.zeros((H, W), np.uint32), fragile=np.zeros((H, W), np.uint8))
+    vals = np.ascontiguousarray(vals, np.uint32); ranges = np.ascontiguousarray(ranges, np.uint32)
+    lib().gso_blend_forward(C.c_int(W), C.c_int(H), _dp(bg), _p(vals, C.c_uint32), _p(ranges, C.c_uint32),
+                            _dp(_f64(mean2d)), _dp(_f64(conic)), _dp(_f64(opacity)), _dp(_f64(color)),
+                            _dp(o.image), _dp(o.final_T), _p(o.n_contrib, C.c_uint32),
+                            _p(o.fragile, C.c_uint8))
+    return o
+
+
+def blend_brute(cam, visible, depth_bits, mean2d, conic, opacity, color):
+    W, H = cam.width, cam.height
+    bg = _f64(cam.background)
+    image = np.zeros((3, H, W)); final_T = np.zeros((H, W))
+    visible = np.ascontiguousarray(visible, np.uint8); db = np.ascontiguousarray(depth_bits, np.uint32)
+    lib().gso_blend_brute(C.c_int64(visible.shape[0]), C.c_int(W), C.c_int(H), _dp(bg),
+                          _p(visible, C.c_uint8), _p(db, C.c_uint32), _dp(_f64(mean2d)), _dp(_f64(conic)),
+                          _dp(_f64(opacity)), _dp(_f64(color)), _dp(image), _dp(final_T))
+    return image, final_T
+
+
+def blend_backward(cam, vals, ranges, mean2d, conic, opacity, color, G, with_abs=False):
+    W, H = cam.width, cam.height
+    bg = _f64(cam.background)
+    n = np.asarray(opacity).shape[0]
+    vals = np.ascontiguousarray(vals, np.uint32); ranges = np.ascontiguousarray(ranges, np.uint32)
+    o = SimpleNamespace(color=np.zeros((n, 3)), opacity=np.zeros(n), conic=np.zeros((n, 3)),
+                        mean2d=np.zeros((n, 2)), abs_sum=np.zeros((n, 9)) if with_abs else None)
+    lib().gso_blend_backward(C.c_int64(n), C.c_int(W), C.c_int(H), _dp(bg), C.c_int64(vals.shape[0]),
+                             _p(vals, C.c_uint32), _p(ranges, C.c_uint32), _dp(_f64(mean2d)),
+                             _dp(_f64(conic)), _dp(_f64(opacity)), _dp(_f64(color)), _dp(_f64(G)),
+                             _dp(o.color), _dp(o.opacity), _dp(o.conic), _dp(o.mean2d), _dp(o.abs_sum))
+    return o
+
+
+def preprocess_backward(means, log_scales, quats, opacity_logits, cam, visible, g_mean2d, g_conic,
+                        g_opacity, g_dir):
+    means, log_scales, quats, logits = _f64(means), _f64(log_scales), _f64(quats), _f64(opacity_logits)
+    n = means.shape[0]
+    visible = np.ascontiguousarray(visible, np.uint8)
+    o = SimpleNamespace(means=np.zeros((n, 3)), log_scales=np.zeros((n, 3)), quats=np.zeros((n, 4)),
+                        opacity_logits=np.zeros(n))
+    cam_a = cam_array(cam)
+    lib().gso_preprocess_backward(C.c_int64(n), _dp(means), _dp(log_scales), _dp(quats), _dp(logits),
+                                  _dp(cam_a), _p(visible, C.c_uint8), _dp(_f64(g_mean2d)),
+                                  _dp(_f64(g_conic)), _dp(_f64(g_opacity)), _dp(_f64(g_dir)),
+                                  _dp(o.means), _dp(o.log_scales), _dp(o.quats), _dp(o.opacity_logits))
+    return o
+
+
+# ------------------------------------------------------------------------------------------
+# The whole path, composed in the paper's order: preprocess (projection + fused colour) ->
+# tile assignment -> sort -> blend -> blend backward -> appearance backward -> preprocess
+# backward.
+# ------------------------------------------------------------------------------------------
+
+def render_forward(scene, cam):
+    pre = preprocess(scene.means, scene.log_scales, scene.quats, scene.opacity_logits, cam)
+    color, resid = appearance_forward(scene, pre.dir, mask=pre.visible)
+    rect, tiles_touched, P = tile_rects_from_px(pre.visible, pre.rect_px)
+    keys, vals, ranges = sorted_instances(rect, pre.depth_bits, cam.width, cam.height, P)
+    bl = blend_forward(cam, vals, ranges, pre.mean2d, pre.conic, pre.opacity, color)
+    return SimpleNamespace(pre=pre, color=color, residual=resid, rect=rect, tiles_touched=tiles_touched,
+                           P=P, keys=keys, vals=vals, ranges=ranges, image=bl.image, final_T=bl.final_T,
+                           n_contrib=bl.n_contrib, fragile=bl.fragile)
+
+
+def render_backward(scene, cam, fwd, G, with_abs=False):
+    pre = fwd.pre
+    g2 = blend_backward(cam, fwd.vals, fwd.ranges, pre.mean2d, pre.conic, pre.opacity, fwd.color, G,
+                        with_abs=with_abs)
+    ga = appearance_backward(scene, pre.dir, g2.color, mask=pre.visible)
+    gp = preprocess_backward(scene.means, scene.log_scales, scene.quats, scene.opacity_logits, cam,
+                             pre.visible, g2.mean2d, g2.conic, g2.opacity, ga.dirs)
+    return SimpleNamespace(means=gp.means, log_scales=gp.log_scales, quats=gp.quats,
+                           opacity_logits=gp.opacity_logits, base_color=ga.base_color,
+                           sh_rest=ga.sh_rest, features=ga.features, mlp_weights=ga.mlp_weights,
+                           blend=g2, dirs=ga.dirs)
+
+
+def render(scene, cam, G=None, with_abs=False):
+    fwd = render_forward(scene, cam)
+    grads = render_backward(scene, cam, fwd, G, with_abs=with_abs) if G is not None else None
+    return fwd, grads
