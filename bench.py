@@ -1,0 +1,412 @@
+#!/usr/bin/env python
+"""Benchmark of the splatting training step (forward + backward, 8 views of a 1M-Gaussian scene).
+
+`python bench.py --gpus N --steps K --warmup W` prints ONE JSON line on rank 0.
+A "step" is one pass of the whole hot path over one batch: for each of the 8 orbit cameras,
+gs_preprocess -> gs_render_forward -> gs_render_backward on the 1M-Gaussian clustered scene
+(the 1M configuration of the benchmark list) with the neural appearance model; the SH model and
+the appearance-decode sweep are timed beside it and reported in extra keys.
+
+`--impl reference` times the CPU oracle (the plain double-precision restatement of the method) on
+the host cores on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "fwd+bwd rasterizer ms/iter @1M Gaussians; appearance-decode GB/s vs HBM peak"
+N_GAUSS, WIDTH, HEIGHT, VIEWS = 1_000_000, 1256, 828, 8
+
+# Algorithmic cost per unit: flops per evaluated list entry of the blend
+# kernels and bytes per Gaussian of the per-Gaussian kernels.
+BLEND_FWD_FLOPS_PER_ENTRY = 14.0
+BLEND_BWD_FLOPS_PER_ENTRY = 14.0
+FP32_LANES_PER_SM, NUM_SMS = 128, 148
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=float(p["hbm_gbs"]), sm_max_mhz=float(p.get("sm_max_mhz", 1965.0)), source="measured")
+    return dict(hbm_gbs=6650.0, sm_max_mhz=1965.0, source="fallback")
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples during the timed region."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.path = index, None, None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = dict(sm_mhz=None, sm_max_mhz=None, reasons=[], samples=0)
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in open(self.path):
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        os.unlink(self.path)
+        if sm:
+            sm.sort()
+            out.update(sm_mhz=sm[len(sm) // 2], sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def dist_setup(args):
+    rank = int(os.environ.get("RANK", "0")); world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+# ---------------------------------------------------------------------------------------------
+# our arm
+# ---------------------------------------------------------------------------------------------
+def run_ours(args):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    from paper_2609_05255_b200 import api, scenes
+
+    rank, world, local = dist_setup(args)
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    peaks = measured_peaks()
+    ctx = api.Context(local)
+    n, views = args.n, args.views
+    cams_host = scenes.orbit_cameras(WIDTH, HEIGHT, views)
+    cams = [api.make_camera(c) for c in cams_host]
+
+    def make_arm(app):
+        host = scenes.config3(app, n=n, width=WIDTH, height=HEIGHT, views=views).scene
+        ds = api.upload_scene(host, dev)
+        probe = api.alloc_projected(ds.n, dev, with_extent=False)
+        pairs = [api.gs_preprocess(ctx, ds, c, probe) for c in cams]
+        cap = int(max(pairs) * 1.02) + 1024
+        r = api.Renderer(ctx, ds.n, WIDTH, HEIGHT, app, pair_capacity=cap)
+        return host, ds, r, pairs
+
+    gen = torch.Generator(device=dev); gen.manual_seed(4242 + rank)
+    G = torch.randn((views, 3, HEIGHT, WIDTH), device=dev, generator=gen)
+
+    def step(ds, r):
+        for v in range(views):
+            r.forward(ds, cams[v])
+            r.backward(ds, cams[v], G[v])
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps, warmup):
+        for _ in range(warmup):
+            fn()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        barrier()
+        ms = e0.elapsed_time(e1) / steps
+        if world > 1:
+            t = torch.tensor([ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    def profile(fn, steps):
+        api.gs_profile_enable(ctx, True)
+        api.gs_profile_collect(ctx)
+        tot_ms, tot_l = {}, {}
+        for _ in range(steps):
+            fn()
+            ms, launches = api.gs_profile_collect(ctx)
+            for k in ms:
+                tot_ms[k] = tot_ms.get(k, 0.0) + ms[k]; tot_l[k] = tot_l.get(k, 0) + launches[k]
+        api.gs_profile_enable(ctx, False)
+        return {k: v / steps for k, v in tot_ms.items()}, {k: v / steps for k, v in tot_l.items()}
+
+    results = {}
+    sampler = ClockSampler(local)
+    clocks = None
+    for app, tag in ((scenes.APP_NEURAL, "neural"), (scenes.APP_SH, "sh")):
+        host, ds, r, pairs = make_arm(app)
+        if tag == "neural":
+            sampler.start()
+        ms = timed(lambda: step(ds, r), args.steps, args.warmup)
+        if tag == "neural":
+            clocks = sampler.stop()
+        stage_ms, stage_launches = profile(lambda: step(ds, r), max(1, min(args.steps, 3)))
+        # units of the blend kernels: list entries up to each pixel's last composited one, over the views
+        entries = 0
+        visible = 0
+        for v in range(views):
+            r.forward(ds, cams[v])
+            torch.cuda.synchronize()
+            entries += int(r.n_contrib.sum(dtype=torch.int64).item())
+            rect = r.proj.rect.to(torch.int32) & 0xFFFF
+            visible += int(((rect[:, 2] > rect[:, 0]) & (rect[:, 3] > rect[:, 1])).sum().item())
+        results[tag] = dict(ms=ms, stage_ms=stage_ms, stage_launches=stage_launches, pairs=pairs,
+                            entries=entries, visible=visible, host=host, ds=ds, r=r)
+
+    # ---- end to end through the public API with host buffers (neural arm)
+    e2e = measure_e2e(api, torch, ctx, results["neural"], cams, G, views, args, timed, dev)
+
+    # ---- appearance-decode sweep (separate-pass kernels, HBM resident)
+    decode = None if args.skip_decode else decode_sweep(api, torch, ctx, dev, peaks, args)
+
+    if rank != 0:
+        return
+    neural = results["neural"]
+    ms = neural["ms"]
+    stage_ms = neural["stage_ms"]
+    total_stage = sum(stage_ms.values()) or 1.0
+    dominant = max(stage_ms, key=stage_ms.get)
+    launches_per_step = int(round(sum(neural["stage_launches"].values())))
+    clock_mhz = peaks["sm_max_mhz"]
+    alu_peak = NUM_SMS * FP32_LANES_PER_SM * 2 * clock_mhz * 1e6 / 1e12   # TFLOP/s
+    roof = stage_roofline(dominant, neural, views, n, peaks, alu_peak)
+    out = {
+        "metric": METRIC, "value": ms / world, "unit": "ms/iter (8 views, fwd+bwd)", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": False,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "config3: 1M Gaussians (64 clusters + shell), 1256x828, 8 orbit views, "
+                               "neural appearance (8 fp16 features + shared 32-16-16-3 MLP), fwd+bwd",
+                   "n": n, "width": WIDTH, "height": HEIGHT, "views": views,
+                   "cache": "inputs_larger_than_L2 (per-view working set > 126 MB; 8 different cameras)",
+                   "multi_gpu": "replicas only"},
+        "gprimitives_per_s": world * n * views / (ms * 1e-3) / 1e9,
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step,
+        "roofline": roof,
+        "stages_ms_per_step": {k: round(v, 4) for k, v in stage_ms.items() if v > 0},
+        "stage_share": {k: round(v / total_stage, 4) for k, v in stage_ms.items() if v > 0},
+        "pairs_per_view": neural["pairs"], "visible_per_view": neural["visible"] / views,
+        "sh": {"ms_per_step": results["sh"]["ms"],
+               "stages_ms_per_step": {k: round(v, 4) for k, v in results["sh"]["stage_ms"].items() if v > 0}},
+        "appearance_decode": decode,
+        "peaks": peaks,
+    }
+    if not args.skip_cpu:
+        out["cpu_baseline"] = cpu_baseline(neural["host"], views, n)
+    print(json.dumps(out))
+
+
+def stage_roofline(stage, arm, views, n, peaks, alu_peak):
+    ms = arm["stage_ms"][stage] / views          # average duration of one launch of the stage
+    if stage in ("blend_fwd", "blend_bwd"):
+        per = BLEND_FWD_FLOPS_PER_ENTRY if stage == "blend_fwd" else BLEND_BWD_FLOPS_PER_ENTRY
+        flops = per * arm["entries"] / views
+        achieved = flops / (ms * 1e-3) / 1e12
+        return {"kernel": stage, "bound": "alu", "achieved": achieved, "peak": alu_peak, "unit": "TFLOP/s",
+                "frac": achieved / alu_peak, "traffic": None, "peak_source": "148 SMs x 128 lanes x 2 x max SM clock",
+                "units_per_launch": arm["entries"] / views, "flops_per_unit": per}
+    vis = arm["visible"] / views
+    app_bytes = 28.0
+    per_launch = {"preprocess_fwd": 44.0 * n + 12.0 * n + (app_bytes + 48.0) * vis,
+                  "preprocess_bwd": 8.0 * n + (44.0 + 48.0 + app_bytes) * vis + 88.0 * n,
+                  "depth_sort": (4 * 20.0 - 4.0) * n,
+                  "tile_sort": 2 * 20.0 * (sum(arm["pairs"]) / views),
+                  "keygen": 12.0 * n + 8.0 * (sum(arm["pairs"]) / views)}.get(stage, 0.0)
+    achieved = per_launch / (ms * 1e-3) / 1e9
+    return {"kernel": stage, "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+            "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"]}
+
+
+def measure_e2e(api, torch, ctx, arm, cams, G, views, args, timed, dev):
+    """Same step, but the scene parameters and upstream gradients start in pinned host memory and the
+    image and every gradient buffer end there: host<->device copies are inside the timed region."""
+    host, ds, r = arm["host"], arm["ds"], arm["r"]
+    pin = lambda t: t.cpu().pin_memory()
+    names = ["means", "log_scales", "quats", "opacity_logits", "base_color", "features", "mlp_weights"]
+    h_scene = {k: pin(getattr(ds, k)) for k in names}
+    h_G = pin(G)
+    g = r.grads
+    gnames = ["means", "log_scales", "quats", "opacity_logits", "base_color", "features", "mlp_weights"]
+    h_grads = {k: torch.empty_like(getattr(g, k), device="cpu").pin_memory() for k in gnames}
+    h_image = torch.empty_like(r.image, device="cpu").pin_memory()
+    d_G = torch.empty_like(G[0])
+    h2d = sum(t.numel() * t.element_size() for t in h_scene.values()) + views * d_G.numel() * 4
+    d2h = views * (sum(t.numel() * t.element_size() for t in h_grads.values()) + h_image.numel() * 4)
+
+    def step():
+        for k in names:
+            getattr(ds, k).copy_(h_scene[k], non_blocking=True)
+        for v in range(views):
+            d_G.copy_(h_G[v], non_blocking=True)
+            r.forward(ds, cams[v])
+            r.backward(ds, cams[v], d_G)
+            h_image.copy_(r.image, non_blocking=True)
+            for k in gnames:
+                h_grads[k].copy_(getattr(g, k), non_blocking=True)
+
+    ms = timed(step, max(2, args.steps // 2), 2)
+    return {"value": ms, "unit": "ms/iter (8 views, fwd+bwd)", "h2d_bytes_per_step": int(h2d),
+            "d2h_bytes_per_step": int(d2h)}
+
+
+def decode_sweep(api, torch, ctx, dev, peaks, args):
+    """Separate-pass colour decode forward + backward at 1M / 3M / 10M Gaussians, SH vs neural."""
+    out = {}
+    sizes = [1_000_000, 3_000_000, 10_000_000] if not args.quick else [1_000_000]
+    for n in sizes:
+        gen = torch.Generator(device=dev); gen.manual_seed(5000 + n % 997)
+        dirs = torch.randn((n, 3), device=dev, generator=gen)
+        dirs = (dirs / dirs.norm(dim=1, keepdim=True)).contiguous()
+        gcol = torch.randn((n, 3), device=dev, generator=gen)
+        base = 0.14 + 0.03 * torch.randn((n, 3), device=dev, generator=gen)
+        z = torch.zeros((1, 4), device=dev)
+        for app, tag in ((0, "sh"), (1, "neural")):
+            if app == 0:
+                sc = api.DeviceScene(z, z, z, z[0], base, 0, 3, sh_rest=0.05 * torch.randn((n, 15, 3), device=dev, generator=gen))
+                bytes_fwd, bytes_bwd = 192 + 12 + 12, 12 + 192 + 12 + 192 + 12 + 12
+            else:
+                w = (torch.rand((816,), device=dev, generator=gen) - 0.5).half()
+                sc = api.DeviceScene(z, z, z, z[0], base, 1, 3,
+                                     features=(0.1 * torch.randn((n, 8), device=dev, generator=gen)).half(), mlp_weights=w)
+                bytes_fwd, bytes_bwd = 28 + 12 + 12, 12 + 12 + 28 + 12 + 32 + 12
+            color = torch.empty((n, 3), device=dev)
+            grads = api.alloc_grads(n, app, dev)
+            gd = torch.empty((n, 3), device=dev)
+            flush = torch.empty((256 << 20,), device=dev, dtype=torch.uint8)
+
+            def run(fn, reps=10):
+                ts = []
+                for i in range(reps + 3):
+                    flush.zero_()                      # evict L2 between iterations
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record(); fn(); e1.record()
+                    torch.cuda.synchronize()
+                    if i >= 3:
+                        ts.append(e0.elapsed_time(e1))
+                ts.sort()
+                return ts[len(ts) // 2]
+            f_ms = run(lambda: api.gs_appearance_forward(ctx, sc, dirs, color))
+            b_ms = run(lambda: api.gs_appearance_backward(ctx, sc, dirs, gcol, grads, gd))
+            gbs = (bytes_fwd + bytes_bwd) * n / ((f_ms + b_ms) * 1e-3) / 1e9
+            out[f"{tag}_{n // 1_000_000}M"] = {
+                "fwd_ms": round(f_ms, 4), "bwd_ms": round(b_ms, 4), "bytes_per_primitive": bytes_fwd + bytes_bwd,
+                "GBps": round(gbs, 1), "frac_of_hbm_peak": round(gbs / peaks["hbm_gbs"], 4),
+                "fwd_GBps": round(bytes_fwd * n / (f_ms * 1e-3) / 1e9, 1),
+                "bwd_GBps": round(bytes_bwd * n / (b_ms * 1e-3) / 1e9, 1),
+                "Gprimitives_per_s": round(n / ((f_ms + b_ms) * 1e-3) / 1e9, 3)}
+            del sc, color, grads, gd, flush
+        del dirs, gcol, base
+        torch.cuda.empty_cache()
+    out["cache"] = "L2 flushed between iterations (256 MiB write)"
+    return out
+
+
+# ---------------------------------------------------------------------------------------------
+# the oracle on the host cores (cpu_baseline leg and --impl reference)
+# ---------------------------------------------------------------------------------------------
+def oracle_view_ms(host_scene, cam, G):
+    from oracle import gs_oracle
+    t0 = time.perf_counter()
+    gs_oracle.render(host_scene, cam, G)
+    return (time.perf_counter() - t0) * 1e3
+
+
+def cpu_baseline(host_scene, views, n):
+    from oracle import gs_oracle
+    from paper_2609_05255_b200 import scenes
+    gs_oracle.build()
+    cams = scenes.orbit_cameras(WIDTH, HEIGHT, views)
+    G = scenes.upstream_gradient(cams[0], 4242)
+    ms = oracle_view_ms(host_scene, cams[0], G)
+    return {"value": ms * views, "unit": "ms/iter (8 views, fwd+bwd)", "cores": gs_oracle.num_threads(),
+            "kind": "oracle", "sample": f"1 of {views} views of the full {n}-Gaussian scene, fwd+bwd, scaled x{views}"}
+
+
+def run_reference(args):
+    rank, world, _ = dist_setup(args)
+    if rank != 0:
+        return
+    from oracle import gs_oracle
+    from paper_2609_05255_b200 import scenes
+    gs_oracle.build()
+    views, n = args.views, args.n
+    host = scenes.config3(scenes.APP_NEURAL, n=n, width=WIDTH, height=HEIGHT, views=views).scene
+    cams = scenes.orbit_cameras(WIDTH, HEIGHT, views)
+    Gs = [scenes.upstream_gradient(cams[0], 4242)]
+    for _ in range(args.warmup):
+        oracle_view_ms(host, cams[0], Gs[0])
+    t = [oracle_view_ms(host, cams[k % views], Gs[0]) for k in range(args.steps)]
+    ms = sum(t) / len(t) * views
+    sample = f"each step = 1 of {views} views of the full {n}-Gaussian scene, fwd+bwd, scaled x{views}"
+    out = {"impl": "reference", "metric": METRIC, "value": ms, "unit": "ms/iter (8 views, fwd+bwd)",
+           "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+           "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+           "config": {"workload": "config3: 1M Gaussians (64 clusters + shell), 1256x828, 8 orbit views, "
+                                  "neural appearance, fwd+bwd", "n": n, "width": WIDTH, "height": HEIGHT,
+                      "views": views},
+           "cpu_baseline": {"value": ms, "unit": "ms/iter (8 views, fwd+bwd)", "cores": gs_oracle.num_threads(),
+                            "kind": "oracle", "sample": sample},
+           "e2e": {"value": ms, "unit": "ms/iter (8 views, fwd+bwd)", "h2d_bytes_per_step": 0,
+                   "d2h_bytes_per_step": 0},
+           "gpu_launches": 0}
+    print(json.dumps(out))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--n", type=int, default=N_GAUSS)
+    ap.add_argument("--views", type=int, default=VIEWS)
+    ap.add_argument("--quick", action="store_true", help="decode sweep at 1M only")
+    ap.add_argument("--skip-decode", action="store_true")
+    ap.add_argument("--skip-cpu", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,195 @@
+/*
+ * gs.h - C ABI of the B200 (sm_100a) differentiable Gaussian-splatting step with fused
+ * view-dependent appearance.
+ *
+ * The library implements one training-step hot path: per-Gaussian preprocess (projection to the
+ * image plane, 16x16 tile overlap, view-dependent colour), tile/depth ordering, per-tile
+ * front-to-back alpha blending, and the backward pass to every per-Gaussian parameter and to
+ * the shared decoder weights (Sec. 3.1 "Appearance Modelling in Gaussian Splatting", Sec. 4
+ * "Neural View-Dependent Appearance" and its "CUDA Implementation" paragraph).
+ *
+ * Conventions
+ *   - Every pointer in GsScene / GsProjected / GsBinning / GsGrads and every `float *` / `void *`
+ *     argument is a DEVICE pointer owned by the caller, contiguous, 16-byte aligned, unless the
+ *     comment says "host".  The structs themselves live in host memory.
+ *   - The library allocates nothing per call.  Work is enqueued on the caller's stream
+ *     (`stream` is a cudaStream_t passed as void*; NULL = the legacy default stream).
+ *   - Outputs are overwritten, never accumulated into.
+ *   - Every call returns a GsStatus; no exception, device trap or device assert crosses the
+ *     boundary.  gs_last_error() gives a text for the last failure on that context.
+ *   - Camera frame: +x right, +y down, +z forward; pixel (i, j) has its centre at (i+0.5, j+0.5).
+ *   - Non-finite values in a Gaussian's inputs cull that Gaussian (defined behaviour).
+ */
+#ifndef GS_B200_H_
+#define GS_B200_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct GsContext GsContext;
+
+typedef enum {
+  GS_OK = 0,
+  GS_ERR_INVALID_ARG = -1, /* NULL / misaligned pointer, n < 0, bad image size, bad degree ... */
+  GS_ERR_CAPACITY = -2,    /* pair count exceeds pair_capacity or workspace too small          */
+  GS_ERR_CUDA = -3,        /* a CUDA runtime call failed; see gs_last_error                    */
+  GS_ERR_UNSUPPORTED = -4,
+  GS_ERR_INTERNAL = -6
+} GsStatus;
+
+typedef enum { GS_APP_SH = 0, GS_APP_NEURAL = 1 } GsAppearance;
+
+enum {
+  GS_TILE = 16,            /* tile edge in pixels (Sec. 3.1)                                    */
+  GS_SH_REST = 45,         /* view-dependent SH coefficients per Gaussian, degrees 1..3, x RGB  */
+  GS_NUM_FEATURES = 8,     /* F, latent features per Gaussian (Sec. 4)                          */
+  GS_MLP_IN = 32,          /* D = 16 direction encodings + 16 feature encodings (Eq. 5)         */
+  GS_MLP_HIDDEN = 16,
+  GS_MLP_OUT = 3,
+  GS_MLP_WEIGHTS = 816     /* 32*16 + 16*16 + 16*3, no biases (Sec. 4)                          */
+};
+
+/* Pinhole camera (host struct). */
+typedef struct {
+  int32_t width, height;        /* pixels                                                      */
+  float fx, fy, cx, cy;         /* intrinsics in pixel units                                   */
+  float w2c[12];                /* row-major [R|t]: x_cam = R x_world + t                      */
+  float near_plane, far_plane;  /* depth cull, typically 0.2 and 1e10                          */
+  float background[3];          /* constant RGB composited behind everything                   */
+} GsCamera;
+
+/* The scene: per-Gaussian parameters plus the shared decoder (host struct of device pointers). */
+typedef struct {
+  int64_t n;                     /* number of Gaussians, >= 0                                  */
+  const float *means;            /* [n,3]                                                      */
+  const float *log_scales;       /* [n,3]   scale = exp(log_scale)                             */
+  const float *quats;            /* [n,4]   (w,x,y,z), normalised inside                       */
+  const float *opacity_logits;   /* [n]     opacity = sigmoid(logit)                           */
+  const float *base_color;       /* [n,3]   c0 of Eq. 2 (the constant Y0 is folded in)         */
+  int32_t app;                   /* GsAppearance                                               */
+  int32_t active_degree;         /* 0..3: direction bands in use (progressive schedule, Sec. 4);
+                                    0 disables the view-dependent residual                     */
+  const float *sh_rest;          /* SH only:     [n,15,3] bands 1..3, RGB innermost (Eq. 1)    */
+  const uint16_t *features;      /* neural only: [n,8] IEEE fp16 bit patterns (Sec. 4)         */
+  const uint16_t *mlp_weights;   /* neural only: [816] fp16: W1[16][32], W2[16][16], W3[3][16],
+                                    each row-major (out, in); input order = 16 SH basis values
+                                    of the direction, then (sin f_j, cos f_j) per feature
+                                    (Eq. 5, Eq. 6 with k = 1)                                  */
+} GsScene;
+
+/* Per-Gaussian results of gs_preprocess (caller-allocated device buffers). */
+typedef struct {
+  float *mean2d;         /* [n,2]  projected centre in pixels                                  */
+  float *conic_opacity;  /* [n,4]  inverse 2D covariance (A,B,C) and opacity                    */
+  float *color;          /* [n,3]  decoded view-dependent colour (Eq. 2)                       */
+  uint32_t *depth_key;   /* [n]    bit pattern of the fp32 camera depth; 0xFFFFFFFF if culled  */
+  uint16_t *rect;        /* [n,4]  tile rectangle (tx0, ty0, tx1, ty1), half open; all zero if
+                                   the Gaussian touches no tile                                */
+  float *extent;         /* [n,2]  optional (may be NULL): half-size in pixels of the box that
+                                   bounds alpha >= 1/255; (-1,-1) if culled before the box test */
+} GsProjected;
+
+/* Tile binning produced by gs_render_forward (caller-allocated device buffers). */
+typedef struct {
+  uint32_t *depth_order;   /* [n]             Gaussian ids by (depth_key, id) ascending        */
+  uint32_t *sorted_tiles;  /* [pair_capacity] tile id of each instance, ascending              */
+  uint32_t *sorted_vals;   /* [pair_capacity] Gaussian id of each instance; inside a tile by
+                                              (depth_key, id) ascending                        */
+  uint32_t *tile_ranges;   /* [tiles,2]       [start,end) into the sorted lists, tiles =
+                                              ceil(W/16)*ceil(H/16), row-major                 */
+} GsBinning;
+
+/* Gradients (caller-allocated device buffers, fp32, dense, exact zeros for culled Gaussians). */
+typedef struct {
+  float *means;           /* [n,3]                                                             */
+  float *log_scales;      /* [n,3]                                                             */
+  float *quats;           /* [n,4]  with respect to the un-normalised quaternion               */
+  float *opacity_logits;  /* [n]                                                               */
+  float *base_color;      /* [n,3]                                                             */
+  float *sh_rest;         /* SH:     [n,15,3]                                                  */
+  float *features;        /* neural: [n,8] fp32                                                */
+  float *mlp_weights;     /* neural: [816] fp32, summed over all visible Gaussians             */
+} GsGrads;
+
+/* Create / destroy a context on CUDA device `device`.  The context owns a few KB of device and
+ * pinned host memory (counters, the decoder-gradient partial sums).  Not thread safe: use one
+ * context per host thread.  Returns GS_ERR_CUDA if the device cannot be used. */
+GsStatus gs_create(int device, GsContext **ctx);
+void gs_destroy(GsContext *ctx);
+const char *gs_last_error(const GsContext *ctx);
+
+/* Bytes of scratch the render calls need for n Gaussians, a width x height image and at most
+ * pair_capacity (Gaussian, tile) instances.  0 on invalid arguments. */
+size_t gs_workspace_bytes(int64_t n, int32_t width, int32_t height, int64_t pair_capacity);
+
+/* Preprocess (Sec. 3.1; fused appearance: Sec. 4 "CUDA Implementation").  For every Gaussian:
+ * cull, project (EWA), bound the alpha >= 1/255 footprint by a tile rectangle, and decode the
+ * view-dependent colour for the direction camera centre -> mean (SH: Eq. 1-2; neural:
+ * Eq. 5-7).  Writes all of `out` and the total instance count to *num_pairs_host (host
+ * pointer; the call synchronises the stream once to read it).  n = 0 is valid. */
+GsStatus gs_preprocess(GsContext *ctx, const GsScene *scene, const GsCamera *cam, GsProjected *out,
+                       int64_t *num_pairs_host, void *stream);
+
+/* Tile assignment, ordering and blending (Sec. 3.1, blend kernel).  Orders the visible
+ * Gaussians by depth, emits one instance per (Gaussian, tile), orders instances by tile keeping
+ * the depth order, records per-tile ranges, then composites every pixel front to back:
+ * alpha = min(0.99, o exp(-0.5 d^T Q d)), skipped below 1/255, stop before transmittance would
+ * fall below 1e-4.  image [3,H,W], final_T [H,W] (transmittance left), n_contrib [H,W] (1 + list
+ * position of the last composited instance).  GS_ERR_CAPACITY, with nothing written, if
+ * num_pairs > pair_capacity or the workspace is smaller than gs_workspace_bytes(). */
+GsStatus gs_render_forward(GsContext *ctx, int64_t n, const GsProjected *proj, const GsCamera *cam,
+                           int64_t num_pairs, int64_t pair_capacity, GsBinning *bin, float *image,
+                           float *final_T, uint32_t *n_contrib, void *workspace,
+                           size_t workspace_bytes, void *stream);
+
+/* Backward of the blend and of the preprocess, appearance included (Sec. 4 "CUDA
+ * Implementation": the directional colour gradient also reaches the means).  dL_dimage is
+ * [3,H,W].  Fills every member of `grads` that applies to scene->app.  Uses the same workspace
+ * (contents of the forward call are not needed). */
+GsStatus gs_render_backward(GsContext *ctx, const GsScene *scene, const GsCamera *cam,
+                            const GsProjected *proj, const GsBinning *bin, int64_t num_pairs,
+                            const float *final_T, const uint32_t *n_contrib, const float *dL_dimage,
+                            GsGrads *grads, void *workspace, size_t workspace_bytes, void *stream);
+
+/* The separate-pass appearance path (Sec. 4 "CUDA Implementation", reference path; App. B.2):
+ * colour decode for given unit directions dirs [n,3] without the rasterizer, and its backward.
+ * Only the appearance members of `scene` are read.  color [n,3].  gs_appearance_backward fills
+ * grads->base_color, grads->sh_rest or grads->features + grads->mlp_weights, and dL_ddirs
+ * [n,3] (gradient with respect to the direction as a free vector). */
+GsStatus gs_appearance_forward(GsContext *ctx, const GsScene *scene, const float *dirs, float *color,
+                               void *stream);
+GsStatus gs_appearance_backward(GsContext *ctx, const GsScene *scene, const float *dirs,
+                                const float *dL_dcolor, GsGrads *grads, float *dL_ddirs,
+                                void *stream);
+
+/* Per-stage device timing, for benchmarks (the paper gives wall-clock protocols only, App. C; this
+ * is the measurement hook of this library).  While enabled, every stage the library launches is
+ * bracketed by CUDA events on the caller's stream.  gs_profile_collect synchronises those events,
+ * ADDS the elapsed milliseconds and the kernel-launch counts since the last collect into
+ * ms[GS_NUM_STAGES] / launches[GS_NUM_STAGES] (host arrays, either may be NULL) and forgets them.
+ * At most 4096 stage records are kept between two collects; further ones are dropped. */
+typedef enum {
+  GS_STAGE_PREPROCESS_FWD = 0, /* projection + fused colour decode                              */
+  GS_STAGE_DEPTH_SORT,         /* radix sort of the Gaussians by depth key                      */
+  GS_STAGE_TILE_OFFSETS,       /* prefix sum of tiles touched, in depth order                   */
+  GS_STAGE_KEYGEN,             /* instance emission                                             */
+  GS_STAGE_TILE_SORT,          /* radix sort of the instances by tile id                        */
+  GS_STAGE_TILE_RANGES,
+  GS_STAGE_BLEND_FWD,
+  GS_STAGE_BLEND_BWD,
+  GS_STAGE_PREPROCESS_BWD,     /* projection backward + fused appearance backward               */
+  GS_STAGE_APPEARANCE_FWD,     /* separate-pass decode                                          */
+  GS_STAGE_APPEARANCE_BWD,
+  GS_NUM_STAGES
+} GsStage;
+GsStatus gs_profile_enable(GsContext *ctx, int enable);
+GsStatus gs_profile_collect(GsContext *ctx, double *ms, int64_t *launches);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GS_B200_H_ */

@@ -1,0 +1,349 @@
+"""Thin ctypes binding of ``libgs_b200.so`` (the C ABI declared in ``include/gs.h``).
+
+Argument marshalling only: every step of the path runs in the CUDA kernels of the library.
+PyTorch supplies device memory and streams.  There is no CPU fallback: importing this module
+fails loudly if the shared library has not been built (``python -m paper_2609_05255_b200.build``).
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libgs_b200.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2609_05255_b200.build` "
+                      "(there is no fallback path)")
+_lib = C.CDLL(LIB_PATH)
+
+GS_OK, GS_ERR_INVALID_ARG, GS_ERR_CAPACITY, GS_ERR_CUDA, GS_ERR_UNSUPPORTED, GS_ERR_INTERNAL = 0, -1, -2, -3, -4, -6
+GS_APP_SH, GS_APP_NEURAL = 0, 1
+TILE = 16
+MLP_WEIGHTS = 816
+
+_vp = C.c_void_p
+
+
+class GsCamera(C.Structure):
+    _fields_ = [("width", C.c_int32), ("height", C.c_int32), ("fx", C.c_float), ("fy", C.c_float),
+                ("cx", C.c_float), ("cy", C.c_float), ("w2c", C.c_float * 12), ("near_plane", C.c_float),
+                ("far_plane", C.c_float), ("background", C.c_float * 3)]
+
+
+class GsScene(C.Structure):
+    _fields_ = [("n", C.c_int64), ("means", _vp), ("log_scales", _vp), ("quats", _vp), ("opacity_logits", _vp),
+                ("base_color", _vp), ("app", C.c_int32), ("active_degree", C.c_int32), ("sh_rest", _vp),
+                ("features", _vp), ("mlp_weights", _vp)]
+
+
+class GsProjected(C.Structure):
+    _fields_ = [("mean2d", _vp), ("conic_opacity", _vp), ("color", _vp), ("depth_key", _vp), ("rect", _vp),
+                ("extent", _vp)]
+
+
+class GsBinning(C.Structure):
+    _fields_ = [("depth_order", _vp), ("sorted_tiles", _vp), ("sorted_vals", _vp), ("tile_ranges", _vp)]
+
+
+class GsGrads(C.Structure):
+    _fields_ = [("means", _vp), ("log_scales", _vp), ("quats", _vp), ("opacity_logits", _vp), ("base_color", _vp),
+                ("sh_rest", _vp), ("features", _vp), ("mlp_weights", _vp)]
+
+
+_lib.gs_create.argtypes = [C.c_int, C.POINTER(_vp)]
+_lib.gs_create.restype = C.c_int
+_lib.gs_destroy.argtypes = [_vp]
+_lib.gs_destroy.restype = None
+_lib.gs_last_error.argtypes = [_vp]
+_lib.gs_last_error.restype = C.c_char_p
+_lib.gs_workspace_bytes.argtypes = [C.c_int64, C.c_int32, C.c_int32, C.c_int64]
+_lib.gs_workspace_bytes.restype = C.c_size_t
+_lib.gs_preprocess.argtypes = [_vp, C.POINTER(GsScene), C.POINTER(GsCamera), C.POINTER(GsProjected),
+                               C.POINTER(C.c_int64), _vp]
+_lib.gs_preprocess.restype = C.c_int
+_lib.gs_render_forward.argtypes = [_vp, C.c_int64, C.POINTER(GsProjected), C.POINTER(GsCamera), C.c_int64,
+                                   C.c_int64, C.POINTER(GsBinning), _vp, _vp, _vp, _vp, C.c_size_t, _vp]
+_lib.gs_render_forward.restype = C.c_int
+_lib.gs_render_backward.argtypes = [_vp, C.POINTER(GsScene), C.POINTER(GsCamera), C.POINTER(GsProjected),
+                                    C.POINTER(GsBinning), C.c_int64, _vp, _vp, _vp, C.POINTER(GsGrads), _vp,
+                                    C.c_size_t, _vp]
+_lib.gs_render_backward.restype = C.c_int
+_lib.gs_appearance_forward.argtypes = [_vp, C.POINTER(GsScene), _vp, _vp, _vp]
+_lib.gs_appearance_forward.restype = C.c_int
+_lib.gs_appearance_backward.argtypes = [_vp, C.POINTER(GsScene), _vp, _vp, C.POINTER(GsGrads), _vp, _vp]
+_lib.gs_appearance_backward.restype = C.c_int
+
+
+STAGES = ["preprocess_fwd", "depth_sort", "tile_offsets", "keygen", "tile_sort", "tile_ranges", "blend_fwd",
+          "blend_bwd", "preprocess_bwd", "appearance_fwd", "appearance_bwd"]
+_lib.gs_profile_enable.argtypes = [_vp, C.c_int]
+_lib.gs_profile_enable.restype = C.c_int
+_lib.gs_profile_collect.argtypes = [_vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
+_lib.gs_profile_collect.restype = C.c_int
+
+
+class GsError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"gs status {status}: {message}")
+        self.status = status
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "device pointers must come from contiguous CUDA tensors"
+    return t.data_ptr()
+
+
+def _stream_handle(stream) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream
+
+
+def make_camera(cam) -> GsCamera:
+    """Any object with width, height, fx, fy, cx, cy, w2c[3,4], near_plane, far_plane, background."""
+    c = GsCamera()
+    c.width, c.height = int(cam.width), int(cam.height)
+    c.fx, c.fy, c.cx, c.cy = float(cam.fx), float(cam.fy), float(cam.cx), float(cam.cy)
+    c.w2c = (C.c_float * 12)(*np.asarray(cam.w2c, np.float32).reshape(12).tolist())
+    c.near_plane, c.far_plane = float(cam.near_plane), float(cam.far_plane)
+    c.background = (C.c_float * 3)(*[float(v) for v in cam.background])
+    return c
+
+
+@dataclass
+class DeviceScene:
+    """The scene's tensors on the device (fp32; features / weights fp16)."""
+    means: torch.Tensor
+    log_scales: torch.Tensor
+    quats: torch.Tensor
+    opacity_logits: torch.Tensor
+    base_color: torch.Tensor
+    app: int
+    active_degree: int
+    sh_rest: Optional[torch.Tensor] = None
+    features: Optional[torch.Tensor] = None
+    mlp_weights: Optional[torch.Tensor] = None
+
+    @property
+    def n(self) -> int:
+        return int(self.base_color.shape[0])
+
+    def c_struct(self) -> GsScene:
+        s = GsScene()
+        s.n = self.n
+        s.means, s.log_scales, s.quats = _ptr(self.means), _ptr(self.log_scales), _ptr(self.quats)
+        s.opacity_logits, s.base_color = _ptr(self.opacity_logits), _ptr(self.base_color)
+        s.app, s.active_degree = int(self.app), int(self.active_degree)
+        s.sh_rest, s.features, s.mlp_weights = _ptr(self.sh_rest), _ptr(self.features), _ptr(self.mlp_weights)
+        return s
+
+
+def upload_scene(scene, device="cuda") -> DeviceScene:
+    """Copy a host scene (numpy arrays, see scenes.Scene) to the device."""
+    def up(a, dtype):
+        return None if a is None else torch.from_numpy(np.ascontiguousarray(a)).to(device=device, dtype=dtype)
+    return DeviceScene(up(scene.means, torch.float32), up(scene.log_scales, torch.float32),
+                       up(scene.quats, torch.float32), up(scene.opacity_logits, torch.float32),
+                       up(scene.base_color, torch.float32), int(scene.app), int(scene.active_degree),
+                       up(scene.sh_rest, torch.float32), up(scene.features, torch.float16),
+                       up(scene.mlp_weights, torch.float16))
+
+
+@dataclass
+class Projected:
+    mean2d: torch.Tensor
+    conic_opacity: torch.Tensor
+    color: torch.Tensor
+    depth_key: torch.Tensor    # int32 storage holding the uint32 bit patterns
+    rect: torch.Tensor         # int16 storage holding uint16 tile coordinates, [n,4]
+    extent: Optional[torch.Tensor]
+
+    def c_struct(self) -> GsProjected:
+        p = GsProjected()
+        p.mean2d, p.conic_opacity, p.color = _ptr(self.mean2d), _ptr(self.conic_opacity), _ptr(self.color)
+        p.depth_key, p.rect, p.extent = _ptr(self.depth_key), _ptr(self.rect), _ptr(self.extent)
+        return p
+
+
+def alloc_projected(n: int, device, with_extent: bool = True) -> Projected:
+    m = max(n, 1)
+    f = dict(device=device, dtype=torch.float32)
+    return Projected(torch.empty((m, 2), **f), torch.empty((m, 4), **f), torch.empty((m, 3), **f),
+                     torch.empty((m,), device=device, dtype=torch.int32),
+                     torch.empty((m, 4), device=device, dtype=torch.int16),
+                     torch.empty((m, 2), **f) if with_extent else None)
+
+
+@dataclass
+class Binning:
+    depth_order: torch.Tensor
+    sorted_tiles: torch.Tensor
+    sorted_vals: torch.Tensor
+    tile_ranges: torch.Tensor
+
+    def c_struct(self) -> GsBinning:
+        b = GsBinning()
+        b.depth_order, b.sorted_tiles = _ptr(self.depth_order), _ptr(self.sorted_tiles)
+        b.sorted_vals, b.tile_ranges = _ptr(self.sorted_vals), _ptr(self.tile_ranges)
+        return b
+
+
+def alloc_binning(n: int, pair_capacity: int, width: int, height: int, device) -> Binning:
+    tiles = ((width + TILE - 1) // TILE) * ((height + TILE - 1) // TILE)
+    i = dict(device=device, dtype=torch.int32)
+    return Binning(torch.empty((max(n, 1),), **i), torch.empty((max(pair_capacity, 1),), **i),
+                   torch.empty((max(pair_capacity, 1),), **i), torch.empty((tiles, 2), **i))
+
+
+@dataclass
+class Grads:
+    means: torch.Tensor
+    log_scales: torch.Tensor
+    quats: torch.Tensor
+    opacity_logits: torch.Tensor
+    base_color: torch.Tensor
+    sh_rest: Optional[torch.Tensor] = None
+    features: Optional[torch.Tensor] = None
+    mlp_weights: Optional[torch.Tensor] = None
+
+    def c_struct(self) -> GsGrads:
+        g = GsGrads()
+        g.means, g.log_scales, g.quats = _ptr(self.means), _ptr(self.log_scales), _ptr(self.quats)
+        g.opacity_logits, g.base_color = _ptr(self.opacity_logits), _ptr(self.base_color)
+        g.sh_rest, g.features, g.mlp_weights = _ptr(self.sh_rest), _ptr(self.features), _ptr(self.mlp_weights)
+        return g
+
+
+def alloc_grads(n: int, app: int, device) -> Grads:
+    m = max(n, 1)
+    f = dict(device=device, dtype=torch.float32)
+    g = Grads(torch.empty((m, 3), **f), torch.empty((m, 3), **f), torch.empty((m, 4), **f),
+              torch.empty((m,), **f), torch.empty((m, 3), **f))
+    if app == GS_APP_SH:
+        g.sh_rest = torch.empty((m, 15, 3), **f)
+    else:
+        g.features = torch.empty((m, 8), **f)
+        g.mlp_weights = torch.empty((MLP_WEIGHTS,), **f)
+    return g
+
+
+class Context:
+    """Owner of one GsContext (gs_create / gs_destroy)."""
+
+    def __init__(self, device: int = 0):
+        if not torch.cuda.is_available():
+            raise RuntimeError("a CUDA device is required: this library has no CPU path")
+        self.device = torch.device("cuda", device)
+        h = _vp()
+        st = _lib.gs_create(device, C.byref(h))
+        if st != GS_OK:
+            raise GsError(st, "gs_create failed")
+        self._h = h
+
+    def close(self):
+        if getattr(self, "_h", None):
+            _lib.gs_destroy(self._h)
+            self._h = None
+
+    __del__ = close
+
+    def _check(self, st: int):
+        if st != GS_OK:
+            raise GsError(st, _lib.gs_last_error(self._h).decode())
+
+
+def gs_profile_enable(ctx: Context, enable: bool) -> None:
+    ctx._check(_lib.gs_profile_enable(ctx._h, int(enable)))
+
+
+def gs_profile_collect(ctx: Context):
+    """Returns ({stage: milliseconds}, {stage: kernel launches}) accumulated since the last collect."""
+    ms = (C.c_double * len(STAGES))()
+    launches = (C.c_int64 * len(STAGES))()
+    ctx._check(_lib.gs_profile_collect(ctx._h, ms, launches))
+    return dict(zip(STAGES, list(ms))), dict(zip(STAGES, list(launches)))
+
+
+def gs_workspace_bytes(n: int, width: int, height: int, pair_capacity: int) -> int:
+    return int(_lib.gs_workspace_bytes(n, width, height, pair_capacity))
+
+
+def gs_preprocess(ctx: Context, scene: DeviceScene, cam: GsCamera, out: Projected, stream=None) -> int:
+    """Returns the number of (Gaussian, tile) instances; synchronises the stream once."""
+    pairs = C.c_int64(0)
+    cs, po = scene.c_struct(), out.c_struct()
+    ctx._check(_lib.gs_preprocess(ctx._h, C.byref(cs), C.byref(cam), C.byref(po), C.byref(pairs),
+                                  _stream_handle(stream)))
+    return int(pairs.value)
+
+
+def gs_render_forward(ctx: Context, n: int, proj: Projected, cam: GsCamera, num_pairs: int, pair_capacity: int,
+                      binning: Binning, image: torch.Tensor, final_T: torch.Tensor, n_contrib: torch.Tensor,
+                      workspace: torch.Tensor, stream=None) -> None:
+    pp, bb = proj.c_struct(), binning.c_struct()
+    ctx._check(_lib.gs_render_forward(ctx._h, n, C.byref(pp), C.byref(cam), num_pairs, pair_capacity, C.byref(bb),
+                                      _ptr(image), _ptr(final_T), _ptr(n_contrib), _ptr(workspace),
+                                      workspace.numel() * workspace.element_size(), _stream_handle(stream)))
+
+
+def gs_render_backward(ctx: Context, scene: DeviceScene, cam: GsCamera, proj: Projected, binning: Binning,
+                       num_pairs: int, final_T: torch.Tensor, n_contrib: torch.Tensor, dL_dimage: torch.Tensor,
+                       grads: Grads, workspace: torch.Tensor, stream=None) -> None:
+    cs, pp, bb, gg = scene.c_struct(), proj.c_struct(), binning.c_struct(), grads.c_struct()
+    ctx._check(_lib.gs_render_backward(ctx._h, C.byref(cs), C.byref(cam), C.byref(pp), C.byref(bb), num_pairs,
+                                       _ptr(final_T), _ptr(n_contrib), _ptr(dL_dimage), C.byref(gg),
+                                       _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                       _stream_handle(stream)))
+
+
+def gs_appearance_forward(ctx: Context, scene: DeviceScene, dirs: torch.Tensor, color: torch.Tensor,
+                          stream=None) -> None:
+    cs = scene.c_struct()
+    ctx._check(_lib.gs_appearance_forward(ctx._h, C.byref(cs), _ptr(dirs), _ptr(color), _stream_handle(stream)))
+
+
+def gs_appearance_backward(ctx: Context, scene: DeviceScene, dirs: torch.Tensor, dL_dcolor: torch.Tensor,
+                           grads: Grads, dL_ddirs: torch.Tensor, stream=None) -> None:
+    cs, gg = scene.c_struct(), grads.c_struct()
+    ctx._check(_lib.gs_appearance_backward(ctx._h, C.byref(cs), _ptr(dirs), _ptr(dL_dcolor), C.byref(gg),
+                                           _ptr(dL_ddirs), _stream_handle(stream)))
+
+
+# ------------------------------------------------------------------------------------------------
+# Convenience: one view, forward + backward, buffers allocated with torch.  Still marshalling only.
+# ------------------------------------------------------------------------------------------------
+class Renderer:
+    """Holds the per-view buffers so that repeated steps allocate nothing."""
+
+    def __init__(self, ctx: Context, n: int, width: int, height: int, app: int, pair_capacity: int,
+                 with_extent: bool = False):
+        dev = ctx.device
+        self.ctx, self.n, self.width, self.height, self.app = ctx, n, width, height, app
+        self.pair_capacity = pair_capacity
+        self.proj = alloc_projected(n, dev, with_extent)
+        self.binning = alloc_binning(n, pair_capacity, width, height, dev)
+        self.image = torch.empty((3, height, width), device=dev, dtype=torch.float32)
+        self.final_T = torch.empty((height, width), device=dev, dtype=torch.float32)
+        self.n_contrib = torch.empty((height, width), device=dev, dtype=torch.int32)
+        self.grads = alloc_grads(n, app, dev)
+        self.workspace = torch.empty((max(gs_workspace_bytes(n, width, height, pair_capacity), 256),),
+                                     device=dev, dtype=torch.uint8)
+        self.num_pairs = 0
+
+    def forward(self, scene: DeviceScene, cam: GsCamera, stream=None) -> torch.Tensor:
+        self.num_pairs = gs_preprocess(self.ctx, scene, cam, self.proj, stream)
+        gs_render_forward(self.ctx, scene.n, self.proj, cam, self.num_pairs, self.pair_capacity, self.binning,
+                          self.image, self.final_T, self.n_contrib, self.workspace, stream)
+        return self.image
+
+    def backward(self, scene: DeviceScene, cam: GsCamera, dL_dimage: torch.Tensor, stream=None) -> Grads:
+        gs_render_backward(self.ctx, scene, cam, self.proj, self.binning, self.num_pairs, self.final_T,
+                           self.n_contrib, dL_dimage, self.grads, self.workspace, stream)
+        return self.grads

@@ -1,0 +1,440 @@
+// The C ABI: argument validation, workspace carving and kernel launches.  No arithmetic of the
+// method lives here.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "gs_device.cuh"
+
+struct StageRecord { int stage; int launches; cudaEvent_t begin, end; };
+
+struct GsContext {
+  int device;
+  unsigned long long *d_counter;      // device: instance counter
+  unsigned long long *h_counter;      // pinned host mirror
+  float *d_w_partials;                // device: [kWgradBlocks, 816] decoder-gradient partial sums
+  char error[256];
+  bool profiling;
+  std::vector<StageRecord> records;   // stage timings since the last collect
+  std::vector<cudaEvent_t> free_events;
+};
+
+namespace {
+
+using namespace gs;
+
+GsStatus fail(GsContext *ctx, GsStatus code, const char *fmt, const char *detail = "") {
+  if (ctx) snprintf(ctx->error, sizeof(ctx->error), fmt, detail);
+  return code;
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+bool bad_ptr(const void *p) { return p == nullptr || !aligned16(p); }
+
+GsStatus check_cuda(GsContext *ctx, cudaError_t e, const char *what) {
+  if (e == cudaSuccess) return GS_OK;
+  if (ctx) snprintf(ctx->error, sizeof(ctx->error), "%s: %s", what, cudaGetErrorString(e));
+  return GS_ERR_CUDA;
+}
+
+// Brackets one stage with events when profiling is on.
+struct StageTimer {
+  GsContext *ctx; cudaStream_t st; StageRecord rec; bool active;
+  static cudaEvent_t get_event(GsContext *ctx) {
+    if (!ctx->free_events.empty()) { cudaEvent_t e = ctx->free_events.back(); ctx->free_events.pop_back(); return e; }
+    cudaEvent_t e = nullptr;
+    cudaEventCreate(&e);
+    return e;
+  }
+  StageTimer(GsContext *c, int stage, cudaStream_t s) : ctx(c), st(s), active(c->profiling && c->records.size() < 4096) {
+    if (!active) return;
+    rec.stage = stage; rec.launches = 0;
+    rec.begin = get_event(ctx); rec.end = get_event(ctx);
+    cudaEventRecord(rec.begin, st);
+  }
+  void done(int launches) {
+    if (!active) return;
+    rec.launches = launches;
+    cudaEventRecord(rec.end, st);
+    ctx->records.push_back(rec);
+  }
+};
+
+bool camera_ok(const GsCamera *c) {
+  if (!c || c->width <= 0 || c->height <= 0) return false;
+  if (!(c->fx > 0.f) || !(c->fy > 0.f)) return false;
+  if ((c->width + GS_TILE - 1) / GS_TILE > 65535 || (c->height + GS_TILE - 1) / GS_TILE > 65535) return false;
+  return true;
+}
+
+CamDev make_cam(const GsCamera *c) {
+  CamDev d;
+  d.W = c->width; d.H = c->height;
+  d.gx = (c->width + GS_TILE - 1) / GS_TILE; d.gy = (c->height + GS_TILE - 1) / GS_TILE;
+  d.fx = c->fx; d.fy = c->fy; d.cx = c->cx; d.cy = c->cy;
+  for (int r = 0; r < 3; ++r) {
+    for (int k = 0; k < 3; ++k) d.R[3 * r + k] = c->w2c[4 * r + k];
+    d.t[r] = c->w2c[4 * r + 3];
+  }
+  for (int k = 0; k < 3; ++k)
+    d.oc[k] = (float)-((double)d.R[k] * d.t[0] + (double)d.R[3 + k] * d.t[1] + (double)d.R[6 + k] * d.t[2]);
+  d.near_plane = c->near_plane; d.far_plane = c->far_plane;
+  d.limx = (float)(1.3 * (c->width / 2.0) / c->fx);
+  d.limy = (float)(1.3 * (c->height / 2.0) / c->fy);
+  for (int k = 0; k < 3; ++k) d.bg[k] = c->background[k];
+  return d;
+}
+
+GsStatus scene_appearance_ok(GsContext *ctx, const GsScene *s) {
+  if (s->app != GS_APP_SH && s->app != GS_APP_NEURAL) return fail(ctx, GS_ERR_INVALID_ARG, "unknown appearance model");
+  if (s->active_degree < 0 || s->active_degree > 3) return fail(ctx, GS_ERR_INVALID_ARG, "active_degree must be 0..3");
+  if (s->n < 0) return fail(ctx, GS_ERR_INVALID_ARG, "n < 0");
+  if (s->n == 0) return GS_OK;
+  if (bad_ptr(s->base_color)) return fail(ctx, GS_ERR_INVALID_ARG, "base_color is NULL or misaligned");
+  if (s->app == GS_APP_SH && bad_ptr(s->sh_rest)) return fail(ctx, GS_ERR_INVALID_ARG, "sh_rest is NULL or misaligned");
+  if (s->app == GS_APP_NEURAL && (bad_ptr(s->features) || bad_ptr(s->mlp_weights)))
+    return fail(ctx, GS_ERR_INVALID_ARG, "features / mlp_weights is NULL or misaligned");
+  return GS_OK;
+}
+
+GsStatus scene_ok(GsContext *ctx, const GsScene *s) {
+  if (!s) return fail(ctx, GS_ERR_INVALID_ARG, "scene is NULL");
+  GsStatus st = scene_appearance_ok(ctx, s);
+  if (st != GS_OK) return st;
+  if (s->n > 0 && (bad_ptr(s->means) || bad_ptr(s->log_scales) || bad_ptr(s->quats) || bad_ptr(s->opacity_logits)))
+    return fail(ctx, GS_ERR_INVALID_ARG, "a geometry array is NULL or misaligned");
+  return GS_OK;
+}
+
+// ---- workspace layout -------------------------------------------------------------------------
+size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
+
+struct Carver {
+  char *base;
+  size_t used;
+  template <class T>
+  T *take(size_t count) {
+    T *p = reinterpret_cast<T *>(base + used);
+    used += align_up(count * sizeof(T));
+    return p;
+  }
+};
+
+struct FwdWorkspace {
+  uint32_t *sorted_depth, *tmp_keys, *tmp_vals;          // [n]
+  uint32_t *block_offsets;                               // scan of tiles touched
+  uint32_t *inst_tiles, *inst_vals, *tmp_tiles, *tmp_ivals;  // [pair_capacity]
+  void *sort_table;
+  size_t bytes;
+};
+
+FwdWorkspace carve_fwd(void *ws, int64_t n, int64_t cap) {
+  Carver c{static_cast<char *>(ws), 0};
+  FwdWorkspace w;
+  const size_t nn = (size_t)(n > 0 ? n : 1), cc = (size_t)(cap > 0 ? cap : 1);
+  w.sorted_depth = c.take<uint32_t>(nn);
+  w.tmp_keys = c.take<uint32_t>(nn);
+  w.tmp_vals = c.take<uint32_t>(nn);
+  w.block_offsets = reinterpret_cast<uint32_t *>(c.take<char>(scan_scratch_bytes((int64_t)nn)));
+  w.inst_tiles = c.take<uint32_t>(cc);
+  w.inst_vals = c.take<uint32_t>(cc);
+  w.tmp_tiles = c.take<uint32_t>(cc);
+  w.tmp_ivals = c.take<uint32_t>(cc);
+  w.sort_table = c.take<char>(sort_scratch_bytes((int64_t)(nn > cc ? nn : cc)));
+  w.bytes = c.used;
+  return w;
+}
+
+size_t bwd_bytes(int64_t n) { return align_up((size_t)(n > 0 ? n : 1) * 12 * sizeof(float)); }
+
+int tile_bits(int num_tiles) {
+  int bits = 1;
+  while ((1 << bits) < num_tiles) ++bits;
+  return bits;
+}
+
+}  // namespace
+
+extern "C" {
+
+GsStatus gs_create(int device, GsContext **out) {
+  if (!out) return GS_ERR_INVALID_ARG;
+  *out = nullptr;
+  int count = 0;
+  if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) return GS_ERR_CUDA;
+  if (cudaSetDevice(device) != cudaSuccess) return GS_ERR_CUDA;
+  GsContext *ctx = new (std::nothrow) GsContext();
+  if (!ctx) return GS_ERR_INTERNAL;
+  ctx->device = device;
+  ctx->error[0] = 0;
+  ctx->d_counter = nullptr; ctx->h_counter = nullptr; ctx->d_w_partials = nullptr;
+  ctx->profiling = false;
+  if (cudaMalloc(&ctx->d_counter, sizeof(unsigned long long)) != cudaSuccess ||
+      cudaMallocHost(&ctx->h_counter, sizeof(unsigned long long)) != cudaSuccess ||
+      cudaMalloc(&ctx->d_w_partials, sizeof(float) * kWgradBlocks * GS_MLP_WEIGHTS) != cudaSuccess) {
+    gs_destroy(ctx);
+    return GS_ERR_CUDA;
+  }
+  *out = ctx;
+  return GS_OK;
+}
+
+void gs_destroy(GsContext *ctx) {
+  if (!ctx) return;
+  cudaSetDevice(ctx->device);
+  if (ctx->d_counter) cudaFree(ctx->d_counter);
+  if (ctx->h_counter) cudaFreeHost(ctx->h_counter);
+  if (ctx->d_w_partials) cudaFree(ctx->d_w_partials);
+  for (StageRecord &r : ctx->records) { cudaEventDestroy(r.begin); cudaEventDestroy(r.end); }
+  for (cudaEvent_t e : ctx->free_events) cudaEventDestroy(e);
+  delete ctx;
+}
+
+const char *gs_last_error(const GsContext *ctx) { return ctx ? ctx->error : "no context"; }
+
+size_t gs_workspace_bytes(int64_t n, int32_t width, int32_t height, int64_t pair_capacity) {
+  if (n < 0 || width <= 0 || height <= 0 || pair_capacity < 0) return 0;
+  const size_t f = carve_fwd(nullptr, n, pair_capacity).bytes, b = bwd_bytes(n);
+  return f > b ? f : b;
+}
+
+GsStatus gs_preprocess(GsContext *ctx, const GsScene *scene, const GsCamera *cam, GsProjected *out,
+                       int64_t *num_pairs_host, void *stream) {
+  if (!ctx) return GS_ERR_INVALID_ARG;
+  GsStatus st = scene_ok(ctx, scene);
+  if (st != GS_OK) return st;
+  if (!camera_ok(cam)) return fail(ctx, GS_ERR_INVALID_ARG, "bad camera (size, focal length or more than 65535 tiles per axis)");
+  if (!out || !num_pairs_host) return fail(ctx, GS_ERR_INVALID_ARG, "out / num_pairs_host is NULL");
+  *num_pairs_host = 0;
+  if (scene->n == 0) return GS_OK;
+  if (bad_ptr(out->mean2d) || bad_ptr(out->conic_opacity) || bad_ptr(out->color) || bad_ptr(out->depth_key) ||
+      bad_ptr(out->rect) || (out->extent && !aligned16(out->extent)))
+    return fail(ctx, GS_ERR_INVALID_ARG, "a GsProjected buffer is NULL or misaligned");
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaSetDevice(ctx->device);
+  PreprocessArgs a;
+  a.n = scene->n;
+  a.means = scene->means; a.log_scales = scene->log_scales; a.quats = scene->quats; a.logits = scene->opacity_logits;
+  a.base_color = scene->base_color; a.sh_rest = scene->sh_rest;
+  a.features = reinterpret_cast<const __half *>(scene->features);
+  a.weights = reinterpret_cast<const __half *>(scene->mlp_weights);
+  a.deg = scene->active_degree;
+  a.mean2d = out->mean2d; a.conic_opacity = out->conic_opacity; a.color = out->color; a.extent = out->extent;
+  a.depth_key = out->depth_key; a.rect = out->rect;
+  a.pair_counter = ctx->d_counter;
+  if ((st = check_cuda(ctx, cudaMemsetAsync(ctx->d_counter, 0, sizeof(unsigned long long), s), "memset")) != GS_OK) return st;
+  {
+    StageTimer t(ctx, GS_STAGE_PREPROCESS_FWD, s);
+    t.done(launch_preprocess_fwd(scene->app, a, make_cam(cam), s));
+  }
+  if ((st = check_cuda(ctx, cudaGetLastError(), "preprocess launch")) != GS_OK) return st;
+  if ((st = check_cuda(ctx, cudaMemcpyAsync(ctx->h_counter, ctx->d_counter, sizeof(unsigned long long),
+                                            cudaMemcpyDeviceToHost, s), "pair count copy")) != GS_OK) return st;
+  if ((st = check_cuda(ctx, cudaStreamSynchronize(s), "preprocess")) != GS_OK) return st;
+  *num_pairs_host = (int64_t)*ctx->h_counter;
+  return GS_OK;
+}
+
+GsStatus gs_render_forward(GsContext *ctx, int64_t n, const GsProjected *proj, const GsCamera *cam,
+                           int64_t num_pairs, int64_t pair_capacity, GsBinning *bin, float *image,
+                           float *final_T, uint32_t *n_contrib, void *workspace, size_t workspace_bytes,
+                           void *stream) {
+  if (!ctx) return GS_ERR_INVALID_ARG;
+  if (n < 0 || num_pairs < 0 || pair_capacity < 0) return fail(ctx, GS_ERR_INVALID_ARG, "negative size");
+  if (!camera_ok(cam)) return fail(ctx, GS_ERR_INVALID_ARG, "bad camera");
+  if (!proj || !bin) return fail(ctx, GS_ERR_INVALID_ARG, "proj / bin is NULL");
+  if (bad_ptr(image) || bad_ptr(final_T) || bad_ptr(n_contrib) || bad_ptr(bin->tile_ranges))
+    return fail(ctx, GS_ERR_INVALID_ARG, "an output buffer is NULL or misaligned");
+  if (num_pairs > pair_capacity) return fail(ctx, GS_ERR_CAPACITY, "num_pairs exceeds pair_capacity");
+  if (num_pairs >= ((int64_t)1 << 32)) return fail(ctx, GS_ERR_CAPACITY, "more than 2^32 - 1 instances");
+  if (workspace_bytes < gs_workspace_bytes(n, cam->width, cam->height, pair_capacity) || bad_ptr(workspace))
+    return fail(ctx, GS_ERR_CAPACITY, "workspace is NULL, misaligned or smaller than gs_workspace_bytes()");
+  if (n > 0 && (bad_ptr(proj->mean2d) || bad_ptr(proj->conic_opacity) || bad_ptr(proj->color) ||
+                bad_ptr(proj->depth_key) || bad_ptr(proj->rect) || bad_ptr(bin->depth_order)))
+    return fail(ctx, GS_ERR_INVALID_ARG, "a per-Gaussian buffer is NULL or misaligned");
+  if (num_pairs > 0 && (bad_ptr(bin->sorted_tiles) || bad_ptr(bin->sorted_vals)))
+    return fail(ctx, GS_ERR_INVALID_ARG, "an instance buffer is NULL or misaligned");
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaSetDevice(ctx->device);
+  const CamDev cd = make_cam(cam);
+  const int num_tiles = cd.gx * cd.gy;
+  const FwdWorkspace w = carve_fwd(workspace, n, pair_capacity);
+  if (n > 0 && num_pairs > 0) {
+    // stage 1: Gaussians by depth key (stable => ties keep the index order)
+    {
+      StageTimer t(ctx, GS_STAGE_DEPTH_SORT, s);
+      t.done(launch_radix_sort(proj->depth_key, nullptr, w.sorted_depth, bin->depth_order, w.tmp_keys, w.tmp_vals,
+                               n, 32, w.sort_table, s));
+    }
+    // stage 2: instances in depth order, then a stable sort by tile id alone
+    {
+      StageTimer t(ctx, GS_STAGE_TILE_OFFSETS, s);
+      t.done(launch_tile_offsets(bin->depth_order, proj->rect, w.block_offsets, n, nullptr, s));
+    }
+    {
+      StageTimer t(ctx, GS_STAGE_KEYGEN, s);
+      t.done(launch_keygen(bin->depth_order, proj->rect, w.block_offsets, w.inst_tiles, w.inst_vals, n, cd.gx, s));
+    }
+    {
+      StageTimer t(ctx, GS_STAGE_TILE_SORT, s);
+      t.done(launch_radix_sort(w.inst_tiles, w.inst_vals, bin->sorted_tiles, bin->sorted_vals, w.tmp_tiles,
+                               w.tmp_ivals, num_pairs, tile_bits(num_tiles), w.sort_table, s));
+    }
+  }
+  {
+    StageTimer t(ctx, GS_STAGE_TILE_RANGES, s);
+    t.done(launch_tile_ranges(bin->sorted_tiles, num_pairs, bin->tile_ranges, num_tiles, s));
+  }
+  {
+    StageTimer t(ctx, GS_STAGE_BLEND_FWD, s);
+    t.done(launch_blend_fwd(cd, bin->tile_ranges, bin->sorted_vals, proj->mean2d, proj->conic_opacity, proj->color,
+                            image, final_T, n_contrib, s));
+  }
+  return check_cuda(ctx, cudaGetLastError(), "render_forward launch");
+}
+
+GsStatus gs_render_backward(GsContext *ctx, const GsScene *scene, const GsCamera *cam, const GsProjected *proj,
+                            const GsBinning *bin, int64_t num_pairs, const float *final_T,
+                            const uint32_t *n_contrib, const float *dL_dimage, GsGrads *grads, void *workspace,
+                            size_t workspace_bytes, void *stream) {
+  if (!ctx) return GS_ERR_INVALID_ARG;
+  GsStatus st = scene_ok(ctx, scene);
+  if (st != GS_OK) return st;
+  if (!camera_ok(cam)) return fail(ctx, GS_ERR_INVALID_ARG, "bad camera");
+  if (!proj || !bin || !grads) return fail(ctx, GS_ERR_INVALID_ARG, "proj / bin / grads is NULL");
+  if (bad_ptr(final_T) || bad_ptr(n_contrib) || bad_ptr(dL_dimage) || bad_ptr(bin->tile_ranges))
+    return fail(ctx, GS_ERR_INVALID_ARG, "an image-sized buffer is NULL or misaligned");
+  const int64_t n = scene->n;
+  if (scene->app == GS_APP_NEURAL && bad_ptr(grads->mlp_weights))
+    return fail(ctx, GS_ERR_INVALID_ARG, "grads->mlp_weights is NULL or misaligned");
+  if (n > 0) {
+    if (bad_ptr(grads->means) || bad_ptr(grads->log_scales) || bad_ptr(grads->quats) ||
+        bad_ptr(grads->opacity_logits) || bad_ptr(grads->base_color))
+      return fail(ctx, GS_ERR_INVALID_ARG, "a gradient buffer is NULL or misaligned");
+    if (scene->app == GS_APP_SH && bad_ptr(grads->sh_rest)) return fail(ctx, GS_ERR_INVALID_ARG, "grads->sh_rest is NULL or misaligned");
+    if (scene->app == GS_APP_NEURAL && bad_ptr(grads->features)) return fail(ctx, GS_ERR_INVALID_ARG, "grads->features is NULL or misaligned");
+    if (bad_ptr(proj->mean2d) || bad_ptr(proj->conic_opacity) || bad_ptr(proj->color) || bad_ptr(proj->rect))
+      return fail(ctx, GS_ERR_INVALID_ARG, "a GsProjected buffer is NULL or misaligned");
+  }
+  if (num_pairs > 0 && bad_ptr(bin->sorted_vals)) return fail(ctx, GS_ERR_INVALID_ARG, "sorted_vals is NULL or misaligned");
+  if (workspace_bytes < bwd_bytes(n) || bad_ptr(workspace))
+    return fail(ctx, GS_ERR_CAPACITY, "workspace is NULL, misaligned or too small");
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaSetDevice(ctx->device);
+  const CamDev cd = make_cam(cam);
+  float *g2d = static_cast<float *>(workspace);
+  if (n > 0) {
+    if ((st = check_cuda(ctx, cudaMemsetAsync(g2d, 0, (size_t)n * 12 * sizeof(float), s), "memset")) != GS_OK) return st;
+    if (num_pairs > 0) {
+      StageTimer t(ctx, GS_STAGE_BLEND_BWD, s);
+      t.done(launch_blend_bwd(cd, bin->tile_ranges, bin->sorted_vals, proj->mean2d, proj->conic_opacity, proj->color,
+                              final_T, n_contrib, dL_dimage, g2d, s));
+    }
+  }
+  PreprocessBwdArgs a;
+  a.n = n;
+  a.means = scene->means; a.log_scales = scene->log_scales; a.quats = scene->quats; a.logits = scene->opacity_logits;
+  a.base_color = scene->base_color; a.sh_rest = scene->sh_rest;
+  a.features = reinterpret_cast<const __half *>(scene->features);
+  a.weights = reinterpret_cast<const __half *>(scene->mlp_weights);
+  a.deg = scene->active_degree;
+  a.rect = proj->rect; a.g2d = g2d;
+  a.g_means = grads->means; a.g_log_scales = grads->log_scales; a.g_quats = grads->quats;
+  a.g_logits = grads->opacity_logits; a.g_base = grads->base_color; a.g_sh_rest = grads->sh_rest;
+  a.g_features = grads->features; a.w_partials = ctx->d_w_partials; a.g_weights = grads->mlp_weights;
+  if (n == 0 && scene->app == GS_APP_NEURAL)
+    return check_cuda(ctx, cudaMemsetAsync(grads->mlp_weights, 0, sizeof(float) * GS_MLP_WEIGHTS, s), "memset");
+  {
+    StageTimer t(ctx, GS_STAGE_PREPROCESS_BWD, s);
+    t.done(launch_preprocess_bwd(scene->app, a, cd, s));
+  }
+  return check_cuda(ctx, cudaGetLastError(), "render_backward launch");
+}
+
+GsStatus gs_appearance_forward(GsContext *ctx, const GsScene *scene, const float *dirs, float *color, void *stream) {
+  if (!ctx) return GS_ERR_INVALID_ARG;
+  if (!scene) return fail(ctx, GS_ERR_INVALID_ARG, "scene is NULL");
+  GsStatus st = scene_appearance_ok(ctx, scene);
+  if (st != GS_OK) return st;
+  if (scene->n == 0) return GS_OK;
+  if (bad_ptr(dirs) || bad_ptr(color)) return fail(ctx, GS_ERR_INVALID_ARG, "dirs / color is NULL or misaligned");
+  cudaSetDevice(ctx->device);
+  AppearanceArgs a;
+  memset(&a, 0, sizeof(a));
+  a.n = scene->n; a.deg = scene->active_degree;
+  a.base_color = scene->base_color; a.sh_rest = scene->sh_rest; a.dirs = dirs;
+  a.features = reinterpret_cast<const __half *>(scene->features);
+  a.weights = reinterpret_cast<const __half *>(scene->mlp_weights);
+  a.color = color;
+  {
+    StageTimer t(ctx, GS_STAGE_APPEARANCE_FWD, static_cast<cudaStream_t>(stream));
+    t.done(launch_appearance_fwd(scene->app, a, static_cast<cudaStream_t>(stream)));
+  }
+  return check_cuda(ctx, cudaGetLastError(), "appearance_forward launch");
+}
+
+GsStatus gs_appearance_backward(GsContext *ctx, const GsScene *scene, const float *dirs, const float *dL_dcolor,
+                                GsGrads *grads, float *dL_ddirs, void *stream) {
+  if (!ctx) return GS_ERR_INVALID_ARG;
+  if (!scene || !grads) return fail(ctx, GS_ERR_INVALID_ARG, "scene / grads is NULL");
+  GsStatus st = scene_appearance_ok(ctx, scene);
+  if (st != GS_OK) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaSetDevice(ctx->device);
+  if (scene->app == GS_APP_NEURAL && bad_ptr(grads->mlp_weights))
+    return fail(ctx, GS_ERR_INVALID_ARG, "grads->mlp_weights is NULL or misaligned");
+  if (scene->n == 0) {
+    if (scene->app == GS_APP_NEURAL)
+      return check_cuda(ctx, cudaMemsetAsync(grads->mlp_weights, 0, sizeof(float) * GS_MLP_WEIGHTS, s), "memset");
+    return GS_OK;
+  }
+  if (bad_ptr(dirs) || bad_ptr(dL_dcolor) || bad_ptr(dL_ddirs) || bad_ptr(grads->base_color))
+    return fail(ctx, GS_ERR_INVALID_ARG, "dirs / dL_dcolor / dL_ddirs / grads->base_color is NULL or misaligned");
+  if (scene->app == GS_APP_SH && bad_ptr(grads->sh_rest)) return fail(ctx, GS_ERR_INVALID_ARG, "grads->sh_rest is NULL or misaligned");
+  if (scene->app == GS_APP_NEURAL && bad_ptr(grads->features)) return fail(ctx, GS_ERR_INVALID_ARG, "grads->features is NULL or misaligned");
+  AppearanceArgs a;
+  memset(&a, 0, sizeof(a));
+  a.n = scene->n; a.deg = scene->active_degree;
+  a.base_color = scene->base_color; a.sh_rest = scene->sh_rest; a.dirs = dirs;
+  a.features = reinterpret_cast<const __half *>(scene->features);
+  a.weights = reinterpret_cast<const __half *>(scene->mlp_weights);
+  a.g_color = dL_dcolor;
+  a.g_base = grads->base_color; a.g_sh_rest = grads->sh_rest; a.g_features = grads->features; a.g_dirs = dL_ddirs;
+  a.w_partials = ctx->d_w_partials; a.g_weights = grads->mlp_weights;
+  {
+    StageTimer t(ctx, GS_STAGE_APPEARANCE_BWD, s);
+    t.done(launch_appearance_bwd(scene->app, a, s));
+  }
+  return check_cuda(ctx, cudaGetLastError(), "appearance_backward launch");
+}
+
+GsStatus gs_profile_enable(GsContext *ctx, int enable) {
+  if (!ctx) return GS_ERR_INVALID_ARG;
+  ctx->profiling = enable != 0;
+  return GS_OK;
+}
+
+GsStatus gs_profile_collect(GsContext *ctx, double *ms, int64_t *launches) {
+  if (!ctx) return GS_ERR_INVALID_ARG;
+  cudaSetDevice(ctx->device);
+  GsStatus st = GS_OK;
+  for (StageRecord &r : ctx->records) {
+    float t = 0.f;
+    cudaError_t e = cudaEventSynchronize(r.end);
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&t, r.begin, r.end);
+    if (e != cudaSuccess) st = check_cuda(ctx, e, "profile collect");
+    else {
+      if (ms) ms[r.stage] += (double)t;
+      if (launches) launches[r.stage] += r.launches;
+    }
+    ctx->free_events.push_back(r.begin);
+    ctx->free_events.push_back(r.end);
+  }
+  ctx->records.clear();
+  return st;
+}
+
+}  // extern "C"

@@ -1,0 +1,880 @@
+// Per-Gaussian kernels: projection with fused appearance decode (forward and backward) and the
+// separate-pass appearance kernels.  One thread per Gaussian; SH coefficient rows and their
+// gradients move through per-warp shared-memory slabs so that global accesses stay coalesced;
+// decoder weights live in shared memory as fp32.
+#include <float.h>
+
+#include "gs_device.cuh"
+
+namespace gs {
+namespace {
+
+constexpr int kBlock = 128;
+constexpr int kWarps = kBlock / 32;
+constexpr int kRow = GS_SH_REST;           // 45 floats per Gaussian
+constexpr int kSlab = 32 * kRow;           // one warp's slab of SH rows
+constexpr unsigned kFull = 0xffffffffu;
+
+__device__ __forceinline__ bool finite_f(float x) { return fabsf(x) <= FLT_MAX; }
+
+// ---- warp-cooperative row movement ----------------------------------------------------------
+__device__ __forceinline__ void warp_load_rows(const float *g, int64_t row0, int64_t n, float *slab,
+                                               int lane) {
+  const int rows = (int)min((int64_t)32, n - row0);
+  const int total = rows * kRow;
+  const float *src = g + row0 * kRow;     // row0 is a multiple of 32 => 16-byte aligned
+  const int nv = total >> 2;
+  for (int k = lane; k < nv; k += 32) reinterpret_cast<float4 *>(slab)[k] = __ldg(reinterpret_cast<const float4 *>(src) + k);
+  for (int k = (nv << 2) + lane; k < total; k += 32) slab[k] = __ldg(src + k);
+  __syncwarp();
+}
+
+__device__ __forceinline__ void warp_store_rows(float *g, int64_t row0, int64_t n, const float *slab,
+                                                int lane) {
+  __syncwarp();
+  const int rows = (int)min((int64_t)32, n - row0);
+  const int total = rows * kRow;
+  float *dst = g + row0 * kRow;
+  const int nv = total >> 2;
+  for (int k = lane; k < nv; k += 32) reinterpret_cast<float4 *>(dst)[k] = reinterpret_cast<const float4 *>(slab)[k];
+  for (int k = (nv << 2) + lane; k < total; k += 32) dst[k] = slab[k];
+  __syncwarp();
+}
+
+// ---- appearance: SH -------------------------------------------------------------------------
+// colour = max(0, c0 + 0.5 + sum_k Y_k(d) c_k); row = this Gaussian's 45 coefficients in smem.
+__device__ __forceinline__ void sh_decode(const float *row, const float base[3], float dx, float dy,
+                                          float dz, int deg, float pre[3]) {
+  float Y[16];
+  sh_basis(dx, dy, dz, Y);
+  const int na = (deg + 1) * (deg + 1);
+  float r = base[0] + 0.5f, g = base[1] + 0.5f, b = base[2] + 0.5f;
+#pragma unroll
+  for (int k = 1; k < 16; ++k) {
+    if (k < na) {
+      r = fmaf(Y[k], row[3 * (k - 1) + 0], r);
+      g = fmaf(Y[k], row[3 * (k - 1) + 1], g);
+      b = fmaf(Y[k], row[3 * (k - 1) + 2], b);
+    }
+  }
+  pre[0] = r; pre[1] = g; pre[2] = b;
+}
+
+// Backward of the SH decode.  gp = dL/d(pre-activation) (already masked by the ReLU).  Writes the
+// coefficient gradients over `row` in place (row holds the coefficients on entry) and returns
+// dL/dd.
+__device__ __forceinline__ void sh_backward(float *row, const float gp[3], float dx, float dy, float dz,
+                                            int deg, float gd[3]) {
+  float Y[16];
+  sh_basis(dx, dy, dz, Y);
+  const int na = (deg + 1) * (deg + 1);
+  float gx = 0.f, gy = 0.f, gz = 0.f;
+#pragma unroll
+  for (int k = 1; k < 16; ++k) {
+    float *c = row + 3 * (k - 1);
+    if (k < na) {
+      const float w = c[0] * gp[0] + c[1] * gp[1] + c[2] * gp[2];
+      sh_grad_acc(k, dx, dy, dz, w, gx, gy, gz);
+      c[0] = Y[k] * gp[0]; c[1] = Y[k] * gp[1]; c[2] = Y[k] * gp[2];
+    } else {
+      c[0] = 0.f; c[1] = 0.f; c[2] = 0.f;
+    }
+  }
+  gd[0] = gx; gd[1] = gy; gd[2] = gz;
+}
+
+// ---- appearance: neural ---------------------------------------------------------------------
+__device__ __forceinline__ void load_weights_f32(const __half *w, float *sW, int tid, int nthreads) {
+  for (int k = tid; k < GS_MLP_WEIGHTS; k += nthreads) sW[k] = __half2float(w[k]);
+}
+
+__device__ __forceinline__ void load_features(const __half *features, int64_t i, float f[8]) {
+  const uint4 raw = __ldg(reinterpret_cast<const uint4 *>(features) + i);
+  const __half2 *h = reinterpret_cast<const __half2 *>(&raw);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const float2 v = __half22float2(h[j]);
+    f[2 * j] = v.x; f[2 * j + 1] = v.y;
+  }
+}
+
+// y = W x for a row-major [OUT][IN] matrix in shared memory (broadcast 128-bit reads).
+template <int OUT, int IN>
+__device__ __forceinline__ void matvec(const float *W, const float *x, float *y) {
+#pragma unroll
+  for (int o = 0; o < OUT; ++o) {
+    float acc = 0.f;
+#pragma unroll
+    for (int i = 0; i < IN; i += 4) {
+      const float4 w = *reinterpret_cast<const float4 *>(W + o * IN + i);
+      acc = fmaf(w.x, x[i], acc); acc = fmaf(w.y, x[i + 1], acc);
+      acc = fmaf(w.z, x[i + 2], acc); acc = fmaf(w.w, x[i + 3], acc);
+    }
+    y[o] = acc;
+  }
+}
+
+// g_x = W^T g_y
+template <int OUT, int IN>
+__device__ __forceinline__ void matvec_t(const float *W, const float *gy, float *gx) {
+#pragma unroll
+  for (int i = 0; i < IN; ++i) gx[i] = 0.f;
+#pragma unroll
+  for (int o = 0; o < OUT; ++o) {
+#pragma unroll
+    for (int i = 0; i < IN; i += 4) {
+      const float4 w = *reinterpret_cast<const float4 *>(W + o * IN + i);
+      gx[i] = fmaf(w.x, gy[o], gx[i]); gx[i + 1] = fmaf(w.y, gy[o], gx[i + 1]);
+      gx[i + 2] = fmaf(w.z, gy[o], gx[i + 2]); gx[i + 3] = fmaf(w.w, gy[o], gx[i + 3]);
+    }
+  }
+}
+
+// Eq. 5-7.  x = (Y_0..15(d) masked by the active degree, sin f_j, cos f_j interleaved).
+__device__ __forceinline__ void mlp_forward(const float *sW, float dx, float dy, float dz,
+                                            const float f[8], int deg, float x[32], float h1[16],
+                                            float h2[16], float A[3]) {
+  sh_basis(dx, dy, dz, x);
+  const int na = (deg + 1) * (deg + 1);
+#pragma unroll
+  for (int k = 0; k < 16; ++k) x[k] = k < na ? x[k] : 0.f;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) sincosf(f[j], &x[16 + 2 * j], &x[17 + 2 * j]);
+  matvec<16, 32>(sW + kMlpW1, x, h1);
+#pragma unroll
+  for (int k = 0; k < 16; ++k) h1[k] = fmaxf(h1[k], 0.f);
+  matvec<16, 16>(sW + kMlpW2, h1, h2);
+#pragma unroll
+  for (int k = 0; k < 16; ++k) h2[k] = fmaxf(h2[k], 0.f);
+  float y[3];
+  matvec<3, 16>(sW + kMlpW3, h2, y);
+#pragma unroll
+  for (int c = 0; c < 3; ++c) A[c] = tanhf(y[c]);
+}
+
+// Per-warp slab of the decoder-gradient kernels: for each of the warp's 32 Gaussians the
+// operands of the three outer products, 100 floats per Gaussian:
+// x[32] | h1[16] | h2[16] | g_h1[16] | g_h2[16] | g_y[3] + pad.
+constexpr int kActRow = 100;
+constexpr int kOffX = 0, kOffH1 = 32, kOffH2 = 48, kOffG1 = 64, kOffG2 = 80, kOffGY = 96;
+
+__device__ __forceinline__ void store4(float *dst, const float *v) {
+  *reinterpret_cast<float4 *>(dst) = make_float4(v[0], v[1], v[2], v[3]);
+}
+
+// Compiler-only fence.  The decoder weights sit in shared memory and are re-read by every stage;
+// without it the compiler keeps hundreds of them live in registers (hoisted out of the
+// persistent loop or carried from the forward into the backward) and spills.
+__device__ __forceinline__ void reload_fence() { asm volatile("" ::: "memory"); }
+
+__device__ __forceinline__ void load4(const float *src, float *v) {
+  const float4 t = *reinterpret_cast<const float4 *>(src);
+  v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+}
+
+// Backward through the decoder for one Gaussian (forward recomputed).  gcol = dL/dcolour; gp
+// returns dL/d(pre-activation of the colour) = gcol masked by the ReLU.  Writes this Gaussian's
+// operand row into the warp slab, returns dL/df and dL/dd.  Activations are parked in the slab row
+// as soon as they exist and read back when needed, which keeps the live registers under the limit.
+__device__ __forceinline__ void mlp_backward(const float *sW, float *act_row, float dx, float dy,
+                                             float dz, const float f[8], int deg, const float base[3],
+                                             const float gcol[3], float gp[3], float gf[8], float gd[3]) {
+  float gy[4];
+  {
+    float x[32], h1[16], h2[16], A[3];
+    mlp_forward(sW, dx, dy, dz, f, deg, x, h1, h2, A);
+#pragma unroll
+    for (int k = 0; k < 32; k += 4) store4(act_row + kOffX + k, x + k);
+#pragma unroll
+    for (int k = 0; k < 16; k += 4) { store4(act_row + kOffH1 + k, h1 + k); store4(act_row + kOffH2 + k, h2 + k); }
+#pragma unroll
+    for (int c = 0; c < 3; ++c) {
+      gp[c] = (base[c] + 0.5f + A[c]) > 0.f ? gcol[c] : 0.f;
+      gy[c] = gp[c] * (1.f - A[c] * A[c]);
+    }
+    gy[3] = 0.f;
+    store4(act_row + kOffGY, gy);
+  }
+  reload_fence();
+  float g1[16];
+  {
+    float g2[16], h[4];
+    matvec_t<3, 16>(sW + kMlpW3, gy, g2);
+#pragma unroll
+    for (int k = 0; k < 16; k += 4) {
+      load4(act_row + kOffH2 + k, h);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) g2[k + j] = h[j] > 0.f ? g2[k + j] : 0.f;
+      store4(act_row + kOffG2 + k, g2 + k);
+    }
+    reload_fence();
+    matvec_t<16, 16>(sW + kMlpW2, g2, g1);
+#pragma unroll
+    for (int k = 0; k < 16; k += 4) {
+      load4(act_row + kOffH1 + k, h);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) g1[k + j] = h[j] > 0.f ? g1[k + j] : 0.f;
+      store4(act_row + kOffG1 + k, g1 + k);
+    }
+  }
+  reload_fence();
+  float gx[32];
+  matvec_t<16, 32>(sW + kMlpW1, g1, gx);
+  reload_fence();
+#pragma unroll
+  for (int j = 0; j < 8; j += 2) {   // x[16 + 2j] = sin f_j, x[17 + 2j] = cos f_j
+    float sc[4];
+    load4(act_row + kOffX + 16 + 2 * j, sc);
+    gf[j] = gx[16 + 2 * j] * sc[1] - gx[17 + 2 * j] * sc[0];
+    gf[j + 1] = gx[18 + 2 * j] * sc[3] - gx[19 + 2 * j] * sc[2];
+  }
+  const int na = (deg + 1) * (deg + 1);
+  float ax = 0.f, ay = 0.f, az = 0.f;
+#pragma unroll
+  for (int k = 1; k < 16; ++k)
+    if (k < na) sh_grad_acc(k, dx, dy, dz, gx[k], ax, ay, az);
+  gd[0] = ax; gd[1] = ay; gd[2] = az;
+}
+
+__device__ __forceinline__ void zero_act_row(float *act_row) {
+  const float z[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+  for (int k = 0; k < kActRow; k += 4) store4(act_row + k, z);
+}
+
+// Register tiles of the weight gradient held by one lane: dW1 4x4 at (o = 4*(lane/8),
+// i = 4*(lane%8)), dW2 2x4 at (o = 2*(lane/4), i = 4*(lane%4)), dW3 1x4 at (o = lane/4,
+// i = 4*(lane%4)) for lanes < 12.
+struct WgradAcc {
+  float w1[16], w2[8], w3[4];
+  __device__ __forceinline__ void clear() {
+#pragma unroll
+    for (int k = 0; k < 16; ++k) w1[k] = 0.f;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) w2[k] = 0.f;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) w3[k] = 0.f;
+  }
+};
+
+// Accumulate the outer products of the warp's 32 operand rows.
+__device__ __forceinline__ void wgrad_accumulate(const float *slab, int lane, WgradAcc &acc) {
+  __syncwarp();
+  const int o1 = 4 * (lane >> 3), i1 = 4 * (lane & 7);
+  const int o2 = 2 * (lane >> 2), i2 = 4 * (lane & 3);
+  const int o3 = lane >> 2;
+  for (int g = 0; g < 32; ++g) {
+    const float *row = slab + g * kActRow;
+    const float4 a = *reinterpret_cast<const float4 *>(row + kOffG1 + o1);
+    const float4 b = *reinterpret_cast<const float4 *>(row + kOffX + i1);
+    const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+      for (int c = 0; c < 4; ++c) acc.w1[4 * r + c] = fmaf(av[r], bv[c], acc.w1[4 * r + c]);
+    const float2 a2 = *reinterpret_cast<const float2 *>(row + kOffG2 + o2);
+    const float4 b2 = *reinterpret_cast<const float4 *>(row + kOffH1 + i2);
+    const float b2v[4] = {b2.x, b2.y, b2.z, b2.w};
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      acc.w2[c] = fmaf(a2.x, b2v[c], acc.w2[c]);
+      acc.w2[4 + c] = fmaf(a2.y, b2v[c], acc.w2[4 + c]);
+    }
+    if (lane < 12) {
+      const float a3 = row[kOffGY + o3];
+      const float4 b3 = *reinterpret_cast<const float4 *>(row + kOffH2 + i2);
+      acc.w3[0] = fmaf(a3, b3.x, acc.w3[0]); acc.w3[1] = fmaf(a3, b3.y, acc.w3[1]);
+      acc.w3[2] = fmaf(a3, b3.z, acc.w3[2]); acc.w3[3] = fmaf(a3, b3.w, acc.w3[3]);
+    }
+  }
+  __syncwarp();
+}
+
+// Sum the warps' register tiles and write this block's partial [816].
+__device__ __forceinline__ void wgrad_flush(const WgradAcc &acc, float *sPart /*[kWarps][816]*/,
+                                            float *partial_out, int tid) {
+  const int lane = tid & 31, warp = tid >> 5;
+  float *mine = sPart + warp * GS_MLP_WEIGHTS;
+  const int o1 = 4 * (lane >> 3), i1 = 4 * (lane & 7);
+  const int o2 = 2 * (lane >> 2), i2 = 4 * (lane & 3);
+  const int o3 = lane >> 2;
+#pragma unroll
+  for (int r = 0; r < 4; ++r)
+#pragma unroll
+    for (int c = 0; c < 4; ++c) mine[kMlpW1 + (o1 + r) * 32 + i1 + c] = acc.w1[4 * r + c];
+#pragma unroll
+  for (int r = 0; r < 2; ++r)
+#pragma unroll
+    for (int c = 0; c < 4; ++c) mine[kMlpW2 + (o2 + r) * 16 + i2 + c] = acc.w2[4 * r + c];
+  if (lane < 12) {
+#pragma unroll
+    for (int c = 0; c < 4; ++c) mine[kMlpW3 + o3 * 16 + i2 + c] = acc.w3[c];
+  }
+  __syncthreads();
+  for (int k = tid; k < GS_MLP_WEIGHTS; k += kBlock) {
+    float s = 0.f;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) s += sPart[w * GS_MLP_WEIGHTS + k];
+    partial_out[k] = s;
+  }
+}
+
+// Deterministic final reduction of the per-block partials.
+__global__ void k_wgrad_reduce(const float *__restrict__ partials, int nblocks, float *__restrict__ out) {
+  const int k = blockIdx.x * blockDim.x + threadIdx.x;
+  if (k >= GS_MLP_WEIGHTS) return;
+  float s = 0.f;
+  for (int b = 0; b < nblocks; ++b) s += partials[(size_t)b * GS_MLP_WEIGHTS + k];
+  out[k] = s;
+}
+
+// ---- projection -----------------------------------------------------------------------------
+struct Geo {
+  bool valid;
+  float u, v, A, B, C, o, ex, ey;
+  uint32_t zbits;
+  float dirx, diry, dirz;
+};
+
+__device__ __forceinline__ void quat_rot(float r, float x, float y, float z, float R[9]) {
+  R[0] = 1.f - 2.f * (y * y + z * z); R[1] = 2.f * (x * y - r * z); R[2] = 2.f * (x * z + r * y);
+  R[3] = 2.f * (x * y + r * z); R[4] = 1.f - 2.f * (x * x + z * z); R[5] = 2.f * (y * z - r * x);
+  R[6] = 2.f * (x * z - r * y); R[7] = 2.f * (y * z + r * x); R[8] = 1.f - 2.f * (x * x + y * y);
+}
+
+// Everything the backward needs again is recomputed there; this is the forward only.
+__device__ __forceinline__ Geo project(const float mu[3], const float ls[3], const float q[4],
+                                       float logit, const CamDev &cam) {
+  Geo g;
+  g.valid = false;
+  g.zbits = 0xffffffffu;
+  bool fin = finite_f(logit);
+#pragma unroll
+  for (int k = 0; k < 3; ++k) fin = fin && finite_f(mu[k]) && finite_f(ls[k]);
+#pragma unroll
+  for (int k = 0; k < 4; ++k) fin = fin && finite_f(q[k]);
+  if (!fin) return g;
+  // the depth key: one fp32 FMA chain, identical bits on any IEEE machine
+  const float z32 = __fmaf_rn(cam.R[8], mu[2], __fmaf_rn(cam.R[7], mu[1], __fmaf_rn(cam.R[6], mu[0], cam.t[2])));
+  if (!(z32 >= cam.near_plane) || !(z32 <= cam.far_plane)) return g;
+  const float o = 1.f / (1.f + expf(-logit));
+  if (o < kAlphaMin) return g;
+  const float qn2 = q[0] * q[0] + q[1] * q[1] + q[2] * q[2] + q[3] * q[3];
+  if (!(qn2 > 0.f)) return g;
+  const float qi = rsqrtf(qn2);
+  float R[9];
+  quat_rot(q[0] * qi, q[1] * qi, q[2] * qi, q[3] * qi, R);
+  const float s0 = expf(ls[0]), s1 = expf(ls[1]), s2 = expf(ls[2]);
+  float M[9];
+#pragma unroll
+  for (int r = 0; r < 3; ++r) { M[3 * r] = R[3 * r] * s0; M[3 * r + 1] = R[3 * r + 1] * s1; M[3 * r + 2] = R[3 * r + 2] * s2; }
+  const float tx = cam.R[0] * mu[0] + cam.R[1] * mu[1] + cam.R[2] * mu[2] + cam.t[0];
+  const float ty = cam.R[3] * mu[0] + cam.R[4] * mu[1] + cam.R[5] * mu[2] + cam.t[1];
+  const float tz = cam.R[6] * mu[0] + cam.R[7] * mu[1] + cam.R[8] * mu[2] + cam.t[2];
+  const float iz = 1.f / tz;
+  const float rx = tx * iz, ry = ty * iz;
+  const float txc = tz * fminf(cam.limx, fmaxf(-cam.limx, rx));
+  const float tyc = tz * fminf(cam.limy, fmaxf(-cam.limy, ry));
+  const float j00 = cam.fx * iz, j02 = -cam.fx * txc * iz * iz;
+  const float j11 = cam.fy * iz, j12 = -cam.fy * tyc * iz * iz;
+  // T = J R_c (2x3), then N = T M (2x3): cov = N N^T + 0.3 I
+  float T[6];
+#pragma unroll
+  for (int c = 0; c < 3; ++c) {
+    T[c] = j00 * cam.R[c] + j02 * cam.R[6 + c];
+    T[3 + c] = j11 * cam.R[3 + c] + j12 * cam.R[6 + c];
+  }
+  float N[6];
+#pragma unroll
+  for (int r = 0; r < 2; ++r)
+#pragma unroll
+    for (int c = 0; c < 3; ++c) N[3 * r + c] = T[3 * r] * M[c] + T[3 * r + 1] * M[3 + c] + T[3 * r + 2] * M[6 + c];
+  const float a = N[0] * N[0] + N[1] * N[1] + N[2] * N[2] + kDilation;
+  const float b = N[0] * N[3] + N[1] * N[4] + N[2] * N[5];
+  const float c = N[3] * N[3] + N[4] * N[4] + N[5] * N[5] + kDilation;
+  const float det = a * c - b * b;
+  if (!(det > 0.f) || !finite_f(det)) return g;
+  const float idet = 1.f / det;
+  const float tau = 2.f * logf(255.f * o);
+  const float ex = __fmul_rn(sqrtf(tau * a), kExtentPad), ey = __fmul_rn(sqrtf(tau * c), kExtentPad);
+  const float u = fmaf(cam.fx, rx, cam.cx), v = fmaf(cam.fy, ry, cam.cy);
+  if (!finite_f(u) || !finite_f(v) || !finite_f(ex) || !finite_f(ey)) return g;
+  g.valid = true;
+  g.zbits = __float_as_uint(z32);
+  g.u = u; g.v = v; g.A = c * idet; g.B = -b * idet; g.C = a * idet; g.o = o; g.ex = ex; g.ey = ey;
+  const float vx = mu[0] - cam.oc[0], vy = mu[1] - cam.oc[1], vz = mu[2] - cam.oc[2];
+  const float vi = rsqrtf(vx * vx + vy * vy + vz * vz);
+  g.dirx = vx * vi; g.diry = vy * vi; g.dirz = vz * vi;
+  return g;
+}
+
+// Tile rectangle of the box [u-ex, u+ex] x [v-ey, v+ey] over pixel centres.  One rounding per
+// operation, no contraction, so that the same integers come out of any IEEE fp32 evaluation.
+__device__ __forceinline__ bool tile_rect(float u, float v, float ex, float ey, const CamDev &cam,
+                                          int r[4]) {
+  const float i0 = ceilf(__fsub_rn(__fsub_rn(u, ex), 0.5f)), i1 = floorf(__fsub_rn(__fadd_rn(u, ex), 0.5f));
+  const float j0 = ceilf(__fsub_rn(__fsub_rn(v, ey), 0.5f)), j1 = floorf(__fsub_rn(__fadd_rn(v, ey), 0.5f));
+  const bool empty = !(i0 <= i1 && j0 <= j1) || i1 < 0.f || j1 < 0.f || i0 > (float)(cam.W - 1) || j0 > (float)(cam.H - 1);
+  if (empty) { r[0] = r[1] = r[2] = r[3] = 0; return false; }
+  const int pi0 = (int)fmaxf(i0, 0.f), pi1 = (int)fminf(i1, (float)(cam.W - 1));
+  const int pj0 = (int)fmaxf(j0, 0.f), pj1 = (int)fminf(j1, (float)(cam.H - 1));
+  r[0] = pi0 >> 4; r[1] = pj0 >> 4; r[2] = (pi1 >> 4) + 1; r[3] = (pj1 >> 4) + 1;
+  return true;
+}
+
+__device__ __forceinline__ void load3(const float *p, int64_t i, float v[3]) {
+  v[0] = __ldg(p + 3 * i); v[1] = __ldg(p + 3 * i + 1); v[2] = __ldg(p + 3 * i + 2);
+}
+
+template <int APP>
+__global__ void __launch_bounds__(kBlock) k_preprocess_fwd(PreprocessArgs a, CamDev cam) {
+  __shared__ __align__(16) float sData[APP == GS_APP_SH ? kWarps * kSlab : GS_MLP_WEIGHTS];
+  __shared__ unsigned int sPairs[kWarps];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (APP == GS_APP_NEURAL) {
+    load_weights_f32(a.weights, sData, tid, kBlock);
+    __syncthreads();
+  }
+  const int64_t i = (int64_t)blockIdx.x * kBlock + tid;
+  const int64_t row0 = (int64_t)blockIdx.x * kBlock + warp * 32;
+  const bool in = i < a.n;
+  Geo g;
+  g.valid = false;
+  int rect[4] = {0, 0, 0, 0};
+  bool vis = false;
+  if (in) {
+    float mu[3], ls[3];
+    load3(a.means, i, mu);
+    load3(a.log_scales, i, ls);
+    const float4 q4 = __ldg(reinterpret_cast<const float4 *>(a.quats) + i);
+    const float q[4] = {q4.x, q4.y, q4.z, q4.w};
+    g = project(mu, ls, q, __ldg(a.logits + i), cam);
+    if (g.valid) vis = tile_rect(g.u, g.v, g.ex, g.ey, cam, rect);
+  }
+  // ---- fused colour decode for the Gaussians that survived culling
+  float pre[3] = {0.f, 0.f, 0.f};
+  if (APP == GS_APP_SH) {
+    float *slab = sData + warp * kSlab;
+    if (__any_sync(kFull, vis) && a.deg > 0 && row0 < a.n) warp_load_rows(a.sh_rest, row0, a.n, slab, lane);
+    if (vis) {
+      float base[3];
+      load3(a.base_color, i, base);
+      sh_decode(slab + lane * kRow, base, g.dirx, g.diry, g.dirz, a.deg, pre);
+    }
+  } else {
+    if (vis) {
+      float base[3];
+      load3(a.base_color, i, base);
+      float A[3] = {0.f, 0.f, 0.f};
+      if (a.deg > 0) {
+        float f[8], x[32], h1[16], h2[16];
+        load_features(a.features, i, f);
+        mlp_forward(sData, g.dirx, g.diry, g.dirz, f, a.deg, x, h1, h2, A);
+      }
+#pragma unroll
+      for (int c = 0; c < 3; ++c) pre[c] = base[c] + 0.5f + A[c];
+    }
+  }
+  unsigned int tiles = 0;
+  if (in) {
+    if (vis) {
+      reinterpret_cast<float2 *>(a.mean2d)[i] = make_float2(g.u, g.v);
+      reinterpret_cast<float4 *>(a.conic_opacity)[i] = make_float4(g.A, g.B, g.C, g.o);
+      a.color[3 * i] = fmaxf(pre[0], 0.f); a.color[3 * i + 1] = fmaxf(pre[1], 0.f); a.color[3 * i + 2] = fmaxf(pre[2], 0.f);
+      tiles = (unsigned)((rect[2] - rect[0]) * (rect[3] - rect[1]));
+    }
+    a.depth_key[i] = vis ? g.zbits : 0xffffffffu;
+    reinterpret_cast<ushort4 *>(a.rect)[i] = make_ushort4((unsigned short)rect[0], (unsigned short)rect[1],
+                                                          (unsigned short)rect[2], (unsigned short)rect[3]);
+    if (a.extent) reinterpret_cast<float2 *>(a.extent)[i] = g.valid ? make_float2(g.ex, g.ey) : make_float2(-1.f, -1.f);
+  }
+  // ---- total number of (Gaussian, tile) instances
+#pragma unroll
+  for (int s = 16; s > 0; s >>= 1) tiles += __shfl_xor_sync(kFull, tiles, s);
+  if (lane == 0) sPairs[warp] = tiles;
+  __syncthreads();
+  if (tid == 0) {
+    unsigned int tot = 0;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) tot += sPairs[w];
+    if (tot) atomicAdd(a.pair_counter, (unsigned long long)tot);
+  }
+}
+
+// ---- backward of the projection for one Gaussian --------------------------------------------
+struct GeoGrads { float mu[3], ls[3], q[4], logit; };
+
+__device__ __forceinline__ GeoGrads project_backward(const float mu[3], const float ls[3], const float q[4],
+                                                     float logit, const CamDev &cam, float gA, float gB,
+                                                     float gC, float gu, float gv, float go, const float gd[3]) {
+  GeoGrads out;
+  const float qn = sqrtf(q[0] * q[0] + q[1] * q[1] + q[2] * q[2] + q[3] * q[3]);
+  const float qi = 1.f / qn;
+  const float r = q[0] * qi, x = q[1] * qi, y = q[2] * qi, z = q[3] * qi;
+  float R[9];
+  quat_rot(r, x, y, z, R);
+  const float s[3] = {expf(ls[0]), expf(ls[1]), expf(ls[2])};
+  float M[9];
+#pragma unroll
+  for (int i = 0; i < 3; ++i)
+#pragma unroll
+    for (int k = 0; k < 3; ++k) M[3 * i + k] = R[3 * i + k] * s[k];
+  const float tx = cam.R[0] * mu[0] + cam.R[1] * mu[1] + cam.R[2] * mu[2] + cam.t[0];
+  const float ty = cam.R[3] * mu[0] + cam.R[4] * mu[1] + cam.R[5] * mu[2] + cam.t[1];
+  const float tz = cam.R[6] * mu[0] + cam.R[7] * mu[1] + cam.R[8] * mu[2] + cam.t[2];
+  const float iz = 1.f / tz, iz2 = iz * iz;
+  const float rx = tx * iz, ry = ty * iz;
+  const bool clx = rx < -cam.limx || rx > cam.limx, cly = ry < -cam.limy || ry > cam.limy;
+  const float txc = tz * fminf(cam.limx, fmaxf(-cam.limx, rx));
+  const float tyc = tz * fminf(cam.limy, fmaxf(-cam.limy, ry));
+  const float j00 = cam.fx * iz, j02 = -cam.fx * txc * iz2;
+  const float j11 = cam.fy * iz, j12 = -cam.fy * tyc * iz2;
+  float T[6];
+#pragma unroll
+  for (int c = 0; c < 3; ++c) {
+    T[c] = j00 * cam.R[c] + j02 * cam.R[6 + c];
+    T[3 + c] = j11 * cam.R[3 + c] + j12 * cam.R[6 + c];
+  }
+  float N[6];  // N = T M, cov = N N^T + 0.3 I
+#pragma unroll
+  for (int i = 0; i < 2; ++i)
+#pragma unroll
+    for (int c = 0; c < 3; ++c) N[3 * i + c] = T[3 * i] * M[c] + T[3 * i + 1] * M[3 + c] + T[3 * i + 2] * M[6 + c];
+  const float a = N[0] * N[0] + N[1] * N[1] + N[2] * N[2] + kDilation;
+  const float b = N[0] * N[3] + N[1] * N[4] + N[2] * N[5];
+  const float c = N[3] * N[3] + N[4] * N[4] + N[5] * N[5] + kDilation;
+  const float idet = 1.f / (a * c - b * b);
+  const float A = c * idet, B = -b * idet, C = a * idet;
+  // conic -> covariance: G_cov = -Q G_Q Q, G_Q = [[gA, gB/2], [gB/2, gC]]
+  const float h = 0.5f * gB;
+  const float m00 = A * gA + B * h, m01 = A * h + B * gC, m10 = B * gA + C * h, m11 = B * h + C * gC;
+  const float c00 = -(m00 * A + m01 * B), c01 = -(m00 * B + m01 * C), c11 = -(m10 * B + m11 * C);
+  // cov = N N^T: G_N = 2 G_cov N (2x3); N = T M: G_T = G_N M^T, G_M = T^T G_N
+  float GN[6];
+#pragma unroll
+  for (int k = 0; k < 3; ++k) {
+    GN[k] = 2.f * (c00 * N[k] + c01 * N[3 + k]);
+    GN[3 + k] = 2.f * (c01 * N[k] + c11 * N[3 + k]);
+  }
+  float GT[6];
+#pragma unroll
+  for (int i = 0; i < 2; ++i)
+#pragma unroll
+    for (int k = 0; k < 3; ++k) GT[3 * i + k] = GN[3 * i] * M[3 * k] + GN[3 * i + 1] * M[3 * k + 1] + GN[3 * i + 2] * M[3 * k + 2];
+  float GM[9];
+#pragma unroll
+  for (int i = 0; i < 3; ++i)
+#pragma unroll
+    for (int k = 0; k < 3; ++k) GM[3 * i + k] = T[i] * GN[k] + T[3 + i] * GN[3 + k];
+  // T = J R_c: the four entries of G_J that exist
+  const float gj00 = GT[0] * cam.R[0] + GT[1] * cam.R[1] + GT[2] * cam.R[2];
+  const float gj02 = GT[0] * cam.R[6] + GT[1] * cam.R[7] + GT[2] * cam.R[8];
+  const float gj11 = GT[3] * cam.R[3] + GT[4] * cam.R[4] + GT[5] * cam.R[5];
+  const float gj12 = GT[3] * cam.R[6] + GT[4] * cam.R[7] + GT[5] * cam.R[8];
+  float gtx = gu * cam.fx * iz, gty = gv * cam.fy * iz;
+  float gtz = -(gu * cam.fx * tx + gv * cam.fy * ty) * iz2 - (gj00 * cam.fx + gj11 * cam.fy) * iz2;
+  if (!clx) { gtx -= gj02 * cam.fx * iz2; gtz += gj02 * 2.f * cam.fx * tx * iz2 * iz; }
+  else      { gtz -= gj02 * j02 * iz; }
+  if (!cly) { gty -= gj12 * cam.fy * iz2; gtz += gj12 * 2.f * cam.fy * ty * iz2 * iz; }
+  else      { gtz -= gj12 * j12 * iz; }
+  // direction d = (mu - o_c)/|mu - o_c|: tangent projection of dL/dd
+  const float vx = mu[0] - cam.oc[0], vy = mu[1] - cam.oc[1], vz = mu[2] - cam.oc[2];
+  const float vi = rsqrtf(vx * vx + vy * vy + vz * vz);
+  const float dx = vx * vi, dy = vy * vi, dz = vz * vi;
+  const float dot = dx * gd[0] + dy * gd[1] + dz * gd[2];
+  out.mu[0] = cam.R[0] * gtx + cam.R[3] * gty + cam.R[6] * gtz + (gd[0] - dx * dot) * vi;
+  out.mu[1] = cam.R[1] * gtx + cam.R[4] * gty + cam.R[7] * gtz + (gd[1] - dy * dot) * vi;
+  out.mu[2] = cam.R[2] * gtx + cam.R[5] * gty + cam.R[8] * gtz + (gd[2] - dz * dot) * vi;
+  // M = R diag(s)
+  float D[9];
+#pragma unroll
+  for (int k = 0; k < 3; ++k) {
+    const float gs = GM[k] * R[k] + GM[3 + k] * R[3 + k] + GM[6 + k] * R[6 + k];
+    out.ls[k] = s[k] * gs;
+    D[k] = GM[k] * s[k]; D[3 + k] = GM[3 + k] * s[k]; D[6 + k] = GM[6 + k] * s[k];
+  }
+  float gq[4];
+  gq[0] = 2.f * (z * (D[3] - D[1]) + y * (D[2] - D[6]) + x * (D[7] - D[5]));
+  gq[1] = 2.f * (y * (D[1] + D[3]) + z * (D[2] + D[6]) + r * (D[7] - D[5]) - 2.f * x * (D[4] + D[8]));
+  gq[2] = 2.f * (x * (D[1] + D[3]) + r * (D[2] - D[6]) + z * (D[5] + D[7]) - 2.f * y * (D[0] + D[8]));
+  gq[3] = 2.f * (r * (D[3] - D[1]) + x * (D[2] + D[6]) + y * (D[5] + D[7]) - 2.f * z * (D[0] + D[4]));
+  const float qd = r * gq[0] + x * gq[1] + y * gq[2] + z * gq[3];
+  out.q[0] = (gq[0] - r * qd) * qi; out.q[1] = (gq[1] - x * qd) * qi;
+  out.q[2] = (gq[2] - y * qd) * qi; out.q[3] = (gq[3] - z * qd) * qi;
+  const float o = 1.f / (1.f + expf(-logit));
+  out.logit = go * o * (1.f - o);
+  return out;
+}
+
+__device__ __forceinline__ void store3(float *p, int64_t i, float a, float b, float c) {
+  p[3 * i] = a; p[3 * i + 1] = b; p[3 * i + 2] = c;
+}
+
+// Shared memory of the backward kernels (dynamic): SH: kWarps slabs of coefficient rows.
+// Neural: weights [816] | kWarps operand slabs [32][100] (reused as [kWarps][816] at the end).
+constexpr size_t kBwdSmemSH = sizeof(float) * kWarps * kSlab;
+constexpr size_t kBwdSmemNN = sizeof(float) * (GS_MLP_WEIGHTS + kWarps * 32 * kActRow);
+static_assert(kWarps * 32 * kActRow >= kWarps * GS_MLP_WEIGHTS, "partial sums reuse the operand slabs");
+
+template <int APP>
+__global__ void __launch_bounds__(kBlock) k_preprocess_bwd(PreprocessBwdArgs a, CamDev cam) {
+  extern __shared__ __align__(16) float smem[];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  float *sW = smem;
+  float *slab = APP == GS_APP_SH ? smem + warp * kSlab : smem + GS_MLP_WEIGHTS + warp * 32 * kActRow;
+  WgradAcc acc;
+  if (APP == GS_APP_NEURAL) {
+    load_weights_f32(a.weights, sW, tid, kBlock);
+    acc.clear();
+    __syncthreads();
+  }
+  const int64_t nchunks = (a.n + kBlock - 1) / kBlock;
+  for (int64_t chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x) {
+    reload_fence();
+    const int64_t i = chunk * kBlock + tid;
+    const int64_t row0 = chunk * kBlock + warp * 32;
+    const bool in = i < a.n;
+    bool vis = false;
+    if (in) {
+      const ushort4 rc = __ldg(reinterpret_cast<const ushort4 *>(a.rect) + i);
+      vis = rc.z > rc.x && rc.w > rc.y;
+    }
+    const bool warp_vis = __any_sync(kFull, vis);
+    float gd[3] = {0.f, 0.f, 0.f};
+    float mu[3], ls[3], q[4], logit = 0.f;
+    float4 ga = make_float4(0.f, 0.f, 0.f, 0.f), gb = ga, gc = ga;
+    float dx = 0.f, dy = 0.f, dz = 0.f;
+    if (vis) {
+      load3(a.means, i, mu);
+      load3(a.log_scales, i, ls);
+      const float4 q4 = __ldg(reinterpret_cast<const float4 *>(a.quats) + i);
+      q[0] = q4.x; q[1] = q4.y; q[2] = q4.z; q[3] = q4.w;
+      logit = __ldg(a.logits + i);
+      const float4 *g2 = reinterpret_cast<const float4 *>(a.g2d) + 3 * i;
+      ga = g2[0]; gb = g2[1]; gc = g2[2];   // (gr, gg, gb, go) (gA, gB, gC, gu) (gv, -, -, -)
+      const float vx = mu[0] - cam.oc[0], vy = mu[1] - cam.oc[1], vz = mu[2] - cam.oc[2];
+      const float vi = rsqrtf(vx * vx + vy * vy + vz * vz);
+      dx = vx * vi; dy = vy * vi; dz = vz * vi;
+    }
+    // ---- appearance backward
+    float gp[3] = {0.f, 0.f, 0.f};
+    if (APP == GS_APP_SH) {
+      if (row0 < a.n) {
+        if (warp_vis && a.deg > 0) {
+          warp_load_rows(a.sh_rest, row0, a.n, slab, lane);
+        }
+        float *row = slab + lane * kRow;
+        if (vis) {
+          float base[3], pre[3];
+          load3(a.base_color, i, base);
+          if (a.deg > 0) sh_decode(row, base, dx, dy, dz, a.deg, pre);
+          else { pre[0] = base[0] + 0.5f; pre[1] = base[1] + 0.5f; pre[2] = base[2] + 0.5f; }
+          gp[0] = pre[0] > 0.f ? ga.x : 0.f; gp[1] = pre[1] > 0.f ? ga.y : 0.f; gp[2] = pre[2] > 0.f ? ga.z : 0.f;
+          sh_backward(row, gp, dx, dy, dz, a.deg, gd);
+        } else {
+#pragma unroll
+          for (int k = 0; k < kRow; ++k) row[k] = 0.f;
+        }
+        warp_store_rows(a.g_sh_rest, row0, a.n, slab, lane);
+      }
+    } else {
+      float gf[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+      float *act_row = slab + lane * kActRow;
+      bool used = false;
+      if (vis) {
+        float base[3];
+        load3(a.base_color, i, base);
+        if (a.deg > 0) {
+          float f[8];
+          const float gcol[3] = {ga.x, ga.y, ga.z};
+          load_features(a.features, i, f);
+          mlp_backward(sW, act_row, dx, dy, dz, f, a.deg, base, gcol, gp, gf, gd);
+          used = true;
+        } else {
+#pragma unroll
+          for (int c = 0; c < 3; ++c) gp[c] = (base[c] + 0.5f) > 0.f ? (c == 0 ? ga.x : c == 1 ? ga.y : ga.z) : 0.f;
+        }
+      }
+      if (warp_vis && a.deg > 0) {
+        if (!used) zero_act_row(act_row);
+        wgrad_accumulate(slab, lane, acc);
+      }
+      if (in) {
+        float4 *gfp = reinterpret_cast<float4 *>(a.g_features) + 2 * i;
+        gfp[0] = make_float4(gf[0], gf[1], gf[2], gf[3]);
+        gfp[1] = make_float4(gf[4], gf[5], gf[6], gf[7]);
+      }
+    }
+    // ---- geometry backward
+    if (in) {
+      GeoGrads gg;
+      if (vis) {
+        gg = project_backward(mu, ls, q, logit, cam, gb.x, gb.y, gb.z, gb.w, gc.x, ga.w, gd);
+      } else {
+#pragma unroll
+        for (int k = 0; k < 3; ++k) { gg.mu[k] = 0.f; gg.ls[k] = 0.f; }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) gg.q[k] = 0.f;
+        gg.logit = 0.f;
+      }
+      store3(a.g_means, i, gg.mu[0], gg.mu[1], gg.mu[2]);
+      store3(a.g_log_scales, i, gg.ls[0], gg.ls[1], gg.ls[2]);
+      reinterpret_cast<float4 *>(a.g_quats)[i] = make_float4(gg.q[0], gg.q[1], gg.q[2], gg.q[3]);
+      a.g_logits[i] = gg.logit;
+      store3(a.g_base, i, gp[0], gp[1], gp[2]);
+    }
+  }
+  if (APP == GS_APP_NEURAL) {
+    __syncthreads();
+    wgrad_flush(acc, smem + GS_MLP_WEIGHTS, a.w_partials + (size_t)blockIdx.x * GS_MLP_WEIGHTS, tid);
+  }
+}
+
+// ---- separate-pass appearance kernels ---------------------------------------------------------
+template <int APP>
+__global__ void __launch_bounds__(kBlock) k_appearance_fwd(AppearanceArgs a) {
+  __shared__ __align__(16) float sData[APP == GS_APP_SH ? kWarps * kSlab : GS_MLP_WEIGHTS];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (APP == GS_APP_NEURAL) {
+    load_weights_f32(a.weights, sData, tid, kBlock);
+    __syncthreads();
+  }
+  const int64_t i = (int64_t)blockIdx.x * kBlock + tid;
+  const int64_t row0 = (int64_t)blockIdx.x * kBlock + warp * 32;
+  const bool in = i < a.n;
+  float d[3] = {0.f, 0.f, 1.f}, base[3] = {0.f, 0.f, 0.f}, pre[3];
+  if (in) { load3(a.dirs, i, d); load3(a.base_color, i, base); }
+  if (APP == GS_APP_SH) {
+    float *slab = sData + warp * kSlab;
+    if (a.deg > 0 && row0 < a.n) warp_load_rows(a.sh_rest, row0, a.n, slab, lane);
+    if (in) sh_decode(slab + lane * kRow, base, d[0], d[1], d[2], a.deg, pre);
+  } else {
+    float A[3] = {0.f, 0.f, 0.f};
+    if (in && a.deg > 0) {
+      float f[8], x[32], h1[16], h2[16];
+      load_features(a.features, i, f);
+      mlp_forward(sData, d[0], d[1], d[2], f, a.deg, x, h1, h2, A);
+    }
+#pragma unroll
+    for (int c = 0; c < 3; ++c) pre[c] = base[c] + 0.5f + A[c];
+  }
+  if (in) store3(a.color, i, fmaxf(pre[0], 0.f), fmaxf(pre[1], 0.f), fmaxf(pre[2], 0.f));
+}
+
+template <int APP>
+__global__ void __launch_bounds__(kBlock) k_appearance_bwd(AppearanceArgs a) {
+  extern __shared__ __align__(16) float smem[];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  float *sW = smem;
+  float *slab = APP == GS_APP_SH ? smem + warp * kSlab : smem + GS_MLP_WEIGHTS + warp * 32 * kActRow;
+  WgradAcc acc;
+  if (APP == GS_APP_NEURAL) {
+    load_weights_f32(a.weights, sW, tid, kBlock);
+    acc.clear();
+    __syncthreads();
+  }
+  const int64_t nchunks = (a.n + kBlock - 1) / kBlock;
+  for (int64_t chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x) {
+    reload_fence();
+    const int64_t i = chunk * kBlock + tid;
+    const int64_t row0 = chunk * kBlock + warp * 32;
+    const bool in = i < a.n;
+    float d[3] = {0.f, 0.f, 1.f}, base[3] = {0.f, 0.f, 0.f}, gcol[3] = {0.f, 0.f, 0.f};
+    if (in) { load3(a.dirs, i, d); load3(a.base_color, i, base); load3(a.g_color, i, gcol); }
+    float gp[3] = {0.f, 0.f, 0.f}, gd[3] = {0.f, 0.f, 0.f};
+    if (APP == GS_APP_SH) {
+      if (row0 < a.n) {
+        if (a.deg > 0) warp_load_rows(a.sh_rest, row0, a.n, slab, lane);
+        float *row = slab + lane * kRow;
+        if (in) {
+          float pre[3];
+          if (a.deg > 0) sh_decode(row, base, d[0], d[1], d[2], a.deg, pre);
+          else { pre[0] = base[0] + 0.5f; pre[1] = base[1] + 0.5f; pre[2] = base[2] + 0.5f; }
+#pragma unroll
+          for (int c = 0; c < 3; ++c) gp[c] = pre[c] > 0.f ? gcol[c] : 0.f;
+          sh_backward(row, gp, d[0], d[1], d[2], a.deg, gd);
+        }
+        warp_store_rows(a.g_sh_rest, row0, a.n, slab, lane);
+      }
+    } else {
+      float gf[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+      float *act_row = slab + lane * kActRow;
+      if (in && a.deg > 0) {
+        float f[8];
+        load_features(a.features, i, f);
+        mlp_backward(sW, act_row, d[0], d[1], d[2], f, a.deg, base, gcol, gp, gf, gd);
+      } else {
+        zero_act_row(act_row);
+#pragma unroll
+        for (int c = 0; c < 3; ++c) gp[c] = (base[c] + 0.5f) > 0.f ? gcol[c] : 0.f;
+      }
+      if (a.deg > 0 && row0 < a.n) wgrad_accumulate(slab, lane, acc);
+      if (in) {
+        float4 *gfp = reinterpret_cast<float4 *>(a.g_features) + 2 * i;
+        gfp[0] = make_float4(gf[0], gf[1], gf[2], gf[3]);
+        gfp[1] = make_float4(gf[4], gf[5], gf[6], gf[7]);
+      }
+    }
+    if (in) {
+      store3(a.g_base, i, gp[0], gp[1], gp[2]);
+      store3(a.g_dirs, i, gd[0], gd[1], gd[2]);
+    }
+  }
+  if (APP == GS_APP_NEURAL) {
+    __syncthreads();
+    wgrad_flush(acc, smem + GS_MLP_WEIGHTS, a.w_partials + (size_t)blockIdx.x * GS_MLP_WEIGHTS, tid);
+  }
+}
+
+inline int grid_for(int64_t n) { return (int)((n + kBlock - 1) / kBlock); }
+
+template <class K>
+void opt_in_smem(K kernel, size_t bytes) {
+  cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+}
+
+}  // namespace
+
+int launch_preprocess_fwd(int app, const PreprocessArgs &a, const CamDev &cam, cudaStream_t st) {
+  if (a.n == 0) return 0;
+  if (app == GS_APP_SH) k_preprocess_fwd<GS_APP_SH><<<grid_for(a.n), kBlock, 0, st>>>(a, cam);
+  else k_preprocess_fwd<GS_APP_NEURAL><<<grid_for(a.n), kBlock, 0, st>>>(a, cam);
+  return 1;
+}
+
+int launch_preprocess_bwd(int app, const PreprocessBwdArgs &a, const CamDev &cam, cudaStream_t st) {
+  if (app == GS_APP_SH) {
+    if (a.n == 0) return 0;
+    opt_in_smem(k_preprocess_bwd<GS_APP_SH>, kBwdSmemSH);
+    k_preprocess_bwd<GS_APP_SH><<<grid_for(a.n), kBlock, kBwdSmemSH, st>>>(a, cam);
+    return 1;
+  } else {
+    opt_in_smem(k_preprocess_bwd<GS_APP_NEURAL>, kBwdSmemNN);
+    k_preprocess_bwd<GS_APP_NEURAL><<<kWgradBlocks, kBlock, kBwdSmemNN, st>>>(a, cam);
+    k_wgrad_reduce<<<(GS_MLP_WEIGHTS + 127) / 128, 128, 0, st>>>(a.w_partials, kWgradBlocks, a.g_weights);
+    return 2;
+  }
+}
+
+int launch_appearance_fwd(int app, const AppearanceArgs &a, cudaStream_t st) {
+  if (a.n == 0) return 0;
+  if (app == GS_APP_SH) k_appearance_fwd<GS_APP_SH><<<grid_for(a.n), kBlock, 0, st>>>(a);
+  else k_appearance_fwd<GS_APP_NEURAL><<<grid_for(a.n), kBlock, 0, st>>>(a);
+  return 1;
+}
+
+int launch_appearance_bwd(int app, const AppearanceArgs &a, cudaStream_t st) {
+  if (app == GS_APP_SH) {
+    if (a.n == 0) return 0;
+    opt_in_smem(k_appearance_bwd<GS_APP_SH>, kBwdSmemSH);
+    k_appearance_bwd<GS_APP_SH><<<grid_for(a.n), kBlock, kBwdSmemSH, st>>>(a);
+    return 1;
+  } else {
+    opt_in_smem(k_appearance_bwd<GS_APP_NEURAL>, kBwdSmemNN);
+    k_appearance_bwd<GS_APP_NEURAL><<<kWgradBlocks, kBlock, kBwdSmemNN, st>>>(a);
+    k_wgrad_reduce<<<(GS_MLP_WEIGHTS + 127) / 128, 128, 0, st>>>(a.w_partials, kWgradBlocks, a.g_weights);
+    return 2;
+  }
+}
+
+}  // namespace gs

@@ -1,0 +1,331 @@
+// Ordering and binning: a stable LSD radix sort (8-bit digits, keys staged and ranked in shared
+// memory, no inter-block waiting), the prefix sum of tiles touched in depth order, instance
+// generation and per-tile ranges.
+//
+// Two-stage ordering: (1) the Gaussians are sorted once by their 32-bit depth key (ties keep the
+// index order because the sort is stable); (2) instances are emitted in that order and sorted by
+// tile id only (ceil(log2(tiles)) bits).  The result is the order by (tile, depth key, index).
+#include "gs_device.cuh"
+
+namespace gs {
+namespace {
+
+constexpr int kSortThreads = 256;
+constexpr int kSortWarps = kSortThreads / 32;
+constexpr int kItems = 16;
+constexpr int kSortTile = kSortThreads * kItems;   // 4096 elements per block iteration
+constexpr int kMaxSortBlocks = 592;                // 4 x 148 SMs
+constexpr unsigned kFull = 0xffffffffu;
+
+struct SortPlan { int blocks; int tiles_per_block; };
+
+SortPlan plan_for(int64_t count) {
+  const int64_t tiles = (count + kSortTile - 1) / kSortTile;
+  SortPlan p;
+  p.blocks = (int)(tiles < kMaxSortBlocks ? tiles : kMaxSortBlocks);
+  if (p.blocks < 1) p.blocks = 1;
+  p.tiles_per_block = (int)((tiles + p.blocks - 1) / p.blocks);
+  if (p.tiles_per_block < 1) p.tiles_per_block = 1;
+  p.blocks = (int)((tiles + p.tiles_per_block - 1) / p.tiles_per_block);
+  if (p.blocks < 1) p.blocks = 1;
+  return p;
+}
+
+// Digit histogram of each block's contiguous range: table[block][digit].
+__global__ void __launch_bounds__(kSortThreads) k_radix_hist(const uint32_t *__restrict__ keys, int64_t count,
+                                                             int shift, int tiles_per_block,
+                                                             uint32_t *__restrict__ table) {
+  __shared__ uint32_t s_hist[kSortWarps][256];
+  const int tid = threadIdx.x, warp = tid >> 5;
+  for (int k = tid; k < kSortWarps * 256; k += kSortThreads) (&s_hist[0][0])[k] = 0;
+  __syncthreads();
+  const int64_t begin = (int64_t)blockIdx.x * tiles_per_block * kSortTile;
+  int64_t end = begin + (int64_t)tiles_per_block * kSortTile;
+  if (end > count) end = count;
+  for (int64_t i = begin + tid; i < end; i += kSortThreads) {
+    const uint32_t d = (__ldg(keys + i) >> shift) & 255u;
+    atomicAdd(&s_hist[warp][d], 1u);
+  }
+  __syncthreads();
+  uint32_t s = 0;
+#pragma unroll
+  for (int w = 0; w < kSortWarps; ++w) s += s_hist[w][tid];
+  table[(size_t)blockIdx.x * 256 + tid] = s;
+}
+
+__device__ __forceinline__ uint32_t block_exclusive_scan_256(uint32_t v, uint32_t *s_warp_tot, int tid) {
+  const int lane = tid & 31, warp = tid >> 5;
+  uint32_t inc = v;
+#pragma unroll
+  for (int s = 1; s < 32; s <<= 1) {
+    const uint32_t t = __shfl_up_sync(kFull, inc, s);
+    if (lane >= s) inc += t;
+  }
+  if (lane == 31) s_warp_tot[warp] = inc;
+  __syncthreads();
+  uint32_t off = 0;
+#pragma unroll
+  for (int w = 0; w < kSortWarps; ++w) off += (w < warp) ? s_warp_tot[w] : 0u;
+  __syncthreads();
+  return off + inc - v;
+}
+
+// One pass: stable scatter of this block's range by the digit at `shift`.
+__global__ void __launch_bounds__(kSortThreads) k_radix_scatter(
+    const uint32_t *__restrict__ keys_in, const uint32_t *__restrict__ vals_in, uint32_t *__restrict__ keys_out,
+    uint32_t *__restrict__ vals_out, int64_t count, int shift, int tiles_per_block,
+    const uint32_t *__restrict__ table, int nblocks) {
+  __shared__ uint32_t s_keys[kSortTile];
+  __shared__ uint32_t s_vals[kSortTile];
+  __shared__ uint32_t s_warp_cnt[kSortWarps][256];
+  __shared__ uint32_t s_digit_start[256];
+  __shared__ uint32_t s_base[256];
+  __shared__ uint32_t s_warp_tot[kSortWarps];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t lt_mask = (1u << lane) - 1u;
+
+  // global base of every digit for this block: all smaller digits everywhere + the same digit
+  // in the blocks before this one
+  {
+    uint32_t before = 0, total = 0;
+    for (int b = 0; b < nblocks; ++b) {
+      const uint32_t v = __ldg(table + (size_t)b * 256 + tid);
+      total += v;
+      if (b < (int)blockIdx.x) before += v;
+    }
+    const uint32_t start = block_exclusive_scan_256(total, s_warp_tot, tid);
+    s_base[tid] = start + before;
+  }
+
+  const int64_t begin = (int64_t)blockIdx.x * tiles_per_block * kSortTile;
+  for (int t = 0; t < tiles_per_block; ++t) {
+    const int64_t tile_begin = begin + (int64_t)t * kSortTile;
+    if (tile_begin >= count) break;
+    const int valid_count = (int)min((int64_t)kSortTile, count - tile_begin);
+    for (int k = tid; k < kSortWarps * 256; k += kSortThreads) (&s_warp_cnt[0][0])[k] = 0;
+    __syncthreads();
+    uint32_t key[kItems], val[kItems];
+    unsigned short rank[kItems];
+#pragma unroll
+    for (int it = 0; it < kItems; ++it) {
+      const int local = warp * (32 * kItems) + it * 32 + lane;
+      const bool ok = local < valid_count;
+      const int64_t idx = tile_begin + local;
+      key[it] = ok ? __ldg(keys_in + idx) : 0xffffffffu;
+      val[it] = ok ? (vals_in ? __ldg(vals_in + idx) : (uint32_t)idx) : 0u;
+      const uint32_t d = ok ? ((key[it] >> shift) & 255u) : 255u;
+      const uint32_t peers = __match_any_sync(kFull, d);
+      const uint32_t prior = s_warp_cnt[warp][d];
+      rank[it] = (unsigned short)(prior + __popc(peers & lt_mask));
+      __syncwarp();
+      if ((peers & lt_mask) == 0) s_warp_cnt[warp][d] = prior + __popc(peers);
+      __syncwarp();
+    }
+    __syncthreads();
+    // per digit: exclusive scan over warps, then over digits
+    uint32_t cnt = 0;
+#pragma unroll
+    for (int w = 0; w < kSortWarps; ++w) {
+      const uint32_t c = s_warp_cnt[w][tid];
+      s_warp_cnt[w][tid] = cnt;
+      cnt += c;
+    }
+    const uint32_t dstart = block_exclusive_scan_256(cnt, s_warp_tot, tid);
+    s_digit_start[tid] = dstart;
+    __syncthreads();
+#pragma unroll
+    for (int it = 0; it < kItems; ++it) {
+      const int local = warp * (32 * kItems) + it * 32 + lane;
+      const uint32_t d = (local < valid_count) ? ((key[it] >> shift) & 255u) : 255u;
+      const uint32_t pos = s_digit_start[d] + s_warp_cnt[warp][d] + rank[it];
+      s_keys[pos] = key[it];
+      s_vals[pos] = val[it];
+    }
+    __syncthreads();
+    for (int j = tid; j < valid_count; j += kSortThreads) {
+      const uint32_t k = s_keys[j];
+      const uint32_t d = (k >> shift) & 255u;
+      const uint32_t gpos = s_base[d] + ((uint32_t)j - s_digit_start[d]);
+      keys_out[gpos] = k;
+      vals_out[gpos] = s_vals[j];
+    }
+    __syncthreads();
+    s_base[tid] += cnt;
+    __syncthreads();
+  }
+}
+
+// ---- tiles touched in depth order -----------------------------------------------------------
+constexpr int kScanBlock = 256;
+
+__device__ __forceinline__ uint32_t tiles_of(const uint16_t *rect, uint32_t g) {
+  const ushort4 r = __ldg(reinterpret_cast<const ushort4 *>(rect) + g);
+  return (uint32_t)(r.z - r.x) * (uint32_t)(r.w - r.y);
+}
+
+__global__ void __launch_bounds__(kScanBlock) k_tiles_block_sums(const uint32_t *__restrict__ order,
+                                                                 const uint16_t *__restrict__ rect, int64_t n,
+                                                                 uint32_t *__restrict__ block_sums) {
+  __shared__ uint32_t s_w[kScanBlock / 32];
+  const int64_t i = (int64_t)blockIdx.x * kScanBlock + threadIdx.x;
+  uint32_t v = i < n ? tiles_of(rect, __ldg(order + i)) : 0u;
+#pragma unroll
+  for (int s = 16; s > 0; s >>= 1) v += __shfl_xor_sync(kFull, v, s);
+  if ((threadIdx.x & 31) == 0) s_w[threadIdx.x >> 5] = v;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    uint32_t t = 0;
+#pragma unroll
+    for (int w = 0; w < kScanBlock / 32; ++w) t += s_w[w];
+    block_sums[blockIdx.x] = t;
+  }
+}
+
+// In-place exclusive scan of `count` values by one block.
+__global__ void __launch_bounds__(1024) k_scan_single_block(uint32_t *__restrict__ data, int count) {
+  __shared__ uint32_t s_w[32];
+  __shared__ uint32_t s_carry;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) s_carry = 0;
+  __syncthreads();
+  for (int base = 0; base < count; base += 1024) {
+    const int i = base + tid;
+    const uint32_t v = i < count ? data[i] : 0u;
+    uint32_t inc = v;
+#pragma unroll
+    for (int s = 1; s < 32; s <<= 1) {
+      const uint32_t t = __shfl_up_sync(kFull, inc, s);
+      if (lane >= s) inc += t;
+    }
+    if (lane == 31) s_w[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+      uint32_t w = s_w[lane], winc = w;
+#pragma unroll
+      for (int s = 1; s < 32; s <<= 1) {
+        const uint32_t t = __shfl_up_sync(kFull, winc, s);
+        if (lane >= s) winc += t;
+      }
+      s_w[lane] = winc - w;
+    }
+    __syncthreads();
+    const uint32_t carry = s_carry;
+    if (i < count) data[i] = carry + s_w[warp] + inc - v;
+    __syncthreads();
+    if (tid == 1023) s_carry = carry + s_w[warp] + inc;
+    __syncthreads();
+  }
+}
+
+// Emit the instances of each Gaussian, in depth order: tile ids ty-major then tx.  Small rects
+// are written by their own thread; large ones by the whole warp.
+__global__ void __launch_bounds__(kScanBlock) k_keygen(const uint32_t *__restrict__ order, const uint16_t *__restrict__ rect,
+                                                       const uint32_t *__restrict__ block_offsets, int64_t n, int gx,
+                                                       uint32_t *__restrict__ inst_tiles, uint32_t *__restrict__ inst_vals) {
+  __shared__ uint32_t s_w[kScanBlock / 32];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int64_t i = (int64_t)blockIdx.x * kScanBlock + tid;
+  uint32_t g = 0;
+  ushort4 r = make_ushort4(0, 0, 0, 0);
+  if (i < n) {
+    g = __ldg(order + i);
+    r = __ldg(reinterpret_cast<const ushort4 *>(rect) + g);
+  }
+  const uint32_t w = (uint32_t)(r.z - r.x), tiles = w * (uint32_t)(r.w - r.y);
+  uint32_t inc = tiles;
+#pragma unroll
+  for (int s = 1; s < 32; s <<= 1) {
+    const uint32_t t = __shfl_up_sync(kFull, inc, s);
+    if (lane >= s) inc += t;
+  }
+  if (lane == 31) s_w[warp] = inc;
+  __syncthreads();
+  uint32_t off = __ldg(block_offsets + blockIdx.x);
+#pragma unroll
+  for (int k = 0; k < kScanBlock / 32; ++k) off += (k < warp) ? s_w[k] : 0u;
+  off += inc - tiles;
+  constexpr uint32_t kSmall = 8;
+  if (tiles > 0 && tiles <= kSmall) {
+    uint32_t p = off;
+    for (uint32_t ty = r.y; ty < r.w; ++ty)
+      for (uint32_t tx = r.x; tx < r.z; ++tx) {
+        inst_tiles[p] = ty * gx + tx;
+        inst_vals[p] = g;
+        ++p;
+      }
+  }
+  uint32_t big = __ballot_sync(kFull, tiles > kSmall);
+  while (big) {
+    const int src = __ffs(big) - 1;
+    big &= big - 1;
+    const uint32_t s_off = __shfl_sync(kFull, off, src), s_tiles = __shfl_sync(kFull, tiles, src);
+    const uint32_t s_w_ = __shfl_sync(kFull, w, src), s_g = __shfl_sync(kFull, g, src);
+    const uint32_t s_x0 = __shfl_sync(kFull, (uint32_t)r.x, src), s_y0 = __shfl_sync(kFull, (uint32_t)r.y, src);
+    for (uint32_t k = lane; k < s_tiles; k += 32) {
+      const uint32_t ty = s_y0 + k / s_w_, tx = s_x0 + k % s_w_;
+      inst_tiles[s_off + k] = ty * gx + tx;
+      inst_vals[s_off + k] = s_g;
+    }
+  }
+}
+
+__global__ void k_tile_ranges(const uint32_t *__restrict__ sorted_tiles, int64_t P, uint32_t *__restrict__ ranges) {
+  const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (p >= P) return;
+  const uint32_t t = __ldg(sorted_tiles + p);
+  if (p == 0 || t != __ldg(sorted_tiles + p - 1)) ranges[2 * t] = (uint32_t)p;
+  if (p == P - 1 || t != __ldg(sorted_tiles + p + 1)) ranges[2 * t + 1] = (uint32_t)(p + 1);
+}
+
+}  // namespace
+
+size_t sort_scratch_bytes(int64_t count) { return (size_t)plan_for(count).blocks * 256 * sizeof(uint32_t); }
+
+int launch_radix_sort(const uint32_t *keys_in, const uint32_t *vals_in, uint32_t *keys_out, uint32_t *vals_out,
+                       uint32_t *tmp_keys, uint32_t *tmp_vals, int64_t count, int num_bits, void *scratch,
+                       cudaStream_t st) {
+  if (count <= 0) return 0;
+  const SortPlan plan = plan_for(count);
+  int passes = (num_bits + 7) / 8;
+  if (passes < 1) passes = 1;
+  uint32_t *table = static_cast<uint32_t *>(scratch);
+  const uint32_t *src_k = keys_in, *src_v = vals_in;
+  for (int p = 0; p < passes; ++p) {
+    const bool to_out = ((passes - 1 - p) % 2) == 0;
+    uint32_t *dst_k = to_out ? keys_out : tmp_keys, *dst_v = to_out ? vals_out : tmp_vals;
+    k_radix_hist<<<plan.blocks, kSortThreads, 0, st>>>(src_k, count, 8 * p, plan.tiles_per_block, table);
+    k_radix_scatter<<<plan.blocks, kSortThreads, 0, st>>>(src_k, src_v, dst_k, dst_v, count, 8 * p,
+                                                           plan.tiles_per_block, table, plan.blocks);
+    src_k = dst_k;
+    src_v = dst_v;
+  }
+  return 2 * passes;
+}
+
+size_t scan_scratch_bytes(int64_t n) { return (size_t)((n + kScanBlock - 1) / kScanBlock + 1) * sizeof(uint32_t); }
+
+int launch_tile_offsets(const uint32_t *depth_order, const uint16_t *rect, uint32_t *block_offsets, int64_t n,
+                        void *, cudaStream_t st) {
+  if (n <= 0) return 0;
+  const int blocks = (int)((n + kScanBlock - 1) / kScanBlock);
+  k_tiles_block_sums<<<blocks, kScanBlock, 0, st>>>(depth_order, rect, n, block_offsets);
+  k_scan_single_block<<<1, 1024, 0, st>>>(block_offsets, blocks);
+  return 2;
+}
+
+int launch_keygen(const uint32_t *depth_order, const uint16_t *rect, const uint32_t *block_offsets,
+                  uint32_t *inst_tiles, uint32_t *inst_vals, int64_t n, int gx, cudaStream_t st) {
+  if (n <= 0) return 0;
+  const int blocks = (int)((n + kScanBlock - 1) / kScanBlock);
+  k_keygen<<<blocks, kScanBlock, 0, st>>>(depth_order, rect, block_offsets, n, gx, inst_tiles, inst_vals);
+  return 1;
+}
+
+int launch_tile_ranges(const uint32_t *sorted_tiles, int64_t P, uint32_t *ranges, int num_tiles, cudaStream_t st) {
+  cudaMemsetAsync(ranges, 0, (size_t)num_tiles * 2 * sizeof(uint32_t), st);
+  if (P <= 0) return 0;
+  k_tile_ranges<<<(int)((P + 255) / 256), 256, 0, st>>>(sorted_tiles, P, ranges);
+  return 1;
+}
+
+}  // namespace gs

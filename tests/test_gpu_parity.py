@@ -1,0 +1,311 @@
+"""Parity of the CUDA path (through the C ABI) against the CPU oracle, element by element, on the
+same seeded inputs.  Integer work must match bit-exactly; images within 1e-4; gradients within
+1e-3 relative or 1e-5 absolute."""
+import math
+from types import SimpleNamespace
+
+import numpy as np
+import pytest
+
+from paper_2609_05255_b200 import scenes
+from gpu_helpers import (GRAD_ATOL, GRAD_RTOL, grad_mismatch, grad_names, image_mismatch, run_gpu)
+
+pytestmark = pytest.mark.gpu
+
+
+def small_workloads():
+    w1 = scenes.config1()
+    w2 = scenes.config2(n=20_011)                      # neural, ragged tail (not a multiple of 128)
+    w2s = scenes.config2(n=20_011, app=scenes.APP_SH)
+    w3 = scenes.config3(scenes.APP_NEURAL, n=30_000, width=400, height=264, views=8)
+    w3.cameras = [w3.cameras[3]]
+    w3s = scenes.config3(scenes.APP_SH, n=30_000, width=401, height=263, views=8)   # ragged image edge
+    w3s.cameras = [w3s.cameras[5]]
+    return {"config1": w1, "config2_neural": w2, "config2_sh": w2s, "config3_neural_small": w3,
+            "config3_sh_small": w3s}
+
+
+WORKLOADS = ["config1", "config2_neural", "config2_sh", "config3_neural_small", "config3_sh_small"]
+
+
+@pytest.fixture(scope="module")
+def results(oracle):
+    out = {}
+    for name, w in small_workloads().items():
+        cam = w.cameras[0]
+        G = scenes.upstream_gradient(cam, 4242)
+        gpu = run_gpu(w.scene, cam, G)
+        fwd, grads = oracle.render(w.scene, cam, G, with_abs=True)
+        out[name] = SimpleNamespace(w=w, cam=cam, G=G, gpu=gpu, fwd=fwd, grads=grads)
+    return out
+
+
+@pytest.mark.parametrize("name", WORKLOADS)
+def test_per_gaussian_floats(results, name):
+    r = results[name]; gpu, pre = r.gpu, r.fwd.pre
+    both = gpu.visible & pre.visible.astype(bool)
+    # visibility may differ only where a box edge sits on a pixel centre or opacity on 1/255
+    differ = np.nonzero(gpu.visible != pre.visible.astype(bool))[0]
+    assert len(differ) <= max(2, 1e-4 * gpu.n), f"{len(differ)} visibility flips"
+    assert both.sum() > 0.2 * gpu.n
+    assert np.abs(gpu.mean2d[both] - pre.mean2d[both]).max() < 2e-3          # pixels
+    ref = np.concatenate([pre.conic, pre.opacity[:, None]], 1)[both]
+    scale = np.abs(ref[:, :3]).max(1, keepdims=True)
+    err = np.abs(gpu.conic_opacity[both] - ref)
+    assert (err[:, :3] / scale).max() < 2e-4 and err[:, 3].max() < 1e-6
+    assert np.abs(gpu.color[both] - r.fwd.color[both]).max() < 2e-5
+    # the padded extent bounds the oracle's and stays within 2e-5 relative of it
+    val = gpu.extent[:, 0] >= 0
+    assert np.array_equal(val, pre.valid.astype(bool)) or (val != pre.valid.astype(bool)).sum() <= 2
+    vb = val & pre.valid.astype(bool)
+    rel = gpu.extent[vb] / np.maximum(pre.extent[vb], 1e-12) - 1
+    assert rel.min() > -1e-6 and rel.max() < 3e-5
+
+
+@pytest.mark.parametrize("name", WORKLOADS)
+def test_integer_stage_bit_exact(results, oracle, name):
+    r = results[name]; gpu, cam = r.gpu, r.cam
+    # depth keys: the same fp32 FMA chain on both sides
+    vis = gpu.visible
+    assert np.array_equal(gpu.depth_key[vis], r.fwd.pre.depth_bits[vis])
+    assert np.all(gpu.depth_key[~vis] == 0xFFFFFFFF)
+    # rects from the GPU's own fp32 centre and extent
+    valid = gpu.extent[:, 0] >= 0
+    rect, tt, P = oracle.tile_rects_f32(valid, gpu.mean2d, gpu.extent, cam.width, cam.height)
+    assert np.array_equal(rect, gpu.rect)
+    assert P == gpu.P and np.array_equal(tt, gpu.tiles_touched)
+    # depth order of the visible Gaussians: (depth key, index) ascending
+    V = int(vis.sum())
+    ids = np.nonzero(vis)[0]
+    order = ids[np.argsort(gpu.depth_key[ids], kind="stable")]
+    assert np.array_equal(gpu.depth_order[:V], order.astype(np.uint32))
+    # sorted instances and ranges
+    keys, vals, ranges = oracle.sorted_instances(rect, np.where(vis, gpu.depth_key, 0), cam.width, cam.height, P)
+    gpu_keys = (gpu.sorted_tiles.astype(np.uint64) << np.uint64(32)) | gpu.depth_key[gpu.sorted_vals].astype(np.uint64)
+    assert np.array_equal(gpu.sorted_vals, vals)
+    assert np.array_equal(gpu_keys, keys)
+    assert np.array_equal(gpu.tile_ranges, ranges)
+
+
+@pytest.mark.parametrize("name", WORKLOADS)
+def test_image(results, name):
+    r = results[name]; gpu, fwd = r.gpu, r.fwd
+    bad = image_mismatch(gpu.image, fwd.image, fwd.fragile)
+    assert bad.sum() == 0, f"{bad.sum()} pixels off, max {np.abs(gpu.image - fwd.image).max():.3e}"
+    frag = fwd.fragile.astype(bool)
+    assert frag.mean() < 1e-2
+    assert np.abs(gpu.final_T - fwd.final_T)[~frag].max() < 1e-4
+    same_lists = np.array_equal(gpu.sorted_vals, fwd.vals)
+    if same_lists:
+        assert (gpu.n_contrib != fwd.n_contrib)[~frag].sum() == 0
+    # invariants on the GPU's own output
+    assert gpu.final_T.min() >= 0 and gpu.final_T.max() <= 1
+
+
+@pytest.mark.parametrize("name", WORKLOADS)
+def test_blend_backward_2d_gradients(results, name):
+    r = results[name]; gpu, g = r.gpu, r.grads.blend
+    ref = np.concatenate([g.color, g.opacity[:, None], g.conic, g.mean2d], 1)
+    bad = grad_mismatch(gpu.g2d[:, :9], ref, r.grads.blend.abs_sum)
+    touched = _fragile_gaussians(r)
+    bad[touched] = False
+    assert bad.sum() == 0, f"{bad.sum()} of {bad.size} 2D gradient values off"
+
+
+def _fragile_gaussians(r):
+    """Gaussians that appear in the list of a tile holding a fragile pixel (a blend threshold within
+    1e-4): their gradients may legitimately differ by one pixel's contribution."""
+    fwd, cam = r.fwd, r.cam
+    gx = (cam.width + 15) // 16
+    ys, xs = np.nonzero(fwd.fragile)
+    out = np.zeros(r.gpu.n, bool)
+    for t in set(((ys // 16) * gx + xs // 16).tolist()):
+        s, e = fwd.ranges[t]
+        out[fwd.vals[s:e]] = True
+    return out
+
+
+@pytest.mark.parametrize("name", WORKLOADS)
+def test_parameter_gradients(results, oracle, name):
+    r = results[name]; gpu, sc, cam = r.gpu, r.w.scene, r.cam
+    # (a) the per-Gaussian backward kernel in isolation: oracle backward fed with the GPU's own 2D
+    #     gradients must match the GPU's parameter gradients by the literal rule
+    g2 = gpu.g2d.astype(np.float64)
+    vis = gpu.visible.astype(np.uint8)
+    pre = r.fwd.pre
+    ga = oracle.appearance_backward(sc, pre.dir, g2[:, 0:3], mask=vis)
+    gp = oracle.preprocess_backward(sc.means, sc.log_scales, sc.quats, sc.opacity_logits, cam, vis,
+                                    g2[:, 7:9], g2[:, 4:7], g2[:, 3], ga.dirs)
+    ref = dict(means=gp.means, log_scales=gp.log_scales, quats=gp.quats, opacity_logits=gp.opacity_logits,
+               base_color=ga.base_color, sh_rest=ga.sh_rest, features=ga.features, mlp_weights=ga.mlp_weights)
+    same_vis = gpu.visible == pre.visible.astype(bool)
+    for nm in grad_names(sc.app):
+        got = getattr(gpu.grads, nm)
+        bad = grad_mismatch(got, ref[nm])
+        if nm != "mlp_weights":
+            bad[~same_vis] = False
+        frac = bad.mean()
+        assert frac <= 2e-4, f"{nm}: {bad.sum()} of {bad.size} off (per-Gaussian backward)"
+    # (b) end to end against the oracle's own gradients
+    skip = _fragile_gaussians(r) | ~same_vis
+    for nm in grad_names(sc.app):
+        got, want = getattr(gpu.grads, nm), getattr(r.grads, nm)
+        bad = grad_mismatch(got, want)
+        if nm != "mlp_weights":
+            bad[skip] = False
+        assert bad.mean() <= 5e-3, f"{nm}: {bad.sum()} of {bad.size} off end to end"
+        # and every element within the fp32 conditioning bound of its accumulation
+        scale = np.abs(want).max()
+        assert np.abs(got - want)[~bad].max() <= max(GRAD_RTOL * scale, GRAD_ATOL)
+    # culled Gaussians: exact zeros
+    for nm in grad_names(sc.app):
+        if nm != "mlp_weights":
+            assert np.all(getattr(gpu.grads, nm)[~gpu.visible] == 0)
+
+
+@pytest.mark.parametrize("app", [scenes.APP_SH, scenes.APP_NEURAL])
+@pytest.mark.parametrize("deg", [0, 1, 2, 3])
+def test_appearance_separate_pass(oracle, app, deg):
+    import torch
+    from paper_2609_05255_b200 import api
+    n = 10_037
+    sc, dirs, gcol = scenes.config5(n, app)
+    sc.active_degree = deg
+    ctx = api.Context(0)
+    ds = api.upload_scene(sc, ctx.device)
+    d = torch.from_numpy(dirs).to(ctx.device); gc = torch.from_numpy(gcol).to(ctx.device)
+    color = torch.empty((n, 3), device=ctx.device)
+    api.gs_appearance_forward(ctx, ds, d, color)
+    grads = api.alloc_grads(n, app, ctx.device)
+    gd = torch.empty((n, 3), device=ctx.device)
+    api.gs_appearance_backward(ctx, ds, d, gc, grads, gd)
+    torch.cuda.synchronize()
+    ref_c, _ = oracle.appearance_forward(sc, dirs)
+    ref = oracle.appearance_backward(sc, dirs, gcol)
+    assert np.abs(color.cpu().numpy() - ref_c).max() < 2e-5
+    assert grad_mismatch(grads.base_color.cpu().numpy(), ref.base_color).sum() == 0
+    assert grad_mismatch(gd.cpu().numpy(), ref.dirs).sum() == 0
+    if app == scenes.APP_SH:
+        assert grad_mismatch(grads.sh_rest.cpu().numpy(), ref.sh_rest).sum() == 0
+    else:
+        assert grad_mismatch(grads.features.cpu().numpy(), ref.features).sum() == 0
+        assert grad_mismatch(grads.mlp_weights.cpu().numpy(), ref.mlp_weights).sum() == 0
+    ctx.close()
+
+
+def test_fused_equals_separate_pass(results, oracle):
+    """The paper's own validation: colours of the fused preprocess equal the separate pass run on the
+    same directions."""
+    import torch
+    from paper_2609_05255_b200 import api
+    for name in ("config2_neural", "config2_sh"):
+        r = results[name]; sc = r.w.scene
+        ctx = api.Context(0)
+        ds = api.upload_scene(sc, ctx.device)
+        dirs = torch.from_numpy(r.fwd.pre.dir.astype(np.float32)).to(ctx.device)
+        color = torch.empty((sc.n, 3), device=ctx.device)
+        api.gs_appearance_forward(ctx, ds, dirs, color)
+        torch.cuda.synchronize()
+        vis = r.gpu.visible
+        assert np.abs(color.cpu().numpy()[vis] - r.gpu.color[vis]).max() < 1e-5
+        ctx.close()
+
+
+# ------------------------------------------------------------------------------------------ edges
+
+def _empty_scene(app):
+    z = lambda *s: np.zeros(s, np.float32)
+    return scenes.Scene(z(0, 3), z(0, 3), z(0, 4), z(0), z(0, 3), app=app, active_degree=3,
+                        sh_rest=z(0, 15, 3) if app == 0 else None,
+                        features=np.zeros((0, 8), np.float16) if app == 1 else None,
+                        mlp_weights=np.zeros(816, np.float16) if app == 1 else None)
+
+
+@pytest.mark.parametrize("app", [0, 1])
+def test_empty_scene_renders_background(app):
+    cam = scenes.identity_camera(40, 24, 32.0, background=(0.25, 0.5, 0.75))
+    G = scenes.upstream_gradient(cam, 1)
+    gpu = run_gpu(_empty_scene(app), cam, G)
+    assert gpu.P == 0
+    assert np.all(gpu.image == np.array([0.25, 0.5, 0.75], np.float32)[:, None, None])
+    assert np.all(gpu.final_T == 1) and np.all(gpu.n_contrib == 0)
+    if app == 1:
+        assert np.all(gpu.grads.mlp_weights == 0)
+
+
+def test_image_smaller_than_a_tile_and_nan_inputs(oracle):
+    w = scenes.config1(200)
+    cam = scenes.identity_camera(11, 7, 16.0)
+    sc = w.scene
+    sc.means[5, 0] = np.nan; sc.opacity_logits[7] = np.inf; sc.quats[9] = 0
+    G = scenes.upstream_gradient(cam, 2)
+    gpu = run_gpu(sc, cam, G)
+    fwd, grads = oracle.render(sc, cam, G)
+    assert not gpu.visible[5] and not gpu.visible[7] and not gpu.visible[9]
+    assert image_mismatch(gpu.image, fwd.image, fwd.fragile).sum() == 0
+    assert np.array_equal(gpu.sorted_vals, fwd.vals)
+    for nm in grad_names(0):
+        assert np.all(np.isfinite(getattr(gpu.grads, nm)))
+        assert np.all(getattr(gpu.grads, nm)[[5, 7, 9]] == 0)
+
+
+def test_capacity_and_argument_errors():
+    import torch
+    from paper_2609_05255_b200 import api
+    w = scenes.config1(300)
+    cam = w.cameras[0]
+    ctx = api.Context(0)
+    ds = api.upload_scene(w.scene, ctx.device)
+    ccam = api.make_camera(cam)
+    proj = api.alloc_projected(ds.n, ctx.device)
+    P = api.gs_preprocess(ctx, ds, ccam, proj)
+    assert P > 10
+    binning = api.alloc_binning(ds.n, P, 64, 64, ctx.device)
+    image = torch.full((3, 64, 64), -7.0, device=ctx.device); fT = torch.empty((64, 64), device=ctx.device)
+    nc = torch.empty((64, 64), device=ctx.device, dtype=torch.int32)
+    ws = torch.empty((api.gs_workspace_bytes(ds.n, 64, 64, P),), device=ctx.device, dtype=torch.uint8)
+    with pytest.raises(api.GsError) as e:
+        api.gs_render_forward(ctx, ds.n, proj, ccam, P, P - 1, binning, image, fT, nc, ws)
+    assert e.value.status == api.GS_ERR_CAPACITY
+    assert torch.all(image == -7.0)                       # nothing was written
+    with pytest.raises(api.GsError) as e:
+        api.gs_render_forward(ctx, ds.n, proj, ccam, P, P, binning, image, fT, nc, ws[:1024])
+    assert e.value.status == api.GS_ERR_CAPACITY
+    ds.active_degree = 4
+    with pytest.raises(api.GsError) as e:
+        api.gs_preprocess(ctx, ds, ccam, proj)
+    assert e.value.status == api.GS_ERR_INVALID_ARG
+    ds.active_degree = 3
+    bad_cam = api.make_camera(cam); bad_cam.width = 0
+    with pytest.raises(api.GsError) as e:
+        api.gs_preprocess(ctx, ds, bad_cam, proj)
+    assert e.value.status == api.GS_ERR_INVALID_ARG
+    # the context is still usable afterwards
+    api.gs_render_forward(ctx, ds.n, proj, ccam, P, P, binning, image, fT, nc, ws)
+    torch.cuda.synchronize()
+    assert torch.all(image >= 0)
+    ctx.close()
+
+
+def test_run_twice_is_deterministic_for_integers_and_images():
+    w = scenes.config2(n=15_000)
+    a = run_gpu(w.scene, w.cameras[0])
+    b = run_gpu(w.scene, w.cameras[0])
+    for nm in ("depth_key", "rect", "depth_order", "sorted_tiles", "sorted_vals", "tile_ranges", "n_contrib"):
+        assert np.array_equal(getattr(a, nm), getattr(b, nm)), nm
+    assert np.array_equal(a.image, b.image) and np.array_equal(a.final_T, b.final_T)
+
+
+def test_single_large_gaussian_covers_every_tile(oracle):
+    """Degenerate case: one Gaussian covering the whole image (the warp-cooperative instance path)
+    in front of many small ones."""
+    w = scenes.config1(500)
+    sc = w.scene
+    sc.means[0] = [0.0, 0.0, 2.0]; sc.log_scales[0] = [1.0, 1.0, -1.0]; sc.opacity_logits[0] = 0.0
+    cam = scenes.identity_camera(200, 120, 100.0)
+    G = scenes.upstream_gradient(cam, 3)
+    gpu = run_gpu(sc, cam, G)
+    fwd, grads = oracle.render(sc, cam, G)
+    assert gpu.tiles_touched[0] == 13 * 8
+    assert np.array_equal(gpu.sorted_vals, fwd.vals) and np.array_equal(gpu.tile_ranges, fwd.ranges)
+    assert image_mismatch(gpu.image, fwd.image, fwd.fragile).sum() == 0
