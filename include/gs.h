@@ -147,8 +147,8 @@ GsStatus gs_render_forward(GsContext *ctx, int64_t n, const GsProjected *proj, c
                            size_t workspace_bytes, void *stream);
 
 /* Backward of the blend and of the preprocess, appearance included (Sec. 4 "CUDA
- * Implementation": the directional colour gradient also reaches the means).  dL_dimage is
- * [3,H,W].  Fills every member of `grads` that applies to scene->app.  Uses the same workspace
+ * Implementation": the directional colour gradient also reaches the means).  `final_T` and
+ * `n_contrib` are the forward's outputs for the same view, dL_dimage is [3,H,W].  Fills every member of `grads` that applies to scene->app.  Uses the same workspace
  * (contents of the forward call are not needed). */
 GsStatus gs_render_backward(GsContext *ctx, const GsScene *scene, const GsCamera *cam,
                             const GsProjected *proj, const GsBinning *bin, int64_t num_pairs,

@@ -502,10 +502,14 @@ struct Composited { uint32_t g; int pos; double alpha, T, power; bool clamped; }
 static void blend_pixel(double px, double py, const uint32_t* list, int64_t len, const double* mean2d,
                         const double* conic, const double* opacity, const double* color,
                         const double bg[3], double out[3], double* final_T, uint32_t* n_contrib,
-                        uint8_t* fragile, std::vector<Composited>* rec) {
+                        uint8_t* fragile, int32_t* fragile_pos, std::vector<Composited>* rec) {
+  // fragile: some evaluated pair lies within 1e-4 (relative) of a blend threshold, so an fp32
+  // evaluation may take the other branch; fragile_pos: list position of the first pair within
+  // 2e-5 (about ten fp32 roundings of alpha), or -1.
   double T = 1.0, C[3] = {0, 0, 0};
   uint32_t last = 0;
   bool frag = false;
+  int32_t fpos = -1;
   for (int64_t k = 0; k < len; ++k) {
     const uint32_t g = list[k];
     const double dx = px - mean2d[2 * g], dy = py - mean2d[2 * g + 1];
@@ -514,9 +518,11 @@ static void blend_pixel(double px, double py, const uint32_t* list, int64_t len,
     const double raw = opacity[g] * std::exp(power);
     const double alpha = std::min(kAlphaMax, raw);
     if (std::fabs(255.0 * alpha - 1.0) < 1e-4) frag = true;
+    if (std::fabs(255.0 * alpha - 1.0) < 2e-5 && fpos < 0) fpos = (int32_t)k;
     if (alpha < kAlphaMin) continue;
     const double Tn = T * (1.0 - alpha);
     if (std::fabs(Tn - kTmin) < 1e-8) frag = true;
+    if (std::fabs(Tn - kTmin) < 2e-9 && fpos < 0) fpos = (int32_t)k;
     if (Tn < kTmin) break;
     for (int c = 0; c < 3; ++c) C[c] += color[3 * g + c] * alpha * T;
     if (rec) rec->push_back({g, (int)k, alpha, T, power, raw > kAlphaMax});
@@ -527,13 +533,14 @@ static void blend_pixel(double px, double py, const uint32_t* list, int64_t len,
   *final_T = T;
   *n_contrib = last;
   if (fragile) *fragile = frag ? 1 : 0;
+  if (fragile_pos) *fragile_pos = fpos;
 }
 
-// Tiled forward: image[3,H,W], final_T[H,W], n_contrib[H,W], fragile[H,W] (u8).
+// Tiled forward: image[3,H,W], final_T[H,W], n_contrib[H,W], fragile[H,W] (u8), fragile_pos[H,W].
 void gso_blend_forward(int W, int H, const double* bg, const uint32_t* vals, const uint32_t* ranges,
                        const double* mean2d, const double* conic, const double* opacity,
                        const double* color, double* image, double* final_T, uint32_t* n_contrib,
-                       uint8_t* fragile) {
+                       uint8_t* fragile, int32_t* fragile_pos) {
   const int gx = (W + kTile - 1) / kTile, gy = (H + kTile - 1) / kTile;
 #pragma omp parallel for schedule(dynamic, 1)
   for (int tile = 0; tile < gx * gy; ++tile) {
@@ -544,7 +551,8 @@ void gso_blend_forward(int W, int H, const double* bg, const uint32_t* vals, con
         double out[3];
         blend_pixel(i + 0.5, j + 0.5, vals + s, (int64_t)e - s, mean2d, conic, opacity, color, bg, out,
                     &final_T[(size_t)j * W + i], &n_contrib[(size_t)j * W + i],
-                    fragile ? &fragile[(size_t)j * W + i] : nullptr, nullptr);
+                    fragile ? &fragile[(size_t)j * W + i] : nullptr,
+                    fragile_pos ? &fragile_pos[(size_t)j * W + i] : nullptr, nullptr);
         for (int c = 0; c < 3; ++c) image[((size_t)c * H + j) * W + i] = out[c];
       }
   }
@@ -563,7 +571,7 @@ void gso_blend_brute(int64_t n, int W, int H, const double* bg, const uint8_t* v
     for (int i = 0; i < W; ++i) {
       double out[3]; uint32_t nc;
       blend_pixel(i + 0.5, j + 0.5, order.data(), (int64_t)order.size(), mean2d, conic, opacity, color,
-                  bg, out, &final_T[(size_t)j * W + i], &nc, nullptr, nullptr);
+                  bg, out, &final_T[(size_t)j * W + i], &nc, nullptr, nullptr, nullptr);
       for (int c = 0; c < 3; ++c) image[((size_t)c * H + j) * W + i] = out[c];
     }
 }
@@ -590,7 +598,7 @@ void gso_blend_backward(int64_t n, int W, int H, const double* bg, int64_t P, co
         double out[3], fT; uint32_t nc;
         const double px = i + 0.5, py = j + 0.5;
         blend_pixel(px, py, vals + s, (int64_t)e - s, mean2d, conic, opacity, color, bg, out, &fT, &nc,
-                    nullptr, &rec);
+                    nullptr, nullptr, &rec);
         double Gp[3];
         for (int c = 0; c < 3; ++c) Gp[c] = G[((size_t)c * H + j) * W + i];
         // S = light arriving from behind the current entry, built back to front

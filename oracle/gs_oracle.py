@@ -192,12 +192,13 @@ def blend_forward(cam, vals, ranges, mean2d, conic, opacity, color):
     W, H = cam.width, cam.height
     bg = _f64(cam.background)
     o = SimpleNamespace(image=np.zeros((3, H, W)), final_T=np.zeros((H, W)),
-                        n_contrib=np.zeros((H, W), np.uint32), fragile=np.zeros((H, W), np.uint8))
+                        n_contrib=np.zeros((H, W), np.uint32), fragile=np.zeros((H, W), np.uint8),
+                        fragile_pos=np.zeros((H, W), np.int32))
     vals = np.ascontiguousarray(vals, np.uint32); ranges = np.ascontiguousarray(ranges, np.uint32)
     lib().gso_blend_forward(C.c_int(W), C.c_int(H), _dp(bg), _p(vals, C.c_uint32), _p(ranges, C.c_uint32),
                             _dp(_f64(mean2d)), _dp(_f64(conic)), _dp(_f64(opacity)), _dp(_f64(color)),
                             _dp(o.image), _dp(o.final_T), _p(o.n_contrib, C.c_uint32),
-                            _p(o.fragile, C.c_uint8))
+                            _p(o.fragile, C.c_uint8), _p(o.fragile_pos, C.c_int32))
     return o
 
 
@@ -255,7 +256,7 @@ def render_forward(scene, cam):
     bl = blend_forward(cam, vals, ranges, pre.mean2d, pre.conic, pre.opacity, color)
     return SimpleNamespace(pre=pre, color=color, residual=resid, rect=rect, tiles_touched=tiles_touched,
                            P=P, keys=keys, vals=vals, ranges=ranges, image=bl.image, final_T=bl.final_T,
-                           n_contrib=bl.n_contrib, fragile=bl.fragile)
+                           n_contrib=bl.n_contrib, fragile=bl.fragile, fragile_pos=bl.fragile_pos)
 
 
 def render_backward(scene, cam, fwd, G, with_abs=False):

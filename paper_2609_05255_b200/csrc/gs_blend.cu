@@ -79,9 +79,12 @@ __global__ void __launch_bounds__(kThreads) k_blend_fwd(CamDev cam, const uint32
   }
 }
 
-// Backward: walk each pixel's composited entries back to front, recover the transmittance in
-// front of each entry by division, and aggregate the nine per-Gaussian partial derivatives over
-// the tile (warp shuffles -> shared-memory accumulators -> one global atomic per value).
+// Backward: walk each pixel's composited entries back to front.  The transmittance in front of
+// an entry is recovered by dividing out (1 - alpha); the light arriving from behind it is summed
+// up on the way (both stay relatively accurate: a front-to-back replay that forms that light as
+// "final pixel - prefix" cancels badly for deep entries).  The nine per-Gaussian partial
+// derivatives are aggregated over the tile: warp shuffles -> shared-memory accumulators -> one
+// global atomic per value.
 // g2d row: (d colour r, g, b, d opacity) (d conic A, B, C, d mean u) (d mean v, -, -, -).
 __global__ void __launch_bounds__(kThreads) k_blend_bwd(CamDev cam, const uint32_t *__restrict__ ranges,
                                                         const uint32_t *__restrict__ vals,
@@ -105,11 +108,11 @@ __global__ void __launch_bounds__(kThreads) k_blend_bwd(CamDev cam, const uint32
   const uint32_t start = __ldg(ranges + 2 * tile), end = __ldg(ranges + 2 * tile + 1);
   const size_t pix = (size_t)py * cam.W + px, plane = (size_t)cam.W * cam.H;
   uint32_t nc = 0;
-  float T = 1.f, Gr = 0.f, Gg = 0.f, Gb = 0.f;
+  float Gr = 0.f, Gg = 0.f, Gb = 0.f, Tfin = 1.f;
   if (inside) {
     nc = __ldg(n_contrib + pix);
-    T = __ldg(final_T + pix);
     Gr = __ldg(dL_dimage + pix); Gg = __ldg(dL_dimage + plane + pix); Gb = __ldg(dL_dimage + 2 * plane + pix);
+    Tfin = __ldg(final_T + pix);
   }
   if (tid == 0) s_max = 0;
   __syncthreads();
@@ -120,7 +123,8 @@ __global__ void __launch_bounds__(kThreads) k_blend_bwd(CamDev cam, const uint32
   __syncthreads();
   const uint32_t maxc = s_max;
   if (maxc == 0 || start + maxc > end) return;   // nothing composited in this tile
-  float Sr = T * cam.bg[0], Sg = T * cam.bg[1], Sb = T * cam.bg[2];
+  float T = Tfin;                                          // transmittance behind the current entry
+  float Sr = Tfin * cam.bg[0], Sg = Tfin * cam.bg[1], Sb = Tfin * cam.bg[2];   // light from behind it
   const int nbatches = (int)((maxc + kBatch - 1) / kBatch);
   for (int b = nbatches - 1; b >= 0; --b) {
     __syncthreads();
@@ -134,7 +138,7 @@ __global__ void __launch_bounds__(kThreads) k_blend_bwd(CamDev cam, const uint32
 #pragma unroll
     for (int k = 0; k < 9; ++k) s_acc[tid][k] = 0.f;
     __syncthreads();
-    int jtop = (int)min((uint32_t)cnt, wmax > first ? wmax - first : 0u);
+    const int jtop = (int)min((uint32_t)cnt, wmax > first ? wmax - first : 0u);
     for (int j = jtop - 1; j >= 0; --j) {
       const uint32_t pos = first + (uint32_t)j;
       bool ok = pos < nc;
@@ -153,6 +157,7 @@ __global__ void __launch_bounds__(kThreads) k_blend_bwd(CamDev cam, const uint32
           const float Tb = T * inv;                 // transmittance in front of this entry
           const float w = alpha * Tb;
           v[0] = w * Gr; v[1] = w * Gg; v[2] = w * Gb;
+          // d pixel / d alpha = T c - S / (1 - alpha), S = everything composited behind this entry
           const float dalpha = Gr * (Tb * col.x - Sr * inv) + Gg * (Tb * col.y - Sg * inv) + Gb * (Tb * col.z - Sb * inv);
           if (c.y * e2 <= kAlphaMax) {              // not clamped: alpha depends on o and power
             v[3] = e2 * dalpha;

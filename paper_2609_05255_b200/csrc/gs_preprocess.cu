@@ -342,6 +342,13 @@ __device__ __forceinline__ void quat_rot(float r, float x, float y, float z, flo
   R[6] = 2.f * (x * z - r * y); R[7] = 2.f * (y * z + r * x); R[8] = 1.f - 2.f * (x * x + y * y);
 }
 
+// det(N N^T + 0.3 I) without the cancellation of a*c - b*b for elongated splats: by Lagrange's
+// identity |N0|^2 |N1|^2 - (N0.N1)^2 = |N0 x N1|^2, so det = |N0 x N1|^2 + 0.3 (|N0|^2 + |N1|^2) + 0.09.
+__device__ __forceinline__ float cov_det(const float N[6], float a, float c) {
+  const float cx = N[1] * N[5] - N[2] * N[4], cy = N[2] * N[3] - N[0] * N[5], cz = N[0] * N[4] - N[1] * N[3];
+  return cx * cx + cy * cy + cz * cz + kDilation * ((a - kDilation) + (c - kDilation)) + kDilation * kDilation;
+}
+
 // Everything the backward needs again is recomputed there; this is the forward only.
 __device__ __forceinline__ Geo project(const float mu[3], const float ls[3], const float q[4],
                                        float logit, const CamDev &cam) {
@@ -392,7 +399,7 @@ __device__ __forceinline__ Geo project(const float mu[3], const float ls[3], con
   const float a = N[0] * N[0] + N[1] * N[1] + N[2] * N[2] + kDilation;
   const float b = N[0] * N[3] + N[1] * N[4] + N[2] * N[5];
   const float c = N[3] * N[3] + N[4] * N[4] + N[5] * N[5] + kDilation;
-  const float det = a * c - b * b;
+  const float det = cov_det(N, a, c);
   if (!(det > 0.f) || !finite_f(det)) return g;
   const float idet = 1.f / det;
   const float tau = 2.f * logf(255.f * o);
@@ -477,8 +484,8 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_fwd(PreprocessArgs a, Cam
   }
   unsigned int tiles = 0;
   if (in) {
+    if (g.valid) reinterpret_cast<float2 *>(a.mean2d)[i] = make_float2(g.u, g.v);
     if (vis) {
-      reinterpret_cast<float2 *>(a.mean2d)[i] = make_float2(g.u, g.v);
       reinterpret_cast<float4 *>(a.conic_opacity)[i] = make_float4(g.A, g.B, g.C, g.o);
       a.color[3 * i] = fmaxf(pre[0], 0.f); a.color[3 * i + 1] = fmaxf(pre[1], 0.f); a.color[3 * i + 2] = fmaxf(pre[2], 0.f);
       tiles = (unsigned)((rect[2] - rect[0]) * (rect[3] - rect[1]));
@@ -543,7 +550,7 @@ __device__ __forceinline__ GeoGrads project_backward(const float mu[3], const fl
   const float a = N[0] * N[0] + N[1] * N[1] + N[2] * N[2] + kDilation;
   const float b = N[0] * N[3] + N[1] * N[4] + N[2] * N[5];
   const float c = N[3] * N[3] + N[4] * N[4] + N[5] * N[5] + kDilation;
-  const float idet = 1.f / (a * c - b * b);
+  const float idet = 1.f / cov_det(N, a, c);
   const float A = c * idet, B = -b * idet, C = a * idet;
   // conic -> covariance: G_cov = -Q G_Q Q, G_Q = [[gA, gB/2], [gB/2, gC]]
   const float h = 0.5f * gB;
