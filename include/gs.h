@@ -166,6 +166,32 @@ GsStatus gs_appearance_backward(GsContext *ctx, const GsScene *scene, const floa
                                 const float *dL_dcolor, GsGrads *grads, float *dL_ddirs,
                                 void *stream);
 
+/* gs_appearance_backward for callers that cannot allocate device memory (the paper has no
+ * counterpart; this entry point exists for integration only).  It is meant for code that runs where
+ * cudaMalloc is not an option: a plugin inside a host application that owns the whole memory budget
+ * and forbids allocations after start-up, a latency-critical loop that may not take the allocator's
+ * implicit synchronisation, or a process that cannot afford gs_create (which allocates the context's
+ * buffers).  It needs no GsContext, and it calls no cudaMalloc, cudaFree or any allocating library
+ * routine.  Neural appearance only (the SH backward uses no scratch: call gs_appearance_backward).
+ *
+ * The scratch the kernel needs - one row of 816 fp32 partial sums of the decoder-weight gradient per
+ * CTA - is a static device array compiled into the library: 1024 rows = 3,342,336 bytes, held by
+ * every GPU that loads the library until the process exits.  Each CTA covers at most 32 x 128
+ * Gaussians, so n may be at most 4,194,304; a larger n is rejected with GS_ERR_CAPACITY and a
+ * message, nothing launched.  Arguments and results are those of gs_appearance_backward (device
+ * pointers on the CURRENT device, 16-byte aligned); per-Gaussian results are bit-identical to it,
+ * grads->mlp_weights is the same sum taken in a different order.  error_text (host, may be NULL)
+ * receives a description when the status is not GS_OK.
+ *
+ * The first call on each device looks up the device address of the array; make that call before any
+ * stream capture begins.  All calls share the one array, which keeps the previous call's values:
+ * every row a launch reads is first overwritten in full by that launch, so nothing needs clearing,
+ * but two calls that overlap on the GPU (different streams, or one device used from two threads)
+ * race on it and give wrong weight gradients - serialise them. */
+GsStatus gs_appearance_backward_noalloc(const GsScene *scene, const float *dirs, const float *dL_dcolor,
+                                        GsGrads *grads, float *dL_ddirs, void *stream, char *error_text,
+                                        size_t error_text_bytes);
+
 /* Per-stage device timing, for benchmarks (the paper gives wall-clock protocols only, App. C; this
  * is the measurement hook of this library).  While enabled, every stage the library launches is
  * bracketed by CUDA events on the caller's stream.  gs_profile_collect synchronises those events,

@@ -347,3 +347,26 @@ class Renderer:
         gs_render_backward(self.ctx, scene, cam, self.proj, self.binning, self.num_pairs, self.final_T,
                            self.n_contrib, dL_dimage, self.grads, self.workspace, stream)
         return self.grads
+
+
+# ------------------------------------------------------------------------------------------------
+# The allocation-free neural appearance backward (no context, static device scratch in the library).
+# ------------------------------------------------------------------------------------------------
+NOALLOC_MAX_N = 4_194_304
+_lib.gs_appearance_backward_noalloc.argtypes = [C.POINTER(GsScene), _vp, _vp, C.POINTER(GsGrads), _vp, _vp,
+                                                C.c_char_p, C.c_size_t]
+_lib.gs_appearance_backward_noalloc.restype = C.c_int
+
+
+def gs_appearance_backward_noalloc(scene: DeviceScene, dirs: torch.Tensor, dL_dcolor: torch.Tensor,
+                                   grads: Grads, dL_ddirs: torch.Tensor, stream=None) -> None:
+    """Same results as gs_appearance_backward for the neural model, for callers that may not allocate:
+    no Context is needed and the library allocates nothing (its scratch is a static device array, good
+    for up to NOALLOC_MAX_N Gaussians).  Calls must not overlap on the GPU; the first call on a device
+    should precede any stream capture.  Raises GsError with the library's message on failure."""
+    cs, gg = scene.c_struct(), grads.c_struct()
+    msg = C.create_string_buffer(256)
+    st = _lib.gs_appearance_backward_noalloc(C.byref(cs), _ptr(dirs), _ptr(dL_dcolor), C.byref(gg), _ptr(dL_ddirs),
+                                             _stream_handle(stream), msg, len(msg))
+    if st != GS_OK:
+        raise GsError(st, msg.value.decode())

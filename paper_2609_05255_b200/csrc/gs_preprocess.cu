@@ -3,6 +3,8 @@
 // gradients move through per-warp shared-memory slabs so that global accesses stay coalesced;
 // decoder weights live in shared memory as fp32.
 #include <float.h>
+#include <stdio.h>
+#include <string.h>
 
 #include "gs_device.cuh"
 
@@ -885,3 +887,83 @@ int launch_appearance_bwd(int app, const AppearanceArgs &a, cudaStream_t st) {
 }
 
 }  // namespace gs
+
+// ---------------------------------------------------------------------------------------------
+// gs_appearance_backward_noalloc: the neural appearance backward for callers that must not
+// allocate.  Its only scratch, the per-block partial sums of the decoder-weight gradient, lives in
+// the file-scope device array below instead of memory obtained from cudaMalloc.
+// ---------------------------------------------------------------------------------------------
+namespace {
+constexpr int kNoAllocChunksPerBlock = 32;                       // chunks of 128 Gaussians per CTA
+constexpr int kNoAllocMaxBlocks = 1024;                          // rows of the static scratch
+constexpr int64_t kNoAllocMaxN = (int64_t)kNoAllocMaxBlocks * kNoAllocChunksPerBlock * 128;   // 4,194,304
+constexpr int kNoAllocMaxDevices = 64;
+}  // namespace
+
+// 1024 rows x 816 floats = 3,342,336 bytes, resident on every GPU that loads the library until the
+// process exits.  Row b is written in full by CTA b of every launch before anything reads it, so no
+// part of it has to start at zero; it keeps the previous call's values in between.
+static __device__ __align__(256) float gs_noalloc_partials[kNoAllocMaxBlocks * GS_MLP_WEIGHTS];
+
+extern "C" GsStatus gs_appearance_backward_noalloc(const GsScene *scene, const float *dirs, const float *dL_dcolor,
+                                                   GsGrads *grads, float *dL_ddirs, void *stream, char *error_text,
+                                                   size_t error_text_bytes) {
+  using namespace gs;
+  auto fail = [&](GsStatus code, const char *msg) {
+    if (error_text && error_text_bytes) snprintf(error_text, error_text_bytes, "%s", msg);
+    return code;
+  };
+  auto misaligned = [](const void *p) { return p == nullptr || (reinterpret_cast<uintptr_t>(p) & 15u) != 0; };
+  if (!scene || !grads) return fail(GS_ERR_INVALID_ARG, "scene / grads is NULL");
+  if (scene->app != GS_APP_NEURAL)
+    return fail(GS_ERR_UNSUPPORTED, "only the neural appearance backward uses scratch memory; call gs_appearance_backward for SH");
+  if (scene->active_degree < 0 || scene->active_degree > 3) return fail(GS_ERR_INVALID_ARG, "active_degree must be 0..3");
+  if (scene->n < 0) return fail(GS_ERR_INVALID_ARG, "n < 0");
+  if (scene->n > kNoAllocMaxN)
+    return fail(GS_ERR_CAPACITY, "n exceeds 4194304 Gaussians, the most the static scratch of this entry point covers; "
+                                 "split the call or use gs_appearance_backward");
+  if (misaligned(grads->mlp_weights)) return fail(GS_ERR_INVALID_ARG, "grads->mlp_weights is NULL or misaligned");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (scene->n == 0) {
+    if (cudaMemsetAsync(grads->mlp_weights, 0, sizeof(float) * GS_MLP_WEIGHTS, st) != cudaSuccess)
+      return fail(GS_ERR_CUDA, "cudaMemsetAsync failed");
+    return GS_OK;
+  }
+  if (misaligned(scene->base_color) || misaligned(scene->features) || misaligned(scene->mlp_weights) ||
+      misaligned(dirs) || misaligned(dL_dcolor) || misaligned(dL_ddirs) || misaligned(grads->base_color) ||
+      misaligned(grads->features))
+    return fail(GS_ERR_INVALID_ARG, "an input or output pointer is NULL or not 16-byte aligned");
+
+  // Set-up, once per device, with that device current: in host code the array's name is only a
+  // stand-in for the symbol, so the kernel must be given the address the runtime reports for it.
+  static float *scratch_of_device[kNoAllocMaxDevices] = {};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kNoAllocMaxDevices)
+    return fail(GS_ERR_CUDA, "cudaGetDevice failed or device index >= 64");
+  float *scratch = scratch_of_device[dev];
+  if (!scratch) {
+    void *p = nullptr;
+    const cudaError_t e = cudaGetSymbolAddress(&p, gs_noalloc_partials);
+    if (e != cudaSuccess || !p) return fail(GS_ERR_CUDA, cudaGetErrorString(e));
+    scratch = static_cast<float *>(p);
+    scratch_of_device[dev] = scratch;      // same value from every thread, so a racing store is benign
+  }
+
+  AppearanceArgs a;
+  memset(&a, 0, sizeof(a));
+  a.n = scene->n; a.deg = scene->active_degree;
+  a.base_color = scene->base_color; a.dirs = dirs;
+  a.features = reinterpret_cast<const __half *>(scene->features);
+  a.weights = reinterpret_cast<const __half *>(scene->mlp_weights);
+  a.g_color = dL_dcolor;
+  a.g_base = grads->base_color; a.g_features = grads->features; a.g_dirs = dL_ddirs;
+  a.w_partials = scratch; a.g_weights = grads->mlp_weights;
+  const int64_t chunks = (a.n + kBlock - 1) / kBlock;
+  const int blocks = (int)((chunks + kNoAllocChunksPerBlock - 1) / kNoAllocChunksPerBlock);   // <= 1024
+  opt_in_smem(k_appearance_bwd<GS_APP_NEURAL>, kBwdSmemNN);
+  k_appearance_bwd<GS_APP_NEURAL><<<blocks, kBlock, kBwdSmemNN, st>>>(a);
+  k_wgrad_reduce<<<(GS_MLP_WEIGHTS + 127) / 128, 128, 0, st>>>(scratch, blocks, a.g_weights);
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(GS_ERR_CUDA, cudaGetErrorString(e));
+  return GS_OK;
+}

@@ -1,0 +1,79 @@
+"""The allocation-free entry point gs_appearance_backward_noalloc (collected last on purpose: a run
+that stops at the first failure has then already run every other test).
+
+Who needs it: code that cannot call cudaMalloc where it runs - a plugin inside an application that
+hands out all device memory at start-up, a real-time loop that may not stall on the allocator, or a
+caller that cannot create a GsContext (gs_create allocates).  The library keeps the kernel's scratch
+(partial sums of the decoder-weight gradient) in a static device array instead.
+
+The test calls it through the C ABI twice in a row, with different sizes and data, and checks every
+output against gs_appearance_backward on the same inputs.
+"""
+import numpy as np
+import pytest
+
+from paper_2609_05255_b200 import scenes
+from gpu_helpers import grad_mismatch
+
+pytestmark = pytest.mark.gpu
+
+
+def _inputs(n, seed, device):
+    import torch
+    from paper_2609_05255_b200 import api
+    sc, dirs, gcol = scenes.config5(n, scenes.APP_NEURAL)
+    rng = np.random.default_rng(seed)
+    sc.features = rng.normal(0, 0.3, sc.features.shape).astype(np.float16)     # differ between the calls
+    gcol = rng.standard_normal(gcol.shape).astype(np.float32)
+    ds = api.upload_scene(sc, device)
+    return ds, torch.from_numpy(dirs).to(device), torch.from_numpy(gcol).to(device)
+
+
+def test_noalloc_matches_the_allocating_entry_point_twice_in_a_row():
+    import torch
+    from paper_2609_05255_b200 import api
+    ctx = api.Context(0)                       # only the existing entry point needs a context
+    dev = ctx.device
+    # second call smaller than the first: rows of the shared scratch left over from call 1 must not leak
+    for n, seed in ((70_001, 1), (9_000, 2)):
+        ds, dirs, gcol = _inputs(n, seed, dev)
+        want = api.alloc_grads(n, api.GS_APP_NEURAL, dev); want_d = torch.empty((n, 3), device=dev)
+        got = api.alloc_grads(n, api.GS_APP_NEURAL, dev); got_d = torch.full((n, 3), float("nan"), device=dev)
+        got.mlp_weights.fill_(float("nan")); got.features.fill_(float("nan")); got.base_color.fill_(float("nan"))
+        api.gs_appearance_backward(ctx, ds, dirs, gcol, want, want_d)
+        torch.cuda.synchronize()
+        before = torch.cuda.memory_allocated(dev)
+        api.gs_appearance_backward_noalloc(ds, dirs, gcol, got, got_d)
+        torch.cuda.synchronize()
+        assert torch.cuda.memory_allocated(dev) == before
+        # per-Gaussian outputs come from the same kernel code: identical bits
+        assert torch.equal(got.base_color, want.base_color)
+        assert torch.equal(got.features, want.features)
+        assert torch.equal(got_d, want_d)
+        # the weight gradient is the same sum in another order: the gradient tolerance of the other tests
+        w_got, w_want = got.mlp_weights.cpu().numpy(), want.mlp_weights.cpu().numpy()
+        assert np.all(np.isfinite(w_got)) and np.abs(w_want).max() > 1
+        assert grad_mismatch(w_got, w_want).sum() == 0
+    ctx.close()
+
+
+def test_noalloc_rejects_what_it_cannot_serve():
+    import torch
+    from paper_2609_05255_b200 import api
+    dev = torch.device("cuda", 0)
+    ds, dirs, gcol = _inputs(256, 3, dev)
+    grads = api.alloc_grads(256, api.GS_APP_NEURAL, dev); gd = torch.empty((256, 3), device=dev)
+    grads.mlp_weights.fill_(7.0)
+    cs = ds.c_struct()
+    cs.n = api.NOALLOC_MAX_N + 1               # only the size is checked before the refusal: nothing is read
+    import ctypes as C
+    msg = C.create_string_buffer(256)
+    st = api._lib.gs_appearance_backward_noalloc(C.byref(cs), dirs.data_ptr(), gcol.data_ptr(),
+                                                 C.byref(grads.c_struct()), gd.data_ptr(), None, msg, len(msg))
+    assert st == api.GS_ERR_CAPACITY and b"4194304" in msg.value
+    torch.cuda.synchronize()
+    assert torch.all(grads.mlp_weights == 7.0)  # nothing was launched
+    ds.app = api.GS_APP_SH
+    with pytest.raises(api.GsError) as e:
+        api.gs_appearance_backward_noalloc(ds, dirs, gcol, grads, gd)
+    assert e.value.status == api.GS_ERR_UNSUPPORTED
