@@ -170,7 +170,8 @@ def run_ours(args):
     results = {}
     sampler = ClockSampler(local)
     clocks = None
-    for app, tag in ((scenes.APP_NEURAL, "neural"), (scenes.APP_SH, "sh")):
+    arms = [(scenes.APP_NEURAL, "neural")] + ([] if args.skip_sh else [(scenes.APP_SH, "sh")])
+    for app, tag in arms:
         host, ds, r, pairs = make_arm(app)
         if tag == "neural":
             sampler.start()
@@ -191,7 +192,7 @@ def run_ours(args):
                             entries=entries, visible=visible, host=host, ds=ds, r=r)
 
     # ---- end to end through the public API with host buffers (neural arm)
-    e2e = measure_e2e(api, torch, ctx, results["neural"], cams, G, views, args, timed, dev)
+    e2e = None if args.skip_e2e else measure_e2e(api, torch, ctx, results["neural"], cams, G, views, args, timed, dev)
 
     # ---- appearance-decode sweep (separate-pass kernels, HBM resident)
     decode = None if args.skip_decode else decode_sweep(api, torch, ctx, dev, peaks, args)
@@ -222,8 +223,9 @@ def run_ours(args):
         "stages_ms_per_step": {k: round(v, 4) for k, v in stage_ms.items() if v > 0},
         "stage_share": {k: round(v / total_stage, 4) for k, v in stage_ms.items() if v > 0},
         "pairs_per_view": neural["pairs"], "visible_per_view": neural["visible"] / views,
-        "sh": {"ms_per_step": results["sh"]["ms"],
-               "stages_ms_per_step": {k: round(v, 4) for k, v in results["sh"]["stage_ms"].items() if v > 0}},
+        "sh": None if args.skip_sh else {
+            "ms_per_step": results["sh"]["ms"],
+            "stages_ms_per_step": {k: round(v, 4) for k, v in results["sh"]["stage_ms"].items() if v > 0}},
         "appearance_decode": decode,
         "peaks": peaks,
     }
@@ -399,6 +401,8 @@ def main():
     ap.add_argument("--quick", action="store_true", help="decode sweep at 1M only")
     ap.add_argument("--skip-decode", action="store_true")
     ap.add_argument("--skip-cpu", action="store_true")
+    ap.add_argument("--skip-sh", action="store_true", help="time the neural arm only (profiling runs)")
+    ap.add_argument("--skip-e2e", action="store_true")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3

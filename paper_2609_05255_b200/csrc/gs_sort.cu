@@ -14,7 +14,7 @@ constexpr int kSortThreads = 256;
 constexpr int kSortWarps = kSortThreads / 32;
 constexpr int kItems = 16;
 constexpr int kSortTile = kSortThreads * kItems;   // 4096 elements per block iteration
-constexpr int kMaxSortBlocks = 592;                // 4 x 148 SMs
+constexpr int kMaxSortBlocks = 444;                // 3 resident CTAs x 148 SMs: one full wave
 constexpr unsigned kFull = 0xffffffffu;
 
 struct SortPlan { int blocks; int tiles_per_block; };
@@ -50,7 +50,40 @@ __global__ void __launch_bounds__(kSortThreads) k_radix_hist(const uint32_t *__r
   uint32_t s = 0;
 #pragma unroll
   for (int w = 0; w < kSortWarps; ++w) s += s_hist[w][tid];
-  table[(size_t)blockIdx.x * 256 + tid] = s;
+  table[(size_t)tid * gridDim.x + blockIdx.x] = s;   // digit-major: one contiguous row per digit
+}
+
+// Per digit (one CTA each): exclusive scan of the row of per-block counts, in place, and the row
+// total.  Done once per pass here instead of by every scatter CTA.
+__global__ void __launch_bounds__(256) k_radix_scan_rows(uint32_t *__restrict__ table, int nblocks,
+                                                         uint32_t *__restrict__ totals) {
+  __shared__ uint32_t s_w[8];
+  __shared__ uint32_t s_carry;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  uint32_t *row = table + (size_t)blockIdx.x * nblocks;
+  if (tid == 0) s_carry = 0;
+  __syncthreads();
+  for (int base = 0; base < nblocks; base += 256) {
+    const int i = base + tid;
+    const uint32_t v = i < nblocks ? row[i] : 0u;
+    uint32_t inc = v;
+#pragma unroll
+    for (int s = 1; s < 32; s <<= 1) {
+      const uint32_t t = __shfl_up_sync(0xffffffffu, inc, s);
+      if (lane >= s) inc += t;
+    }
+    if (lane == 31) s_w[warp] = inc;
+    __syncthreads();
+    uint32_t off = 0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) off += (w < warp) ? s_w[w] : 0u;
+    const uint32_t carry = s_carry;
+    if (i < nblocks) row[i] = carry + off + inc - v;
+    __syncthreads();
+    if (tid == 255) s_carry = carry + off + inc;
+    __syncthreads();
+  }
+  if (tid == 0) totals[blockIdx.x] = s_carry;
 }
 
 __device__ __forceinline__ uint32_t block_exclusive_scan_256(uint32_t v, uint32_t *s_warp_tot, int tid) {
@@ -71,10 +104,10 @@ __device__ __forceinline__ uint32_t block_exclusive_scan_256(uint32_t v, uint32_
 }
 
 // One pass: stable scatter of this block's range by the digit at `shift`.
-__global__ void __launch_bounds__(kSortThreads) k_radix_scatter(
+__global__ void __launch_bounds__(kSortThreads, 3) k_radix_scatter(
     const uint32_t *__restrict__ keys_in, const uint32_t *__restrict__ vals_in, uint32_t *__restrict__ keys_out,
     uint32_t *__restrict__ vals_out, int64_t count, int shift, int tiles_per_block,
-    const uint32_t *__restrict__ table, int nblocks) {
+    const uint32_t *__restrict__ table, const uint32_t *__restrict__ totals, int nblocks) {
   __shared__ uint32_t s_keys[kSortTile];
   __shared__ uint32_t s_vals[kSortTile];
   __shared__ uint32_t s_warp_cnt[kSortWarps][256];
@@ -84,17 +117,11 @@ __global__ void __launch_bounds__(kSortThreads) k_radix_scatter(
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t lt_mask = (1u << lane) - 1u;
 
-  // global base of every digit for this block: all smaller digits everywhere + the same digit
-  // in the blocks before this one
+  // global base of every digit for this block: all smaller digits everywhere (scan of the row
+  // totals) + the same digit in the blocks before this one (the row prefix from k_radix_scan_rows)
   {
-    uint32_t before = 0, total = 0;
-    for (int b = 0; b < nblocks; ++b) {
-      const uint32_t v = __ldg(table + (size_t)b * 256 + tid);
-      total += v;
-      if (b < (int)blockIdx.x) before += v;
-    }
-    const uint32_t start = block_exclusive_scan_256(total, s_warp_tot, tid);
-    s_base[tid] = start + before;
+    const uint32_t start = block_exclusive_scan_256(__ldg(totals + tid), s_warp_tot, tid);
+    s_base[tid] = start + __ldg(table + (size_t)tid * nblocks + blockIdx.x);
   }
 
   const int64_t begin = (int64_t)blockIdx.x * tiles_per_block * kSortTile;
@@ -106,6 +133,7 @@ __global__ void __launch_bounds__(kSortThreads) k_radix_scatter(
     __syncthreads();
     uint32_t key[kItems], val[kItems];
     unsigned short rank[kItems];
+    // all loads first (independent, in flight together), then the serial ranking chain
 #pragma unroll
     for (int it = 0; it < kItems; ++it) {
       const int local = warp * (32 * kItems) + it * 32 + lane;
@@ -113,13 +141,21 @@ __global__ void __launch_bounds__(kSortThreads) k_radix_scatter(
       const int64_t idx = tile_begin + local;
       key[it] = ok ? __ldg(keys_in + idx) : 0xffffffffu;
       val[it] = ok ? (vals_in ? __ldg(vals_in + idx) : (uint32_t)idx) : 0u;
+    }
+#pragma unroll
+    for (int it = 0; it < kItems; ++it) {
+      const int local = warp * (32 * kItems) + it * 32 + lane;
+      const bool ok = local < valid_count;
       const uint32_t d = ok ? ((key[it] >> shift) & 255u) : 255u;
+      // lanes with the same digit form a group; its first lane bumps the warp's counter once and
+      // hands the old value to the group.  A warp's shared-memory atomics execute in program order,
+      // so the 16 items need no barrier between them and their latencies overlap.
       const uint32_t peers = __match_any_sync(kFull, d);
-      const uint32_t prior = s_warp_cnt[warp][d];
+      const int leader = __ffs(peers) - 1;
+      uint32_t prior = 0;
+      if (lane == leader) prior = atomicAdd(&s_warp_cnt[warp][d], (uint32_t)__popc(peers));
+      prior = __shfl_sync(kFull, prior, leader);
       rank[it] = (unsigned short)(prior + __popc(peers & lt_mask));
-      __syncwarp();
-      if ((peers & lt_mask) == 0) s_warp_cnt[warp][d] = prior + __popc(peers);
-      __syncwarp();
     }
     __syncthreads();
     // per digit: exclusive scan over warps, then over digits
@@ -279,7 +315,7 @@ __global__ void k_tile_ranges(const uint32_t *__restrict__ sorted_tiles, int64_t
 
 }  // namespace
 
-size_t sort_scratch_bytes(int64_t count) { return (size_t)plan_for(count).blocks * 256 * sizeof(uint32_t); }
+size_t sort_scratch_bytes(int64_t count) { return ((size_t)plan_for(count).blocks + 1) * 256 * sizeof(uint32_t); }
 
 int launch_radix_sort(const uint32_t *keys_in, const uint32_t *vals_in, uint32_t *keys_out, uint32_t *vals_out,
                        uint32_t *tmp_keys, uint32_t *tmp_vals, int64_t count, int num_bits, void *scratch,
@@ -289,17 +325,19 @@ int launch_radix_sort(const uint32_t *keys_in, const uint32_t *vals_in, uint32_t
   int passes = (num_bits + 7) / 8;
   if (passes < 1) passes = 1;
   uint32_t *table = static_cast<uint32_t *>(scratch);
+  uint32_t *totals = table + (size_t)plan.blocks * 256;
   const uint32_t *src_k = keys_in, *src_v = vals_in;
   for (int p = 0; p < passes; ++p) {
     const bool to_out = ((passes - 1 - p) % 2) == 0;
     uint32_t *dst_k = to_out ? keys_out : tmp_keys, *dst_v = to_out ? vals_out : tmp_vals;
     k_radix_hist<<<plan.blocks, kSortThreads, 0, st>>>(src_k, count, 8 * p, plan.tiles_per_block, table);
+    k_radix_scan_rows<<<256, 256, 0, st>>>(table, plan.blocks, totals);
     k_radix_scatter<<<plan.blocks, kSortThreads, 0, st>>>(src_k, src_v, dst_k, dst_v, count, 8 * p,
-                                                           plan.tiles_per_block, table, plan.blocks);
+                                                           plan.tiles_per_block, table, totals, plan.blocks);
     src_k = dst_k;
     src_v = dst_v;
   }
-  return 2 * passes;
+  return 3 * passes;
 }
 
 size_t scan_scratch_bytes(int64_t n) { return (size_t)((n + kScanBlock - 1) / kScanBlock + 1) * sizeof(uint32_t); }
