@@ -84,7 +84,9 @@ typedef struct {
 /* Per-Gaussian results of gs_preprocess (caller-allocated device buffers). */
 typedef struct {
   float *mean2d;         /* [n,2]  projected centre in pixels                                  */
-  float *conic_opacity;  /* [n,4]  inverse 2D covariance (A,B,C) and opacity                    */
+  float *conic_opacity;  /* [n,4]  (l11, l21, l22, opacity): the inverse 2D covariance ("conic") in
+                                   Cholesky form, Q = L L^T with L = [[l11, 0], [l21, l22]], i.e.
+                                   Q = [[l11^2, l11 l21], [l11 l21, l21^2 + l22^2]]                */
   float *color;          /* [n,3]  decoded view-dependent colour (Eq. 2)                       */
   uint32_t *depth_key;   /* [n]    bit pattern of the fp32 camera depth; 0xFFFFFFFF if culled  */
   uint16_t *rect;        /* [n,4]  tile rectangle (tx0, ty0, tx1, ty1), half open; all zero if

@@ -497,7 +497,9 @@ void gso_tile_ranges(int64_t P, const uint64_t* keys, int num_tiles, uint32_t* r
 // Blend.  One pixel, one ordered list.  Returns through the pointers; `rec` (optional)
 // records every composited entry for the backward pass.
 // ---------------------------------------------------------------------------------------
-struct Composited { uint32_t g; int pos; double alpha, T, power; bool clamped; };
+// `ghost`: a pair the oracle did NOT composite although it sits within 1e-4 of a threshold, so an
+// fp32 evaluation might; it only feeds the flip allowance of the backward.
+struct Composited { uint32_t g; int pos; double alpha, T, power; bool clamped; bool ghost; };
 
 static void blend_pixel(double px, double py, const uint32_t* list, int64_t len, const double* mean2d,
                         const double* conic, const double* opacity, const double* color,
@@ -505,7 +507,8 @@ static void blend_pixel(double px, double py, const uint32_t* list, int64_t len,
                         uint8_t* fragile, int32_t* fragile_pos, std::vector<Composited>* rec) {
   // fragile: some evaluated pair lies within 1e-4 (relative) of a blend threshold, so an fp32
   // evaluation may take the other branch; fragile_pos: list position of the first pair within
-  // 2e-5 (about ten fp32 roundings of alpha), or -1.
+  // tolerance, or -1.  (fp32 alpha can be off by 1e-4 for footprints hundreds of pixels wide, and the
+  // transmittance is a product of up to a thousand fp32 factors.)
   double T = 1.0, C[3] = {0, 0, 0};
   uint32_t last = 0;
   bool frag = false;
@@ -518,14 +521,41 @@ static void blend_pixel(double px, double py, const uint32_t* list, int64_t len,
     const double raw = opacity[g] * std::exp(power);
     const double alpha = std::min(kAlphaMax, raw);
     if (std::fabs(255.0 * alpha - 1.0) < 1e-4) frag = true;
-    if (std::fabs(255.0 * alpha - 1.0) < 2e-5 && fpos < 0) fpos = (int32_t)k;
-    if (alpha < kAlphaMin) continue;
+    const bool near_alpha = std::fabs(255.0 * alpha - 1.0) < 1e-4;
+    if (near_alpha && fpos < 0) fpos = (int32_t)k;
+    // the 0.99 clamp switches the gradient of the pair on and off: also a branch fp32 may flip
+    if (std::fabs(raw - kAlphaMax) < 1e-4 * kAlphaMax) { frag = true; if (fpos < 0) fpos = (int32_t)k; }
+    if (alpha < kAlphaMin) {
+      if (near_alpha && rec) rec->push_back({g, (int)k, alpha, T, power, false, true});
+      continue;
+    }
     const double Tn = T * (1.0 - alpha);
-    if (std::fabs(Tn - kTmin) < 1e-8) frag = true;
-    if (std::fabs(Tn - kTmin) < 2e-9 && fpos < 0) fpos = (int32_t)k;
-    if (Tn < kTmin) break;
+    if (std::fabs(Tn - kTmin) < 1e-7) frag = true;
+    const bool near_stop = std::fabs(Tn - kTmin) < 1e-7;
+    if (near_stop && fpos < 0) fpos = (int32_t)k;
+    if (Tn < kTmin) {
+      if (near_stop && rec) {
+        // The stop is within tolerance: an fp32 evaluation may composite this pair and walk on.
+        // Record what it would then add, as ghosts, until the transmittance is clearly below the
+        // threshold.
+        double Tg = T;
+        for (int64_t kk = k; kk < len; ++kk) {
+          const uint32_t gg = list[kk];
+          const double ex = px - mean2d[2 * gg], ey = py - mean2d[2 * gg + 1];
+          const double pw = -0.5 * (conic[3 * gg] * ex * ex + conic[3 * gg + 2] * ey * ey) - conic[3 * gg + 1] * ex * ey;
+          if (pw > 0) continue;
+          const double rw = opacity[gg] * std::exp(pw), al = std::min(kAlphaMax, rw);
+          if (al < kAlphaMin) continue;
+          const double Tgn = Tg * (1.0 - al);
+          if (kk > k && Tgn < kTmin - 1e-7) break;
+          rec->push_back({gg, (int)kk, al, Tg, pw, rw > kAlphaMax, true});
+          Tg = Tgn;
+        }
+      }
+      break;
+    }
     for (int c = 0; c < 3; ++c) C[c] += color[3 * g + c] * alpha * T;
-    if (rec) rec->push_back({g, (int)k, alpha, T, power, raw > kAlphaMax});
+    if (rec) rec->push_back({g, (int)k, alpha, T, power, raw > kAlphaMax, false});
     T = Tn;
     last = (uint32_t)(k + 1);
   }
@@ -578,15 +608,18 @@ void gso_blend_brute(int64_t n, int W, int H, const double* bg, const uint8_t* v
 
 // Backward of the blend for L with upstream G = dL/dimage [3,H,W].
 // Outputs per Gaussian: g_color[n,3], g_opacity[n], g_conic[n,3] (A,B,C), g_mean2d[n,2];
-// abs_* (optional, same shapes packed as [n,9] = colour3, opacity, conic3, mean2): the sums of
-// the absolute values of the accumulated terms (conditioning of the fp32 summation).
+// abs_sum (optional, [n,9] = colour3, opacity, conic3, mean2): the sums of the absolute values of
+// the accumulated terms (conditioning of the fp32 summation).  flip_sum (optional, [n,9]): the
+// absolute values of the terms that an fp32 evaluation could add, drop or rescale because some pair
+// of the pixel sits within 1e-4 of a blend threshold - that pair and every entry behind it.
 void gso_blend_backward(int64_t n, int W, int H, const double* bg, int64_t P, const uint32_t* vals,
                         const uint32_t* ranges, const double* mean2d, const double* conic,
                         const double* opacity, const double* color, const double* G,
                         double* g_color, double* g_opacity, double* g_conic, double* g_mean2d,
-                        double* abs_sum) {
+                        double* abs_sum, double* flip_sum) {
   const int gx = (W + kTile - 1) / kTile, gy = (H + kTile - 1) / kTile;
-  std::vector<double> inst((size_t)P * 9, 0.0), inst_abs(abs_sum ? (size_t)P * 9 : 0, 0.0);
+  std::vector<double> inst((size_t)P * 9, 0.0), inst_abs(abs_sum ? (size_t)P * 9 : 0, 0.0),
+      inst_flip(flip_sum ? (size_t)P * 9 : 0, 0.0);
 #pragma omp parallel for schedule(dynamic, 1)
   for (int tile = 0; tile < gx * gy; ++tile) {
     const int tx = tile % gx, ty = tile / gx;
@@ -595,10 +628,10 @@ void gso_blend_backward(int64_t n, int W, int H, const double* bg, int64_t P, co
     for (int j = ty * kTile; j < std::min(H, (ty + 1) * kTile); ++j)
       for (int i = tx * kTile; i < std::min(W, (tx + 1) * kTile); ++i) {
         rec.clear();
-        double out[3], fT; uint32_t nc;
+        double out[3], fT; uint32_t nc; int32_t fpos = -1;
         const double px = i + 0.5, py = j + 0.5;
         blend_pixel(px, py, vals + s, (int64_t)e - s, mean2d, conic, opacity, color, bg, out, &fT, &nc,
-                    nullptr, nullptr, &rec);
+                    nullptr, &fpos, &rec);
         double Gp[3];
         for (int c = 0; c < 3; ++c) Gp[c] = G[((size_t)c * H + j) * W + i];
         // S = light arriving from behind the current entry, built back to front
@@ -608,13 +641,20 @@ void gso_blend_backward(int64_t n, int W, int H, const double* bg, int64_t P, co
           const uint32_t g = r.g;
           double* acc = inst.data() + ((size_t)s + r.pos) * 9;
           double* aab = abs_sum ? inst_abs.data() + ((size_t)s + r.pos) * 9 : nullptr;
-          auto add = [&](int slot, double v) { acc[slot] += v; if (aab) aab[slot] += std::fabs(v); };
+          double* afl = (flip_sum && fpos >= 0 && r.pos >= fpos) ? inst_flip.data() + ((size_t)s + r.pos) * 9 : nullptr;
+          bool real = !r.ghost;
+          auto add = [&](int slot, double v) {
+            if (real) { acc[slot] += v; if (aab) aab[slot] += std::fabs(v); }
+            if (afl) afl[slot] += std::fabs(v);
+          };
           double dalpha = 0;
           for (int c = 0; c < 3; ++c) {
             add(c, r.alpha * r.T * Gp[c]);
             dalpha += Gp[c] * (r.T * color[3 * g + c] - S[c] / (1.0 - r.alpha));
           }
-          if (!r.clamped) {
+          const bool near_clamp = std::fabs(opacity[g] * std::exp(r.power) - kAlphaMax) < 1e-4 * kAlphaMax;
+          if (!r.clamped || near_clamp) {
+            if (r.clamped) real = false;   // clamped here, but fp32 may not clamp: flip allowance only
             const double dpower = r.alpha * dalpha;
             const double dx = px - mean2d[2 * g], dy = py - mean2d[2 * g + 1];
             add(3, std::exp(r.power) * dalpha);
@@ -625,7 +665,7 @@ void gso_blend_backward(int64_t n, int W, int H, const double* bg, int64_t P, co
             add(7, dpower * (conic[3 * g] * dx + conic[3 * g + 1] * dy));
             add(8, dpower * (conic[3 * g + 1] * dx + conic[3 * g + 2] * dy));
           }
-          for (int c = 0; c < 3; ++c) S[c] += color[3 * g + c] * r.alpha * r.T;
+          if (!r.ghost) for (int c = 0; c < 3; ++c) S[c] += color[3 * g + c] * r.alpha * r.T;
         }
       }
   }
@@ -633,6 +673,7 @@ void gso_blend_backward(int64_t n, int W, int H, const double* bg, int64_t P, co
     for (int c = 0; c < 3; ++c) { g_color[3 * i + c] = 0; g_conic[3 * i + c] = 0; }
     g_opacity[i] = 0; g_mean2d[2 * i] = g_mean2d[2 * i + 1] = 0;
     if (abs_sum) for (int c = 0; c < 9; ++c) abs_sum[9 * i + c] = 0;
+    if (flip_sum) for (int c = 0; c < 9; ++c) flip_sum[9 * i + c] = 0;
   }
   for (int64_t p = 0; p < P; ++p) {
     const uint32_t g = vals[p];
@@ -642,6 +683,7 @@ void gso_blend_backward(int64_t n, int W, int H, const double* bg, int64_t P, co
     for (int c = 0; c < 3; ++c) g_conic[3 * g + c] += a[4 + c];
     g_mean2d[2 * g] += a[7]; g_mean2d[2 * g + 1] += a[8];
     if (abs_sum) for (int c = 0; c < 9; ++c) abs_sum[9 * g + c] += inst_abs[(size_t)p * 9 + c];
+    if (flip_sum) for (int c = 0; c < 9; ++c) flip_sum[9 * g + c] += inst_flip[(size_t)p * 9 + c];
   }
 }
 

@@ -219,11 +219,13 @@ def blend_backward(cam, vals, ranges, mean2d, conic, opacity, color, G, with_abs
     n = np.asarray(opacity).shape[0]
     vals = np.ascontiguousarray(vals, np.uint32); ranges = np.ascontiguousarray(ranges, np.uint32)
     o = SimpleNamespace(color=np.zeros((n, 3)), opacity=np.zeros(n), conic=np.zeros((n, 3)),
-                        mean2d=np.zeros((n, 2)), abs_sum=np.zeros((n, 9)) if with_abs else None)
+                        mean2d=np.zeros((n, 2)), abs_sum=np.zeros((n, 9)) if with_abs else None,
+                        flip_sum=np.zeros((n, 9)) if with_abs else None)
     lib().gso_blend_backward(C.c_int64(n), C.c_int(W), C.c_int(H), _dp(bg), C.c_int64(vals.shape[0]),
                              _p(vals, C.c_uint32), _p(ranges, C.c_uint32), _dp(_f64(mean2d)),
                              _dp(_f64(conic)), _dp(_f64(opacity)), _dp(_f64(color)), _dp(_f64(G)),
-                             _dp(o.color), _dp(o.opacity), _dp(o.conic), _dp(o.mean2d), _dp(o.abs_sum))
+                             _dp(o.color), _dp(o.opacity), _dp(o.conic), _dp(o.mean2d), _dp(o.abs_sum),
+                             _dp(o.flip_sum))
     return o
 
 

@@ -21,35 +21,39 @@ __device__ __forceinline__ void quad_of(int tile, int gx, int tid, int &px, int 
   py = ty * GS_TILE + warp * 8 + 2 * (lane >> 3);
 }
 
-// Stage one batch entry: (x, y, qa, qb) (qc, o) (r, g, b, -) with the conic pre-scaled so that
-// exp(power) = 2^(qa dx^2 + qb dx dy + qc dy^2).
+// Stage one batch entry: (x, y, la, lb) (lc, o) (r, g, b, -).  (la, lb, lc) is the Cholesky factor
+// of the conic, scaled by sqrt(0.5 log2 e), so that exp(power) = 2^-((la dx + lb dy)^2 + (lc dy)^2):
+// a sum of two squares has no cancellation, which keeps alpha accurate to a few ulp even for
+// footprints hundreds of pixels wide (the expanded quadratic form loses 1e-4 there).
 __device__ __forceinline__ void stage_entry(uint32_t g, const float *mean2d, const float *conic_opacity,
                                             const float *color, float4 &xyab, float2 &co, float4 &rgb) {
   const float2 m = __ldg(reinterpret_cast<const float2 *>(mean2d) + g);
   const float4 q = __ldg(reinterpret_cast<const float4 *>(conic_opacity) + g);
-  xyab = make_float4(m.x, m.y, -0.5f * kLog2e * q.x, -kLog2e * q.y);
-  co = make_float2(-0.5f * kLog2e * q.z, q.w);
+  const float kS = 0.8493218002880191f;   // sqrt(0.5 * log2(e))
+  xyab = make_float4(m.x, m.y, kS * q.x, kS * q.y);   // q = (l11, l21, l22, opacity)
+  co = make_float2(kS * q.z, q.w);
   rgb = make_float4(__ldg(color + 3 * (size_t)g), __ldg(color + 3 * (size_t)g + 1), __ldg(color + 3 * (size_t)g + 2), 0.f);
 }
 
 // log2 of the Gaussian falloff at the four pixels of a quad; dx0, dy0 are the offsets of the
 // top-left pixel centre from the mean.  Index k = 2 * row + column.  One explicit operation order,
 // shared by the forward and the backward so that both take identical skip decisions.
-__device__ __forceinline__ void quad_power(float dx0, float dy0, float qa, float qb, float qc, float p[4]) {
+// t1[k] = la dx + lb dy is returned too: the backward needs it for the gradient of the mean.
+__device__ __forceinline__ void quad_power(float dx0, float dy0, float la, float lb, float lc, float p[4],
+                                           float t1[4], float t2[2]) {
   const float dx1 = __fadd_rn(dx0, 1.f), dy1 = __fadd_rn(dy0, 1.f);
-  const float a0 = __fmul_rn(qa, dx0), a1 = __fmul_rn(qa, dx1);
-  const float b0 = __fmul_rn(qb, dy0), b1 = __fmul_rn(qb, dy1);
-  const float c0 = __fmul_rn(__fmul_rn(qc, dy0), dy0), c1 = __fmul_rn(__fmul_rn(qc, dy1), dy1);
-  p[0] = __fmaf_rn(__fadd_rn(a0, b0), dx0, c0);
-  p[1] = __fmaf_rn(__fadd_rn(a1, b0), dx1, c0);
-  p[2] = __fmaf_rn(__fadd_rn(a0, b1), dx0, c1);
-  p[3] = __fmaf_rn(__fadd_rn(a1, b1), dx1, c1);
+  const float a0 = __fmul_rn(la, dx0), a1 = __fmul_rn(la, dx1);
+  t2[0] = __fmul_rn(lc, dy0); t2[1] = __fmul_rn(lc, dy1);
+  const float s0 = __fmul_rn(t2[0], t2[0]), s1 = __fmul_rn(t2[1], t2[1]);
+  t1[0] = __fmaf_rn(lb, dy0, a0); t1[1] = __fmaf_rn(lb, dy0, a1);
+  t1[2] = __fmaf_rn(lb, dy1, a0); t1[3] = __fmaf_rn(lb, dy1, a1);
+  p[0] = -__fmaf_rn(t1[0], t1[0], s0); p[1] = -__fmaf_rn(t1[1], t1[1], s0);
+  p[2] = -__fmaf_rn(t1[2], t1[2], s1); p[3] = -__fmaf_rn(t1[3], t1[3], s1);
 }
 
 // alpha of one pixel from its log2 falloff; false if the pair is skipped.
 __device__ __forceinline__ bool alpha_of(float p, float o, float &e2, float &alpha) {
-  if (p > 0.f) return false;
-  e2 = ex2_approx(p);
+  e2 = ex2_approx(p);             // p <= 0 by construction
   alpha = fminf(kAlphaMax, __fmul_rn(o, e2));
   return alpha >= kAlphaMin;
 }
@@ -89,8 +93,8 @@ __global__ void __launch_bounds__(kThreads) k_blend_fwd(CamDev cam, const uint32
     for (int j = 0; j < cnt && live; ++j) {
       const float4 a = s_xyab[j];
       const float2 c = s_co[j];
-      float p[4];
-      quad_power(fx - a.x, fy - a.y, a.z, a.w, c.x, p);
+      float p[4], t1[4], t2[2];
+      quad_power(fx - a.x, fy - a.y, a.z, a.w, c.x, p, t1, t2);
       const float4 col = s_rgb[j];
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
@@ -230,8 +234,8 @@ __global__ void __launch_bounds__(kThreads) k_blend_bwd(CamDev cam, const uint32
       const float4 a = s_xyab[j];
       const float2 c = s_co[j];
       const float dx0 = fx - a.x, dy0 = fy - a.y;
-      float p[4];
-      quad_power(dx0, dy0, a.z, a.w, c.x, p);
+      float p[4], t1[4], t2[2];
+      quad_power(dx0, dy0, a.z, a.w, c.x, p, t1, t2);
       const float4 col = s_rgb[j];
       float v[9];
 #pragma unroll
@@ -253,12 +257,12 @@ __global__ void __launch_bounds__(kThreads) k_blend_bwd(CamDev cam, const uint32
         if (c.y * e2 <= kAlphaMax) {              // not clamped: alpha depends on o and power
           v[8] = fmaf(e2, dalpha, v[8]);
           const float dp = alpha * dalpha;
-          const float dp2 = dp * kLn2;            // the staged conic carries a factor log2(e)
+          const float dp2 = dp * (2.f * kLn2);    // power = -ln2 (t1^2 + t2^2), d power / d mean = -d / d (dx, dy)
           v[0] = fmaf(-0.5f * dx * dx, dp, v[0]);
           v[1] = fmaf(-dx * dy, dp, v[1]);
           v[2] = fmaf(-0.5f * dy * dy, dp, v[2]);
-          v[3] = fmaf(-dp2, 2.f * a.z * dx + a.w * dy, v[3]);
-          v[4] = fmaf(-dp2, a.w * dx + 2.f * c.x * dy, v[4]);
+          v[3] = fmaf(dp2, t1[k] * a.z, v[3]);
+          v[4] = fmaf(dp2, fmaf(t1[k], a.w, t2[k >> 1] * c.x), v[4]);
         }
         Sr[k] = fmaf(col.x, w, Sr[k]); Sg[k] = fmaf(col.y, w, Sg[k]); Sb[k] = fmaf(col.z, w, Sb[k]);
         T[k] = Tb;

@@ -333,7 +333,7 @@ __global__ void k_wgrad_reduce(const float *__restrict__ partials, int nblocks, 
 // ---- projection -----------------------------------------------------------------------------
 struct Geo {
   bool valid;
-  float u, v, A, B, C, o, ex, ey;
+  float u, v, A, B, C, o, ex, ey;   // (A, B, C) = (l11, l21, l22), the Cholesky factor of the conic
   uint32_t zbits;
   float dirx, diry, dirz;
 };
@@ -410,7 +410,11 @@ __device__ __forceinline__ Geo project(const float mu[3], const float ls[3], con
   if (!finite_f(u) || !finite_f(v) || !finite_f(ex) || !finite_f(ey)) return g;
   g.valid = true;
   g.zbits = __float_as_uint(z32);
-  g.u = u; g.v = v; g.A = c * idet; g.B = -b * idet; g.C = a * idet; g.o = o; g.ex = ex; g.ey = ey;
+  // Cholesky factor of the conic Q = cov^-1 = L L^T, straight from the covariance entries (no
+  // cancellation even for needle-like splats): l22 = 1/sqrt(c), l11 = sqrt(c/det), l21 = -b/sqrt(c det)
+  const float isd = 1.f / sqrtf(det), l22 = 1.f / sqrtf(c);
+  (void)idet;
+  g.u = u; g.v = v; g.A = sqrtf(c) * isd; g.B = -b * l22 * isd; g.C = l22; g.o = o; g.ex = ex; g.ey = ey;
   const float vx = mu[0] - cam.oc[0], vy = mu[1] - cam.oc[1], vz = mu[2] - cam.oc[2];
   const float vi = rsqrtf(vx * vx + vy * vy + vz * vz);
   g.dirx = vx * vi; g.diry = vy * vi; g.dirz = vz * vi;

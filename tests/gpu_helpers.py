@@ -31,6 +31,13 @@ def image_mismatch(gpu, ref, fragile):
     return d > tol
 
 
+def _conic_from_cholesky(lo):
+    """The library stores the conic as its Cholesky factor (l11, l21, l22) + opacity; rebuild (A, B, C, o)
+    in double, exactly."""
+    lo = lo.astype(np.float64)
+    return np.stack([lo[:, 0] ** 2, lo[:, 0] * lo[:, 1], lo[:, 1] ** 2 + lo[:, 2] ** 2, lo[:, 3]], 1)
+
+
 def run_gpu(scene, cam, G=None, pair_capacity=None, with_extent=True, device=0):
     """One view through gs_preprocess / gs_render_forward / gs_render_backward.  Returns numpy copies."""
     import torch
@@ -51,7 +58,7 @@ def run_gpu(scene, cam, G=None, pair_capacity=None, with_extent=True, device=0):
     torch.cuda.synchronize()
     u32 = lambda t: t.cpu().numpy().view(np.uint32)
     out = SimpleNamespace(
-        P=P, n=n, mean2d=proj.mean2d.cpu().numpy()[:n], conic_opacity=proj.conic_opacity.cpu().numpy()[:n],
+        P=P, n=n, mean2d=proj.mean2d.cpu().numpy()[:n], conic_opacity=_conic_from_cholesky(proj.conic_opacity.cpu().numpy()[:n]),
         color=proj.color.cpu().numpy()[:n], depth_key=u32(proj.depth_key)[:n],
         rect=proj.rect.cpu().numpy().view(np.uint16)[:n].astype(np.int32),
         extent=proj.extent.cpu().numpy()[:n] if with_extent else None,
