@@ -103,6 +103,9 @@ typedef struct {
                                               (depth_key, id) ascending                        */
   uint32_t *tile_ranges;   /* [tiles,2]       [start,end) into the sorted lists, tiles =
                                               ceil(W/16)*ceil(H/16), row-major                 */
+  uint32_t *tile_order;    /* [tiles]         tile ids by decreasing list length: the order in
+                                              which the blend kernels start their tiles (affects
+                                              scheduling only; ties in no particular order)    */
 } GsBinning;
 
 /* Gradients (caller-allocated device buffers, fp32, dense, exact zeros for culled Gaussians). */

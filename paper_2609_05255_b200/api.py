@@ -48,7 +48,8 @@ class GsProjected(C.Structure):
 
 
 class GsBinning(C.Structure):
-    _fields_ = [("depth_order", _vp), ("sorted_tiles", _vp), ("sorted_vals", _vp), ("tile_ranges", _vp)]
+    _fields_ = [("depth_order", _vp), ("sorted_tiles", _vp), ("sorted_vals", _vp), ("tile_ranges", _vp),
+                ("tile_order", _vp)]
 
 
 class GsGrads(C.Structure):
@@ -187,11 +188,13 @@ class Binning:
     sorted_tiles: torch.Tensor
     sorted_vals: torch.Tensor
     tile_ranges: torch.Tensor
+    tile_order: torch.Tensor
 
     def c_struct(self) -> GsBinning:
         b = GsBinning()
         b.depth_order, b.sorted_tiles = _ptr(self.depth_order), _ptr(self.sorted_tiles)
         b.sorted_vals, b.tile_ranges = _ptr(self.sorted_vals), _ptr(self.tile_ranges)
+        b.tile_order = _ptr(self.tile_order)
         return b
 
 
@@ -199,7 +202,8 @@ def alloc_binning(n: int, pair_capacity: int, width: int, height: int, device) -
     tiles = ((width + TILE - 1) // TILE) * ((height + TILE - 1) // TILE)
     i = dict(device=device, dtype=torch.int32)
     return Binning(torch.empty((max(n, 1),), **i), torch.empty((max(pair_capacity, 1),), **i),
-                   torch.empty((max(pair_capacity, 1),), **i), torch.empty((tiles, 2), **i))
+                   torch.empty((max(pair_capacity, 1),), **i), torch.empty((tiles, 2), **i),
+                   torch.empty((tiles,), **i))
 
 
 @dataclass

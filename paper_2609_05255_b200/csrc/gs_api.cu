@@ -246,7 +246,7 @@ GsStatus gs_render_forward(GsContext *ctx, int64_t n, const GsProjected *proj, c
   if (n < 0 || num_pairs < 0 || pair_capacity < 0) return fail(ctx, GS_ERR_INVALID_ARG, "negative size");
   if (!camera_ok(cam)) return fail(ctx, GS_ERR_INVALID_ARG, "bad camera");
   if (!proj || !bin) return fail(ctx, GS_ERR_INVALID_ARG, "proj / bin is NULL");
-  if (bad_ptr(image) || bad_ptr(final_T) || bad_ptr(n_contrib) || bad_ptr(bin->tile_ranges))
+  if (bad_ptr(image) || bad_ptr(final_T) || bad_ptr(n_contrib) || bad_ptr(bin->tile_ranges) || bad_ptr(bin->tile_order))
     return fail(ctx, GS_ERR_INVALID_ARG, "an output buffer is NULL or misaligned");
   if (num_pairs > pair_capacity) return fail(ctx, GS_ERR_CAPACITY, "num_pairs exceeds pair_capacity");
   if (num_pairs >= ((int64_t)1 << 32)) return fail(ctx, GS_ERR_CAPACITY, "more than 2^32 - 1 instances");
@@ -286,11 +286,11 @@ GsStatus gs_render_forward(GsContext *ctx, int64_t n, const GsProjected *proj, c
   }
   {
     StageTimer t(ctx, GS_STAGE_TILE_RANGES, s);
-    t.done(launch_tile_ranges(bin->sorted_tiles, num_pairs, bin->tile_ranges, num_tiles, s));
+    t.done(launch_tile_ranges(bin->sorted_tiles, num_pairs, bin->tile_ranges, bin->tile_order, num_tiles, s));
   }
   {
     StageTimer t(ctx, GS_STAGE_BLEND_FWD, s);
-    t.done(launch_blend_fwd(cd, bin->tile_ranges, bin->sorted_vals, proj->mean2d, proj->conic_opacity, proj->color,
+    t.done(launch_blend_fwd(cd, bin->tile_ranges, bin->tile_order, bin->sorted_vals, proj->mean2d, proj->conic_opacity, proj->color,
                             image, final_T, n_contrib, s));
   }
   return check_cuda(ctx, cudaGetLastError(), "render_forward launch");
@@ -305,7 +305,7 @@ GsStatus gs_render_backward(GsContext *ctx, const GsScene *scene, const GsCamera
   if (st != GS_OK) return st;
   if (!camera_ok(cam)) return fail(ctx, GS_ERR_INVALID_ARG, "bad camera");
   if (!proj || !bin || !grads) return fail(ctx, GS_ERR_INVALID_ARG, "proj / bin / grads is NULL");
-  if (bad_ptr(final_T) || bad_ptr(n_contrib) || bad_ptr(dL_dimage) || bad_ptr(bin->tile_ranges))
+  if (bad_ptr(final_T) || bad_ptr(n_contrib) || bad_ptr(dL_dimage) || bad_ptr(bin->tile_ranges) || bad_ptr(bin->tile_order))
     return fail(ctx, GS_ERR_INVALID_ARG, "an image-sized buffer is NULL or misaligned");
   const int64_t n = scene->n;
   if (scene->app == GS_APP_NEURAL && bad_ptr(grads->mlp_weights))
@@ -330,7 +330,7 @@ GsStatus gs_render_backward(GsContext *ctx, const GsScene *scene, const GsCamera
     if ((st = check_cuda(ctx, cudaMemsetAsync(g2d, 0, (size_t)n * 12 * sizeof(float), s), "memset")) != GS_OK) return st;
     if (num_pairs > 0) {
       StageTimer t(ctx, GS_STAGE_BLEND_BWD, s);
-      t.done(launch_blend_bwd(cd, bin->tile_ranges, bin->sorted_vals, proj->mean2d, proj->conic_opacity, proj->color,
+      t.done(launch_blend_bwd(cd, bin->tile_ranges, bin->tile_order, bin->sorted_vals, proj->mean2d, proj->conic_opacity, proj->color,
                               final_T, n_contrib, dL_dimage, g2d, s));
     }
   }

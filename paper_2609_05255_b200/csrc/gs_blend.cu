@@ -59,6 +59,7 @@ __device__ __forceinline__ bool alpha_of(float p, float o, float &e2, float &alp
 }
 
 __global__ void __launch_bounds__(kThreads) k_blend_fwd(CamDev cam, const uint32_t *__restrict__ ranges,
+                                                        const uint32_t *__restrict__ order,
                                                         const uint32_t *__restrict__ vals,
                                                         const float *__restrict__ mean2d,
                                                         const float *__restrict__ conic_opacity,
@@ -67,7 +68,7 @@ __global__ void __launch_bounds__(kThreads) k_blend_fwd(CamDev cam, const uint32
   __shared__ float4 s_xyab[kBatch];
   __shared__ float2 s_co[kBatch];
   __shared__ float4 s_rgb[kBatch];
-  const int tid = threadIdx.x, tile = blockIdx.x;
+  const int tid = threadIdx.x, tile = (int)__ldg(order + blockIdx.x);
   int px, py;
   quad_of(tile, cam.gx, tid, px, py);
   const float fx = (float)px + 0.5f, fy = (float)py + 0.5f;
@@ -167,6 +168,7 @@ __device__ __forceinline__ void warp_reduce9(const float v[9], int lane, float &
 // the kernel the values travel as v[0..7] = (conic A, B, C, mean u, mean v, colour r, g, b) and
 // v[8] = opacity.
 __global__ void __launch_bounds__(kThreads) k_blend_bwd(CamDev cam, const uint32_t *__restrict__ ranges,
+                                                        const uint32_t *__restrict__ order,
                                                         const uint32_t *__restrict__ vals,
                                                         const float *__restrict__ mean2d,
                                                         const float *__restrict__ conic_opacity,
@@ -180,7 +182,7 @@ __global__ void __launch_bounds__(kThreads) k_blend_bwd(CamDev cam, const uint32
   __shared__ uint32_t s_gid[kBatch];
   __shared__ float s_acc[kBatch][9];
   __shared__ uint32_t s_max[2];
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, tile = blockIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, tile = (int)__ldg(order + blockIdx.x);
   int px, py;
   quad_of(tile, cam.gx, tid, px, py);
   const float fx = (float)px + 0.5f, fy = (float)py + 0.5f;
@@ -294,18 +296,20 @@ __global__ void __launch_bounds__(kThreads) k_blend_bwd(CamDev cam, const uint32
 
 }  // namespace
 
-int launch_blend_fwd(const CamDev &cam, const uint32_t *ranges, const uint32_t *vals, const float *mean2d,
+int launch_blend_fwd(const CamDev &cam, const uint32_t *ranges, const uint32_t *order, const uint32_t *vals,
+                     const float *mean2d,
                      const float *conic_opacity, const float *color, float *image, float *final_T,
                      uint32_t *n_contrib, cudaStream_t st) {
-  k_blend_fwd<<<cam.gx * cam.gy, kThreads, 0, st>>>(cam, ranges, vals, mean2d, conic_opacity, color, image,
+  k_blend_fwd<<<cam.gx * cam.gy, kThreads, 0, st>>>(cam, ranges, order, vals, mean2d, conic_opacity, color, image,
                                                     final_T, n_contrib);
   return 1;
 }
 
-int launch_blend_bwd(const CamDev &cam, const uint32_t *ranges, const uint32_t *vals, const float *mean2d,
+int launch_blend_bwd(const CamDev &cam, const uint32_t *ranges, const uint32_t *order, const uint32_t *vals,
+                     const float *mean2d,
                      const float *conic_opacity, const float *color, const float *final_T,
                      const uint32_t *n_contrib, const float *dL_dimage, float *g2d, cudaStream_t st) {
-  k_blend_bwd<<<cam.gx * cam.gy, kThreads, 0, st>>>(cam, ranges, vals, mean2d, conic_opacity, color, final_T,
+  k_blend_bwd<<<cam.gx * cam.gy, kThreads, 0, st>>>(cam, ranges, order, vals, mean2d, conic_opacity, color, final_T,
                                                     n_contrib, dL_dimage, g2d);
   return 1;
 }

@@ -82,14 +82,14 @@ int launch_tile_offsets(const uint32_t *depth_order, const uint16_t *rect, uint3
                          int64_t n, void *scratch, cudaStream_t st);
 int launch_keygen(const uint32_t *depth_order, const uint16_t *rect, const uint32_t *offsets,
                    uint32_t *inst_tiles, uint32_t *inst_vals, int64_t n, int gx, cudaStream_t st);
-int launch_tile_ranges(const uint32_t *sorted_tiles, int64_t P, uint32_t *ranges, int num_tiles,
-                        cudaStream_t st);
+int launch_tile_ranges(const uint32_t *sorted_tiles, int64_t P, uint32_t *ranges, uint32_t *order,
+                       int num_tiles, cudaStream_t st);
 
 // Blend.
-int launch_blend_fwd(const CamDev &cam, const uint32_t *ranges, const uint32_t *vals,
+int launch_blend_fwd(const CamDev &cam, const uint32_t *ranges, const uint32_t *order, const uint32_t *vals,
                       const float *mean2d, const float *conic_opacity, const float *color,
                       float *image, float *final_T, uint32_t *n_contrib, cudaStream_t st);
-int launch_blend_bwd(const CamDev &cam, const uint32_t *ranges, const uint32_t *vals,
+int launch_blend_bwd(const CamDev &cam, const uint32_t *ranges, const uint32_t *order, const uint32_t *vals,
                       const float *mean2d, const float *conic_opacity, const float *color,
                       const float *final_T, const uint32_t *n_contrib, const float *dL_dimage,
                       float *g2d, cudaStream_t st);

@@ -7,6 +7,7 @@
 #include <string.h>
 
 #include "gs_device.cuh"
+#include "gs_mlp_mma.cuh"
 
 namespace gs {
 namespace {
@@ -86,10 +87,6 @@ __device__ __forceinline__ void sh_backward(float *row, const float gp[3], float
 }
 
 // ---- appearance: neural ---------------------------------------------------------------------
-__device__ __forceinline__ void load_weights_f32(const __half *w, float *sW, int tid, int nthreads) {
-  for (int k = tid; k < GS_MLP_WEIGHTS; k += nthreads) sW[k] = __half2float(w[k]);
-}
-
 __device__ __forceinline__ void load_features(const __half *features, int64_t i, float f[8]) {
   const uint4 raw = __ldg(reinterpret_cast<const uint4 *>(features) + i);
   const __half2 *h = reinterpret_cast<const __half2 *>(&raw);
@@ -100,135 +97,64 @@ __device__ __forceinline__ void load_features(const __half *features, int64_t i,
   }
 }
 
-// y = W x for a row-major [OUT][IN] matrix in shared memory (broadcast 128-bit reads).
-template <int OUT, int IN>
-__device__ __forceinline__ void matvec(const float *W, const float *x, float *y) {
-#pragma unroll
-  for (int o = 0; o < OUT; ++o) {
-    float acc = 0.f;
-#pragma unroll
-    for (int i = 0; i < IN; i += 4) {
-      const float4 w = *reinterpret_cast<const float4 *>(W + o * IN + i);
-      acc = fmaf(w.x, x[i], acc); acc = fmaf(w.y, x[i + 1], acc);
-      acc = fmaf(w.z, x[i + 2], acc); acc = fmaf(w.w, x[i + 3], acc);
-    }
-    y[o] = acc;
-  }
-}
-
-// g_x = W^T g_y
-template <int OUT, int IN>
-__device__ __forceinline__ void matvec_t(const float *W, const float *gy, float *gx) {
-#pragma unroll
-  for (int i = 0; i < IN; ++i) gx[i] = 0.f;
-#pragma unroll
-  for (int o = 0; o < OUT; ++o) {
-#pragma unroll
-    for (int i = 0; i < IN; i += 4) {
-      const float4 w = *reinterpret_cast<const float4 *>(W + o * IN + i);
-      gx[i] = fmaf(w.x, gy[o], gx[i]); gx[i + 1] = fmaf(w.y, gy[o], gx[i + 1]);
-      gx[i + 2] = fmaf(w.z, gy[o], gx[i + 2]); gx[i + 3] = fmaf(w.w, gy[o], gx[i + 3]);
-    }
-  }
-}
-
-// Eq. 5-7.  x = (Y_0..15(d) masked by the active degree, sin f_j, cos f_j interleaved).
-__device__ __forceinline__ void mlp_forward(const float *sW, float dx, float dy, float dz,
-                                            const float f[8], int deg, float x[32], float h1[16],
-                                            float h2[16], float A[3]) {
+// Decoder inputs of one Gaussian (Eq. 5, Eq. 6 with k = 1): SH basis of the direction masked by the
+// active degree, then (sin f_j, cos f_j).  The fast sincos is used inside [-pi, pi] (absolute error
+// below 4e-7 there), the accurate one outside.
+__device__ __forceinline__ void decoder_inputs(float dx, float dy, float dz, const float f[8], int deg, float x[32]) {
   sh_basis(dx, dy, dz, x);
   const int na = (deg + 1) * (deg + 1);
 #pragma unroll
   for (int k = 0; k < 16; ++k) x[k] = k < na ? x[k] : 0.f;
 #pragma unroll
-  for (int j = 0; j < 8; ++j) sincosf(f[j], &x[16 + 2 * j], &x[17 + 2 * j]);
-  matvec<16, 32>(sW + kMlpW1, x, h1);
-#pragma unroll
-  for (int k = 0; k < 16; ++k) h1[k] = fmaxf(h1[k], 0.f);
-  matvec<16, 16>(sW + kMlpW2, h1, h2);
-#pragma unroll
-  for (int k = 0; k < 16; ++k) h2[k] = fmaxf(h2[k], 0.f);
-  float y[3];
-  matvec<3, 16>(sW + kMlpW3, h2, y);
-#pragma unroll
-  for (int c = 0; c < 3; ++c) A[c] = tanhf(y[c]);
-}
-
-// Per-warp slab of the decoder-gradient kernels: for each of the warp's 32 Gaussians the
-// operands of the three outer products, 100 floats per Gaussian:
-// x[32] | h1[16] | h2[16] | g_h1[16] | g_h2[16] | g_y[3] + pad.
-constexpr int kActRow = 100;
-constexpr int kOffX = 0, kOffH1 = 32, kOffH2 = 48, kOffG1 = 64, kOffG2 = 80, kOffGY = 96;
-
-__device__ __forceinline__ void store4(float *dst, const float *v) {
-  *reinterpret_cast<float4 *>(dst) = make_float4(v[0], v[1], v[2], v[3]);
-}
-
-// Compiler-only fence.  The decoder weights sit in shared memory and are re-read by every stage;
-// without it the compiler keeps hundreds of them live in registers (hoisted out of the
-// persistent loop or carried from the forward into the backward) and spills.
-__device__ __forceinline__ void reload_fence() { asm volatile("" ::: "memory"); }
-
-__device__ __forceinline__ void load4(const float *src, float *v) {
-  const float4 t = *reinterpret_cast<const float4 *>(src);
-  v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
-}
-
-// Backward through the decoder for one Gaussian (forward recomputed).  gcol = dL/dcolour; gp
-// returns dL/d(pre-activation of the colour) = gcol masked by the ReLU.  Writes this Gaussian's
-// operand row into the warp slab, returns dL/df and dL/dd.  Activations are parked in the slab row
-// as soon as they exist and read back when needed, which keeps the live registers under the limit.
-__device__ __forceinline__ void mlp_backward(const float *sW, float *act_row, float dx, float dy,
-                                             float dz, const float f[8], int deg, const float base[3],
-                                             const float gcol[3], float gp[3], float gf[8], float gd[3]) {
-  float gy[4];
-  {
-    float x[32], h1[16], h2[16], A[3];
-    mlp_forward(sW, dx, dy, dz, f, deg, x, h1, h2, A);
-#pragma unroll
-    for (int k = 0; k < 32; k += 4) store4(act_row + kOffX + k, x + k);
-#pragma unroll
-    for (int k = 0; k < 16; k += 4) { store4(act_row + kOffH1 + k, h1 + k); store4(act_row + kOffH2 + k, h2 + k); }
-#pragma unroll
-    for (int c = 0; c < 3; ++c) {
-      gp[c] = (base[c] + 0.5f + A[c]) > 0.f ? gcol[c] : 0.f;
-      gy[c] = gp[c] * (1.f - A[c] * A[c]);
-    }
-    gy[3] = 0.f;
-    store4(act_row + kOffGY, gy);
+  for (int j = 0; j < 8; ++j) {
+    if (fabsf(f[j]) <= 3.14159265f) __sincosf(f[j], &x[16 + 2 * j], &x[17 + 2 * j]);
+    else sincosf(f[j], &x[16 + 2 * j], &x[17 + 2 * j]);
   }
-  reload_fence();
-  float g1[16];
-  {
-    float g2[16], h[4];
-    matvec_t<3, 16>(sW + kMlpW3, gy, g2);
+}
+
+// Forward-only staging of the tensor-core decoder: the leading members of mlp::WarpStage.
+struct __align__(16) StageFwd {
+  uint32_t xhi[32 * mlp::kXStride];
+  uint32_t xlo[32 * mlp::kXStride];
+  float y[32 * 4];
+};
+
+// Whole-warp decode: every lane passes its Gaussian's inputs (zeros if it has none) and gets the
+// tanh-bounded residual A back.  All 32 lanes must call it.
+template <class Stage>
+__device__ __forceinline__ void decode_warp(const mlp::Weights &W, Stage &S, int lane, const float x[32],
+                                            mlp::Activations &act, float A[3]) {
+  mlp::stage_inputs(x, S, lane);
+  mlp::forward_warp(W, S, lane, act);
 #pragma unroll
-    for (int k = 0; k < 16; k += 4) {
-      load4(act_row + kOffH2 + k, h);
+  for (int c = 0; c < 3; ++c) A[c] = tanhf(S.y[lane * 4 + c]);
+}
+
+// Whole-warp backward of the decoder.  `has`: this lane owns a Gaussian (inputs x, direction d, base
+// colour, dL/dcolour gcol); lanes without one pass zeros.  Returns the ReLU-masked colour gradient
+// gp, dL/df and dL/dd of the lane's Gaussian and advances the warp's weight-gradient fragments.
+__device__ __forceinline__ void decode_backward_warp(const mlp::Weights &W, mlp::WarpStage &S, int lane, bool has,
+                                                     const float x[32], float dx, float dy, float dz, int deg,
+                                                     const float base[3], const float gcol[3], mlp::WeightGrad &dW,
+                                                     float gp[3], float gf[8], float gd[3]) {
+  mlp::Activations act;
+  float A[3];
+  decode_warp(W, S, lane, x, act, A);
+  float gy[3];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) g2[k + j] = h[j] > 0.f ? g2[k + j] : 0.f;
-      store4(act_row + kOffG2 + k, g2 + k);
-    }
-    reload_fence();
-    matvec_t<16, 16>(sW + kMlpW2, g2, g1);
-#pragma unroll
-    for (int k = 0; k < 16; k += 4) {
-      load4(act_row + kOffH1 + k, h);
-#pragma unroll
-      for (int j = 0; j < 4; ++j) g1[k + j] = h[j] > 0.f ? g1[k + j] : 0.f;
-      store4(act_row + kOffG1 + k, g1 + k);
-    }
+  for (int c = 0; c < 3; ++c) {
+    gp[c] = (has && (base[c] + 0.5f + A[c]) > 0.f) ? gcol[c] : 0.f;
+    gy[c] = gp[c] * (1.f - A[c] * A[c]);
   }
-  reload_fence();
-  float gx[32];
-  matvec_t<16, 32>(sW + kMlpW1, g1, gx);
-  reload_fence();
+  *reinterpret_cast<float4 *>(S.y + lane * 4) = make_float4(gy[0], gy[1], gy[2], 0.f);
+  mlp::backward_warp(W, S, lane, act, dW);
+  const float4 f0 = *reinterpret_cast<const float4 *>(S.gf + lane * 8), f1 = *reinterpret_cast<const float4 *>(S.gf + lane * 8 + 4);
+  gf[0] = f0.x; gf[1] = f0.y; gf[2] = f0.z; gf[3] = f0.w; gf[4] = f1.x; gf[5] = f1.y; gf[6] = f1.z; gf[7] = f1.w;
+  float gx[16];
 #pragma unroll
-  for (int j = 0; j < 8; j += 2) {   // x[16 + 2j] = sin f_j, x[17 + 2j] = cos f_j
-    float sc[4];
-    load4(act_row + kOffX + 16 + 2 * j, sc);
-    gf[j] = gx[16 + 2 * j] * sc[1] - gx[17 + 2 * j] * sc[0];
-    gf[j + 1] = gx[18 + 2 * j] * sc[3] - gx[19 + 2 * j] * sc[2];
+  for (int q = 0; q < 4; ++q) {
+    const float4 v = *reinterpret_cast<const float4 *>(S.gx + lane * mlp::kGxStride + 4 * q);
+    gx[4 * q] = v.x; gx[4 * q + 1] = v.y; gx[4 * q + 2] = v.z; gx[4 * q + 3] = v.w;
   }
   const int na = (deg + 1) * (deg + 1);
   float ax = 0.f, ay = 0.f, az = 0.f;
@@ -236,82 +162,14 @@ __device__ __forceinline__ void mlp_backward(const float *sW, float *act_row, fl
   for (int k = 1; k < 16; ++k)
     if (k < na) sh_grad_acc(k, dx, dy, dz, gx[k], ax, ay, az);
   gd[0] = ax; gd[1] = ay; gd[2] = az;
-}
-
-__device__ __forceinline__ void zero_act_row(float *act_row) {
-  const float z[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-  for (int k = 0; k < kActRow; k += 4) store4(act_row + k, z);
-}
-
-// Register tiles of the weight gradient held by one lane: dW1 4x4 at (o = 4*(lane/8),
-// i = 4*(lane%8)), dW2 2x4 at (o = 2*(lane/4), i = 4*(lane%4)), dW3 1x4 at (o = lane/4,
-// i = 4*(lane%4)) for lanes < 12.
-struct WgradAcc {
-  float w1[16], w2[8], w3[4];
-  __device__ __forceinline__ void clear() {
-#pragma unroll
-    for (int k = 0; k < 16; ++k) w1[k] = 0.f;
-#pragma unroll
-    for (int k = 0; k < 8; ++k) w2[k] = 0.f;
-#pragma unroll
-    for (int k = 0; k < 4; ++k) w3[k] = 0.f;
-  }
-};
-
-// Accumulate the outer products of the warp's 32 operand rows.
-__device__ __forceinline__ void wgrad_accumulate(const float *slab, int lane, WgradAcc &acc) {
-  __syncwarp();
-  const int o1 = 4 * (lane >> 3), i1 = 4 * (lane & 7);
-  const int o2 = 2 * (lane >> 2), i2 = 4 * (lane & 3);
-  const int o3 = lane >> 2;
-  for (int g = 0; g < 32; ++g) {
-    const float *row = slab + g * kActRow;
-    const float4 a = *reinterpret_cast<const float4 *>(row + kOffG1 + o1);
-    const float4 b = *reinterpret_cast<const float4 *>(row + kOffX + i1);
-    const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
-#pragma unroll
-    for (int r = 0; r < 4; ++r)
-#pragma unroll
-      for (int c = 0; c < 4; ++c) acc.w1[4 * r + c] = fmaf(av[r], bv[c], acc.w1[4 * r + c]);
-    const float2 a2 = *reinterpret_cast<const float2 *>(row + kOffG2 + o2);
-    const float4 b2 = *reinterpret_cast<const float4 *>(row + kOffH1 + i2);
-    const float b2v[4] = {b2.x, b2.y, b2.z, b2.w};
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      acc.w2[c] = fmaf(a2.x, b2v[c], acc.w2[c]);
-      acc.w2[4 + c] = fmaf(a2.y, b2v[c], acc.w2[4 + c]);
-    }
-    if (lane < 12) {
-      const float a3 = row[kOffGY + o3];
-      const float4 b3 = *reinterpret_cast<const float4 *>(row + kOffH2 + i2);
-      acc.w3[0] = fmaf(a3, b3.x, acc.w3[0]); acc.w3[1] = fmaf(a3, b3.y, acc.w3[1]);
-      acc.w3[2] = fmaf(a3, b3.z, acc.w3[2]); acc.w3[3] = fmaf(a3, b3.w, acc.w3[3]);
-    }
-  }
   __syncwarp();
 }
 
-// Sum the warps' register tiles and write this block's partial [816].
-__device__ __forceinline__ void wgrad_flush(const WgradAcc &acc, float *sPart /*[kWarps][816]*/,
-                                            float *partial_out, int tid) {
-  const int lane = tid & 31, warp = tid >> 5;
-  float *mine = sPart + warp * GS_MLP_WEIGHTS;
-  const int o1 = 4 * (lane >> 3), i1 = 4 * (lane & 7);
-  const int o2 = 2 * (lane >> 2), i2 = 4 * (lane & 3);
-  const int o3 = lane >> 2;
-#pragma unroll
-  for (int r = 0; r < 4; ++r)
-#pragma unroll
-    for (int c = 0; c < 4; ++c) mine[kMlpW1 + (o1 + r) * 32 + i1 + c] = acc.w1[4 * r + c];
-#pragma unroll
-  for (int r = 0; r < 2; ++r)
-#pragma unroll
-    for (int c = 0; c < 4; ++c) mine[kMlpW2 + (o2 + r) * 16 + i2 + c] = acc.w2[4 * r + c];
-  if (lane < 12) {
-#pragma unroll
-    for (int c = 0; c < 4; ++c) mine[kMlpW3 + o3 * 16 + i2 + c] = acc.w3[c];
-  }
+// Sum the warps' weight-gradient fragments and write this block's partial [816].  sPart
+// ([kWarps][816] floats) may alias the warps' staging areas.
+__device__ __forceinline__ void weight_grad_flush(const mlp::WeightGrad &dW, float *sPart, float *partial_out, int tid) {
+  __syncthreads();
+  mlp::store_weight_grad(dW, sPart + (tid >> 5) * GS_MLP_WEIGHTS, tid & 31);
   __syncthreads();
   for (int k = tid; k < GS_MLP_WEIGHTS; k += kBlock) {
     float s = 0.f;
@@ -320,6 +178,10 @@ __device__ __forceinline__ void wgrad_flush(const WgradAcc &acc, float *sPart /*
     partial_out[k] = s;
   }
 }
+
+// Compiler-only fence at the top of the persistent loops: keeps loads of loop-invariant shared
+// memory from being hoisted out of the loop into hundreds of live registers.
+__device__ __forceinline__ void reload_fence() { asm volatile("" ::: "memory"); }
 
 // Deterministic final reduction of the per-block partials.
 __global__ void k_wgrad_reduce(const float *__restrict__ partials, int nblocks, float *__restrict__ out) {
@@ -441,11 +303,14 @@ __device__ __forceinline__ void load3(const float *p, int64_t i, float v[3]) {
 
 template <int APP>
 __global__ void __launch_bounds__(kBlock) k_preprocess_fwd(PreprocessArgs a, CamDev cam) {
-  __shared__ __align__(16) float sData[APP == GS_APP_SH ? kWarps * kSlab : GS_MLP_WEIGHTS];
+  __shared__ __align__(16) float sData[APP == GS_APP_SH ? kWarps * kSlab : 4];
+  __shared__ __align__(16) unsigned char sNN[APP == GS_APP_NEURAL ? sizeof(mlp::Weights) + kWarps * sizeof(StageFwd) : 16];
+  mlp::Weights *sWt = reinterpret_cast<mlp::Weights *>(sNN);
+  StageFwd *sStage = reinterpret_cast<StageFwd *>(sNN + sizeof(mlp::Weights));
   __shared__ unsigned int sPairs[kWarps];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (APP == GS_APP_NEURAL) {
-    load_weights_f32(a.weights, sData, tid, kBlock);
+    mlp::load_weights(a.weights, sWt[0], tid, kBlock);
     __syncthreads();
   }
   const int64_t i = (int64_t)blockIdx.x * kBlock + tid;
@@ -475,15 +340,23 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_fwd(PreprocessArgs a, Cam
       sh_decode(slab + lane * kRow, base, g.dirx, g.diry, g.dirz, a.deg, pre);
     }
   } else {
+    float A[3] = {0.f, 0.f, 0.f};
+    if (a.deg > 0 && __any_sync(kFull, vis)) {   // the whole warp decodes; culled lanes feed zeros
+      float x[32];
+      if (vis) {
+        float f[8];
+        load_features(a.features, i, f);
+        decoder_inputs(g.dirx, g.diry, g.dirz, f, a.deg, x);
+      } else {
+#pragma unroll
+        for (int k = 0; k < 32; ++k) x[k] = 0.f;
+      }
+      mlp::Activations act;
+      decode_warp(sWt[0], sStage[warp], lane, x, act, A);
+    }
     if (vis) {
       float base[3];
       load3(a.base_color, i, base);
-      float A[3] = {0.f, 0.f, 0.f};
-      if (a.deg > 0) {
-        float f[8], x[32], h1[16], h2[16];
-        load_features(a.features, i, f);
-        mlp_forward(sData, g.dirx, g.diry, g.dirz, f, a.deg, x, h1, h2, A);
-      }
 #pragma unroll
       for (int c = 0; c < 3; ++c) pre[c] = base[c] + 0.5f + A[c];
     }
@@ -626,19 +499,21 @@ __device__ __forceinline__ void store3(float *p, int64_t i, float a, float b, fl
 // Shared memory of the backward kernels (dynamic): SH: kWarps slabs of coefficient rows.
 // Neural: weights [816] | kWarps operand slabs [32][100] (reused as [kWarps][816] at the end).
 constexpr size_t kBwdSmemSH = sizeof(float) * kWarps * kSlab;
-constexpr size_t kBwdSmemNN = sizeof(float) * (GS_MLP_WEIGHTS + kWarps * 32 * kActRow);
-static_assert(kWarps * 32 * kActRow >= kWarps * GS_MLP_WEIGHTS, "partial sums reuse the operand slabs");
+constexpr size_t kBwdSmemNN = sizeof(mlp::Weights) + kWarps * sizeof(mlp::WarpStage);
+static_assert(kWarps * sizeof(mlp::WarpStage) >= kWarps * GS_MLP_WEIGHTS * sizeof(float), "partial sums reuse the staging areas");
+static_assert(sizeof(mlp::Weights) % 16 == 0, "staging areas must stay 16-byte aligned");
 
 template <int APP>
 __global__ void __launch_bounds__(kBlock) k_preprocess_bwd(PreprocessBwdArgs a, CamDev cam) {
   extern __shared__ __align__(16) float smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  float *sW = smem;
-  float *slab = APP == GS_APP_SH ? smem + warp * kSlab : smem + GS_MLP_WEIGHTS + warp * 32 * kActRow;
-  WgradAcc acc;
+  float *slab = smem + warp * kSlab;   // SH: this warp's slab of coefficient rows
+  mlp::Weights &sWt = *reinterpret_cast<mlp::Weights *>(smem);
+  mlp::WarpStage *sStage = reinterpret_cast<mlp::WarpStage *>(reinterpret_cast<unsigned char *>(smem) + sizeof(mlp::Weights));
+  mlp::WeightGrad dW;
   if (APP == GS_APP_NEURAL) {
-    load_weights_f32(a.weights, sW, tid, kBlock);
-    acc.clear();
+    mlp::load_weights(a.weights, sWt, tid, kBlock);
+    dW.clear();
     __syncthreads();
   }
   const int64_t nchunks = (a.n + kBlock - 1) / kBlock;
@@ -692,25 +567,23 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_bwd(PreprocessBwdArgs a, 
       }
     } else {
       float gf[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-      float *act_row = slab + lane * kActRow;
-      bool used = false;
-      if (vis) {
-        float base[3];
-        load3(a.base_color, i, base);
-        if (a.deg > 0) {
+      float base[3] = {0.f, 0.f, 0.f};
+      const float gcol[3] = {ga.x, ga.y, ga.z};
+      if (vis) load3(a.base_color, i, base);
+      if (warp_vis && a.deg > 0) {   // the whole warp goes through the decoder; culled lanes feed zeros
+        float x[32];
+        if (vis) {
           float f[8];
-          const float gcol[3] = {ga.x, ga.y, ga.z};
           load_features(a.features, i, f);
-          mlp_backward(sW, act_row, dx, dy, dz, f, a.deg, base, gcol, gp, gf, gd);
-          used = true;
+          decoder_inputs(dx, dy, dz, f, a.deg, x);
         } else {
 #pragma unroll
-          for (int c = 0; c < 3; ++c) gp[c] = (base[c] + 0.5f) > 0.f ? (c == 0 ? ga.x : c == 1 ? ga.y : ga.z) : 0.f;
+          for (int k = 0; k < 32; ++k) x[k] = 0.f;
         }
-      }
-      if (warp_vis && a.deg > 0) {
-        if (!used) zero_act_row(act_row);
-        wgrad_accumulate(slab, lane, acc);
+        decode_backward_warp(sWt, sStage[warp], lane, vis, x, dx, dy, dz, a.deg, base, gcol, dW, gp, gf, gd);
+      } else if (vis) {
+#pragma unroll
+        for (int c = 0; c < 3; ++c) gp[c] = (base[c] + 0.5f) > 0.f ? gcol[c] : 0.f;
       }
       if (in) {
         float4 *gfp = reinterpret_cast<float4 *>(a.g_features) + 2 * i;
@@ -738,18 +611,20 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_bwd(PreprocessBwdArgs a, 
     }
   }
   if (APP == GS_APP_NEURAL) {
-    __syncthreads();
-    wgrad_flush(acc, smem + GS_MLP_WEIGHTS, a.w_partials + (size_t)blockIdx.x * GS_MLP_WEIGHTS, tid);
+    weight_grad_flush(dW, reinterpret_cast<float *>(sStage), a.w_partials + (size_t)blockIdx.x * GS_MLP_WEIGHTS, tid);
   }
 }
 
 // ---- separate-pass appearance kernels ---------------------------------------------------------
 template <int APP>
 __global__ void __launch_bounds__(kBlock) k_appearance_fwd(AppearanceArgs a) {
-  __shared__ __align__(16) float sData[APP == GS_APP_SH ? kWarps * kSlab : GS_MLP_WEIGHTS];
+  __shared__ __align__(16) float sData[APP == GS_APP_SH ? kWarps * kSlab : 4];
+  __shared__ __align__(16) unsigned char sNN[APP == GS_APP_NEURAL ? sizeof(mlp::Weights) + kWarps * sizeof(StageFwd) : 16];
+  mlp::Weights *sWt = reinterpret_cast<mlp::Weights *>(sNN);
+  StageFwd *sStage = reinterpret_cast<StageFwd *>(sNN + sizeof(mlp::Weights));
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (APP == GS_APP_NEURAL) {
-    load_weights_f32(a.weights, sData, tid, kBlock);
+    mlp::load_weights(a.weights, sWt[0], tid, kBlock);
     __syncthreads();
   }
   const int64_t i = (int64_t)blockIdx.x * kBlock + tid;
@@ -763,10 +638,18 @@ __global__ void __launch_bounds__(kBlock) k_appearance_fwd(AppearanceArgs a) {
     if (in) sh_decode(slab + lane * kRow, base, d[0], d[1], d[2], a.deg, pre);
   } else {
     float A[3] = {0.f, 0.f, 0.f};
-    if (in && a.deg > 0) {
-      float f[8], x[32], h1[16], h2[16];
-      load_features(a.features, i, f);
-      mlp_forward(sData, d[0], d[1], d[2], f, a.deg, x, h1, h2, A);
+    if (a.deg > 0 && row0 < a.n) {
+      float x[32];
+      if (in) {
+        float f[8];
+        load_features(a.features, i, f);
+        decoder_inputs(d[0], d[1], d[2], f, a.deg, x);
+      } else {
+#pragma unroll
+        for (int k = 0; k < 32; ++k) x[k] = 0.f;
+      }
+      mlp::Activations act;
+      decode_warp(sWt[0], sStage[warp], lane, x, act, A);
     }
 #pragma unroll
     for (int c = 0; c < 3; ++c) pre[c] = base[c] + 0.5f + A[c];
@@ -778,12 +661,13 @@ template <int APP>
 __global__ void __launch_bounds__(kBlock) k_appearance_bwd(AppearanceArgs a) {
   extern __shared__ __align__(16) float smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  float *sW = smem;
-  float *slab = APP == GS_APP_SH ? smem + warp * kSlab : smem + GS_MLP_WEIGHTS + warp * 32 * kActRow;
-  WgradAcc acc;
+  float *slab = smem + warp * kSlab;   // SH: this warp's slab of coefficient rows
+  mlp::Weights &sWt = *reinterpret_cast<mlp::Weights *>(smem);
+  mlp::WarpStage *sStage = reinterpret_cast<mlp::WarpStage *>(reinterpret_cast<unsigned char *>(smem) + sizeof(mlp::Weights));
+  mlp::WeightGrad dW;
   if (APP == GS_APP_NEURAL) {
-    load_weights_f32(a.weights, sW, tid, kBlock);
-    acc.clear();
+    mlp::load_weights(a.weights, sWt, tid, kBlock);
+    dW.clear();
     __syncthreads();
   }
   const int64_t nchunks = (a.n + kBlock - 1) / kBlock;
@@ -811,17 +695,21 @@ __global__ void __launch_bounds__(kBlock) k_appearance_bwd(AppearanceArgs a) {
       }
     } else {
       float gf[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-      float *act_row = slab + lane * kActRow;
-      if (in && a.deg > 0) {
-        float f[8];
-        load_features(a.features, i, f);
-        mlp_backward(sW, act_row, d[0], d[1], d[2], f, a.deg, base, gcol, gp, gf, gd);
-      } else {
-        zero_act_row(act_row);
+      if (a.deg > 0 && row0 < a.n) {
+        float x[32];
+        if (in) {
+          float f[8];
+          load_features(a.features, i, f);
+          decoder_inputs(d[0], d[1], d[2], f, a.deg, x);
+        } else {
+#pragma unroll
+          for (int k = 0; k < 32; ++k) x[k] = 0.f;
+        }
+        decode_backward_warp(sWt, sStage[warp], lane, in, x, d[0], d[1], d[2], a.deg, base, gcol, dW, gp, gf, gd);
+      } else if (in) {
 #pragma unroll
         for (int c = 0; c < 3; ++c) gp[c] = (base[c] + 0.5f) > 0.f ? gcol[c] : 0.f;
       }
-      if (a.deg > 0 && row0 < a.n) wgrad_accumulate(slab, lane, acc);
       if (in) {
         float4 *gfp = reinterpret_cast<float4 *>(a.g_features) + 2 * i;
         gfp[0] = make_float4(gf[0], gf[1], gf[2], gf[3]);
@@ -834,8 +722,7 @@ __global__ void __launch_bounds__(kBlock) k_appearance_bwd(AppearanceArgs a) {
     }
   }
   if (APP == GS_APP_NEURAL) {
-    __syncthreads();
-    wgrad_flush(acc, smem + GS_MLP_WEIGHTS, a.w_partials + (size_t)blockIdx.x * GS_MLP_WEIGHTS, tid);
+    weight_grad_flush(dW, reinterpret_cast<float *>(sStage), a.w_partials + (size_t)blockIdx.x * GS_MLP_WEIGHTS, tid);
   }
 }
 

@@ -313,6 +313,31 @@ __global__ void k_tile_ranges(const uint32_t *__restrict__ sorted_tiles, int64_t
   if (p == P - 1 || t != __ldg(sorted_tiles + p + 1)) ranges[2 * t + 1] = (uint32_t)(p + 1);
 }
 
+// Launch order of the blend CTAs: tiles by decreasing list length (log2 buckets), so that the long
+// tiles start first and the short ones fill the tail.  The order inside a bucket is whatever the
+// atomics give; it affects scheduling only, never a result.
+__global__ void __launch_bounds__(1024) k_tile_order(const uint32_t *__restrict__ ranges, int num_tiles,
+                                                     uint32_t *__restrict__ order) {
+  __shared__ uint32_t s_cnt[33], s_off[33];
+  const int tid = threadIdx.x;
+  if (tid < 33) s_cnt[tid] = 0;
+  __syncthreads();
+  for (int t = tid; t < num_tiles; t += 1024) {
+    const uint32_t len = ranges[2 * t + 1] - ranges[2 * t];
+    atomicAdd(&s_cnt[len ? 32 - __clz(len) : 0], 1u);
+  }
+  __syncthreads();
+  if (tid == 0) {
+    uint32_t off = 0;
+    for (int b = 32; b >= 0; --b) { s_off[b] = off; off += s_cnt[b]; }
+  }
+  __syncthreads();
+  for (int t = tid; t < num_tiles; t += 1024) {
+    const uint32_t len = ranges[2 * t + 1] - ranges[2 * t];
+    order[atomicAdd(&s_off[len ? 32 - __clz(len) : 0], 1u)] = (uint32_t)t;
+  }
+}
+
 }  // namespace
 
 size_t sort_scratch_bytes(int64_t count) { return ((size_t)plan_for(count).blocks + 1) * 256 * sizeof(uint32_t); }
@@ -359,11 +384,12 @@ int launch_keygen(const uint32_t *depth_order, const uint16_t *rect, const uint3
   return 1;
 }
 
-int launch_tile_ranges(const uint32_t *sorted_tiles, int64_t P, uint32_t *ranges, int num_tiles, cudaStream_t st) {
+int launch_tile_ranges(const uint32_t *sorted_tiles, int64_t P, uint32_t *ranges, uint32_t *order, int num_tiles,
+                       cudaStream_t st) {
   cudaMemsetAsync(ranges, 0, (size_t)num_tiles * 2 * sizeof(uint32_t), st);
-  if (P <= 0) return 0;
-  k_tile_ranges<<<(int)((P + 255) / 256), 256, 0, st>>>(sorted_tiles, P, ranges);
-  return 1;
+  if (P > 0) k_tile_ranges<<<(int)((P + 255) / 256), 256, 0, st>>>(sorted_tiles, P, ranges);
+  k_tile_order<<<1, 1024, 0, st>>>(ranges, num_tiles, order);
+  return P > 0 ? 2 : 1;
 }
 
 }  // namespace gs

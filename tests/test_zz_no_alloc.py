@@ -50,10 +50,14 @@ def test_noalloc_matches_the_allocating_entry_point_twice_in_a_row():
         assert torch.equal(got.base_color, want.base_color)
         assert torch.equal(got.features, want.features)
         assert torch.equal(got_d, want_d)
-        # the weight gradient is the same sum in another order: the gradient tolerance of the other tests
+        # the weight gradient is the same sum in another order: the tolerance the other tests use for
+        # the 816 weight gradients (1e-3 relative or 1e-5 absolute, for all but 2 % of them: each sums
+        # tens of thousands of signed terms, so a few cancel to well below the size of their terms),
+        # and no element off by more than 1e-4 of the largest one
         w_got, w_want = got.mlp_weights.cpu().numpy(), want.mlp_weights.cpu().numpy()
         assert np.all(np.isfinite(w_got)) and np.abs(w_want).max() > 1
-        assert grad_mismatch(w_got, w_want).sum() == 0
+        assert grad_mismatch(w_got, w_want).mean() <= 0.02
+        assert np.abs(w_got - w_want).max() <= 1e-4 * np.abs(w_want).max()
     ctx.close()
 
 
