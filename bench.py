@@ -28,8 +28,11 @@ N_GAUSS, WIDTH, HEIGHT, VIEWS = 1_000_000, 1256, 828, 8
 
 # Algorithmic cost per unit: flops per evaluated list entry of the blend
 # kernels and bytes per Gaussian of the per-Gaussian kernels.
-BLEND_FWD_FLOPS_PER_ENTRY = 14.0
-BLEND_BWD_FLOPS_PER_ENTRY = 14.0
+# Blend kernels (fp32 ALU bound): flops per list entry evaluated for a pixel (the alpha test) and per
+# pair composited, counted from the kernels' arithmetic.
+BLEND_FLOPS_PER_EVALUATED = 8.0       # 3.5 (quad falloff, shared by 4 pixels) + ex2 + mul + min + compare
+BLEND_FWD_FLOPS_PER_COMPOSITED = 10.0  # 1-a, T(1-a), compare, aT, three FMAs
+BLEND_BWD_FLOPS_PER_COMPOSITED = 45.0  # reciprocal, T and S recovery, d/d alpha, nine gradient FMAs
 FP32_LANES_PER_SM, NUM_SMS = 128, 148
 
 
@@ -182,14 +185,18 @@ def run_ours(args):
         # units of the blend kernels: list entries up to each pixel's last composited one, over the views
         entries = 0
         visible = 0
+        evaluated = composited = 0
         for v in range(views):
             r.forward(ds, cams[v])
             torch.cuda.synchronize()
             entries += int(r.n_contrib.sum(dtype=torch.int64).item())
+            ev, co = api.gs_profile_blend_counts(ctx, r.proj, r.binning, cams[v])
+            evaluated += ev; composited += co
             rect = r.proj.rect.to(torch.int32) & 0xFFFF
             visible += int(((rect[:, 2] > rect[:, 0]) & (rect[:, 3] > rect[:, 1])).sum().item())
         results[tag] = dict(ms=ms, stage_ms=stage_ms, stage_launches=stage_launches, pairs=pairs,
-                            entries=entries, visible=visible, host=host, ds=ds, r=r)
+                            entries=entries, visible=visible, evaluated=evaluated, composited=composited,
+                            host=host, ds=ds, r=r)
 
     # ---- end to end through the public API with host buffers (neural arm)
     e2e = None if args.skip_e2e else measure_e2e(api, torch, ctx, results["neural"], cams, G, views, args, timed, dev)
@@ -220,6 +227,9 @@ def run_ours(args):
         "gprimitives_per_s": world * n * views / (ms * 1e-3) / 1e9,
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step,
         "roofline": roof,
+        "rooflines": {k: stage_roofline(k, neural, views, n, peaks, alu_peak)
+                      for k in ("preprocess_fwd", "depth_sort", "keygen", "tile_sort", "blend_fwd", "blend_bwd",
+                                "preprocess_bwd") if stage_ms.get(k, 0) > 0},
         "stages_ms_per_step": {k: round(v, 4) for k, v in stage_ms.items() if v > 0},
         "stage_share": {k: round(v / total_stage, 4) for k, v in stage_ms.items() if v > 0},
         "pairs_per_view": neural["pairs"], "visible_per_view": neural["visible"] / views,
@@ -237,12 +247,17 @@ def run_ours(args):
 def stage_roofline(stage, arm, views, n, peaks, alu_peak):
     ms = arm["stage_ms"][stage] / views          # average duration of one launch of the stage
     if stage in ("blend_fwd", "blend_bwd"):
-        per = BLEND_FWD_FLOPS_PER_ENTRY if stage == "blend_fwd" else BLEND_BWD_FLOPS_PER_ENTRY
-        flops = per * arm["entries"] / views
+        if stage == "blend_fwd":
+            ev, per_c = arm["evaluated"] / views, BLEND_FWD_FLOPS_PER_COMPOSITED
+        else:   # the backward walks each pixel's list only up to its last composited entry
+            ev, per_c = arm["entries"] / views, BLEND_BWD_FLOPS_PER_COMPOSITED
+        co = arm["composited"] / views
+        flops = BLEND_FLOPS_PER_EVALUATED * ev + per_c * co
         achieved = flops / (ms * 1e-3) / 1e12
         return {"kernel": stage, "bound": "alu", "achieved": achieved, "peak": alu_peak, "unit": "TFLOP/s",
                 "frac": achieved / alu_peak, "traffic": None, "peak_source": "148 SMs x 128 lanes x 2 x max SM clock",
-                "units_per_launch": arm["entries"] / views, "flops_per_unit": per}
+                "evaluated_per_launch": ev, "composited_per_launch": co,
+                "flops_per_evaluated": BLEND_FLOPS_PER_EVALUATED, "flops_per_composited": per_c}
     vis = arm["visible"] / views
     app_bytes = 28.0
     per_launch = {"preprocess_fwd": 44.0 * n + 12.0 * n + (app_bytes + 48.0) * vis,

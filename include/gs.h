@@ -89,10 +89,13 @@ typedef struct {
                                    Q = [[l11^2, l11 l21], [l11 l21, l21^2 + l22^2]]                */
   float *color;          /* [n,3]  decoded view-dependent colour (Eq. 2)                       */
   uint32_t *depth_key;   /* [n]    bit pattern of the fp32 camera depth; 0xFFFFFFFF if culled  */
-  uint16_t *rect;        /* [n,4]  tile rectangle (tx0, ty0, tx1, ty1), half open; all zero if
-                                   the Gaussian touches no tile                                */
-  float *extent;         /* [n,2]  optional (may be NULL): half-size in pixels of the box that
-                                   bounds alpha >= 1/255; (-1,-1) if culled before the box test */
+  uint16_t *rect;        /* [n,4]  tile rectangle (tx0, ty0, tx1, ty1), half open, bounding the
+                                   alpha >= 1/255 footprint; all zero if the Gaussian touches no tile */
+  uint32_t *tiles_touched; /* [n]  tiles inside rect that the alpha >= 1/255 ellipse really meets
+                                   (= instances emitted for the Gaussian)                      */
+  float *extent;         /* [n,4]  optional (may be NULL): (ex, ey, tau, 0): half-size in pixels of the
+                                   box that bounds alpha >= 1/255 and tau = 2 ln(255 opacity);
+                                   ex = ey = -1 if culled before the box test                  */
 } GsProjected;
 
 /* Tile binning produced by gs_render_forward (caller-allocated device buffers). */
@@ -218,6 +221,11 @@ typedef enum {
   GS_NUM_STAGES
 } GsStage;
 GsStatus gs_profile_enable(GsContext *ctx, int enable);
+/* Measurement only: for the view last rendered into (proj, bin), count over all pixels the list
+ * entries the blend evaluates (until each pixel stops) and the pairs it composites; these are the
+ * work units of the blend kernels' roofline.  counts_host[2] is a host array; synchronises. */
+GsStatus gs_profile_blend_counts(GsContext *ctx, const GsProjected *proj, const GsBinning *bin, const GsCamera *cam,
+                                 int64_t *counts_host, void *stream);
 GsStatus gs_profile_collect(GsContext *ctx, double *ms, int64_t *launches);
 
 #ifdef __cplusplus

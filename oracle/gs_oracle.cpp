@@ -426,62 +426,138 @@ void gso_appearance_backward(int64_t n, int app, int deg, const double* base_col
 }
 
 // ---------------------------------------------------------------------------------------
-// Integer stage on FP32 per-Gaussian values (u, v, ex, ey) as produced by either side:
-// pixel rect -> tile rect -> tiles touched.  Returns the pair count P.
-// rect = (tx0, ty0, tx1, ty1), half open.
+// Integer stage on per-Gaussian values (centre, Cholesky factor of the conic, box half-extents and
+// tau = 2 ln(255 o)) as produced by either side, in the precision F they come in (float for the
+// GPU's values, double for the oracle's own).
+//
+// A Gaussian's instances are the tiles that its alpha >= 1/255 ellipse
+//     (la dx + lb dy)^2 + (lc dy)^2 <= tau
+// meets, found row of tiles by row of tiles inside the bounding tile rectangle: over the band of
+// pixel-centre rows of one tile row the set is convex, so the tiles it meets are those between
+// its leftmost and rightmost point in the band; the rightmost point is at the band end nearest
+// to dy_r = -lb sqrt(tau/C)/lc (C = lb^2 + lc^2, where the ellipse's tangent is vertical), the
+// leftmost at the end nearest to -dy_r.  tau and the band are padded (2e-5, 1e-5) so that
+// rounding can only add a tile.  Each operation is rounded once, in this order.
 // ---------------------------------------------------------------------------------------
-int64_t gso_tile_rects_f32(int64_t n, const uint8_t* valid, const float* mean2d, const float* extent,
-                           int W, int H, int32_t* rect, uint32_t* tiles_touched) {
+}  // extern "C"
+
+namespace {
+
+template <class F>
+struct Spans {
+  F u, v, ila, lb, lc, taup, dys, eyp;
+  int W, H;
+  void setup(F u_, F v_, F la, F lb_, F lc_, F tau, int W_, int H_) {
+    u = u_; v = v_; lb = lb_; lc = lc_; W = W_; H = H_;
+    taup = tau * (F)1.00002f;
+    const F rl = (F)1 / lc;
+    ila = (F)1 / la;
+    const F b2 = lb * lb, c2 = lc * lc;
+    const F C = b2 + c2;
+    const F q = taup / C;
+    const F br = lb * rl;
+    dys = br * std::sqrt(q);
+    const F st = std::sqrt(taup) * rl;
+    eyp = st * (F)1.00001f;
+  }
+  bool row(int ty, int tx0, int tx1, int& xa, int& xb) const {
+    const F ylo = (F)(16 * ty) + (F)0.5, yhi = std::min((F)(16 * ty) + (F)15.5, (F)H - (F)0.5);
+    const F da = std::max(ylo - v, -eyp), db = std::min(yhi - v, eyp);
+    if (!(da <= db)) return false;
+    const F dyR = std::min(std::max(-dys, da), db), dyL = std::min(std::max(dys, da), db);
+    const F tR = lc * dyR, tL = lc * dyL;
+    const F tR2 = tR * tR, tL2 = tL * tL;
+    const F sR = std::sqrt(std::max(taup - tR2, (F)0)), sL = std::sqrt(std::max(taup - tL2, (F)0));
+    const F bR = lb * dyR, bL = lb * dyL;
+    const F xr = (sR - bR) * ila, xl = (-sL - bL) * ila;
+    const F hi0 = u + xr, lo0 = u + xl;
+    const F ihi = std::floor(hi0 - (F)0.5), ilo = std::ceil(lo0 - (F)0.5);
+    if (!(ilo <= ihi) || ihi < 0 || ilo > (F)(W - 1)) return false;
+    const int pa = (int)std::max(ilo, (F)0), pb = (int)std::min(ihi, (F)(W - 1));
+    xa = std::max(pa >> 4, tx0);
+    xb = std::min((pb >> 4) + 1, tx1);
+    return xa < xb;
+  }
+};
+
+template <class F>
+int64_t tile_spans(int64_t n, const uint8_t* valid, const F* mean2d, const F* chol, const F* ext, int W, int H,
+                   int32_t* rect, uint32_t* tiles_touched) {
   int64_t P = 0;
   for (int64_t i = 0; i < n; ++i) {
     for (int j = 0; j < 4; ++j) rect[4 * i + j] = 0;
     tiles_touched[i] = 0;
     if (!valid[i]) continue;
     int px[4]; bool empty;
-    pixel_rect<float>(mean2d[2 * i], mean2d[2 * i + 1], extent[2 * i], extent[2 * i + 1], W, H, px, empty);
+    pixel_rect<F>(mean2d[2 * i], mean2d[2 * i + 1], ext[4 * i], ext[4 * i + 1], W, H, px, empty);
     if (empty) continue;
     int t[4];
     tile_rect(px, t);
+    Spans<F> sp;
+    sp.setup(mean2d[2 * i], mean2d[2 * i + 1], chol[3 * i], chol[3 * i + 1], chol[3 * i + 2], ext[4 * i + 2], W, H);
+    uint32_t c = 0;
+    for (int ty = t[1]; ty < t[3]; ++ty) {
+      int xa, xb;
+      if (sp.row(ty, t[0], t[2], xa, xb)) c += (uint32_t)(xb - xa);
+    }
+    if (c == 0) continue;
     for (int j = 0; j < 4; ++j) rect[4 * i + j] = t[j];
-    tiles_touched[i] = (uint32_t)((t[2] - t[0]) * (t[3] - t[1]));
-    P += tiles_touched[i];
+    tiles_touched[i] = c;
+    P += c;
   }
   return P;
 }
 
-// Same from the oracle's own double-precision pixel rects.
-int64_t gso_tile_rects_from_px(int64_t n, const uint8_t* visible, const int32_t* rect_px,
-                               int32_t* rect, uint32_t* tiles_touched) {
-  int64_t P = 0;
-  for (int64_t i = 0; i < n; ++i) {
-    for (int j = 0; j < 4; ++j) rect[4 * i + j] = 0;
-    tiles_touched[i] = 0;
-    if (!visible[i]) continue;
-    int px[4] = {rect_px[4 * i], rect_px[4 * i + 1], rect_px[4 * i + 2], rect_px[4 * i + 3]};
-    int t[4];
-    tile_rect(px, t);
-    for (int j = 0; j < 4; ++j) rect[4 * i + j] = t[j];
-    tiles_touched[i] = (uint32_t)((t[2] - t[0]) * (t[3] - t[1]));
-    P += tiles_touched[i];
-  }
-  return P;
-}
-
-// Emit instances for Gaussian index ascending, inside a rect ty-major then tx; key =
-// (tile_id << 32) | depth_bits; stable sort by key; per-tile [start, end).
-void gso_sorted_instances(int64_t n, const int32_t* rect, const uint32_t* depth_bits, int gx,
-                          int64_t P, uint64_t* keys, uint32_t* vals) {
+// Emit instances for Gaussian index ascending, tile rows top to bottom, tiles left to right;
+// key = (tile_id << 32) | depth_bits; stable sort by key.
+template <class F>
+void sorted_instances(int64_t n, const int32_t* rect, const uint32_t* tiles_touched, const F* mean2d, const F* chol,
+                      const F* ext, const uint32_t* depth_bits, int W, int H, int64_t P, uint64_t* keys,
+                      uint32_t* vals) {
+  const int gx = (W + kTile - 1) / kTile;
   std::vector<std::pair<uint64_t, uint32_t>> inst;
   inst.reserve((size_t)P);
-  for (int64_t i = 0; i < n; ++i)
-    for (int ty = rect[4 * i + 1]; ty < rect[4 * i + 3]; ++ty)
-      for (int tx = rect[4 * i]; tx < rect[4 * i + 2]; ++tx)
+  for (int64_t i = 0; i < n; ++i) {
+    if (!tiles_touched[i]) continue;
+    Spans<F> sp;
+    sp.setup(mean2d[2 * i], mean2d[2 * i + 1], chol[3 * i], chol[3 * i + 1], chol[3 * i + 2], ext[4 * i + 2], W, H);
+    for (int ty = rect[4 * i + 1]; ty < rect[4 * i + 3]; ++ty) {
+      int xa, xb;
+      if (!sp.row(ty, rect[4 * i], rect[4 * i + 2], xa, xb)) continue;
+      for (int tx = xa; tx < xb; ++tx)
         inst.emplace_back(((uint64_t)(ty * gx + tx) << 32) | depth_bits[i], (uint32_t)i);
+    }
+  }
   std::stable_sort(inst.begin(), inst.end(),
                    [](const std::pair<uint64_t, uint32_t>& a, const std::pair<uint64_t, uint32_t>& b) {
                      return a.first < b.first;
                    });
-  for (int64_t p = 0; p < P; ++p) { keys[p] = inst[p].first; vals[p] = inst[p].second; }
+  for (int64_t p = 0; p < P && p < (int64_t)inst.size(); ++p) { keys[p] = inst[p].first; vals[p] = inst[p].second; }
+}
+
+}  // namespace
+
+extern "C" {
+
+// mean2d [n,2], chol [n,3] = (la, lb, lc), ext [n,4] = (ex, ey, tau, -).  rect = (tx0, ty0, tx1, ty1),
+// half open (all zero when no tile is met).  Return the pair count P.
+int64_t gso_tile_spans_f32(int64_t n, const uint8_t* valid, const float* mean2d, const float* chol, const float* ext,
+                           int W, int H, int32_t* rect, uint32_t* tiles_touched) {
+  return tile_spans<float>(n, valid, mean2d, chol, ext, W, H, rect, tiles_touched);
+}
+int64_t gso_tile_spans_f64(int64_t n, const uint8_t* valid, const double* mean2d, const double* chol,
+                           const double* ext, int W, int H, int32_t* rect, uint32_t* tiles_touched) {
+  return tile_spans<double>(n, valid, mean2d, chol, ext, W, H, rect, tiles_touched);
+}
+void gso_sorted_instances_f32(int64_t n, const int32_t* rect, const uint32_t* tiles_touched, const float* mean2d,
+                              const float* chol, const float* ext, const uint32_t* depth_bits, int W, int H,
+                              int64_t P, uint64_t* keys, uint32_t* vals) {
+  sorted_instances<float>(n, rect, tiles_touched, mean2d, chol, ext, depth_bits, W, H, P, keys, vals);
+}
+void gso_sorted_instances_f64(int64_t n, const int32_t* rect, const uint32_t* tiles_touched, const double* mean2d,
+                              const double* chol, const double* ext, const uint32_t* depth_bits, int W, int H,
+                              int64_t P, uint64_t* keys, uint32_t* vals) {
+  sorted_instances<double>(n, rect, tiles_touched, mean2d, chol, ext, depth_bits, W, H, P, keys, vals);
 }
 
 void gso_tile_ranges(int64_t P, const uint64_t* keys, int num_tiles, uint32_t* ranges) {

@@ -44,8 +44,6 @@ def lib():
     if _lib is None:
         build()
         _lib = C.CDLL(_LIB)
-        _lib.gso_tile_rects_f32.restype = C.c_int64
-        _lib.gso_tile_rects_from_px.restype = C.c_int64
         _lib.gso_num_mlp_weights.restype = C.c_int
         _lib.gso_mlp_macs.restype = C.c_int
     return _lib
@@ -157,35 +155,61 @@ def appearance_backward(scene, dirs, g_color, mask=None, deg=None):
     return o
 
 
-def tile_rects_f32(valid, mean2d_f32, extent_f32, width, height):
-    """Integer stage on fp32 per-Gaussian values (from either side)."""
+def _tile_spans(suffix, dtype, ctype, valid, mean2d, chol, ext, width, height):
     valid = np.ascontiguousarray(valid, np.uint8)
-    m = np.ascontiguousarray(mean2d_f32, np.float32); e = np.ascontiguousarray(extent_f32, np.float32)
+    m = np.ascontiguousarray(mean2d, dtype); c = np.ascontiguousarray(chol, dtype)
+    e = np.ascontiguousarray(ext, dtype)
     n = valid.shape[0]
+    assert m.shape == (n, 2) and c.shape == (n, 3) and e.shape == (n, 4)
     rect = np.zeros((n, 4), np.int32); tt = np.zeros(n, np.uint32)
-    P = lib().gso_tile_rects_f32(C.c_int64(n), _p(valid, C.c_uint8), _p(m, C.c_float), _p(e, C.c_float),
-                                 C.c_int(width), C.c_int(height), _p(rect, C.c_int32), _p(tt, C.c_uint32))
+    f = getattr(lib(), "gso_tile_spans_" + suffix)
+    f.restype = C.c_int64
+    P = f(C.c_int64(n), _p(valid, C.c_uint8), _p(m, ctype), _p(c, ctype), _p(e, ctype), C.c_int(width),
+          C.c_int(height), _p(rect, C.c_int32), _p(tt, C.c_uint32))
     return rect, tt, int(P)
 
 
-def tile_rects_from_px(visible, rect_px):
-    visible = np.ascontiguousarray(visible, np.uint8); rect_px = np.ascontiguousarray(rect_px, np.int32)
-    n = visible.shape[0]
-    rect = np.zeros((n, 4), np.int32); tt = np.zeros(n, np.uint32)
-    P = lib().gso_tile_rects_from_px(C.c_int64(n), _p(visible, C.c_uint8), _p(rect_px, C.c_int32),
-                                     _p(rect, C.c_int32), _p(tt, C.c_uint32))
-    return rect, tt, int(P)
-
-
-def sorted_instances(rect, depth_bits, width, height, P):
-    rect = np.ascontiguousarray(rect, np.int32); db = np.ascontiguousarray(depth_bits, np.uint32)
+def _sorted_instances(suffix, dtype, ctype, rect, tt, mean2d, chol, ext, depth_bits, width, height, P):
+    rect = np.ascontiguousarray(rect, np.int32); tt = np.ascontiguousarray(tt, np.uint32)
+    m = np.ascontiguousarray(mean2d, dtype); c = np.ascontiguousarray(chol, dtype)
+    e = np.ascontiguousarray(ext, dtype); db = np.ascontiguousarray(depth_bits, np.uint32)
     gx, gy = (width + TILE - 1) // TILE, (height + TILE - 1) // TILE
     keys = np.zeros(P, np.uint64); vals = np.zeros(P, np.uint32)
     ranges = np.zeros((gx * gy, 2), np.uint32)
-    lib().gso_sorted_instances(C.c_int64(rect.shape[0]), _p(rect, C.c_int32), _p(db, C.c_uint32),
-                               C.c_int(gx), C.c_int64(P), _p(keys, C.c_uint64), _p(vals, C.c_uint32))
+    getattr(lib(), "gso_sorted_instances_" + suffix)(
+        C.c_int64(rect.shape[0]), _p(rect, C.c_int32), _p(tt, C.c_uint32), _p(m, ctype), _p(c, ctype), _p(e, ctype),
+        _p(db, C.c_uint32), C.c_int(width), C.c_int(height), C.c_int64(P), _p(keys, C.c_uint64), _p(vals, C.c_uint32))
     lib().gso_tile_ranges(C.c_int64(P), _p(keys, C.c_uint64), C.c_int(gx * gy), _p(ranges, C.c_uint32))
     return keys, vals, ranges
+
+
+def tile_spans_f32(valid, mean2d, chol, ext, width, height):
+    """Integer stage on fp32 per-Gaussian values (from either side): bounding tile rectangle, tiles
+    the alpha >= 1/255 ellipse meets, pair count.  chol = (la, lb, lc), ext = (ex, ey, tau, -)."""
+    return _tile_spans("f32", np.float32, C.c_float, valid, mean2d, chol, ext, width, height)
+
+
+def sorted_instances_f32(rect, tt, mean2d, chol, ext, depth_bits, width, height, P):
+    return _sorted_instances("f32", np.float32, C.c_float, rect, tt, mean2d, chol, ext, depth_bits, width, height, P)
+
+
+def tile_spans_f64(valid, mean2d, chol, ext, width, height):
+    return _tile_spans("f64", np.float64, C.c_double, valid, mean2d, chol, ext, width, height)
+
+
+def sorted_instances_f64(rect, tt, mean2d, chol, ext, depth_bits, width, height, P):
+    return _sorted_instances("f64", np.float64, C.c_double, rect, tt, mean2d, chol, ext, depth_bits, width, height, P)
+
+
+def cholesky_of_conic(conic):
+    """(la, lb, lc) with conic = [[la^2, la lb], [la lb, lb^2 + lc^2]]."""
+    conic = np.asarray(conic, np.float64)
+    with np.errstate(invalid="ignore", divide="ignore"):
+        la = np.sqrt(conic[:, 0]); lb = conic[:, 1] / la
+        lc = np.sqrt(np.maximum(conic[:, 2] - lb * lb, 0.0))
+    out = np.stack([la, lb, lc], 1)
+    out[~np.isfinite(out).all(1)] = 0
+    return out
 
 
 def blend_forward(cam, vals, ranges, mean2d, conic, opacity, color):
@@ -252,9 +276,16 @@ def preprocess_backward(means, log_scales, quats, opacity_logits, cam, visible, 
 
 def render_forward(scene, cam):
     pre = preprocess(scene.means, scene.log_scales, scene.quats, scene.opacity_logits, cam)
+    chol = cholesky_of_conic(pre.conic)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        tau = np.where(pre.valid > 0, 2.0 * np.log(255.0 * pre.opacity), 0.0)
+    ext = np.concatenate([pre.extent, tau[:, None], np.zeros_like(tau)[:, None]], 1)
+    rect, tiles_touched, P = tile_spans_f64(pre.valid, pre.mean2d, chol, ext, cam.width, cam.height)
+    pre.visible = (tiles_touched > 0).astype(np.uint8)      # visible = meets at least one tile
+    pre.chol, pre.ext = chol, ext
     color, resid = appearance_forward(scene, pre.dir, mask=pre.visible)
-    rect, tiles_touched, P = tile_rects_from_px(pre.visible, pre.rect_px)
-    keys, vals, ranges = sorted_instances(rect, pre.depth_bits, cam.width, cam.height, P)
+    keys, vals, ranges = sorted_instances_f64(rect, tiles_touched, pre.mean2d, chol, ext, pre.depth_bits,
+                                              cam.width, cam.height, P)
     bl = blend_forward(cam, vals, ranges, pre.mean2d, pre.conic, pre.opacity, color)
     return SimpleNamespace(pre=pre, color=color, residual=resid, rect=rect, tiles_touched=tiles_touched,
                            P=P, keys=keys, vals=vals, ranges=ranges, image=bl.image, final_T=bl.final_T,

@@ -44,7 +44,7 @@ class GsScene(C.Structure):
 
 class GsProjected(C.Structure):
     _fields_ = [("mean2d", _vp), ("conic_opacity", _vp), ("color", _vp), ("depth_key", _vp), ("rect", _vp),
-                ("extent", _vp)]
+                ("tiles_touched", _vp), ("extent", _vp)]
 
 
 class GsBinning(C.Structure):
@@ -87,6 +87,11 @@ _lib.gs_profile_enable.argtypes = [_vp, C.c_int]
 _lib.gs_profile_enable.restype = C.c_int
 _lib.gs_profile_collect.argtypes = [_vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
 _lib.gs_profile_collect.restype = C.c_int
+
+
+_lib.gs_profile_blend_counts.argtypes = [_vp, C.POINTER(GsProjected), C.POINTER(GsBinning), C.POINTER(GsCamera),
+                                         C.POINTER(C.c_int64), _vp]
+_lib.gs_profile_blend_counts.restype = C.c_int
 
 
 class GsError(RuntimeError):
@@ -164,12 +169,14 @@ class Projected:
     color: torch.Tensor
     depth_key: torch.Tensor    # int32 storage holding the uint32 bit patterns
     rect: torch.Tensor         # int16 storage holding uint16 tile coordinates, [n,4]
+    tiles_touched: torch.Tensor
     extent: Optional[torch.Tensor]
 
     def c_struct(self) -> GsProjected:
         p = GsProjected()
         p.mean2d, p.conic_opacity, p.color = _ptr(self.mean2d), _ptr(self.conic_opacity), _ptr(self.color)
         p.depth_key, p.rect, p.extent = _ptr(self.depth_key), _ptr(self.rect), _ptr(self.extent)
+        p.tiles_touched = _ptr(self.tiles_touched)
         return p
 
 
@@ -179,7 +186,8 @@ def alloc_projected(n: int, device, with_extent: bool = True) -> Projected:
     return Projected(torch.empty((m, 2), **f), torch.empty((m, 4), **f), torch.empty((m, 3), **f),
                      torch.empty((m,), device=device, dtype=torch.int32),
                      torch.empty((m, 4), device=device, dtype=torch.int16),
-                     torch.empty((m, 2), **f) if with_extent else None)
+                     torch.empty((m,), device=device, dtype=torch.int32),
+                     torch.empty((m, 4), **f) if with_extent else None)
 
 
 @dataclass
@@ -273,6 +281,15 @@ def gs_profile_collect(ctx: Context):
     launches = (C.c_int64 * len(STAGES))()
     ctx._check(_lib.gs_profile_collect(ctx._h, ms, launches))
     return dict(zip(STAGES, list(ms))), dict(zip(STAGES, list(launches)))
+
+
+def gs_profile_blend_counts(ctx: Context, proj: "Projected", binning: "Binning", cam: GsCamera, stream=None):
+    """(list entries evaluated, pairs composited) over all pixels of the view held in proj / binning."""
+    out = (C.c_int64 * 2)()
+    pp, bb = proj.c_struct(), binning.c_struct()
+    ctx._check(_lib.gs_profile_blend_counts(ctx._h, C.byref(pp), C.byref(bb), C.byref(cam), out,
+                                            _stream_handle(stream)))
+    return int(out[0]), int(out[1])
 
 
 def gs_workspace_bytes(n: int, width: int, height: int, pair_capacity: int) -> int:

@@ -13,7 +13,7 @@ struct StageRecord { int stage; int launches; cudaEvent_t begin, end; };
 
 struct GsContext {
   int device;
-  unsigned long long *d_counter;      // device: instance counter
+  unsigned long long *d_counter;      // device: instance counter (+ one more word for gs_profile_blend_counts)
   unsigned long long *h_counter;      // pinned host mirror
   float *d_w_partials;                // device: [kWgradBlocks, 816] decoder-gradient partial sums
   char error[256];
@@ -172,8 +172,8 @@ GsStatus gs_create(int device, GsContext **out) {
   ctx->error[0] = 0;
   ctx->d_counter = nullptr; ctx->h_counter = nullptr; ctx->d_w_partials = nullptr;
   ctx->profiling = false;
-  if (cudaMalloc(&ctx->d_counter, sizeof(unsigned long long)) != cudaSuccess ||
-      cudaMallocHost(&ctx->h_counter, sizeof(unsigned long long)) != cudaSuccess ||
+  if (cudaMalloc(&ctx->d_counter, 2 * sizeof(unsigned long long)) != cudaSuccess ||
+      cudaMallocHost(&ctx->h_counter, 2 * sizeof(unsigned long long)) != cudaSuccess ||
       cudaMalloc(&ctx->d_w_partials, sizeof(float) * kWgradBlocks * GS_MLP_WEIGHTS) != cudaSuccess) {
     gs_destroy(ctx);
     return GS_ERR_CUDA;
@@ -211,7 +211,7 @@ GsStatus gs_preprocess(GsContext *ctx, const GsScene *scene, const GsCamera *cam
   *num_pairs_host = 0;
   if (scene->n == 0) return GS_OK;
   if (bad_ptr(out->mean2d) || bad_ptr(out->conic_opacity) || bad_ptr(out->color) || bad_ptr(out->depth_key) ||
-      bad_ptr(out->rect) || (out->extent && !aligned16(out->extent)))
+      bad_ptr(out->rect) || bad_ptr(out->tiles_touched) || (out->extent && !aligned16(out->extent)))
     return fail(ctx, GS_ERR_INVALID_ARG, "a GsProjected buffer is NULL or misaligned");
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   cudaSetDevice(ctx->device);
@@ -223,7 +223,7 @@ GsStatus gs_preprocess(GsContext *ctx, const GsScene *scene, const GsCamera *cam
   a.weights = reinterpret_cast<const __half *>(scene->mlp_weights);
   a.deg = scene->active_degree;
   a.mean2d = out->mean2d; a.conic_opacity = out->conic_opacity; a.color = out->color; a.extent = out->extent;
-  a.depth_key = out->depth_key; a.rect = out->rect;
+  a.depth_key = out->depth_key; a.rect = out->rect; a.tiles_touched = out->tiles_touched;
   a.pair_counter = ctx->d_counter;
   if ((st = check_cuda(ctx, cudaMemsetAsync(ctx->d_counter, 0, sizeof(unsigned long long), s), "memset")) != GS_OK) return st;
   {
@@ -253,7 +253,8 @@ GsStatus gs_render_forward(GsContext *ctx, int64_t n, const GsProjected *proj, c
   if (workspace_bytes < gs_workspace_bytes(n, cam->width, cam->height, pair_capacity) || bad_ptr(workspace))
     return fail(ctx, GS_ERR_CAPACITY, "workspace is NULL, misaligned or smaller than gs_workspace_bytes()");
   if (n > 0 && (bad_ptr(proj->mean2d) || bad_ptr(proj->conic_opacity) || bad_ptr(proj->color) ||
-                bad_ptr(proj->depth_key) || bad_ptr(proj->rect) || bad_ptr(bin->depth_order)))
+                bad_ptr(proj->depth_key) || bad_ptr(proj->rect) || bad_ptr(proj->tiles_touched) ||
+                bad_ptr(bin->depth_order)))
     return fail(ctx, GS_ERR_INVALID_ARG, "a per-Gaussian buffer is NULL or misaligned");
   if (num_pairs > 0 && (bad_ptr(bin->sorted_tiles) || bad_ptr(bin->sorted_vals)))
     return fail(ctx, GS_ERR_INVALID_ARG, "an instance buffer is NULL or misaligned");
@@ -272,11 +273,12 @@ GsStatus gs_render_forward(GsContext *ctx, int64_t n, const GsProjected *proj, c
     // stage 2: instances in depth order, then a stable sort by tile id alone
     {
       StageTimer t(ctx, GS_STAGE_TILE_OFFSETS, s);
-      t.done(launch_tile_offsets(bin->depth_order, proj->rect, w.block_offsets, n, nullptr, s));
+      t.done(launch_tile_offsets(bin->depth_order, proj->tiles_touched, w.block_offsets, n, nullptr, s));
     }
     {
       StageTimer t(ctx, GS_STAGE_KEYGEN, s);
-      t.done(launch_keygen(bin->depth_order, proj->rect, w.block_offsets, w.inst_tiles, w.inst_vals, n, cd.gx, s));
+      t.done(launch_keygen(bin->depth_order, proj->rect, proj->mean2d, proj->conic_opacity, proj->tiles_touched,
+                           w.block_offsets, w.inst_tiles, w.inst_vals, n, cd.gx, cd.W, cd.H, s));
     }
     {
       StageTimer t(ctx, GS_STAGE_TILE_SORT, s);
@@ -409,6 +411,24 @@ GsStatus gs_appearance_backward(GsContext *ctx, const GsScene *scene, const floa
     t.done(launch_appearance_bwd(scene->app, a, s));
   }
   return check_cuda(ctx, cudaGetLastError(), "appearance_backward launch");
+}
+
+GsStatus gs_profile_blend_counts(GsContext *ctx, const GsProjected *proj, const GsBinning *bin, const GsCamera *cam,
+                                 int64_t *counts_host, void *stream) {
+  if (!ctx) return GS_ERR_INVALID_ARG;
+  if (!proj || !bin || !counts_host || !camera_ok(cam)) return fail(ctx, GS_ERR_INVALID_ARG, "bad argument");
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaSetDevice(ctx->device);
+  GsStatus st;
+  if ((st = check_cuda(ctx, cudaMemsetAsync(ctx->d_counter, 0, 2 * sizeof(unsigned long long), s), "memset")) != GS_OK) return st;
+  launch_blend_count(make_cam(cam), bin->tile_ranges, bin->sorted_vals, proj->mean2d, proj->conic_opacity, proj->color,
+                     ctx->d_counter, s);
+  if ((st = check_cuda(ctx, cudaMemcpyAsync(ctx->h_counter, ctx->d_counter, 2 * sizeof(unsigned long long),
+                                            cudaMemcpyDeviceToHost, s), "count copy")) != GS_OK) return st;
+  if ((st = check_cuda(ctx, cudaStreamSynchronize(s), "blend counts")) != GS_OK) return st;
+  counts_host[0] = (int64_t)ctx->h_counter[0];
+  counts_host[1] = (int64_t)ctx->h_counter[1];
+  return GS_OK;
 }
 
 GsStatus gs_profile_enable(GsContext *ctx, int enable) {

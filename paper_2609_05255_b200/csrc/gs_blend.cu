@@ -294,7 +294,71 @@ __global__ void __launch_bounds__(kThreads) k_blend_bwd(CamDev cam, const uint32
   }
 }
 
+// Measurement only: replay the forward's decisions and count, over all pixels, the list entries
+// evaluated (until each pixel stopped) and the pairs composited.  counts[0] += evaluated,
+// counts[1] += composited.
+__global__ void __launch_bounds__(kThreads) k_blend_count(CamDev cam, const uint32_t *__restrict__ ranges,
+                                                          const uint32_t *__restrict__ vals,
+                                                          const float *__restrict__ mean2d,
+                                                          const float *__restrict__ conic_opacity,
+                                                          const float *__restrict__ color,
+                                                          unsigned long long *__restrict__ counts) {
+  __shared__ float4 s_xyab[kBatch];
+  __shared__ float2 s_co[kBatch];
+  __shared__ float4 s_rgb[kBatch];
+  const int tid = threadIdx.x, tile = blockIdx.x;
+  int px, py;
+  quad_of(tile, cam.gx, tid, px, py);
+  const float fx = (float)px + 0.5f, fy = (float)py + 0.5f;
+  const uint32_t start = __ldg(ranges + 2 * tile), end = __ldg(ranges + 2 * tile + 1);
+  float T[4] = {1.f, 1.f, 1.f, 1.f};
+  unsigned live = 0;
+  unsigned long long evaluated = 0, composited = 0;
+#pragma unroll
+  for (int k = 0; k < 4; ++k)
+    if (px + (k & 1) < cam.W && py + (k >> 1) < cam.H) live |= 1u << k;
+  for (uint32_t base = start; base < end; base += kBatch) {
+    if (__syncthreads_and(live == 0)) break;
+#pragma unroll
+    for (int h = 0; h < kBatch / kThreads; ++h) {
+      const int slot = tid + h * kThreads;
+      const uint32_t idx = base + slot;
+      if (idx < end) stage_entry(__ldg(vals + idx), mean2d, conic_opacity, color, s_xyab[slot], s_co[slot], s_rgb[slot]);
+    }
+    __syncthreads();
+    const int cnt = (int)min((uint32_t)kBatch, end - base);
+    for (int j = 0; j < cnt && live; ++j) {
+      const float4 a = s_xyab[j];
+      const float2 c = s_co[j];
+      float p[4], t1[4], t2[2];
+      quad_power(fx - a.x, fy - a.y, a.z, a.w, c.x, p, t1, t2);
+      evaluated += __popc(live);
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        float e2, alpha;
+        if (!((live >> k) & 1u) || !alpha_of(p[k], c.y, e2, alpha)) continue;
+        const float Tn = __fmul_rn(T[k], 1.f - alpha);
+        if (Tn < kTmin) { live &= ~(1u << k); continue; }
+        T[k] = Tn;
+        ++composited;
+      }
+    }
+  }
+#pragma unroll
+  for (int s = 16; s > 0; s >>= 1) {
+    evaluated += __shfl_xor_sync(kFull, evaluated, s);
+    composited += __shfl_xor_sync(kFull, composited, s);
+  }
+  if ((tid & 31) == 0) { atomicAdd(counts, evaluated); atomicAdd(counts + 1, composited); }
+}
+
 }  // namespace
+
+int launch_blend_count(const CamDev &cam, const uint32_t *ranges, const uint32_t *vals, const float *mean2d,
+                       const float *conic_opacity, const float *color, unsigned long long *counts, cudaStream_t st) {
+  k_blend_count<<<cam.gx * cam.gy, kThreads, 0, st>>>(cam, ranges, vals, mean2d, conic_opacity, color, counts);
+  return 1;
+}
 
 int launch_blend_fwd(const CamDev &cam, const uint32_t *ranges, const uint32_t *order, const uint32_t *vals,
                      const float *mean2d,

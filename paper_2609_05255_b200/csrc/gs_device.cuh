@@ -36,7 +36,7 @@ struct PreprocessArgs {
   const __half *features, *weights;
   int deg;
   float *mean2d, *conic_opacity, *color, *extent;
-  uint32_t *depth_key;
+  uint32_t *depth_key, *tiles_touched;
   uint16_t *rect;
   unsigned long long *pair_counter;
 };
@@ -78,10 +78,11 @@ int launch_radix_sort(const uint32_t *keys_in, const uint32_t *vals_in, uint32_t
                        uint32_t *vals_out, uint32_t *tmp_keys, uint32_t *tmp_vals, int64_t count,
                        int num_bits, void *scratch, cudaStream_t st);
 size_t scan_scratch_bytes(int64_t n);
-int launch_tile_offsets(const uint32_t *depth_order, const uint16_t *rect, uint32_t *offsets,
-                         int64_t n, void *scratch, cudaStream_t st);
-int launch_keygen(const uint32_t *depth_order, const uint16_t *rect, const uint32_t *offsets,
-                   uint32_t *inst_tiles, uint32_t *inst_vals, int64_t n, int gx, cudaStream_t st);
+int launch_tile_offsets(const uint32_t *depth_order, const uint32_t *tiles_touched, uint32_t *offsets,
+                        int64_t n, void *scratch, cudaStream_t st);
+int launch_keygen(const uint32_t *depth_order, const uint16_t *rect, const float *mean2d, const float *conic_opacity,
+                  const uint32_t *tiles_touched, const uint32_t *offsets, uint32_t *inst_tiles, uint32_t *inst_vals,
+                  int64_t n, int gx, int W, int H, cudaStream_t st);
 int launch_tile_ranges(const uint32_t *sorted_tiles, int64_t P, uint32_t *ranges, uint32_t *order,
                        int num_tiles, cudaStream_t st);
 
@@ -93,6 +94,9 @@ int launch_blend_bwd(const CamDev &cam, const uint32_t *ranges, const uint32_t *
                       const float *mean2d, const float *conic_opacity, const float *color,
                       const float *final_T, const uint32_t *n_contrib, const float *dL_dimage,
                       float *g2d, cudaStream_t st);
+
+int launch_blend_count(const CamDev &cam, const uint32_t *ranges, const uint32_t *vals, const float *mean2d,
+                       const float *conic_opacity, const float *color, unsigned long long *counts, cudaStream_t st);
 
 // ---- device helpers -------------------------------------------------------------------------
 #ifdef __CUDACC__
@@ -147,6 +151,58 @@ __device__ __forceinline__ void sh_grad_acc(int k, float x, float y, float z, fl
     default: break;
   }
 }
+
+// tau = 2 ln(255 o): the alpha >= 1/255 ellipse is conic-form <= tau.  One function, so that the
+// preprocess and the instance emission get identical bits.
+__device__ __forceinline__ float footprint_tau(float o) { return 2.f * logf(255.f * o); }
+
+// Exact tile overlap of the alpha >= 1/255 ellipse, row of tiles by row of tiles.  The ellipse is
+// (la dx + lb dy)^2 + (lc dy)^2 <= tau with (la, lb, lc) the Cholesky factor of the conic.  Over a
+// band of pixel-centre rows dy in [da, db] the set is convex, so the tiles it meets in that row are
+// exactly those between its leftmost and rightmost point; the rightmost point over the band is at
+// the band end nearest to dy_r = -lb sqrt(tau / C) / lc (C = lb^2 + lc^2), the leftmost at the one
+// nearest to -dy_r.  Every operation is rounded once, in a fixed order (no contraction), so the
+// same integers come out of any IEEE fp32 evaluation; tau and the band are padded by 2e-5 / 1e-5
+// so that rounding can only add a tile, never drop a pixel the blend would accept.
+struct TileSpans {
+  float u, v, ila, lb, lc, taup, dys, eyp;
+  int W, H;
+  __device__ __forceinline__ void setup(float u_, float v_, float la, float lb_, float lc_, float tau, int W_, int H_) {
+    u = u_; v = v_; lb = lb_; lc = lc_; W = W_; H = H_;
+    taup = __fmul_rn(tau, 1.00002f);
+    const float rl = __frcp_rn(lc);
+    ila = __frcp_rn(la);
+    const float C = __fadd_rn(__fmul_rn(lb, lb), __fmul_rn(lc, lc));
+    dys = __fmul_rn(__fmul_rn(lb, rl), __fsqrt_rn(__fdiv_rn(taup, C)));
+    eyp = __fmul_rn(__fmul_rn(__fsqrt_rn(taup), rl), 1.00001f);
+  }
+  // Tiles [xa, xb) of tile row ty, clipped to the bounding rectangle's columns [tx0, tx1).
+  __device__ __forceinline__ bool row(int ty, int tx0, int tx1, int &xa, int &xb) const {
+    const float ylo = (float)(16 * ty) + 0.5f, yhi = fminf((float)(16 * ty) + 15.5f, (float)H - 0.5f);
+    const float da = fmaxf(__fsub_rn(ylo, v), -eyp), db = fminf(__fsub_rn(yhi, v), eyp);
+    if (!(da <= db)) return false;
+    const float dyR = fminf(fmaxf(-dys, da), db), dyL = fminf(fmaxf(dys, da), db);
+    const float tR = __fmul_rn(lc, dyR), tL = __fmul_rn(lc, dyL);
+    const float sR = __fsqrt_rn(fmaxf(__fsub_rn(taup, __fmul_rn(tR, tR)), 0.f));
+    const float sL = __fsqrt_rn(fmaxf(__fsub_rn(taup, __fmul_rn(tL, tL)), 0.f));
+    const float xr = __fmul_rn(__fsub_rn(sR, __fmul_rn(lb, dyR)), ila);
+    const float xl = __fmul_rn(__fsub_rn(-sL, __fmul_rn(lb, dyL)), ila);
+    const float ihi = floorf(__fsub_rn(__fadd_rn(u, xr), 0.5f)), ilo = ceilf(__fsub_rn(__fadd_rn(u, xl), 0.5f));
+    if (!(ilo <= ihi) || ihi < 0.f || ilo > (float)(W - 1)) return false;
+    const int pa = (int)fmaxf(ilo, 0.f), pb = (int)fminf(ihi, (float)(W - 1));
+    xa = max(pa >> 4, tx0);
+    xb = min((pb >> 4) + 1, tx1);
+    return xa < xb;
+  }
+  __device__ __forceinline__ unsigned count(int tx0, int ty0, int tx1, int ty1) const {
+    unsigned c = 0;
+    for (int ty = ty0; ty < ty1; ++ty) {
+      int xa, xb;
+      if (row(ty, tx0, tx1, xa, xb)) c += (unsigned)(xb - xa);
+    }
+    return c;
+  }
+};
 
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;

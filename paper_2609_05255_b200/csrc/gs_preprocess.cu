@@ -195,7 +195,7 @@ __global__ void k_wgrad_reduce(const float *__restrict__ partials, int nblocks, 
 // ---- projection -----------------------------------------------------------------------------
 struct Geo {
   bool valid;
-  float u, v, A, B, C, o, ex, ey;   // (A, B, C) = (l11, l21, l22), the Cholesky factor of the conic
+  float u, v, A, B, C, o, ex, ey, tau;   // (A, B, C) = (l11, l21, l22), the Cholesky factor of the conic
   uint32_t zbits;
   float dirx, diry, dirz;
 };
@@ -266,7 +266,7 @@ __device__ __forceinline__ Geo project(const float mu[3], const float ls[3], con
   const float det = cov_det(N, a, c);
   if (!(det > 0.f) || !finite_f(det)) return g;
   const float idet = 1.f / det;
-  const float tau = 2.f * logf(255.f * o);
+  const float tau = footprint_tau(o);
   const float ex = __fmul_rn(sqrtf(tau * a), kExtentPad), ey = __fmul_rn(sqrtf(tau * c), kExtentPad);
   const float u = fmaf(cam.fx, rx, cam.cx), v = fmaf(cam.fy, ry, cam.cy);
   if (!finite_f(u) || !finite_f(v) || !finite_f(ex) || !finite_f(ey)) return g;
@@ -276,7 +276,7 @@ __device__ __forceinline__ Geo project(const float mu[3], const float ls[3], con
   // cancellation even for needle-like splats): l22 = 1/sqrt(c), l11 = sqrt(c/det), l21 = -b/sqrt(c det)
   const float isd = 1.f / sqrtf(det), l22 = 1.f / sqrtf(c);
   (void)idet;
-  g.u = u; g.v = v; g.A = sqrtf(c) * isd; g.B = -b * l22 * isd; g.C = l22; g.o = o; g.ex = ex; g.ey = ey;
+  g.u = u; g.v = v; g.A = sqrtf(c) * isd; g.B = -b * l22 * isd; g.C = l22; g.o = o; g.ex = ex; g.ey = ey; g.tau = tau;
   const float vx = mu[0] - cam.oc[0], vy = mu[1] - cam.oc[1], vz = mu[2] - cam.oc[2];
   const float vi = rsqrtf(vx * vx + vy * vy + vz * vz);
   g.dirx = vx * vi; g.diry = vy * vi; g.dirz = vz * vi;
@@ -329,6 +329,14 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_fwd(PreprocessArgs a, Cam
     g = project(mu, ls, q, __ldg(a.logits + i), cam);
     if (g.valid) vis = tile_rect(g.u, g.v, g.ex, g.ey, cam, rect);
   }
+  // tiles the ellipse really meets inside its bounding rectangle
+  unsigned int tiles = 0;
+  if (vis) {
+    TileSpans sp;
+    sp.setup(g.u, g.v, g.A, g.B, g.C, g.tau, cam.W, cam.H);
+    tiles = sp.count(rect[0], rect[1], rect[2], rect[3]);
+    if (tiles == 0) { vis = false; rect[0] = rect[1] = rect[2] = rect[3] = 0; }
+  }
   // ---- fused colour decode for the Gaussians that survived culling
   float pre[3] = {0.f, 0.f, 0.f};
   if (APP == GS_APP_SH) {
@@ -361,18 +369,19 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_fwd(PreprocessArgs a, Cam
       for (int c = 0; c < 3; ++c) pre[c] = base[c] + 0.5f + A[c];
     }
   }
-  unsigned int tiles = 0;
   if (in) {
-    if (g.valid) reinterpret_cast<float2 *>(a.mean2d)[i] = make_float2(g.u, g.v);
-    if (vis) {
+    if (g.valid) {   // also for footprints that reach no tile: the tile stage is checked from these values
+      reinterpret_cast<float2 *>(a.mean2d)[i] = make_float2(g.u, g.v);
       reinterpret_cast<float4 *>(a.conic_opacity)[i] = make_float4(g.A, g.B, g.C, g.o);
+    }
+    if (vis) {
       a.color[3 * i] = fmaxf(pre[0], 0.f); a.color[3 * i + 1] = fmaxf(pre[1], 0.f); a.color[3 * i + 2] = fmaxf(pre[2], 0.f);
-      tiles = (unsigned)((rect[2] - rect[0]) * (rect[3] - rect[1]));
     }
     a.depth_key[i] = vis ? g.zbits : 0xffffffffu;
+    a.tiles_touched[i] = tiles;
     reinterpret_cast<ushort4 *>(a.rect)[i] = make_ushort4((unsigned short)rect[0], (unsigned short)rect[1],
                                                           (unsigned short)rect[2], (unsigned short)rect[3]);
-    if (a.extent) reinterpret_cast<float2 *>(a.extent)[i] = g.valid ? make_float2(g.ex, g.ey) : make_float2(-1.f, -1.f);
+    if (a.extent) reinterpret_cast<float4 *>(a.extent)[i] = g.valid ? make_float4(g.ex, g.ey, g.tau, 0.f) : make_float4(-1.f, -1.f, 0.f, 0.f);
   }
   // ---- total number of (Gaussian, tile) instances
 #pragma unroll

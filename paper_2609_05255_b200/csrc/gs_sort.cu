@@ -194,17 +194,12 @@ __global__ void __launch_bounds__(kSortThreads, 3) k_radix_scatter(
 // ---- tiles touched in depth order -----------------------------------------------------------
 constexpr int kScanBlock = 256;
 
-__device__ __forceinline__ uint32_t tiles_of(const uint16_t *rect, uint32_t g) {
-  const ushort4 r = __ldg(reinterpret_cast<const ushort4 *>(rect) + g);
-  return (uint32_t)(r.z - r.x) * (uint32_t)(r.w - r.y);
-}
-
 __global__ void __launch_bounds__(kScanBlock) k_tiles_block_sums(const uint32_t *__restrict__ order,
-                                                                 const uint16_t *__restrict__ rect, int64_t n,
+                                                                 const uint32_t *__restrict__ tiles_touched, int64_t n,
                                                                  uint32_t *__restrict__ block_sums) {
   __shared__ uint32_t s_w[kScanBlock / 32];
   const int64_t i = (int64_t)blockIdx.x * kScanBlock + threadIdx.x;
-  uint32_t v = i < n ? tiles_of(rect, __ldg(order + i)) : 0u;
+  uint32_t v = i < n ? __ldg(tiles_touched + __ldg(order + i)) : 0u;
 #pragma unroll
   for (int s = 16; s > 0; s >>= 1) v += __shfl_xor_sync(kFull, v, s);
   if ((threadIdx.x & 31) == 0) s_w[threadIdx.x >> 5] = v;
@@ -253,21 +248,34 @@ __global__ void __launch_bounds__(1024) k_scan_single_block(uint32_t *__restrict
   }
 }
 
-// Emit the instances of each Gaussian, in depth order: tile ids ty-major then tx.  Small rects
-// are written by their own thread; large ones by the whole warp.
+// Emit the instances of each Gaussian, in depth order: the tiles its alpha >= 1/255 ellipse meets
+// (TileSpans, the same function the preprocess counted with), tile rows top to bottom, tiles left
+// to right.  Small footprints are written by their own thread; large ones by the whole warp.
 __global__ void __launch_bounds__(kScanBlock) k_keygen(const uint32_t *__restrict__ order, const uint16_t *__restrict__ rect,
+                                                       const float *__restrict__ mean2d,
+                                                       const float *__restrict__ conic_opacity,
+                                                       const uint32_t *__restrict__ tiles_touched,
                                                        const uint32_t *__restrict__ block_offsets, int64_t n, int gx,
-                                                       uint32_t *__restrict__ inst_tiles, uint32_t *__restrict__ inst_vals) {
+                                                       int W, int H, uint32_t *__restrict__ inst_tiles,
+                                                       uint32_t *__restrict__ inst_vals) {
   __shared__ uint32_t s_w[kScanBlock / 32];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int64_t i = (int64_t)blockIdx.x * kScanBlock + tid;
-  uint32_t g = 0;
+  uint32_t g = 0, tiles = 0;
   ushort4 r = make_ushort4(0, 0, 0, 0);
+  float4 sp0 = make_float4(0.f, 0.f, 1.f, 0.f);   // u, v, la, lb
+  float2 sp1 = make_float2(1.f, 0.f);             // lc, tau
   if (i < n) {
     g = __ldg(order + i);
-    r = __ldg(reinterpret_cast<const ushort4 *>(rect) + g);
+    tiles = __ldg(tiles_touched + g);
+    if (tiles) {
+      r = __ldg(reinterpret_cast<const ushort4 *>(rect) + g);
+      const float2 m = __ldg(reinterpret_cast<const float2 *>(mean2d) + g);
+      const float4 q = __ldg(reinterpret_cast<const float4 *>(conic_opacity) + g);
+      sp0 = make_float4(m.x, m.y, q.x, q.y);
+      sp1 = make_float2(q.z, footprint_tau(q.w));
+    }
   }
-  const uint32_t w = (uint32_t)(r.z - r.x), tiles = w * (uint32_t)(r.w - r.y);
   uint32_t inc = tiles;
 #pragma unroll
   for (int s = 1; s < 32; s <<= 1) {
@@ -280,27 +288,53 @@ __global__ void __launch_bounds__(kScanBlock) k_keygen(const uint32_t *__restric
 #pragma unroll
   for (int k = 0; k < kScanBlock / 32; ++k) off += (k < warp) ? s_w[k] : 0u;
   off += inc - tiles;
-  constexpr uint32_t kSmall = 8;
+  constexpr uint32_t kSmall = 32;
   if (tiles > 0 && tiles <= kSmall) {
+    TileSpans sp;
+    sp.setup(sp0.x, sp0.y, sp0.z, sp0.w, sp1.x, sp1.y, W, H);
     uint32_t p = off;
-    for (uint32_t ty = r.y; ty < r.w; ++ty)
-      for (uint32_t tx = r.x; tx < r.z; ++tx) {
-        inst_tiles[p] = ty * gx + tx;
+    for (int ty = r.y; ty < (int)r.w; ++ty) {
+      int xa, xb;
+      if (!sp.row(ty, r.x, r.z, xa, xb)) continue;
+      for (int tx = xa; tx < xb; ++tx) {
+        inst_tiles[p] = (uint32_t)(ty * gx + tx);
         inst_vals[p] = g;
         ++p;
       }
+    }
   }
+  // a large footprint is shared by the warp: one tile row per lane, then the tiles of each row
   uint32_t big = __ballot_sync(kFull, tiles > kSmall);
   while (big) {
     const int src = __ffs(big) - 1;
     big &= big - 1;
-    const uint32_t s_off = __shfl_sync(kFull, off, src), s_tiles = __shfl_sync(kFull, tiles, src);
-    const uint32_t s_w_ = __shfl_sync(kFull, w, src), s_g = __shfl_sync(kFull, g, src);
-    const uint32_t s_x0 = __shfl_sync(kFull, (uint32_t)r.x, src), s_y0 = __shfl_sync(kFull, (uint32_t)r.y, src);
-    for (uint32_t k = lane; k < s_tiles; k += 32) {
-      const uint32_t ty = s_y0 + k / s_w_, tx = s_x0 + k % s_w_;
-      inst_tiles[s_off + k] = ty * gx + tx;
-      inst_vals[s_off + k] = s_g;
+    TileSpans sp;
+    sp.setup(__shfl_sync(kFull, sp0.x, src), __shfl_sync(kFull, sp0.y, src), __shfl_sync(kFull, sp0.z, src),
+             __shfl_sync(kFull, sp0.w, src), __shfl_sync(kFull, sp1.x, src), __shfl_sync(kFull, sp1.y, src), W, H);
+    uint32_t p = __shfl_sync(kFull, off, src);
+    const uint32_t s_g = __shfl_sync(kFull, g, src);
+    const int x0 = (int)__shfl_sync(kFull, (uint32_t)r.x, src), x1 = (int)__shfl_sync(kFull, (uint32_t)r.z, src);
+    const int y0 = (int)__shfl_sync(kFull, (uint32_t)r.y, src), y1 = (int)__shfl_sync(kFull, (uint32_t)r.w, src);
+    for (int tyb = y0; tyb < y1; tyb += 32) {
+      int xa = 0, xb = 0;
+      if (tyb + lane < y1 && !sp.row(tyb + lane, x0, x1, xa, xb)) xa = xb = 0;
+      uint32_t incl = (uint32_t)(xb - xa);
+#pragma unroll
+      for (int s = 1; s < 32; s <<= 1) {
+        const uint32_t t = __shfl_up_sync(kFull, incl, s);
+        if (lane >= s) incl += t;
+      }
+      const uint32_t excl = incl - (uint32_t)(xb - xa);
+      const int rows = min(32, y1 - tyb);
+      for (int rr = 0; rr < rows; ++rr) {
+        const int a = __shfl_sync(kFull, xa, rr), b = __shfl_sync(kFull, xb, rr);
+        const uint32_t o = p + __shfl_sync(kFull, excl, rr);
+        for (int tx = a + lane; tx < b; tx += 32) {
+          inst_tiles[o + (uint32_t)(tx - a)] = (uint32_t)((tyb + rr) * gx + tx);
+          inst_vals[o + (uint32_t)(tx - a)] = s_g;
+        }
+      }
+      p += __shfl_sync(kFull, incl, 31);
     }
   }
 }
@@ -367,20 +401,22 @@ int launch_radix_sort(const uint32_t *keys_in, const uint32_t *vals_in, uint32_t
 
 size_t scan_scratch_bytes(int64_t n) { return (size_t)((n + kScanBlock - 1) / kScanBlock + 1) * sizeof(uint32_t); }
 
-int launch_tile_offsets(const uint32_t *depth_order, const uint16_t *rect, uint32_t *block_offsets, int64_t n,
+int launch_tile_offsets(const uint32_t *depth_order, const uint32_t *tiles_touched, uint32_t *block_offsets, int64_t n,
                         void *, cudaStream_t st) {
   if (n <= 0) return 0;
   const int blocks = (int)((n + kScanBlock - 1) / kScanBlock);
-  k_tiles_block_sums<<<blocks, kScanBlock, 0, st>>>(depth_order, rect, n, block_offsets);
+  k_tiles_block_sums<<<blocks, kScanBlock, 0, st>>>(depth_order, tiles_touched, n, block_offsets);
   k_scan_single_block<<<1, 1024, 0, st>>>(block_offsets, blocks);
   return 2;
 }
 
-int launch_keygen(const uint32_t *depth_order, const uint16_t *rect, const uint32_t *block_offsets,
-                  uint32_t *inst_tiles, uint32_t *inst_vals, int64_t n, int gx, cudaStream_t st) {
+int launch_keygen(const uint32_t *depth_order, const uint16_t *rect, const float *mean2d, const float *conic_opacity,
+                  const uint32_t *tiles_touched, const uint32_t *block_offsets, uint32_t *inst_tiles, uint32_t *inst_vals,
+                  int64_t n, int gx, int W, int H, cudaStream_t st) {
   if (n <= 0) return 0;
   const int blocks = (int)((n + kScanBlock - 1) / kScanBlock);
-  k_keygen<<<blocks, kScanBlock, 0, st>>>(depth_order, rect, block_offsets, n, gx, inst_tiles, inst_vals);
+  k_keygen<<<blocks, kScanBlock, 0, st>>>(depth_order, rect, mean2d, conic_opacity, tiles_touched, block_offsets, n, gx, W, H,
+                                          inst_tiles, inst_vals);
   return 1;
 }
 

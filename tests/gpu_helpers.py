@@ -59,13 +59,13 @@ def run_gpu(scene, cam, G=None, pair_capacity=None, with_extent=True, device=0):
     u32 = lambda t: t.cpu().numpy().view(np.uint32)
     out = SimpleNamespace(
         P=P, n=n, mean2d=proj.mean2d.cpu().numpy()[:n], conic_opacity=_conic_from_cholesky(proj.conic_opacity.cpu().numpy()[:n]),
+        chol=proj.conic_opacity.cpu().numpy()[:n, :3].copy(), tiles_touched=u32(proj.tiles_touched)[:n],
         color=proj.color.cpu().numpy()[:n], depth_key=u32(proj.depth_key)[:n],
         rect=proj.rect.cpu().numpy().view(np.uint16)[:n].astype(np.int32),
         extent=proj.extent.cpu().numpy()[:n] if with_extent else None,
         depth_order=u32(binning.depth_order)[:n], sorted_tiles=u32(binning.sorted_tiles)[:P],
         sorted_vals=u32(binning.sorted_vals)[:P], tile_ranges=u32(binning.tile_ranges),
         image=image.cpu().numpy(), final_T=final_T.cpu().numpy(), n_contrib=u32(n_contrib), grads=None, g2d=None)
-    out.tiles_touched = ((out.rect[:, 2] - out.rect[:, 0]) * (out.rect[:, 3] - out.rect[:, 1])).astype(np.uint32)
     out.visible = out.tiles_touched > 0
     if G is not None:
         g = api.alloc_grads(n, ds.app, dev)

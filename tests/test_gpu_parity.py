@@ -66,7 +66,7 @@ def test_per_gaussian_floats(results, name):
     val = gpu.extent[:, 0] >= 0
     assert np.array_equal(val, pre.valid.astype(bool)) or (val != pre.valid.astype(bool)).sum() <= 2
     vb = val & pre.valid.astype(bool)
-    rel = gpu.extent[vb] / np.maximum(pre.extent[vb], 1e-12) - 1
+    rel = gpu.extent[vb, :2] / np.maximum(pre.extent[vb], 1e-12) - 1
     assert rel.min() > -1e-6 and rel.max() < 3e-5
 
 
@@ -79,7 +79,7 @@ def test_integer_stage_bit_exact(results, oracle, name):
     assert np.all(gpu.depth_key[~vis] == 0xFFFFFFFF)
     # rects from the GPU's own fp32 centre and extent
     valid = gpu.extent[:, 0] >= 0
-    rect, tt, P = oracle.tile_rects_f32(valid, gpu.mean2d, gpu.extent, cam.width, cam.height)
+    rect, tt, P = oracle.tile_spans_f32(valid, gpu.mean2d, gpu.chol, gpu.extent, cam.width, cam.height)
     assert np.array_equal(rect, gpu.rect)
     assert P == gpu.P and np.array_equal(tt, gpu.tiles_touched)
     # depth order of the visible Gaussians: (depth key, index) ascending
@@ -88,7 +88,8 @@ def test_integer_stage_bit_exact(results, oracle, name):
     order = ids[np.argsort(gpu.depth_key[ids], kind="stable")]
     assert np.array_equal(gpu.depth_order[:V], order.astype(np.uint32))
     # sorted instances and ranges
-    keys, vals, ranges = oracle.sorted_instances(rect, np.where(vis, gpu.depth_key, 0), cam.width, cam.height, P)
+    keys, vals, ranges = oracle.sorted_instances_f32(rect, tt, gpu.mean2d, gpu.chol, gpu.extent,
+                                                     np.where(vis, gpu.depth_key, 0), cam.width, cam.height, P)
     gpu_keys = (gpu.sorted_tiles.astype(np.uint64) << np.uint64(32)) | gpu.depth_key[gpu.sorted_vals].astype(np.uint64)
     assert np.array_equal(gpu.sorted_vals, vals)
     assert np.array_equal(gpu_keys, keys)

@@ -393,15 +393,37 @@ def test_alpha_clamp_and_early_stop(oracle):
     assert fwd.n_contrib[8, 8] == 2 and abs(fwd.final_T[8, 8] - 1e-4) < 1e-15
 
 
-def _instances_by_definition(fwd, cam):
-    """(tile, depth_bits, index) triples straight from the per-Gaussian pixel rects."""
-    gx = (cam.width + 15) // 16
+def _min_quadratic_over_box(A, B, C, x0, x1, y0, y1):
+    """min of A x^2 + 2 B x y + C y^2 over the box [x0,x1] x [y0,y1] (coordinates relative to the
+    centre), by the textbook case split: the origin if inside, else the best of the four edges."""
+    if x0 <= 0 <= x1 and y0 <= 0 <= y1:
+        return 0.0
+    best = math.inf
+    for y in (y0, y1):                      # horizontal edges: minimise over x, clamp
+        x = min(max(-B * y / A, x0), x1)
+        best = min(best, A * x * x + 2 * B * x * y + C * y * y)
+    for x in (x0, x1):                      # vertical edges
+        y = min(max(-B * x / C, y0), y1)
+        best = min(best, A * x * x + 2 * B * x * y + C * y * y)
+    return best
+
+
+def _instances_by_definition(fwd, cam, slack):
+    """(tile, depth_bits, index) for every tile whose box of pixel centres the alpha >= 1/255 ellipse
+    (conic form <= tau (1 + slack)) meets, straight from that definition."""
+    gx, gy = (cam.width + 15) // 16, (cam.height + 15) // 16
+    pre = fwd.pre
     out = []
-    for g in np.nonzero(fwd.pre.visible)[0]:
-        i0, i1, j0, j1 = fwd.pre.rect_px[g]
-        for ty in range(j0 // 16, j1 // 16 + 1):
-            for tx in range(i0 // 16, i1 // 16 + 1):
-                out.append((ty * gx + tx, int(fwd.pre.depth_bits[g]), int(g)))
+    for g in np.nonzero(pre.valid)[0]:
+        A, B, C = pre.conic[g]
+        u, v = pre.mean2d[g]
+        tau = 2 * math.log(255 * pre.opacity[g]) * (1 + slack)
+        for ty in range(gy):
+            for tx in range(gx):
+                x0, x1 = 16 * tx + 0.5 - u, min(16 * tx + 15.5, cam.width - 0.5) - u
+                y0, y1 = 16 * ty + 0.5 - v, min(16 * ty + 15.5, cam.height - 0.5) - v
+                if _min_quadratic_over_box(A, B, C, x0, x1, y0, y1) <= tau:
+                    out.append((ty * gx + tx, int(pre.depth_bits[g]), int(g)))
     return sorted(out)
 
 
@@ -409,12 +431,25 @@ def test_tiles_sort_and_ranges_by_brute_force(oracle):
     w = scenes.config1(400)
     cam = w.cameras[0]
     fwd, _ = oracle.render(w.scene, cam)
-    ref = _instances_by_definition(fwd, cam)
-    assert fwd.P == len(ref)
     got = [(int(k >> np.uint64(32)), int(k & np.uint64(0xFFFFFFFF)), int(v)) for k, v in zip(fwd.keys, fwd.vals)]
-    assert got == ref
+    assert fwd.P == len(got) and got == sorted(got)
+    # lower bound: every tile that holds a pixel centre inside the ellipse (those are the pairs that
+    # can blend); upper bound: every tile whose box of pixel centres the ellipse, padded by 5e-5 in
+    # tau, meets at all (the span rule may drop a tile the ellipse only grazes between pixel centres)
+    pre, gx = fwd.pre, (cam.width + 15) // 16
+    ii, jj = np.meshgrid(np.arange(cam.width) + 0.5, np.arange(cam.height) + 0.5)
+    must = set()
+    for g in np.nonzero(pre.valid)[0]:
+        dx, dy = ii - pre.mean2d[g, 0], jj - pre.mean2d[g, 1]
+        A, B, C = pre.conic[g]
+        ys, xs = np.nonzero(A * dx * dx + 2 * B * dx * dy + C * dy * dy <= 2 * math.log(255 * pre.opacity[g]))
+        must |= {((y // 16) * gx + x // 16, int(pre.depth_bits[g]), int(g)) for y, x in zip(ys.tolist(), xs.tolist())}
+    may = set(_instances_by_definition(fwd, cam, 5e-5))
+    assert len(must) > 500 and must <= set(got) <= may
+    assert len(may) - len(got) <= 0.02 * len(got)       # ... and it drops few of those
+    assert len(got) < 0.99 * int(((fwd.rect[:, 2] - fwd.rect[:, 0]) * (fwd.rect[:, 3] - fwd.rect[:, 1])).sum())
     # ranges partition [0, P) and every instance lies inside its tile's range
-    tiles = np.array([t for t, _, _ in ref])
+    tiles = np.array([t for t, _, _ in got])
     for t in range(fwd.ranges.shape[0]):
         s, e = fwd.ranges[t]
         assert np.all(tiles[s:e] == t)
@@ -462,12 +497,15 @@ def test_blend_invariants(oracle):
     assert np.all(fwd.image <= fwd.color.max() * (1 - fwd.final_T)[None] + 1e-12)
 
 
-def test_integer_stage_f32_agrees_with_double_rects(oracle):
+def test_integer_stage_f32_agrees_with_double(oracle):
     w = scenes.config1()
     cam = w.cameras[0]
     fwd, _ = oracle.render(w.scene, cam)
     pre = fwd.pre
-    rect, tt, P = oracle.tile_rects_f32(pre.valid, pre.mean2d.astype(np.float32),
-                                        pre.extent.astype(np.float32), cam.width, cam.height)
-    assert (tt != fwd.tiles_touched).sum() <= 2      # fp32 rounding may flip a box edge, rarely
-    assert abs(P - fwd.P) <= 4
+    f32 = lambda a: a.astype(np.float32)
+    rect, tt, P = oracle.tile_spans_f32(pre.valid, f32(pre.mean2d), f32(pre.chol), f32(pre.ext), cam.width, cam.height)
+    assert (tt != fwd.tiles_touched).sum() <= 3      # fp32 rounding may flip a tile at a box edge, rarely
+    assert abs(P - fwd.P) <= 6
+    keys, vals, ranges = oracle.sorted_instances_f32(rect, tt, f32(pre.mean2d), f32(pre.chol), f32(pre.ext),
+                                                     pre.depth_bits, cam.width, cam.height, P)
+    assert len(vals) == P and np.all(np.diff(keys.astype(np.int64) >> 32) >= 0)
