@@ -196,7 +196,7 @@ def run_ours(args):
             visible += int(((rect[:, 2] > rect[:, 0]) & (rect[:, 3] > rect[:, 1])).sum().item())
         results[tag] = dict(ms=ms, stage_ms=stage_ms, stage_launches=stage_launches, pairs=pairs,
                             entries=entries, visible=visible, evaluated=evaluated, composited=composited,
-                            host=host, ds=ds, r=r)
+                            host=host, ds=ds, r=r, app=tag)
 
     # ---- end to end through the public API with host buffers (neural arm)
     e2e = None if args.skip_e2e else measure_e2e(api, torch, ctx, results["neural"], cams, G, views, args, timed, dev)
@@ -244,7 +244,20 @@ def run_ours(args):
     print(json.dumps(out))
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum of ONE launch (orbit view 0 of the default workload), from the
+# ncu --set full captures summarised under profiles/ (k_<kernel>_config3_neural_1M_view0.md).  Bytes.
+NCU_TRAFFIC_1M_NEURAL = {"blend_bwd": 47.37e6, "blend_fwd": 25.73e6, "preprocess_bwd": 181.99e6,
+                         "preprocess_fwd": 89.63e6}
+
+
 def stage_roofline(stage, arm, views, n, peaks, alu_peak):
+    out = _stage_roofline(stage, arm, views, n, peaks, alu_peak)
+    if n == 1_000_000 and arm.get("app") == "neural":
+        out["traffic"] = NCU_TRAFFIC_1M_NEURAL.get(stage)
+    return out
+
+
+def _stage_roofline(stage, arm, views, n, peaks, alu_peak):
     ms = arm["stage_ms"][stage] / views          # average duration of one launch of the stage
     if stage in ("blend_fwd", "blend_bwd"):
         if stage == "blend_fwd":
