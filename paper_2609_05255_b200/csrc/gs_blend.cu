@@ -125,13 +125,20 @@ __global__ void __launch_bounds__(kThreads) k_blend_fwd(CamDev cam, const uint32
   }
 }
 
-// Sum nine per-lane values over the warp with 14 shuffles instead of 45.  Values 0..7: at each of
+__device__ __forceinline__ float rcp_approx(float x) {
+  float y;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// Sum ten per-lane values over the warp with 14 shuffles instead of 50.  Values 0..7: at each of
 // the first three butterfly levels a lane keeps only the half of the values it is "responsible"
 // for and trades the other half with its partner, so the exchanged volume halves each level
 // (4 + 2 + 1 shuffles); two plain levels finish the one value left per lane.  Afterwards the
 // lanes 0, 4, .., 28 hold the totals: lane 16 * b4 + 8 * b3 + 4 * b2 owns value 4 * b4 + 2 * b3 + b2.
-// Value 8 takes a plain five-level butterfly and ends in every lane.
-__device__ __forceinline__ void warp_reduce9(const float v[9], int lane, float &mine, float &ninth) {
+// Values 8 and 9 are traded once between the half warps and then take four plain levels: every
+// lane below 16 ends with the total of value 8, every lane from 16 up with that of value 9.
+__device__ __forceinline__ void warp_reduce10(const float v[10], int lane, float &mine, float &tail) {
   float a[4], b[2], c;
   const bool hi16 = lane & 16, hi8 = lane & 8, hi4 = lane & 4;
 #pragma unroll
@@ -151,22 +158,27 @@ __device__ __forceinline__ void warp_reduce9(const float v[9], int lane, float &
   c += __shfl_xor_sync(kFull, c, 2);
   c += __shfl_xor_sync(kFull, c, 1);
   mine = c;
-  float n = v[8];
+  float t = (hi16 ? v[9] : v[8]) + __shfl_xor_sync(kFull, hi16 ? v[8] : v[9], 16);
 #pragma unroll
-  for (int s = 16; s > 0; s >>= 1) n += __shfl_xor_sync(kFull, n, s);
-  ninth = n;
+  for (int s = 8; s > 0; s >>= 1) t += __shfl_xor_sync(kFull, t, s);
+  tail = t;
 }
 
 // Backward: walk each pixel's composited entries back to front.  The transmittance in front of
 // an entry is recovered by dividing out (1 - alpha); the light arriving from behind it is summed
 // up on the way (both stay relatively accurate: a front-to-back replay that forms that light as
-// "final pixel - prefix" cancels badly for deep entries).  The nine per-Gaussian partial
-// derivatives are summed over the thread's four pixels in registers, over the warp with
-// warp_reduce9, over the tile's two warps in shared memory, and leave with one global atomic per
-// value.
-// g2d row: (d colour r, g, b, d opacity) (d conic A, B, C, d mean u) (d mean v, -, -, -).  Inside
-// the kernel the values travel as v[0..7] = (conic A, B, C, mean u, mean v, colour r, g, b) and
-// v[8] = opacity.
+// "final pixel - prefix" cancels badly for deep entries).  Only its product with the pixel's
+// upstream gradient is needed, so one scalar per pixel carries it.
+//
+// What a pixel sends to a Gaussian's conic and mean is linear in dp = dL/d(power) times
+// (1, dx, dy, dx^2, dx dy, dy^2).  The threads therefore sum the six moments of dp in tile-local
+// pixel coordinates (half-integers up to 7.5, so the products are exact), a quad of pixels at a
+// time, and the moments are shifted to the Gaussian's own centre once per (tile, Gaussian) when
+// the batch leaves shared memory.  Ten values per entry cross the warp: the six moments, the
+// colour gradient and the opacity gradient (warp_reduce10); each warp owns its own copy of the
+// batch's accumulators, so no shared-memory atomics are needed; the sums leave with one global
+// atomic per value.
+// g2d row: (d colour r, g, b, d opacity) (d conic A, B, C, d mean u) (d mean v, -, -, -).
 __global__ void __launch_bounds__(kThreads) k_blend_bwd(CamDev cam, const uint32_t *__restrict__ ranges,
                                                         const uint32_t *__restrict__ order,
                                                         const uint32_t *__restrict__ vals,
@@ -180,16 +192,20 @@ __global__ void __launch_bounds__(kThreads) k_blend_bwd(CamDev cam, const uint32
   __shared__ float2 s_co[kBatch];
   __shared__ float4 s_rgb[kBatch];
   __shared__ uint32_t s_gid[kBatch];
-  __shared__ float s_acc[kBatch][9];
+  __shared__ float s_acc[kThreads / 32][kBatch][10];
   __shared__ uint32_t s_max[2];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, tile = (int)__ldg(order + blockIdx.x);
   int px, py;
   quad_of(tile, cam.gx, tid, px, py);
   const float fx = (float)px + 0.5f, fy = (float)py + 0.5f;
+  // tile-local coordinates of the quad's pixel centres, origin at the middle of the tile
+  const float ox_tile = (float)((tile % cam.gx) * GS_TILE + GS_TILE / 2), oy_tile = (float)((tile / cam.gx) * GS_TILE + GS_TILE / 2);
+  const float X0 = fx - ox_tile, X1 = X0 + 1.f, Y0 = fy - oy_tile, Y1 = Y0 + 1.f;
+  const float XX0 = X0 * X0, XX1 = X1 * X1, YY0 = Y0 * Y0, YY1 = Y1 * Y1;
   const uint32_t start = __ldg(ranges + 2 * tile), end = __ldg(ranges + 2 * tile + 1);
   const size_t plane = (size_t)cam.W * cam.H;
   uint32_t nc[4];
-  float T[4], Gr[4], Gg[4], Gb[4], Sr[4], Sg[4], Sb[4];
+  float T[4], Gr[4], Gg[4], Gb[4], GS[4];
   uint32_t wmax = 0;
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
@@ -201,7 +217,7 @@ __global__ void __launch_bounds__(kThreads) k_blend_bwd(CamDev cam, const uint32
       T[k] = __ldg(final_T + pix);
       Gr[k] = __ldg(dL_dimage + pix); Gg[k] = __ldg(dL_dimage + plane + pix); Gb[k] = __ldg(dL_dimage + 2 * plane + pix);
     }
-    Sr[k] = T[k] * cam.bg[0]; Sg[k] = T[k] * cam.bg[1]; Sb[k] = T[k] * cam.bg[2];
+    GS[k] = T[k] * fmaf(Gb[k], cam.bg[2], fmaf(Gg[k], cam.bg[1], Gr[k] * cam.bg[0]));   // G . (light from behind)
     wmax = max(wmax, nc[k]);
   }
 #pragma unroll
@@ -210,9 +226,8 @@ __global__ void __launch_bounds__(kThreads) k_blend_bwd(CamDev cam, const uint32
   __syncthreads();
   const uint32_t maxc = max(s_max[0], s_max[1]);
   if (maxc == 0 || start + maxc > end) return;   // nothing composited in this tile
-  // column of the g2d row that this lane's reduced value belongs to (lanes 0, 4, .., 28)
+  // value that this lane holds after the reduction (lanes 0, 4, .., 28: one of 0..7; lanes 1 and 17: 8 and 9)
   const int my_value = ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1);
-  const int my_col = my_value < 5 ? my_value + 4 : my_value - 5;
   const int nbatches = (int)((maxc + kBatch - 1) / kBatch);
   for (int b = nbatches - 1; b >= 0; --b) {
     __syncthreads();
@@ -227,7 +242,7 @@ __global__ void __launch_bounds__(kThreads) k_blend_bwd(CamDev cam, const uint32
         stage_entry(g, mean2d, conic_opacity, color, s_xyab[slot], s_co[slot], s_rgb[slot]);
       }
 #pragma unroll
-      for (int k = 0; k < 9; ++k) s_acc[slot][k] = 0.f;
+      for (int k = 0; k < 10; ++k) s_acc[0][slot][k] = s_acc[1][slot][k] = 0.f;
     }
     __syncthreads();
     const int jtop = (int)min((uint32_t)cnt, wmax > first ? wmax - first : 0u);
@@ -235,45 +250,47 @@ __global__ void __launch_bounds__(kThreads) k_blend_bwd(CamDev cam, const uint32
       const uint32_t pos = first + (uint32_t)j;
       const float4 a = s_xyab[j];
       const float2 c = s_co[j];
-      const float dx0 = fx - a.x, dy0 = fy - a.y;
       float p[4], t1[4], t2[2];
-      quad_power(dx0, dy0, a.z, a.w, c.x, p, t1, t2);
+      quad_power(fx - a.x, fy - a.y, a.z, a.w, c.x, p, t1, t2);
       const float4 col = s_rgb[j];
-      float v[9];
-#pragma unroll
-      for (int k = 0; k < 9; ++k) v[k] = 0.f;
+      float dp[4] = {0.f, 0.f, 0.f, 0.f};
+      float v[10];
+      v[6] = v[7] = v[8] = v[9] = 0.f;
       bool any = false;
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
-        float e2, alpha;
-        if (pos >= nc[k] || !alpha_of(p[k], c.y, e2, alpha)) continue;
+        if (pos >= nc[k]) continue;
+        const float e2 = ex2_approx(p[k]);
+        const float raw = __fmul_rn(c.y, e2);
+        const float alpha = fminf(kAlphaMax, raw);
+        if (alpha < kAlphaMin) continue;
         any = true;
-        const float dx = dx0 + (float)(k & 1), dy = dy0 + (float)(k >> 1);
-        const float inv = __frcp_rn(1.f - alpha);
+        const float inv = rcp_approx(1.f - alpha);
         const float Tb = T[k] * inv;              // transmittance in front of this entry
         const float w = alpha * Tb;
-        v[5] = fmaf(w, Gr[k], v[5]); v[6] = fmaf(w, Gg[k], v[6]); v[7] = fmaf(w, Gb[k], v[7]);
+        v[6] = fmaf(w, Gr[k], v[6]); v[7] = fmaf(w, Gg[k], v[7]); v[8] = fmaf(w, Gb[k], v[8]);
         // d pixel / d alpha = T c - S / (1 - alpha), S = everything composited behind this entry
-        const float dalpha = Gr[k] * (Tb * col.x - Sr[k] * inv) + Gg[k] * (Tb * col.y - Sg[k] * inv) +
-                             Gb[k] * (Tb * col.z - Sb[k] * inv);
-        if (c.y * e2 <= kAlphaMax) {              // not clamped: alpha depends on o and power
-          v[8] = fmaf(e2, dalpha, v[8]);
-          const float dp = alpha * dalpha;
-          const float dp2 = dp * (2.f * kLn2);    // power = -ln2 (t1^2 + t2^2), d power / d mean = -d / d (dx, dy)
-          v[0] = fmaf(-0.5f * dx * dx, dp, v[0]);
-          v[1] = fmaf(-dx * dy, dp, v[1]);
-          v[2] = fmaf(-0.5f * dy * dy, dp, v[2]);
-          v[3] = fmaf(dp2, t1[k] * a.z, v[3]);
-          v[4] = fmaf(dp2, fmaf(t1[k], a.w, t2[k >> 1] * c.x), v[4]);
+        const float gc = fmaf(Gb[k], col.z, fmaf(Gg[k], col.y, Gr[k] * col.x));
+        const float dalpha = fmaf(T[k], gc, -GS[k]) * inv;
+        if (raw <= kAlphaMax) {                   // not clamped: alpha depends on o and power
+          v[9] = fmaf(e2, dalpha, v[9]);
+          dp[k] = alpha * dalpha;
         }
-        Sr[k] = fmaf(col.x, w, Sr[k]); Sg[k] = fmaf(col.y, w, Sg[k]); Sb[k] = fmaf(col.z, w, Sb[k]);
+        GS[k] = fmaf(w, gc, GS[k]);
         T[k] = Tb;
       }
       if (__any_sync(kFull, any)) {
-        float mine, ninth;
-        warp_reduce9(v, lane, mine, ninth);
-        if ((lane & 3) == 0) atomicAdd(&s_acc[j][my_col], mine);
-        if (lane == 1) atomicAdd(&s_acc[j][3], ninth);
+        const float sL = dp[0] + dp[2], sR = dp[1] + dp[3], sT = dp[0] + dp[1], sB = dp[2] + dp[3];
+        v[0] = sL + sR;
+        v[1] = fmaf(X0, sL, X1 * sR);
+        v[2] = fmaf(Y0, sT, Y1 * sB);
+        v[3] = fmaf(XX0, sL, XX1 * sR);
+        v[4] = fmaf(X0, fmaf(Y0, dp[0], Y1 * dp[2]), X1 * fmaf(Y0, dp[1], Y1 * dp[3]));
+        v[5] = fmaf(YY0, sT, YY1 * sB);
+        float mine, tail;
+        warp_reduce10(v, lane, mine, tail);
+        if ((lane & 3) == 0) s_acc[warp][j][my_value] = mine;
+        if ((lane & 15) == 1) s_acc[warp][j][8 + (lane >> 4)] = tail;
       }
     }
     __syncthreads();
@@ -281,13 +298,28 @@ __global__ void __launch_bounds__(kThreads) k_blend_bwd(CamDev cam, const uint32
     for (int h = 0; h < kBatch / kThreads; ++h) {
       const int slot = tid + h * kThreads;
       if (slot < cnt) {
-        float *dst = g2d + (size_t)s_gid[slot] * 12;
+        float M[10];
         bool touched = false;
 #pragma unroll
-        for (int k = 0; k < 9; ++k) touched = touched || (s_acc[slot][k] != 0.f);
+        for (int k = 0; k < 10; ++k) {
+          M[k] = s_acc[0][slot][k] + s_acc[1][slot][k];
+          touched = touched || (M[k] != 0.f);
+        }
         if (touched) {
-#pragma unroll
-          for (int k = 0; k < 9; ++k) atomicAdd(dst + k, s_acc[slot][k]);
+          // moments about the Gaussian's centre from the tile-local ones: d = (X + ox, Y + oy)
+          const float4 a = s_xyab[slot];
+          const float lc = s_co[slot].x;
+          const float ox = ox_tile - a.x, oy = oy_tile - a.y;
+          const float sx = fmaf(ox, M[0], M[1]), sy = fmaf(oy, M[0], M[2]);
+          const float sxx = fmaf(ox, M[1] + sx, M[3]);
+          const float sxy = fmaf(oy, sx, fmaf(ox, M[2], M[4]));
+          const float syy = fmaf(oy, M[2] + sy, M[5]);
+          // the staged factor is the conic's Cholesky factor times sqrt(0.5 log2 e)
+          const float A = 2.f * kLn2 * a.z * a.z, B = 2.f * kLn2 * a.z * a.w, C = 2.f * kLn2 * fmaf(a.w, a.w, lc * lc);
+          float *dst = g2d + (size_t)s_gid[slot] * 12;
+          atomicAdd(dst + 0, M[6]); atomicAdd(dst + 1, M[7]); atomicAdd(dst + 2, M[8]); atomicAdd(dst + 3, M[9]);
+          atomicAdd(dst + 4, -0.5f * sxx); atomicAdd(dst + 5, -sxy); atomicAdd(dst + 6, -0.5f * syy);
+          atomicAdd(dst + 7, fmaf(A, sx, B * sy)); atomicAdd(dst + 8, fmaf(B, sx, C * sy));
         }
       }
     }
