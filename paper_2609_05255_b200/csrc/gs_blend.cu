@@ -41,14 +41,18 @@ __device__ __forceinline__ void stage_entry(uint32_t g, const float *mean2d, con
 // t1[k] = la dx + lb dy is returned too: the backward needs it for the gradient of the mean.
 __device__ __forceinline__ void quad_power(float dx0, float dy0, float la, float lb, float lc, float p[4],
                                            float t1[4], float t2[2]) {
-  const float dx1 = __fadd_rn(dx0, 1.f), dy1 = __fadd_rn(dy0, 1.f);
-  const float a0 = __fmul_rn(la, dx0), a1 = __fmul_rn(la, dx1);
-  t2[0] = __fmul_rn(lc, dy0); t2[1] = __fmul_rn(lc, dy1);
-  const float s0 = __fmul_rn(t2[0], t2[0]), s1 = __fmul_rn(t2[1], t2[1]);
-  t1[0] = __fmaf_rn(lb, dy0, a0); t1[1] = __fmaf_rn(lb, dy0, a1);
-  t1[2] = __fmaf_rn(lb, dy1, a0); t1[3] = __fmaf_rn(lb, dy1, a1);
-  p[0] = -__fmaf_rn(t1[0], t1[0], s0); p[1] = -__fmaf_rn(t1[1], t1[1], s0);
-  p[2] = -__fmaf_rn(t1[2], t1[2], s1); p[3] = -__fmaf_rn(t1[3], t1[3], s1);
+  // packed fp32 pairs (one instruction, two IEEE operations): the bits equal the scalar sequence
+  const float2 one = make_float2(1.f, 1.f);
+  const float2 d1 = __fadd2_rn(make_float2(dx0, dy0), one);            // (dx1, dy1)
+  const float2 a = __fmul2_rn(make_float2(la, la), make_float2(dx0, d1.x));
+  const float2 c = __fmul2_rn(make_float2(lc, lc), make_float2(dy0, d1.y));
+  const float2 s = __fmul2_rn(c, c);
+  const float2 lb2 = make_float2(lb, lb);
+  const float2 u = __ffma2_rn(lb2, make_float2(dy0, dy0), a), w = __ffma2_rn(lb2, make_float2(d1.y, d1.y), a);
+  const float2 pu = __ffma2_rn(u, u, make_float2(s.x, s.x)), pw = __ffma2_rn(w, w, make_float2(s.y, s.y));
+  t2[0] = c.x; t2[1] = c.y;
+  t1[0] = u.x; t1[1] = u.y; t1[2] = w.x; t1[3] = w.y;
+  p[0] = -pu.x; p[1] = -pu.y; p[2] = -pw.x; p[3] = -pw.y;
 }
 
 // alpha of one pixel from its log2 falloff; false if the pair is skipped.
