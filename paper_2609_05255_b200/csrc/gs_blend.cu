@@ -10,6 +10,7 @@ namespace {
 
 constexpr int kThreads = 64;
 constexpr int kBatch = 128;
+constexpr int kBatchBwd = 64;   // the backward keeps ten accumulators per entry and warp in shared memory
 constexpr unsigned kFull = 0xffffffffu;
 constexpr float kLn2 = 0.6931471805599453f;
 
@@ -183,7 +184,7 @@ __device__ __forceinline__ void warp_reduce10(const float v[10], int lane, float
 // batch's accumulators, so no shared-memory atomics are needed; the sums leave with one global
 // atomic per value.
 // g2d row: (d colour r, g, b, d opacity) (d conic A, B, C, d mean u) (d mean v, -, -, -).
-__global__ void __launch_bounds__(kThreads) k_blend_bwd(CamDev cam, const uint32_t *__restrict__ ranges,
+__global__ void __launch_bounds__(kThreads, 16) k_blend_bwd(CamDev cam, const uint32_t *__restrict__ ranges,
                                                         const uint32_t *__restrict__ order,
                                                         const uint32_t *__restrict__ vals,
                                                         const float *__restrict__ mean2d,
@@ -192,11 +193,11 @@ __global__ void __launch_bounds__(kThreads) k_blend_bwd(CamDev cam, const uint32
                                                         const float *__restrict__ final_T,
                                                         const uint32_t *__restrict__ n_contrib,
                                                         const float *__restrict__ dL_dimage, float *__restrict__ g2d) {
-  __shared__ float4 s_xyab[kBatch];
-  __shared__ float2 s_co[kBatch];
-  __shared__ float4 s_rgb[kBatch];
-  __shared__ uint32_t s_gid[kBatch];
-  __shared__ float s_acc[kThreads / 32][kBatch][10];
+  __shared__ float4 s_xyab[kBatchBwd];
+  __shared__ float2 s_co[kBatchBwd];
+  __shared__ float4 s_rgb[kBatchBwd];
+  __shared__ uint32_t s_gid[kBatchBwd];
+  __shared__ float s_acc[kThreads / 32][kBatchBwd][10];
   __shared__ uint32_t s_max[2];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, tile = (int)__ldg(order + blockIdx.x);
   int px, py;
@@ -232,13 +233,13 @@ __global__ void __launch_bounds__(kThreads) k_blend_bwd(CamDev cam, const uint32
   if (maxc == 0 || start + maxc > end) return;   // nothing composited in this tile
   // value that this lane holds after the reduction (lanes 0, 4, .., 28: one of 0..7; lanes 1 and 17: 8 and 9)
   const int my_value = ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1);
-  const int nbatches = (int)((maxc + kBatch - 1) / kBatch);
+  const int nbatches = (int)((maxc + kBatchBwd - 1) / kBatchBwd);
   for (int b = nbatches - 1; b >= 0; --b) {
     __syncthreads();
-    const uint32_t first = (uint32_t)b * kBatch;
-    const int cnt = (int)min((uint32_t)kBatch, maxc - first);
+    const uint32_t first = (uint32_t)b * kBatchBwd;
+    const int cnt = (int)min((uint32_t)kBatchBwd, maxc - first);
 #pragma unroll
-    for (int h = 0; h < kBatch / kThreads; ++h) {
+    for (int h = 0; h < kBatchBwd / kThreads; ++h) {
       const int slot = tid + h * kThreads;
       if (slot < cnt) {
         const uint32_t g = __ldg(vals + start + first + slot);
@@ -299,7 +300,7 @@ __global__ void __launch_bounds__(kThreads) k_blend_bwd(CamDev cam, const uint32
     }
     __syncthreads();
 #pragma unroll
-    for (int h = 0; h < kBatch / kThreads; ++h) {
+    for (int h = 0; h < kBatchBwd / kThreads; ++h) {
       const int slot = tid + h * kThreads;
       if (slot < cnt) {
         float M[10];
