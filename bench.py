@@ -97,6 +97,35 @@ def dist_setup(args):
     return replicas.rank_env()
 
 
+def workload_of(args, scenes):
+    """The seeded synthetic workload of --config: name, sizes, cameras, a scene factory per appearance model
+    and the arms timed (the first one carries the headline numbers)."""
+    c = args.config
+    if c == 3:
+        n, views = args.n or N_GAUSS, args.views or VIEWS
+        return dict(name=f"config3: {n} Gaussians (64 clusters + shell), {WIDTH}x{HEIGHT}, {views} orbit views, "
+                         "neural appearance (8 fp16 features + shared 32-16-16-3 MLP) with SH degree 3 beside it, fwd+bwd",
+                    n=n, views=views, width=WIDTH, height=HEIGHT, cams=scenes.orbit_cameras(WIDTH, HEIGHT, views),
+                    scene=lambda app: scenes.config3(app, n=n, width=WIDTH, height=HEIGHT, views=views).scene,
+                    arms=[(scenes.APP_NEURAL, "neural"), (scenes.APP_SH, "sh")])
+    if c == 1:
+        w = scenes.config1()
+        return dict(name="config1: 1000 Gaussians in a box, 64x64, identity camera, SH degree 3, fwd+bwd",
+                    n=w.scene.n, views=1, width=64, height=64, cams=w.cameras, scene=lambda app: w.scene,
+                    arms=[(scenes.APP_SH, "sh")])
+    if c == 2:
+        w = scenes.config2()
+        return dict(name="config2: 100k Gaussians in a box, 512x512, identity camera, neural appearance, fwd+bwd",
+                    n=w.scene.n, views=1, width=512, height=512, cams=w.cameras, scene=lambda app: w.scene,
+                    arms=[(scenes.APP_NEURAL, "neural")])
+    views = args.views or 16
+    w = scenes.config4(views=views)
+    return dict(name=f"config4: 3M Gaussians (256 clusters, depths 1-50, + shell), 1920x1080, {views} orbit views, "
+                     "neural appearance, fwd+bwd",
+                n=w.scene.n, views=views, width=1920, height=1080, cams=w.cameras, scene=lambda app: w.scene,
+                arms=[(scenes.APP_NEURAL, "neural")])
+
+
 # ---------------------------------------------------------------------------------------------
 # our arm
 # ---------------------------------------------------------------------------------------------
@@ -111,12 +140,12 @@ def run_ours(args):
     dist = replicas.init_process_group("nccl", world, dev)
     peaks = measured_peaks()
     ctx = api.Context(local)
-    n, views = args.n, args.views
-    cams_host = scenes.orbit_cameras(WIDTH, HEIGHT, views)
+    wl = workload_of(args, scenes)
+    n, views, WIDTH, HEIGHT, cams_host = wl["n"], wl["views"], wl["width"], wl["height"], wl["cams"]
     cams = [api.make_camera(c) for c in cams_host]
 
     def make_arm(app):
-        host = scenes.config3(app, n=n, width=WIDTH, height=HEIGHT, views=views).scene
+        host = wl["scene"](app)
         ds = api.upload_scene(host, dev)
         probe = api.alloc_projected(ds.n, dev, with_extent=False)
         pairs = [api.gs_preprocess(ctx, ds, c, probe) for c in cams]
@@ -126,6 +155,7 @@ def run_ours(args):
 
     gen = torch.Generator(device=dev); gen.manual_seed(4242 + rank)
     G = torch.randn((views, 3, HEIGHT, WIDTH), device=dev, generator=gen)
+    head = wl["arms"][0][1]                     # the arm the headline numbers are quoted on
 
     def step(ds, r):
         for v in range(views):
@@ -164,14 +194,14 @@ def run_ours(args):
     results = {}
     sampler = ClockSampler(local)
     clocks = None
-    arms = [(scenes.APP_NEURAL, "neural")] + ([] if args.skip_sh else [(scenes.APP_SH, "sh")])
+    arms = [a for a in wl["arms"] if not (args.skip_sh and a[1] == "sh" and a[1] != head)]
     for app, tag in arms:
         host, ds, r, pairs = make_arm(app)
-        if tag == "neural":
+        if tag == head:
             sampler.start()
         ms = timed(lambda: step(ds, r), args.steps, args.warmup)
         stage_ms, stage_launches = profile(lambda: step(ds, r), max(1, min(args.steps, 3)))
-        if tag == "neural":
+        if tag == head:
             # keep the GPU under the same load until the sampler has a few readings (100 ms apart)
             t_end = time.perf_counter() + max(0.0, 1.0 - args.steps * ms * 1e-3)
             while time.perf_counter() < t_end:
@@ -195,14 +225,14 @@ def run_ours(args):
                             host=host, ds=ds, r=r, app=tag)
 
     # ---- end to end through the public API with host buffers (neural arm)
-    e2e = None if args.skip_e2e else measure_e2e(api, torch, ctx, results["neural"], cams, G, views, args, timed, dev)
+    e2e = None if args.skip_e2e else measure_e2e(api, torch, ctx, results[head], cams, G, views, args, timed, dev)
 
     # ---- appearance-decode sweep (separate-pass kernels, HBM resident)
-    decode = None if args.skip_decode else decode_sweep(api, torch, ctx, dev, peaks, args)
+    decode = None if (args.skip_decode or args.config != 3) else decode_sweep(api, torch, ctx, dev, peaks, args)
 
     if rank != 0:
         return
-    neural = results["neural"]
+    neural = results[head]
     ms = neural["ms"]
     stage_ms = neural["stage_ms"]
     total_stage = sum(stage_ms.values()) or 1.0
@@ -212,11 +242,10 @@ def run_ours(args):
     alu_peak = NUM_SMS * FP32_LANES_PER_SM * 2 * clock_mhz * 1e6 / 1e12   # TFLOP/s
     roof = stage_roofline(dominant, neural, views, n, peaks, alu_peak)
     out = {
-        "metric": METRIC, "value": replicas.job_ms_per_iteration(ms, 1, world), "unit": "ms/iter (8 views, fwd+bwd)", "n_gpus": world,
+        "metric": METRIC, "value": replicas.job_ms_per_iteration(ms, 1, world), "unit": f"ms/iter ({views} views, fwd+bwd)", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": False,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": "config3: 1M Gaussians (64 clusters + shell), 1256x828, 8 orbit views, "
-                               "neural appearance (8 fp16 features + shared 32-16-16-3 MLP), fwd+bwd",
+        "config": {"workload": wl["name"], "appearance": head,
                    "n": n, "width": WIDTH, "height": HEIGHT, "views": views,
                    "cache": "inputs_larger_than_L2 (per-view working set > 126 MB; 8 different cameras)",
                    "multi_gpu": "replicas only"},
@@ -229,14 +258,14 @@ def run_ours(args):
         "stages_ms_per_step": {k: round(v, 4) for k, v in stage_ms.items() if v > 0},
         "stage_share": {k: round(v / total_stage, 4) for k, v in stage_ms.items() if v > 0},
         "pairs_per_view": neural["pairs"], "visible_per_view": neural["visible"] / views,
-        "sh": None if args.skip_sh else {
+        "sh": None if "sh" not in results or head == "sh" else {
             "ms_per_step": results["sh"]["ms"],
             "stages_ms_per_step": {k: round(v, 4) for k, v in results["sh"]["stage_ms"].items() if v > 0}},
         "appearance_decode": decode,
         "peaks": peaks,
     }
     if not args.skip_cpu:
-        out["cpu_baseline"] = cpu_baseline(neural["host"], views, n)
+        out["cpu_baseline"] = cpu_baseline(neural["host"], cams_host, n)
     print(json.dumps(out))
 
 
@@ -281,34 +310,63 @@ def _stage_roofline(stage, arm, views, n, peaks, alu_peak):
 
 def measure_e2e(api, torch, ctx, arm, cams, G, views, args, timed, dev):
     """Same step, but the scene parameters and upstream gradients start in pinned host memory and the
-    image and every gradient buffer end there: host<->device copies are inside the timed region."""
+    image and every gradient buffer of every view end there: the host<->device copies are inside the
+    timed region.  The copies run on their own streams (one per direction) against double-buffered
+    device buffers, so that view v's results travel while view v+1 is computed; the step ends when the
+    last copy has landed."""
     host, ds, r = arm["host"], arm["ds"], arm["r"]
     pin = lambda t: t.cpu().pin_memory()
-    names = ["means", "log_scales", "quats", "opacity_logits", "base_color", "features", "mlp_weights"]
+    app_names = ["features", "mlp_weights"] if arm["app"] == "neural" else ["sh_rest"]
+    names = ["means", "log_scales", "quats", "opacity_logits", "base_color"] + app_names
     h_scene = {k: pin(getattr(ds, k)) for k in names}
     h_G = pin(G)
-    g = r.grads
-    gnames = ["means", "log_scales", "quats", "opacity_logits", "base_color", "features", "mlp_weights"]
-    h_grads = {k: torch.empty_like(getattr(g, k), device="cpu").pin_memory() for k in gnames}
+    grads = [r.grads, api.alloc_grads(ds.n, r.app, dev)]
+    images = [r.image, torch.empty_like(r.image)]
+    h_grads = {k: torch.empty_like(getattr(grads[0], k), device="cpu").pin_memory() for k in names}
     h_image = torch.empty_like(r.image, device="cpu").pin_memory()
-    d_G = torch.empty_like(G[0])
-    h2d = sum(t.numel() * t.element_size() for t in h_scene.values()) + views * d_G.numel() * 4
+    d_G = [torch.empty_like(G[0]), torch.empty_like(G[0])]
+    h2d = sum(t.numel() * t.element_size() for t in h_scene.values()) + views * d_G[0].numel() * 4
     d2h = views * (sum(t.numel() * t.element_size() for t in h_grads.values()) + h_image.numel() * 4)
+    main = torch.cuda.current_stream(dev)
+    up, down = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+    ev_up = [torch.cuda.Event(), torch.cuda.Event()]
+    ev_down = [torch.cuda.Event(), torch.cuda.Event()]
+    ev_done = [torch.cuda.Event() for _ in range(views)]
 
     def step():
-        for k in names:
-            getattr(ds, k).copy_(h_scene[k], non_blocking=True)
+        up.wait_stream(main)                       # the previous step no longer reads the scene
+        with torch.cuda.stream(up):
+            for k in names:
+                getattr(ds, k).copy_(h_scene[k], non_blocking=True)
+            d_G[0].copy_(h_G[0], non_blocking=True)
+            ev_up[0].record(up)
         for v in range(views):
-            d_G.copy_(h_G[v], non_blocking=True)
+            b = v & 1
+            if v + 1 < views:
+                with torch.cuda.stream(up):
+                    if v >= 1:
+                        up.wait_event(ev_done[v - 1])   # d_G[1 - b] was the input of view v - 1
+                    d_G[1 - b].copy_(h_G[v + 1], non_blocking=True)
+                    ev_up[1 - b].record(up)
+            main.wait_event(ev_up[b])
+            if v >= 2:
+                main.wait_event(ev_down[b])         # view v - 2 has left buffer set b
+            r.image, r.grads = images[b], grads[b]
             r.forward(ds, cams[v])
-            r.backward(ds, cams[v], d_G)
-            h_image.copy_(r.image, non_blocking=True)
-            for k in gnames:
-                h_grads[k].copy_(getattr(g, k), non_blocking=True)
+            r.backward(ds, cams[v], d_G[b])
+            ev_done[v].record(main)
+            with torch.cuda.stream(down):
+                down.wait_event(ev_done[v])
+                h_image.copy_(images[b], non_blocking=True)
+                for k in names:
+                    h_grads[k].copy_(getattr(grads[b], k), non_blocking=True)
+                ev_down[b].record(down)
+        main.wait_stream(down)
 
     ms = timed(step, max(2, args.steps // 2), 2)
-    return {"value": ms, "unit": "ms/iter (8 views, fwd+bwd)", "h2d_bytes_per_step": int(h2d),
-            "d2h_bytes_per_step": int(d2h)}
+    r.image, r.grads = images[0], grads[0]
+    return {"value": ms, "unit": f"ms/iter ({views} views, fwd+bwd)", "h2d_bytes_per_step": int(h2d),
+            "d2h_bytes_per_step": int(d2h), "overlap": "copies on their own streams, double-buffered"}
 
 
 def decode_sweep(api, torch, ctx, dev, peaks, args):
@@ -373,14 +431,14 @@ def oracle_view_ms(host_scene, cam, G):
     return (time.perf_counter() - t0) * 1e3
 
 
-def cpu_baseline(host_scene, views, n):
+def cpu_baseline(host_scene, cams, n):
     from oracle import gs_oracle
     from paper_2609_05255_b200 import scenes
     gs_oracle.build()
-    cams = scenes.orbit_cameras(WIDTH, HEIGHT, views)
+    views = len(cams)
     G = scenes.upstream_gradient(cams[0], 4242)
     ms = oracle_view_ms(host_scene, cams[0], G)
-    return {"value": ms * views, "unit": "ms/iter (8 views, fwd+bwd)", "cores": gs_oracle.num_threads(),
+    return {"value": ms * views, "unit": f"ms/iter ({views} views, fwd+bwd)", "cores": gs_oracle.num_threads(),
             "kind": "oracle", "sample": f"1 of {views} views of the full {n}-Gaussian scene, fwd+bwd, scaled x{views}"}
 
 
@@ -391,24 +449,23 @@ def run_reference(args):
     from oracle import gs_oracle
     from paper_2609_05255_b200 import scenes
     gs_oracle.build()
-    views, n = args.views, args.n
-    host = scenes.config3(scenes.APP_NEURAL, n=n, width=WIDTH, height=HEIGHT, views=views).scene
-    cams = scenes.orbit_cameras(WIDTH, HEIGHT, views)
+    wl = workload_of(args, scenes)
+    views, n, WIDTH, HEIGHT, cams = wl["views"], wl["n"], wl["width"], wl["height"], wl["cams"]
+    host = wl["scene"](wl["arms"][0][0])
     Gs = [scenes.upstream_gradient(cams[0], 4242)]
     for _ in range(args.warmup):
         oracle_view_ms(host, cams[0], Gs[0])
     t = [oracle_view_ms(host, cams[k % views], Gs[0]) for k in range(args.steps)]
     ms = sum(t) / len(t) * views
     sample = f"each step = 1 of {views} views of the full {n}-Gaussian scene, fwd+bwd, scaled x{views}"
-    out = {"impl": "reference", "metric": METRIC, "value": ms, "unit": "ms/iter (8 views, fwd+bwd)",
+    out = {"impl": "reference", "metric": METRIC, "value": ms, "unit": f"ms/iter ({views} views, fwd+bwd)",
            "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
            "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-           "config": {"workload": "config3: 1M Gaussians (64 clusters + shell), 1256x828, 8 orbit views, "
-                                  "neural appearance, fwd+bwd", "n": n, "width": WIDTH, "height": HEIGHT,
-                      "views": views},
-           "cpu_baseline": {"value": ms, "unit": "ms/iter (8 views, fwd+bwd)", "cores": gs_oracle.num_threads(),
+           "config": {"workload": wl["name"], "appearance": wl["arms"][0][1], "n": n, "width": WIDTH,
+                      "height": HEIGHT, "views": views},
+           "cpu_baseline": {"value": ms, "unit": f"ms/iter ({views} views, fwd+bwd)", "cores": gs_oracle.num_threads(),
                             "kind": "oracle", "sample": sample},
-           "e2e": {"value": ms, "unit": "ms/iter (8 views, fwd+bwd)", "h2d_bytes_per_step": 0,
+           "e2e": {"value": ms, "unit": f"ms/iter ({views} views, fwd+bwd)", "h2d_bytes_per_step": 0,
                    "d2h_bytes_per_step": 0},
            "gpu_launches": 0}
     print(json.dumps(out))
@@ -420,8 +477,10 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--n", type=int, default=N_GAUSS)
-    ap.add_argument("--views", type=int, default=VIEWS)
+    ap.add_argument("--config", type=int, default=3, choices=[1, 2, 3, 4],
+                    help="workload (3 = the headline: 1M Gaussians, 8 views; the others fill the results table)")
+    ap.add_argument("--n", type=int, default=None, help="override the Gaussian count of config 3")
+    ap.add_argument("--views", type=int, default=None, help="override the number of views of configs 3 and 4")
     ap.add_argument("--quick", action="store_true", help="decode sweep at 1M only")
     ap.add_argument("--skip-decode", action="store_true")
     ap.add_argument("--skip-cpu", action="store_true")

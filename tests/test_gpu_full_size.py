@@ -1,5 +1,6 @@
-"""Parity at the full benchmark sizes, in the launch configuration bench.py times: one view of the
-1M-Gaussian 1256x828 scene (neural and SH) and one view of the 3M-Gaussian 1920x1080 scene, checked
+"""Parity at the full benchmark sizes, in the launch configuration bench.py times: the 100k-Gaussian
+512x512 scene, one view of the 1M-Gaussian 1256x828 scene (neural and SH) and one view of the
+3M-Gaussian 1920x1080 scene (config 1 runs at its full size among the small cases), checked
 against the oracle with the same stage-by-stage rules as the small cases."""
 from types import SimpleNamespace
 
@@ -13,6 +14,7 @@ import test_gpu_parity as small
 pytestmark = pytest.mark.gpu
 
 CASES = {
+    "config2_neural_100k": lambda: (scenes.config2(), 0),
     "config3_neural_1M": lambda: (scenes.config3(scenes.APP_NEURAL), 2),
     "config3_sh_1M": lambda: (scenes.config3(scenes.APP_SH), 5),
     "config4_neural_3M": lambda: (scenes.config4(), 7),
