@@ -22,7 +22,7 @@ __device__ __forceinline__ void quad_of(int tile, int gx, int tid, int &px, int 
   py = ty * GS_TILE + warp * 8 + 2 * (lane >> 3);
 }
 
-// Stage one batch entry: (x, y, la, lb) (lc, o) (r, g, b, -).  (la, lb, lc) is the Cholesky factor
+// Stage one batch entry: (x, y, la, lb) (lc, o) (r, g, b, pmin).  (la, lb, lc) is the Cholesky factor
 // of the conic, scaled by sqrt(0.5 log2 e), so that exp(power) = 2^-((la dx + lb dy)^2 + (lc dy)^2):
 // a sum of two squares has no cancellation, which keeps alpha accurate to a few ulp even for
 // footprints hundreds of pixels wide (the expanded quadratic form loses 1e-4 there).
@@ -33,7 +33,10 @@ __device__ __forceinline__ void stage_entry(uint32_t g, const float *mean2d, con
   const float kS = 0.8493218002880191f;   // sqrt(0.5 * log2(e))
   xyab = make_float4(m.x, m.y, kS * q.x, kS * q.y);   // q = (l11, l21, l22, opacity)
   co = make_float2(kS * q.z, q.w);
-  rgb = make_float4(__ldg(color + 3 * (size_t)g), __ldg(color + 3 * (size_t)g + 1), __ldg(color + 3 * (size_t)g + 2), 0.f);
+  // alpha >= 1/255 <=> log2 falloff >= pmin = -log2(255 o): the test is taken on the exponent, before the
+  // exponential, by the forward, the backward and the pair counter alike
+  rgb = make_float4(__ldg(color + 3 * (size_t)g), __ldg(color + 3 * (size_t)g + 1), __ldg(color + 3 * (size_t)g + 2),
+                    -__log2f(255.f * q.w));
 }
 
 // log2 of the Gaussian falloff at the four pixels of a quad; dx0, dy0 are the offsets of the
@@ -56,11 +59,14 @@ __device__ __forceinline__ void quad_power(float dx0, float dy0, float la, float
   p[0] = -pu.x; p[1] = -pu.y; p[2] = -pw.x; p[3] = -pw.y;
 }
 
-// alpha of one pixel from its log2 falloff; false if the pair is skipped.
-__device__ __forceinline__ bool alpha_of(float p, float o, float &e2, float &alpha) {
+// alpha of one pixel from its log2 falloff p; false if the pair is skipped (alpha < 1/255, decided as
+// p < pmin).  raw = o * exp(power) before the clamp at 0.99.
+__device__ __forceinline__ bool alpha_of(float p, float o, float pmin, float &e2, float &raw, float &alpha) {
+  if (p < pmin) return false;
   e2 = ex2_approx(p);             // p <= 0 by construction
-  alpha = fminf(kAlphaMax, __fmul_rn(o, e2));
-  return alpha >= kAlphaMin;
+  raw = __fmul_rn(o, e2);
+  alpha = fminf(kAlphaMax, raw);
+  return true;
 }
 
 __global__ void __launch_bounds__(kThreads) k_blend_fwd(CamDev cam, const uint32_t *__restrict__ ranges,
@@ -104,8 +110,8 @@ __global__ void __launch_bounds__(kThreads) k_blend_fwd(CamDev cam, const uint32
       const float4 col = s_rgb[j];
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
-        float e2, alpha;
-        if (!((live >> k) & 1u) || !alpha_of(p[k], c.y, e2, alpha)) continue;
+        float e2, raw, alpha;
+        if (!((live >> k) & 1u) || !alpha_of(p[k], c.y, col.w, e2, raw, alpha)) continue;
         const float Tn = __fmul_rn(T[k], 1.f - alpha);
         if (Tn < kTmin) { live &= ~(1u << k); continue; }
         const float w = __fmul_rn(alpha, T[k]);
@@ -136,14 +142,13 @@ __device__ __forceinline__ float rcp_approx(float x) {
   return y;
 }
 
-// Sum ten per-lane values over the warp with 14 shuffles instead of 50.  Values 0..7: at each of
+// Sum nine per-lane values over the warp with 14 shuffles instead of 45.  Values 0..7: at each of
 // the first three butterfly levels a lane keeps only the half of the values it is "responsible"
 // for and trades the other half with its partner, so the exchanged volume halves each level
 // (4 + 2 + 1 shuffles); two plain levels finish the one value left per lane.  Afterwards the
 // lanes 0, 4, .., 28 hold the totals: lane 16 * b4 + 8 * b3 + 4 * b2 owns value 4 * b4 + 2 * b3 + b2.
-// Values 8 and 9 are traded once between the half warps and then take four plain levels: every
-// lane below 16 ends with the total of value 8, every lane from 16 up with that of value 9.
-__device__ __forceinline__ void warp_reduce10(const float v[10], int lane, float &mine, float &tail) {
+// Value 8 takes a plain five-level butterfly and ends in every lane.
+__device__ __forceinline__ void warp_reduce9(const float v[9], int lane, float &mine, float &ninth) {
   float a[4], b[2], c;
   const bool hi16 = lane & 16, hi8 = lane & 8, hi4 = lane & 4;
 #pragma unroll
@@ -163,10 +168,10 @@ __device__ __forceinline__ void warp_reduce10(const float v[10], int lane, float
   c += __shfl_xor_sync(kFull, c, 2);
   c += __shfl_xor_sync(kFull, c, 1);
   mine = c;
-  float t = (hi16 ? v[9] : v[8]) + __shfl_xor_sync(kFull, hi16 ? v[8] : v[9], 16);
+  float n = v[8];
 #pragma unroll
-  for (int s = 8; s > 0; s >>= 1) t += __shfl_xor_sync(kFull, t, s);
-  tail = t;
+  for (int s = 16; s > 0; s >>= 1) n += __shfl_xor_sync(kFull, n, s);
+  ninth = n;
 }
 
 // Backward: walk each pixel's composited entries back to front.  The transmittance in front of
@@ -179,8 +184,9 @@ __device__ __forceinline__ void warp_reduce10(const float v[10], int lane, float
 // (1, dx, dy, dx^2, dx dy, dy^2).  The threads therefore sum the six moments of dp in tile-local
 // pixel coordinates (half-integers up to 7.5, so the products are exact), a quad of pixels at a
 // time, and the moments are shifted to the Gaussian's own centre once per (tile, Gaussian) when
-// the batch leaves shared memory.  Ten values per entry cross the warp: the six moments, the
-// colour gradient and the opacity gradient (warp_reduce10); each warp owns its own copy of the
+// the batch leaves shared memory.  The opacity gradient needs no sum of its own: alpha = o exp(power)
+// where it is not clamped, so dL/do = (sum of dp) / o, the zeroth moment.  Nine values per entry cross
+// the warp: the six moments and the colour gradient (warp_reduce9); each warp owns its own copy of the
 // batch's accumulators, so no shared-memory atomics are needed; the sums leave with one global
 // atomic per value.
 // g2d row: (d colour r, g, b, d opacity) (d conic A, B, C, d mean u) (d mean v, -, -, -).
@@ -197,7 +203,7 @@ __global__ void __launch_bounds__(kThreads, 16) k_blend_bwd(CamDev cam, const ui
   __shared__ float2 s_co[kBatchBwd];
   __shared__ float4 s_rgb[kBatchBwd];
   __shared__ uint32_t s_gid[kBatchBwd];
-  __shared__ float s_acc[kThreads / 32][kBatchBwd][10];
+  __shared__ float s_acc[kThreads / 32][kBatchBwd][9];
   __shared__ uint32_t s_max[2];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, tile = (int)__ldg(order + blockIdx.x);
   int px, py;
@@ -231,7 +237,7 @@ __global__ void __launch_bounds__(kThreads, 16) k_blend_bwd(CamDev cam, const ui
   __syncthreads();
   const uint32_t maxc = max(s_max[0], s_max[1]);
   if (maxc == 0 || start + maxc > end) return;   // nothing composited in this tile
-  // value that this lane holds after the reduction (lanes 0, 4, .., 28: one of 0..7; lanes 1 and 17: 8 and 9)
+  // value that this lane holds after the reduction (lanes 0, 4, .., 28: one of 0..7; lane 1 stores value 8)
   const int my_value = ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1);
   const int nbatches = (int)((maxc + kBatchBwd - 1) / kBatchBwd);
   for (int b = nbatches - 1; b >= 0; --b) {
@@ -247,7 +253,7 @@ __global__ void __launch_bounds__(kThreads, 16) k_blend_bwd(CamDev cam, const ui
         stage_entry(g, mean2d, conic_opacity, color, s_xyab[slot], s_co[slot], s_rgb[slot]);
       }
 #pragma unroll
-      for (int k = 0; k < 10; ++k) s_acc[0][slot][k] = s_acc[1][slot][k] = 0.f;
+      for (int k = 0; k < 9; ++k) s_acc[0][slot][k] = s_acc[1][slot][k] = 0.f;
     }
     __syncthreads();
     const int jtop = (int)min((uint32_t)cnt, wmax > first ? wmax - first : 0u);
@@ -259,16 +265,13 @@ __global__ void __launch_bounds__(kThreads, 16) k_blend_bwd(CamDev cam, const ui
       quad_power(fx - a.x, fy - a.y, a.z, a.w, c.x, p, t1, t2);
       const float4 col = s_rgb[j];
       float dp[4] = {0.f, 0.f, 0.f, 0.f};
-      float v[10];
-      v[6] = v[7] = v[8] = v[9] = 0.f;
+      float v[9];
+      v[6] = v[7] = v[8] = 0.f;
       bool any = false;
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
-        if (pos >= nc[k]) continue;
-        const float e2 = ex2_approx(p[k]);
-        const float raw = __fmul_rn(c.y, e2);
-        const float alpha = fminf(kAlphaMax, raw);
-        if (alpha < kAlphaMin) continue;
+        float e2, raw, alpha;
+        if (pos >= nc[k] || !alpha_of(p[k], c.y, col.w, e2, raw, alpha)) continue;
         any = true;
         const float inv = rcp_approx(1.f - alpha);
         const float Tb = T[k] * inv;              // transmittance in front of this entry
@@ -277,10 +280,7 @@ __global__ void __launch_bounds__(kThreads, 16) k_blend_bwd(CamDev cam, const ui
         // d pixel / d alpha = T c - S / (1 - alpha), S = everything composited behind this entry
         const float gc = fmaf(Gb[k], col.z, fmaf(Gg[k], col.y, Gr[k] * col.x));
         const float dalpha = fmaf(T[k], gc, -GS[k]) * inv;
-        if (raw <= kAlphaMax) {                   // not clamped: alpha depends on o and power
-          v[9] = fmaf(e2, dalpha, v[9]);
-          dp[k] = alpha * dalpha;
-        }
+        if (raw <= kAlphaMax) dp[k] = alpha * dalpha;   // not clamped: alpha depends on o and power
         GS[k] = fmaf(w, gc, GS[k]);
         T[k] = Tb;
       }
@@ -292,10 +292,10 @@ __global__ void __launch_bounds__(kThreads, 16) k_blend_bwd(CamDev cam, const ui
         v[3] = fmaf(XX0, sL, XX1 * sR);
         v[4] = fmaf(X0, fmaf(Y0, dp[0], Y1 * dp[2]), X1 * fmaf(Y0, dp[1], Y1 * dp[3]));
         v[5] = fmaf(YY0, sT, YY1 * sB);
-        float mine, tail;
-        warp_reduce10(v, lane, mine, tail);
+        float mine, ninth;
+        warp_reduce9(v, lane, mine, ninth);
         if ((lane & 3) == 0) s_acc[warp][j][my_value] = mine;
-        if ((lane & 15) == 1) s_acc[warp][j][8 + (lane >> 4)] = tail;
+        if (lane == 1) s_acc[warp][j][8] = ninth;
       }
     }
     __syncthreads();
@@ -303,17 +303,17 @@ __global__ void __launch_bounds__(kThreads, 16) k_blend_bwd(CamDev cam, const ui
     for (int h = 0; h < kBatchBwd / kThreads; ++h) {
       const int slot = tid + h * kThreads;
       if (slot < cnt) {
-        float M[10];
+        float M[9];
         bool touched = false;
 #pragma unroll
-        for (int k = 0; k < 10; ++k) {
+        for (int k = 0; k < 9; ++k) {
           M[k] = s_acc[0][slot][k] + s_acc[1][slot][k];
           touched = touched || (M[k] != 0.f);
         }
         if (touched) {
           // moments about the Gaussian's centre from the tile-local ones: d = (X + ox, Y + oy)
           const float4 a = s_xyab[slot];
-          const float lc = s_co[slot].x;
+          const float lc = s_co[slot].x, o = s_co[slot].y;
           const float ox = ox_tile - a.x, oy = oy_tile - a.y;
           const float sx = fmaf(ox, M[0], M[1]), sy = fmaf(oy, M[0], M[2]);
           const float sxx = fmaf(ox, M[1] + sx, M[3]);
@@ -322,7 +322,7 @@ __global__ void __launch_bounds__(kThreads, 16) k_blend_bwd(CamDev cam, const ui
           // the staged factor is the conic's Cholesky factor times sqrt(0.5 log2 e)
           const float A = 2.f * kLn2 * a.z * a.z, B = 2.f * kLn2 * a.z * a.w, C = 2.f * kLn2 * fmaf(a.w, a.w, lc * lc);
           float *dst = g2d + (size_t)s_gid[slot] * 12;
-          atomicAdd(dst + 0, M[6]); atomicAdd(dst + 1, M[7]); atomicAdd(dst + 2, M[8]); atomicAdd(dst + 3, M[9]);
+          atomicAdd(dst + 0, M[6]); atomicAdd(dst + 1, M[7]); atomicAdd(dst + 2, M[8]); atomicAdd(dst + 3, __fdividef(M[0], o));
           atomicAdd(dst + 4, -0.5f * sxx); atomicAdd(dst + 5, -sxy); atomicAdd(dst + 6, -0.5f * syy);
           atomicAdd(dst + 7, fmaf(A, sx, B * sy)); atomicAdd(dst + 8, fmaf(B, sx, C * sy));
         }
@@ -369,11 +369,12 @@ __global__ void __launch_bounds__(kThreads) k_blend_count(CamDev cam, const uint
       const float2 c = s_co[j];
       float p[4], t1[4], t2[2];
       quad_power(fx - a.x, fy - a.y, a.z, a.w, c.x, p, t1, t2);
+      const float4 col = s_rgb[j];
       evaluated += __popc(live);
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
-        float e2, alpha;
-        if (!((live >> k) & 1u) || !alpha_of(p[k], c.y, e2, alpha)) continue;
+        float e2, raw, alpha;
+        if (!((live >> k) & 1u) || !alpha_of(p[k], c.y, col.w, e2, raw, alpha)) continue;
         const float Tn = __fmul_rn(T[k], 1.f - alpha);
         if (Tn < kTmin) { live &= ~(1u << k); continue; }
         T[k] = Tn;
