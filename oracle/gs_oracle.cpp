@@ -187,6 +187,25 @@ int gso_num_mlp_weights() { return kNumW; }
 // per Gaussian (App. B.3, first-layer folding).
 int gso_mlp_macs(int fold) { return (fold ? 16 : kIn) * kHid + kHid * kHid + kHid * kOut; }
 
+// One Adam step on a [rows, cols] parameter tensor with one learning rate per column (App. C.1:
+// the optimiser is Adam with the single change that it takes a learning rate per column of a
+// parameter tensor).  Plain textbook form, step = 1, 2, ...:
+//   m <- b1 m + (1 - b1) g;  v <- b2 v + (1 - b2) g^2;
+//   theta <- theta - lr_c (m / (1 - b1^step)) / (sqrt(v / (1 - b2^step)) + eps).
+void gso_adam_step(int64_t rows, int cols, double* param, const double* grad, double* m, double* v,
+                   const double* lr, double beta1, double beta2, double eps, int64_t step) {
+  const double c1 = 1.0 - std::pow(beta1, (double)step), c2 = 1.0 - std::pow(beta2, (double)step);
+  for (int64_t r = 0; r < rows; ++r)
+    for (int c = 0; c < cols; ++c) {
+      const int64_t i = r * cols + c;
+      const double g = grad[i];
+      m[i] = beta1 * m[i] + (1.0 - beta1) * g;
+      v[i] = beta2 * v[i] + (1.0 - beta2) * g * g;
+      const double mhat = m[i] / c1, vhat = v[i] / c2;
+      param[i] -= lr[c] * mhat / (std::sqrt(vhat) + eps);
+    }
+}
+
 void gso_sh_basis(const double* d, double* Y) { sh_basis(d, Y); }
 void gso_sh_basis_grad(const double* d, double* G) {
   double g[16][3];

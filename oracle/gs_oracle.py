@@ -103,6 +103,19 @@ def num_mlp_weights() -> int:
     return lib().gso_num_mlp_weights()
 
 
+def adam_step(param, grad, m, v, lr, beta1=0.9, beta2=0.999, eps=1e-15, step=1):
+    """One Adam step with one learning rate per column (App. C.1).  param, grad, m, v: [rows, cols] (or
+    [cols] for a single row); lr: [cols].  Returns new (param, m, v) as float64 arrays of the input shape."""
+    shape = np.shape(param)
+    lr = _f64(np.atleast_1d(lr))
+    cols = lr.shape[0]
+    p2, g2 = _f64(param).reshape(-1, cols).copy(), _f64(grad).reshape(-1, cols)
+    m2, v2 = _f64(m).reshape(-1, cols).copy(), _f64(v).reshape(-1, cols).copy()
+    lib().gso_adam_step(C.c_int64(p2.shape[0]), C.c_int(cols), _dp(p2), _dp(np.ascontiguousarray(g2)), _dp(m2), _dp(v2),
+                        _dp(lr), C.c_double(beta1), C.c_double(beta2), C.c_double(eps), C.c_int64(step))
+    return p2.reshape(shape), m2.reshape(shape), v2.reshape(shape)
+
+
 def preprocess(means, log_scales, quats, opacity_logits, cam):
     means, log_scales, quats, logits = _f64(means), _f64(log_scales), _f64(quats), _f64(opacity_logits)
     n = means.shape[0]
