@@ -200,6 +200,41 @@ GsStatus gs_appearance_backward_noalloc(const GsScene *scene, const float *dirs,
                                         GsGrads *grads, float *dL_ddirs, void *stream, char *error_text,
                                         size_t error_text_bytes);
 
+/* ---- NEXT step after the rendering path: the fused Adam update (App. C.1, App. C.2) ------------
+ * The paper's optimiser is Adam with one change: it takes ONE LEARNING RATE PER COLUMN of a
+ * parameter tensor (App. C.1), so that e.g. base colour, coefficients or the parameters of a site
+ * keep their own rates without being split into separate tensors.  Features and decoder weights are
+ * stored and updated in single precision, and a half-precision copy is made for the next
+ * iteration's forward and backward pass (App. C.2).  The update touches every row, also those of
+ * Gaussians that were invisible this iteration (Tab. 3, footnote).
+ *
+ * One tensor of an update, row-major [rows, cols]:
+ *   m <- beta1 m + (1 - beta1) g;   v <- beta2 v + (1 - beta2) g^2;
+ *   param <- param - lr[c] (m / (1 - beta1^step)) / (sqrt(v / (1 - beta2^step)) + eps)
+ * param, grad, exp_avg (m), exp_avg_sq (v): DEVICE pointers, fp32, 16-byte aligned, owned by the
+ * caller; param, exp_avg, exp_avg_sq are updated in place, grad is only read.  half_copy: DEVICE
+ * pointer to [rows, cols] IEEE fp16 bits (8-byte aligned) that receives the updated values rounded
+ * to nearest even, or NULL.  lr: HOST array of cols rates (read during the call).  A decoder-weight
+ * vector is a tensor with rows = 816, cols = 1 (App. B.2 sets its beta2 to 0.99). */
+enum { GS_ADAM_MAX_COLS = 64, GS_ADAM_MAX_TENSORS = 8 };
+typedef struct {
+  float *param;
+  const float *grad;
+  float *exp_avg;
+  float *exp_avg_sq;
+  uint16_t *half_copy;
+  int64_t rows;
+  int32_t cols;          /* 1 .. GS_ADAM_MAX_COLS; rows * cols < 2^32 */
+  const float *lr;
+  float beta1, beta2, eps;
+} GsAdamTensor;
+/* Updates up to GS_ADAM_MAX_TENSORS tensors with ONE kernel launch on `stream` (asynchronous; no
+ * allocation, no synchronisation).  step = 1, 2, ... is the number of this update, shared by the
+ * tensors.  Tensors with rows = 0 are skipped.  GS_ERR_INVALID_ARG (nothing launched) for a NULL or
+ * misaligned pointer, cols out of range, step < 1, betas outside [0, 1) or too many tensors;
+ * GS_ERR_CAPACITY if a tensor has 2^32 elements or more. */
+GsStatus gs_adam_step(GsContext *ctx, const GsAdamTensor *tensors, int32_t num_tensors, int64_t step, void *stream);
+
 /* Per-stage device timing, for benchmarks (the paper gives wall-clock protocols only, App. C; this
  * is the measurement hook of this library).  While enabled, every stage the library launches is
  * bracketed by CUDA events on the caller's stream.  gs_profile_collect synchronises those events,
@@ -218,6 +253,7 @@ typedef enum {
   GS_STAGE_PREPROCESS_BWD,     /* projection backward + fused appearance backward               */
   GS_STAGE_APPEARANCE_FWD,     /* separate-pass decode                                          */
   GS_STAGE_APPEARANCE_BWD,
+  GS_STAGE_ADAM,               /* fused parameter update                                        */
   GS_NUM_STAGES
 } GsStage;
 GsStatus gs_profile_enable(GsContext *ctx, int enable);

@@ -82,7 +82,7 @@ _lib.gs_appearance_backward.restype = C.c_int
 
 
 STAGES = ["preprocess_fwd", "depth_sort", "tile_offsets", "keygen", "tile_sort", "tile_ranges", "blend_fwd",
-          "blend_bwd", "preprocess_bwd", "appearance_fwd", "appearance_bwd"]
+          "blend_bwd", "preprocess_bwd", "appearance_fwd", "appearance_bwd", "adam"]
 _lib.gs_profile_enable.argtypes = [_vp, C.c_int]
 _lib.gs_profile_enable.restype = C.c_int
 _lib.gs_profile_collect.argtypes = [_vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
@@ -92,6 +92,19 @@ _lib.gs_profile_collect.restype = C.c_int
 _lib.gs_profile_blend_counts.argtypes = [_vp, C.POINTER(GsProjected), C.POINTER(GsBinning), C.POINTER(GsCamera),
                                          C.POINTER(C.c_int64), _vp]
 _lib.gs_profile_blend_counts.restype = C.c_int
+
+
+GS_ADAM_MAX_COLS, GS_ADAM_MAX_TENSORS = 64, 8
+
+
+class GsAdamTensor(C.Structure):
+    _fields_ = [("param", _vp), ("grad", _vp), ("exp_avg", _vp), ("exp_avg_sq", _vp), ("half_copy", _vp),
+                ("rows", C.c_int64), ("cols", C.c_int32), ("lr", C.POINTER(C.c_float)), ("beta1", C.c_float),
+                ("beta2", C.c_float), ("eps", C.c_float)]
+
+
+_lib.gs_adam_step.argtypes = [_vp, C.POINTER(GsAdamTensor), C.c_int32, C.c_int64, _vp]
+_lib.gs_adam_step.restype = C.c_int
 
 
 class GsError(RuntimeError):
@@ -368,6 +381,38 @@ class Renderer:
         gs_render_backward(self.ctx, scene, cam, self.proj, self.binning, self.num_pairs, self.final_T,
                            self.n_contrib, dL_dimage, self.grads, self.workspace, stream)
         return self.grads
+
+
+# ------------------------------------------------------------------------------------------------
+# Fused Adam update
+# ------------------------------------------------------------------------------------------------
+class AdamTensor:
+    """One parameter tensor of an update: fp32 param / grad / exp_avg / exp_avg_sq of the same shape
+    (viewed as [rows, cols] with cols = len(lr)), an optional fp16 tensor that receives the updated
+    values, and the hyper-parameters.  Marshalling only."""
+
+    def __init__(self, param, grad, exp_avg, exp_avg_sq, lr, beta1=0.9, beta2=0.999, eps=1e-15, half_copy=None):
+        lr = [float(x) for x in (lr if hasattr(lr, "__len__") else [lr])]
+        self.cols = len(lr)
+        assert param.numel() % self.cols == 0
+        self.rows = param.numel() // self.cols
+        self.param, self.grad, self.exp_avg, self.exp_avg_sq, self.half_copy = param, grad, exp_avg, exp_avg_sq, half_copy
+        self.lr = (C.c_float * self.cols)(*lr)          # host array, kept alive by this object
+        self.beta1, self.beta2, self.eps = beta1, beta2, eps
+
+    def c_struct(self) -> GsAdamTensor:
+        t = GsAdamTensor()
+        t.param, t.grad, t.exp_avg, t.exp_avg_sq = _ptr(self.param), _ptr(self.grad), _ptr(self.exp_avg), _ptr(self.exp_avg_sq)
+        t.half_copy = _ptr(self.half_copy)
+        t.rows, t.cols, t.lr = self.rows, self.cols, C.cast(self.lr, C.POINTER(C.c_float))
+        t.beta1, t.beta2, t.eps = self.beta1, self.beta2, self.eps
+        return t
+
+
+def gs_adam_step(ctx: Context, tensors, step: int, stream=None) -> None:
+    """Update all `tensors` (AdamTensor objects, at most GS_ADAM_MAX_TENSORS) with one kernel launch."""
+    arr = (GsAdamTensor * max(1, len(tensors)))(*[t.c_struct() for t in tensors])
+    ctx._check(_lib.gs_adam_step(ctx._h, arr, len(tensors), step, _stream_handle(stream)))
 
 
 # ------------------------------------------------------------------------------------------------

@@ -13,6 +13,7 @@ struct StageRecord { int stage; int launches; cudaEvent_t begin, end; };
 
 struct GsContext {
   int device;
+  int num_sms;
   unsigned long long *d_counter;      // device: instance counter (+ one more word for gs_profile_blend_counts)
   unsigned long long *h_counter;      // pinned host mirror
   float *d_w_partials;                // device: [kWgradBlocks, 816] decoder-gradient partial sums
@@ -169,6 +170,8 @@ GsStatus gs_create(int device, GsContext **out) {
   GsContext *ctx = new (std::nothrow) GsContext();
   if (!ctx) return GS_ERR_INTERNAL;
   ctx->device = device;
+  ctx->num_sms = 148;
+  cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, device);
   ctx->error[0] = 0;
   ctx->d_counter = nullptr; ctx->h_counter = nullptr; ctx->d_w_partials = nullptr;
   ctx->profiling = false;
@@ -429,6 +432,32 @@ GsStatus gs_profile_blend_counts(GsContext *ctx, const GsProjected *proj, const 
   counts_host[0] = (int64_t)ctx->h_counter[0];
   counts_host[1] = (int64_t)ctx->h_counter[1];
   return GS_OK;
+}
+
+GsStatus gs_adam_step(GsContext *ctx, const GsAdamTensor *tensors, int32_t num_tensors, int64_t step, void *stream) {
+  if (!ctx) return GS_ERR_INVALID_ARG;
+  if (num_tensors < 0 || num_tensors > GS_ADAM_MAX_TENSORS || (num_tensors > 0 && !tensors))
+    return fail(ctx, GS_ERR_INVALID_ARG, "num_tensors must be 0..8 and tensors non-NULL");
+  if (step < 1) return fail(ctx, GS_ERR_INVALID_ARG, "step counts from 1");
+  for (int i = 0; i < num_tensors; ++i) {
+    const GsAdamTensor &t = tensors[i];
+    if (t.rows < 0 || t.cols < 1 || t.cols > GS_ADAM_MAX_COLS) return fail(ctx, GS_ERR_INVALID_ARG, "rows < 0 or cols outside 1..64");
+    if (t.rows == 0) continue;
+    if (!t.lr) return fail(ctx, GS_ERR_INVALID_ARG, "lr is NULL");
+    if (bad_ptr(t.param) || bad_ptr(t.grad) || bad_ptr(t.exp_avg) || bad_ptr(t.exp_avg_sq) ||
+        (t.half_copy && (reinterpret_cast<uintptr_t>(t.half_copy) & 7u)))
+      return fail(ctx, GS_ERR_INVALID_ARG, "an Adam tensor pointer is NULL or misaligned");
+    if (!(t.beta1 >= 0.f && t.beta1 < 1.f && t.beta2 >= 0.f && t.beta2 < 1.f) || !(t.eps >= 0.f))
+      return fail(ctx, GS_ERR_INVALID_ARG, "betas must lie in [0, 1) and eps be >= 0");
+    if ((uint64_t)t.rows * (uint64_t)t.cols >= (1ull << 32)) return fail(ctx, GS_ERR_CAPACITY, "an Adam tensor has 2^32 elements or more");
+  }
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaSetDevice(ctx->device);
+  {
+    StageTimer t(ctx, GS_STAGE_ADAM, s);
+    t.done(launch_adam(tensors, num_tensors, step, ctx->num_sms, s));
+  }
+  return check_cuda(ctx, cudaGetLastError(), "adam launch");
 }
 
 GsStatus gs_profile_enable(GsContext *ctx, int enable) {
