@@ -252,6 +252,7 @@ def run_ours(args):
 
     # ---- appearance-decode sweep (separate-pass kernels, HBM resident)
     decode = None if (args.skip_decode or args.config != 3) else decode_sweep(api, torch, ctx, dev, peaks, args)
+    adam = None if (args.skip_decode or args.config != 3) else adam_sweep(api, torch, ctx, dev, peaks, n)
 
     if rank != 0:
         return
@@ -287,6 +288,7 @@ def run_ours(args):
             "ms_per_step": results["sh"]["ms"],
             "stages_ms_per_step": {k: round(v, 4) for k, v in results["sh"]["stage_ms"].items() if v > 0}},
         "appearance_decode": decode,
+        "adam_update": adam,
         "peaks": peaks,
     }
     if not args.skip_cpu:
@@ -392,6 +394,47 @@ def measure_e2e(api, torch, ctx, arm, cams, G, views, args, timed, dev):
     r.image, r.grads = images[0], grads[0]
     return {"value": ms, "unit": f"ms/iter ({views} views, fwd+bwd)", "h2d_bytes_per_step": int(h2d),
             "d2h_bytes_per_step": int(d2h), "overlap": "copies on their own streams, double-buffered"}
+
+
+def adam_sweep(api, torch, ctx, dev, peaks, n):
+    """The step that follows the rendering path: one fused Adam update of every parameter of a model, SH
+    (59 floats per Gaussian) against neural (22 floats + 816 weights), one launch each.  The tensors are far
+    larger than L2 (16 B of state per element), so the stream is measured from HBM."""
+    y0 = 0.28209479177387814
+    geo = [("means", 3, 1.6e-4), ("log_scales", 3, 5e-3), ("quats", 4, 1e-3), ("opacity_logits", 1, 5e-2)]
+    sets = {"sh": geo + [("base_color", 3, 0.0025 * y0), ("sh_rest", 45, 0.000125)],
+            "neural": geo + [("base_color", 3, 0.00025), ("features", 8, 0.008), ("mlp_weights", 1, 0.003)]}
+    out = {}
+    for tag, spec in sets.items():
+        gen = torch.Generator(device=dev); gen.manual_seed(77)
+        tensors, nbytes = [], 0
+        for name, cols, lr in spec:
+            rows = 816 if name == "mlp_weights" else n
+            p = torch.randn((rows, cols), device=dev, generator=gen)
+            g = torch.randn((rows, cols), device=dev, generator=gen) * 1e-3
+            m, v = torch.zeros_like(p), torch.zeros_like(p)
+            half = torch.empty((rows, cols), device=dev, dtype=torch.float16) if name in ("features", "mlp_weights") else None
+            tensors.append(api.AdamTensor(p, g, m, v, [lr] * cols, 0.9, 0.99 if name == "mlp_weights" else 0.999, 1e-15,
+                                          half_copy=half))
+            nbytes += rows * cols * (28 + (2 if half is not None else 0))
+        for it in range(3):
+            api.gs_adam_step(ctx, tensors, it + 1)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = 20
+        e0.record()
+        for it in range(reps):
+            api.gs_adam_step(ctx, tensors, it + 4)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / reps
+        gbs = nbytes / (ms * 1e-3) / 1e9
+        out[tag] = {"ms": round(ms, 4), "bytes_per_gaussian": round(nbytes / n, 1), "GBps": round(gbs, 1),
+                    "frac_of_hbm_peak": round(gbs / peaks["hbm_gbs"], 4), "launches_per_update": 1}
+        del tensors
+    out["n"] = n
+    out["cache"] = "tensors larger than L2 (352 MB neural, 944 MB SH at 1M)"
+    return out
 
 
 def decode_sweep(api, torch, ctx, dev, peaks, args):

@@ -42,11 +42,17 @@ __device__ __forceinline__ void adam_element(float &p, float g, float &m, float 
 }
 
 __global__ void __launch_bounds__(kAdamThreads) k_adam(const __grid_constant__ AdamArgs a) {
+  // the per-column step sizes of the chunk's tensor, in shared memory: the lanes of a warp want
+  // different columns, which the constant bank would serve one address at a time
+  __shared__ float s_step[GS_ADAM_MAX_COLS];
   const uint32_t total_chunks = a.chunk_start[a.num_tensors];
   for (uint32_t chunk = blockIdx.x; chunk < total_chunks; chunk += gridDim.x) {
     int ti = 0;
     while (ti + 1 < a.num_tensors && chunk >= a.chunk_start[ti + 1]) ++ti;
     const AdamTensorDev &t = a.t[ti];
+    __syncthreads();
+    if (threadIdx.x < t.cols) s_step[threadIdx.x] = t.step_size[threadIdx.x];
+    __syncthreads();
     const uint32_t base = (chunk - a.chunk_start[ti]) * kAdamChunk;
     float4 p[kAdamUnroll], g[kAdamUnroll], m[kAdamUnroll], v[kAdamUnroll];
     uint32_t e[kAdamUnroll];
@@ -71,7 +77,7 @@ __global__ void __launch_bounds__(kAdamThreads) k_adam(const __grid_constant__ A
         const float *gg = &g[u].x;
 #pragma unroll
         for (int k = 0; k < kAdamVec; ++k) {
-          adam_element(pp[k], gg[k], mm[k], vv[k], t.step_size[c], t.beta1, t.beta2, t.eps, t.inv_sqrt_c2);
+          adam_element(pp[k], gg[k], mm[k], vv[k], s_step[c], t.beta1, t.beta2, t.eps, t.inv_sqrt_c2);
           c = (c + 1 == t.cols) ? 0u : c + 1;
         }
         *reinterpret_cast<float4 *>(t.param + e[u]) = p[u];
@@ -88,7 +94,7 @@ __global__ void __launch_bounds__(kAdamThreads) k_adam(const __grid_constant__ A
         uint32_t c = e[u] % t.cols;
         for (uint32_t i = e[u]; i < t.count; ++i) {
           float pv = t.param[i], mv = t.m[i], vv = t.v[i];
-          adam_element(pv, t.grad[i], mv, vv, t.step_size[c], t.beta1, t.beta2, t.eps, t.inv_sqrt_c2);
+          adam_element(pv, t.grad[i], mv, vv, s_step[c], t.beta1, t.beta2, t.eps, t.inv_sqrt_c2);
           t.param[i] = pv; t.m[i] = mv; t.v[i] = vv;
           if (t.half_copy) t.half_copy[i] = __float2half_rn(pv);
           c = (c + 1 == t.cols) ? 0u : c + 1;
