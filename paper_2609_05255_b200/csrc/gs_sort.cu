@@ -150,7 +150,15 @@ __global__ void __launch_bounds__(kSortThreads, 3) k_radix_scatter(
       // lanes with the same digit form a group; its first lane bumps the warp's counter once and
       // hands the old value to the group.  A warp's shared-memory atomics execute in program order,
       // so the 16 items need no barrier between them and their latencies overlap.
-      const uint32_t peers = __match_any_sync(kFull, d);
+      // The group comes from one ballot per digit bit: a fixed cost, where the match instruction
+      // takes time in proportion to the number of different digits in the warp.
+      uint32_t peers = kFull;
+#pragma unroll
+      for (int b = 0; b < 8; ++b) {
+        const bool bit = (d >> b) & 1u;
+        const uint32_t m = __ballot_sync(kFull, bit);
+        peers &= bit ? m : ~m;
+      }
       const int leader = __ffs(peers) - 1;
       uint32_t prior = 0;
       if (lane == leader) prior = atomicAdd(&s_warp_cnt[warp][d], (uint32_t)__popc(peers));
