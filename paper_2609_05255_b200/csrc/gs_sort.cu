@@ -33,7 +33,7 @@ SortPlan plan_for(int64_t count) {
 
 // Digit histogram of each block's contiguous range: table[block][digit].
 __global__ void __launch_bounds__(kSortThreads) k_radix_hist(const uint32_t *__restrict__ keys, int64_t count,
-                                                             int shift, int tiles_per_block,
+                                                             int shift, uint32_t mask, int tiles_per_block,
                                                              uint32_t *__restrict__ table) {
   __shared__ uint32_t s_hist[kSortWarps][256];
   const int tid = threadIdx.x, warp = tid >> 5;
@@ -43,7 +43,7 @@ __global__ void __launch_bounds__(kSortThreads) k_radix_hist(const uint32_t *__r
   int64_t end = begin + (int64_t)tiles_per_block * kSortTile;
   if (end > count) end = count;
   for (int64_t i = begin + tid; i < end; i += kSortThreads) {
-    const uint32_t d = (__ldg(keys + i) >> shift) & 255u;
+    const uint32_t d = (__ldg(keys + i) >> shift) & mask;
     atomicAdd(&s_hist[warp][d], 1u);
   }
   __syncthreads();
@@ -103,7 +103,10 @@ __device__ __forceinline__ uint32_t block_exclusive_scan_256(uint32_t v, uint32_
   return off + inc - v;
 }
 
-// One pass: stable scatter of this block's range by the digit at `shift`.
+// One pass: stable scatter of this block's range by the BITS-wide digit at `shift`.  Slots past the
+// end of the input carry the largest digit and sit at the end of the last tile, so they rank after
+// every real key and are never written.
+template <int BITS>
 __global__ void __launch_bounds__(kSortThreads, 3) k_radix_scatter(
     const uint32_t *__restrict__ keys_in, const uint32_t *__restrict__ vals_in, uint32_t *__restrict__ keys_out,
     uint32_t *__restrict__ vals_out, int64_t count, int shift, int tiles_per_block,
@@ -116,6 +119,7 @@ __global__ void __launch_bounds__(kSortThreads, 3) k_radix_scatter(
   __shared__ uint32_t s_warp_tot[kSortWarps];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t lt_mask = (1u << lane) - 1u;
+  constexpr uint32_t kDigitMask = (1u << BITS) - 1u;
 
   // global base of every digit for this block: all smaller digits everywhere (scan of the row
   // totals) + the same digit in the blocks before this one (the row prefix from k_radix_scan_rows)
@@ -146,7 +150,7 @@ __global__ void __launch_bounds__(kSortThreads, 3) k_radix_scatter(
     for (int it = 0; it < kItems; ++it) {
       const int local = warp * (32 * kItems) + it * 32 + lane;
       const bool ok = local < valid_count;
-      const uint32_t d = ok ? ((key[it] >> shift) & 255u) : 255u;
+      const uint32_t d = ok ? ((key[it] >> shift) & kDigitMask) : kDigitMask;
       // lanes with the same digit form a group; its first lane bumps the warp's counter once and
       // hands the old value to the group.  A warp's shared-memory atomics execute in program order,
       // so the 16 items need no barrier between them and their latencies overlap.
@@ -154,7 +158,7 @@ __global__ void __launch_bounds__(kSortThreads, 3) k_radix_scatter(
       // takes time in proportion to the number of different digits in the warp.
       uint32_t peers = kFull;
 #pragma unroll
-      for (int b = 0; b < 8; ++b) {
+      for (int b = 0; b < BITS; ++b) {
         const bool bit = (d >> b) & 1u;
         const uint32_t m = __ballot_sync(kFull, bit);
         peers &= bit ? m : ~m;
@@ -180,7 +184,7 @@ __global__ void __launch_bounds__(kSortThreads, 3) k_radix_scatter(
 #pragma unroll
     for (int it = 0; it < kItems; ++it) {
       const int local = warp * (32 * kItems) + it * 32 + lane;
-      const uint32_t d = (local < valid_count) ? ((key[it] >> shift) & 255u) : 255u;
+      const uint32_t d = (local < valid_count) ? ((key[it] >> shift) & kDigitMask) : kDigitMask;
       const uint32_t pos = s_digit_start[d] + s_warp_cnt[warp][d] + rank[it];
       s_keys[pos] = key[it];
       s_vals[pos] = val[it];
@@ -188,7 +192,7 @@ __global__ void __launch_bounds__(kSortThreads, 3) k_radix_scatter(
     __syncthreads();
     for (int j = tid; j < valid_count; j += kSortThreads) {
       const uint32_t k = s_keys[j];
-      const uint32_t d = (k >> shift) & 255u;
+      const uint32_t d = (k >> shift) & kDigitMask;
       const uint32_t gpos = s_base[d] + ((uint32_t)j - s_digit_start[d]);
       keys_out[gpos] = k;
       vals_out[gpos] = s_vals[j];
@@ -391,16 +395,27 @@ int launch_radix_sort(const uint32_t *keys_in, const uint32_t *vals_in, uint32_t
   const SortPlan plan = plan_for(count);
   int passes = (num_bits + 7) / 8;
   if (passes < 1) passes = 1;
+  const int bits = (num_bits + passes - 1) / passes;     // digits of equal width: 13 bits sort as 7 + 6
   uint32_t *table = static_cast<uint32_t *>(scratch);
   uint32_t *totals = table + (size_t)plan.blocks * 256;
   const uint32_t *src_k = keys_in, *src_v = vals_in;
   for (int p = 0; p < passes; ++p) {
     const bool to_out = ((passes - 1 - p) % 2) == 0;
     uint32_t *dst_k = to_out ? keys_out : tmp_keys, *dst_v = to_out ? vals_out : tmp_vals;
-    k_radix_hist<<<plan.blocks, kSortThreads, 0, st>>>(src_k, count, 8 * p, plan.tiles_per_block, table);
+    k_radix_hist<<<plan.blocks, kSortThreads, 0, st>>>(src_k, count, bits * p, (1u << bits) - 1u, plan.tiles_per_block, table);
     k_radix_scan_rows<<<256, 256, 0, st>>>(table, plan.blocks, totals);
-    k_radix_scatter<<<plan.blocks, kSortThreads, 0, st>>>(src_k, src_v, dst_k, dst_v, count, 8 * p,
-                                                           plan.tiles_per_block, table, totals, plan.blocks);
+#define GS_SCATTER(B)                                                                                              \
+  case B:                                                                                                          \
+    k_radix_scatter<B><<<plan.blocks, kSortThreads, 0, st>>>(src_k, src_v, dst_k, dst_v, count, bits * p,         \
+                                                              plan.tiles_per_block, table, totals, plan.blocks);   \
+    break;
+    switch (bits) {
+      GS_SCATTER(1) GS_SCATTER(2) GS_SCATTER(3) GS_SCATTER(4) GS_SCATTER(5) GS_SCATTER(6) GS_SCATTER(7)
+      default:
+        k_radix_scatter<8><<<plan.blocks, kSortThreads, 0, st>>>(src_k, src_v, dst_k, dst_v, count, bits * p,
+                                                                  plan.tiles_per_block, table, totals, plan.blocks);
+    }
+#undef GS_SCATTER
     src_k = dst_k;
     src_v = dst_v;
   }
