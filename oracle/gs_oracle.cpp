@@ -187,6 +187,66 @@ int gso_num_mlp_weights() { return kNumW; }
 // per Gaussian (App. B.3, first-layer folding).
 int gso_mlp_macs(int fold) { return (fold ? 16 : kIn) * kHid + kHid * kHid + kHid * kOut; }
 
+// Viewer-side evaluation of the neural model (App. C.3, "Neural").  The 16 encoded feature inputs and
+// the constant degree-0 input do not depend on the view, so their 17 columns of the first layer are
+// folded into 16 pre-activations per Gaussian when the model is exported:
+//   pre[o] = W1[o][0] Y_0 + sum_j (W1[o][16+2j] sin f_j + W1[o][17+2j] cos f_j).
+// deg >= 1 (with deg = 0 the residual is disabled and nothing is folded).
+void gso_neural_fold(int64_t n, const double* features, const double* weights, double* pre) {
+  const double d0[3] = {0, 0, 1};
+  double Y[16];
+  sh_basis(d0, Y);   // Y[0] is the constant
+#pragma omp parallel for schedule(static)
+  for (int64_t i = 0; i < n; ++i)
+    for (int o = 0; o < kHid; ++o) {
+      double a = weights[kW1 + o * kIn + 0] * Y[0];
+      for (int j = 0; j < kFeat; ++j) {
+        a += weights[kW1 + o * kIn + 16 + 2 * j] * std::sin(features[kFeat * i + j]);
+        a += weights[kW1 + o * kIn + 17 + 2 * j] * std::cos(features[kFeat * i + j]);
+      }
+      pre[kHid * i + o] = a;
+    }
+}
+
+// Per frame: only the 15 direction-dependent columns (SH degrees 1..3, masked by the active degree)
+// of the first layer remain, 15 (padded to 16) x 16 + 16 x 16 + 16 x 3 = 560 multiply-accumulates:
+//   h1 = ReLU(pre + W1[:, 1..15] Y_1..15(d)); h2 = ReLU(W2 h1); A = tanh(W3 h2); c = ReLU(c0 + 0.5 + A).
+// d = (mean - eye) / |mean - eye|.
+void gso_neural_prepass(int64_t n, int deg, const double* means, const double* base_color, const double* pre,
+                        const double* weights, const double* eye, double* color) {
+  const int na = num_active(deg);
+#pragma omp parallel for schedule(static)
+  for (int64_t i = 0; i < n; ++i) {
+    double A[3] = {0, 0, 0};
+    if (deg > 0) {
+      double d[3] = {means[3 * i] - eye[0], means[3 * i + 1] - eye[1], means[3 * i + 2] - eye[2]};
+      const double len = std::sqrt(d[0] * d[0] + d[1] * d[1] + d[2] * d[2]);
+      for (int c = 0; c < 3; ++c) d[c] /= len;
+      double Y[16], h1[kHid], h2[kHid];
+      sh_basis(d, Y);
+      for (int o = 0; o < kHid; ++o) {
+        double a = pre[kHid * i + o];
+        for (int k = 1; k < na; ++k) a += weights[kW1 + o * kIn + k] * Y[k];
+        h1[o] = a > 0 ? a : 0;
+      }
+      for (int o = 0; o < kHid; ++o) {
+        double a = 0;
+        for (int k = 0; k < kHid; ++k) a += weights[kW2 + o * kHid + k] * h1[k];
+        h2[o] = a > 0 ? a : 0;
+      }
+      for (int o = 0; o < kOut; ++o) {
+        double a = 0;
+        for (int k = 0; k < kHid; ++k) a += weights[kW3 + o * kHid + k] * h2[k];
+        A[o] = std::tanh(a);
+      }
+    }
+    for (int c = 0; c < 3; ++c) {
+      const double v = base_color[3 * i + c] + 0.5 + A[c];
+      color[3 * i + c] = v > 0 ? v : 0;
+    }
+  }
+}
+
 // One Adam step on a [rows, cols] parameter tensor with one learning rate per column (App. C.1:
 // the optimiser is Adam with the single change that it takes a learning rate per column of a
 // parameter tensor).  Plain textbook form, step = 1, 2, ...:

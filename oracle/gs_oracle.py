@@ -103,6 +103,31 @@ def num_mlp_weights() -> int:
     return lib().gso_num_mlp_weights()
 
 
+def neural_fold(scene):
+    """Export step of the viewer (App. C.3): [n,16] pre-activations of the first layer from the features,
+    the constant degree-0 input and their 17 weight columns, in double (not yet rounded to fp16)."""
+    n = scene.means.shape[0]
+    pre = np.zeros((n, 16))
+    lib().gso_neural_fold(C.c_int64(n), _dp(_f64(scene.features)), _dp(_f64(scene.mlp_weights)), _dp(pre))
+    return pre
+
+
+def neural_prepass(scene, pre, eye, deg=None):
+    """Per-frame colour of every Gaussian from the folded pre-activations and the camera position `eye`."""
+    n = scene.means.shape[0]
+    color = np.zeros((n, 3))
+    lib().gso_neural_prepass(C.c_int64(n), C.c_int(scene.active_degree if deg is None else deg), _dp(_f64(scene.means)),
+                             _dp(_f64(scene.base_color)), _dp(_f64(pre)), _dp(_f64(scene.mlp_weights)), _dp(_f64(eye)),
+                             _dp(color))
+    return color
+
+
+def rgba8(color, opacity):
+    """The prepass output texel: colour clamped to [0,1] and opacity, each to 8 bits, round to nearest."""
+    c = np.clip(np.concatenate([np.asarray(color, np.float64), np.asarray(opacity, np.float64)[:, None]], 1), 0.0, 1.0)
+    return np.floor(c * 255.0 + 0.5).astype(np.uint8)
+
+
 def adam_step(param, grad, m, v, lr, beta1=0.9, beta2=0.999, eps=1e-15, step=1):
     """One Adam step with one learning rate per column (App. C.1).  param, grad, m, v: [rows, cols] (or
     [cols] for a single row); lr: [cols].  Returns new (param, m, v) as float64 arrays of the input shape."""
