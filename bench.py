@@ -253,6 +253,7 @@ def run_ours(args):
     # ---- appearance-decode sweep (separate-pass kernels, HBM resident)
     decode = None if (args.skip_decode or args.config != 3) else decode_sweep(api, torch, ctx, dev, peaks, args)
     adam = None if (args.skip_decode or args.config != 3) else adam_sweep(api, torch, ctx, dev, peaks, n)
+    prepass = None if (args.skip_decode or args.config != 3) else prepass_sweep(api, torch, ctx, dev, peaks, args, scenes)
 
     if rank != 0:
         return
@@ -289,6 +290,7 @@ def run_ours(args):
             "stages_ms_per_step": {k: round(v, 4) for k, v in results["sh"]["stage_ms"].items() if v > 0}},
         "appearance_decode": decode,
         "adam_update": adam,
+        "viewer_prepass": prepass,
         "peaks": peaks,
     }
     if not args.skip_cpu:
@@ -434,6 +436,43 @@ def adam_sweep(api, torch, ctx, dev, peaks, n):
         del tensors
     out["n"] = n
     out["cache"] = "tensors larger than L2 (352 MB neural, 944 MB SH at 1M)"
+    return out
+
+
+def prepass_sweep(api, torch, ctx, dev, peaks, args, scenes):
+    """The viewer's per-frame colour prepass of the neural model (560 MAC per Gaussian on tensor cores, one RGBA8
+    texel out) and its one-off export fold, at 1M / 3M / 10M Gaussians.  64 B move per Gaussian and frame."""
+    out = {}
+    sizes = [1_000_000, 3_000_000, 10_000_000] if not args.quick else [1_000_000]
+    cam = api.make_camera(scenes.orbit_cameras(WIDTH, HEIGHT, 8)[1])
+    flush = torch.empty(64 * 1024 * 1024, device=dev, dtype=torch.float32)
+    for n in sizes:
+        sc, _, _ = scenes.config5(n, scenes.APP_NEURAL)
+        ds = api.upload_scene(sc, dev)
+        pre = torch.empty((n, 16), device=dev, dtype=torch.float16)
+        rgba = torch.empty((n, 4), device=dev, dtype=torch.uint8)
+        api.gs_neural_fold(ctx, ds, pre)
+        for _ in range(3):
+            api.gs_neural_prepass(ctx, ds, pre, cam, rgba)
+        torch.cuda.synchronize()
+        t_fold = t_pre = 0.0
+        reps = 10
+        for _ in range(reps):
+            flush.zero_()
+            e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+            e0.record(); api.gs_neural_fold(ctx, ds, pre); e1.record()
+            flush.zero_()
+            e0b = torch.cuda.Event(enable_timing=True); e0b.record()
+            api.gs_neural_prepass(ctx, ds, pre, cam, rgba); e2.record()
+            torch.cuda.synchronize()
+            t_fold += e0.elapsed_time(e1); t_pre += e0b.elapsed_time(e2)
+        ms = t_pre / reps
+        gbs = 64.0 * n / (ms * 1e-3) / 1e9
+        out[f"{n // 1_000_000}M"] = {"prepass_ms": round(ms, 4), "fold_ms": round(t_fold / reps, 4), "bytes_per_gaussian": 64,
+                                      "GBps": round(gbs, 1), "frac_of_hbm_peak": round(gbs / peaks["hbm_gbs"], 4),
+                                      "Ggaussians_per_s": round(n / (ms * 1e-3) / 1e9, 3), "mac_per_gaussian": 560}
+        del ds, pre, rgba
+    out["cache"] = "L2 flushed between iterations (256 MiB write)"
     return out
 
 

@@ -235,6 +235,26 @@ typedef struct {
  * GS_ERR_CAPACITY if a tensor has 2^32 elements or more. */
 GsStatus gs_adam_step(GsContext *ctx, const GsAdamTensor *tensors, int32_t num_tensors, int64_t step, void *stream);
 
+/* ---- NEXT: the viewer's colour prepass of the neural model as CUDA kernels (App. C.3, "Neural") --
+ * Export: gs_neural_fold folds the 17 view-independent columns of the decoder's first layer (the 16
+ * encoded feature inputs and the constant degree-0 input) into 16 half-precision pre-activations per
+ * Gaussian, stored in place of the features' encodings (32 B per Gaussian).  scene->features,
+ * scene->mlp_weights and preact [n,16] (IEEE fp16 bits, 16-byte aligned) are device pointers.
+ *
+ * Per frame: gs_neural_prepass evaluates what depends on the view - the 15 direction columns of the
+ * first layer (SH degrees 1..active_degree of d = normalize(mean - camera centre)), the second and
+ * the output layer, 560 instead of 816 multiply-accumulates per Gaussian - in half precision with
+ * fp32 accumulation, composes the residual with the base colour, c = max(0, c0 + 0.5 + tanh(.)), and
+ * writes one texel per Gaussian: rgba [n,4] bytes = (c clamped to [0,1], sigmoid(opacity logit)),
+ * each times 255 and rounded to nearest.  color (optional, may be NULL) receives the unquantised
+ * colour [n,3] fp32.  Uses scene->n, means, opacity_logits, base_color, mlp_weights, active_degree
+ * (0 disables the residual); of the camera only its centre matters.  Asynchronous on `stream`;
+ * GS_ERR_INVALID_ARG for NULL or misaligned pointers, GS_ERR_UNSUPPORTED for a scene that is not
+ * GS_APP_NEURAL.  The WebGL viewer itself is out of reach here; this is its shader arithmetic. */
+GsStatus gs_neural_fold(GsContext *ctx, const GsScene *scene, uint16_t *preact, void *stream);
+GsStatus gs_neural_prepass(GsContext *ctx, const GsScene *scene, const uint16_t *preact, const GsCamera *cam,
+                           uint8_t *rgba, float *color, void *stream);
+
 /* Per-stage device timing, for benchmarks (the paper gives wall-clock protocols only, App. C; this
  * is the measurement hook of this library).  While enabled, every stage the library launches is
  * bracketed by CUDA events on the caller's stream.  gs_profile_collect synchronises those events,
@@ -254,6 +274,7 @@ typedef enum {
   GS_STAGE_APPEARANCE_FWD,     /* separate-pass decode                                          */
   GS_STAGE_APPEARANCE_BWD,
   GS_STAGE_ADAM,               /* fused parameter update                                        */
+  GS_STAGE_PREPASS,            /* viewer-side fold / colour prepass                             */
   GS_NUM_STAGES
 } GsStage;
 GsStatus gs_profile_enable(GsContext *ctx, int enable);

@@ -82,7 +82,7 @@ _lib.gs_appearance_backward.restype = C.c_int
 
 
 STAGES = ["preprocess_fwd", "depth_sort", "tile_offsets", "keygen", "tile_sort", "tile_ranges", "blend_fwd",
-          "blend_bwd", "preprocess_bwd", "appearance_fwd", "appearance_bwd", "adam"]
+          "blend_bwd", "preprocess_bwd", "appearance_fwd", "appearance_bwd", "adam", "prepass"]
 _lib.gs_profile_enable.argtypes = [_vp, C.c_int]
 _lib.gs_profile_enable.restype = C.c_int
 _lib.gs_profile_collect.argtypes = [_vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
@@ -105,6 +105,10 @@ class GsAdamTensor(C.Structure):
 
 _lib.gs_adam_step.argtypes = [_vp, C.POINTER(GsAdamTensor), C.c_int32, C.c_int64, _vp]
 _lib.gs_adam_step.restype = C.c_int
+_lib.gs_neural_fold.argtypes = [_vp, C.POINTER(GsScene), _vp, _vp]
+_lib.gs_neural_fold.restype = C.c_int
+_lib.gs_neural_prepass.argtypes = [_vp, C.POINTER(GsScene), _vp, C.POINTER(GsCamera), _vp, _vp, _vp]
+_lib.gs_neural_prepass.restype = C.c_int
 
 
 class GsError(RuntimeError):
@@ -381,6 +385,23 @@ class Renderer:
         gs_render_backward(self.ctx, scene, cam, self.proj, self.binning, self.num_pairs, self.final_T,
                            self.n_contrib, dL_dimage, self.grads, self.workspace, stream)
         return self.grads
+
+
+# ------------------------------------------------------------------------------------------------
+# Viewer-side colour prepass of the neural model
+# ------------------------------------------------------------------------------------------------
+def gs_neural_fold(ctx: Context, scene: "DeviceScene", preact: torch.Tensor, stream=None) -> None:
+    """preact: [n,16] float16 tensor that receives the folded first-layer pre-activations."""
+    cs = scene.c_struct()
+    ctx._check(_lib.gs_neural_fold(ctx._h, C.byref(cs), _ptr(preact), _stream_handle(stream)))
+
+
+def gs_neural_prepass(ctx: Context, scene: "DeviceScene", preact: torch.Tensor, cam: GsCamera, rgba: torch.Tensor,
+                      color: Optional[torch.Tensor] = None, stream=None) -> None:
+    """rgba: [n,4] uint8 texels; color: optional [n,3] float32 unquantised colour."""
+    cs = scene.c_struct()
+    ctx._check(_lib.gs_neural_prepass(ctx._h, C.byref(cs), _ptr(preact), C.byref(cam), _ptr(rgba), _ptr(color),
+                                      _stream_handle(stream)))
 
 
 # ------------------------------------------------------------------------------------------------

@@ -460,6 +460,45 @@ GsStatus gs_adam_step(GsContext *ctx, const GsAdamTensor *tensors, int32_t num_t
   return check_cuda(ctx, cudaGetLastError(), "adam launch");
 }
 
+GsStatus gs_neural_fold(GsContext *ctx, const GsScene *scene, uint16_t *preact, void *stream) {
+  if (!ctx) return GS_ERR_INVALID_ARG;
+  if (!scene || scene->n < 0) return fail(ctx, GS_ERR_INVALID_ARG, "scene is NULL or n < 0");
+  if (scene->app != GS_APP_NEURAL) return fail(ctx, GS_ERR_UNSUPPORTED, "the fold exists for the neural model only");
+  if (scene->n == 0) return GS_OK;
+  if (bad_ptr(scene->features) || bad_ptr(scene->mlp_weights) || bad_ptr(preact))
+    return fail(ctx, GS_ERR_INVALID_ARG, "features, mlp_weights or preact is NULL or misaligned");
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaSetDevice(ctx->device);
+  {
+    StageTimer t(ctx, GS_STAGE_PREPASS, s);
+    t.done(launch_neural_fold(scene->n, reinterpret_cast<const __half *>(scene->features),
+                              reinterpret_cast<const __half *>(scene->mlp_weights), reinterpret_cast<__half *>(preact), s));
+  }
+  return check_cuda(ctx, cudaGetLastError(), "neural fold launch");
+}
+
+GsStatus gs_neural_prepass(GsContext *ctx, const GsScene *scene, const uint16_t *preact, const GsCamera *cam,
+                           uint8_t *rgba, float *color, void *stream) {
+  if (!ctx) return GS_ERR_INVALID_ARG;
+  if (!scene || scene->n < 0 || !cam) return fail(ctx, GS_ERR_INVALID_ARG, "scene or cam is NULL, or n < 0");
+  if (scene->app != GS_APP_NEURAL) return fail(ctx, GS_ERR_UNSUPPORTED, "the prepass exists for the neural model only");
+  if (scene->active_degree < 0 || scene->active_degree > 3) return fail(ctx, GS_ERR_INVALID_ARG, "active_degree outside 0..3");
+  if (scene->n == 0) return GS_OK;
+  if (bad_ptr(scene->means) || bad_ptr(scene->opacity_logits) || bad_ptr(scene->base_color) || bad_ptr(scene->mlp_weights) ||
+      bad_ptr(preact) || !rgba || (reinterpret_cast<uintptr_t>(rgba) & 3u) || (color && !aligned16(color)))
+    return fail(ctx, GS_ERR_INVALID_ARG, "a prepass pointer is NULL or misaligned");
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaSetDevice(ctx->device);
+  const CamDev cd = make_cam(cam);
+  {
+    StageTimer t(ctx, GS_STAGE_PREPASS, s);
+    t.done(launch_neural_prepass(scene->n, scene->active_degree, scene->means, scene->opacity_logits, scene->base_color,
+                                 reinterpret_cast<const __half *>(preact), reinterpret_cast<const __half *>(scene->mlp_weights),
+                                 cd.oc, rgba, color, s));
+  }
+  return check_cuda(ctx, cudaGetLastError(), "neural prepass launch");
+}
+
 GsStatus gs_profile_enable(GsContext *ctx, int enable) {
   if (!ctx) return GS_ERR_INVALID_ARG;
   ctx->profiling = enable != 0;

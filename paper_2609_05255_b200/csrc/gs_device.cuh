@@ -95,6 +95,10 @@ int launch_blend_bwd(const CamDev &cam, const uint32_t *ranges, const uint32_t *
                       const float *final_T, const uint32_t *n_contrib, const float *dL_dimage,
                       float *g2d, cudaStream_t st);
 
+int launch_neural_fold(int64_t n, const __half *features, const __half *weights, __half *preact, cudaStream_t st);
+int launch_neural_prepass(int64_t n, int deg, const float *means, const float *logits, const float *base_color,
+                          const __half *preact, const __half *weights, const float eye[3], uint8_t *rgba, float *color,
+                          cudaStream_t st);
 int launch_adam(const GsAdamTensor *tensors, int num_tensors, int64_t step, int num_sms, cudaStream_t st);
 int launch_blend_count(const CamDev &cam, const uint32_t *ranges, const uint32_t *vals, const float *mean2d,
                        const float *conic_opacity, const float *color, unsigned long long *counts, cudaStream_t st);
