@@ -74,7 +74,7 @@ __global__ void __launch_bounds__(kPrepassThreads) k_neural_prepass(int64_t n, i
                                                                     float ez, uchar4 *__restrict__ rgba,
                                                                     float *__restrict__ color) {
   __shared__ uint32_t s_x[kPrepassWarps][32][kXRow];
-  __shared__ float4 s_c[kPrepassWarps][32];
+  __shared__ float s_y[kPrepassWarps][32][3];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, t = lane & 3;
   // B fragments: B[k][nn] = W[nn][k]; b0 holds k = 2t, 2t+1 and b1 k = 2t+8, 2t+9 of column nn = 8 nt + g.
   // Layer 1 keeps only the direction columns 1..15 (column 0 is the folded constant: its weight is dropped).
@@ -96,11 +96,11 @@ __global__ void __launch_bounds__(kPrepassThreads) k_neural_prepass(int64_t n, i
   if (row0 >= n) return;
   const int64_t i = row0 + lane;
   // ---- this lane's Gaussian: direction, direction inputs, base colour, alpha
+  float4 c = make_float4(0.f, 0.f, 0.f, 0.f);   // base colour and the alpha texel value
   {
     float Y[16];
 #pragma unroll
     for (int k = 0; k < 16; ++k) Y[k] = 0.f;
-    float4 c = make_float4(0.f, 0.f, 0.f, 0.f);
     if (i < n) {
       const float dx = __ldg(means + 3 * i) - ex, dy = __ldg(means + 3 * i + 1) - ey, dz = __ldg(means + 3 * i + 2) - ez;
       const float inv = rsqrtf(fmaf(dx, dx, fmaf(dy, dy, dz * dz)));
@@ -113,7 +113,6 @@ __global__ void __launch_bounds__(kPrepassThreads) k_neural_prepass(int64_t n, i
 #pragma unroll
     for (int k = 0; k < 8; ++k)
       s_x[warp][lane][k] = pack_half2(2 * k < na ? Y[2 * k] : 0.f, 2 * k + 1 < na ? Y[2 * k + 1] : 0.f);
-    s_c[warp][lane] = c;
   }
   __syncwarp();
   float y[2][4];
@@ -147,30 +146,31 @@ __global__ void __launch_bounds__(kPrepassThreads) k_neural_prepass(int64_t n, i
     y[mt][0] = y[mt][1] = y[mt][2] = y[mt][3] = 0.f;
     mlp::mma16816(y[mt], a, w3b0, w3b1);
   }
-  // ---- colour and texel: lanes with t = 0 hold outputs 0, 1 of rows g and g + 8; output 2 sits in lane t = 1
+  // ---- the three outputs go back from the fragment layout (lanes t = 0 hold outputs 0, 1 of rows g and
+  // g + 8, lanes t = 1 output 2) to one row per lane, so that every lane finishes its own Gaussian
 #pragma unroll
   for (int mt = 0; mt < 2; ++mt) {
-    const float b_lo = __shfl_down_sync(kFull, y[mt][0], 1), b_hi = __shfl_down_sync(kFull, y[mt][2], 1);
     if (t == 0) {
-#pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        const int r = mt * 16 + g + 8 * half;
-        if (row0 + r < n) {
-          const float4 c = s_c[warp][r];
-          float A[3] = {half ? y[mt][2] : y[mt][0], half ? y[mt][3] : y[mt][1], half ? b_hi : b_lo};
-          float col[3];
-          unsigned q[3];
-#pragma unroll
-          for (int ch = 0; ch < 3; ++ch) {
-            const float res = deg > 0 ? tanhf(A[ch]) : 0.f;
-            col[ch] = fmaxf((ch == 0 ? c.x : ch == 1 ? c.y : c.z) + 0.5f + res, 0.f);
-            q[ch] = (unsigned)floorf(fmaf(fminf(col[ch], 1.f), 255.f, 0.5f));
-          }
-          rgba[row0 + r] = make_uchar4((unsigned char)q[0], (unsigned char)q[1], (unsigned char)q[2], (unsigned char)c.w);
-          if (color) { color[3 * (row0 + r)] = col[0]; color[3 * (row0 + r) + 1] = col[1]; color[3 * (row0 + r) + 2] = col[2]; }
-        }
-      }
+      s_y[warp][mt * 16 + g][0] = y[mt][0]; s_y[warp][mt * 16 + g][1] = y[mt][1];
+      s_y[warp][mt * 16 + g + 8][0] = y[mt][2]; s_y[warp][mt * 16 + g + 8][1] = y[mt][3];
+    } else if (t == 1) {
+      s_y[warp][mt * 16 + g][2] = y[mt][0];
+      s_y[warp][mt * 16 + g + 8][2] = y[mt][2];
     }
+  }
+  __syncwarp();
+  if (i < n) {
+    float col[3];
+    unsigned q[3];
+#pragma unroll
+    for (int ch = 0; ch < 3; ++ch) {
+      // tanh(a) = 1 - 2 / (exp(2a) + 1); the fast exponential and division are far inside the texel's step
+      const float res = deg > 0 ? 1.f - __fdividef(2.f, __expf(2.f * s_y[warp][lane][ch]) + 1.f) : 0.f;
+      col[ch] = fmaxf((ch == 0 ? c.x : ch == 1 ? c.y : c.z) + 0.5f + res, 0.f);
+      q[ch] = (unsigned)floorf(fmaf(fminf(col[ch], 1.f), 255.f, 0.5f));
+    }
+    rgba[i] = make_uchar4((unsigned char)q[0], (unsigned char)q[1], (unsigned char)q[2], (unsigned char)c.w);
+    if (color) { color[3 * i] = col[0]; color[3 * i + 1] = col[1]; color[3 * i + 2] = col[2]; }
   }
 }
 
