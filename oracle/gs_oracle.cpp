@@ -127,6 +127,26 @@ struct MlpState {
   double x[kIn], h1[kHid], h2[kHid], y[kOut], A[kOut];
 };
 
+// Colour activations of Sec. 3.1, as functions of x = c0 + A(d).  All map 0 to (about) 0.5 with slope
+// (about) 1:  0: ReLU(x + 0.5)   1: softplus(x + 0.5), beta = 10   2: sigmoid(4 x)   3: clamp(x + 0.5, 0, 1).
+// The derivative at a kink is the one-sided value 0.
+double color_act(int act, double x) {
+  switch (act) {
+    case 1: { const double z = 10.0 * (x + 0.5); return (z > 30 ? z : std::log1p(std::exp(z))) / 10.0; }
+    case 2: return 1.0 / (1.0 + std::exp(-4.0 * x));
+    case 3: { const double z = x + 0.5; return z < 0 ? 0.0 : (z > 1 ? 1.0 : z); }
+    default: { const double z = x + 0.5; return z > 0 ? z : 0.0; }
+  }
+}
+double color_act_grad(int act, double x) {
+  switch (act) {
+    case 1: return 1.0 / (1.0 + std::exp(-10.0 * (x + 0.5)));
+    case 2: { const double y = 1.0 / (1.0 + std::exp(-4.0 * x)); return 4.0 * y * (1.0 - y); }
+    case 3: { const double z = x + 0.5; return (z > 0 && z < 1) ? 1.0 : 0.0; }
+    default: return (x + 0.5) > 0 ? 1.0 : 0.0;
+  }
+}
+
 // Eq. 5-7: x = (Y_0..15(d) masked by the active degree, (sin f_j, cos f_j)_j); two ReLU
 // layers; A = tanh(W3 h2).
 void mlp_forward(const double* W, const double d[3], const double* f, int deg, MlpState& s) {
@@ -210,9 +230,9 @@ void gso_neural_fold(int64_t n, const double* features, const double* weights, d
 
 // Per frame: only the 15 direction-dependent columns (SH degrees 1..3, masked by the active degree)
 // of the first layer remain, 15 (padded to 16) x 16 + 16 x 16 + 16 x 3 = 560 multiply-accumulates:
-//   h1 = ReLU(pre + W1[:, 1..15] Y_1..15(d)); h2 = ReLU(W2 h1); A = tanh(W3 h2); c = ReLU(c0 + 0.5 + A).
+//   h1 = ReLU(pre + W1[:, 1..15] Y_1..15(d)); h2 = ReLU(W2 h1); A = tanh(W3 h2); c = phi(c0 + A).
 // d = (mean - eye) / |mean - eye|.
-void gso_neural_prepass(int64_t n, int deg, const double* means, const double* base_color, const double* pre,
+void gso_neural_prepass(int64_t n, int deg, int act, const double* means, const double* base_color, const double* pre,
                         const double* weights, const double* eye, double* color) {
   const int na = num_active(deg);
 #pragma omp parallel for schedule(static)
@@ -241,8 +261,7 @@ void gso_neural_prepass(int64_t n, int deg, const double* means, const double* b
       }
     }
     for (int c = 0; c < 3; ++c) {
-      const double v = base_color[3 * i + c] + 0.5 + A[c];
-      color[3 * i + c] = v > 0 ? v : 0;
+      color[3 * i + c] = color_act(act, base_color[3 * i + c] + A[c]);
     }
   }
 }
@@ -377,7 +396,7 @@ void gso_preprocess(int64_t n, const double* means, const double* log_scales, co
 // sh_rest is [n,15,3]; features [n,8]; weights [816] = W1[16][32], W2[16][16], W3[3][16].
 // residual_out (may be null) receives A(d).
 // ---------------------------------------------------------------------------------------
-void gso_appearance_forward(int64_t n, int app, int deg, const double* base_color,
+void gso_appearance_forward(int64_t n, int app, int deg, int act, const double* base_color,
                             const double* sh_rest, const double* features, const double* weights,
                             const double* dirs, const uint8_t* mask, double* color,
                             double* residual_out) {
@@ -398,8 +417,7 @@ void gso_appearance_forward(int64_t n, int app, int deg, const double* base_colo
       for (int c = 0; c < 3; ++c) A[c] = s.A[c];
     }
     for (int c = 0; c < 3; ++c) {
-      const double pre = base_color[3 * i + c] + 0.5 + A[c];
-      color[3 * i + c] = pre > 0 ? pre : 0;
+      color[3 * i + c] = color_act(act, base_color[3 * i + c] + A[c]);
       if (residual_out) residual_out[3 * i + c] = A[c];
     }
   }
@@ -408,7 +426,7 @@ void gso_appearance_forward(int64_t n, int app, int deg, const double* base_colo
 // Backward of the decode.  g_color = dL/dc.  Outputs: g_base[n,3], g_sh_rest[n,15,3] or
 // g_features[n,8], g_weights[816] (sum over Gaussians in index order), g_dirs[n,3] (gradient
 // with respect to the direction as a free R^3 vector).
-void gso_appearance_backward(int64_t n, int app, int deg, const double* base_color,
+void gso_appearance_backward(int64_t n, int app, int deg, int act, const double* base_color,
                              const double* sh_rest, const double* features, const double* weights,
                              const double* dirs, const uint8_t* mask, const double* g_color,
                              double* g_base, double* g_sh_rest, double* g_features,
@@ -444,8 +462,7 @@ void gso_appearance_backward(int64_t n, int app, int deg, const double* base_col
         for (int k = 1; k < na; ++k)
           for (int c = 0; c < 3; ++c) A[c] += Y[k] * sh_rest[(i * 15 + (k - 1)) * 3 + c];
         for (int c = 0; c < 3; ++c) {
-          const double pre = base_color[3 * i + c] + 0.5 + A[c];
-          const double gp = pre > 0 ? g_color[3 * i + c] : 0.0;
+          const double gp = color_act_grad(act, base_color[3 * i + c] + A[c]) * g_color[3 * i + c];
           g_base[3 * i + c] = gp;
           for (int k = 1; k < na; ++k) {
             g_sh_rest[(i * 15 + (k - 1)) * 3 + c] = Y[k] * gp;
@@ -456,8 +473,7 @@ void gso_appearance_backward(int64_t n, int app, int deg, const double* base_col
       } else {
         if (deg == 0) {
           for (int c = 0; c < 3; ++c) {
-            const double pre = base_color[3 * i + c] + 0.5;
-            g_base[3 * i + c] = pre > 0 ? g_color[3 * i + c] : 0.0;
+            g_base[3 * i + c] = color_act_grad(act, base_color[3 * i + c]) * g_color[3 * i + c];
           }
           continue;
         }
@@ -466,8 +482,7 @@ void gso_appearance_backward(int64_t n, int app, int deg, const double* base_col
         double* gw = gw_rows.data() + ii * kNumW;
         double gy[kOut], gh2[kHid], gh1[kHid], gx[kIn];
         for (int c = 0; c < 3; ++c) {
-          const double pre = base_color[3 * i + c] + 0.5 + s.A[c];
-          const double gp = pre > 0 ? g_color[3 * i + c] : 0.0;
+          const double gp = color_act_grad(act, base_color[3 * i + c] + s.A[c]) * g_color[3 * i + c];
           g_base[3 * i + c] = gp;
           gy[c] = gp * (1.0 - s.A[c] * s.A[c]);
         }
@@ -965,3 +980,8 @@ void gso_preprocess_backward(int64_t n, const double* means, const double* log_s
 }
 
 }  // extern "C"
+
+extern "C" {
+double gso_color_act(int act, double x) { return color_act(act, x); }
+double gso_color_act_grad(int act, double x) { return color_act_grad(act, x); }
+}

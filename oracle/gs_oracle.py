@@ -103,6 +103,27 @@ def num_mlp_weights() -> int:
     return lib().gso_num_mlp_weights()
 
 
+ACT_RELU, ACT_SOFTPLUS, ACT_SIGMOID, ACT_HARD_SIGMOID = 0, 1, 2, 3
+
+
+def _act(scene) -> int:
+    return int(getattr(scene, "color_activation", 0))
+
+
+def color_act(act: int, x: float) -> float:
+    """phi(x), x = c0 + A(d) (Sec. 3.1): 0 ReLU(x + 0.5), 1 softplus(x + 0.5) with beta = 10, 2 sigmoid(4x),
+    3 clamp(x + 0.5, 0, 1)."""
+    f = lib().gso_color_act
+    f.restype = C.c_double
+    return float(f(C.c_int(act), C.c_double(x)))
+
+
+def color_act_grad(act: int, x: float) -> float:
+    f = lib().gso_color_act_grad
+    f.restype = C.c_double
+    return float(f(C.c_int(act), C.c_double(x)))
+
+
 def neural_fold(scene):
     """Export step of the viewer (App. C.3): [n,16] pre-activations of the first layer from the features,
     the constant degree-0 input and their 17 weight columns, in double (not yet rounded to fp16)."""
@@ -116,7 +137,8 @@ def neural_prepass(scene, pre, eye, deg=None):
     """Per-frame colour of every Gaussian from the folded pre-activations and the camera position `eye`."""
     n = scene.means.shape[0]
     color = np.zeros((n, 3))
-    lib().gso_neural_prepass(C.c_int64(n), C.c_int(scene.active_degree if deg is None else deg), _dp(_f64(scene.means)),
+    lib().gso_neural_prepass(C.c_int64(n), C.c_int(scene.active_degree if deg is None else deg), C.c_int(_act(scene)),
+                             _dp(_f64(scene.means)),
                              _dp(_f64(scene.base_color)), _dp(_f64(pre)), _dp(_f64(scene.mlp_weights)), _dp(_f64(eye)),
                              _dp(color))
     return color
@@ -170,7 +192,7 @@ def appearance_forward(scene, dirs, mask=None, deg=None):
     color, resid = np.zeros((n, 3)), np.zeros((n, 3))
     deg = scene.active_degree if deg is None else deg
     m = None if mask is None else np.ascontiguousarray(mask, np.uint8)
-    lib().gso_appearance_forward(C.c_int64(n), C.c_int(scene.app), C.c_int(deg), _dp(base), _dp(sh),
+    lib().gso_appearance_forward(C.c_int64(n), C.c_int(scene.app), C.c_int(deg), C.c_int(_act(scene)), _dp(base), _dp(sh),
                                  _dp(ft), _dp(wt), _dp(dirs), _p(m, C.c_uint8), _dp(color), _dp(resid))
     return color, resid
 
@@ -186,7 +208,7 @@ def appearance_backward(scene, dirs, g_color, mask=None, deg=None):
         o.sh_rest = np.zeros((n, 15, 3))
     else:
         o.features = np.zeros((n, 8)); o.mlp_weights = np.zeros(num_mlp_weights())
-    lib().gso_appearance_backward(C.c_int64(n), C.c_int(scene.app), C.c_int(deg), _dp(base), _dp(sh),
+    lib().gso_appearance_backward(C.c_int64(n), C.c_int(scene.app), C.c_int(deg), C.c_int(_act(scene)), _dp(base), _dp(sh),
                                   _dp(ft), _dp(wt), _dp(dirs), _p(m, C.c_uint8), _dp(g_color),
                                   _dp(o.base_color), _dp(o.sh_rest), _dp(o.features),
                                   _dp(o.mlp_weights), _dp(o.dirs))

@@ -55,6 +55,7 @@ class Scene:
     sh_rest: Optional[np.ndarray] = None      # [n,15,3] f32
     features: Optional[np.ndarray] = None     # [n,8]  f16
     mlp_weights: Optional[np.ndarray] = None  # [816]  f16: W1[16][32], W2[16][16], W3[3][16]
+    color_activation: int = 0                 # 0 ReLU(x+0.5), 1 softplus(x+0.5) beta 10, 2 sigmoid(4x), 3 clamp(x+0.5,0,1)
 
     @property
     def n(self) -> int:
