@@ -53,6 +53,15 @@ enum {
   GS_MLP_WEIGHTS = 816     /* 32*16 + 16*16 + 16*3, no biases (Sec. 4)                          */
 };
 
+/* Colour activation phi of Sec. 3.1, applied to x = c0 + A(d).  All four map 0 to (about) 0.5 with slope
+ * (about) 1 there; the paper uses the first unless it says otherwise. */
+typedef enum {
+  GS_ACT_RELU = 0,         /* ReLU(x + 0.5), the standard one                                   */
+  GS_ACT_SOFTPLUS = 1,     /* softplus(x + 0.5) with beta = 10                                  */
+  GS_ACT_SIGMOID = 2,      /* sigmoid(4 x)                                                      */
+  GS_ACT_HARD_SIGMOID = 3  /* clamp(x + 0.5, 0, 1)                                              */
+} GsColorActivation;
+
 /* Pinhole camera (host struct). */
 typedef struct {
   int32_t width, height;        /* pixels                                                      */
@@ -79,6 +88,7 @@ typedef struct {
                                     each row-major (out, in); input order = 16 SH basis values
                                     of the direction, then (sin f_j, cos f_j) per feature
                                     (Eq. 5, Eq. 6 with k = 1)                                  */
+  int32_t color_activation;      /* GsColorActivation: phi of c = phi(c0 + A(d)) (Sec. 3.1)    */
 } GsScene;
 
 /* Per-Gaussian results of gs_preprocess (caller-allocated device buffers). */

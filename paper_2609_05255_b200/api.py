@@ -39,7 +39,7 @@ class GsCamera(C.Structure):
 class GsScene(C.Structure):
     _fields_ = [("n", C.c_int64), ("means", _vp), ("log_scales", _vp), ("quats", _vp), ("opacity_logits", _vp),
                 ("base_color", _vp), ("app", C.c_int32), ("active_degree", C.c_int32), ("sh_rest", _vp),
-                ("features", _vp), ("mlp_weights", _vp)]
+                ("features", _vp), ("mlp_weights", _vp), ("color_activation", C.c_int32)]
 
 
 class GsProjected(C.Structure):
@@ -153,6 +153,7 @@ class DeviceScene:
     sh_rest: Optional[torch.Tensor] = None
     features: Optional[torch.Tensor] = None
     mlp_weights: Optional[torch.Tensor] = None
+    color_activation: int = 0        # GS_ACT_*: 0 ReLU(x+0.5), 1 softplus beta 10, 2 sigmoid(4x), 3 clamp(x+0.5, 0, 1)
 
     @property
     def n(self) -> int:
@@ -165,6 +166,7 @@ class DeviceScene:
         s.opacity_logits, s.base_color = _ptr(self.opacity_logits), _ptr(self.base_color)
         s.app, s.active_degree = int(self.app), int(self.active_degree)
         s.sh_rest, s.features, s.mlp_weights = _ptr(self.sh_rest), _ptr(self.features), _ptr(self.mlp_weights)
+        s.color_activation = int(self.color_activation)
         return s
 
 
@@ -176,7 +178,7 @@ def upload_scene(scene, device="cuda") -> DeviceScene:
                        up(scene.quats, torch.float32), up(scene.opacity_logits, torch.float32),
                        up(scene.base_color, torch.float32), int(scene.app), int(scene.active_degree),
                        up(scene.sh_rest, torch.float32), up(scene.features, torch.float16),
-                       up(scene.mlp_weights, torch.float16))
+                       up(scene.mlp_weights, torch.float16), int(getattr(scene, "color_activation", 0)))
 
 
 @dataclass

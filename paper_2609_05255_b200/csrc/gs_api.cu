@@ -92,6 +92,8 @@ CamDev make_cam(const GsCamera *c) {
 GsStatus scene_appearance_ok(GsContext *ctx, const GsScene *s) {
   if (s->app != GS_APP_SH && s->app != GS_APP_NEURAL) return fail(ctx, GS_ERR_INVALID_ARG, "unknown appearance model");
   if (s->active_degree < 0 || s->active_degree > 3) return fail(ctx, GS_ERR_INVALID_ARG, "active_degree must be 0..3");
+  if (s->color_activation < GS_ACT_RELU || s->color_activation > GS_ACT_HARD_SIGMOID)
+    return fail(ctx, GS_ERR_INVALID_ARG, "unknown colour activation");
   if (s->n < 0) return fail(ctx, GS_ERR_INVALID_ARG, "n < 0");
   if (s->n == 0) return GS_OK;
   if (bad_ptr(s->base_color)) return fail(ctx, GS_ERR_INVALID_ARG, "base_color is NULL or misaligned");
@@ -224,7 +226,7 @@ GsStatus gs_preprocess(GsContext *ctx, const GsScene *scene, const GsCamera *cam
   a.base_color = scene->base_color; a.sh_rest = scene->sh_rest;
   a.features = reinterpret_cast<const __half *>(scene->features);
   a.weights = reinterpret_cast<const __half *>(scene->mlp_weights);
-  a.deg = scene->active_degree;
+  a.deg = scene->active_degree; a.act = scene->color_activation;
   a.mean2d = out->mean2d; a.conic_opacity = out->conic_opacity; a.color = out->color; a.extent = out->extent;
   a.depth_key = out->depth_key; a.rect = out->rect; a.tiles_touched = out->tiles_touched;
   a.pair_counter = ctx->d_counter;
@@ -345,7 +347,7 @@ GsStatus gs_render_backward(GsContext *ctx, const GsScene *scene, const GsCamera
   a.base_color = scene->base_color; a.sh_rest = scene->sh_rest;
   a.features = reinterpret_cast<const __half *>(scene->features);
   a.weights = reinterpret_cast<const __half *>(scene->mlp_weights);
-  a.deg = scene->active_degree;
+  a.deg = scene->active_degree; a.act = scene->color_activation;
   a.rect = proj->rect; a.g2d = g2d;
   a.g_means = grads->means; a.g_log_scales = grads->log_scales; a.g_quats = grads->quats;
   a.g_logits = grads->opacity_logits; a.g_base = grads->base_color; a.g_sh_rest = grads->sh_rest;
@@ -369,7 +371,7 @@ GsStatus gs_appearance_forward(GsContext *ctx, const GsScene *scene, const float
   cudaSetDevice(ctx->device);
   AppearanceArgs a;
   memset(&a, 0, sizeof(a));
-  a.n = scene->n; a.deg = scene->active_degree;
+  a.n = scene->n; a.deg = scene->active_degree; a.act = scene->color_activation;
   a.base_color = scene->base_color; a.sh_rest = scene->sh_rest; a.dirs = dirs;
   a.features = reinterpret_cast<const __half *>(scene->features);
   a.weights = reinterpret_cast<const __half *>(scene->mlp_weights);
@@ -402,7 +404,7 @@ GsStatus gs_appearance_backward(GsContext *ctx, const GsScene *scene, const floa
   if (scene->app == GS_APP_NEURAL && bad_ptr(grads->features)) return fail(ctx, GS_ERR_INVALID_ARG, "grads->features is NULL or misaligned");
   AppearanceArgs a;
   memset(&a, 0, sizeof(a));
-  a.n = scene->n; a.deg = scene->active_degree;
+  a.n = scene->n; a.deg = scene->active_degree; a.act = scene->color_activation;
   a.base_color = scene->base_color; a.sh_rest = scene->sh_rest; a.dirs = dirs;
   a.features = reinterpret_cast<const __half *>(scene->features);
   a.weights = reinterpret_cast<const __half *>(scene->mlp_weights);
@@ -483,6 +485,8 @@ GsStatus gs_neural_prepass(GsContext *ctx, const GsScene *scene, const uint16_t 
   if (!scene || scene->n < 0 || !cam) return fail(ctx, GS_ERR_INVALID_ARG, "scene or cam is NULL, or n < 0");
   if (scene->app != GS_APP_NEURAL) return fail(ctx, GS_ERR_UNSUPPORTED, "the prepass exists for the neural model only");
   if (scene->active_degree < 0 || scene->active_degree > 3) return fail(ctx, GS_ERR_INVALID_ARG, "active_degree outside 0..3");
+  if (scene->color_activation < GS_ACT_RELU || scene->color_activation > GS_ACT_HARD_SIGMOID)
+    return fail(ctx, GS_ERR_INVALID_ARG, "unknown colour activation");
   if (scene->n == 0) return GS_OK;
   if (bad_ptr(scene->means) || bad_ptr(scene->opacity_logits) || bad_ptr(scene->base_color) || bad_ptr(scene->mlp_weights) ||
       bad_ptr(preact) || !rgba || (reinterpret_cast<uintptr_t>(rgba) & 3u) || (color && !aligned16(color)))
@@ -492,7 +496,7 @@ GsStatus gs_neural_prepass(GsContext *ctx, const GsScene *scene, const uint16_t 
   const CamDev cd = make_cam(cam);
   {
     StageTimer t(ctx, GS_STAGE_PREPASS, s);
-    t.done(launch_neural_prepass(scene->n, scene->active_degree, scene->means, scene->opacity_logits, scene->base_color,
+    t.done(launch_neural_prepass(scene->n, scene->active_degree, scene->color_activation, scene->means, scene->opacity_logits, scene->base_color,
                                  reinterpret_cast<const __half *>(preact), reinterpret_cast<const __half *>(scene->mlp_weights),
                                  cd.oc, rgba, color, s));
   }

@@ -34,7 +34,7 @@ struct PreprocessArgs {
   int64_t n;
   const float *means, *log_scales, *quats, *logits, *base_color, *sh_rest;
   const __half *features, *weights;
-  int deg;
+  int deg, act;
   float *mean2d, *conic_opacity, *color, *extent;
   uint32_t *depth_key, *tiles_touched;
   uint16_t *rect;
@@ -46,7 +46,7 @@ struct PreprocessBwdArgs {
   int64_t n;
   const float *means, *log_scales, *quats, *logits, *base_color, *sh_rest;
   const __half *features, *weights;
-  int deg;
+  int deg, act;
   const uint16_t *rect;
   const float *g2d;            // [n,12]: dL/dcolor(3), dL/dopacity, dL/dconic(3), dL/dmean2d(2), pad
   float *g_means, *g_log_scales, *g_quats, *g_logits, *g_base, *g_sh_rest, *g_features;
@@ -57,7 +57,7 @@ int launch_preprocess_bwd(int app, const PreprocessBwdArgs &a, const CamDev &cam
 
 struct AppearanceArgs {
   int64_t n;
-  int deg;
+  int deg, act;
   const float *base_color, *sh_rest, *dirs;
   const __half *features, *weights;
   float *color;                // forward
@@ -96,7 +96,7 @@ int launch_blend_bwd(const CamDev &cam, const uint32_t *ranges, const uint32_t *
                       float *g2d, cudaStream_t st);
 
 int launch_neural_fold(int64_t n, const __half *features, const __half *weights, __half *preact, cudaStream_t st);
-int launch_neural_prepass(int64_t n, int deg, const float *means, const float *logits, const float *base_color,
+int launch_neural_prepass(int64_t n, int deg, int act, const float *means, const float *logits, const float *base_color,
                           const __half *preact, const __half *weights, const float eye[3], uint8_t *rgba, float *color,
                           cudaStream_t st);
 int launch_adam(const GsAdamTensor *tensors, int num_tensors, int64_t step, int num_sms, cudaStream_t st);
@@ -208,6 +208,21 @@ struct TileSpans {
     return c;
   }
 };
+
+// Colour activations (Sec. 3.1) of z = c0 + 0.5 + A(d) and their derivatives: 0 ReLU(z), 1 softplus(z) with
+// beta = 10, 2 sigmoid(4 (z - 0.5)), 3 clamp(z, 0, 1).  The derivative at a kink is 0.
+__device__ __forceinline__ float color_act_z(int act, float z) {
+  if (act == GS_ACT_SOFTPLUS) { const float t = 10.f * z; return t > 15.f ? z : 0.1f * log1pf(expf(t)); }
+  if (act == GS_ACT_SIGMOID) return 1.f / (1.f + expf(fmaf(-4.f, z, 2.f)));
+  if (act == GS_ACT_HARD_SIGMOID) return fminf(fmaxf(z, 0.f), 1.f);
+  return fmaxf(z, 0.f);
+}
+__device__ __forceinline__ float color_act_grad_z(int act, float z) {
+  if (act == GS_ACT_SOFTPLUS) return 1.f / (1.f + expf(-10.f * z));
+  if (act == GS_ACT_SIGMOID) { const float y = 1.f / (1.f + expf(fmaf(-4.f, z, 2.f))); return 4.f * y * (1.f - y); }
+  if (act == GS_ACT_HARD_SIGMOID) return (z > 0.f && z < 1.f) ? 1.f : 0.f;
+  return z > 0.f ? 1.f : 0.f;
+}
 
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;

@@ -66,7 +66,7 @@ __device__ __forceinline__ uint32_t pack_weights(const __half *w, int idx) {   /
 // One warp per 32 Gaussians.  Lane L prepares row L (direction, SH basis, base colour, alpha byte);
 // the rows reach the tensor-core fragment layout through a small shared-memory tile; the weights
 // live in ten registers per lane for the whole kernel.
-__global__ void __launch_bounds__(kPrepassThreads) k_neural_prepass(int64_t n, int deg, const float *__restrict__ means,
+__global__ void __launch_bounds__(kPrepassThreads) k_neural_prepass(int64_t n, int deg, int act, const float *__restrict__ means,
                                                                     const float *__restrict__ logits,
                                                                     const float *__restrict__ base_color,
                                                                     const __half *__restrict__ preact,
@@ -166,7 +166,7 @@ __global__ void __launch_bounds__(kPrepassThreads) k_neural_prepass(int64_t n, i
     for (int ch = 0; ch < 3; ++ch) {
       // tanh(a) = 1 - 2 / (exp(2a) + 1); the fast exponential and division are far inside the texel's step
       const float res = deg > 0 ? 1.f - __fdividef(2.f, __expf(2.f * s_y[warp][lane][ch]) + 1.f) : 0.f;
-      col[ch] = fmaxf((ch == 0 ? c.x : ch == 1 ? c.y : c.z) + 0.5f + res, 0.f);
+      col[ch] = color_act_z(act, (ch == 0 ? c.x : ch == 1 ? c.y : c.z) + 0.5f + res);
       q[ch] = (unsigned)floorf(fmaf(fminf(col[ch], 1.f), 255.f, 0.5f));
     }
     rgba[i] = make_uchar4((unsigned char)q[0], (unsigned char)q[1], (unsigned char)q[2], (unsigned char)c.w);
@@ -182,12 +182,12 @@ int launch_neural_fold(int64_t n, const __half *features, const __half *weights,
   return 1;
 }
 
-int launch_neural_prepass(int64_t n, int deg, const float *means, const float *logits, const float *base_color,
+int launch_neural_prepass(int64_t n, int deg, int act, const float *means, const float *logits, const float *base_color,
                           const __half *preact, const __half *weights, const float eye[3], uint8_t *rgba, float *color,
                           cudaStream_t st) {
   if (n <= 0) return 0;
   k_neural_prepass<<<(unsigned)((n + kPrepassThreads - 1) / kPrepassThreads), kPrepassThreads, 0, st>>>(
-      n, deg, means, logits, base_color, preact, weights, eye[0], eye[1], eye[2], reinterpret_cast<uchar4 *>(rgba), color);
+      n, deg, act, means, logits, base_color, preact, weights, eye[0], eye[1], eye[2], reinterpret_cast<uchar4 *>(rgba), color);
   return 1;
 }
 

@@ -131,10 +131,10 @@ __device__ __forceinline__ void decode_warp(const mlp::Weights &W, Stage &S, int
 }
 
 // Whole-warp backward of the decoder.  `has`: this lane owns a Gaussian (inputs x, direction d, base
-// colour, dL/dcolour gcol); lanes without one pass zeros.  Returns the ReLU-masked colour gradient
+// colour, dL/dcolour gcol); lanes without one pass zeros.  Returns the colour gradient through the activation
 // gp, dL/df and dL/dd of the lane's Gaussian and advances the warp's weight-gradient fragments.
 __device__ __forceinline__ void decode_backward_warp(const mlp::Weights &W, mlp::WarpStage &S, int lane, bool has,
-                                                     const float x[32], float dx, float dy, float dz, int deg,
+                                                     const float x[32], float dx, float dy, float dz, int deg, int cact,
                                                      const float base[3], const float gcol[3], mlp::WeightGrad &dW,
                                                      float gp[3], float gf[8], float gd[3]) {
   mlp::Activations act;
@@ -143,7 +143,7 @@ __device__ __forceinline__ void decode_backward_warp(const mlp::Weights &W, mlp:
   float gy[3];
 #pragma unroll
   for (int c = 0; c < 3; ++c) {
-    gp[c] = (has && (base[c] + 0.5f + A[c]) > 0.f) ? gcol[c] : 0.f;
+    gp[c] = has ? color_act_grad_z(cact, base[c] + 0.5f + A[c]) * gcol[c] : 0.f;
     gy[c] = gp[c] * (1.f - A[c] * A[c]);
   }
   *reinterpret_cast<float4 *>(S.y + lane * 4) = make_float4(gy[0], gy[1], gy[2], 0.f);
@@ -375,7 +375,7 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_fwd(PreprocessArgs a, Cam
       reinterpret_cast<float4 *>(a.conic_opacity)[i] = make_float4(g.A, g.B, g.C, g.o);
     }
     if (vis) {
-      a.color[3 * i] = fmaxf(pre[0], 0.f); a.color[3 * i + 1] = fmaxf(pre[1], 0.f); a.color[3 * i + 2] = fmaxf(pre[2], 0.f);
+      a.color[3 * i] = color_act_z(a.act, pre[0]); a.color[3 * i + 1] = color_act_z(a.act, pre[1]); a.color[3 * i + 2] = color_act_z(a.act, pre[2]);
     }
     a.depth_key[i] = vis ? g.zbits : 0xffffffffu;
     a.tiles_touched[i] = tiles;
@@ -566,7 +566,8 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_bwd(PreprocessBwdArgs a, 
           load3(a.base_color, i, base);
           if (a.deg > 0) sh_decode(row, base, dx, dy, dz, a.deg, pre);
           else { pre[0] = base[0] + 0.5f; pre[1] = base[1] + 0.5f; pre[2] = base[2] + 0.5f; }
-          gp[0] = pre[0] > 0.f ? ga.x : 0.f; gp[1] = pre[1] > 0.f ? ga.y : 0.f; gp[2] = pre[2] > 0.f ? ga.z : 0.f;
+          gp[0] = color_act_grad_z(a.act, pre[0]) * ga.x; gp[1] = color_act_grad_z(a.act, pre[1]) * ga.y;
+          gp[2] = color_act_grad_z(a.act, pre[2]) * ga.z;
           sh_backward(row, gp, dx, dy, dz, a.deg, gd);
         } else {
 #pragma unroll
@@ -589,10 +590,10 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_bwd(PreprocessBwdArgs a, 
 #pragma unroll
           for (int k = 0; k < 32; ++k) x[k] = 0.f;
         }
-        decode_backward_warp(sWt, sStage[warp], lane, vis, x, dx, dy, dz, a.deg, base, gcol, dW, gp, gf, gd);
+        decode_backward_warp(sWt, sStage[warp], lane, vis, x, dx, dy, dz, a.deg, a.act, base, gcol, dW, gp, gf, gd);
       } else if (vis) {
 #pragma unroll
-        for (int c = 0; c < 3; ++c) gp[c] = (base[c] + 0.5f) > 0.f ? gcol[c] : 0.f;
+        for (int c = 0; c < 3; ++c) gp[c] = color_act_grad_z(a.act, base[c] + 0.5f) * gcol[c];
       }
       if (in) {
         float4 *gfp = reinterpret_cast<float4 *>(a.g_features) + 2 * i;
@@ -663,7 +664,7 @@ __global__ void __launch_bounds__(kBlock) k_appearance_fwd(AppearanceArgs a) {
 #pragma unroll
     for (int c = 0; c < 3; ++c) pre[c] = base[c] + 0.5f + A[c];
   }
-  if (in) store3(a.color, i, fmaxf(pre[0], 0.f), fmaxf(pre[1], 0.f), fmaxf(pre[2], 0.f));
+  if (in) store3(a.color, i, color_act_z(a.act, pre[0]), color_act_z(a.act, pre[1]), color_act_z(a.act, pre[2]));
 }
 
 template <int APP>
@@ -697,7 +698,7 @@ __global__ void __launch_bounds__(kBlock) k_appearance_bwd(AppearanceArgs a) {
           if (a.deg > 0) sh_decode(row, base, d[0], d[1], d[2], a.deg, pre);
           else { pre[0] = base[0] + 0.5f; pre[1] = base[1] + 0.5f; pre[2] = base[2] + 0.5f; }
 #pragma unroll
-          for (int c = 0; c < 3; ++c) gp[c] = pre[c] > 0.f ? gcol[c] : 0.f;
+          for (int c = 0; c < 3; ++c) gp[c] = color_act_grad_z(a.act, pre[c]) * gcol[c];
           sh_backward(row, gp, d[0], d[1], d[2], a.deg, gd);
         }
         warp_store_rows(a.g_sh_rest, row0, a.n, slab, lane);
@@ -714,10 +715,10 @@ __global__ void __launch_bounds__(kBlock) k_appearance_bwd(AppearanceArgs a) {
 #pragma unroll
           for (int k = 0; k < 32; ++k) x[k] = 0.f;
         }
-        decode_backward_warp(sWt, sStage[warp], lane, in, x, d[0], d[1], d[2], a.deg, base, gcol, dW, gp, gf, gd);
+        decode_backward_warp(sWt, sStage[warp], lane, in, x, d[0], d[1], d[2], a.deg, a.act, base, gcol, dW, gp, gf, gd);
       } else if (in) {
 #pragma unroll
-        for (int c = 0; c < 3; ++c) gp[c] = (base[c] + 0.5f) > 0.f ? gcol[c] : 0.f;
+        for (int c = 0; c < 3; ++c) gp[c] = color_act_grad_z(a.act, base[c] + 0.5f) * gcol[c];
       }
       if (in) {
         float4 *gfp = reinterpret_cast<float4 *>(a.g_features) + 2 * i;
@@ -851,7 +852,7 @@ extern "C" GsStatus gs_appearance_backward_noalloc(const GsScene *scene, const f
 
   AppearanceArgs a;
   memset(&a, 0, sizeof(a));
-  a.n = scene->n; a.deg = scene->active_degree;
+  a.n = scene->n; a.deg = scene->active_degree; a.act = scene->color_activation;
   a.base_color = scene->base_color; a.dirs = dirs;
   a.features = reinterpret_cast<const __half *>(scene->features);
   a.weights = reinterpret_cast<const __half *>(scene->mlp_weights);

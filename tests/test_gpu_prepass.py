@@ -101,3 +101,16 @@ def test_prepass_at_full_size_agrees_with_the_training_decoder(oracle):
     want = oracle.neural_prepass(sub, oracle.neural_fold(sub), _eye(cam))
     assert np.abs(color.cpu().numpy()[idx] - want).max() < 6e-3
     ctx.close()
+
+
+@pytest.mark.parametrize("act", [1, 2, 3])
+def test_prepass_with_other_colour_activations(oracle, act):
+    sc, cam = _scene(4_001, 30 + act)
+    sc.color_activation = act
+    sc.base_color = np.random.default_rng(act).uniform(-0.8, 0.8, sc.base_color.shape).astype(np.float32)
+    pre, rgba, color = _run(sc, cam, 3)
+    want = oracle.neural_prepass(sc, pre.astype(np.float64), _eye(cam), deg=3)
+    assert np.abs(color - want).max() < 4e-3
+    assert np.abs(want - np.maximum(sc.base_color + 0.5, 0)).max() > 1e-2
+    texel = oracle.rgba8(want, 1 / (1 + np.exp(-sc.opacity_logits.astype(np.float64))))
+    assert np.abs(rgba.astype(int) - texel.astype(int)).max() <= 1
