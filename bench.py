@@ -175,7 +175,7 @@ def run_ours(args):
             s.wait_stream(main)
         for v in range(views):
             r, s = pair[v % n_lanes], lanes[v % n_lanes]
-            r.forward(ds, cams[v], stream=s)
+            r.forward_async(ds, cams[v], stream=s)      # no host wait: the instance count stays on the device
             r.backward(ds, cams[v], G[v], stream=s)
         for s in lanes:
             main.wait_stream(s)
@@ -222,6 +222,8 @@ def run_ours(args):
         if views > 1 and n_lanes > 1:
             rs = [r] + [api.Renderer(c, ds.n, WIDTH, HEIGHT, app, pair_capacity=r.pair_capacity) for c in lane_ctx[1:]]
             ms = timed(lambda: step_two_streams(ds, rs), args.steps, args.warmup)
+            for c, s_ in zip(lane_ctx, lanes):
+                api.gs_async_status(c, s_)              # raises if a view had outgrown its pair capacity
             del rs
         stage_ms, stage_launches = profile(lambda: step(ds, r), max(1, min(args.steps, 3)))
         if tag == head:

@@ -152,6 +152,24 @@ size_t gs_workspace_bytes(int64_t n, int32_t width, int32_t height, int64_t pair
 GsStatus gs_preprocess(GsContext *ctx, const GsScene *scene, const GsCamera *cam, GsProjected *out,
                        int64_t *num_pairs_host, void *stream);
 
+/* The same without the host read: nothing is copied back and the call does not wait for the GPU.
+ * The instance count stays in the context, on the device, for the gs_render_forward that follows on
+ * the same stream with num_pairs = GS_PAIRS_ON_DEVICE.  With it a whole view (and the next ones, on
+ * other streams with contexts of their own) can be queued without the host ever waiting, which is
+ * what lets independent views overlap on the GPU.  Not in the paper, whose rasterizer reads the
+ * count back as usual. */
+GsStatus gs_preprocess_async(GsContext *ctx, const GsScene *scene, const GsCamera *cam, GsProjected *out,
+                             void *stream);
+/* gs_render_forward / gs_render_backward accept this as num_pairs: the count is the one the
+ * context's last gs_preprocess(_async) left on the device.  Buffers and kernel grids are then sized
+ * by pair_capacity.  If the true count exceeds pair_capacity the instance lists are cut off at
+ * pair_capacity (no write ever leaves the caller's buffers), the image of that view is wrong, and a
+ * flag is set that gs_async_status reports. */
+#define GS_PAIRS_ON_DEVICE ((int64_t)-1)
+/* Waits for `stream`, then returns GS_ERR_CAPACITY if any device-counted view on this context
+ * overflowed its pair_capacity since the last call (and clears the flag), else GS_OK. */
+GsStatus gs_async_status(GsContext *ctx, void *stream);
+
 /* Tile assignment, ordering and blending (Sec. 3.1, blend kernel).  Orders the visible
  * Gaussians by depth, emits one instance per (Gaussian, tile), orders instances by tile keeping
  * the depth order, records per-tile ranges, then composites every pixel front to back:

@@ -68,6 +68,11 @@ _lib.gs_workspace_bytes.restype = C.c_size_t
 _lib.gs_preprocess.argtypes = [_vp, C.POINTER(GsScene), C.POINTER(GsCamera), C.POINTER(GsProjected),
                                C.POINTER(C.c_int64), _vp]
 _lib.gs_preprocess.restype = C.c_int
+_lib.gs_preprocess_async.argtypes = [_vp, C.POINTER(GsScene), C.POINTER(GsCamera), C.POINTER(GsProjected), _vp]
+_lib.gs_preprocess_async.restype = C.c_int
+_lib.gs_async_status.argtypes = [_vp, _vp]
+_lib.gs_async_status.restype = C.c_int
+GS_PAIRS_ON_DEVICE = -1
 _lib.gs_render_forward.argtypes = [_vp, C.c_int64, C.POINTER(GsProjected), C.POINTER(GsCamera), C.c_int64,
                                    C.c_int64, C.POINTER(GsBinning), _vp, _vp, _vp, _vp, C.c_size_t, _vp]
 _lib.gs_render_forward.restype = C.c_int
@@ -324,6 +329,17 @@ def gs_preprocess(ctx: Context, scene: DeviceScene, cam: GsCamera, out: Projecte
     return int(pairs.value)
 
 
+def gs_preprocess_async(ctx: Context, scene: "DeviceScene", cam: GsCamera, out: "Projected", stream=None) -> None:
+    """gs_preprocess without the host read of the instance count (it stays on the device, see GS_PAIRS_ON_DEVICE)."""
+    cs, pp = scene.c_struct(), out.c_struct()
+    ctx._check(_lib.gs_preprocess_async(ctx._h, C.byref(cs), C.byref(cam), C.byref(pp), _stream_handle(stream)))
+
+
+def gs_async_status(ctx: Context, stream=None) -> None:
+    """Wait for the stream; raise GsError(GS_ERR_CAPACITY) if a device-counted view overflowed its capacity."""
+    ctx._check(_lib.gs_async_status(ctx._h, _stream_handle(stream)))
+
+
 def gs_render_forward(ctx: Context, n: int, proj: Projected, cam: GsCamera, num_pairs: int, pair_capacity: int,
                       binning: Binning, image: torch.Tensor, final_T: torch.Tensor, n_contrib: torch.Tensor,
                       workspace: torch.Tensor, stream=None) -> None:
@@ -380,6 +396,15 @@ class Renderer:
     def forward(self, scene: DeviceScene, cam: GsCamera, stream=None) -> torch.Tensor:
         self.num_pairs = gs_preprocess(self.ctx, scene, cam, self.proj, stream)
         gs_render_forward(self.ctx, scene.n, self.proj, cam, self.num_pairs, self.pair_capacity, self.binning,
+                          self.image, self.final_T, self.n_contrib, self.workspace, stream)
+        return self.image
+
+    def forward_async(self, scene: DeviceScene, cam: GsCamera, stream=None) -> torch.Tensor:
+        """forward() without any host wait: the instance count stays on the device and the lists are sized by
+        pair_capacity.  Check gs_async_status(ctx, stream) once the work is done."""
+        gs_preprocess_async(self.ctx, scene, cam, self.proj, stream)
+        self.num_pairs = GS_PAIRS_ON_DEVICE
+        gs_render_forward(self.ctx, scene.n, self.proj, cam, GS_PAIRS_ON_DEVICE, self.pair_capacity, self.binning,
                           self.image, self.final_T, self.n_contrib, self.workspace, stream)
         return self.image
 

@@ -14,7 +14,8 @@ struct StageRecord { int stage; int launches; cudaEvent_t begin, end; };
 struct GsContext {
   int device;
   int num_sms;
-  unsigned long long *d_counter;      // device: instance counter (+ one more word for gs_profile_blend_counts)
+  unsigned long long *d_counter;      // device: [0] instance counter of the last gs_preprocess, [1] second word of
+                                      // gs_profile_blend_counts, [2] set when a device-counted view overflowed its capacity
   unsigned long long *h_counter;      // pinned host mirror
   float *d_w_partials;                // device: [kWgradBlocks, 816] decoder-gradient partial sums
   char error[256];
@@ -177,8 +178,9 @@ GsStatus gs_create(int device, GsContext **out) {
   ctx->error[0] = 0;
   ctx->d_counter = nullptr; ctx->h_counter = nullptr; ctx->d_w_partials = nullptr;
   ctx->profiling = false;
-  if (cudaMalloc(&ctx->d_counter, 2 * sizeof(unsigned long long)) != cudaSuccess ||
-      cudaMallocHost(&ctx->h_counter, 2 * sizeof(unsigned long long)) != cudaSuccess ||
+  if (cudaMalloc(&ctx->d_counter, 4 * sizeof(unsigned long long)) != cudaSuccess ||
+      cudaMemset(ctx->d_counter, 0, 4 * sizeof(unsigned long long)) != cudaSuccess ||
+      cudaMallocHost(&ctx->h_counter, 4 * sizeof(unsigned long long)) != cudaSuccess ||
       cudaMalloc(&ctx->d_w_partials, sizeof(float) * kWgradBlocks * GS_MLP_WEIGHTS) != cudaSuccess) {
     gs_destroy(ctx);
     return GS_ERR_CUDA;
@@ -206,20 +208,21 @@ size_t gs_workspace_bytes(int64_t n, int32_t width, int32_t height, int64_t pair
   return f > b ? f : b;
 }
 
-GsStatus gs_preprocess(GsContext *ctx, const GsScene *scene, const GsCamera *cam, GsProjected *out,
-                       int64_t *num_pairs_host, void *stream) {
-  if (!ctx) return GS_ERR_INVALID_ARG;
+namespace {
+GsStatus preprocess_impl(GsContext *ctx, const GsScene *scene, const GsCamera *cam, GsProjected *out,
+                         int64_t *num_pairs_host, void *stream) {
   GsStatus st = scene_ok(ctx, scene);
   if (st != GS_OK) return st;
   if (!camera_ok(cam)) return fail(ctx, GS_ERR_INVALID_ARG, "bad camera (size, focal length or more than 65535 tiles per axis)");
-  if (!out || !num_pairs_host) return fail(ctx, GS_ERR_INVALID_ARG, "out / num_pairs_host is NULL");
-  *num_pairs_host = 0;
+  if (!out) return fail(ctx, GS_ERR_INVALID_ARG, "out is NULL");
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaSetDevice(ctx->device);
+  // the counter is cleared even for an empty scene: a device-counted forward reads it
+  if ((st = check_cuda(ctx, cudaMemsetAsync(ctx->d_counter, 0, sizeof(unsigned long long), s), "memset")) != GS_OK) return st;
   if (scene->n == 0) return GS_OK;
   if (bad_ptr(out->mean2d) || bad_ptr(out->conic_opacity) || bad_ptr(out->color) || bad_ptr(out->depth_key) ||
       bad_ptr(out->rect) || bad_ptr(out->tiles_touched) || (out->extent && !aligned16(out->extent)))
     return fail(ctx, GS_ERR_INVALID_ARG, "a GsProjected buffer is NULL or misaligned");
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
-  cudaSetDevice(ctx->device);
   PreprocessArgs a;
   a.n = scene->n;
   a.means = scene->means; a.log_scales = scene->log_scales; a.quats = scene->quats; a.logits = scene->opacity_logits;
@@ -230,16 +233,44 @@ GsStatus gs_preprocess(GsContext *ctx, const GsScene *scene, const GsCamera *cam
   a.mean2d = out->mean2d; a.conic_opacity = out->conic_opacity; a.color = out->color; a.extent = out->extent;
   a.depth_key = out->depth_key; a.rect = out->rect; a.tiles_touched = out->tiles_touched;
   a.pair_counter = ctx->d_counter;
-  if ((st = check_cuda(ctx, cudaMemsetAsync(ctx->d_counter, 0, sizeof(unsigned long long), s), "memset")) != GS_OK) return st;
   {
     StageTimer t(ctx, GS_STAGE_PREPROCESS_FWD, s);
     t.done(launch_preprocess_fwd(scene->app, a, make_cam(cam), s));
   }
   if ((st = check_cuda(ctx, cudaGetLastError(), "preprocess launch")) != GS_OK) return st;
+  if (!num_pairs_host) return GS_OK;
   if ((st = check_cuda(ctx, cudaMemcpyAsync(ctx->h_counter, ctx->d_counter, sizeof(unsigned long long),
                                             cudaMemcpyDeviceToHost, s), "pair count copy")) != GS_OK) return st;
   if ((st = check_cuda(ctx, cudaStreamSynchronize(s), "preprocess")) != GS_OK) return st;
   *num_pairs_host = (int64_t)*ctx->h_counter;
+  return GS_OK;
+}
+}  // namespace
+
+GsStatus gs_preprocess(GsContext *ctx, const GsScene *scene, const GsCamera *cam, GsProjected *out,
+                       int64_t *num_pairs_host, void *stream) {
+  if (!ctx) return GS_ERR_INVALID_ARG;
+  if (!num_pairs_host) return fail(ctx, GS_ERR_INVALID_ARG, "num_pairs_host is NULL");
+  *num_pairs_host = 0;
+  return preprocess_impl(ctx, scene, cam, out, num_pairs_host, stream);
+}
+
+GsStatus gs_preprocess_async(GsContext *ctx, const GsScene *scene, const GsCamera *cam, GsProjected *out, void *stream) {
+  if (!ctx) return GS_ERR_INVALID_ARG;
+  return preprocess_impl(ctx, scene, cam, out, nullptr, stream);
+}
+
+GsStatus gs_async_status(GsContext *ctx, void *stream) {
+  if (!ctx) return GS_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaSetDevice(ctx->device);
+  GsStatus st;
+  if ((st = check_cuda(ctx, cudaMemcpyAsync(ctx->h_counter + 2, ctx->d_counter + 2, sizeof(unsigned long long),
+                                            cudaMemcpyDeviceToHost, s), "status copy")) != GS_OK) return st;
+  if ((st = check_cuda(ctx, cudaMemsetAsync(ctx->d_counter + 2, 0, sizeof(unsigned long long), s), "status reset")) != GS_OK) return st;
+  if ((st = check_cuda(ctx, cudaStreamSynchronize(s), "status")) != GS_OK) return st;
+  if (ctx->h_counter[2] != 0)
+    return fail(ctx, GS_ERR_CAPACITY, "a device-counted gs_render_forward had more instances than pair_capacity: that view's lists were cut off");
   return GS_OK;
 }
 
@@ -248,6 +279,9 @@ GsStatus gs_render_forward(GsContext *ctx, int64_t n, const GsProjected *proj, c
                            float *final_T, uint32_t *n_contrib, void *workspace, size_t workspace_bytes,
                            void *stream) {
   if (!ctx) return GS_ERR_INVALID_ARG;
+  const bool on_device = num_pairs == GS_PAIRS_ON_DEVICE;   // the count of the context's last gs_preprocess(_async)
+  const unsigned long long *count_dev = on_device ? ctx->d_counter : nullptr;
+  if (on_device) num_pairs = pair_capacity;
   if (n < 0 || num_pairs < 0 || pair_capacity < 0) return fail(ctx, GS_ERR_INVALID_ARG, "negative size");
   if (!camera_ok(cam)) return fail(ctx, GS_ERR_INVALID_ARG, "bad camera");
   if (!proj || !bin) return fail(ctx, GS_ERR_INVALID_ARG, "proj / bin is NULL");
@@ -273,7 +307,7 @@ GsStatus gs_render_forward(GsContext *ctx, int64_t n, const GsProjected *proj, c
     {
       StageTimer t(ctx, GS_STAGE_DEPTH_SORT, s);
       t.done(launch_radix_sort(proj->depth_key, nullptr, w.sorted_depth, bin->depth_order, w.tmp_keys, w.tmp_vals,
-                               n, 32, w.sort_table, s));
+                               n, nullptr, 32, w.sort_table, s));
     }
     // stage 2: instances in depth order, then a stable sort by tile id alone
     {
@@ -283,17 +317,18 @@ GsStatus gs_render_forward(GsContext *ctx, int64_t n, const GsProjected *proj, c
     {
       StageTimer t(ctx, GS_STAGE_KEYGEN, s);
       t.done(launch_keygen(bin->depth_order, proj->rect, proj->mean2d, proj->conic_opacity, proj->tiles_touched,
-                           w.block_offsets, w.inst_tiles, w.inst_vals, n, cd.gx, cd.W, cd.H, s));
+                           w.block_offsets, w.inst_tiles, w.inst_vals, n, cd.gx, cd.W, cd.H, pair_capacity, s));
     }
     {
       StageTimer t(ctx, GS_STAGE_TILE_SORT, s);
       t.done(launch_radix_sort(w.inst_tiles, w.inst_vals, bin->sorted_tiles, bin->sorted_vals, w.tmp_tiles,
-                               w.tmp_ivals, num_pairs, tile_bits(num_tiles), w.sort_table, s));
+                               w.tmp_ivals, num_pairs, count_dev, tile_bits(num_tiles), w.sort_table, s));
     }
   }
   {
     StageTimer t(ctx, GS_STAGE_TILE_RANGES, s);
-    t.done(launch_tile_ranges(bin->sorted_tiles, num_pairs, bin->tile_ranges, bin->tile_order, num_tiles, s));
+    t.done(launch_tile_ranges(bin->sorted_tiles, num_pairs, count_dev, reinterpret_cast<uint32_t *>(ctx->d_counter + 2),
+                              bin->tile_ranges, bin->tile_order, num_tiles, s));
   }
   {
     StageTimer t(ctx, GS_STAGE_BLEND_FWD, s);
@@ -312,6 +347,7 @@ GsStatus gs_render_backward(GsContext *ctx, const GsScene *scene, const GsCamera
   if (st != GS_OK) return st;
   if (!camera_ok(cam)) return fail(ctx, GS_ERR_INVALID_ARG, "bad camera");
   if (!proj || !bin || !grads) return fail(ctx, GS_ERR_INVALID_ARG, "proj / bin / grads is NULL");
+  if (num_pairs == GS_PAIRS_ON_DEVICE) num_pairs = 1;   // unknown here; the tile ranges bound every list
   if (bad_ptr(final_T) || bad_ptr(n_contrib) || bad_ptr(dL_dimage) || bad_ptr(bin->tile_ranges) || bad_ptr(bin->tile_order))
     return fail(ctx, GS_ERR_INVALID_ARG, "an image-sized buffer is NULL or misaligned");
   const int64_t n = scene->n;

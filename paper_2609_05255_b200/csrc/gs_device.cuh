@@ -76,15 +76,15 @@ size_t sort_scratch_bytes(int64_t count);
 // the element indices.  Result lands in keys_out / vals_out; tmp_* are same-sized alternates.
 int launch_radix_sort(const uint32_t *keys_in, const uint32_t *vals_in, uint32_t *keys_out,
                        uint32_t *vals_out, uint32_t *tmp_keys, uint32_t *tmp_vals, int64_t count,
-                       int num_bits, void *scratch, cudaStream_t st);
+                       const unsigned long long *count_dev, int num_bits, void *scratch, cudaStream_t st);
 size_t scan_scratch_bytes(int64_t n);
 int launch_tile_offsets(const uint32_t *depth_order, const uint32_t *tiles_touched, uint32_t *offsets,
                         int64_t n, void *scratch, cudaStream_t st);
 int launch_keygen(const uint32_t *depth_order, const uint16_t *rect, const float *mean2d, const float *conic_opacity,
                   const uint32_t *tiles_touched, const uint32_t *offsets, uint32_t *inst_tiles, uint32_t *inst_vals,
-                  int64_t n, int gx, int W, int H, cudaStream_t st);
-int launch_tile_ranges(const uint32_t *sorted_tiles, int64_t P, uint32_t *ranges, uint32_t *order,
-                       int num_tiles, cudaStream_t st);
+                  int64_t n, int gx, int W, int H, int64_t capacity, cudaStream_t st);
+int launch_tile_ranges(const uint32_t *sorted_tiles, int64_t P, const unsigned long long *count_dev, uint32_t *overflow,
+                       uint32_t *ranges, uint32_t *order, int num_tiles, cudaStream_t st);
 
 // Blend.
 int launch_blend_fwd(const CamDev &cam, const uint32_t *ranges, const uint32_t *order, const uint32_t *vals,

@@ -33,8 +33,10 @@ SortPlan plan_for(int64_t count) {
 
 // Digit histogram of each block's contiguous range: table[block][digit].
 __global__ void __launch_bounds__(kSortThreads) k_radix_hist(const uint32_t *__restrict__ keys, int64_t count,
+                                                             const unsigned long long *__restrict__ count_dev,
                                                              int shift, uint32_t mask, int tiles_per_block,
                                                              uint32_t *__restrict__ table) {
+  if (count_dev) count = min(count, (int64_t)__ldg(count_dev));   // the true length lives on the device
   __shared__ uint32_t s_hist[kSortWarps][256];
   const int tid = threadIdx.x, warp = tid >> 5;
   for (int k = tid; k < kSortWarps * 256; k += kSortThreads) (&s_hist[0][0])[k] = 0;
@@ -109,7 +111,8 @@ __device__ __forceinline__ uint32_t block_exclusive_scan_256(uint32_t v, uint32_
 template <int BITS>
 __global__ void __launch_bounds__(kSortThreads, 3) k_radix_scatter(
     const uint32_t *__restrict__ keys_in, const uint32_t *__restrict__ vals_in, uint32_t *__restrict__ keys_out,
-    uint32_t *__restrict__ vals_out, int64_t count, int shift, int tiles_per_block,
+    uint32_t *__restrict__ vals_out, int64_t count, const unsigned long long *__restrict__ count_dev, int shift,
+    int tiles_per_block,
     const uint32_t *__restrict__ table, const uint32_t *__restrict__ totals, int nblocks) {
   __shared__ uint32_t s_keys[kSortTile];
   __shared__ uint32_t s_vals[kSortTile];
@@ -119,6 +122,7 @@ __global__ void __launch_bounds__(kSortThreads, 3) k_radix_scatter(
   __shared__ uint32_t s_warp_tot[kSortWarps];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t lt_mask = (1u << lane) - 1u;
+  if (count_dev) count = min(count, (int64_t)__ldg(count_dev));
   constexpr uint32_t kDigitMask = (1u << BITS) - 1u;
 
   // global base of every digit for this block: all smaller digits everywhere (scan of the row
@@ -268,7 +272,8 @@ __global__ void __launch_bounds__(kScanBlock) k_keygen(const uint32_t *__restric
                                                        const float *__restrict__ conic_opacity,
                                                        const uint32_t *__restrict__ tiles_touched,
                                                        const uint32_t *__restrict__ block_offsets, int64_t n, int gx,
-                                                       int W, int H, uint32_t *__restrict__ inst_tiles,
+                                                       int W, int H, uint32_t capacity,
+                                                       uint32_t *__restrict__ inst_tiles,
                                                        uint32_t *__restrict__ inst_vals) {
   __shared__ uint32_t s_w[kScanBlock / 32];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -309,8 +314,10 @@ __global__ void __launch_bounds__(kScanBlock) k_keygen(const uint32_t *__restric
       int xa, xb;
       if (!sp.row(ty, r.x, r.z, xa, xb)) continue;
       for (int tx = xa; tx < xb; ++tx) {
-        inst_tiles[p] = (uint32_t)(ty * gx + tx);
-        inst_vals[p] = g;
+        if (p < capacity) {   // never past the caller's buffers, even if the count was taken on the device
+          inst_tiles[p] = (uint32_t)(ty * gx + tx);
+          inst_vals[p] = g;
+        }
         ++p;
       }
     }
@@ -342,8 +349,11 @@ __global__ void __launch_bounds__(kScanBlock) k_keygen(const uint32_t *__restric
         const int a = __shfl_sync(kFull, xa, rr), b = __shfl_sync(kFull, xb, rr);
         const uint32_t o = p + __shfl_sync(kFull, excl, rr);
         for (int tx = a + lane; tx < b; tx += 32) {
-          inst_tiles[o + (uint32_t)(tx - a)] = (uint32_t)((tyb + rr) * gx + tx);
-          inst_vals[o + (uint32_t)(tx - a)] = s_g;
+          const uint32_t q = o + (uint32_t)(tx - a);
+          if (q < capacity) {
+            inst_tiles[q] = (uint32_t)((tyb + rr) * gx + tx);
+            inst_vals[q] = s_g;
+          }
         }
       }
       p += __shfl_sync(kFull, incl, 31);
@@ -351,8 +361,15 @@ __global__ void __launch_bounds__(kScanBlock) k_keygen(const uint32_t *__restric
   }
 }
 
-__global__ void k_tile_ranges(const uint32_t *__restrict__ sorted_tiles, int64_t P, uint32_t *__restrict__ ranges) {
+__global__ void k_tile_ranges(const uint32_t *__restrict__ sorted_tiles, int64_t P,
+                              const unsigned long long *__restrict__ count_dev, uint32_t *__restrict__ overflow,
+                              uint32_t *__restrict__ ranges) {
   const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (count_dev) {   // P is the capacity here; more instances than that were cut off: tell the host
+    const int64_t c = (int64_t)__ldg(count_dev);
+    if (p == 0 && c > P) *overflow = 1u;
+    P = min(P, c);
+  }
   if (p >= P) return;
   const uint32_t t = __ldg(sorted_tiles + p);
   if (p == 0 || t != __ldg(sorted_tiles + p - 1)) ranges[2 * t] = (uint32_t)p;
@@ -389,8 +406,8 @@ __global__ void __launch_bounds__(1024) k_tile_order(const uint32_t *__restrict_
 size_t sort_scratch_bytes(int64_t count) { return ((size_t)plan_for(count).blocks + 1) * 256 * sizeof(uint32_t); }
 
 int launch_radix_sort(const uint32_t *keys_in, const uint32_t *vals_in, uint32_t *keys_out, uint32_t *vals_out,
-                       uint32_t *tmp_keys, uint32_t *tmp_vals, int64_t count, int num_bits, void *scratch,
-                       cudaStream_t st) {
+                       uint32_t *tmp_keys, uint32_t *tmp_vals, int64_t count, const unsigned long long *count_dev,
+                       int num_bits, void *scratch, cudaStream_t st) {
   if (count <= 0) return 0;
   const SortPlan plan = plan_for(count);
   int passes = (num_bits + 7) / 8;
@@ -402,17 +419,18 @@ int launch_radix_sort(const uint32_t *keys_in, const uint32_t *vals_in, uint32_t
   for (int p = 0; p < passes; ++p) {
     const bool to_out = ((passes - 1 - p) % 2) == 0;
     uint32_t *dst_k = to_out ? keys_out : tmp_keys, *dst_v = to_out ? vals_out : tmp_vals;
-    k_radix_hist<<<plan.blocks, kSortThreads, 0, st>>>(src_k, count, bits * p, (1u << bits) - 1u, plan.tiles_per_block, table);
+    k_radix_hist<<<plan.blocks, kSortThreads, 0, st>>>(src_k, count, count_dev, bits * p, (1u << bits) - 1u,
+                                                        plan.tiles_per_block, table);
     k_radix_scan_rows<<<256, 256, 0, st>>>(table, plan.blocks, totals);
 #define GS_SCATTER(B)                                                                                              \
   case B:                                                                                                          \
-    k_radix_scatter<B><<<plan.blocks, kSortThreads, 0, st>>>(src_k, src_v, dst_k, dst_v, count, bits * p,         \
+    k_radix_scatter<B><<<plan.blocks, kSortThreads, 0, st>>>(src_k, src_v, dst_k, dst_v, count, count_dev, bits * p, \
                                                               plan.tiles_per_block, table, totals, plan.blocks);   \
     break;
     switch (bits) {
       GS_SCATTER(1) GS_SCATTER(2) GS_SCATTER(3) GS_SCATTER(4) GS_SCATTER(5) GS_SCATTER(6) GS_SCATTER(7)
       default:
-        k_radix_scatter<8><<<plan.blocks, kSortThreads, 0, st>>>(src_k, src_v, dst_k, dst_v, count, bits * p,
+        k_radix_scatter<8><<<plan.blocks, kSortThreads, 0, st>>>(src_k, src_v, dst_k, dst_v, count, count_dev, bits * p,
                                                                   plan.tiles_per_block, table, totals, plan.blocks);
     }
 #undef GS_SCATTER
@@ -435,18 +453,19 @@ int launch_tile_offsets(const uint32_t *depth_order, const uint32_t *tiles_touch
 
 int launch_keygen(const uint32_t *depth_order, const uint16_t *rect, const float *mean2d, const float *conic_opacity,
                   const uint32_t *tiles_touched, const uint32_t *block_offsets, uint32_t *inst_tiles, uint32_t *inst_vals,
-                  int64_t n, int gx, int W, int H, cudaStream_t st) {
+                  int64_t n, int gx, int W, int H, int64_t capacity, cudaStream_t st) {
   if (n <= 0) return 0;
   const int blocks = (int)((n + kScanBlock - 1) / kScanBlock);
+  const uint32_t cap = capacity > 0xffffffffll ? 0xffffffffu : (uint32_t)capacity;
   k_keygen<<<blocks, kScanBlock, 0, st>>>(depth_order, rect, mean2d, conic_opacity, tiles_touched, block_offsets, n, gx, W, H,
-                                          inst_tiles, inst_vals);
+                                          cap, inst_tiles, inst_vals);
   return 1;
 }
 
-int launch_tile_ranges(const uint32_t *sorted_tiles, int64_t P, uint32_t *ranges, uint32_t *order, int num_tiles,
-                       cudaStream_t st) {
+int launch_tile_ranges(const uint32_t *sorted_tiles, int64_t P, const unsigned long long *count_dev, uint32_t *overflow,
+                       uint32_t *ranges, uint32_t *order, int num_tiles, cudaStream_t st) {
   cudaMemsetAsync(ranges, 0, (size_t)num_tiles * 2 * sizeof(uint32_t), st);
-  if (P > 0) k_tile_ranges<<<(int)((P + 255) / 256), 256, 0, st>>>(sorted_tiles, P, ranges);
+  if (P > 0) k_tile_ranges<<<(int)((P + 255) / 256), 256, 0, st>>>(sorted_tiles, P, count_dev, overflow, ranges);
   k_tile_order<<<1, 1024, 0, st>>>(ranges, num_tiles, order);
   return P > 0 ? 2 : 1;
 }

@@ -1,0 +1,82 @@
+"""The path without host waits: gs_preprocess_async + gs_render_forward(GS_PAIRS_ON_DEVICE) must give the
+same bits as the path that reads the instance count back, and an overflow of the capacity must be
+reported (with every write kept inside the caller's buffers)."""
+import numpy as np
+import pytest
+
+from paper_2609_05255_b200 import scenes
+
+pytestmark = pytest.mark.gpu
+
+
+def _setup(n=20_011, app=scenes.APP_NEURAL):
+    import torch
+    from paper_2609_05255_b200 import api
+    w = scenes.config2(n=n, app=app)
+    ctx = api.Context(0)
+    ds = api.upload_scene(w.scene, ctx.device)
+    cam = api.make_camera(w.cameras[0])
+    return torch, api, ctx, ds, cam, w
+
+
+def test_device_counted_view_equals_host_counted_view():
+    torch, api, ctx, ds, cam, w = _setup()
+    W, H = w.cameras[0].width, w.cameras[0].height
+    probe = api.alloc_projected(ds.n, ctx.device, False)
+    P = api.gs_preprocess(ctx, ds, cam, probe)
+    cap = int(P * 1.3) + 777
+    a = api.Renderer(ctx, ds.n, W, H, ds.app, pair_capacity=cap)
+    b = api.Renderer(ctx, ds.n, W, H, ds.app, pair_capacity=cap)
+    G = torch.from_numpy(scenes.upstream_gradient(w.cameras[0], 5)).to(ctx.device)
+    a.forward(ds, cam); a.backward(ds, cam, G)
+    b.forward_async(ds, cam); b.backward(ds, cam, G)
+    api.gs_async_status(ctx)
+    assert torch.equal(a.image, b.image) and torch.equal(a.final_T, b.final_T) and torch.equal(a.n_contrib, b.n_contrib)
+    assert torch.equal(a.binning.tile_ranges, b.binning.tile_ranges)
+    assert torch.equal(a.binning.sorted_vals[:P], b.binning.sorted_vals[:P])
+    for k in ("means", "log_scales", "quats", "opacity_logits", "base_color", "features"):
+        x, y = getattr(a.grads, k), getattr(b.grads, k)
+        # the blend backward sums with atomics: equal up to the order of those sums
+        assert torch.allclose(x, y, rtol=1e-4, atol=1e-6), k
+    ctx.close()
+
+
+def test_overflow_is_reported_and_nothing_is_written_past_the_capacity():
+    torch, api, ctx, ds, cam, w = _setup()
+    W, H = w.cameras[0].width, w.cameras[0].height
+    probe = api.alloc_projected(ds.n, ctx.device, False)
+    P = api.gs_preprocess(ctx, ds, cam, probe)
+    cap = P // 3
+    r = api.Renderer(ctx, ds.n, W, H, ds.app, pair_capacity=cap)
+    # canaries behind the instance lists (the buffers hold exactly `cap` entries, allocated apart)
+    guard = 4096
+    big_t = torch.full((cap + guard,), 0x5A5A5A5A, device=ctx.device, dtype=torch.int32)
+    big_v = torch.full((cap + guard,), 0x5A5A5A5A, device=ctx.device, dtype=torch.int32)
+    r.binning.sorted_tiles, r.binning.sorted_vals = big_t[:cap], big_v[:cap]
+    r.forward_async(ds, cam)
+    with pytest.raises(api.GsError) as e:
+        api.gs_async_status(ctx)
+    assert e.value.status == api.GS_ERR_CAPACITY
+    assert torch.all(big_t[cap:] == 0x5A5A5A5A) and torch.all(big_v[cap:] == 0x5A5A5A5A)
+    api.gs_async_status(ctx)                      # the flag was cleared
+    # the same renderer with the host-counted call refuses up front
+    with pytest.raises(api.GsError) as e:
+        r.forward(ds, cam)
+    assert e.value.status == api.GS_ERR_CAPACITY
+    ctx.close()
+
+
+def test_empty_scene_through_the_async_calls():
+    import torch
+    from paper_2609_05255_b200 import api
+    ctx = api.Context(0)
+    sc = scenes.config1(0).scene if hasattr(scenes, "config1") else None
+    ds = api.upload_scene(sc, ctx.device)
+    cam_h = scenes.identity_camera(64, 64, 64.0)
+    cam = api.make_camera(cam_h)
+    r = api.Renderer(ctx, 0, 64, 64, ds.app, pair_capacity=16)
+    r.forward_async(ds, cam)
+    api.gs_async_status(ctx)
+    bg = torch.tensor(np.asarray(cam_h.background, np.float32), device=ctx.device)
+    assert torch.equal(r.image, bg[:, None, None].expand(3, 64, 64))
+    ctx.close()
