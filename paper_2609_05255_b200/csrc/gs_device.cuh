@@ -230,18 +230,6 @@ __device__ __forceinline__ float ex2_approx(float x) {
   return y;
 }
 
-// One pixel-Gaussian evaluation, shared by the forward and the backward blend so that both
-// take identical skip decisions.  q = (-0.5 A log2e, -B log2e, -0.5 C log2e).  Returns false if
-// the pair is skipped; e2 = exp(power), alpha = min(0.99, o * e2).
-__device__ __forceinline__ bool eval_alpha(float dx, float dy, float qa, float qb, float qc, float o,
-                                           float &e2, float &alpha) {
-  const float p = __fmaf_rn(__fmaf_rn(qa, dx, __fmul_rn(qb, dy)), dx, __fmul_rn(__fmul_rn(qc, dy), dy));
-  if (p > 0.f) return false;
-  e2 = ex2_approx(p);
-  alpha = fminf(kAlphaMax, __fmul_rn(o, e2));
-  return alpha >= kAlphaMin;
-}
-
 #endif  // __CUDACC__
 
 }  // namespace gs

@@ -12,7 +12,6 @@
 namespace gs {
 namespace {
 
-constexpr unsigned kFull = 0xffffffffu;
 constexpr int kFoldThreads = 128;
 constexpr int kPrepassThreads = 128;
 constexpr int kPrepassWarps = kPrepassThreads / 32;

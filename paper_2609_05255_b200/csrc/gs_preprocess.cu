@@ -306,7 +306,7 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_fwd(PreprocessArgs a, Cam
   __shared__ __align__(16) float sData[APP == GS_APP_SH ? kWarps * kSlab : 4];
   __shared__ __align__(16) unsigned char sNN[APP == GS_APP_NEURAL ? sizeof(mlp::Weights) + kWarps * sizeof(StageFwd) : 16];
   mlp::Weights *sWt = reinterpret_cast<mlp::Weights *>(sNN);
-  StageFwd *sStage = reinterpret_cast<StageFwd *>(sNN + sizeof(mlp::Weights));
+  StageFwd *sStage = reinterpret_cast<StageFwd *>(sNN + (APP == GS_APP_NEURAL ? sizeof(mlp::Weights) : 0));   // unused for SH
   __shared__ unsigned int sPairs[kWarps];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (APP == GS_APP_NEURAL) {
@@ -631,7 +631,7 @@ __global__ void __launch_bounds__(kBlock) k_appearance_fwd(AppearanceArgs a) {
   __shared__ __align__(16) float sData[APP == GS_APP_SH ? kWarps * kSlab : 4];
   __shared__ __align__(16) unsigned char sNN[APP == GS_APP_NEURAL ? sizeof(mlp::Weights) + kWarps * sizeof(StageFwd) : 16];
   mlp::Weights *sWt = reinterpret_cast<mlp::Weights *>(sNN);
-  StageFwd *sStage = reinterpret_cast<StageFwd *>(sNN + sizeof(mlp::Weights));
+  StageFwd *sStage = reinterpret_cast<StageFwd *>(sNN + (APP == GS_APP_NEURAL ? sizeof(mlp::Weights) : 0));   // unused for SH
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (APP == GS_APP_NEURAL) {
     mlp::load_weights(a.weights, sWt[0], tid, kBlock);
