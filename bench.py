@@ -250,7 +250,9 @@ def run_ours(args):
                             host=host, ds=ds, r=r, app=tag)
 
     # ---- end to end through the public API with host buffers (neural arm)
-    e2e = None if args.skip_e2e else measure_e2e(api, torch, ctx, results[head], cams, G, views, args, timed, dev)
+    e2e_host = None if args.skip_e2e else measure_e2e(api, torch, ctx, results[head], cams, G, views, args, timed, dev)
+    e2e = None if args.skip_e2e else measure_e2e_training(api, torch, lane_ctx, lanes, results[head], cams, G, views, args,
+                                                           timed, dev, WIDTH, HEIGHT)
 
     # ---- appearance-decode sweep (separate-pass kernels, HBM resident)
     decode = None if (args.skip_decode or args.config != 3) else decode_sweep(api, torch, ctx, dev, peaks, args)
@@ -279,7 +281,7 @@ def run_ours(args):
         "gprimitives_per_s": world * n * views / (ms * 1e-3) / 1e9,
         "ms_per_step_single_stream": neural["ms_one"],
         "streams": 1 if views == 1 else n_lanes,
-        "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step,
+        "clocks": clocks, "e2e": e2e, "e2e_gradients_to_host": e2e_host, "gpu_launches": launches_per_step,
         "roofline": roof,
         "rooflines": {k: stage_roofline(k, neural, views, n, peaks, alu_peak)
                       for k in ("preprocess_fwd", "depth_sort", "keygen", "tile_sort", "blend_fwd", "blend_bwd",
@@ -398,6 +400,78 @@ def measure_e2e(api, torch, ctx, arm, cams, G, views, args, timed, dev):
     r.image, r.grads = images[0], grads[0]
     return {"value": ms, "unit": f"ms/iter ({views} views, fwd+bwd)", "h2d_bytes_per_step": int(h2d),
             "d2h_bytes_per_step": int(d2h), "overlap": "copies on their own streams, double-buffered"}
+
+
+def measure_e2e_training(api, torch, lane_ctx, lanes, arm, cams, G, views, args, timed, dev, WIDTH, HEIGHT):
+    """One training iteration end to end, as a trainer would run it: the scene lives on the device; every step
+    the upstream gradients of the views come from pinned host memory, the views are rendered forward and
+    backward (each into gradient buffers of its own, on the lanes' streams, without host waits), ONE fused Adam
+    launch sums the views' gradients and updates all parameters (fp32 masters, half copies for the next step),
+    and the rendered images go back to pinned host memory.  Copies run on streams of their own."""
+    ds, r0 = arm["ds"], arm["r"]
+    neural = arm["app"] == "neural"
+    n = ds.n
+    rs = [r0] + [api.Renderer(c, n, WIDTH, HEIGHT, r0.app, pair_capacity=r0.pair_capacity) for c in lane_ctx[1:]]
+    grads = [r0.grads] + [api.alloc_grads(n, r0.app, dev) for _ in range(views - 1)]
+    images = [r0.image] + [torch.empty_like(r0.image) for _ in range(views - 1)]
+    h_G = G.cpu().pin_memory()
+    d_G = torch.empty_like(G)
+    h_images = torch.empty((views,) + tuple(r0.image.shape), dtype=torch.float32).pin_memory()
+    y0 = 0.28209479177387814
+    spec = [("means", 3, 1.6e-6), ("log_scales", 3, 5e-5), ("quats", 4, 1e-5), ("opacity_logits", 1, 5e-4)]
+    spec += [("base_color", 3, 0.00025), ("features", 8, 0.008e-2), ("mlp_weights", 1, 0.003e-2)] if neural else \
+            [("base_color", 3, 0.0025 * y0 * 1e-2), ("sh_rest", 45, 0.000125e-2)]
+    tensors, masters = [], {}
+    for name, cols, lr in spec:        # rates scaled down: random upstream gradients must not wreck the synthetic scene
+        stored = getattr(ds, name)
+        master = stored.float().contiguous() if stored.dtype != torch.float32 else stored
+        masters[name] = master
+        g0 = getattr(grads[0], name)
+        more = [getattr(g, name) for g in grads[1:]]
+        tensors.append(api.AdamTensor(master, g0, torch.zeros_like(master), torch.zeros_like(master), [lr] * cols, 0.9,
+                                      0.99 if name == "mlp_weights" else 0.999, 1e-15,
+                                      half_copy=stored if stored.dtype == torch.float16 else None, more_grads=more))
+    main = torch.cuda.current_stream(dev)
+    up, down = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+    ev_up = [torch.cuda.Event() for _ in range(views)]
+    ev_done = [torch.cuda.Event() for _ in range(views)]
+    state = {"step": 0}
+    L = len(lanes)
+
+    def step():
+        state["step"] += 1
+        up.wait_stream(main)                       # the previous step's kernels have read d_G
+        with torch.cuda.stream(up):
+            for v in range(views):
+                d_G[v].copy_(h_G[v], non_blocking=True)
+                ev_up[v].record(up)
+        down.wait_stream(main)
+        for s in lanes:
+            s.wait_stream(main)                    # the parameters of this step are in place
+        for v in range(views):
+            r, s = rs[v % L], lanes[v % L]
+            s.wait_event(ev_up[v])
+            r.image, r.grads = images[v], grads[v]
+            r.forward_async(ds, cams[v], stream=s)
+            r.backward(ds, cams[v], d_G[v], stream=s)
+            ev_done[v].record(s)
+            with torch.cuda.stream(down):
+                down.wait_event(ev_done[v])
+                h_images[v].copy_(images[v], non_blocking=True)
+        for s in lanes:
+            main.wait_stream(s)
+        api.gs_adam_step(lane_ctx[0], tensors, state["step"])
+        main.wait_stream(down)
+
+    ms = timed(step, max(2, args.steps // 2), 2)
+    for c, s_ in zip(lane_ctx, lanes):
+        api.gs_async_status(c, s_)
+    finite = all(bool(torch.isfinite(m).all()) for m in masters.values())
+    r0.image, r0.grads = images[0], grads[0]
+    return {"value": ms, "unit": f"ms/iter ({views} views, fwd+bwd, + one fused Adam update)",
+            "h2d_bytes_per_step": int(h_G.numel() * 4), "d2h_bytes_per_step": int(h_images.numel() * 4),
+            "what": "upstream gradients in, rendered images out, parameters stay on the device and are updated by Adam",
+            "streams": L, "parameters_finite_after_run": finite}
 
 
 def adam_sweep(api, torch, ctx, dev, peaks, n):

@@ -244,7 +244,7 @@ GsStatus gs_appearance_backward_noalloc(const GsScene *scene, const float *dirs,
  * pointer to [rows, cols] IEEE fp16 bits (8-byte aligned) that receives the updated values rounded
  * to nearest even, or NULL.  lr: HOST array of cols rates (read during the call).  A decoder-weight
  * vector is a tensor with rows = 816, cols = 1 (App. B.2 sets its beta2 to 0.99). */
-enum { GS_ADAM_MAX_COLS = 64, GS_ADAM_MAX_TENSORS = 8 };
+enum { GS_ADAM_MAX_COLS = 64, GS_ADAM_MAX_TENSORS = 8, GS_ADAM_MAX_MORE_GRADS = 7 };
 typedef struct {
   float *param;
   const float *grad;
@@ -255,6 +255,10 @@ typedef struct {
   int32_t cols;          /* 1 .. GS_ADAM_MAX_COLS; rows * cols < 2^32 */
   const float *lr;
   float beta1, beta2, eps;
+  const float *const *more_grads; /* HOST array of num_more_grads DEVICE pointers, each [rows, cols] fp32 and
+                                     16-byte aligned, or NULL: the gradient of the step is grad plus these
+                                     (the views of an iteration, each with a gradient buffer of its own)  */
+  int32_t num_more_grads;         /* 0 .. GS_ADAM_MAX_MORE_GRADS                                           */
 } GsAdamTensor;
 /* Updates up to GS_ADAM_MAX_TENSORS tensors with ONE kernel launch on `stream` (asynchronous; no
  * allocation, no synchronisation).  step = 1, 2, ... is the number of this update, shared by the

@@ -105,7 +105,7 @@ GS_ADAM_MAX_COLS, GS_ADAM_MAX_TENSORS = 64, 8
 class GsAdamTensor(C.Structure):
     _fields_ = [("param", _vp), ("grad", _vp), ("exp_avg", _vp), ("exp_avg_sq", _vp), ("half_copy", _vp),
                 ("rows", C.c_int64), ("cols", C.c_int32), ("lr", C.POINTER(C.c_float)), ("beta1", C.c_float),
-                ("beta2", C.c_float), ("eps", C.c_float)]
+                ("beta2", C.c_float), ("eps", C.c_float), ("more_grads", C.POINTER(_vp)), ("num_more_grads", C.c_int32)]
 
 
 _lib.gs_adam_step.argtypes = [_vp, C.POINTER(GsAdamTensor), C.c_int32, C.c_int64, _vp]
@@ -439,7 +439,8 @@ class AdamTensor:
     (viewed as [rows, cols] with cols = len(lr)), an optional fp16 tensor that receives the updated
     values, and the hyper-parameters.  Marshalling only."""
 
-    def __init__(self, param, grad, exp_avg, exp_avg_sq, lr, beta1=0.9, beta2=0.999, eps=1e-15, half_copy=None):
+    def __init__(self, param, grad, exp_avg, exp_avg_sq, lr, beta1=0.9, beta2=0.999, eps=1e-15, half_copy=None,
+                 more_grads=()):
         lr = [float(x) for x in (lr if hasattr(lr, "__len__") else [lr])]
         self.cols = len(lr)
         assert param.numel() % self.cols == 0
@@ -447,6 +448,8 @@ class AdamTensor:
         self.param, self.grad, self.exp_avg, self.exp_avg_sq, self.half_copy = param, grad, exp_avg, exp_avg_sq, half_copy
         self.lr = (C.c_float * self.cols)(*lr)          # host array, kept alive by this object
         self.beta1, self.beta2, self.eps = beta1, beta2, eps
+        self.more_grads = list(more_grads)                       # further gradient tensors, summed with grad
+        self._more = (_vp * max(1, len(self.more_grads)))(*[_ptr(g) for g in self.more_grads])
 
     def c_struct(self) -> GsAdamTensor:
         t = GsAdamTensor()
@@ -454,6 +457,8 @@ class AdamTensor:
         t.half_copy = _ptr(self.half_copy)
         t.rows, t.cols, t.lr = self.rows, self.cols, C.cast(self.lr, C.POINTER(C.c_float))
         t.beta1, t.beta2, t.eps = self.beta1, self.beta2, self.eps
+        t.more_grads = C.cast(self._more, C.POINTER(_vp)) if self.more_grads else None
+        t.num_more_grads = len(self.more_grads)
         return t
 
 

@@ -25,6 +25,8 @@ struct AdamTensorDev {
   float beta1, beta2, eps;
   float inv_sqrt_c2;         // 1 / sqrt(1 - beta2^step)
   float step_size[GS_ADAM_MAX_COLS];   // lr_c / (1 - beta1^step)
+  int num_more;
+  const float *more[GS_ADAM_MAX_MORE_GRADS];   // further gradient buffers, summed with grad
 };
 
 struct AdamArgs {
@@ -65,6 +67,10 @@ __global__ void __launch_bounds__(kAdamThreads) k_adam(const __grid_constant__ A
       if (full[u]) {
         p[u] = *reinterpret_cast<const float4 *>(t.param + e[u]);
         g[u] = __ldcs(reinterpret_cast<const float4 *>(t.grad + e[u]));
+        for (int k = 0; k < t.num_more; ++k) {
+          const float4 x = __ldcs(reinterpret_cast<const float4 *>(t.more[k] + e[u]));
+          g[u].x += x.x; g[u].y += x.y; g[u].z += x.z; g[u].w += x.w;
+        }
         m[u] = *reinterpret_cast<const float4 *>(t.m + e[u]);
         v[u] = *reinterpret_cast<const float4 *>(t.v + e[u]);
       }
@@ -93,8 +99,9 @@ __global__ void __launch_bounds__(kAdamThreads) k_adam(const __grid_constant__ A
       } else if (e[u] < t.count) {   // ragged end of the tensor, element by element
         uint32_t c = e[u] % t.cols;
         for (uint32_t i = e[u]; i < t.count; ++i) {
-          float pv = t.param[i], mv = t.m[i], vv = t.v[i];
-          adam_element(pv, t.grad[i], mv, vv, s_step[c], t.beta1, t.beta2, t.eps, t.inv_sqrt_c2);
+          float pv = t.param[i], mv = t.m[i], vv = t.v[i], gv = t.grad[i];
+          for (int k = 0; k < t.num_more; ++k) gv += t.more[k][i];
+          adam_element(pv, gv, mv, vv, s_step[c], t.beta1, t.beta2, t.eps, t.inv_sqrt_c2);
           t.param[i] = pv; t.m[i] = mv; t.v[i] = vv;
           if (t.half_copy) t.half_copy[i] = __float2half_rn(pv);
           c = (c + 1 == t.cols) ? 0u : c + 1;
@@ -124,6 +131,8 @@ int launch_adam(const GsAdamTensor *tensors, int num_tensors, int64_t step, int 
     const double c1 = 1.0 - pow((double)s.beta1, (double)step), c2 = 1.0 - pow((double)s.beta2, (double)step);
     d.inv_sqrt_c2 = (float)(1.0 / sqrt(c2));
     for (int c = 0; c < s.cols; ++c) d.step_size[c] = (float)((double)s.lr[c] / c1);
+    d.num_more = s.more_grads ? s.num_more_grads : 0;
+    for (int k = 0; k < d.num_more; ++k) d.more[k] = s.more_grads[k];
     a.chunk_start[a.num_tensors + 1] = a.chunk_start[a.num_tensors] + (uint32_t)((count + kAdamChunk - 1) / kAdamChunk);
     ++a.num_tensors;
   }

@@ -488,6 +488,10 @@ GsStatus gs_adam_step(GsContext *ctx, const GsAdamTensor *tensors, int32_t num_t
     if (!(t.beta1 >= 0.f && t.beta1 < 1.f && t.beta2 >= 0.f && t.beta2 < 1.f) || !(t.eps >= 0.f))
       return fail(ctx, GS_ERR_INVALID_ARG, "betas must lie in [0, 1) and eps be >= 0");
     if ((uint64_t)t.rows * (uint64_t)t.cols >= (1ull << 32)) return fail(ctx, GS_ERR_CAPACITY, "an Adam tensor has 2^32 elements or more");
+    if (t.num_more_grads < 0 || t.num_more_grads > GS_ADAM_MAX_MORE_GRADS || (t.num_more_grads > 0 && !t.more_grads))
+      return fail(ctx, GS_ERR_INVALID_ARG, "num_more_grads outside 0..7 or more_grads is NULL");
+    for (int k = 0; k < t.num_more_grads; ++k)
+      if (bad_ptr(t.more_grads[k])) return fail(ctx, GS_ERR_INVALID_ARG, "a further gradient pointer is NULL or misaligned");
   }
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   cudaSetDevice(ctx->device);

@@ -126,3 +126,36 @@ def test_adam_argument_errors():
         api.gs_adam_step(ctx, [mis], 1)
     torch.cuda.synchronize()
     ctx.close()
+
+
+def test_adam_sums_the_gradient_buffers_of_several_views(oracle):
+    """grad + more_grads[0..6] is the gradient of the step: against the oracle fed with their sum."""
+    import torch
+    from paper_2609_05255_b200 import api
+    ctx = api.Context(0)
+    dev = ctx.device
+    rng = np.random.default_rng(41)
+    rows, cols, views = 3_001, 8, 8
+    p0 = rng.normal(size=(rows, cols)).astype(np.float32)
+    gs = [(rng.normal(size=(rows, cols)) * 10.0 ** rng.uniform(-4, 0)).astype(np.float32) for _ in range(views)]
+    lr = np.full(cols, 0.008, np.float32)
+    p, m, v = (torch.from_numpy(a).to(dev) for a in (p0.copy(), np.zeros_like(p0), np.zeros_like(p0)))
+    dg = [torch.from_numpy(g).to(dev) for g in gs]
+    half = torch.empty((rows, cols), device=dev, dtype=torch.float16)
+    t = api.AdamTensor(p, dg[0], m, v, lr, 0.9, 0.999, 1e-15, half_copy=half, more_grads=dg[1:])
+    hp, hm, hv = p0.astype(np.float64), np.zeros((rows, cols)), np.zeros((rows, cols))
+    for step in (1, 2, 3):
+        api.gs_adam_step(ctx, [t], step)
+        hp, hm, hv = oracle.adam_step(hp, np.sum([g.astype(np.float64) for g in gs], 0), hm, hv, lr.astype(np.float64),
+                                      F32(0.9), F32(0.999), F32(1e-15), step)
+    torch.cuda.synchronize()
+    # the sum of eight fp32 gradients carries up to 4 ulp of the largest one
+    assert np.all(np.abs(p.cpu().numpy() - hp) <= 1e-6 * np.abs(hp) + 1e-4 * 3 * lr[0])
+    # v is made of (sum g_k)^2: where the eight terms cancel, the fp32 sum is off by up to 5e-7 of sum |g_k|
+    g_sum = np.sum([g.astype(np.float64) for g in gs], 0)
+    e_g = 5e-7 * np.sum([np.abs(g).astype(np.float64) for g in gs], 0)
+    tol_v = 1e-5 * hv + 3 * (1 - F32(0.999)) * (2 * np.abs(g_sum) * e_g + e_g ** 2)
+    assert np.all(np.abs(v.cpu().numpy() - hv) <= tol_v)
+    with pytest.raises(api.GsError):
+        api.gs_adam_step(ctx, [api.AdamTensor(p, dg[0], m, v, lr, more_grads=dg + dg[:1])], 4)      # nine in all: too many
+    ctx.close()
