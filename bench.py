@@ -412,8 +412,9 @@ def measure_e2e_training(api, torch, lane_ctx, lanes, arm, cams, G, views, args,
     neural = arm["app"] == "neural"
     n = ds.n
     rs = [r0] + [api.Renderer(c, n, WIDTH, HEIGHT, r0.app, pair_capacity=r0.pair_capacity) for c in lane_ctx[1:]]
-    grads = [r0.grads] + [api.alloc_grads(n, r0.app, dev) for _ in range(views - 1)]
-    images = [r0.image] + [torch.empty_like(r0.image) for _ in range(views - 1)]
+    group = min(views, 8)              # views per Adam update: one launch sums at most eight gradient sets
+    grads = [r0.grads] + [api.alloc_grads(n, r0.app, dev) for _ in range(group - 1)]
+    images = [r0.image] + [torch.empty_like(r0.image) for _ in range(group - 1)]
     h_G = G.cpu().pin_memory()
     d_G = torch.empty_like(G)
     h_images = torch.empty((views,) + tuple(r0.image.shape), dtype=torch.float32).pin_memory()
@@ -421,16 +422,23 @@ def measure_e2e_training(api, torch, lane_ctx, lanes, arm, cams, G, views, args,
     spec = [("means", 3, 1.6e-6), ("log_scales", 3, 5e-5), ("quats", 4, 1e-5), ("opacity_logits", 1, 5e-4)]
     spec += [("base_color", 3, 0.00025), ("features", 8, 0.008e-2), ("mlp_weights", 1, 0.003e-2)] if neural else \
             [("base_color", 3, 0.0025 * y0 * 1e-2), ("sh_rest", 45, 0.000125e-2)]
-    tensors, masters = [], {}
+    masters, moments = {}, {}
     for name, cols, lr in spec:        # rates scaled down: random upstream gradients must not wreck the synthetic scene
         stored = getattr(ds, name)
-        master = stored.float().contiguous() if stored.dtype != torch.float32 else stored
-        masters[name] = master
-        g0 = getattr(grads[0], name)
-        more = [getattr(g, name) for g in grads[1:]]
-        tensors.append(api.AdamTensor(master, g0, torch.zeros_like(master), torch.zeros_like(master), [lr] * cols, 0.9,
-                                      0.99 if name == "mlp_weights" else 0.999, 1e-15,
-                                      half_copy=stored if stored.dtype == torch.float16 else None, more_grads=more))
+        masters[name] = stored.float().contiguous() if stored.dtype != torch.float32 else stored
+        moments[name] = (torch.zeros_like(masters[name]), torch.zeros_like(masters[name]))
+
+    def adam_tensors(count):           # the update that sums the first `count` gradient sets
+        out = []
+        for name, cols, lr in spec:
+            stored = getattr(ds, name)
+            out.append(api.AdamTensor(masters[name], getattr(grads[0], name), moments[name][0], moments[name][1], [lr] * cols,
+                                      0.9, 0.99 if name == "mlp_weights" else 0.999, 1e-15,
+                                      half_copy=stored if stored.dtype == torch.float16 else None,
+                                      more_grads=[getattr(g, name) for g in grads[1:count]]))
+        return out
+
+    tensors_for = {c: adam_tensors(c) for c in {min(group, views - b) for b in range(0, views, group)}}
     main = torch.cuda.current_stream(dev)
     up, down = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
     ev_up = [torch.cuda.Event() for _ in range(views)]
@@ -439,28 +447,33 @@ def measure_e2e_training(api, torch, lane_ctx, lanes, arm, cams, G, views, args,
     L = len(lanes)
 
     def step():
-        state["step"] += 1
         up.wait_stream(main)                       # the previous step's kernels have read d_G
         with torch.cuda.stream(up):
             for v in range(views):
                 d_G[v].copy_(h_G[v], non_blocking=True)
                 ev_up[v].record(up)
         down.wait_stream(main)
-        for s in lanes:
-            s.wait_stream(main)                    # the parameters of this step are in place
-        for v in range(views):
-            r, s = rs[v % L], lanes[v % L]
-            s.wait_event(ev_up[v])
-            r.image, r.grads = images[v], grads[v]
-            r.forward_async(ds, cams[v], stream=s)
-            r.backward(ds, cams[v], d_G[v], stream=s)
-            ev_done[v].record(s)
-            with torch.cuda.stream(down):
-                down.wait_event(ev_done[v])
-                h_images[v].copy_(images[v], non_blocking=True)
-        for s in lanes:
-            main.wait_stream(s)
-        api.gs_adam_step(lane_ctx[0], tensors, state["step"])
+        for b in range(0, views, group):
+            for s in lanes:
+                s.wait_stream(main)                # the parameters of this group are in place
+            count = min(group, views - b)
+            for k in range(count):
+                v = b + k
+                r, s = rs[v % L], lanes[v % L]
+                s.wait_event(ev_up[v])
+                r.image, r.grads = images[k], grads[k]
+                r.forward_async(ds, cams[v], stream=s)
+                r.backward(ds, cams[v], d_G[v], stream=s)
+                ev_done[v].record(s)
+                with torch.cuda.stream(down):
+                    down.wait_event(ev_done[v])
+                    h_images[v].copy_(images[k], non_blocking=True)
+            for s in lanes:
+                main.wait_stream(s)
+            if b + group < views:
+                main.wait_stream(down)             # the next group renders into the same image buffers
+            state["step"] += 1
+            api.gs_adam_step(lane_ctx[0], tensors_for[count], state["step"])
         main.wait_stream(down)
 
     ms = timed(step, max(2, args.steps // 2), 2)
@@ -468,7 +481,7 @@ def measure_e2e_training(api, torch, lane_ctx, lanes, arm, cams, G, views, args,
         api.gs_async_status(c, s_)
     finite = all(bool(torch.isfinite(m).all()) for m in masters.values())
     r0.image, r0.grads = images[0], grads[0]
-    return {"value": ms, "unit": f"ms/iter ({views} views, fwd+bwd, + one fused Adam update)",
+    return {"value": ms, "unit": f"ms/iter ({views} views, fwd+bwd, + one fused Adam update per {group} views)",
             "h2d_bytes_per_step": int(h_G.numel() * 4), "d2h_bytes_per_step": int(h_images.numel() * 4),
             "what": "upstream gradients in, rendered images out, parameters stay on the device and are updated by Adam",
             "streams": L, "parameters_finite_after_run": finite}
