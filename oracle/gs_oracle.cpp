@@ -147,6 +147,55 @@ double color_act_grad(int act, double x) {
   }
 }
 
+// Spherical Voronoi residual (Eq. 3, App. B "Spherical Voronoi"): kSites sites per Gaussian, seven raw
+// parameters each, in the order (a_r, a_g, a_b, s_x, s_y, s_z, t): colour a, unnormalised site direction,
+// log-temperature.  s = raw / |raw|, tau = exp(t), rho = |s - d| (chord distance),
+//   A(d) = sum_i softmax_i(-tau_i rho_i) a_i.
+constexpr int kSites = 7, kSiteP = 7;
+struct SvState { double s[kSites][3], tau[kSites], rho[kSites], w[kSites], len[kSites]; };
+void sv_forward(const double* site, const double d[3], double A[3], SvState& st) {
+  double logit[kSites], mx = -1e300;
+  for (int i = 0; i < kSites; ++i) {
+    const double* p = site + kSiteP * i;
+    st.len[i] = std::sqrt(p[3] * p[3] + p[4] * p[4] + p[5] * p[5]);
+    for (int c = 0; c < 3; ++c) st.s[i][c] = p[3 + c] / st.len[i];
+    st.tau[i] = std::exp(p[6]);
+    const double e[3] = {st.s[i][0] - d[0], st.s[i][1] - d[1], st.s[i][2] - d[2]};
+    st.rho[i] = std::sqrt(e[0] * e[0] + e[1] * e[1] + e[2] * e[2]);
+    logit[i] = -st.tau[i] * st.rho[i];
+    mx = std::max(mx, logit[i]);
+  }
+  double z = 0;
+  for (int i = 0; i < kSites; ++i) { st.w[i] = std::exp(logit[i] - mx); z += st.w[i]; }
+  A[0] = A[1] = A[2] = 0;
+  for (int i = 0; i < kSites; ++i) {
+    st.w[i] /= z;
+    for (int c = 0; c < 3; ++c) A[c] += st.w[i] * site[kSiteP * i + c];
+  }
+}
+// gA = dL/dA.  g_site [7,7] (written), g_d[3] (added to).  Where rho = 0 the distance has no gradient.
+void sv_backward(const double* site, const double d[3], const double gA[3], const SvState& st, const double A[3],
+                 double* g_site, double g_d[3]) {
+  const double Ag = A[0] * gA[0] + A[1] * gA[1] + A[2] * gA[2];
+  for (int i = 0; i < kSites; ++i) {
+    const double* p = site + kSiteP * i;
+    double* g = g_site + kSiteP * i;
+    for (int c = 0; c < 3; ++c) g[c] = st.w[i] * gA[c];
+    const double g_logit = st.w[i] * (p[0] * gA[0] + p[1] * gA[1] + p[2] * gA[2] - Ag);
+    g[6] = -st.rho[i] * g_logit * st.tau[i];                 // through tau = exp(t)
+    const double g_rho = -st.tau[i] * g_logit;
+    double gs[3] = {0, 0, 0};
+    if (st.rho[i] > 0)
+      for (int c = 0; c < 3; ++c) {
+        const double u = (st.s[i][c] - d[c]) / st.rho[i];
+        gs[c] = g_rho * u;
+        g_d[c] -= g_rho * u;
+      }
+    const double dot = gs[0] * st.s[i][0] + gs[1] * st.s[i][1] + gs[2] * st.s[i][2];   // through the normalisation
+    for (int c = 0; c < 3; ++c) g[3 + c] = (gs[c] - dot * st.s[i][c]) / st.len[i];
+  }
+}
+
 // Eq. 5-7: x = (Y_0..15(d) masked by the active degree, (sin f_j, cos f_j)_j); two ReLU
 // layers; A = tanh(W3 h2).
 void mlp_forward(const double* W, const double d[3], const double* f, int deg, MlpState& s) {
@@ -411,6 +460,8 @@ void gso_appearance_forward(int64_t n, int app, int deg, int act, const double* 
       sh_basis(dirs + 3 * i, Y);
       for (int k = 1; k < num_active(deg); ++k)
         for (int c = 0; c < 3; ++c) A[c] += Y[k] * sh_rest[(i * 15 + (k - 1)) * 3 + c];
+    } else if (app == 2) {   // Spherical Voronoi: the sites travel in the sh_rest argument, [n,7,7]
+      if (deg > 0) { SvState st; sv_forward(sh_rest + (size_t)i * kSites * kSiteP, dirs + 3 * i, A, st); }
     } else if (deg > 0) {
       MlpState s;
       mlp_forward(weights, dirs + 3 * i, features + kFeat * i, deg, s);
@@ -447,6 +498,7 @@ void gso_appearance_backward(int64_t n, int app, int deg, int act, const double*
       const int64_t i = base + ii;
       for (int c = 0; c < 3; ++c) { g_base[3 * i + c] = 0; g_dirs[3 * i + c] = 0; }
       if (app == 0) for (int k = 0; k < 45; ++k) g_sh_rest[45 * i + k] = 0;
+      if (app == 2) for (int k = 0; k < kSites * kSiteP; ++k) g_sh_rest[(size_t)kSites * kSiteP * i + k] = 0;
       if (app == 1) {
         for (int k = 0; k < kFeat; ++k) g_features[kFeat * i + k] = 0;
         std::fill(gw_rows.begin() + ii * kNumW, gw_rows.begin() + (ii + 1) * kNumW, 0.0);
@@ -470,6 +522,15 @@ void gso_appearance_backward(int64_t n, int app, int deg, int act, const double*
             for (int a = 0; a < 3; ++a) g_dirs[3 * i + a] += G[k][a] * w;
           }
         }
+      } else if (app == 2) {   // Spherical Voronoi: sites in sh_rest, their gradients in g_sh_rest, [n,7,7]
+        double A[3] = {0, 0, 0}, gp[3];
+        SvState st;
+        if (deg > 0) sv_forward(sh_rest + (size_t)i * kSites * kSiteP, d, A, st);
+        for (int c = 0; c < 3; ++c) {
+          gp[c] = color_act_grad(act, base_color[3 * i + c] + A[c]) * g_color[3 * i + c];
+          g_base[3 * i + c] = gp[c];
+        }
+        if (deg > 0) sv_backward(sh_rest + (size_t)i * kSites * kSiteP, d, gp, st, A, g_sh_rest + (size_t)i * kSites * kSiteP, g_dirs + 3 * i);
       } else {
         if (deg == 0) {
           for (int c = 0; c < 3; ++c) {

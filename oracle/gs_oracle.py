@@ -180,7 +180,7 @@ def preprocess(means, log_scales, quats, opacity_logits, cam):
 
 
 def _app_args(scene):
-    sh = _f64(scene.sh_rest) if scene.app == 0 else None
+    sh = _f64(scene.sh_rest) if scene.app == 0 else (_f64(scene.sv_sites) if scene.app == 2 else None)
     ft = _f64(scene.features) if scene.app == 1 else None
     wt = _f64(scene.mlp_weights) if scene.app == 1 else None
     return _f64(scene.base_color), sh, ft, wt
@@ -203,14 +203,16 @@ def appearance_backward(scene, dirs, g_color, mask=None, deg=None):
     deg = scene.active_degree if deg is None else deg
     m = None if mask is None else np.ascontiguousarray(mask, np.uint8)
     o = SimpleNamespace(base_color=np.zeros((n, 3)), dirs=np.zeros((n, 3)), sh_rest=None,
-                        features=None, mlp_weights=None)
+                        features=None, mlp_weights=None, sv_sites=None)
     if scene.app == 0:
         o.sh_rest = np.zeros((n, 15, 3))
+    elif scene.app == 2:
+        o.sv_sites = np.zeros((n, 7, 7))
     else:
         o.features = np.zeros((n, 8)); o.mlp_weights = np.zeros(num_mlp_weights())
     lib().gso_appearance_backward(C.c_int64(n), C.c_int(scene.app), C.c_int(deg), C.c_int(_act(scene)), _dp(base), _dp(sh),
                                   _dp(ft), _dp(wt), _dp(dirs), _p(m, C.c_uint8), _dp(g_color),
-                                  _dp(o.base_color), _dp(o.sh_rest), _dp(o.features),
+                                  _dp(o.base_color), _dp(o.sv_sites if scene.app == 2 else o.sh_rest), _dp(o.features),
                                   _dp(o.mlp_weights), _dp(o.dirs))
     return o
 
@@ -361,7 +363,7 @@ def render_backward(scene, cam, fwd, G, with_abs=False):
                              pre.visible, g2.mean2d, g2.conic, g2.opacity, ga.dirs)
     return SimpleNamespace(means=gp.means, log_scales=gp.log_scales, quats=gp.quats,
                            opacity_logits=gp.opacity_logits, base_color=ga.base_color,
-                           sh_rest=ga.sh_rest, features=ga.features, mlp_weights=ga.mlp_weights,
+                           sh_rest=ga.sh_rest, features=ga.features, mlp_weights=ga.mlp_weights, sv_sites=ga.sv_sites,
                            blend=g2, dirs=ga.dirs)
 
 

@@ -18,6 +18,8 @@ import numpy as np
 
 APP_SH = 0
 APP_NEURAL = 1
+APP_SV = 2          # Spherical Voronoi (Eq. 3)
+SV_SITES = 7
 
 # Layer sizes of the shared decoder (Sec. 4, "two hidden layers of 16 neurons, three
 # outputs", 32 inputs): 32*16 + 16*16 + 16*3 = 816 weights, no biases.
@@ -56,6 +58,7 @@ class Scene:
     features: Optional[np.ndarray] = None     # [n,8]  f16
     mlp_weights: Optional[np.ndarray] = None  # [816]  f16: W1[16][32], W2[16][16], W3[3][16]
     color_activation: int = 0                 # 0 ReLU(x+0.5), 1 softplus(x+0.5) beta 10, 2 sigmoid(4x), 3 clamp(x+0.5,0,1)
+    sv_sites: Optional[np.ndarray] = None     # [n,7,7] f32: per site (a_r, a_g, a_b, s_x, s_y, s_z, log tau)
 
     @property
     def n(self) -> int:
@@ -115,10 +118,36 @@ def draw_neural_appearance(rng, n):
     return base_color, features, mlp_weights
 
 
+def fibonacci_sites(count: int) -> np.ndarray:
+    """`count` directions spread over the sphere on a Fibonacci lattice."""
+    k = np.arange(count) + 0.5
+    z = 1.0 - 2.0 * k / count
+    phi = math.pi * (1.0 + math.sqrt(5.0)) * k
+    r = np.sqrt(1.0 - z * z)
+    return np.stack([r * np.cos(phi), r * np.sin(phi), z], 1)
+
+
+def draw_sv_appearance(rng, n):
+    """Spherical Voronoi: 7 sites per Gaussian, each (colour a [3], unnormalised direction s [3], log-temperature t).
+    Sites start on a shared Fibonacci lattice (as the paper initialises them) and are perturbed and rescaled so
+    that normalisation, temperatures and colours all matter."""
+    dc = rng.normal(0.5, 0.1, (n, 3))
+    base_color = _f32(_Y0 * dc)
+    sites = np.empty((n, SV_SITES, 7))
+    sites[:, :, 0:3] = rng.normal(0.0, 0.15, (n, SV_SITES, 3))
+    lattice = fibonacci_sites(SV_SITES)[None] + rng.normal(0.0, 0.25, (n, SV_SITES, 3))
+    sites[:, :, 3:6] = lattice * rng.uniform(0.5, 2.0, (n, SV_SITES, 1))
+    sites[:, :, 6] = rng.normal(0.5, 0.5, (n, SV_SITES))
+    return base_color, _f32(sites)
+
+
 def _attach_appearance(rng, n, app, geom) -> Scene:
     if app == APP_SH:
         base_color, sh_rest = draw_sh_appearance(rng, n)
         return Scene(*geom, base_color=base_color, app=APP_SH, active_degree=3, sh_rest=sh_rest)
+    if app == APP_SV:
+        base_color, sites = draw_sv_appearance(rng, n)
+        return Scene(*geom, base_color=base_color, app=APP_SV, active_degree=3, sv_sites=sites)
     base_color, features, weights = draw_neural_appearance(rng, n)
     return Scene(*geom, base_color=base_color, app=APP_NEURAL, active_degree=3,
                  features=features, mlp_weights=weights)
