@@ -41,10 +41,16 @@ typedef enum {
   GS_ERR_INTERNAL = -6
 } GsStatus;
 
-typedef enum { GS_APP_SH = 0, GS_APP_NEURAL = 1 } GsAppearance;
+typedef enum {
+  GS_APP_SH = 0,      /* spherical harmonics, degrees 1..3 (Eq. 1)                              */
+  GS_APP_NEURAL = 1,  /* latent features + shared decoder (Eq. 5-7)                             */
+  GS_APP_SV = 2       /* Spherical Voronoi: soft interpolation over seven sites (Eq. 3)         */
+} GsAppearance;
 
 enum {
   GS_TILE = 16,            /* tile edge in pixels (Sec. 3.1)                                    */
+  GS_SV_SITES = 7,         /* Spherical Voronoi sites per Gaussian (App. B)                       */
+  GS_SV_ROW = 49,          /* 7 sites x (colour a [3], unnormalised direction s [3], log-temperature) */
   GS_SH_REST = 45,         /* view-dependent SH coefficients per Gaussian, degrees 1..3, x RGB  */
   GS_NUM_FEATURES = 8,     /* F, latent features per Gaussian (Sec. 4)                          */
   GS_MLP_IN = 32,          /* D = 16 direction encodings + 16 feature encodings (Eq. 5)         */
@@ -89,6 +95,10 @@ typedef struct {
                                     of the direction, then (sin f_j, cos f_j) per feature
                                     (Eq. 5, Eq. 6 with k = 1)                                  */
   int32_t color_activation;      /* GsColorActivation: phi of c = phi(c0 + A(d)) (Sec. 3.1)    */
+  const float *sv_sites;         /* SV only: [n,7,7] raw site parameters, per site (a_r, a_g, a_b, s_x,
+                                    s_y, s_z, t): A(d) = sum_i softmax_i(-exp(t_i) |s_i/|s_i| - d|) a_i
+                                    (Eq. 3 with the chord distance of App. B); any active_degree >= 1
+                                    uses all seven sites, 0 disables the residual                  */
 } GsScene;
 
 /* Per-Gaussian results of gs_preprocess (caller-allocated device buffers). */
@@ -131,6 +141,7 @@ typedef struct {
   float *sh_rest;         /* SH:     [n,15,3]                                                  */
   float *features;        /* neural: [n,8] fp32                                                */
   float *mlp_weights;     /* neural: [816] fp32, summed over all visible Gaussians             */
+  float *sv_sites;        /* SV:     [n,7,7] with respect to the raw site parameters            */
 } GsGrads;
 
 /* Create / destroy a context on CUDA device `device`.  The context owns a few KB of device and

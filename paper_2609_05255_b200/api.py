@@ -23,7 +23,7 @@ if not os.path.exists(LIB_PATH):
 _lib = C.CDLL(LIB_PATH)
 
 GS_OK, GS_ERR_INVALID_ARG, GS_ERR_CAPACITY, GS_ERR_CUDA, GS_ERR_UNSUPPORTED, GS_ERR_INTERNAL = 0, -1, -2, -3, -4, -6
-GS_APP_SH, GS_APP_NEURAL = 0, 1
+GS_APP_SH, GS_APP_NEURAL, GS_APP_SV = 0, 1, 2
 TILE = 16
 MLP_WEIGHTS = 816
 
@@ -39,7 +39,7 @@ class GsCamera(C.Structure):
 class GsScene(C.Structure):
     _fields_ = [("n", C.c_int64), ("means", _vp), ("log_scales", _vp), ("quats", _vp), ("opacity_logits", _vp),
                 ("base_color", _vp), ("app", C.c_int32), ("active_degree", C.c_int32), ("sh_rest", _vp),
-                ("features", _vp), ("mlp_weights", _vp), ("color_activation", C.c_int32)]
+                ("features", _vp), ("mlp_weights", _vp), ("color_activation", C.c_int32), ("sv_sites", _vp)]
 
 
 class GsProjected(C.Structure):
@@ -54,7 +54,7 @@ class GsBinning(C.Structure):
 
 class GsGrads(C.Structure):
     _fields_ = [("means", _vp), ("log_scales", _vp), ("quats", _vp), ("opacity_logits", _vp), ("base_color", _vp),
-                ("sh_rest", _vp), ("features", _vp), ("mlp_weights", _vp)]
+                ("sh_rest", _vp), ("features", _vp), ("mlp_weights", _vp), ("sv_sites", _vp)]
 
 
 _lib.gs_create.argtypes = [C.c_int, C.POINTER(_vp)]
@@ -159,6 +159,7 @@ class DeviceScene:
     features: Optional[torch.Tensor] = None
     mlp_weights: Optional[torch.Tensor] = None
     color_activation: int = 0        # GS_ACT_*: 0 ReLU(x+0.5), 1 softplus beta 10, 2 sigmoid(4x), 3 clamp(x+0.5, 0, 1)
+    sv_sites: Optional[torch.Tensor] = None      # Spherical Voronoi: [n,7,7]
 
     @property
     def n(self) -> int:
@@ -172,6 +173,7 @@ class DeviceScene:
         s.app, s.active_degree = int(self.app), int(self.active_degree)
         s.sh_rest, s.features, s.mlp_weights = _ptr(self.sh_rest), _ptr(self.features), _ptr(self.mlp_weights)
         s.color_activation = int(self.color_activation)
+        s.sv_sites = _ptr(self.sv_sites)
         return s
 
 
@@ -183,7 +185,8 @@ def upload_scene(scene, device="cuda") -> DeviceScene:
                        up(scene.quats, torch.float32), up(scene.opacity_logits, torch.float32),
                        up(scene.base_color, torch.float32), int(scene.app), int(scene.active_degree),
                        up(scene.sh_rest, torch.float32), up(scene.features, torch.float16),
-                       up(scene.mlp_weights, torch.float16), int(getattr(scene, "color_activation", 0)))
+                       up(scene.mlp_weights, torch.float16), int(getattr(scene, "color_activation", 0)),
+                       up(getattr(scene, "sv_sites", None), torch.float32))
 
 
 @dataclass
@@ -248,12 +251,14 @@ class Grads:
     sh_rest: Optional[torch.Tensor] = None
     features: Optional[torch.Tensor] = None
     mlp_weights: Optional[torch.Tensor] = None
+    sv_sites: Optional[torch.Tensor] = None
 
     def c_struct(self) -> GsGrads:
         g = GsGrads()
         g.means, g.log_scales, g.quats = _ptr(self.means), _ptr(self.log_scales), _ptr(self.quats)
         g.opacity_logits, g.base_color = _ptr(self.opacity_logits), _ptr(self.base_color)
         g.sh_rest, g.features, g.mlp_weights = _ptr(self.sh_rest), _ptr(self.features), _ptr(self.mlp_weights)
+        g.sv_sites = _ptr(self.sv_sites)
         return g
 
 
@@ -264,6 +269,8 @@ def alloc_grads(n: int, app: int, device) -> Grads:
               torch.empty((m,), **f), torch.empty((m, 3), **f))
     if app == GS_APP_SH:
         g.sh_rest = torch.empty((m, 15, 3), **f)
+    elif app == GS_APP_SV:
+        g.sv_sites = torch.empty((m, 7, 7), **f)
     else:
         g.features = torch.empty((m, 8), **f)
         g.mlp_weights = torch.empty((MLP_WEIGHTS,), **f)

@@ -91,7 +91,7 @@ CamDev make_cam(const GsCamera *c) {
 }
 
 GsStatus scene_appearance_ok(GsContext *ctx, const GsScene *s) {
-  if (s->app != GS_APP_SH && s->app != GS_APP_NEURAL) return fail(ctx, GS_ERR_INVALID_ARG, "unknown appearance model");
+  if (s->app != GS_APP_SH && s->app != GS_APP_NEURAL && s->app != GS_APP_SV) return fail(ctx, GS_ERR_INVALID_ARG, "unknown appearance model");
   if (s->active_degree < 0 || s->active_degree > 3) return fail(ctx, GS_ERR_INVALID_ARG, "active_degree must be 0..3");
   if (s->color_activation < GS_ACT_RELU || s->color_activation > GS_ACT_HARD_SIGMOID)
     return fail(ctx, GS_ERR_INVALID_ARG, "unknown colour activation");
@@ -99,6 +99,7 @@ GsStatus scene_appearance_ok(GsContext *ctx, const GsScene *s) {
   if (s->n == 0) return GS_OK;
   if (bad_ptr(s->base_color)) return fail(ctx, GS_ERR_INVALID_ARG, "base_color is NULL or misaligned");
   if (s->app == GS_APP_SH && bad_ptr(s->sh_rest)) return fail(ctx, GS_ERR_INVALID_ARG, "sh_rest is NULL or misaligned");
+  if (s->app == GS_APP_SV && bad_ptr(s->sv_sites)) return fail(ctx, GS_ERR_INVALID_ARG, "sv_sites is NULL or misaligned");
   if (s->app == GS_APP_NEURAL && (bad_ptr(s->features) || bad_ptr(s->mlp_weights)))
     return fail(ctx, GS_ERR_INVALID_ARG, "features / mlp_weights is NULL or misaligned");
   return GS_OK;
@@ -226,7 +227,7 @@ GsStatus preprocess_impl(GsContext *ctx, const GsScene *scene, const GsCamera *c
   PreprocessArgs a;
   a.n = scene->n;
   a.means = scene->means; a.log_scales = scene->log_scales; a.quats = scene->quats; a.logits = scene->opacity_logits;
-  a.base_color = scene->base_color; a.sh_rest = scene->sh_rest;
+  a.base_color = scene->base_color; a.sh_rest = scene->app == GS_APP_SV ? scene->sv_sites : scene->sh_rest;
   a.features = reinterpret_cast<const __half *>(scene->features);
   a.weights = reinterpret_cast<const __half *>(scene->mlp_weights);
   a.deg = scene->active_degree; a.act = scene->color_activation;
@@ -358,6 +359,8 @@ GsStatus gs_render_backward(GsContext *ctx, const GsScene *scene, const GsCamera
         bad_ptr(grads->opacity_logits) || bad_ptr(grads->base_color))
       return fail(ctx, GS_ERR_INVALID_ARG, "a gradient buffer is NULL or misaligned");
     if (scene->app == GS_APP_SH && bad_ptr(grads->sh_rest)) return fail(ctx, GS_ERR_INVALID_ARG, "grads->sh_rest is NULL or misaligned");
+  if (scene->app == GS_APP_SV && bad_ptr(grads->sv_sites)) return fail(ctx, GS_ERR_INVALID_ARG, "grads->sv_sites is NULL or misaligned");
+    if (scene->app == GS_APP_SV && bad_ptr(grads->sv_sites)) return fail(ctx, GS_ERR_INVALID_ARG, "grads->sv_sites is NULL or misaligned");
     if (scene->app == GS_APP_NEURAL && bad_ptr(grads->features)) return fail(ctx, GS_ERR_INVALID_ARG, "grads->features is NULL or misaligned");
     if (bad_ptr(proj->mean2d) || bad_ptr(proj->conic_opacity) || bad_ptr(proj->color) || bad_ptr(proj->rect))
       return fail(ctx, GS_ERR_INVALID_ARG, "a GsProjected buffer is NULL or misaligned");
@@ -380,13 +383,14 @@ GsStatus gs_render_backward(GsContext *ctx, const GsScene *scene, const GsCamera
   PreprocessBwdArgs a;
   a.n = n;
   a.means = scene->means; a.log_scales = scene->log_scales; a.quats = scene->quats; a.logits = scene->opacity_logits;
-  a.base_color = scene->base_color; a.sh_rest = scene->sh_rest;
+  a.base_color = scene->base_color; a.sh_rest = scene->app == GS_APP_SV ? scene->sv_sites : scene->sh_rest;
   a.features = reinterpret_cast<const __half *>(scene->features);
   a.weights = reinterpret_cast<const __half *>(scene->mlp_weights);
   a.deg = scene->active_degree; a.act = scene->color_activation;
   a.rect = proj->rect; a.g2d = g2d;
   a.g_means = grads->means; a.g_log_scales = grads->log_scales; a.g_quats = grads->quats;
-  a.g_logits = grads->opacity_logits; a.g_base = grads->base_color; a.g_sh_rest = grads->sh_rest;
+  a.g_logits = grads->opacity_logits; a.g_base = grads->base_color;
+  a.g_sh_rest = scene->app == GS_APP_SV ? grads->sv_sites : grads->sh_rest;
   a.g_features = grads->features; a.w_partials = ctx->d_w_partials; a.g_weights = grads->mlp_weights;
   if (n == 0 && scene->app == GS_APP_NEURAL)
     return check_cuda(ctx, cudaMemsetAsync(grads->mlp_weights, 0, sizeof(float) * GS_MLP_WEIGHTS, s), "memset");
@@ -408,7 +412,7 @@ GsStatus gs_appearance_forward(GsContext *ctx, const GsScene *scene, const float
   AppearanceArgs a;
   memset(&a, 0, sizeof(a));
   a.n = scene->n; a.deg = scene->active_degree; a.act = scene->color_activation;
-  a.base_color = scene->base_color; a.sh_rest = scene->sh_rest; a.dirs = dirs;
+  a.base_color = scene->base_color; a.sh_rest = scene->app == GS_APP_SV ? scene->sv_sites : scene->sh_rest; a.dirs = dirs;
   a.features = reinterpret_cast<const __half *>(scene->features);
   a.weights = reinterpret_cast<const __half *>(scene->mlp_weights);
   a.color = color;
@@ -437,15 +441,17 @@ GsStatus gs_appearance_backward(GsContext *ctx, const GsScene *scene, const floa
   if (bad_ptr(dirs) || bad_ptr(dL_dcolor) || bad_ptr(dL_ddirs) || bad_ptr(grads->base_color))
     return fail(ctx, GS_ERR_INVALID_ARG, "dirs / dL_dcolor / dL_ddirs / grads->base_color is NULL or misaligned");
   if (scene->app == GS_APP_SH && bad_ptr(grads->sh_rest)) return fail(ctx, GS_ERR_INVALID_ARG, "grads->sh_rest is NULL or misaligned");
+  if (scene->app == GS_APP_SV && bad_ptr(grads->sv_sites)) return fail(ctx, GS_ERR_INVALID_ARG, "grads->sv_sites is NULL or misaligned");
   if (scene->app == GS_APP_NEURAL && bad_ptr(grads->features)) return fail(ctx, GS_ERR_INVALID_ARG, "grads->features is NULL or misaligned");
   AppearanceArgs a;
   memset(&a, 0, sizeof(a));
   a.n = scene->n; a.deg = scene->active_degree; a.act = scene->color_activation;
-  a.base_color = scene->base_color; a.sh_rest = scene->sh_rest; a.dirs = dirs;
+  a.base_color = scene->base_color; a.sh_rest = scene->app == GS_APP_SV ? scene->sv_sites : scene->sh_rest; a.dirs = dirs;
   a.features = reinterpret_cast<const __half *>(scene->features);
   a.weights = reinterpret_cast<const __half *>(scene->mlp_weights);
   a.g_color = dL_dcolor;
-  a.g_base = grads->base_color; a.g_sh_rest = grads->sh_rest; a.g_features = grads->features; a.g_dirs = dL_ddirs;
+  a.g_base = grads->base_color; a.g_sh_rest = scene->app == GS_APP_SV ? grads->sv_sites : grads->sh_rest;
+  a.g_features = grads->features; a.g_dirs = dL_ddirs;
   a.w_partials = ctx->d_w_partials; a.g_weights = grads->mlp_weights;
   {
     StageTimer t(ctx, GS_STAGE_APPEARANCE_BWD, s);

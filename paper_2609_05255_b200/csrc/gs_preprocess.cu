@@ -14,13 +14,17 @@ namespace {
 
 constexpr int kBlock = 128;
 constexpr int kWarps = kBlock / 32;
-constexpr int kRow = GS_SH_REST;           // 45 floats per Gaussian
-constexpr int kSlab = 32 * kRow;           // one warp's slab of SH rows
+// Floats per Gaussian of the explicit models' parameter rows: 45 SH coefficients (bands 1..3, RGB) or the
+// 7 x 7 raw site parameters of Spherical Voronoi.  Both are odd, so a lane reading its own row in a
+// warp's shared-memory slab of 32 rows meets no bank conflict.
+template <int APP> struct RowOf { static constexpr int value = APP == GS_APP_SV ? GS_SV_ROW : GS_SH_REST; };
+template <int APP> struct SlabOf { static constexpr int value = 32 * RowOf<APP>::value; };
 constexpr unsigned kFull = 0xffffffffu;
 
 __device__ __forceinline__ bool finite_f(float x) { return fabsf(x) <= FLT_MAX; }
 
 // ---- warp-cooperative row movement ----------------------------------------------------------
+template <int kRow>
 __device__ __forceinline__ void warp_load_rows(const float *g, int64_t row0, int64_t n, float *slab,
                                                int lane) {
   const int rows = (int)min((int64_t)32, n - row0);
@@ -32,6 +36,7 @@ __device__ __forceinline__ void warp_load_rows(const float *g, int64_t row0, int
   __syncwarp();
 }
 
+template <int kRow>
 __device__ __forceinline__ void warp_store_rows(float *g, int64_t row0, int64_t n, const float *slab,
                                                 int lane) {
   __syncwarp();
@@ -84,6 +89,88 @@ __device__ __forceinline__ void sh_backward(float *row, const float gp[3], float
     }
   }
   gd[0] = gx; gd[1] = gy; gd[2] = gz;
+}
+
+// ---- appearance: Spherical Voronoi (Eq. 3) ---------------------------------------------------
+// row = this Gaussian's 7 sites x (a_r, a_g, a_b, s_x, s_y, s_z, t) in shared memory.  s = raw / |raw|,
+// tau = exp(t), rho = |s - d|, A = sum_i softmax_i(-tau_i rho_i) a_i.  One pass over the sites with a running
+// maximum (App. B): when a larger logit turns up, what has been summed so far is rescaled.
+__device__ __forceinline__ float sv_logit(const float *p, float dx, float dy, float dz) {
+  const float inv = rsqrtf(fmaf(p[3], p[3], fmaf(p[4], p[4], p[5] * p[5])));
+  const float ex = fmaf(p[3], inv, -dx), ey = fmaf(p[4], inv, -dy), ez = fmaf(p[5], inv, -dz);
+  return -expf(p[6]) * sqrtf(fmaf(ex, ex, fmaf(ey, ey, ez * ez)));
+}
+__device__ __forceinline__ void sv_decode(const float *row, float dx, float dy, float dz, float A[3], float &mx, float &z) {
+  mx = -FLT_MAX; z = 0.f;
+  float r = 0.f, g = 0.f, b = 0.f;
+#pragma unroll
+  for (int i = 0; i < GS_SV_SITES; ++i) {
+    const float *p = row + 7 * i;
+    const float l = sv_logit(p, dx, dy, dz);
+    if (l > mx) { const float sc = expf(mx - l); z *= sc; r *= sc; g *= sc; b *= sc; mx = l; }
+    const float e = expf(l - mx);
+    z += e; r = fmaf(e, p[0], r); g = fmaf(e, p[1], g); b = fmaf(e, p[2], b);
+  }
+  const float iz = 1.f / z;
+  A[0] = r * iz; A[1] = g * iz; A[2] = b * iz;
+}
+// Backward, second pass (the first is sv_decode, which leaves A, the maximum and the normaliser): writes the
+// site gradients over `row` in place and returns dL/dd.  gA = dL/dA.
+__device__ __forceinline__ void sv_backward(float *row, const float gA[3], const float A[3], float mx, float z, float dx,
+                                            float dy, float dz, float gd[3]) {
+  const float Ag = A[0] * gA[0] + A[1] * gA[1] + A[2] * gA[2], iz = 1.f / z;
+  float gx = 0.f, gy = 0.f, gz = 0.f;
+#pragma unroll
+  for (int i = 0; i < GS_SV_SITES; ++i) {
+    float *p = row + 7 * i;
+    const float a0 = p[0], a1 = p[1], a2 = p[2];
+    const float len2 = fmaf(p[3], p[3], fmaf(p[4], p[4], p[5] * p[5]));
+    const float inv = rsqrtf(len2);
+    const float sx = p[3] * inv, sy = p[4] * inv, sz = p[5] * inv;
+    const float ex = sx - dx, ey = sy - dy, ez = sz - dz;
+    const float rho = sqrtf(fmaf(ex, ex, fmaf(ey, ey, ez * ez)));
+    const float tau = expf(p[6]);
+    const float w = expf(-tau * rho - mx) * iz;
+    const float g_logit = w * (a0 * gA[0] + a1 * gA[1] + a2 * gA[2] - Ag);
+    const float g_rho = -tau * g_logit;
+    const float ir = rho > 0.f ? 1.f / rho : 0.f;      // no gradient of the distance where it vanishes
+    const float ux = g_rho * ex * ir, uy = g_rho * ey * ir, uz = g_rho * ez * ir;   // dL/ds
+    gx -= ux; gy -= uy; gz -= uz;
+    const float dot = ux * sx + uy * sy + uz * sz;     // through the normalisation
+    p[0] = w * gA[0]; p[1] = w * gA[1]; p[2] = w * gA[2];
+    p[3] = (ux - dot * sx) * inv; p[4] = (uy - dot * sy) * inv; p[5] = (uz - dot * sz) * inv;
+    p[6] = -rho * g_logit * tau;
+  }
+  gd[0] = gx; gd[1] = gy; gd[2] = gz;
+}
+
+// ---- the two explicit models behind one pair of calls -----------------------------------------
+struct SvCarry { float A[3], mx, z; };   // what the SV backward needs from its first pass
+template <int APP>
+__device__ __forceinline__ void explicit_pre(const float *row, const float base[3], float dx, float dy, float dz, int deg,
+                                             float pre[3], SvCarry &cy) {
+  if (APP == GS_APP_SV) {
+    cy.A[0] = cy.A[1] = cy.A[2] = 0.f; cy.mx = 0.f; cy.z = 1.f;
+    if (deg > 0) sv_decode(row, dx, dy, dz, cy.A, cy.mx, cy.z);
+    pre[0] = base[0] + 0.5f + cy.A[0]; pre[1] = base[1] + 0.5f + cy.A[1]; pre[2] = base[2] + 0.5f + cy.A[2];
+  } else {
+    sh_decode(row, base, dx, dy, dz, deg, pre);
+  }
+}
+template <int APP>
+__device__ __forceinline__ void explicit_bwd(float *row, const float gp[3], float dx, float dy, float dz, int deg,
+                                             const SvCarry &cy, float gd[3]) {
+  if (APP == GS_APP_SV) {
+    if (deg > 0) {
+      sv_backward(row, gp, cy.A, cy.mx, cy.z, dx, dy, dz, gd);
+    } else {
+#pragma unroll
+      for (int k = 0; k < GS_SV_ROW; ++k) row[k] = 0.f;
+      gd[0] = gd[1] = gd[2] = 0.f;
+    }
+  } else {
+    sh_backward(row, gp, dx, dy, dz, deg, gd);
+  }
 }
 
 // ---- appearance: neural ---------------------------------------------------------------------
@@ -303,7 +390,7 @@ __device__ __forceinline__ void load3(const float *p, int64_t i, float v[3]) {
 
 template <int APP>
 __global__ void __launch_bounds__(kBlock) k_preprocess_fwd(PreprocessArgs a, CamDev cam) {
-  __shared__ __align__(16) float sData[APP == GS_APP_SH ? kWarps * kSlab : 4];
+  __shared__ __align__(16) float sData[APP != GS_APP_NEURAL ? kWarps * SlabOf<APP>::value : 4];
   __shared__ __align__(16) unsigned char sNN[APP == GS_APP_NEURAL ? sizeof(mlp::Weights) + kWarps * sizeof(StageFwd) : 16];
   mlp::Weights *sWt = reinterpret_cast<mlp::Weights *>(sNN);
   StageFwd *sStage = reinterpret_cast<StageFwd *>(sNN + (APP == GS_APP_NEURAL ? sizeof(mlp::Weights) : 0));   // unused for SH
@@ -339,13 +426,14 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_fwd(PreprocessArgs a, Cam
   }
   // ---- fused colour decode for the Gaussians that survived culling
   float pre[3] = {0.f, 0.f, 0.f};
-  if (APP == GS_APP_SH) {
-    float *slab = sData + warp * kSlab;
-    if (__any_sync(kFull, vis) && a.deg > 0 && row0 < a.n) warp_load_rows(a.sh_rest, row0, a.n, slab, lane);
+  if (APP != GS_APP_NEURAL) {   // SH or Spherical Voronoi: parameter rows through the warp's slab
+    float *slab = sData + warp * SlabOf<APP>::value;
+    if (__any_sync(kFull, vis) && a.deg > 0 && row0 < a.n) warp_load_rows<RowOf<APP>::value>(a.sh_rest, row0, a.n, slab, lane);
     if (vis) {
       float base[3];
       load3(a.base_color, i, base);
-      sh_decode(slab + lane * kRow, base, g.dirx, g.diry, g.dirz, a.deg, pre);
+      SvCarry cy;
+      explicit_pre<APP>(slab + lane * RowOf<APP>::value, base, g.dirx, g.diry, g.dirz, a.deg, pre, cy);
     }
   } else {
     float A[3] = {0.f, 0.f, 0.f};
@@ -507,7 +595,8 @@ __device__ __forceinline__ void store3(float *p, int64_t i, float a, float b, fl
 
 // Shared memory of the backward kernels (dynamic): SH: kWarps slabs of coefficient rows.
 // Neural: weights [816] | kWarps operand slabs [32][100] (reused as [kWarps][816] at the end).
-constexpr size_t kBwdSmemSH = sizeof(float) * kWarps * kSlab;
+constexpr size_t kBwdSmemSH = sizeof(float) * kWarps * SlabOf<GS_APP_SH>::value;
+constexpr size_t kBwdSmemSV = sizeof(float) * kWarps * SlabOf<GS_APP_SV>::value;
 constexpr size_t kBwdSmemNN = sizeof(mlp::Weights) + kWarps * sizeof(mlp::WarpStage);
 static_assert(kWarps * sizeof(mlp::WarpStage) >= kWarps * GS_MLP_WEIGHTS * sizeof(float), "partial sums reuse the staging areas");
 static_assert(sizeof(mlp::Weights) % 16 == 0, "staging areas must stay 16-byte aligned");
@@ -516,7 +605,7 @@ template <int APP>
 __global__ void __launch_bounds__(kBlock) k_preprocess_bwd(PreprocessBwdArgs a, CamDev cam) {
   extern __shared__ __align__(16) float smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  float *slab = smem + warp * kSlab;   // SH: this warp's slab of coefficient rows
+  float *slab = smem + warp * SlabOf<APP>::value;   // SH / SV: this warp's slab of parameter rows
   mlp::Weights &sWt = *reinterpret_cast<mlp::Weights *>(smem);
   mlp::WarpStage *sStage = reinterpret_cast<mlp::WarpStage *>(reinterpret_cast<unsigned char *>(smem) + sizeof(mlp::Weights));
   mlp::WeightGrad dW;
@@ -555,25 +644,26 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_bwd(PreprocessBwdArgs a, 
     }
     // ---- appearance backward
     float gp[3] = {0.f, 0.f, 0.f};
-    if (APP == GS_APP_SH) {
+    if (APP != GS_APP_NEURAL) {
       if (row0 < a.n) {
         if (warp_vis && a.deg > 0) {
-          warp_load_rows(a.sh_rest, row0, a.n, slab, lane);
+          warp_load_rows<RowOf<APP>::value>(a.sh_rest, row0, a.n, slab, lane);
         }
-        float *row = slab + lane * kRow;
+        float *row = slab + lane * RowOf<APP>::value;
         if (vis) {
           float base[3], pre[3];
           load3(a.base_color, i, base);
-          if (a.deg > 0) sh_decode(row, base, dx, dy, dz, a.deg, pre);
+          SvCarry cy;
+          if (a.deg > 0) explicit_pre<APP>(row, base, dx, dy, dz, a.deg, pre, cy);
           else { pre[0] = base[0] + 0.5f; pre[1] = base[1] + 0.5f; pre[2] = base[2] + 0.5f; }
           gp[0] = color_act_grad_z(a.act, pre[0]) * ga.x; gp[1] = color_act_grad_z(a.act, pre[1]) * ga.y;
           gp[2] = color_act_grad_z(a.act, pre[2]) * ga.z;
-          sh_backward(row, gp, dx, dy, dz, a.deg, gd);
+          explicit_bwd<APP>(row, gp, dx, dy, dz, a.deg, cy, gd);
         } else {
 #pragma unroll
-          for (int k = 0; k < kRow; ++k) row[k] = 0.f;
+          for (int k = 0; k < RowOf<APP>::value; ++k) row[k] = 0.f;
         }
-        warp_store_rows(a.g_sh_rest, row0, a.n, slab, lane);
+        warp_store_rows<RowOf<APP>::value>(a.g_sh_rest, row0, a.n, slab, lane);
       }
     } else {
       float gf[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
@@ -628,7 +718,7 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_bwd(PreprocessBwdArgs a, 
 // ---- separate-pass appearance kernels ---------------------------------------------------------
 template <int APP>
 __global__ void __launch_bounds__(kBlock) k_appearance_fwd(AppearanceArgs a) {
-  __shared__ __align__(16) float sData[APP == GS_APP_SH ? kWarps * kSlab : 4];
+  __shared__ __align__(16) float sData[APP != GS_APP_NEURAL ? kWarps * SlabOf<APP>::value : 4];
   __shared__ __align__(16) unsigned char sNN[APP == GS_APP_NEURAL ? sizeof(mlp::Weights) + kWarps * sizeof(StageFwd) : 16];
   mlp::Weights *sWt = reinterpret_cast<mlp::Weights *>(sNN);
   StageFwd *sStage = reinterpret_cast<StageFwd *>(sNN + (APP == GS_APP_NEURAL ? sizeof(mlp::Weights) : 0));   // unused for SH
@@ -642,10 +732,11 @@ __global__ void __launch_bounds__(kBlock) k_appearance_fwd(AppearanceArgs a) {
   const bool in = i < a.n;
   float d[3] = {0.f, 0.f, 1.f}, base[3] = {0.f, 0.f, 0.f}, pre[3];
   if (in) { load3(a.dirs, i, d); load3(a.base_color, i, base); }
-  if (APP == GS_APP_SH) {
-    float *slab = sData + warp * kSlab;
-    if (a.deg > 0 && row0 < a.n) warp_load_rows(a.sh_rest, row0, a.n, slab, lane);
-    if (in) sh_decode(slab + lane * kRow, base, d[0], d[1], d[2], a.deg, pre);
+  if (APP != GS_APP_NEURAL) {
+    float *slab = sData + warp * SlabOf<APP>::value;
+    if (a.deg > 0 && row0 < a.n) warp_load_rows<RowOf<APP>::value>(a.sh_rest, row0, a.n, slab, lane);
+    SvCarry cy;
+    if (in) explicit_pre<APP>(slab + lane * RowOf<APP>::value, base, d[0], d[1], d[2], a.deg, pre, cy);
   } else {
     float A[3] = {0.f, 0.f, 0.f};
     if (a.deg > 0 && row0 < a.n) {
@@ -671,7 +762,7 @@ template <int APP>
 __global__ void __launch_bounds__(kBlock) k_appearance_bwd(AppearanceArgs a) {
   extern __shared__ __align__(16) float smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  float *slab = smem + warp * kSlab;   // SH: this warp's slab of coefficient rows
+  float *slab = smem + warp * SlabOf<APP>::value;   // SH / SV: this warp's slab of parameter rows
   mlp::Weights &sWt = *reinterpret_cast<mlp::Weights *>(smem);
   mlp::WarpStage *sStage = reinterpret_cast<mlp::WarpStage *>(reinterpret_cast<unsigned char *>(smem) + sizeof(mlp::Weights));
   mlp::WeightGrad dW;
@@ -689,19 +780,20 @@ __global__ void __launch_bounds__(kBlock) k_appearance_bwd(AppearanceArgs a) {
     float d[3] = {0.f, 0.f, 1.f}, base[3] = {0.f, 0.f, 0.f}, gcol[3] = {0.f, 0.f, 0.f};
     if (in) { load3(a.dirs, i, d); load3(a.base_color, i, base); load3(a.g_color, i, gcol); }
     float gp[3] = {0.f, 0.f, 0.f}, gd[3] = {0.f, 0.f, 0.f};
-    if (APP == GS_APP_SH) {
+    if (APP != GS_APP_NEURAL) {
       if (row0 < a.n) {
-        if (a.deg > 0) warp_load_rows(a.sh_rest, row0, a.n, slab, lane);
-        float *row = slab + lane * kRow;
+        if (a.deg > 0) warp_load_rows<RowOf<APP>::value>(a.sh_rest, row0, a.n, slab, lane);
+        float *row = slab + lane * RowOf<APP>::value;
         if (in) {
           float pre[3];
-          if (a.deg > 0) sh_decode(row, base, d[0], d[1], d[2], a.deg, pre);
+          SvCarry cy;
+          if (a.deg > 0) explicit_pre<APP>(row, base, d[0], d[1], d[2], a.deg, pre, cy);
           else { pre[0] = base[0] + 0.5f; pre[1] = base[1] + 0.5f; pre[2] = base[2] + 0.5f; }
 #pragma unroll
           for (int c = 0; c < 3; ++c) gp[c] = color_act_grad_z(a.act, pre[c]) * gcol[c];
-          sh_backward(row, gp, d[0], d[1], d[2], a.deg, gd);
+          explicit_bwd<APP>(row, gp, d[0], d[1], d[2], a.deg, cy, gd);
         }
-        warp_store_rows(a.g_sh_rest, row0, a.n, slab, lane);
+        warp_store_rows<RowOf<APP>::value>(a.g_sh_rest, row0, a.n, slab, lane);
       }
     } else {
       float gf[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
@@ -748,6 +840,7 @@ void opt_in_smem(K kernel, size_t bytes) {
 int launch_preprocess_fwd(int app, const PreprocessArgs &a, const CamDev &cam, cudaStream_t st) {
   if (a.n == 0) return 0;
   if (app == GS_APP_SH) k_preprocess_fwd<GS_APP_SH><<<grid_for(a.n), kBlock, 0, st>>>(a, cam);
+  else if (app == GS_APP_SV) k_preprocess_fwd<GS_APP_SV><<<grid_for(a.n), kBlock, 0, st>>>(a, cam);
   else k_preprocess_fwd<GS_APP_NEURAL><<<grid_for(a.n), kBlock, 0, st>>>(a, cam);
   return 1;
 }
@@ -757,6 +850,11 @@ int launch_preprocess_bwd(int app, const PreprocessBwdArgs &a, const CamDev &cam
     if (a.n == 0) return 0;
     opt_in_smem(k_preprocess_bwd<GS_APP_SH>, kBwdSmemSH);
     k_preprocess_bwd<GS_APP_SH><<<grid_for(a.n), kBlock, kBwdSmemSH, st>>>(a, cam);
+    return 1;
+  } else if (app == GS_APP_SV) {
+    if (a.n == 0) return 0;
+    opt_in_smem(k_preprocess_bwd<GS_APP_SV>, kBwdSmemSV);
+    k_preprocess_bwd<GS_APP_SV><<<grid_for(a.n), kBlock, kBwdSmemSV, st>>>(a, cam);
     return 1;
   } else {
     opt_in_smem(k_preprocess_bwd<GS_APP_NEURAL>, kBwdSmemNN);
@@ -769,6 +867,7 @@ int launch_preprocess_bwd(int app, const PreprocessBwdArgs &a, const CamDev &cam
 int launch_appearance_fwd(int app, const AppearanceArgs &a, cudaStream_t st) {
   if (a.n == 0) return 0;
   if (app == GS_APP_SH) k_appearance_fwd<GS_APP_SH><<<grid_for(a.n), kBlock, 0, st>>>(a);
+  else if (app == GS_APP_SV) k_appearance_fwd<GS_APP_SV><<<grid_for(a.n), kBlock, 0, st>>>(a);
   else k_appearance_fwd<GS_APP_NEURAL><<<grid_for(a.n), kBlock, 0, st>>>(a);
   return 1;
 }
@@ -778,6 +877,11 @@ int launch_appearance_bwd(int app, const AppearanceArgs &a, cudaStream_t st) {
     if (a.n == 0) return 0;
     opt_in_smem(k_appearance_bwd<GS_APP_SH>, kBwdSmemSH);
     k_appearance_bwd<GS_APP_SH><<<grid_for(a.n), kBlock, kBwdSmemSH, st>>>(a);
+    return 1;
+  } else if (app == GS_APP_SV) {
+    if (a.n == 0) return 0;
+    opt_in_smem(k_appearance_bwd<GS_APP_SV>, kBwdSmemSV);
+    k_appearance_bwd<GS_APP_SV><<<grid_for(a.n), kBlock, kBwdSmemSV, st>>>(a);
     return 1;
   } else {
     opt_in_smem(k_appearance_bwd<GS_APP_NEURAL>, kBwdSmemNN);

@@ -77,6 +77,7 @@ def run_gpu(scene, cam, G=None, pair_capacity=None, with_extent=True, device=0):
                                     opacity_logits=cp(g.opacity_logits)[:n], base_color=cp(g.base_color)[:n],
                                     sh_rest=cp(g.sh_rest)[:n] if g.sh_rest is not None else None,
                                     features=cp(g.features)[:n] if g.features is not None else None,
+                                    sv_sites=cp(g.sv_sites)[:n] if g.sv_sites is not None else None,
                                     mlp_weights=cp(g.mlp_weights))
         # the backward leaves the per-Gaussian 2D gradients at the start of the workspace, [n,12]
         out.g2d = ws[: n * 48].view(torch.float32).reshape(n, 12).cpu().numpy() if n else np.zeros((0, 12), np.float32)
@@ -86,4 +87,4 @@ def run_gpu(scene, cam, G=None, pair_capacity=None, with_extent=True, device=0):
 
 def grad_names(app):
     base = ["means", "log_scales", "quats", "opacity_logits", "base_color"]
-    return base + (["sh_rest"] if app == 0 else ["features", "mlp_weights"])
+    return base + (["sh_rest"] if app == 0 else ["sv_sites"] if app == 2 else ["features", "mlp_weights"])

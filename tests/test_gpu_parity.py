@@ -173,7 +173,8 @@ def test_parameter_gradients(results, oracle, name):
     gp = oracle.preprocess_backward(sc.means, sc.log_scales, sc.quats, sc.opacity_logits, cam, vis,
                                     g2[:, 7:9], g2[:, 4:7], g2[:, 3], ga.dirs)
     ref = dict(means=gp.means, log_scales=gp.log_scales, quats=gp.quats, opacity_logits=gp.opacity_logits,
-               base_color=ga.base_color, sh_rest=ga.sh_rest, features=ga.features, mlp_weights=ga.mlp_weights)
+               base_color=ga.base_color, sh_rest=ga.sh_rest, features=ga.features, mlp_weights=ga.mlp_weights,
+               sv_sites=ga.sv_sites)
     same_vis = gpu.visible == pre.visible.astype(bool)
     for nm in grad_names(sc.app):
         got = getattr(gpu.grads, nm)
