@@ -104,10 +104,10 @@ def workload_of(args, scenes):
     if c == 3:
         n, views = args.n or N_GAUSS, args.views or VIEWS
         return dict(name=f"config3: {n} Gaussians (64 clusters + shell), {WIDTH}x{HEIGHT}, {views} orbit views, "
-                         "neural appearance (8 fp16 features + shared 32-16-16-3 MLP) with SH degree 3 beside it, fwd+bwd",
+                         "neural appearance (8 fp16 features + shared 32-16-16-3 MLP), with SH degree 3 and Spherical Voronoi beside it, fwd+bwd",
                     n=n, views=views, width=WIDTH, height=HEIGHT, cams=scenes.orbit_cameras(WIDTH, HEIGHT, views),
                     scene=lambda app: scenes.config3(app, n=n, width=WIDTH, height=HEIGHT, views=views).scene,
-                    arms=[(scenes.APP_NEURAL, "neural"), (scenes.APP_SH, "sh")])
+                    arms=[(scenes.APP_NEURAL, "neural"), (scenes.APP_SH, "sh"), (scenes.APP_SV, "sv")])
     if c == 1:
         w = scenes.config1()
         return dict(name="config1: 1000 Gaussians in a box, 64x64, identity camera, SH degree 3, fwd+bwd",
@@ -212,7 +212,7 @@ def run_ours(args):
     results = {}
     sampler = ClockSampler(local)
     clocks = None
-    arms = [a for a in wl["arms"] if not (args.skip_sh and a[1] == "sh" and a[1] != head)]
+    arms = [a for a in wl["arms"] if not (args.skip_sh and a[1] != head)]
     for app, tag in arms:
         host, ds, r, pairs = make_arm(app)
         if tag == head:
@@ -290,8 +290,11 @@ def run_ours(args):
         "stage_share": {k: round(v / total_stage, 4) for k, v in stage_ms.items() if v > 0},
         "pairs_per_view": neural["pairs"], "visible_per_view": neural["visible"] / views,
         "sh": None if "sh" not in results or head == "sh" else {
-            "ms_per_step": results["sh"]["ms"],
+            "ms_per_step": results["sh"]["ms"], "ms_per_step_single_stream": results["sh"]["ms_one"],
             "stages_ms_per_step": {k: round(v, 4) for k, v in results["sh"]["stage_ms"].items() if v > 0}},
+        "sv": None if "sv" not in results or head == "sv" else {
+            "ms_per_step": results["sv"]["ms"], "ms_per_step_single_stream": results["sv"]["ms_one"],
+            "stages_ms_per_step": {k: round(v, 4) for k, v in results["sv"]["stage_ms"].items() if v > 0}},
         "appearance_decode": decode,
         "adam_update": adam,
         "viewer_prepass": prepass,
@@ -493,8 +496,10 @@ def adam_sweep(api, torch, ctx, dev, peaks, n):
     larger than L2 (16 B of state per element), so the stream is measured from HBM."""
     y0 = 0.28209479177387814
     geo = [("means", 3, 1.6e-4), ("log_scales", 3, 5e-3), ("quats", 4, 1e-3), ("opacity_logits", 1, 5e-2)]
+    sv_rates = ([0.0008] * 3 + [0.002] * 3 + [0.006]) * 7      # per site: colour, site direction, temperature (App. B)
     sets = {"sh": geo + [("base_color", 3, 0.0025 * y0), ("sh_rest", 45, 0.000125)],
-            "neural": geo + [("base_color", 3, 0.00025), ("features", 8, 0.008), ("mlp_weights", 1, 0.003)]}
+            "neural": geo + [("base_color", 3, 0.00025), ("features", 8, 0.008), ("mlp_weights", 1, 0.003)],
+            "sv": geo + [("base_color", 3, 0.0008), ("sv_sites", 49, sv_rates)]}
     out = {}
     for tag, spec in sets.items():
         gen = torch.Generator(device=dev); gen.manual_seed(77)
@@ -505,8 +510,8 @@ def adam_sweep(api, torch, ctx, dev, peaks, n):
             g = torch.randn((rows, cols), device=dev, generator=gen) * 1e-3
             m, v = torch.zeros_like(p), torch.zeros_like(p)
             half = torch.empty((rows, cols), device=dev, dtype=torch.float16) if name in ("features", "mlp_weights") else None
-            tensors.append(api.AdamTensor(p, g, m, v, [lr] * cols, 0.9, 0.99 if name == "mlp_weights" else 0.999, 1e-15,
-                                          half_copy=half))
+            tensors.append(api.AdamTensor(p, g, m, v, lr if isinstance(lr, list) else [lr] * cols, 0.9,
+                                          0.99 if name == "mlp_weights" else 0.999, 1e-15, half_copy=half))
             nbytes += rows * cols * (28 + (2 if half is not None else 0))
         for it in range(3):
             api.gs_adam_step(ctx, tensors, it + 1)
@@ -566,7 +571,7 @@ def prepass_sweep(api, torch, ctx, dev, peaks, args, scenes):
 
 
 def decode_sweep(api, torch, ctx, dev, peaks, args):
-    """Separate-pass colour decode forward + backward at 1M / 3M / 10M Gaussians, SH vs neural."""
+    """Separate-pass colour decode forward + backward at 1M / 3M / 10M Gaussians: SH, neural, Spherical Voronoi."""
     out = {}
     sizes = [1_000_000, 3_000_000, 10_000_000] if not args.quick else [1_000_000]
     for n in sizes:
@@ -576,8 +581,13 @@ def decode_sweep(api, torch, ctx, dev, peaks, args):
         gcol = torch.randn((n, 3), device=dev, generator=gen)
         base = 0.14 + 0.03 * torch.randn((n, 3), device=dev, generator=gen)
         z = torch.zeros((1, 4), device=dev)
-        for app, tag in ((0, "sh"), (1, "neural")):
-            if app == 0:
+        for app, tag in ((0, "sh"), (1, "neural"), (2, "sv")):
+            if app == 2:     # Spherical Voronoi: 7 sites x 7 raw parameters = 196 B per primitive
+                sites = torch.randn((n, 7, 7), device=dev, generator=gen)
+                sites[:, :, 0:3] *= 0.15
+                sc = api.DeviceScene(z, z, z, z[0], base, 2, 3, sv_sites=sites.contiguous())
+                bytes_fwd, bytes_bwd = 196 + 12 + 12, 12 + 196 + 12 + 196 + 12 + 12
+            elif app == 0:
                 sc = api.DeviceScene(z, z, z, z[0], base, 0, 3, sh_rest=0.05 * torch.randn((n, 15, 3), device=dev, generator=gen))
                 bytes_fwd, bytes_bwd = 192 + 12 + 12, 12 + 192 + 12 + 192 + 12 + 12
             else:

@@ -258,7 +258,7 @@ def config3(app: int, n: int = 1_000_000, width: int = 1256, height: int = 828,
             views: int = 8) -> Workload:
     """1M Gaussians in 64 clusters + shell, 8 orbit cameras."""
     scene = clustered_scene(n, 64, -4.0, 0.7, app, seed=1003)
-    tag = "sh" if app == APP_SH else "neural"
+    tag = {APP_SH: "sh", APP_SV: "sv"}.get(app, "neural")
     return Workload(f"config3_1M_{tag}", scene, orbit_cameras(width, height, views))
 
 
