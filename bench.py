@@ -224,6 +224,29 @@ def run_ours(args):
             ms = timed(lambda: step_two_streams(ds, rs), args.steps, args.warmup)
             for c, s_ in zip(lane_ctx, lanes):
                 api.gs_async_status(c, s_)              # raises if a view had outgrown its pair capacity
+            ms_streams, graph_note = ms, None
+            if not args.no_graph:
+                # The same iteration captured once as a CUDA graph (nothing in it waits for the host) and replayed:
+                # the kernels, their order and their arguments are unchanged, only the launching is.
+                try:
+                    cap = torch.cuda.Stream(dev)
+                    cap.wait_stream(torch.cuda.current_stream(dev))
+                    graph = torch.cuda.CUDAGraph()
+                    with torch.cuda.stream(cap):
+                        step_two_streams(ds, rs)            # once more outside the capture, on the capture stream
+                        torch.cuda.synchronize()
+                        with torch.cuda.graph(graph, stream=cap):
+                            step_two_streams(ds, rs)
+                    torch.cuda.current_stream(dev).wait_stream(cap)
+                    ms_graph = timed(graph.replay, args.steps, args.warmup)
+                    for c, s_ in zip(lane_ctx, lanes):
+                        api.gs_async_status(c, s_)
+                    graph_note = {"ms_per_step": ms_graph, "captured": True}
+                    ms = min(ms, ms_graph)
+                    del graph
+                except Exception as e:                      # capture is an optimisation of the launching only
+                    graph_note = {"captured": False, "why": str(e)[:200]}
+                    torch.cuda.synchronize()
             del rs
         stage_ms, stage_launches = profile(lambda: step(ds, r), max(1, min(args.steps, 3)))
         if tag == head:
@@ -245,7 +268,8 @@ def run_ours(args):
             evaluated += ev; composited += co
             rect = r.proj.rect.to(torch.int32) & 0xFFFF
             visible += int(((rect[:, 2] > rect[:, 0]) & (rect[:, 3] > rect[:, 1])).sum().item())
-        results[tag] = dict(ms=ms, ms_one=ms_one, stage_ms=stage_ms, stage_launches=stage_launches, pairs=pairs,
+        results[tag] = dict(ms=ms, ms_one=ms_one, ms_streams=locals().get("ms_streams", ms), graph=locals().get("graph_note"),
+                            stage_ms=stage_ms, stage_launches=stage_launches, pairs=pairs,
                             entries=entries, visible=visible, evaluated=evaluated, composited=composited,
                             host=host, ds=ds, r=r, app=tag)
 
@@ -279,7 +303,8 @@ def run_ours(args):
                    "cache": "inputs_larger_than_L2 (per-view working set > 126 MB; 8 different cameras)",
                    "multi_gpu": "replicas only"},
         "gprimitives_per_s": world * n * views / (ms * 1e-3) / 1e9,
-        "ms_per_step_single_stream": neural["ms_one"],
+        "ms_per_step_single_stream": neural["ms_one"], "ms_per_step_streams_no_graph": neural["ms_streams"],
+        "cuda_graph": neural["graph"],
         "streams": 1 if views == 1 else n_lanes,
         "clocks": clocks, "e2e": e2e, "e2e_gradients_to_host": e2e_host, "gpu_launches": launches_per_step,
         "roofline": roof,
@@ -693,6 +718,7 @@ def main():
     ap.add_argument("--skip-sh", action="store_true", help="time the neural arm only (profiling runs)")
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--single-stream", action="store_true", help="time the views one after another on one stream only")
+    ap.add_argument("--no-graph", action="store_true", help="do not try the CUDA-graph replay of the multi-stream iteration")
     ap.add_argument("--streams", type=int, default=4, help="views in flight (each on its own stream, context and buffers)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
