@@ -156,9 +156,9 @@ const char *gs_last_error(const GsContext *ctx);
 size_t gs_workspace_bytes(int64_t n, int32_t width, int32_t height, int64_t pair_capacity);
 
 /* Preprocess (Sec. 3.1; fused appearance: Sec. 4 "CUDA Implementation").  For every Gaussian:
- * cull, project (EWA), bound the alpha >= 1/255 footprint by a tile rectangle, and decode the
- * view-dependent colour for the direction camera centre -> mean (SH: Eq. 1-2; neural:
- * Eq. 5-7).  Writes all of `out` and the total instance count to *num_pairs_host (host
+ * cull, project (EWA), bound the alpha >= 1/255 ellipse by a tile rectangle and count the tiles
+ * inside it that the ellipse reaches, and decode the view-dependent colour for the direction
+ * camera centre -> mean (SH: Eq. 1-2; neural: Eq. 5-7; Spherical Voronoi: Eq. 3).  Writes all of `out` and the total instance count to *num_pairs_host (host
  * pointer; the call synchronises the stream once to read it).  n = 0 is valid. */
 GsStatus gs_preprocess(GsContext *ctx, const GsScene *scene, const GsCamera *cam, GsProjected *out,
                        int64_t *num_pairs_host, void *stream);
@@ -195,8 +195,9 @@ GsStatus gs_render_forward(GsContext *ctx, int64_t n, const GsProjected *proj, c
 
 /* Backward of the blend and of the preprocess, appearance included (Sec. 4 "CUDA
  * Implementation": the directional colour gradient also reaches the means).  `final_T` and
- * `n_contrib` are the forward's outputs for the same view, dL_dimage is [3,H,W].  Fills every member of `grads` that applies to scene->app.  Uses the same workspace
- * (contents of the forward call are not needed). */
+ * `n_contrib` are the forward's outputs for the same view, dL_dimage is [3,H,W].  Fills every
+ * member of `grads` that applies to scene->app.  Uses the same workspace (contents of the forward
+ * call are not needed). */
 GsStatus gs_render_backward(GsContext *ctx, const GsScene *scene, const GsCamera *cam,
                             const GsProjected *proj, const GsBinning *bin, int64_t num_pairs,
                             const float *final_T, const uint32_t *n_contrib, const float *dL_dimage,
@@ -205,7 +206,7 @@ GsStatus gs_render_backward(GsContext *ctx, const GsScene *scene, const GsCamera
 /* The separate-pass appearance path (Sec. 4 "CUDA Implementation", reference path; App. B.2):
  * colour decode for given unit directions dirs [n,3] without the rasterizer, and its backward.
  * Only the appearance members of `scene` are read.  color [n,3].  gs_appearance_backward fills
- * grads->base_color, grads->sh_rest or grads->features + grads->mlp_weights, and dL_ddirs
+ * grads->base_color, grads->sh_rest or grads->features + grads->mlp_weights or grads->sv_sites, and dL_ddirs
  * [n,3] (gradient with respect to the direction as a free vector). */
 GsStatus gs_appearance_forward(GsContext *ctx, const GsScene *scene, const float *dirs, float *color,
                                void *stream);
