@@ -336,10 +336,19 @@ NCU_TRAFFIC_1M_NEURAL = {"blend_bwd": 47.37e6, "blend_fwd": 25.73e6, "preprocess
                          "preprocess_fwd": 89.63e6}
 
 
+# smsp__issue_active.avg.pct_of_peak_sustained_active of the same captures: the share of issue slots the kernel
+# fills while it runs.  For the ALU-bound blend kernels this, not the flop rate, says how close to the machine they
+# are: the flop count above is the method's minimum arithmetic, the issue slots also carry loads, predicates,
+# shuffles and loop control.
+NCU_ISSUE_ACTIVE_1M_NEURAL = {"blend_bwd": 0.81, "blend_fwd": 0.70, "preprocess_bwd": 0.38, "preprocess_fwd": 0.72,
+                              "keygen": 0.46}
+
+
 def stage_roofline(stage, arm, views, n, peaks, alu_peak):
     out = _stage_roofline(stage, arm, views, n, peaks, alu_peak)
     if n == 1_000_000 and arm.get("app") == "neural":
         out["traffic"] = NCU_TRAFFIC_1M_NEURAL.get(stage)
+        out["issue_active_frac_ncu"] = NCU_ISSUE_ACTIVE_1M_NEURAL.get(stage)
     return out
 
 
