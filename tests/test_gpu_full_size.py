@@ -17,6 +17,7 @@ CASES = {
     "config2_neural_100k": lambda: (scenes.config2(), 0),
     "config3_neural_1M": lambda: (scenes.config3(scenes.APP_NEURAL), 2),
     "config3_sh_1M": lambda: (scenes.config3(scenes.APP_SH), 5),
+    "config3_sv_1M": lambda: (scenes.config3(scenes.APP_SV), 1),
     "config4_neural_3M": lambda: (scenes.config4(), 7),
 }
 
