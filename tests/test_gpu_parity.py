@@ -352,3 +352,32 @@ def test_single_large_gaussian_covers_every_tile(oracle):
     assert gpu.tiles_touched[0] == 13 * 8
     assert np.array_equal(gpu.sorted_vals, fwd.vals) and np.array_equal(gpu.tile_ranges, fwd.ranges)
     assert image_mismatch(gpu.image, fwd.image, fwd.fragile).sum() == 0
+
+
+def test_large_image_many_tiles(oracle):
+    """A 4K-wide image: 240 x 135 = 32 400 tiles, so the tile id takes 15 bits (two 8-bit digits) and a
+    single Gaussian can cover thousands of tiles; few Gaussians, so the oracle stays quick."""
+    w = scenes.config1(3000)
+    sc = w.scene
+    sc.log_scales += np.float32(0.8)                        # footprints of tens to hundreds of pixels
+    sc.means[0] = [0.0, 0.0, 2.5]; sc.log_scales[0] = [0.6, 0.2, -1.0]; sc.opacity_logits[0] = 1.0   # one huge one
+    cam = scenes.identity_camera(3840, 2160, 1900.0)
+    G = scenes.upstream_gradient(cam, 8)
+    gpu = run_gpu(sc, cam, G)
+    fwd, grads = oracle.render(sc, cam, G)
+    assert gpu.tiles_touched.max() > 4000 and gpu.P > 100_000
+    valid = gpu.extent[:, 0] >= 0
+    rect, tt, P = oracle.tile_spans_f32(valid, gpu.mean2d, gpu.chol, gpu.extent, cam.width, cam.height)
+    assert P == gpu.P and np.array_equal(rect, gpu.rect) and np.array_equal(tt, gpu.tiles_touched)
+    keys, vals, ranges = oracle.sorted_instances_f32(rect, tt, gpu.mean2d, gpu.chol, gpu.extent,
+                                                     np.where(gpu.visible, gpu.depth_key, 0), cam.width, cam.height, P)
+    assert np.array_equal(gpu.sorted_vals, vals) and np.array_equal(gpu.tile_ranges, ranges)
+    assert np.array_equal(gpu.sorted_tiles, (keys >> np.uint64(32)).astype(np.uint32))
+    assert image_mismatch(gpu.image, fwd.image, fwd.fragile).sum() == 0
+    # footprints of 1e4-1e6 pixels sum upstream gradients of both signs: what an fp32 sum keeps of such a result
+    # is bounded by the size of its terms, not of the result (test_blend_backward_2d_gradients states that bound);
+    # here: nearly all elements by the literal rule, none off by more than 1e-2 of the largest of its kind
+    for nm in grad_names(sc.app):
+        got, want = getattr(gpu.grads, nm), getattr(grads, nm)
+        assert grad_mismatch(got, want).mean() <= 5e-2, nm
+        assert np.abs(got - want).max() <= 1e-2 * np.abs(want).max(), nm
