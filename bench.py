@@ -26,8 +26,8 @@ sys.path.insert(0, ROOT)
 METRIC = "fwd+bwd rasterizer ms/iter @1M Gaussians; appearance-decode GB/s vs HBM peak"
 N_GAUSS, WIDTH, HEIGHT, VIEWS = 1_000_000, 1256, 828, 8
 
-# Algorithmic cost per unit: flops per evaluated list entry of the blend
-# kernels and bytes per Gaussian of the per-Gaussian kernels.
+# Algorithmic cost per unit: flops per evaluated list entry of the blend kernels and bytes per Gaussian of
+# the per-Gaussian kernels.
 # Blend kernels (fp32 ALU bound): flops per list entry evaluated for a pixel (the alpha test) and per
 # pair composited, counted from the kernels' arithmetic.
 BLEND_FLOPS_PER_EVALUATED = 8.0       # 3.5 (quad falloff, shared by 4 pixels) + ex2 + mul + min + compare
@@ -331,7 +331,7 @@ def run_ours(args):
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum of ONE launch (orbit view 0 of the default workload), from the
-# ncu --set full captures summarised under profiles/ (k_<kernel>_config3_neural_1M_view0.md).  Bytes.
+# ncu --set full captures summarised under profiles/.  Bytes.
 NCU_TRAFFIC_1M_NEURAL = {"blend_bwd": 47.37e6, "blend_fwd": 25.73e6, "preprocess_bwd": 181.99e6,
                          "preprocess_fwd": 89.63e6}
 
