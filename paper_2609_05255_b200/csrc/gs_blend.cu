@@ -2,7 +2,7 @@
 // thread owns a 2x2 pixel quad (a warp covers 16x8 pixels), so one shared-memory read of a
 // Gaussian serves four pixels and, in the backward, four pixels are summed in registers before
 // anything crosses lanes.  The tile's depth-ordered instance list is staged through shared memory
-// in batches of 128 Gaussians.
+// in batches of 128 Gaussians (64 in the backward, which also keeps the batch's gradient sums there).
 #include "gs_device.cuh"
 
 namespace gs {

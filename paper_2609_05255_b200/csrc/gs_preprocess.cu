@@ -1,7 +1,8 @@
 // Per-Gaussian kernels: projection with fused appearance decode (forward and backward) and the
-// separate-pass appearance kernels.  One thread per Gaussian; SH coefficient rows and their
-// gradients move through per-warp shared-memory slabs so that global accesses stay coalesced;
-// decoder weights live in shared memory as fp32.
+// separate-pass appearance kernels.  One thread per Gaussian; the parameter rows of the explicit models
+// (SH coefficients, Spherical Voronoi sites) and their gradients move through per-warp shared-memory
+// slabs so that global accesses stay coalesced; the neural decoder runs on warp-level tensor-core tiles
+// with its weights in shared memory.
 #include <float.h>
 #include <stdio.h>
 #include <string.h>

@@ -1,4 +1,4 @@
-// Ordering and binning: a stable LSD radix sort (8-bit digits, keys staged and ranked in shared
+// Ordering and binning: a stable LSD radix sort (digits of up to 8 bits, keys staged and ranked in shared
 // memory, no inter-block waiting), the prefix sum of tiles touched in depth order, instance
 // generation and per-tile ranges.
 //
