@@ -102,6 +102,7 @@ __global__ void __launch_bounds__(kThreads) k_blend_fwd(CamDev cam, const uint32
     }
     __syncthreads();
     const int cnt = (int)min((uint32_t)kBatch, end - base);
+#pragma unroll 2
     for (int j = 0; j < cnt && live; ++j) {
       const float4 a = s_xyab[j];
       const float2 c = s_co[j];
