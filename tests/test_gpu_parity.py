@@ -381,3 +381,21 @@ def test_large_image_many_tiles(oracle):
         got, want = getattr(gpu.grads, nm), getattr(grads, nm)
         assert grad_mismatch(got, want).mean() <= 5e-2, nm
         assert np.abs(got - want).max() <= 1e-2 * np.abs(want).max(), nm
+
+
+@pytest.mark.parametrize("n", [1, 2, 31, 33, 127, 129])
+@pytest.mark.parametrize("app", [scenes.APP_SH, scenes.APP_NEURAL, scenes.APP_SV])
+def test_tiny_gaussian_counts(oracle, n, app):
+    """Fewer Gaussians than a warp, a warp plus one, a block plus one: every ragged-tail path at once."""
+    w = scenes.config2(n=n, app=app)
+    sc = w.scene
+    sc.log_scales += np.float32(1.0)                         # big enough to be seen
+    cam = scenes.identity_camera(96, 64, 96.0)
+    G = scenes.upstream_gradient(cam, n)
+    gpu = run_gpu(sc, cam, G)
+    fwd, grads = oracle.render(sc, cam, G)
+    assert gpu.P == fwd.P and np.array_equal(gpu.sorted_vals, fwd.vals) and np.array_equal(gpu.tile_ranges, fwd.ranges)
+    assert image_mismatch(gpu.image, fwd.image, fwd.fragile).sum() == 0
+    for nm in grad_names(app):
+        got, want = getattr(gpu.grads, nm), getattr(grads, nm)
+        assert np.abs(got - want).max() <= 2e-3 * max(np.abs(want).max(), 1e-6) + GRAD_ATOL, nm
