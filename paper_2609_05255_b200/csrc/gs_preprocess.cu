@@ -271,13 +271,27 @@ __device__ __forceinline__ void weight_grad_flush(const mlp::WeightGrad &dW, flo
 // memory from being hoisted out of the loop into hundreds of live registers.
 __device__ __forceinline__ void reload_fence() { asm volatile("" ::: "memory"); }
 
-// Deterministic final reduction of the per-block partials.
-__global__ void k_wgrad_reduce(const float *__restrict__ partials, int nblocks, float *__restrict__ out) {
-  const int k = blockIdx.x * blockDim.x + threadIdx.x;
-  if (k >= GS_MLP_WEIGHTS) return;
+// Deterministic final reduction of the per-block partials: 32 weights per CTA, the rows shared out over
+// eight groups of threads (each sums every eighth row, in order), the eight sums added in a fixed order.
+constexpr int kReduceGroups = 8;
+__global__ void __launch_bounds__(32 * kReduceGroups) k_wgrad_reduce(const float *__restrict__ partials, int nblocks,
+                                                                    float *__restrict__ out) {
+  __shared__ float s_part[kReduceGroups][32];
+  const int k = blockIdx.x * 32 + threadIdx.x, grp = threadIdx.y;
   float s = 0.f;
-  for (int b = 0; b < nblocks; ++b) s += partials[(size_t)b * GS_MLP_WEIGHTS + k];
-  out[k] = s;
+  if (k < GS_MLP_WEIGHTS)
+    for (int b = grp; b < nblocks; b += kReduceGroups) s += partials[(size_t)b * GS_MLP_WEIGHTS + k];
+  s_part[grp][threadIdx.x] = s;
+  __syncthreads();
+  if (grp == 0 && k < GS_MLP_WEIGHTS) {
+    float t = 0.f;
+#pragma unroll
+    for (int q = 0; q < kReduceGroups; ++q) t += s_part[q][threadIdx.x];
+    out[k] = t;
+  }
+}
+inline void launch_wgrad_reduce(const float *partials, int nblocks, float *out, cudaStream_t st) {
+  k_wgrad_reduce<<<(GS_MLP_WEIGHTS + 31) / 32, dim3(32, kReduceGroups), 0, st>>>(partials, nblocks, out);
 }
 
 // ---- projection -----------------------------------------------------------------------------
@@ -860,7 +874,7 @@ int launch_preprocess_bwd(int app, const PreprocessBwdArgs &a, const CamDev &cam
   } else {
     opt_in_smem(k_preprocess_bwd<GS_APP_NEURAL>, kBwdSmemNN);
     k_preprocess_bwd<GS_APP_NEURAL><<<kWgradBlocks, kBlock, kBwdSmemNN, st>>>(a, cam);
-    k_wgrad_reduce<<<(GS_MLP_WEIGHTS + 127) / 128, 128, 0, st>>>(a.w_partials, kWgradBlocks, a.g_weights);
+    launch_wgrad_reduce(a.w_partials, kWgradBlocks, a.g_weights, st);
     return 2;
   }
 }
@@ -887,7 +901,7 @@ int launch_appearance_bwd(int app, const AppearanceArgs &a, cudaStream_t st) {
   } else {
     opt_in_smem(k_appearance_bwd<GS_APP_NEURAL>, kBwdSmemNN);
     k_appearance_bwd<GS_APP_NEURAL><<<kWgradBlocks, kBlock, kBwdSmemNN, st>>>(a);
-    k_wgrad_reduce<<<(GS_MLP_WEIGHTS + 127) / 128, 128, 0, st>>>(a.w_partials, kWgradBlocks, a.g_weights);
+    launch_wgrad_reduce(a.w_partials, kWgradBlocks, a.g_weights, st);
     return 2;
   }
 }
@@ -968,7 +982,7 @@ extern "C" GsStatus gs_appearance_backward_noalloc(const GsScene *scene, const f
   const int blocks = (int)((chunks + kNoAllocChunksPerBlock - 1) / kNoAllocChunksPerBlock);   // <= 1024
   opt_in_smem(k_appearance_bwd<GS_APP_NEURAL>, kBwdSmemNN);
   k_appearance_bwd<GS_APP_NEURAL><<<blocks, kBlock, kBwdSmemNN, st>>>(a);
-  k_wgrad_reduce<<<(GS_MLP_WEIGHTS + 127) / 128, 128, 0, st>>>(scratch, blocks, a.g_weights);
+  launch_wgrad_reduce(scratch, blocks, a.g_weights, st);
   const cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return fail(GS_ERR_CUDA, cudaGetErrorString(e));
   return GS_OK;
