@@ -509,3 +509,23 @@ def test_integer_stage_f32_agrees_with_double(oracle):
     keys, vals, ranges = oracle.sorted_instances_f32(rect, tt, f32(pre.mean2d), f32(pre.chol), f32(pre.ext),
                                                      pre.depth_bits, cam.width, cam.height, P)
     assert len(vals) == P and np.all(np.diff(keys.astype(np.int64) >> 32) >= 0)
+
+
+def test_oracle_output_has_not_drifted(oracle):
+    """The oracle's summary numbers on small seeded scenes equal the stored ones (written by
+    tests/golden/make_oracle_regression.py from the oracle alone): its arithmetic is changed on purpose or not
+    at all."""
+    import importlib.util
+    here = os.path.dirname(__file__)
+    spec = importlib.util.spec_from_file_location("make_oracle_regression", os.path.join(here, "golden", "make_oracle_regression.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    stored = {}
+    for line in open(os.path.join(here, "golden", "oracle_regression.txt")):
+        if line.strip() and not line.startswith("#"):
+            k, v = line.split("=")
+            stored[k.strip()] = float(v)
+    now = mod.summary()
+    assert set(now) == set(stored)
+    for k, v in now.items():
+        assert abs(v - stored[k]) <= 1e-9 * max(1.0, abs(stored[k])), k
