@@ -399,3 +399,34 @@ def test_tiny_gaussian_counts(oracle, n, app):
     for nm in grad_names(app):
         got, want = getattr(gpu.grads, nm), getattr(grads, nm)
         assert np.abs(got - want).max() <= 2e-3 * max(np.abs(want).max(), 1e-6) + GRAD_ATOL, nm
+
+
+@pytest.mark.parametrize("app", [scenes.APP_SH, scenes.APP_NEURAL, scenes.APP_SV])
+def test_extreme_parameter_values_stay_finite_and_agree(oracle, app):
+    """Needle-thin and sheet-flat Gaussians, scales of e^+-6, opacity logits of +-25, unnormalised quaternions of
+    length 1e-3 and 1e3, a Gaussian at the camera centre, one behind the camera, features of +-20 (far outside
+    the fast sine's range), huge site vectors: visibility must agree with the oracle, nothing may be non-finite,
+    and the image must match."""
+    w = scenes.config2(n=600, app=app)
+    sc = w.scene
+    rng = np.random.default_rng(77)
+    sc.log_scales[:100] = rng.choice([-6.0, 0.5, 2.0], (100, 3)).astype(np.float32)
+    sc.opacity_logits[100:160] = rng.choice([-25.0, 25.0], 60).astype(np.float32)
+    sc.quats[160:200] *= np.float32(1e-3); sc.quats[200:240] *= np.float32(1e3)
+    sc.means[240] = [0.0, 0.0, 0.0]; sc.means[241] = [0.1, 0.1, -3.0]; sc.means[242] = [0.0, 0.0, 0.2]
+    if app == scenes.APP_NEURAL:
+        sc.features[250:300] = rng.choice([-20.0, 20.0, 3.2, -3.2], (50, 8)).astype(np.float16)
+    if app == scenes.APP_SV:
+        sc.sv_sites[250:300, :, 3:6] *= np.float32(1e4); sc.sv_sites[300:330, :, 6] = np.float32(5.0)
+    cam = w.cameras[0]
+    G = scenes.upstream_gradient(cam, 6)
+    gpu = run_gpu(sc, cam, G)
+    fwd, grads = oracle.render(sc, cam, G)
+    differ = gpu.visible != fwd.pre.visible.astype(bool)
+    assert differ.sum() <= 1
+    assert np.all(np.isfinite(gpu.image)) and np.all(np.isfinite(gpu.final_T))
+    for nm in grad_names(app):
+        assert np.all(np.isfinite(getattr(gpu.grads, nm))), nm
+    if differ.sum() == 0:
+        assert image_mismatch(gpu.image, fwd.image, fwd.fragile).sum() == 0
+        assert np.array_equal(gpu.sorted_vals, fwd.vals)
