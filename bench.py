@@ -218,13 +218,14 @@ def run_ours(args):
         if tag == head:
             sampler.start()
         ms_one = timed(lambda: step(ds, r), args.steps, args.warmup)
-        ms = ms_one
+        ms = ms_streams = ms_one
+        graph_note = None
         if views > 1 and n_lanes > 1:
             rs = [r] + [api.Renderer(c, ds.n, WIDTH, HEIGHT, app, pair_capacity=r.pair_capacity) for c in lane_ctx[1:]]
             ms = timed(lambda: step_two_streams(ds, rs), args.steps, args.warmup)
             for c, s_ in zip(lane_ctx, lanes):
                 api.gs_async_status(c, s_)              # raises if a view had outgrown its pair capacity
-            ms_streams, graph_note = ms, None
+            ms_streams = ms
             if not args.no_graph:
                 # The same iteration captured once as a CUDA graph (nothing in it waits for the host) and replayed:
                 # the kernels, their order and their arguments are unchanged, only the launching is.
@@ -268,7 +269,7 @@ def run_ours(args):
             evaluated += ev; composited += co
             rect = r.proj.rect.to(torch.int32) & 0xFFFF
             visible += int(((rect[:, 2] > rect[:, 0]) & (rect[:, 3] > rect[:, 1])).sum().item())
-        results[tag] = dict(ms=ms, ms_one=ms_one, ms_streams=locals().get("ms_streams", ms), graph=locals().get("graph_note"),
+        results[tag] = dict(ms=ms, ms_one=ms_one, ms_streams=ms_streams, graph=graph_note,
                             stage_ms=stage_ms, stage_launches=stage_launches, pairs=pairs,
                             entries=entries, visible=visible, evaluated=evaluated, composited=composited,
                             host=host, ds=ds, r=r, app=tag)
