@@ -1042,6 +1042,128 @@ void gso_preprocess_backward(int64_t n, const double* means, const double* log_s
 
 }  // extern "C"
 
+// ---------------------------------------------------------------------------------------------
+// The decoder with its architecture as a parameter (App. D, architecture table): `layers` hidden layers
+// (1..3) of `hidden` neurons (16 or 32), ReLU, no biases, three tanh outputs; input = 16 SH basis values of
+// the direction (masked by the active degree) followed by 16 feature inputs: nfeat = 8 features as
+// (sin f_j, cos f_j) pairs (Eq. 6, k = 1), or nfeat = 16 raw features without frequency encoding.
+// Weights: W_1[hidden][32], then layers - 1 matrices [hidden][hidden], then W_out[3][hidden], row-major.
+// A second, independent statement of Eq. 5-7: for hidden = 16, layers = 2, nfeat = 8 it must agree with
+// the fixed-size decoder above.
+// ---------------------------------------------------------------------------------------------
+namespace {
+constexpr int kMaxHid = 32, kMaxLayers = 3;
+struct DecState { double x[32], h[kMaxLayers][kMaxHid], A[3]; };
+int dec_num_weights(int hidden, int layers) { return 32 * hidden + (layers - 1) * hidden * hidden + 3 * hidden; }
+void dec_inputs(const double* d, const double* f, int nfeat, int deg, double x[32]) {
+  double Y[16];
+  sh_basis(d, Y);
+  const int na = num_active(deg);
+  for (int k = 0; k < 16; ++k) x[k] = k < na ? Y[k] : 0.0;
+  if (nfeat == 8)
+    for (int j = 0; j < 8; ++j) { x[16 + 2 * j] = std::sin(f[j]); x[17 + 2 * j] = std::cos(f[j]); }
+  else
+    for (int j = 0; j < 16; ++j) x[16 + j] = f[j];
+}
+void dec_forward(const double* W, int hidden, int layers, const double x[32], DecState& s) {
+  const double* w = W;
+  const double* in = x;
+  int nin = 32;
+  for (int l = 0; l < layers; ++l) {
+    for (int o = 0; o < hidden; ++o) {
+      double a = 0;
+      for (int i = 0; i < nin; ++i) a += w[o * nin + i] * in[i];
+      s.h[l][o] = a > 0 ? a : 0;
+    }
+    w += hidden * nin; in = s.h[l]; nin = hidden;
+  }
+  for (int o = 0; o < 3; ++o) {
+    double a = 0;
+    for (int i = 0; i < hidden; ++i) a += w[o * hidden + i] * in[i];
+    s.A[o] = std::tanh(a);
+  }
+}
+}  // namespace
+
+extern "C" {
+int gso_decoder_num_weights(int hidden, int layers) { return dec_num_weights(hidden, layers); }
+// Multiply-accumulates per Gaussian; fold = 1: the 17 view-independent columns of the first layer are
+// pre-multiplied per Gaussian (only worthwhile while hidden <= 16, App. C.3).
+int gso_decoder_macs(int hidden, int layers, int fold) {
+  return (fold ? 16 : 32) * hidden + (layers - 1) * hidden * hidden + 3 * hidden;
+}
+void gso_decoder_forward(int64_t n, int hidden, int layers, int nfeat, int deg, int act, const double* base_color,
+                         const double* features, const double* weights, const double* dirs, double* color) {
+#pragma omp parallel for schedule(static)
+  for (int64_t i = 0; i < n; ++i) {
+    DecState s;
+    s.A[0] = s.A[1] = s.A[2] = 0;
+    if (deg > 0) {
+      double x[32];
+      dec_inputs(dirs + 3 * i, features + (size_t)nfeat * i, nfeat, deg, x);
+      dec_forward(weights, hidden, layers, x, s);
+    }
+    for (int c = 0; c < 3; ++c) color[3 * i + c] = color_act(act, base_color[3 * i + c] + s.A[c]);
+  }
+}
+// g_weights is the sum over the Gaussians in index order.
+void gso_decoder_backward(int64_t n, int hidden, int layers, int nfeat, int deg, int act, const double* base_color,
+                          const double* features, const double* weights, const double* dirs, const double* g_color,
+                          double* g_base, double* g_features, double* g_weights, double* g_dirs) {
+  const int nw = dec_num_weights(hidden, layers);
+  for (int k = 0; k < nw; ++k) g_weights[k] = 0;
+  const int na = num_active(deg);
+  for (int64_t i = 0; i < n; ++i) {
+    for (int c = 0; c < 3; ++c) g_dirs[3 * i + c] = 0;
+    for (int j = 0; j < nfeat; ++j) g_features[(size_t)nfeat * i + j] = 0;
+    if (deg == 0) {
+      for (int c = 0; c < 3; ++c) g_base[3 * i + c] = color_act_grad(act, base_color[3 * i + c]) * g_color[3 * i + c];
+      continue;
+    }
+    DecState s;
+    double x[32];
+    dec_inputs(dirs + 3 * i, features + (size_t)nfeat * i, nfeat, deg, x);
+    dec_forward(weights, hidden, layers, x, s);
+    double g_out[kMaxHid], g_in[kMaxHid > 32 ? kMaxHid : 32];
+    for (int c = 0; c < 3; ++c) {
+      const double gp = color_act_grad(act, base_color[3 * i + c] + s.A[c]) * g_color[3 * i + c];
+      g_base[3 * i + c] = gp;
+      g_out[c] = gp * (1.0 - s.A[c] * s.A[c]);
+    }
+    // walk the layers from the output back: offsets of each matrix
+    int off[kMaxLayers + 1];
+    off[0] = 0;
+    for (int l = 1; l <= layers; ++l) off[l] = off[l - 1] + hidden * (l == 1 ? 32 : hidden);
+    int nout = 3;
+    for (int l = layers; l >= 0; --l) {
+      const double* in = l == 0 ? x : s.h[l - 1];
+      const int nin = l == 0 ? 32 : hidden;
+      const double* w = weights + off[l];
+      double* gw = g_weights + off[l];
+      for (int o = 0; o < nout; ++o)
+        for (int k = 0; k < nin; ++k) gw[o * nin + k] += g_out[o] * in[k];
+      for (int k = 0; k < nin; ++k) {
+        double a = 0;
+        for (int o = 0; o < nout; ++o) a += w[o * nin + k] * g_out[o];
+        g_in[k] = (l == 0 || in[k] > 0) ? a : 0.0;     // ReLU of the layer below (the inputs have none)
+      }
+      for (int k = 0; k < nin; ++k) g_out[k] = g_in[k];
+      nout = hidden;
+      if (l == 0) break;
+    }
+    // g_out now holds dL/dx[0..31]
+    if (nfeat == 8)
+      for (int j = 0; j < 8; ++j) g_features[8 * i + j] = g_out[16 + 2 * j] * x[17 + 2 * j] - g_out[17 + 2 * j] * x[16 + 2 * j];
+    else
+      for (int j = 0; j < 16; ++j) g_features[16 * i + j] = g_out[16 + j];
+    double G[16][3];
+    sh_basis_grad(dirs + 3 * i, G);
+    for (int k = 1; k < na; ++k)
+      for (int a = 0; a < 3; ++a) g_dirs[3 * i + a] += G[k][a] * g_out[k];
+  }
+}
+}
+
 extern "C" {
 double gso_color_act(int act, double x) { return color_act(act, x); }
 double gso_color_act_grad(int act, double x) { return color_act_grad(act, x); }

@@ -103,6 +103,44 @@ def num_mlp_weights() -> int:
     return lib().gso_num_mlp_weights()
 
 
+def decoder_arch(scene):
+    """(hidden, layers, nfeat) of a scene's decoder; the default is the paper's 16 / 2 / 8."""
+    return (int(getattr(scene, "mlp_hidden", 0) or 16), int(getattr(scene, "mlp_layers", 0) or 2),
+            int(scene.features.shape[1]))
+
+
+def decoder_num_weights(hidden: int, layers: int) -> int:
+    return int(lib().gso_decoder_num_weights(C.c_int(hidden), C.c_int(layers)))
+
+
+def decoder_macs(hidden: int, layers: int, fold: bool) -> int:
+    return int(lib().gso_decoder_macs(C.c_int(hidden), C.c_int(layers), C.c_int(1 if fold else 0)))
+
+
+def decoder_forward(scene, dirs, deg=None):
+    """Colour of the neural model for any of the decoder architectures of the paper's architecture table."""
+    hidden, layers, nfeat = decoder_arch(scene)
+    dirs = _f64(dirs); n = dirs.shape[0]
+    color = np.zeros((n, 3))
+    lib().gso_decoder_forward(C.c_int64(n), C.c_int(hidden), C.c_int(layers), C.c_int(nfeat),
+                              C.c_int(scene.active_degree if deg is None else deg), C.c_int(_act(scene)),
+                              _dp(_f64(scene.base_color)), _dp(_f64(scene.features)), _dp(_f64(scene.mlp_weights)),
+                              _dp(dirs), _dp(color))
+    return color
+
+
+def decoder_backward(scene, dirs, g_color, deg=None):
+    hidden, layers, nfeat = decoder_arch(scene)
+    dirs, g_color = _f64(dirs), _f64(g_color); n = dirs.shape[0]
+    o = SimpleNamespace(base_color=np.zeros((n, 3)), features=np.zeros((n, nfeat)),
+                        mlp_weights=np.zeros(decoder_num_weights(hidden, layers)), dirs=np.zeros((n, 3)))
+    lib().gso_decoder_backward(C.c_int64(n), C.c_int(hidden), C.c_int(layers), C.c_int(nfeat),
+                               C.c_int(scene.active_degree if deg is None else deg), C.c_int(_act(scene)),
+                               _dp(_f64(scene.base_color)), _dp(_f64(scene.features)), _dp(_f64(scene.mlp_weights)),
+                               _dp(dirs), _dp(g_color), _dp(o.base_color), _dp(o.features), _dp(o.mlp_weights), _dp(o.dirs))
+    return o
+
+
 ACT_RELU, ACT_SOFTPLUS, ACT_SIGMOID, ACT_HARD_SIGMOID = 0, 1, 2, 3
 
 

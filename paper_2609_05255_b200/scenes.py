@@ -59,6 +59,8 @@ class Scene:
     mlp_weights: Optional[np.ndarray] = None  # [816]  f16: W1[16][32], W2[16][16], W3[3][16]
     color_activation: int = 0                 # 0 ReLU(x+0.5), 1 softplus(x+0.5) beta 10, 2 sigmoid(4x), 3 clamp(x+0.5,0,1)
     sv_sites: Optional[np.ndarray] = None     # [n,7,7] f32: per site (a_r, a_g, a_b, s_x, s_y, s_z, log tau)
+    mlp_hidden: int = 0                       # decoder variant: neurons per hidden layer (0 = the default 16)
+    mlp_layers: int = 0                       # decoder variant: hidden layers (0 = the default 2)
 
     @property
     def n(self) -> int:
@@ -106,12 +108,15 @@ def draw_sh_appearance(rng, n):
     return base_color, sh_rest
 
 
-def draw_neural_appearance(rng, n):
+def draw_neural_appearance(rng, n, hidden: int = MLP_HIDDEN, layers: int = 2, num_features: int = NUM_FEATURES):
+    """Features and Xavier-uniform weights of a decoder with `layers` hidden layers of `hidden` neurons;
+    num_features = 8 (frequency encoded) or 16 (raw).  The defaults are the paper's decoder."""
     dc = rng.normal(0.5, 0.1, (n, 3))
     base_color = _f32(_Y0 * dc)
-    features = _f32(rng.normal(0.0, 0.1, (n, NUM_FEATURES))).astype(np.float16)
+    features = _f32(rng.normal(0.0, 0.1, (n, num_features))).astype(np.float16)
     weights = []
-    for fan_out, fan_in in ((MLP_HIDDEN, MLP_IN), (MLP_HIDDEN, MLP_HIDDEN), (MLP_OUT, MLP_HIDDEN)):
+    shapes = [(hidden, MLP_IN)] + [(hidden, hidden)] * (layers - 1) + [(MLP_OUT, hidden)]
+    for fan_out, fan_in in shapes:
         bound = math.sqrt(6.0 / (fan_in + fan_out))
         weights.append(rng.uniform(-bound, bound, (fan_out, fan_in)).reshape(-1))
     mlp_weights = _f32(np.concatenate(weights)).astype(np.float16)
@@ -266,6 +271,17 @@ def config4(n: int = 3_000_000, width: int = 1920, height: int = 1080, views: in
     """3M Gaussians, 256 clusters with depth range 1-50, neural appearance, 16 orbit cameras."""
     scene = clustered_scene(n, 256, -4.5, 0.8, APP_NEURAL, seed=1004, deep=True)
     return Workload("config4_3M_neural", scene, orbit_cameras(width, height, views))
+
+
+def decoder_variant(n: int, hidden: int, layers: int, num_features: int, seed: int = 1006):
+    """Appearance-sweep inputs for a decoder variant of the paper's architecture table."""
+    rng = np.random.default_rng(np.random.PCG64(seed))
+    geom = (np.zeros((n, 3), np.float32), np.zeros((n, 3), np.float32),
+            np.zeros((n, 4), np.float32), np.zeros((n,), np.float32))
+    base_color, features, weights = draw_neural_appearance(rng, n, hidden, layers, num_features)
+    scene = Scene(*geom, base_color=base_color, app=APP_NEURAL, active_degree=3, features=features,
+                  mlp_weights=weights, mlp_hidden=hidden, mlp_layers=layers)
+    return scene, unit_directions(n, 2006), color_gradient(n, 3006)
 
 
 def config5(n: int, app: int):
