@@ -99,6 +99,16 @@ typedef struct {
                                     s_y, s_z, t): A(d) = sum_i softmax_i(-exp(t_i) |s_i/|s_i| - d|) a_i
                                     (Eq. 3 with the chord distance of App. B); any active_degree >= 1
                                     uses all seven sites, 0 disables the residual                  */
+  int32_t mlp_hidden;            /* neural only: neurons per hidden layer, 16 or 32; 0 means 16   */
+  int32_t mlp_layers;            /* neural only: hidden layers, 1..3; 0 means 2                   */
+  int32_t num_features;          /* neural only: 8 (frequency encoded, Eq. 6) or 16 (fed to the decoder
+                                    as they are, features then [n,16]); 0 means 8.  These three select a
+                                    decoder of the architecture table (App. D): mlp_weights then holds
+                                    W_1[hidden][32], (layers - 1) x [hidden][hidden], W_out[3][hidden],
+                                    32 hidden + (layers - 1) hidden^2 + 3 hidden values.  Anything but
+                                    the default 16 / 2 / 8 is served by gs_appearance_forward and
+                                    gs_appearance_backward only (plain fp32 kernels); every other entry
+                                    point returns GS_ERR_UNSUPPORTED for it                        */
 } GsScene;
 
 /* Per-Gaussian results of gs_preprocess (caller-allocated device buffers). */
@@ -139,8 +149,9 @@ typedef struct {
   float *opacity_logits;  /* [n]                                                               */
   float *base_color;      /* [n,3]                                                             */
   float *sh_rest;         /* SH:     [n,15,3]                                                  */
-  float *features;        /* neural: [n,8] fp32                                                */
-  float *mlp_weights;     /* neural: [816] fp32, summed over all visible Gaussians             */
+  float *features;        /* neural: [n,8] fp32 ([n,16] with num_features = 16)                */
+  float *mlp_weights;     /* neural: [816] fp32 (the variant's weight count otherwise), summed
+                                     over all visible Gaussians                                */
   float *sv_sites;        /* SV:     [n,7,7] with respect to the raw site parameters            */
 } GsGrads;
 

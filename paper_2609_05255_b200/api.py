@@ -39,7 +39,8 @@ class GsCamera(C.Structure):
 class GsScene(C.Structure):
     _fields_ = [("n", C.c_int64), ("means", _vp), ("log_scales", _vp), ("quats", _vp), ("opacity_logits", _vp),
                 ("base_color", _vp), ("app", C.c_int32), ("active_degree", C.c_int32), ("sh_rest", _vp),
-                ("features", _vp), ("mlp_weights", _vp), ("color_activation", C.c_int32), ("sv_sites", _vp)]
+                ("features", _vp), ("mlp_weights", _vp), ("color_activation", C.c_int32), ("sv_sites", _vp),
+                ("mlp_hidden", C.c_int32), ("mlp_layers", C.c_int32), ("num_features", C.c_int32)]
 
 
 class GsProjected(C.Structure):
@@ -160,6 +161,9 @@ class DeviceScene:
     mlp_weights: Optional[torch.Tensor] = None
     color_activation: int = 0        # GS_ACT_*: 0 ReLU(x+0.5), 1 softplus beta 10, 2 sigmoid(4x), 3 clamp(x+0.5, 0, 1)
     sv_sites: Optional[torch.Tensor] = None      # Spherical Voronoi: [n,7,7]
+    mlp_hidden: int = 16             # decoder architecture (App. D); anything but 16 / 2 / 8 runs in
+    mlp_layers: int = 2              # gs_appearance_forward / backward only
+    num_features: int = 8
 
     @property
     def n(self) -> int:
@@ -174,6 +178,7 @@ class DeviceScene:
         s.sh_rest, s.features, s.mlp_weights = _ptr(self.sh_rest), _ptr(self.features), _ptr(self.mlp_weights)
         s.color_activation = int(self.color_activation)
         s.sv_sites = _ptr(self.sv_sites)
+        s.mlp_hidden, s.mlp_layers, s.num_features = int(self.mlp_hidden), int(self.mlp_layers), int(self.num_features)
         return s
 
 
@@ -186,7 +191,9 @@ def upload_scene(scene, device="cuda") -> DeviceScene:
                        up(scene.base_color, torch.float32), int(scene.app), int(scene.active_degree),
                        up(scene.sh_rest, torch.float32), up(scene.features, torch.float16),
                        up(scene.mlp_weights, torch.float16), int(getattr(scene, "color_activation", 0)),
-                       up(getattr(scene, "sv_sites", None), torch.float32))
+                       up(getattr(scene, "sv_sites", None), torch.float32),
+                       int(getattr(scene, "mlp_hidden", 0)) or 16, int(getattr(scene, "mlp_layers", 0)) or 2,
+                       int(scene.features.shape[1]) if scene.features is not None else 8)
 
 
 @dataclass
@@ -262,7 +269,11 @@ class Grads:
         return g
 
 
-def alloc_grads(n: int, app: int, device) -> Grads:
+def decoder_num_weights(hidden: int = 16, layers: int = 2) -> int:
+    return 32 * hidden + (layers - 1) * hidden * hidden + 3 * hidden
+
+
+def alloc_grads(n: int, app: int, device, num_features: int = 8, num_weights: int = MLP_WEIGHTS) -> Grads:
     m = max(n, 1)
     f = dict(device=device, dtype=torch.float32)
     g = Grads(torch.empty((m, 3), **f), torch.empty((m, 3), **f), torch.empty((m, 4), **f),
@@ -272,8 +283,8 @@ def alloc_grads(n: int, app: int, device) -> Grads:
     elif app == GS_APP_SV:
         g.sv_sites = torch.empty((m, 7, 7), **f)
     else:
-        g.features = torch.empty((m, 8), **f)
-        g.mlp_weights = torch.empty((MLP_WEIGHTS,), **f)
+        g.features = torch.empty((m, num_features), **f)
+        g.mlp_weights = torch.empty((num_weights,), **f)
     return g
 
 

@@ -9,7 +9,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libgs_b200.so")
-SOURCES = ["gs_api.cu", "gs_preprocess.cu", "gs_sort.cu", "gs_blend.cu", "gs_adam.cu", "gs_prepass.cu"]
+SOURCES = ["gs_api.cu", "gs_preprocess.cu", "gs_sort.cu", "gs_blend.cu", "gs_adam.cu", "gs_prepass.cu",
+           "gs_decoder_variants.cu"]
 HEADERS = [os.path.join(CSRC, "gs_device.cuh"), os.path.join(_ROOT, "include", "gs.h")]
 
 

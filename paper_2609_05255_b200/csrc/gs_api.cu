@@ -4,6 +4,7 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <algorithm>
 #include <new>
 #include <vector>
 
@@ -90,12 +91,26 @@ CamDev make_cam(const GsCamera *c) {
   return d;
 }
 
+struct DecoderArch { int hidden, layers, nfeat; };
+DecoderArch decoder_arch(const GsScene *s) {
+  return {s->mlp_hidden ? s->mlp_hidden : 16, s->mlp_layers ? s->mlp_layers : 2, s->num_features ? s->num_features : 8};
+}
+bool default_decoder(const GsScene *s) {
+  const DecoderArch d = decoder_arch(s);
+  return s->app != GS_APP_NEURAL || (d.hidden == 16 && d.layers == 2 && d.nfeat == 8);
+}
+
 GsStatus scene_appearance_ok(GsContext *ctx, const GsScene *s) {
   if (s->app != GS_APP_SH && s->app != GS_APP_NEURAL && s->app != GS_APP_SV) return fail(ctx, GS_ERR_INVALID_ARG, "unknown appearance model");
   if (s->active_degree < 0 || s->active_degree > 3) return fail(ctx, GS_ERR_INVALID_ARG, "active_degree must be 0..3");
   if (s->color_activation < GS_ACT_RELU || s->color_activation > GS_ACT_HARD_SIGMOID)
     return fail(ctx, GS_ERR_INVALID_ARG, "unknown colour activation");
   if (s->n < 0) return fail(ctx, GS_ERR_INVALID_ARG, "n < 0");
+  if (s->app == GS_APP_NEURAL) {
+    const DecoderArch d = decoder_arch(s);
+    if ((d.hidden != 16 && d.hidden != 32) || d.layers < 1 || d.layers > 3 || (d.nfeat != 8 && d.nfeat != 16))
+      return fail(ctx, GS_ERR_INVALID_ARG, "decoder must have 1..3 hidden layers of 16 or 32 neurons and 8 or 16 features");
+  }
   if (s->n == 0) return GS_OK;
   if (bad_ptr(s->base_color)) return fail(ctx, GS_ERR_INVALID_ARG, "base_color is NULL or misaligned");
   if (s->app == GS_APP_SH && bad_ptr(s->sh_rest)) return fail(ctx, GS_ERR_INVALID_ARG, "sh_rest is NULL or misaligned");
@@ -109,6 +124,8 @@ GsStatus scene_ok(GsContext *ctx, const GsScene *s) {
   if (!s) return fail(ctx, GS_ERR_INVALID_ARG, "scene is NULL");
   GsStatus st = scene_appearance_ok(ctx, s);
   if (st != GS_OK) return st;
+  if (!default_decoder(s))
+    return fail(ctx, GS_ERR_UNSUPPORTED, "only the 16 / 2 / 8 decoder is fused into the rendering step; the variants run in gs_appearance_forward / backward");
   if (s->n > 0 && (bad_ptr(s->means) || bad_ptr(s->log_scales) || bad_ptr(s->quats) || bad_ptr(s->opacity_logits)))
     return fail(ctx, GS_ERR_INVALID_ARG, "a geometry array is NULL or misaligned");
   return GS_OK;
@@ -182,7 +199,7 @@ GsStatus gs_create(int device, GsContext **out) {
   if (cudaMalloc(&ctx->d_counter, 4 * sizeof(unsigned long long)) != cudaSuccess ||
       cudaMemset(ctx->d_counter, 0, 4 * sizeof(unsigned long long)) != cudaSuccess ||
       cudaMallocHost(&ctx->h_counter, 4 * sizeof(unsigned long long)) != cudaSuccess ||
-      cudaMalloc(&ctx->d_w_partials, sizeof(float) * kWgradBlocks * GS_MLP_WEIGHTS) != cudaSuccess) {
+      cudaMalloc(&ctx->d_w_partials, sizeof(float) * std::max((size_t)kWgradBlocks * GS_MLP_WEIGHTS, variant_partials_floats())) != cudaSuccess) {
     gs_destroy(ctx);
     return GS_ERR_CUDA;
   }
@@ -418,7 +435,9 @@ GsStatus gs_appearance_forward(GsContext *ctx, const GsScene *scene, const float
   a.color = color;
   {
     StageTimer t(ctx, GS_STAGE_APPEARANCE_FWD, static_cast<cudaStream_t>(stream));
-    t.done(launch_appearance_fwd(scene->app, a, static_cast<cudaStream_t>(stream)));
+    const DecoderArch d = decoder_arch(scene);
+    t.done(default_decoder(scene) ? launch_appearance_fwd(scene->app, a, static_cast<cudaStream_t>(stream))
+                                  : launch_variant_fwd(d.hidden, d.layers, d.nfeat, a, static_cast<cudaStream_t>(stream)));
   }
   return check_cuda(ctx, cudaGetLastError(), "appearance_forward launch");
 }
@@ -434,8 +453,10 @@ GsStatus gs_appearance_backward(GsContext *ctx, const GsScene *scene, const floa
   if (scene->app == GS_APP_NEURAL && bad_ptr(grads->mlp_weights))
     return fail(ctx, GS_ERR_INVALID_ARG, "grads->mlp_weights is NULL or misaligned");
   if (scene->n == 0) {
-    if (scene->app == GS_APP_NEURAL)
-      return check_cuda(ctx, cudaMemsetAsync(grads->mlp_weights, 0, sizeof(float) * GS_MLP_WEIGHTS, s), "memset");
+    if (scene->app == GS_APP_NEURAL) {
+      const DecoderArch d = decoder_arch(scene);
+      return check_cuda(ctx, cudaMemsetAsync(grads->mlp_weights, 0, sizeof(float) * variant_num_weights(d.hidden, d.layers), s), "memset");
+    }
     return GS_OK;
   }
   if (bad_ptr(dirs) || bad_ptr(dL_dcolor) || bad_ptr(dL_ddirs) || bad_ptr(grads->base_color))
@@ -455,7 +476,8 @@ GsStatus gs_appearance_backward(GsContext *ctx, const GsScene *scene, const floa
   a.w_partials = ctx->d_w_partials; a.g_weights = grads->mlp_weights;
   {
     StageTimer t(ctx, GS_STAGE_APPEARANCE_BWD, s);
-    t.done(launch_appearance_bwd(scene->app, a, s));
+    const DecoderArch d = decoder_arch(scene);
+    t.done(default_decoder(scene) ? launch_appearance_bwd(scene->app, a, s) : launch_variant_bwd(d.hidden, d.layers, d.nfeat, a, s));
   }
   return check_cuda(ctx, cudaGetLastError(), "appearance_backward launch");
 }
@@ -512,6 +534,7 @@ GsStatus gs_neural_fold(GsContext *ctx, const GsScene *scene, uint16_t *preact, 
   if (!ctx) return GS_ERR_INVALID_ARG;
   if (!scene || scene->n < 0) return fail(ctx, GS_ERR_INVALID_ARG, "scene is NULL or n < 0");
   if (scene->app != GS_APP_NEURAL) return fail(ctx, GS_ERR_UNSUPPORTED, "the fold exists for the neural model only");
+  if (!default_decoder(scene)) return fail(ctx, GS_ERR_UNSUPPORTED, "the fold is built for the 16 / 2 / 8 decoder only");
   if (scene->n == 0) return GS_OK;
   if (bad_ptr(scene->features) || bad_ptr(scene->mlp_weights) || bad_ptr(preact))
     return fail(ctx, GS_ERR_INVALID_ARG, "features, mlp_weights or preact is NULL or misaligned");
@@ -530,6 +553,7 @@ GsStatus gs_neural_prepass(GsContext *ctx, const GsScene *scene, const uint16_t 
   if (!ctx) return GS_ERR_INVALID_ARG;
   if (!scene || scene->n < 0 || !cam) return fail(ctx, GS_ERR_INVALID_ARG, "scene or cam is NULL, or n < 0");
   if (scene->app != GS_APP_NEURAL) return fail(ctx, GS_ERR_UNSUPPORTED, "the prepass exists for the neural model only");
+  if (!default_decoder(scene)) return fail(ctx, GS_ERR_UNSUPPORTED, "the prepass is built for the 16 / 2 / 8 decoder only");
   if (scene->active_degree < 0 || scene->active_degree > 3) return fail(ctx, GS_ERR_INVALID_ARG, "active_degree outside 0..3");
   if (scene->color_activation < GS_ACT_RELU || scene->color_activation > GS_ACT_HARD_SIGMOID)
     return fail(ctx, GS_ERR_INVALID_ARG, "unknown colour activation");

@@ -68,6 +68,12 @@ struct AppearanceArgs {
 int launch_appearance_fwd(int app, const AppearanceArgs &a, cudaStream_t st);
 int launch_appearance_bwd(int app, const AppearanceArgs &a, cudaStream_t st);
 
+// Decoder variants (1-3 hidden layers of 16 or 32 neurons, 8 encoded or 16 raw features): fp32 kernels.
+int variant_num_weights(int hidden, int layers);
+size_t variant_partials_floats();   // floats of per-block weight-gradient partials the backward needs
+int launch_variant_fwd(int hidden, int layers, int nfeat, const AppearanceArgs &a, cudaStream_t st);
+int launch_variant_bwd(int hidden, int layers, int nfeat, const AppearanceArgs &a, cudaStream_t st);
+
 constexpr int kWgradBlocks = 592;   // persistent blocks of the decoder-gradient kernels (4 x 148)
 
 // Sorting / binning.

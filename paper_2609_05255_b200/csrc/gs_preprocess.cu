@@ -938,6 +938,9 @@ extern "C" GsStatus gs_appearance_backward_noalloc(const GsScene *scene, const f
   if (scene->app != GS_APP_NEURAL)
     return fail(GS_ERR_UNSUPPORTED, "only the neural appearance backward uses scratch memory; call gs_appearance_backward for SH");
   if (scene->active_degree < 0 || scene->active_degree > 3) return fail(GS_ERR_INVALID_ARG, "active_degree must be 0..3");
+  if ((scene->mlp_hidden != 0 && scene->mlp_hidden != 16) || (scene->mlp_layers != 0 && scene->mlp_layers != 2) ||
+      (scene->num_features != 0 && scene->num_features != 8))
+    return fail(GS_ERR_UNSUPPORTED, "this entry point serves the 16 / 2 / 8 decoder only");
   if (scene->n < 0) return fail(GS_ERR_INVALID_ARG, "n < 0");
   if (scene->n > kNoAllocMaxN)
     return fail(GS_ERR_CAPACITY, "n exceeds 4194304 Gaussians, the most the static scratch of this entry point covers; "

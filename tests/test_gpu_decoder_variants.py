@@ -1,0 +1,133 @@
+"""The decoder variants of the architecture table (App. D) through the CUDA path: separate-pass decode and
+its backward for 1 to 3 hidden layers of 16 or 32 neurons with 8 encoded or 16 raw features, element by
+element against the oracle's decoder with the same architecture; the entry points that are built for the
+default decoder only must refuse the others."""
+import numpy as np
+import pytest
+
+from paper_2609_05255_b200 import scenes
+from gpu_helpers import grad_mismatch
+
+pytestmark = pytest.mark.gpu
+
+# (hidden, layers, features): the table's rows, the default through the variant kernels' sibling sizes, and
+# the corners of the supported range
+ARCHS = [(16, 1, 8), (16, 3, 8), (32, 2, 8), (16, 2, 16), (32, 1, 16), (32, 3, 16), (32, 3, 8), (16, 1, 16)]
+
+
+def run(api, torch, sc, dirs, gcol):
+    n = dirs.shape[0]
+    ctx = api.Context(0)
+    ds = api.upload_scene(sc, ctx.device)
+    d = torch.from_numpy(dirs).to(ctx.device); gc = torch.from_numpy(gcol).to(ctx.device)
+    color = torch.full((max(n, 1), 3), float("nan"), device=ctx.device)
+    api.gs_appearance_forward(ctx, ds, d, color)
+    grads = api.alloc_grads(n, scenes.APP_NEURAL, ctx.device, ds.num_features,
+                            api.decoder_num_weights(ds.mlp_hidden, ds.mlp_layers))
+    for t in (grads.base_color, grads.features, grads.mlp_weights):
+        t.fill_(float("nan"))
+    gd = torch.full((max(n, 1), 3), float("nan"), device=ctx.device)
+    api.gs_appearance_backward(ctx, ds, d, gc, grads, gd)
+    torch.cuda.synchronize()
+    out = (color.cpu().numpy()[:n], grads.base_color.cpu().numpy()[:n], grads.features.cpu().numpy()[:n],
+           grads.mlp_weights.cpu().numpy(), gd.cpu().numpy()[:n])
+    ctx.close()
+    return out
+
+
+@pytest.mark.parametrize("arch", ARCHS, ids=lambda a: "h%d_l%d_f%d" % a)
+@pytest.mark.parametrize("deg", [3, 1])
+def test_variant_matches_oracle(oracle, arch, deg):
+    import torch
+    from paper_2609_05255_b200 import api
+    hidden, layers, nfeat = arch
+    n = 40_003 if deg == 3 else 4_099       # 313 blocks: more than the backward's persistent grid, ragged tail
+    sc, dirs, gcol = scenes.decoder_variant(n, hidden, layers, nfeat)
+    sc.active_degree = deg
+    color, g_base, g_feat, g_w, g_dirs = run(api, torch, sc, dirs, gcol)
+    ref_c = oracle.decoder_forward(sc, dirs)
+    ref = oracle.decoder_backward(sc, dirs, gcol)
+    assert np.abs(color - ref_c).max() < 2e-5
+    assert grad_mismatch(g_base, ref.base_color).sum() == 0
+    # a hidden unit within rounding of its ReLU kink may switch: allow a handful of Gaussians
+    bad_rows = grad_mismatch(g_feat, ref.features).any(1) | grad_mismatch(g_dirs, ref.dirs).any(1)
+    assert bad_rows.sum() <= max(1, n // 10_000), bad_rows.sum()
+    assert g_w.shape == ref.mlp_weights.shape
+    scale = np.abs(ref.mlp_weights).max()
+    assert np.abs(g_w - ref.mlp_weights).max() < 2e-4 * scale
+
+
+def test_variant_degree_zero_and_activations(oracle):
+    import torch
+    from paper_2609_05255_b200 import api
+    n = 2_050
+    for act, deg in ((0, 0), (1, 3), (2, 3), (3, 0)):
+        sc, dirs, gcol = scenes.decoder_variant(n, 32, 2, 16)
+        sc.active_degree = deg; sc.color_activation = act
+        color, g_base, g_feat, g_w, g_dirs = run(api, torch, sc, dirs, gcol)
+        ref_c = oracle.decoder_forward(sc, dirs)
+        ref = oracle.decoder_backward(sc, dirs, gcol)
+        assert np.abs(color - ref_c).max() < 2e-5
+        near_kink = (np.abs(ref_c) < 1e-5) | (np.abs(ref_c - 1) < 1e-5) if act == 3 else np.zeros((n, 3), bool)
+        assert (grad_mismatch(g_base, ref.base_color) & ~near_kink).sum() == 0
+        if deg == 0:
+            assert not g_feat.any() and not g_dirs.any() and not g_w.any()
+        else:
+            assert grad_mismatch(g_feat, ref.features).any(1).sum() <= 1
+            assert np.abs(g_w - ref.mlp_weights).max() < 2e-4 * np.abs(ref.mlp_weights).max()
+
+
+def test_variant_tiny_and_empty(oracle):
+    import torch
+    from paper_2609_05255_b200 import api
+    for n in (0, 1, 31, 129):
+        sc, dirs, gcol = scenes.decoder_variant(n, 16, 3, 8)
+        color, g_base, g_feat, g_w, g_dirs = run(api, torch, sc, dirs, gcol)
+        if n == 0:
+            assert not g_w.any()
+            continue
+        ref = oracle.decoder_backward(sc, dirs, gcol)
+        assert np.abs(color - oracle.decoder_forward(sc, dirs)).max() < 2e-5
+        assert grad_mismatch(g_feat, ref.features).sum() == 0
+        assert grad_mismatch(g_w, ref.mlp_weights).sum() == 0
+
+
+def test_default_architecture_takes_the_tensor_core_path(oracle):
+    """16 / 2 / 8 named explicitly is the default decoder: same result as leaving the fields at zero."""
+    import torch
+    from paper_2609_05255_b200 import api
+    n = 5_003
+    sc, dirs, gcol = scenes.config5(n, scenes.APP_NEURAL)
+    a = run(api, torch, sc, dirs, gcol)
+    sc.mlp_hidden, sc.mlp_layers = 16, 2
+    b = run(api, torch, sc, dirs, gcol)
+    for x, y in zip(a[:3] + a[4:], b[:3] + b[4:]):
+        assert np.array_equal(x, y)
+    ref = oracle.decoder_backward(sc, dirs, gcol)
+    assert grad_mismatch(b[2], ref.features).any(1).sum() <= 1
+
+
+def test_fused_entry_points_refuse_variants():
+    import torch
+    from paper_2609_05255_b200 import api
+    w = scenes.config2(n=500, app=scenes.APP_NEURAL)
+    sc = w.scene
+    sc.mlp_hidden = 32
+    sc.mlp_weights = np.zeros(api.decoder_num_weights(32, 2), np.float16)
+    ctx = api.Context(0)
+    ds = api.upload_scene(sc, ctx.device)
+    cam = api.make_camera(w.cameras[0])
+    proj = api.alloc_projected(ds.n, ctx.device, False)
+    with pytest.raises(api.GsError) as e:
+        api.gs_preprocess(ctx, ds, cam, proj)
+    assert e.value.status == api.GS_ERR_UNSUPPORTED
+    preact = torch.empty((ds.n, 16), dtype=torch.float16, device=ctx.device)
+    with pytest.raises(api.GsError) as e:
+        api.gs_neural_fold(ctx, ds, preact)
+    assert e.value.status == api.GS_ERR_UNSUPPORTED
+    bad = api.upload_scene(sc, ctx.device)
+    bad.mlp_hidden = 24
+    with pytest.raises(api.GsError) as e:
+        api.gs_appearance_forward(ctx, bad, torch.zeros((ds.n, 3), device=ctx.device), torch.zeros((ds.n, 3), device=ctx.device))
+    assert e.value.status == api.GS_ERR_INVALID_ARG
+    ctx.close()
