@@ -34,6 +34,7 @@ BLEND_FLOPS_PER_EVALUATED = 8.0       # 3.5 (quad falloff, shared by 4 pixels) +
 BLEND_FWD_FLOPS_PER_COMPOSITED = 10.0  # 1-a, T(1-a), compare, aT, three FMAs
 BLEND_BWD_FLOPS_PER_COMPOSITED = 45.0  # reciprocal, T and S recovery, d/d alpha, nine gradient FMAs
 FP32_LANES_PER_SM, NUM_SMS = 128, 148
+FP32_ALU_PEAK_TFLOPS = NUM_SMS * FP32_LANES_PER_SM * 2 * 1965e6 / 1e12   # 74.4 at the maximum SM clock
 
 
 def measured_peaks():
@@ -654,6 +655,44 @@ def decode_sweep(api, torch, ctx, dev, peaks, args):
                 "GBps": round(gbs, 1), "frac_of_hbm_peak": round(gbs / peaks["hbm_gbs"], 4),
                 "fwd_GBps": round(bytes_fwd * n / (f_ms * 1e-3) / 1e9, 1),
                 "bwd_GBps": round(bytes_bwd * n / (b_ms * 1e-3) / 1e9, 1),
+                "Gprimitives_per_s": round(n / ((f_ms + b_ms) * 1e-3) / 1e9, 3)}
+            del sc, color, grads, gd, flush
+        # the decoder variants of the architecture table (App. D), fp32 CUDA-core kernels: 1M only
+        for hidden, layers, nfeat in (((16, 1, 8), (16, 3, 8), (32, 2, 8), (16, 2, 16)) if n == 1_000_000 else ()):
+            nw = api.decoder_num_weights(hidden, layers)
+            w = ((torch.rand((nw,), device=dev, generator=gen) - 0.5) * (16.0 / hidden) ** 0.5).half()
+            sc = api.DeviceScene(z, z, z, z[0], base, 1, 3,
+                                 features=(0.1 * torch.randn((n, nfeat), device=dev, generator=gen)).half(), mlp_weights=w,
+                                 mlp_hidden=hidden, mlp_layers=layers, num_features=nfeat)
+            fb = 2 * nfeat
+            bytes_fwd, bytes_bwd = fb + 12 + 12 + 12, 12 + 12 + fb + 12 + 12 + 4 * nfeat + 12
+            color = torch.empty((n, 3), device=dev)
+            grads = api.alloc_grads(n, 1, dev, nfeat, nw)
+            gd = torch.empty((n, 3), device=dev)
+            flush = torch.empty((256 << 20,), device=dev, dtype=torch.uint8)
+
+            def run_v(fn, reps=10):
+                ts = []
+                for i in range(reps + 3):
+                    flush.zero_()
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record(); fn(); e1.record()
+                    torch.cuda.synchronize()
+                    if i >= 3:
+                        ts.append(e0.elapsed_time(e1))
+                ts.sort()
+                return ts[len(ts) // 2]
+            f_ms = run_v(lambda: api.gs_appearance_forward(ctx, sc, dirs, color))
+            b_ms = run_v(lambda: api.gs_appearance_backward(ctx, sc, dirs, gcol, grads, gd))
+            # forward: one pass over the weights; backward: the forward again, the transposed pass and the weight gradient
+            flop_fwd, flop_bwd = 2 * nw * n, 6 * nw * n
+            out[f"neural_h{hidden}_l{layers}_f{nfeat}_{n // 1_000_000}M"] = {
+                "weights": nw, "fwd_ms": round(f_ms, 4), "bwd_ms": round(b_ms, 4),
+                "bytes_per_primitive": bytes_fwd + bytes_bwd,
+                "GBps": round((bytes_fwd + bytes_bwd) * n / ((f_ms + b_ms) * 1e-3) / 1e9, 1),
+                "fwd_fp32_TFLOPs": round(flop_fwd / (f_ms * 1e-3) / 1e12, 2),
+                "bwd_fp32_TFLOPs": round(flop_bwd / (b_ms * 1e-3) / 1e12, 2),
+                "frac_of_fp32_alu_peak": round((flop_fwd + flop_bwd) / ((f_ms + b_ms) * 1e-3) / 1e12 / FP32_ALU_PEAK_TFLOPS, 4),
                 "Gprimitives_per_s": round(n / ((f_ms + b_ms) * 1e-3) / 1e9, 3)}
             del sc, color, grads, gd, flush
         del dirs, gcol, base
