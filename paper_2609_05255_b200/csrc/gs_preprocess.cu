@@ -175,14 +175,16 @@ __device__ __forceinline__ void explicit_bwd(float *row, const float gp[3], floa
 }
 
 // ---- appearance: neural ---------------------------------------------------------------------
-__device__ __forceinline__ void load_features(const __half *features, int64_t i, float f[8]) {
-  const uint4 raw = __ldg(reinterpret_cast<const uint4 *>(features) + i);
+__device__ __forceinline__ void unpack_features(const uint4 &raw, float f[8]) {
   const __half2 *h = reinterpret_cast<const __half2 *>(&raw);
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
     const float2 v = __half22float2(h[j]);
     f[2 * j] = v.x; f[2 * j + 1] = v.y;
   }
+}
+__device__ __forceinline__ void load_features(const __half *features, int64_t i, float f[8]) {
+  unpack_features(__ldg(reinterpret_cast<const uint4 *>(features) + i), f);
 }
 
 // Decoder inputs of one Gaussian (Eq. 5, Eq. 6 with k = 1): SH basis of the direction masked by the
@@ -635,24 +637,31 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_bwd(PreprocessBwdArgs a, 
     const int64_t i = chunk * kBlock + tid;
     const int64_t row0 = chunk * kBlock + warp * 32;
     const bool in = i < a.n;
+    // Every input row of this Gaussian is requested here, before anything depends on one of them (also for
+    // culled Gaussians, whose rows are then ignored): one memory round trip per trip of the loop instead of one
+    // per branch that needs a value.
     bool vis = false;
+    float gd[3] = {0.f, 0.f, 0.f};
+    float mu[3] = {0.f, 0.f, 0.f}, ls[3] = {0.f, 0.f, 0.f}, q[4] = {1.f, 0.f, 0.f, 0.f}, logit = 0.f;
+    float4 ga = make_float4(0.f, 0.f, 0.f, 0.f), gb = ga, gc = ga;
+    float base_in[3] = {0.f, 0.f, 0.f};
+    uint4 feat_raw = make_uint4(0u, 0u, 0u, 0u);
+    float dx = 0.f, dy = 0.f, dz = 0.f;
     if (in) {
       const ushort4 rc = __ldg(reinterpret_cast<const ushort4 *>(a.rect) + i);
-      vis = rc.z > rc.x && rc.w > rc.y;
-    }
-    const bool warp_vis = __any_sync(kFull, vis);
-    float gd[3] = {0.f, 0.f, 0.f};
-    float mu[3], ls[3], q[4], logit = 0.f;
-    float4 ga = make_float4(0.f, 0.f, 0.f, 0.f), gb = ga, gc = ga;
-    float dx = 0.f, dy = 0.f, dz = 0.f;
-    if (vis) {
       load3(a.means, i, mu);
       load3(a.log_scales, i, ls);
       const float4 q4 = __ldg(reinterpret_cast<const float4 *>(a.quats) + i);
-      q[0] = q4.x; q[1] = q4.y; q[2] = q4.z; q[3] = q4.w;
       logit = __ldg(a.logits + i);
       const float4 *g2 = reinterpret_cast<const float4 *>(a.g2d) + 3 * i;
       ga = g2[0]; gb = g2[1]; gc = g2[2];   // (gr, gg, gb, go) (gA, gB, gC, gu) (gv, -, -, -)
+      load3(a.base_color, i, base_in);
+      if (APP == GS_APP_NEURAL) feat_raw = __ldg(reinterpret_cast<const uint4 *>(a.features) + i);
+      q[0] = q4.x; q[1] = q4.y; q[2] = q4.z; q[3] = q4.w;
+      vis = rc.z > rc.x && rc.w > rc.y;
+    }
+    const bool warp_vis = __any_sync(kFull, vis);
+    if (vis) {
       const float vx = mu[0] - cam.oc[0], vy = mu[1] - cam.oc[1], vz = mu[2] - cam.oc[2];
       const float vi = rsqrtf(vx * vx + vy * vy + vz * vz);
       dx = vx * vi; dy = vy * vi; dz = vz * vi;
@@ -666,8 +675,8 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_bwd(PreprocessBwdArgs a, 
         }
         float *row = slab + lane * RowOf<APP>::value;
         if (vis) {
-          float base[3], pre[3];
-          load3(a.base_color, i, base);
+          float pre[3];
+          const float (&base)[3] = base_in;
           SvCarry cy;
           if (a.deg > 0) explicit_pre<APP>(row, base, dx, dy, dz, a.deg, pre, cy);
           else { pre[0] = base[0] + 0.5f; pre[1] = base[1] + 0.5f; pre[2] = base[2] + 0.5f; }
@@ -684,12 +693,12 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_bwd(PreprocessBwdArgs a, 
       float gf[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
       float base[3] = {0.f, 0.f, 0.f};
       const float gcol[3] = {ga.x, ga.y, ga.z};
-      if (vis) load3(a.base_color, i, base);
+      if (vis) { base[0] = base_in[0]; base[1] = base_in[1]; base[2] = base_in[2]; }
       if (warp_vis && a.deg > 0) {   // the whole warp goes through the decoder; culled lanes feed zeros
         float x[32];
         if (vis) {
           float f[8];
-          load_features(a.features, i, f);
+          unpack_features(feat_raw, f);
           decoder_inputs(dx, dy, dz, f, a.deg, x);
         } else {
 #pragma unroll
@@ -850,6 +859,24 @@ void opt_in_smem(K kernel, size_t bytes) {
   cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
 }
 
+// Grid of a persistent kernel: as many CTAs as fit on the device at once (a second, thinner wave of a
+// grid-stride loop would run at a fraction of the occupancy), at most kWgradBlocks (rows of the partial buffer).
+template <class K>
+int resident_blocks(K kernel, size_t smem_bytes) {
+  static int cached[64] = {};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (dev < 0 || dev >= 64) return kWgradBlocks;
+  if (!cached[dev]) {
+    int per_sm = 0, sms = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kBlock, smem_bytes) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || per_sm <= 0 || sms <= 0)
+      return kWgradBlocks;
+    cached[dev] = per_sm * sms < kWgradBlocks ? per_sm * sms : kWgradBlocks;
+  }
+  return cached[dev];
+}
+
 }  // namespace
 
 int launch_preprocess_fwd(int app, const PreprocessArgs &a, const CamDev &cam, cudaStream_t st) {
@@ -873,8 +900,9 @@ int launch_preprocess_bwd(int app, const PreprocessBwdArgs &a, const CamDev &cam
     return 1;
   } else {
     opt_in_smem(k_preprocess_bwd<GS_APP_NEURAL>, kBwdSmemNN);
-    k_preprocess_bwd<GS_APP_NEURAL><<<kWgradBlocks, kBlock, kBwdSmemNN, st>>>(a, cam);
-    launch_wgrad_reduce(a.w_partials, kWgradBlocks, a.g_weights, st);
+    const int blocks = resident_blocks(k_preprocess_bwd<GS_APP_NEURAL>, kBwdSmemNN);
+    k_preprocess_bwd<GS_APP_NEURAL><<<blocks, kBlock, kBwdSmemNN, st>>>(a, cam);
+    launch_wgrad_reduce(a.w_partials, blocks, a.g_weights, st);
     return 2;
   }
 }
@@ -900,8 +928,9 @@ int launch_appearance_bwd(int app, const AppearanceArgs &a, cudaStream_t st) {
     return 1;
   } else {
     opt_in_smem(k_appearance_bwd<GS_APP_NEURAL>, kBwdSmemNN);
-    k_appearance_bwd<GS_APP_NEURAL><<<kWgradBlocks, kBlock, kBwdSmemNN, st>>>(a);
-    launch_wgrad_reduce(a.w_partials, kWgradBlocks, a.g_weights, st);
+    const int blocks = resident_blocks(k_appearance_bwd<GS_APP_NEURAL>, kBwdSmemNN);
+    k_appearance_bwd<GS_APP_NEURAL><<<blocks, kBlock, kBwdSmemNN, st>>>(a);
+    launch_wgrad_reduce(a.w_partials, blocks, a.g_weights, st);
     return 2;
   }
 }
