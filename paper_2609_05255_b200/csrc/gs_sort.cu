@@ -267,6 +267,8 @@ __global__ void __launch_bounds__(1024) k_scan_single_block(uint32_t *__restrict
 // Emit the instances of each Gaussian, in depth order: the tiles its alpha >= 1/255 ellipse meets
 // (TileSpans, the same function the preprocess counted with), tile rows top to bottom, tiles left
 // to right.  Small footprints are written by their own thread; large ones by the whole warp.
+constexpr uint32_t kKeygenStage = 512;   // instances a warp stages in shared memory (4 KB per warp)
+
 __global__ void __launch_bounds__(kScanBlock) k_keygen(const uint32_t *__restrict__ order, const uint16_t *__restrict__ rect,
                                                        const float *__restrict__ mean2d,
                                                        const float *__restrict__ conic_opacity,
@@ -276,6 +278,7 @@ __global__ void __launch_bounds__(kScanBlock) k_keygen(const uint32_t *__restric
                                                        uint32_t *__restrict__ inst_tiles,
                                                        uint32_t *__restrict__ inst_vals) {
   __shared__ uint32_t s_w[kScanBlock / 32];
+  __shared__ uint32_t s_stage[kScanBlock / 32][2 * kKeygenStage];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int64_t i = (int64_t)blockIdx.x * kScanBlock + tid;
   uint32_t g = 0, tiles = 0;
@@ -284,11 +287,13 @@ __global__ void __launch_bounds__(kScanBlock) k_keygen(const uint32_t *__restric
   float2 sp1 = make_float2(1.f, 0.f);             // lc, tau
   if (i < n) {
     g = __ldg(order + i);
+    // the four gathers go out together (also for Gaussians without tiles, whose rows are then ignored)
     tiles = __ldg(tiles_touched + g);
+    const ushort4 rr = __ldg(reinterpret_cast<const ushort4 *>(rect) + g);
+    const float2 m = __ldg(reinterpret_cast<const float2 *>(mean2d) + g);
+    const float4 q = __ldg(reinterpret_cast<const float4 *>(conic_opacity) + g);
     if (tiles) {
-      r = __ldg(reinterpret_cast<const ushort4 *>(rect) + g);
-      const float2 m = __ldg(reinterpret_cast<const float2 *>(mean2d) + g);
-      const float4 q = __ldg(reinterpret_cast<const float4 *>(conic_opacity) + g);
+      r = rr;
       sp0 = make_float4(m.x, m.y, q.x, q.y);
       sp1 = make_float2(q.z, footprint_tau(q.w));
     }
@@ -306,6 +311,17 @@ __global__ void __launch_bounds__(kScanBlock) k_keygen(const uint32_t *__restric
   for (int k = 0; k < kScanBlock / 32; ++k) off += (k < warp) ? s_w[k] : 0u;
   off += inc - tiles;
   constexpr uint32_t kSmall = 32;
+  // A warp whose footprints add up to at most kKeygenStage instances writes them to shared memory first and
+  // copies the block out with coalesced stores; lanes writing their own short runs directly would touch a
+  // different sector with every store.  Staged or not, the emission below is the same: only the destination
+  // and the origin of the positions differ.
+  const uint32_t warp_total = __shfl_sync(kFull, inc, 31);
+  const uint32_t warp_base = __shfl_sync(kFull, off, 0);
+  const bool staged = warp_total <= kKeygenStage;
+  uint32_t *dst_tiles = staged ? s_stage[warp] : inst_tiles;
+  uint32_t *dst_vals = staged ? s_stage[warp] + kKeygenStage : inst_vals;
+  const uint32_t limit = staged ? kKeygenStage : capacity;   // never past the buffers, even if the count was taken on the device
+  if (staged) off -= warp_base;
   if (tiles > 0 && tiles <= kSmall) {
     TileSpans sp;
     sp.setup(sp0.x, sp0.y, sp0.z, sp0.w, sp1.x, sp1.y, W, H);
@@ -314,9 +330,9 @@ __global__ void __launch_bounds__(kScanBlock) k_keygen(const uint32_t *__restric
       int xa, xb;
       if (!sp.row(ty, r.x, r.z, xa, xb)) continue;
       for (int tx = xa; tx < xb; ++tx) {
-        if (p < capacity) {   // never past the caller's buffers, even if the count was taken on the device
-          inst_tiles[p] = (uint32_t)(ty * gx + tx);
-          inst_vals[p] = g;
+        if (p < limit) {
+          dst_tiles[p] = (uint32_t)(ty * gx + tx);
+          dst_vals[p] = g;
         }
         ++p;
       }
@@ -350,13 +366,23 @@ __global__ void __launch_bounds__(kScanBlock) k_keygen(const uint32_t *__restric
         const uint32_t o = p + __shfl_sync(kFull, excl, rr);
         for (int tx = a + lane; tx < b; tx += 32) {
           const uint32_t q = o + (uint32_t)(tx - a);
-          if (q < capacity) {
-            inst_tiles[q] = (uint32_t)((tyb + rr) * gx + tx);
-            inst_vals[q] = s_g;
+          if (q < limit) {
+            dst_tiles[q] = (uint32_t)((tyb + rr) * gx + tx);
+            dst_vals[q] = s_g;
           }
         }
       }
       p += __shfl_sync(kFull, incl, 31);
+    }
+  }
+  if (staged) {
+    __syncwarp();
+    const uint32_t *st = s_stage[warp], *sv = st + kKeygenStage;
+    for (uint32_t q = lane; q < warp_total; q += 32) {
+      if (warp_base + q < capacity) {
+        inst_tiles[warp_base + q] = st[q];
+        inst_vals[warp_base + q] = sv[q];
+      }
     }
   }
 }
