@@ -17,32 +17,42 @@ constexpr int kSortTile = kSortThreads * kItems;   // 4096 elements per block it
 constexpr int kMaxSortBlocks = 444;                // 3 resident CTAs x 148 SMs: one full wave
 constexpr unsigned kFull = 0xffffffffu;
 
-struct SortPlan { int blocks; int tiles_per_block; };
+// Block b sorts tiles_per_block (+ 1 if b < extra) consecutive tiles of kSortTile elements: the tiles are dealt
+// out as evenly as whole tiles allow over one full wave of CTAs.
+struct SortPlan { int blocks; int tiles_per_block; int extra; };
 
 SortPlan plan_for(int64_t count) {
   const int64_t tiles = (count + kSortTile - 1) / kSortTile;
   SortPlan p;
   p.blocks = (int)(tiles < kMaxSortBlocks ? tiles : kMaxSortBlocks);
   if (p.blocks < 1) p.blocks = 1;
-  p.tiles_per_block = (int)((tiles + p.blocks - 1) / p.blocks);
-  if (p.tiles_per_block < 1) p.tiles_per_block = 1;
-  p.blocks = (int)((tiles + p.tiles_per_block - 1) / p.tiles_per_block);
-  if (p.blocks < 1) p.blocks = 1;
+  p.tiles_per_block = (int)(tiles / p.blocks);
+  p.extra = (int)(tiles - (int64_t)p.tiles_per_block * p.blocks);
   return p;
+}
+
+// First tile and number of tiles of a block under the plan.
+__device__ __forceinline__ void block_tiles(int tiles_per_block, int extra, int64_t &first, int &num) {
+  const int b = (int)blockIdx.x;
+  first = (int64_t)b * tiles_per_block + min(b, extra);
+  num = tiles_per_block + (b < extra ? 1 : 0);
 }
 
 // Digit histogram of each block's contiguous range: table[block][digit].
 __global__ void __launch_bounds__(kSortThreads) k_radix_hist(const uint32_t *__restrict__ keys, int64_t count,
                                                              const unsigned long long *__restrict__ count_dev,
-                                                             int shift, uint32_t mask, int tiles_per_block,
+                                                             int shift, uint32_t mask, int tiles_per_block, int extra,
                                                              uint32_t *__restrict__ table) {
   if (count_dev) count = min(count, (int64_t)__ldg(count_dev));   // the true length lives on the device
   __shared__ uint32_t s_hist[kSortWarps][256];
   const int tid = threadIdx.x, warp = tid >> 5;
   for (int k = tid; k < kSortWarps * 256; k += kSortThreads) (&s_hist[0][0])[k] = 0;
   __syncthreads();
-  const int64_t begin = (int64_t)blockIdx.x * tiles_per_block * kSortTile;
-  int64_t end = begin + (int64_t)tiles_per_block * kSortTile;
+  int64_t first_tile;
+  int my_tiles;
+  block_tiles(tiles_per_block, extra, first_tile, my_tiles);
+  const int64_t begin = first_tile * kSortTile;
+  int64_t end = begin + (int64_t)my_tiles * kSortTile;
   if (end > count) end = count;
   for (int64_t i = begin + tid; i < end; i += kSortThreads) {
     const uint32_t d = (__ldg(keys + i) >> shift) & mask;
@@ -112,7 +122,7 @@ template <int BITS>
 __global__ void __launch_bounds__(kSortThreads, 3) k_radix_scatter(
     const uint32_t *__restrict__ keys_in, const uint32_t *__restrict__ vals_in, uint32_t *__restrict__ keys_out,
     uint32_t *__restrict__ vals_out, int64_t count, const unsigned long long *__restrict__ count_dev, int shift,
-    int tiles_per_block,
+    int tiles_per_block, int extra,
     const uint32_t *__restrict__ table, const uint32_t *__restrict__ totals, int nblocks) {
   __shared__ uint32_t s_keys[kSortTile];
   __shared__ uint32_t s_vals[kSortTile];
@@ -132,8 +142,11 @@ __global__ void __launch_bounds__(kSortThreads, 3) k_radix_scatter(
     s_base[tid] = start + __ldg(table + (size_t)tid * nblocks + blockIdx.x);
   }
 
-  const int64_t begin = (int64_t)blockIdx.x * tiles_per_block * kSortTile;
-  for (int t = 0; t < tiles_per_block; ++t) {
+  int64_t first_tile;
+  int my_tiles;
+  block_tiles(tiles_per_block, extra, first_tile, my_tiles);
+  const int64_t begin = first_tile * kSortTile;
+  for (int t = 0; t < my_tiles; ++t) {
     const int64_t tile_begin = begin + (int64_t)t * kSortTile;
     if (tile_begin >= count) break;
     const int valid_count = (int)min((int64_t)kSortTile, count - tile_begin);
@@ -387,19 +400,34 @@ __global__ void __launch_bounds__(kScanBlock) k_keygen(const uint32_t *__restric
   }
 }
 
-__global__ void k_tile_ranges(const uint32_t *__restrict__ sorted_tiles, int64_t P,
-                              const unsigned long long *__restrict__ count_dev, uint32_t *__restrict__ overflow,
-                              uint32_t *__restrict__ ranges) {
-  const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+// Four consecutive entries per thread (one 16-byte load plus the two neighbours).
+__global__ void __launch_bounds__(256) k_tile_ranges(const uint32_t *__restrict__ sorted_tiles, int64_t P,
+                                                     const unsigned long long *__restrict__ count_dev,
+                                                     uint32_t *__restrict__ overflow, uint32_t *__restrict__ ranges) {
+  const int64_t p0 = 4 * ((int64_t)blockIdx.x * blockDim.x + threadIdx.x);
   if (count_dev) {   // P is the capacity here; more instances than that were cut off: tell the host
     const int64_t c = (int64_t)__ldg(count_dev);
-    if (p == 0 && c > P) *overflow = 1u;
+    if (p0 == 0 && c > P) *overflow = 1u;
     P = min(P, c);
   }
-  if (p >= P) return;
-  const uint32_t t = __ldg(sorted_tiles + p);
-  if (p == 0 || t != __ldg(sorted_tiles + p - 1)) ranges[2 * t] = (uint32_t)p;
-  if (p == P - 1 || t != __ldg(sorted_tiles + p + 1)) ranges[2 * t + 1] = (uint32_t)(p + 1);
+  if (p0 >= P) return;
+  uint32_t t[6];   // entries p0 - 1 .. p0 + 4
+  if (p0 + 4 <= P) {
+    const uint4 v = __ldg(reinterpret_cast<const uint4 *>(sorted_tiles + p0));
+    t[1] = v.x; t[2] = v.y; t[3] = v.z; t[4] = v.w;
+  } else {
+#pragma unroll
+    for (int k = 0; k < 4; ++k) t[1 + k] = p0 + k < P ? __ldg(sorted_tiles + p0 + k) : 0u;
+  }
+  t[0] = p0 > 0 ? __ldg(sorted_tiles + p0 - 1) : 0u;
+  t[5] = p0 + 4 < P ? __ldg(sorted_tiles + p0 + 4) : 0u;
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const int64_t p = p0 + k;
+    if (p >= P) break;
+    if (p == 0 || t[1 + k] != t[k]) ranges[2 * t[1 + k]] = (uint32_t)p;
+    if (p == P - 1 || t[1 + k] != t[2 + k]) ranges[2 * t[1 + k] + 1] = (uint32_t)(p + 1);
+  }
 }
 
 // Launch order of the blend CTAs: tiles by decreasing list length (log2 buckets), so that the long
@@ -446,18 +474,18 @@ int launch_radix_sort(const uint32_t *keys_in, const uint32_t *vals_in, uint32_t
     const bool to_out = ((passes - 1 - p) % 2) == 0;
     uint32_t *dst_k = to_out ? keys_out : tmp_keys, *dst_v = to_out ? vals_out : tmp_vals;
     k_radix_hist<<<plan.blocks, kSortThreads, 0, st>>>(src_k, count, count_dev, bits * p, (1u << bits) - 1u,
-                                                        plan.tiles_per_block, table);
+                                                        plan.tiles_per_block, plan.extra, table);
     k_radix_scan_rows<<<256, 256, 0, st>>>(table, plan.blocks, totals);
 #define GS_SCATTER(B)                                                                                              \
   case B:                                                                                                          \
     k_radix_scatter<B><<<plan.blocks, kSortThreads, 0, st>>>(src_k, src_v, dst_k, dst_v, count, count_dev, bits * p, \
-                                                              plan.tiles_per_block, table, totals, plan.blocks);   \
+                                                              plan.tiles_per_block, plan.extra, table, totals, plan.blocks);   \
     break;
     switch (bits) {
       GS_SCATTER(1) GS_SCATTER(2) GS_SCATTER(3) GS_SCATTER(4) GS_SCATTER(5) GS_SCATTER(6) GS_SCATTER(7)
       default:
         k_radix_scatter<8><<<plan.blocks, kSortThreads, 0, st>>>(src_k, src_v, dst_k, dst_v, count, count_dev, bits * p,
-                                                                  plan.tiles_per_block, table, totals, plan.blocks);
+                                                                  plan.tiles_per_block, plan.extra, table, totals, plan.blocks);
     }
 #undef GS_SCATTER
     src_k = dst_k;
@@ -491,7 +519,7 @@ int launch_keygen(const uint32_t *depth_order, const uint16_t *rect, const float
 int launch_tile_ranges(const uint32_t *sorted_tiles, int64_t P, const unsigned long long *count_dev, uint32_t *overflow,
                        uint32_t *ranges, uint32_t *order, int num_tiles, cudaStream_t st) {
   cudaMemsetAsync(ranges, 0, (size_t)num_tiles * 2 * sizeof(uint32_t), st);
-  if (P > 0) k_tile_ranges<<<(int)((P + 255) / 256), 256, 0, st>>>(sorted_tiles, P, count_dev, overflow, ranges);
+  if (P > 0) k_tile_ranges<<<(int)((P + 1023) / 1024), 256, 0, st>>>(sorted_tiles, P, count_dev, overflow, ranges);
   k_tile_order<<<1, 1024, 0, st>>>(ranges, num_tiles, order);
   return P > 0 ? 2 : 1;
 }
