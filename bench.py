@@ -334,7 +334,7 @@ def run_ours(args):
 
 # dram__bytes_read.sum + dram__bytes_write.sum of ONE launch (orbit view 0 of the default workload), from the
 # ncu --set full captures summarised under profiles/.  Bytes.
-NCU_TRAFFIC_1M_NEURAL = {"blend_bwd": 47.37e6, "blend_fwd": 25.73e6, "preprocess_bwd": 181.99e6,
+NCU_TRAFFIC_1M_NEURAL = {"blend_bwd": 47.37e6, "blend_fwd": 25.73e6, "preprocess_bwd": 180.64e6,
                          "preprocess_fwd": 89.63e6}
 
 
@@ -342,8 +342,8 @@ NCU_TRAFFIC_1M_NEURAL = {"blend_bwd": 47.37e6, "blend_fwd": 25.73e6, "preprocess
 # fills while it runs.  For the ALU-bound blend kernels this, not the flop rate, says how close to the machine they
 # are: the flop count above is the method's minimum arithmetic, the issue slots also carry loads, predicates,
 # shuffles and loop control.
-NCU_ISSUE_ACTIVE_1M_NEURAL = {"blend_bwd": 0.81, "blend_fwd": 0.70, "preprocess_bwd": 0.38, "preprocess_fwd": 0.72,
-                              "keygen": 0.46}
+NCU_ISSUE_ACTIVE_1M_NEURAL = {"blend_bwd": 0.81, "blend_fwd": 0.70, "preprocess_bwd": 0.53, "preprocess_fwd": 0.72,
+                              "keygen": 0.57}
 
 
 def stage_roofline(stage, arm, views, n, peaks, alu_peak):

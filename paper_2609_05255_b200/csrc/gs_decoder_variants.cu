@@ -15,7 +15,7 @@ namespace {
 
 constexpr int kVarBlock = 128;
 constexpr int kVarWarps = kVarBlock / 32;
-constexpr int kVarPartialBlocks = 296;   // persistent CTAs of the backward (2 x 148)
+constexpr int kVarPartialBlocks = 592;   // most persistent CTAs of the backward (rows of the partial buffer)
 
 template <int H, int L> struct VarDims {
   static constexpr int kNumW = 32 * H + (L - 1) * H * H + 3 * H;
@@ -119,15 +119,36 @@ __global__ void __launch_bounds__(kVarBlock) k_variant_fwd(AppearanceArgs a, int
 }
 
 // Weight gradient of one layer for the warp's 32 Gaussians: sX [32][NIN] inputs, sG [32][NOUT] output gradients
-// (rows of Gaussians without one are zero); lane owns weights lane, lane + 32, ...
+// (rows of Gaussians without one are zero).  A lane owns one input column and four output rows at a time, so one
+// load of the input and one 16-byte load of the gradients feed four FMAs; the sums of every element are taken in
+// Gaussian order by its one owner.
 template <int NOUT, int NIN>
 __device__ __forceinline__ void warp_weight_grad(const float *sX, const float *sG, float *sDW, int lane) {
-  for (int w = lane; w < NOUT * NIN; w += 32) {
-    const int o = w / NIN, i = w % NIN;
-    float acc = sDW[w];
+  if (NOUT % 4 != 0) {   // the three output rows
+    for (int w = lane; w < NOUT * NIN; w += 32) {
+      const int o = w / NIN, i = w % NIN;
+      float acc = sDW[w];
 #pragma unroll 8
-    for (int g = 0; g < 32; ++g) acc = fmaf(sG[g * NOUT + o], sX[g * NIN + i], acc);
-    sDW[w] = acc;
+      for (int g = 0; g < 32; ++g) acc = fmaf(sG[g * NOUT + o], sX[g * NIN + i], acc);
+      sDW[w] = acc;
+    }
+    return;
+  }
+  constexpr int kGroups = 32 / NIN;   // lanes per column
+  const int i = lane % NIN, og = lane / NIN;
+  for (int c = og; c < NOUT / 4; c += kGroups) {
+    float acc[4];
+#pragma unroll
+    for (int r = 0; r < 4; ++r) acc[r] = sDW[(4 * c + r) * NIN + i];
+#pragma unroll 8
+    for (int g = 0; g < 32; ++g) {
+      const float x = sX[g * NIN + i];
+      const float4 gg = *reinterpret_cast<const float4 *>(sG + g * NOUT + 4 * c);
+      acc[0] = fmaf(gg.x, x, acc[0]); acc[1] = fmaf(gg.y, x, acc[1]);
+      acc[2] = fmaf(gg.z, x, acc[2]); acc[3] = fmaf(gg.w, x, acc[3]);
+    }
+#pragma unroll
+    for (int r = 0; r < 4; ++r) sDW[(4 * c + r) * NIN + i] = acc[r];
   }
 }
 
@@ -275,7 +296,13 @@ int run_bwd(const AppearanceArgs &a, int nfeat, cudaStream_t st) {
   const size_t smem = sizeof(float) * ((1 + kVarWarps) * D::kNumW + kVarWarps * 2048);
   opt_in(k_variant_bwd<H, L>, smem);
   const int64_t chunks = (a.n + kVarBlock - 1) / kVarBlock;
-  const int blocks = (int)(chunks < kVarPartialBlocks ? chunks : kVarPartialBlocks);
+  // one full wave: as many CTAs as are resident at once
+  int per_sm = 0, sms = 0, dev = 0, wave = kVarPartialBlocks;
+  if (cudaGetDevice(&dev) == cudaSuccess &&
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_variant_bwd<H, L>, kVarBlock, smem) == cudaSuccess &&
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && per_sm > 0 && sms > 0)
+    wave = per_sm * sms < kVarPartialBlocks ? per_sm * sms : kVarPartialBlocks;
+  const int blocks = (int)(chunks < wave ? chunks : wave);
   k_variant_bwd<H, L><<<blocks, kVarBlock, smem, st>>>(a, nfeat);
   k_variant_wreduce<<<(D::kNumW + 127) / 128, 128, 0, st>>>(a.w_partials, blocks, D::kNumW, a.g_weights);
   return 2;
