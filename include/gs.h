@@ -70,7 +70,8 @@ typedef enum {
 
 /* Pinhole camera (host struct). */
 typedef struct {
-  int32_t width, height;        /* pixels                                                      */
+  int32_t width, height;        /* pixels; at most 65535 tiles of 16 pixels per axis and 2^24
+                                   tiles in all (GS_ERR_INVALID_ARG beyond)                    */
   float fx, fy, cx, cy;         /* intrinsics in pixel units                                   */
   float w2c[12];                /* row-major [R|t]: x_cam = R x_world + t                      */
   float near_plane, far_plane;  /* depth cull, typically 0.2 and 1e10                          */
@@ -79,7 +80,7 @@ typedef struct {
 
 /* The scene: per-Gaussian parameters plus the shared decoder (host struct of device pointers). */
 typedef struct {
-  int64_t n;                     /* number of Gaussians, >= 0                                  */
+  int64_t n;                     /* number of Gaussians, >= 0 and < 2^31 (GS_ERR_CAPACITY)     */
   const float *means;            /* [n,3]                                                      */
   const float *log_scales;       /* [n,3]   scale = exp(log_scale)                             */
   const float *quats;            /* [n,4]   (w,x,y,z), normalised inside                       */

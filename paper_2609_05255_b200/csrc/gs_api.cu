@@ -18,7 +18,8 @@ struct GsContext {
   unsigned long long *d_counter;      // device: [0] instance counter of the last gs_preprocess, [1] second word of
                                       // gs_profile_blend_counts, [2] set when a device-counted view overflowed its capacity
   unsigned long long *h_counter;      // pinned host mirror
-  float *d_w_partials;                // device: [kWgradBlocks, 816] decoder-gradient partial sums
+  float *d_w_partials;                // device: per-CTA partial sums of the decoder gradient ([kWgradBlocks, 816];
+                                      // sized for the decoder variants' largest case as well)
   char error[256];
   bool profiling;
   std::vector<StageRecord> records;   // stage timings since the last collect
@@ -69,7 +70,8 @@ struct StageTimer {
 bool camera_ok(const GsCamera *c) {
   if (!c || c->width <= 0 || c->height <= 0) return false;
   if (!(c->fx > 0.f) || !(c->fy > 0.f)) return false;
-  if ((c->width + GS_TILE - 1) / GS_TILE > 65535 || (c->height + GS_TILE - 1) / GS_TILE > 65535) return false;
+  const int64_t gx = (c->width + GS_TILE - 1) / GS_TILE, gy = (c->height + GS_TILE - 1) / GS_TILE;
+  if (gx > 65535 || gy > 65535 || gx * gy > ((int64_t)1 << 24)) return false;   // rect is u16; tile ids and grids stay small
   return true;
 }
 
@@ -106,6 +108,7 @@ GsStatus scene_appearance_ok(GsContext *ctx, const GsScene *s) {
   if (s->color_activation < GS_ACT_RELU || s->color_activation > GS_ACT_HARD_SIGMOID)
     return fail(ctx, GS_ERR_INVALID_ARG, "unknown colour activation");
   if (s->n < 0) return fail(ctx, GS_ERR_INVALID_ARG, "n < 0");
+  if (s->n >= ((int64_t)1 << 31)) return fail(ctx, GS_ERR_CAPACITY, "n must stay below 2^31 (32-bit Gaussian ids and grids)");
   if (s->app == GS_APP_NEURAL) {
     const DecoderArch d = decoder_arch(s);
     if ((d.hidden != 16 && d.hidden != 32) || d.layers < 1 || d.layers > 3 || (d.nfeat != 8 && d.nfeat != 16))
@@ -231,7 +234,7 @@ GsStatus preprocess_impl(GsContext *ctx, const GsScene *scene, const GsCamera *c
                          int64_t *num_pairs_host, void *stream) {
   GsStatus st = scene_ok(ctx, scene);
   if (st != GS_OK) return st;
-  if (!camera_ok(cam)) return fail(ctx, GS_ERR_INVALID_ARG, "bad camera (size, focal length or more than 65535 tiles per axis)");
+  if (!camera_ok(cam)) return fail(ctx, GS_ERR_INVALID_ARG, "bad camera (size, focal length, more than 65535 tiles per axis or more than 2^24 tiles)");
   if (!out) return fail(ctx, GS_ERR_INVALID_ARG, "out is NULL");
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   cudaSetDevice(ctx->device);
@@ -376,7 +379,6 @@ GsStatus gs_render_backward(GsContext *ctx, const GsScene *scene, const GsCamera
         bad_ptr(grads->opacity_logits) || bad_ptr(grads->base_color))
       return fail(ctx, GS_ERR_INVALID_ARG, "a gradient buffer is NULL or misaligned");
     if (scene->app == GS_APP_SH && bad_ptr(grads->sh_rest)) return fail(ctx, GS_ERR_INVALID_ARG, "grads->sh_rest is NULL or misaligned");
-  if (scene->app == GS_APP_SV && bad_ptr(grads->sv_sites)) return fail(ctx, GS_ERR_INVALID_ARG, "grads->sv_sites is NULL or misaligned");
     if (scene->app == GS_APP_SV && bad_ptr(grads->sv_sites)) return fail(ctx, GS_ERR_INVALID_ARG, "grads->sv_sites is NULL or misaligned");
     if (scene->app == GS_APP_NEURAL && bad_ptr(grads->features)) return fail(ctx, GS_ERR_INVALID_ARG, "grads->features is NULL or misaligned");
     if (bad_ptr(proj->mean2d) || bad_ptr(proj->conic_opacity) || bad_ptr(proj->color) || bad_ptr(proj->rect))

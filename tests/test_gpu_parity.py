@@ -323,6 +323,10 @@ def test_capacity_and_argument_errors():
     with pytest.raises(api.GsError) as e:
         api.gs_preprocess(ctx, ds, bad_cam, proj)
     assert e.value.status == api.GS_ERR_INVALID_ARG
+    huge = api.make_camera(cam); huge.width = 70_000; huge.height = 70_000      # 4375 x 4375 tiles > 2^24
+    with pytest.raises(api.GsError) as e:
+        api.gs_preprocess(ctx, ds, huge, proj)
+    assert e.value.status == api.GS_ERR_INVALID_ARG
     # the context is still usable afterwards
     api.gs_render_forward(ctx, ds.n, proj, ccam, P, P, binning, image, fT, nc, ws)
     torch.cuda.synchronize()
