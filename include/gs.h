@@ -156,9 +156,10 @@ typedef struct {
   float *sv_sites;        /* SV:     [n,7,7] with respect to the raw site parameters            */
 } GsGrads;
 
-/* Create / destroy a context on CUDA device `device`.  The context owns a few KB of device and
- * pinned host memory (counters, the decoder-gradient partial sums).  Not thread safe: use one
- * context per host thread.  Returns GS_ERR_CUDA if the device cannot be used. */
+/* Create / destroy a context on CUDA device `device`.  The context owns 32 bytes of counters
+ * (device and pinned host) and 7.5 MB of device memory for the per-CTA partial sums of the decoder
+ * gradient.  Not thread safe: use one context per host thread, and one per stream whose calls may
+ * overlap on the GPU.  Returns GS_ERR_CUDA if the device cannot be used. */
 GsStatus gs_create(int device, GsContext **ctx);
 void gs_destroy(GsContext *ctx);
 const char *gs_last_error(const GsContext *ctx);
