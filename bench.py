@@ -286,6 +286,7 @@ def run_ours(args):
     decode = None if (args.skip_decode or args.config != 3) else decode_sweep(api, torch, ctx, dev, peaks, args)
     adam = None if (args.skip_decode or args.config != 3) else adam_sweep(api, torch, ctx, dev, peaks, n)
     prepass = None if (args.skip_decode or args.config != 3) else prepass_sweep(api, torch, ctx, dev, peaks, args, scenes)
+    sort_ref = None if (args.skip_decode or args.config != 3) else sort_reference(torch, results[head], cams, views, dev)
 
     if rank != 0:
         return
@@ -327,6 +328,7 @@ def run_ours(args):
         "appearance_decode": decode,
         "adam_update": adam,
         "viewer_prepass": prepass,
+        "sort_reference": sort_ref,
         "peaks": peaks,
     }
     if not args.skip_cpu:
@@ -539,6 +541,38 @@ def measure_e2e_training(api, torch, lane_ctx, lanes, arm, cams, G, views, args,
             "what": "upstream gradients in, rendered images out, parameters stay on the device and are updated by Adam; "
                     "two buffer sets, so one step's copies overlap the next step's kernels",
             "streams": L, "parameters_finite_after_run": finite}
+
+
+def sort_reference(torch, arm, cams, views, dev):
+    """Context for the ordering stages: the library's stable sort of one view's instance list as 64-bit
+    (tile, depth bits) keys with the Gaussian ids as values - the one-key formulation - timed as a library
+    call beside this library's two-stage ordering (depth sort of the Gaussians + tile sort of the instances)."""
+    r = arm["r"]
+    r.forward(arm["ds"], cams[0])      # view 0's lists, with the host-side count
+    torch.cuda.synchronize()
+    P = int(r.num_pairs)
+    tiles = r.binning.sorted_tiles[:P].to(torch.int64)
+    vals = r.binning.sorted_vals[:P].to(torch.int64)
+    depth = r.proj.depth_key.view(torch.int32).to(torch.int64) & 0xffffffff
+    keys = (tiles << 32) | depth[vals]
+    gen = torch.Generator(device=dev); gen.manual_seed(9)
+    perm = torch.randperm(P, device=dev, generator=gen)
+    keys, vals = keys[perm].contiguous(), vals[perm].to(torch.int32).contiguous()
+    ts = []
+    for i in range(8):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        sk, order = torch.sort(keys, stable=True)
+        sv = vals[order]
+        e1.record()
+        torch.cuda.synchronize()
+        if i >= 3:
+            ts.append(e0.elapsed_time(e1))
+    ts.sort()
+    ours = (arm["stage_ms"]["depth_sort"] + arm["stage_ms"]["tile_sort"]) / views
+    return {"instances": P, "library_sort_64bit_keys_ms": round(ts[len(ts) // 2], 4),
+            "two_stage_ordering_ms_per_view": round(ours, 4),
+            "what": "torch.sort(stable) of (tile << 32 | depth bits) keys + gather of the ids, against depth_sort + tile_sort of one view"}
 
 
 def adam_sweep(api, torch, ctx, dev, peaks, n):
