@@ -107,9 +107,18 @@ typedef struct {
                                     decoder of the architecture table (App. D): mlp_weights then holds
                                     W_1[hidden][32], (layers - 1) x [hidden][hidden], W_out[3][hidden],
                                     32 hidden + (layers - 1) hidden^2 + 3 hidden values.  Anything but
-                                    the default 16 / 2 / 8 is served by gs_appearance_forward and
-                                    gs_appearance_backward only (plain fp32 kernels); every other entry
-                                    point returns GS_ERR_UNSUPPORTED for it                        */
+                                    the default 16 / 2 / 8 runs on plain fp32 kernels and, in the
+                                    rendering step, always through the separate-pass path below;
+                                    gs_neural_fold, gs_neural_prepass and
+                                    gs_appearance_backward_noalloc return GS_ERR_UNSUPPORTED for it */
+  int32_t separate_pass;         /* 0: appearance fused into the preprocess kernels (Sec. 4 "CUDA
+                                    Implementation").  1: the unfused reference path of Sec. 4 / App. D
+                                    "Fusion": gs_preprocess leaves the view directions of the visible
+                                    Gaussians in GsProjected.color and a separate appearance pass turns
+                                    them into colours in place; gs_render_backward runs the appearance
+                                    backward as a pass of its own between the blend backward and the
+                                    projection backward, exchanging directions, dL/dcolor and dL/dd
+                                    through the workspace.  Same results up to rounding             */
 } GsScene;
 
 /* Per-Gaussian results of gs_preprocess (caller-allocated device buffers). */

@@ -224,7 +224,16 @@ def _app_args(scene):
     return _f64(scene.base_color), sh, ft, wt
 
 
+def _is_variant(scene) -> bool:
+    return scene.app == 1 and decoder_arch(scene) != (16, 2, 8)
+
+
 def appearance_forward(scene, dirs, mask=None, deg=None):
+    if _is_variant(scene):      # a decoder of another size: the generic decoder, masked rows left at zero
+        keep = np.ones(len(dirs), bool) if mask is None else np.asarray(mask) > 0
+        color = np.zeros((len(dirs), 3))
+        color[keep] = decoder_forward(scene_rows(scene, keep), _f64(dirs)[keep], deg)
+        return color, np.zeros((len(dirs), 3))
     base, sh, ft, wt = _app_args(scene)
     dirs = _f64(dirs); n = dirs.shape[0]
     color, resid = np.zeros((n, 3)), np.zeros((n, 3))
@@ -235,7 +244,24 @@ def appearance_forward(scene, dirs, mask=None, deg=None):
     return color, resid
 
 
+def scene_rows(scene, keep):
+    """The appearance parameters of the Gaussians selected by the boolean array `keep` (decoder shared)."""
+    return SimpleNamespace(app=scene.app, active_degree=scene.active_degree, base_color=np.asarray(scene.base_color)[keep],
+                           features=np.asarray(scene.features)[keep], mlp_weights=scene.mlp_weights,
+                           mlp_hidden=getattr(scene, "mlp_hidden", 0), mlp_layers=getattr(scene, "mlp_layers", 0),
+                           color_activation=_act(scene))
+
+
 def appearance_backward(scene, dirs, g_color, mask=None, deg=None):
+    if _is_variant(scene):
+        n = len(dirs)
+        keep = np.ones(n, bool) if mask is None else np.asarray(mask) > 0
+        g = decoder_backward(scene_rows(scene, keep), _f64(dirs)[keep], _f64(g_color)[keep], deg)
+        nfeat = scene.features.shape[1]
+        o = SimpleNamespace(base_color=np.zeros((n, 3)), dirs=np.zeros((n, 3)), sh_rest=None, sv_sites=None,
+                            features=np.zeros((n, nfeat)), mlp_weights=g.mlp_weights)
+        o.base_color[keep], o.dirs[keep], o.features[keep] = g.base_color, g.dirs, g.features
+        return o
     base, sh, ft, wt = _app_args(scene)
     dirs, g_color = _f64(dirs), _f64(g_color); n = dirs.shape[0]
     deg = scene.active_degree if deg is None else deg

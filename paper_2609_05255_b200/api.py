@@ -40,7 +40,8 @@ class GsScene(C.Structure):
     _fields_ = [("n", C.c_int64), ("means", _vp), ("log_scales", _vp), ("quats", _vp), ("opacity_logits", _vp),
                 ("base_color", _vp), ("app", C.c_int32), ("active_degree", C.c_int32), ("sh_rest", _vp),
                 ("features", _vp), ("mlp_weights", _vp), ("color_activation", C.c_int32), ("sv_sites", _vp),
-                ("mlp_hidden", C.c_int32), ("mlp_layers", C.c_int32), ("num_features", C.c_int32)]
+                ("mlp_hidden", C.c_int32), ("mlp_layers", C.c_int32), ("num_features", C.c_int32),
+                ("separate_pass", C.c_int32)]
 
 
 class GsProjected(C.Structure):
@@ -164,6 +165,7 @@ class DeviceScene:
     mlp_hidden: int = 16             # decoder architecture (App. D); anything but 16 / 2 / 8 runs in
     mlp_layers: int = 2              # gs_appearance_forward / backward only
     num_features: int = 8
+    separate_pass: int = 0           # 1: the unfused reference path (appearance as passes of its own)
 
     @property
     def n(self) -> int:
@@ -179,6 +181,7 @@ class DeviceScene:
         s.color_activation = int(self.color_activation)
         s.sv_sites = _ptr(self.sv_sites)
         s.mlp_hidden, s.mlp_layers, s.num_features = int(self.mlp_hidden), int(self.mlp_layers), int(self.num_features)
+        s.separate_pass = int(self.separate_pass)
         return s
 
 
@@ -193,7 +196,8 @@ def upload_scene(scene, device="cuda") -> DeviceScene:
                        up(scene.mlp_weights, torch.float16), int(getattr(scene, "color_activation", 0)),
                        up(getattr(scene, "sv_sites", None), torch.float32),
                        int(getattr(scene, "mlp_hidden", 0)) or 16, int(getattr(scene, "mlp_layers", 0)) or 2,
-                       int(scene.features.shape[1]) if scene.features is not None else 8)
+                       int(scene.features.shape[1]) if scene.features is not None else 8,
+                       int(getattr(scene, "separate_pass", 0)))
 
 
 @dataclass
@@ -286,6 +290,12 @@ def alloc_grads(n: int, app: int, device, num_features: int = 8, num_weights: in
         g.features = torch.empty((m, num_features), **f)
         g.mlp_weights = torch.empty((num_weights,), **f)
     return g
+
+
+def alloc_grads_for(scene: DeviceScene, device) -> Grads:
+    """Gradient buffers shaped for the scene's appearance model and decoder."""
+    return alloc_grads(scene.n, scene.app, device, scene.num_features,
+                       decoder_num_weights(scene.mlp_hidden, scene.mlp_layers))
 
 
 class Context:

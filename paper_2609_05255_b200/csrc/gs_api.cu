@@ -101,6 +101,26 @@ bool default_decoder(const GsScene *s) {
   const DecoderArch d = decoder_arch(s);
   return s->app != GS_APP_NEURAL || (d.hidden == 16 && d.layers == 2 && d.nfeat == 8);
 }
+// The rendering step with the appearance as passes of its own (asked for, or the only way for a decoder variant).
+bool unfused(const GsScene *s) { return s->separate_pass != 0 || !default_decoder(s); }
+
+AppearanceArgs appearance_args(const GsScene *scene) {
+  AppearanceArgs a;
+  memset(&a, 0, sizeof(a));
+  a.n = scene->n; a.deg = scene->active_degree; a.act = scene->color_activation;
+  a.base_color = scene->base_color; a.sh_rest = scene->app == GS_APP_SV ? scene->sv_sites : scene->sh_rest;
+  a.features = reinterpret_cast<const __half *>(scene->features);
+  a.weights = reinterpret_cast<const __half *>(scene->mlp_weights);
+  return a;
+}
+int run_appearance_fwd(const GsScene *scene, const AppearanceArgs &a, cudaStream_t s) {
+  const DecoderArch d = decoder_arch(scene);
+  return default_decoder(scene) ? launch_appearance_fwd(scene->app, a, s) : launch_variant_fwd(d.hidden, d.layers, d.nfeat, a, s);
+}
+int run_appearance_bwd(const GsScene *scene, const AppearanceArgs &a, cudaStream_t s) {
+  const DecoderArch d = decoder_arch(scene);
+  return default_decoder(scene) ? launch_appearance_bwd(scene->app, a, s) : launch_variant_bwd(d.hidden, d.layers, d.nfeat, a, s);
+}
 
 GsStatus scene_appearance_ok(GsContext *ctx, const GsScene *s) {
   if (s->app != GS_APP_SH && s->app != GS_APP_NEURAL && s->app != GS_APP_SV) return fail(ctx, GS_ERR_INVALID_ARG, "unknown appearance model");
@@ -127,8 +147,6 @@ GsStatus scene_ok(GsContext *ctx, const GsScene *s) {
   if (!s) return fail(ctx, GS_ERR_INVALID_ARG, "scene is NULL");
   GsStatus st = scene_appearance_ok(ctx, s);
   if (st != GS_OK) return st;
-  if (!default_decoder(s))
-    return fail(ctx, GS_ERR_UNSUPPORTED, "only the 16 / 2 / 8 decoder is fused into the rendering step; the variants run in gs_appearance_forward / backward");
   if (s->n > 0 && (bad_ptr(s->means) || bad_ptr(s->log_scales) || bad_ptr(s->quats) || bad_ptr(s->opacity_logits)))
     return fail(ctx, GS_ERR_INVALID_ARG, "a geometry array is NULL or misaligned");
   return GS_OK;
@@ -173,7 +191,21 @@ FwdWorkspace carve_fwd(void *ws, int64_t n, int64_t cap) {
   return w;
 }
 
-size_t bwd_bytes(int64_t n) { return align_up((size_t)(n > 0 ? n : 1) * 12 * sizeof(float)); }
+// Backward scratch: the 2D gradients [n,12], then (used by the separate-pass path only) directions, dL/dcolor and
+// dL/dd as [n,3] each.
+struct BwdWorkspace { float *g2d, *dirs, *g_color, *g_dirs; size_t bytes; };
+BwdWorkspace carve_bwd(void *ws, int64_t n) {
+  Carver c{static_cast<char *>(ws), 0};
+  const size_t nn = (size_t)(n > 0 ? n : 1);
+  BwdWorkspace w;
+  w.g2d = c.take<float>(nn * 12);
+  w.dirs = c.take<float>(nn * 3);
+  w.g_color = c.take<float>(nn * 3);
+  w.g_dirs = c.take<float>(nn * 3);
+  w.bytes = c.used;
+  return w;
+}
+size_t bwd_bytes(int64_t n) { return carve_bwd(nullptr, n).bytes; }
 
 int tile_bits(int num_tiles) {
   int bits = 1;
@@ -256,7 +288,13 @@ GsStatus preprocess_impl(GsContext *ctx, const GsScene *scene, const GsCamera *c
   a.pair_counter = ctx->d_counter;
   {
     StageTimer t(ctx, GS_STAGE_PREPROCESS_FWD, s);
-    t.done(launch_preprocess_fwd(scene->app, a, make_cam(cam), s));
+    t.done(launch_preprocess_fwd(unfused(scene) ? kAppExternal : scene->app, a, make_cam(cam), s));
+  }
+  if (unfused(scene)) {   // directions sit in out->color: decode them in place, visible Gaussians only
+    AppearanceArgs ap = appearance_args(scene);
+    ap.dirs = out->color; ap.color = out->color; ap.mask = out->tiles_touched;
+    StageTimer t(ctx, GS_STAGE_APPEARANCE_FWD, s);
+    t.done(run_appearance_fwd(scene, ap, s));
   }
   if ((st = check_cuda(ctx, cudaGetLastError(), "preprocess launch")) != GS_OK) return st;
   if (!num_pairs_host) return GS_OK;
@@ -390,7 +428,10 @@ GsStatus gs_render_backward(GsContext *ctx, const GsScene *scene, const GsCamera
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   cudaSetDevice(ctx->device);
   const CamDev cd = make_cam(cam);
-  float *g2d = static_cast<float *>(workspace);
+  const BwdWorkspace bw = carve_bwd(workspace, n);
+  float *g2d = bw.g2d;
+  const bool ext = unfused(scene);
+  if (ext && n > 0 && bad_ptr(proj->tiles_touched)) return fail(ctx, GS_ERR_INVALID_ARG, "proj->tiles_touched is NULL or misaligned");
   if (n > 0) {
     if ((st = check_cuda(ctx, cudaMemsetAsync(g2d, 0, (size_t)n * 12 * sizeof(float), s), "memset")) != GS_OK) return st;
     if (num_pairs > 0) {
@@ -411,11 +452,24 @@ GsStatus gs_render_backward(GsContext *ctx, const GsScene *scene, const GsCamera
   a.g_logits = grads->opacity_logits; a.g_base = grads->base_color;
   a.g_sh_rest = scene->app == GS_APP_SV ? grads->sv_sites : grads->sh_rest;
   a.g_features = grads->features; a.w_partials = ctx->d_w_partials; a.g_weights = grads->mlp_weights;
-  if (n == 0 && scene->app == GS_APP_NEURAL)
-    return check_cuda(ctx, cudaMemsetAsync(grads->mlp_weights, 0, sizeof(float) * GS_MLP_WEIGHTS, s), "memset");
+  a.gd_in = bw.g_dirs;
+  if (n == 0 && scene->app == GS_APP_NEURAL) {
+    const DecoderArch d = decoder_arch(scene);
+    return check_cuda(ctx, cudaMemsetAsync(grads->mlp_weights, 0, sizeof(float) * variant_num_weights(d.hidden, d.layers), s), "memset");
+  }
+  if (ext && n > 0) {   // the appearance backward as a pass of its own, through dense arrays in the workspace
+    AppearanceArgs ap = appearance_args(scene);
+    ap.dirs = bw.dirs; ap.g_color = bw.g_color; ap.mask = proj->tiles_touched;
+    ap.g_base = grads->base_color; ap.g_sh_rest = scene->app == GS_APP_SV ? grads->sv_sites : grads->sh_rest;
+    ap.g_features = grads->features; ap.g_dirs = bw.g_dirs;
+    ap.w_partials = ctx->d_w_partials; ap.g_weights = grads->mlp_weights;
+    StageTimer t(ctx, GS_STAGE_APPEARANCE_BWD, s);
+    t.done(launch_unfused_prepare(n, scene->means, cd, g2d, proj->tiles_touched, bw.dirs, bw.g_color, s) +
+           run_appearance_bwd(scene, ap, s));
+  }
   {
     StageTimer t(ctx, GS_STAGE_PREPROCESS_BWD, s);
-    t.done(launch_preprocess_bwd(scene->app, a, cd, s));
+    t.done(launch_preprocess_bwd(ext ? kAppExternal : scene->app, a, cd, s));
   }
   return check_cuda(ctx, cudaGetLastError(), "render_backward launch");
 }
@@ -437,9 +491,7 @@ GsStatus gs_appearance_forward(GsContext *ctx, const GsScene *scene, const float
   a.color = color;
   {
     StageTimer t(ctx, GS_STAGE_APPEARANCE_FWD, static_cast<cudaStream_t>(stream));
-    const DecoderArch d = decoder_arch(scene);
-    t.done(default_decoder(scene) ? launch_appearance_fwd(scene->app, a, static_cast<cudaStream_t>(stream))
-                                  : launch_variant_fwd(d.hidden, d.layers, d.nfeat, a, static_cast<cudaStream_t>(stream)));
+    t.done(run_appearance_fwd(scene, a, static_cast<cudaStream_t>(stream)));
   }
   return check_cuda(ctx, cudaGetLastError(), "appearance_forward launch");
 }
@@ -478,8 +530,7 @@ GsStatus gs_appearance_backward(GsContext *ctx, const GsScene *scene, const floa
   a.w_partials = ctx->d_w_partials; a.g_weights = grads->mlp_weights;
   {
     StageTimer t(ctx, GS_STAGE_APPEARANCE_BWD, s);
-    const DecoderArch d = decoder_arch(scene);
-    t.done(default_decoder(scene) ? launch_appearance_bwd(scene->app, a, s) : launch_variant_bwd(d.hidden, d.layers, d.nfeat, a, s));
+    t.done(run_appearance_bwd(scene, a, s));
   }
   return check_cuda(ctx, cudaGetLastError(), "appearance_backward launch");
 }

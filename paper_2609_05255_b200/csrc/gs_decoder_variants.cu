@@ -104,7 +104,7 @@ __global__ void __launch_bounds__(kVarBlock) k_variant_fwd(AppearanceArgs a, int
   for (int k = threadIdx.x; k < VarDims<H, L>::kNumW; k += kVarBlock) sW[k] = __half2float(a.weights[k]);
   __syncthreads();
   const int64_t i = (int64_t)blockIdx.x * kVarBlock + threadIdx.x;
-  if (i >= a.n) return;
+  if (i >= a.n || (a.mask && __ldg(a.mask + i) == 0u)) return;   // masked-out Gaussians are skipped
   float d[3], base[3];
   d[0] = __ldg(a.dirs + 3 * i); d[1] = __ldg(a.dirs + 3 * i + 1); d[2] = __ldg(a.dirs + 3 * i + 2);
   base[0] = __ldg(a.base_color + 3 * i); base[1] = __ldg(a.base_color + 3 * i + 1); base[2] = __ldg(a.base_color + 3 * i + 2);
@@ -168,7 +168,8 @@ __global__ void __launch_bounds__(kVarBlock) k_variant_bwd(AppearanceArgs a, int
   const int64_t nchunks = (a.n + kVarBlock - 1) / kVarBlock;
   for (int64_t chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x) {
     const int64_t i = chunk * kVarBlock + tid;
-    const bool in = i < a.n;
+    const bool exists = i < a.n;
+    const bool in = exists && (!a.mask || __ldg(a.mask + i) != 0u);   // masked out: zero gradient rows
     float d[3] = {0.f, 0.f, 1.f}, base[3] = {0.f, 0.f, 0.f}, gcol[3] = {0.f, 0.f, 0.f};
     if (in) {
 #pragma unroll
@@ -232,12 +233,12 @@ __global__ void __launch_bounds__(kVarBlock) k_variant_bwd(AppearanceArgs a, int
       warp_weight_grad<H, 32>(sX, sG, sDW, lane);
       matvec_t<H, 32>(sW, g_hi, gx);
     }
-    if (in) {
+    if (exists) {
       a.g_base[3 * i] = gp[0]; a.g_base[3 * i + 1] = gp[1]; a.g_base[3 * i + 2] = gp[2];
       // features
       if (nfeat == 8) {
         float gf[8];
-        if (a.deg > 0) {
+        if (a.deg > 0 && in) {
           float x[32];
           variant_inputs(a, i, nfeat, d, x);
 #pragma unroll

@@ -30,6 +30,11 @@ struct CamDev {
 
 // ---- launches (all enqueue on `st`; none synchronises; each returns the number of kernels it
 // launched) ---------------------------------------------------------------------------------
+// Appearance "model" of the preprocess kernels in the separate-pass (unfused) step: no colour is decoded; the
+// forward leaves the view directions of the visible Gaussians where the colours go, the backward takes dL/dd
+// from a buffer.  The appearance kernels run as launches of their own around them.
+constexpr int kAppExternal = 3;
+
 struct PreprocessArgs {
   int64_t n;
   const float *means, *log_scales, *quats, *logits, *base_color, *sh_rest;
@@ -49,6 +54,7 @@ struct PreprocessBwdArgs {
   int deg, act;
   const uint16_t *rect;
   const float *g2d;            // [n,12]: dL/dcolor(3), dL/dopacity, dL/dconic(3), dL/dmean2d(2), pad
+  const float *gd_in;          // kAppExternal only: [n,3] dL/dd from the separate appearance backward
   float *g_means, *g_log_scales, *g_quats, *g_logits, *g_base, *g_sh_rest, *g_features;
   float *w_partials;           // [kWgradBlocks, 816]
   float *g_weights;            // [816]
@@ -64,6 +70,8 @@ struct AppearanceArgs {
   const float *g_color;        // backward
   float *g_base, *g_sh_rest, *g_features, *g_dirs;
   float *w_partials, *g_weights;
+  const uint32_t *mask;        // optional [n]: Gaussians with a zero here are skipped (no colour written; zero
+                               // gradient rows written); the tiles-touched array in the unfused step
 };
 int launch_appearance_fwd(int app, const AppearanceArgs &a, cudaStream_t st);
 int launch_appearance_bwd(int app, const AppearanceArgs &a, cudaStream_t st);
@@ -73,6 +81,11 @@ int variant_num_weights(int hidden, int layers);
 size_t variant_partials_floats();   // floats of per-block weight-gradient partials the backward needs
 int launch_variant_fwd(int hidden, int layers, int nfeat, const AppearanceArgs &a, cudaStream_t st);
 int launch_variant_bwd(int hidden, int layers, int nfeat, const AppearanceArgs &a, cudaStream_t st);
+
+// Unfused step, backward: view directions of the masked-in Gaussians and their dL/dcolor (columns 0..2 of the
+// [n,12] rows) as dense [n,3] arrays for the separate appearance backward.
+int launch_unfused_prepare(int64_t n, const float *means, const CamDev &cam, const float *g2d, const uint32_t *mask,
+                           float *dirs, float *g_color, cudaStream_t st);
 
 constexpr int kWgradBlocks = 592;   // persistent blocks of the decoder-gradient kernels (4 x 148)
 

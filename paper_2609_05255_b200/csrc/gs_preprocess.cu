@@ -20,6 +20,7 @@ constexpr int kWarps = kBlock / 32;
 // warp's shared-memory slab of 32 rows meets no bank conflict.
 template <int APP> struct RowOf { static constexpr int value = APP == GS_APP_SV ? GS_SV_ROW : GS_SH_REST; };
 template <int APP> struct SlabOf { static constexpr int value = 32 * RowOf<APP>::value; };
+template <int APP> struct Explicit { static constexpr bool value = APP == GS_APP_SH || APP == GS_APP_SV; };
 constexpr unsigned kFull = 0xffffffffu;
 
 __device__ __forceinline__ bool finite_f(float x) { return fabsf(x) <= FLT_MAX; }
@@ -407,7 +408,7 @@ __device__ __forceinline__ void load3(const float *p, int64_t i, float v[3]) {
 
 template <int APP>
 __global__ void __launch_bounds__(kBlock) k_preprocess_fwd(PreprocessArgs a, CamDev cam) {
-  __shared__ __align__(16) float sData[APP != GS_APP_NEURAL ? kWarps * SlabOf<APP>::value : 4];
+  __shared__ __align__(16) float sData[Explicit<APP>::value ? kWarps * SlabOf<APP>::value : 4];
   __shared__ __align__(16) unsigned char sNN[APP == GS_APP_NEURAL ? sizeof(mlp::Weights) + kWarps * sizeof(StageFwd) : 16];
   mlp::Weights *sWt = reinterpret_cast<mlp::Weights *>(sNN);
   StageFwd *sStage = reinterpret_cast<StageFwd *>(sNN + (APP == GS_APP_NEURAL ? sizeof(mlp::Weights) : 0));   // unused for SH
@@ -443,7 +444,7 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_fwd(PreprocessArgs a, Cam
   }
   // ---- fused colour decode for the Gaussians that survived culling
   float pre[3] = {0.f, 0.f, 0.f};
-  if (APP != GS_APP_NEURAL) {   // SH or Spherical Voronoi: parameter rows through the warp's slab
+  if (Explicit<APP>::value) {   // SH or Spherical Voronoi: parameter rows through the warp's slab
     float *slab = sData + warp * SlabOf<APP>::value;
     if (__any_sync(kFull, vis) && a.deg > 0 && row0 < a.n) warp_load_rows<RowOf<APP>::value>(a.sh_rest, row0, a.n, slab, lane);
     if (vis) {
@@ -452,7 +453,7 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_fwd(PreprocessArgs a, Cam
       SvCarry cy;
       explicit_pre<APP>(slab + lane * RowOf<APP>::value, base, g.dirx, g.diry, g.dirz, a.deg, pre, cy);
     }
-  } else {
+  } else if (APP == GS_APP_NEURAL) {
     float A[3] = {0.f, 0.f, 0.f};
     if (a.deg > 0 && __any_sync(kFull, vis)) {   // the whole warp decodes; culled lanes feed zeros
       float x[32];
@@ -480,7 +481,11 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_fwd(PreprocessArgs a, Cam
       reinterpret_cast<float4 *>(a.conic_opacity)[i] = make_float4(g.A, g.B, g.C, g.o);
     }
     if (vis) {
-      a.color[3 * i] = color_act_z(a.act, pre[0]); a.color[3 * i + 1] = color_act_z(a.act, pre[1]); a.color[3 * i + 2] = color_act_z(a.act, pre[2]);
+      if (APP == kAppExternal) {   // the separate appearance pass reads the direction here and writes the colour over it
+        a.color[3 * i] = g.dirx; a.color[3 * i + 1] = g.diry; a.color[3 * i + 2] = g.dirz;
+      } else {
+        a.color[3 * i] = color_act_z(a.act, pre[0]); a.color[3 * i + 1] = color_act_z(a.act, pre[1]); a.color[3 * i + 2] = color_act_z(a.act, pre[2]);
+      }
     }
     a.depth_key[i] = vis ? g.zbits : 0xffffffffu;
     a.tiles_touched[i] = tiles;
@@ -655,7 +660,8 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_bwd(PreprocessBwdArgs a, 
       logit = __ldg(a.logits + i);
       const float4 *g2 = reinterpret_cast<const float4 *>(a.g2d) + 3 * i;
       ga = g2[0]; gb = g2[1]; gc = g2[2];   // (gr, gg, gb, go) (gA, gB, gC, gu) (gv, -, -, -)
-      load3(a.base_color, i, base_in);
+      if (APP != kAppExternal) load3(a.base_color, i, base_in);
+      else load3(a.gd_in, i, gd);
       if (APP == GS_APP_NEURAL) feat_raw = __ldg(reinterpret_cast<const uint4 *>(a.features) + i);
       q[0] = q4.x; q[1] = q4.y; q[2] = q4.z; q[3] = q4.w;
       vis = rc.z > rc.x && rc.w > rc.y;
@@ -668,7 +674,9 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_bwd(PreprocessBwdArgs a, 
     }
     // ---- appearance backward
     float gp[3] = {0.f, 0.f, 0.f};
-    if (APP != GS_APP_NEURAL) {
+    if (APP == kAppExternal) {
+      // dL/dd came from the separate appearance backward (zero rows for culled Gaussians)
+    } else if (Explicit<APP>::value) {
       if (row0 < a.n) {
         if (warp_vis && a.deg > 0) {
           warp_load_rows<RowOf<APP>::value>(a.sh_rest, row0, a.n, slab, lane);
@@ -731,7 +739,7 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_bwd(PreprocessBwdArgs a, 
       store3(a.g_log_scales, i, gg.ls[0], gg.ls[1], gg.ls[2]);
       reinterpret_cast<float4 *>(a.g_quats)[i] = make_float4(gg.q[0], gg.q[1], gg.q[2], gg.q[3]);
       a.g_logits[i] = gg.logit;
-      store3(a.g_base, i, gp[0], gp[1], gp[2]);
+      if (APP != kAppExternal) store3(a.g_base, i, gp[0], gp[1], gp[2]);
     }
   }
   if (APP == GS_APP_NEURAL) {
@@ -753,7 +761,7 @@ __global__ void __launch_bounds__(kBlock) k_appearance_fwd(AppearanceArgs a) {
   }
   const int64_t i = (int64_t)blockIdx.x * kBlock + tid;
   const int64_t row0 = (int64_t)blockIdx.x * kBlock + warp * 32;
-  const bool in = i < a.n;
+  const bool in = i < a.n && (!a.mask || __ldg(a.mask + i) != 0u);   // masked-out Gaussians are skipped
   float d[3] = {0.f, 0.f, 1.f}, base[3] = {0.f, 0.f, 0.f}, pre[3];
   if (in) { load3(a.dirs, i, d); load3(a.base_color, i, base); }
   if (APP != GS_APP_NEURAL) {
@@ -800,7 +808,8 @@ __global__ void __launch_bounds__(kBlock) k_appearance_bwd(AppearanceArgs a) {
     reload_fence();
     const int64_t i = chunk * kBlock + tid;
     const int64_t row0 = chunk * kBlock + warp * 32;
-    const bool in = i < a.n;
+    const bool exists = i < a.n;
+    const bool in = exists && (!a.mask || __ldg(a.mask + i) != 0u);   // masked out: zero gradient rows
     float d[3] = {0.f, 0.f, 1.f}, base[3] = {0.f, 0.f, 0.f}, gcol[3] = {0.f, 0.f, 0.f};
     if (in) { load3(a.dirs, i, d); load3(a.base_color, i, base); load3(a.g_color, i, gcol); }
     float gp[3] = {0.f, 0.f, 0.f}, gd[3] = {0.f, 0.f, 0.f};
@@ -816,6 +825,9 @@ __global__ void __launch_bounds__(kBlock) k_appearance_bwd(AppearanceArgs a) {
 #pragma unroll
           for (int c = 0; c < 3; ++c) gp[c] = color_act_grad_z(a.act, pre[c]) * gcol[c];
           explicit_bwd<APP>(row, gp, d[0], d[1], d[2], a.deg, cy, gd);
+        } else if (exists) {
+#pragma unroll
+          for (int k = 0; k < RowOf<APP>::value; ++k) row[k] = 0.f;
         }
         warp_store_rows<RowOf<APP>::value>(a.g_sh_rest, row0, a.n, slab, lane);
       }
@@ -836,13 +848,13 @@ __global__ void __launch_bounds__(kBlock) k_appearance_bwd(AppearanceArgs a) {
 #pragma unroll
         for (int c = 0; c < 3; ++c) gp[c] = color_act_grad_z(a.act, base[c] + 0.5f) * gcol[c];
       }
-      if (in) {
+      if (exists) {
         float4 *gfp = reinterpret_cast<float4 *>(a.g_features) + 2 * i;
         gfp[0] = make_float4(gf[0], gf[1], gf[2], gf[3]);
         gfp[1] = make_float4(gf[4], gf[5], gf[6], gf[7]);
       }
     }
-    if (in) {
+    if (exists) {
       store3(a.g_base, i, gp[0], gp[1], gp[2]);
       store3(a.g_dirs, i, gd[0], gd[1], gd[2]);
     }
@@ -850,6 +862,26 @@ __global__ void __launch_bounds__(kBlock) k_appearance_bwd(AppearanceArgs a) {
   if (APP == GS_APP_NEURAL) {
     weight_grad_flush(dW, reinterpret_cast<float *>(sStage), a.w_partials + (size_t)blockIdx.x * GS_MLP_WEIGHTS, tid);
   }
+}
+
+// Unfused step, backward: what the separate appearance backward reads, as dense arrays.
+__global__ void __launch_bounds__(kBlock) k_unfused_prepare(int64_t n, const float *__restrict__ means, CamDev cam,
+                                                            const float *__restrict__ g2d, const uint32_t *__restrict__ mask,
+                                                            float *__restrict__ dirs, float *__restrict__ g_color) {
+  const int64_t i = (int64_t)blockIdx.x * kBlock + threadIdx.x;
+  if (i >= n) return;
+  float d[3] = {0.f, 0.f, 1.f}, g[3] = {0.f, 0.f, 0.f};
+  if (__ldg(mask + i) != 0u) {
+    float mu[3];
+    load3(means, i, mu);
+    const float vx = mu[0] - cam.oc[0], vy = mu[1] - cam.oc[1], vz = mu[2] - cam.oc[2];
+    const float vi = rsqrtf(vx * vx + vy * vy + vz * vz);
+    d[0] = vx * vi; d[1] = vy * vi; d[2] = vz * vi;
+    const float4 ga = __ldg(reinterpret_cast<const float4 *>(g2d) + 3 * i);
+    g[0] = ga.x; g[1] = ga.y; g[2] = ga.z;
+  }
+  store3(dirs, i, d[0], d[1], d[2]);
+  store3(g_color, i, g[0], g[1], g[2]);
 }
 
 inline int grid_for(int64_t n) { return (int)((n + kBlock - 1) / kBlock); }
@@ -883,7 +915,15 @@ int launch_preprocess_fwd(int app, const PreprocessArgs &a, const CamDev &cam, c
   if (a.n == 0) return 0;
   if (app == GS_APP_SH) k_preprocess_fwd<GS_APP_SH><<<grid_for(a.n), kBlock, 0, st>>>(a, cam);
   else if (app == GS_APP_SV) k_preprocess_fwd<GS_APP_SV><<<grid_for(a.n), kBlock, 0, st>>>(a, cam);
+  else if (app == kAppExternal) k_preprocess_fwd<kAppExternal><<<grid_for(a.n), kBlock, 0, st>>>(a, cam);
   else k_preprocess_fwd<GS_APP_NEURAL><<<grid_for(a.n), kBlock, 0, st>>>(a, cam);
+  return 1;
+}
+
+int launch_unfused_prepare(int64_t n, const float *means, const CamDev &cam, const float *g2d, const uint32_t *mask,
+                           float *dirs, float *g_color, cudaStream_t st) {
+  if (n == 0) return 0;
+  k_unfused_prepare<<<grid_for(n), kBlock, 0, st>>>(n, means, cam, g2d, mask, dirs, g_color);
   return 1;
 }
 
@@ -897,6 +937,10 @@ int launch_preprocess_bwd(int app, const PreprocessBwdArgs &a, const CamDev &cam
     if (a.n == 0) return 0;
     opt_in_smem(k_preprocess_bwd<GS_APP_SV>, kBwdSmemSV);
     k_preprocess_bwd<GS_APP_SV><<<grid_for(a.n), kBlock, kBwdSmemSV, st>>>(a, cam);
+    return 1;
+  } else if (app == kAppExternal) {
+    if (a.n == 0) return 0;
+    k_preprocess_bwd<kAppExternal><<<grid_for(a.n), kBlock, 16, st>>>(a, cam);
     return 1;
   } else {
     opt_in_smem(k_preprocess_bwd<GS_APP_NEURAL>, kBwdSmemNN);

@@ -61,6 +61,7 @@ class Scene:
     sv_sites: Optional[np.ndarray] = None     # [n,7,7] f32: per site (a_r, a_g, a_b, s_x, s_y, s_z, log tau)
     mlp_hidden: int = 0                       # decoder variant: neurons per hidden layer (0 = the default 16)
     mlp_layers: int = 0                       # decoder variant: hidden layers (0 = the default 2)
+    separate_pass: int = 0                    # 1: ask the library for its unfused reference path (same results)
 
     @property
     def n(self) -> int:

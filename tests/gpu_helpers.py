@@ -68,7 +68,7 @@ def run_gpu(scene, cam, G=None, pair_capacity=None, with_extent=True, device=0):
         image=image.cpu().numpy(), final_T=final_T.cpu().numpy(), n_contrib=u32(n_contrib), grads=None, g2d=None)
     out.visible = out.tiles_touched > 0
     if G is not None:
-        g = api.alloc_grads(n, ds.app, dev)
+        g = api.alloc_grads_for(ds, dev)
         Gd = torch.from_numpy(np.ascontiguousarray(G, np.float32)).to(dev)
         api.gs_render_backward(ctx, ds, ccam, proj, binning, P, final_T, n_contrib, Gd, g, ws)
         torch.cuda.synchronize()

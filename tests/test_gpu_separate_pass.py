@@ -1,0 +1,111 @@
+"""The unfused reference path of the rendering step (Sec. 4 "CUDA Implementation", App. D "Fusion"): the
+appearance model evaluated as passes of its own around the rasterizer, exchanging directions, colours and
+their gradients through global memory.  It must give what the fused step gives (the paper's own validation of
+its fused kernels), and it is the way a decoder of another size goes through the whole step: those are
+checked against the oracle."""
+import copy
+
+import numpy as np
+import pytest
+
+from paper_2609_05255_b200 import scenes
+from gpu_helpers import GRAD_ATOL, grad_mismatch, grad_names, image_mismatch, run_gpu
+
+pytestmark = pytest.mark.gpu
+
+INT_FIELDS = ("depth_key", "rect", "tiles_touched", "depth_order", "sorted_tiles", "sorted_vals", "tile_ranges", "n_contrib")
+
+
+@pytest.mark.parametrize("app", [scenes.APP_SH, scenes.APP_NEURAL, scenes.APP_SV], ids=["sh", "neural", "sv"])
+def test_unfused_step_equals_fused_step(app):
+    w = scenes.config2(n=12_011, app=app)
+    cam = w.cameras[0]
+    G = scenes.upstream_gradient(cam, 7)
+    fused = run_gpu(w.scene, cam, G)
+    sc = copy.copy(w.scene)
+    sc.separate_pass = 1
+    unfused = run_gpu(sc, cam, G)
+    for nm in INT_FIELDS:
+        assert np.array_equal(getattr(fused, nm), getattr(unfused, nm)), nm
+    vis = fused.visible
+    assert vis.sum() > 5_000
+    assert np.abs(fused.color[vis] - unfused.color[vis]).max() < 1e-5
+    assert np.abs(fused.image - unfused.image).max() < 1e-5
+    for nm in grad_names(app):
+        a, b = getattr(fused.grads, nm), getattr(unfused.grads, nm)
+        # both runs sum the blend's atomics in their own order: the rule of the parity tests, between the two
+        bad = grad_mismatch(a, b)
+        assert bad.mean() <= (2e-2 if nm == "mlp_weights" else 5e-4), f"{nm}: {bad.sum()} of {bad.size}"
+        assert np.abs(a - b).max() <= max(2e-3 * np.abs(a).max(), GRAD_ATOL), nm
+        if nm != "mlp_weights":
+            assert np.all(b[~vis] == 0), nm        # culled Gaussians: exact zeros from the separate passes too
+
+
+def test_unfused_step_with_nan_appearance_on_a_culled_gaussian():
+    """A Gaussian that is culled never reaches the appearance passes: its parameters may hold anything."""
+    w = scenes.config2(n=3_001, app=scenes.APP_NEURAL)
+    cam = w.cameras[0]
+    G = scenes.upstream_gradient(cam, 8)
+    sc = copy.copy(w.scene)
+    sc.separate_pass = 1
+    sc.means = sc.means.copy(); sc.features = sc.features.copy(); sc.base_color = sc.base_color.copy()
+    sc.means[5] = (0.0, 0.0, -3.0)                       # behind the camera
+    sc.features[5] = np.float16("nan"); sc.base_color[5] = np.nan
+    out = run_gpu(sc, cam, G)
+    assert not out.visible[5]
+    for nm in grad_names(scenes.APP_NEURAL):
+        assert np.isfinite(getattr(out.grads, nm)).all(), nm
+    assert np.isfinite(out.image).all()
+
+
+@pytest.mark.parametrize("arch", [(16, 1, 8), (32, 2, 8), (16, 2, 16), (16, 3, 8)], ids=lambda a: "h%d_l%d_f%d" % a)
+def test_decoder_variant_through_the_whole_step(oracle, arch):
+    hidden, layers, nfeat = arch
+    w = scenes.config2(n=20_011, app=scenes.APP_NEURAL)      # the size of the fused parity tests: same tolerances
+    cam = w.cameras[0]
+    sc = w.scene
+    rng = np.random.default_rng(np.random.PCG64(4242))
+    _, sc.features, sc.mlp_weights = scenes.draw_neural_appearance(rng, sc.n, hidden, layers, nfeat)
+    sc.mlp_hidden, sc.mlp_layers = hidden, layers
+    G = scenes.upstream_gradient(cam, 9)
+    gpu = run_gpu(sc, cam, G)
+    fwd, grads = oracle.render(sc, cam, G)
+    same_vis = gpu.visible == fwd.pre.visible.astype(bool)
+    assert (~same_vis).sum() <= 2
+    both = gpu.visible & same_vis
+    assert np.abs(gpu.color[both] - fwd.color[both]).max() < 2e-5
+    assert image_mismatch(gpu.image, fwd.image, fwd.fragile).sum() == 0
+    # the appearance passes in isolation: the oracle's decoder fed with the GPU's own dL/dcolor
+    vis = gpu.visible.astype(np.uint8)
+    ga = oracle.appearance_backward(sc, fwd.pre.dir, gpu.g2d[:, 0:3].astype(np.float64), mask=vis)
+    gp = oracle.preprocess_backward(sc.means, sc.log_scales, sc.quats, sc.opacity_logits, cam, vis,
+                                    gpu.g2d[:, 7:9], gpu.g2d[:, 4:7], gpu.g2d[:, 3], ga.dirs)
+    ref = dict(means=gp.means, log_scales=gp.log_scales, quats=gp.quats, opacity_logits=gp.opacity_logits,
+               base_color=ga.base_color, features=ga.features, mlp_weights=ga.mlp_weights)
+    assert gpu.grads.features.shape == (sc.n, nfeat) and gpu.grads.mlp_weights.shape == ref["mlp_weights"].shape
+    for nm in grad_names(scenes.APP_NEURAL):
+        got = getattr(gpu.grads, nm)
+        bad = grad_mismatch(got, ref[nm])
+        if nm != "mlp_weights":
+            bad[~same_vis] = False
+            assert bad.mean() <= 2e-4, f"{nm}: {bad.sum()} of {bad.size} off (separate passes)"
+        else:
+            assert np.abs(got - ref[nm]).max() <= 2e-4 * np.abs(ref[nm]).max()
+    # end to end against the oracle's own gradients, by the rule of the fused parity tests
+    for nm in grad_names(scenes.APP_NEURAL):
+        got, want = getattr(gpu.grads, nm), getattr(grads, nm)
+        bad = grad_mismatch(got, want)
+        d = np.abs(got - want)
+        if nm != "mlp_weights":
+            bad[~same_vis] = False; d[~same_vis] = 0
+        assert bad.mean() <= (2e-2 if nm == "mlp_weights" else 2e-3), f"{nm}: {bad.sum()} of {bad.size} off end to end"
+        assert d.max() <= max(1e-2 * np.abs(want).max(), GRAD_ATOL), nm
+        if nm != "mlp_weights":
+            assert np.all(got[~gpu.visible] == 0)
+
+
+def test_workspace_covers_the_separate_passes():
+    from paper_2609_05255_b200 import api
+    n = 100_000
+    # backward scratch: [n,12] + three [n,3] arrays, each rounded up to 256 bytes
+    assert api.gs_workspace_bytes(n, 64, 64, 0) >= n * (12 + 9) * 4
