@@ -272,7 +272,16 @@ def run_ours(args):
             evaluated += ev; composited += co
             rect = r.proj.rect.to(torch.int32) & 0xFFFF
             visible += int(((rect[:, 2] > rect[:, 0]) & (rect[:, 3] > rect[:, 1])).sum().item())
-        results[tag] = dict(ms=ms, ms_one=ms_one, ms_streams=ms_streams, graph=graph_note,
+        # the same step through the unfused reference path (App. D "Fusion"): appearance as passes of its own
+        unfused = None
+        if args.config == 3 and not args.skip_decode:
+            ds.separate_pass = 1
+            u_one = timed(lambda: step(ds, r), args.steps, args.warmup)
+            u_stage, _ = profile(lambda: step(ds, r), max(1, min(args.steps, 3)))
+            ds.separate_pass = 0
+            unfused = {"ms_per_step_single_stream": u_one, "fused_ms_per_step_single_stream": ms_one,
+                       "stages_ms_per_step": {k: round(v, 4) for k, v in u_stage.items() if v > 0}}
+        results[tag] = dict(ms=ms, ms_one=ms_one, ms_streams=ms_streams, graph=graph_note, unfused=unfused,
                             stage_ms=stage_ms, stage_launches=stage_launches, pairs=pairs,
                             entries=entries, visible=visible, evaluated=evaluated, composited=composited,
                             host=host, ds=ds, r=r, app=tag)
@@ -325,6 +334,7 @@ def run_ours(args):
         "sv": None if "sv" not in results or head == "sv" else {
             "ms_per_step": results["sv"]["ms"], "ms_per_step_single_stream": results["sv"]["ms_one"],
             "stages_ms_per_step": {k: round(v, 4) for k, v in results["sv"]["stage_ms"].items() if v > 0}},
+        "separate_pass_step": {t: results[t]["unfused"] for t in results if results[t].get("unfused")} or None,
         "appearance_decode": decode,
         "adam_update": adam,
         "viewer_prepass": prepass,
