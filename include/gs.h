@@ -200,7 +200,9 @@ GsStatus gs_preprocess_async(GsContext *ctx, const GsScene *scene, const GsCamer
  * flag is set that gs_async_status reports. */
 #define GS_PAIRS_ON_DEVICE ((int64_t)-1)
 /* Waits for `stream`, then returns GS_ERR_CAPACITY if any device-counted view on this context
- * overflowed its pair_capacity since the last call (and clears the flag), else GS_OK. */
+ * overflowed its pair_capacity since the last call (and clears the flag), GS_ERR_INTERNAL if a kernel
+ * gave up a bounded wait on one of its own bulk copies (never expected; the waits exist so that a
+ * kernel cannot hang), else GS_OK. */
 GsStatus gs_async_status(GsContext *ctx, void *stream);
 
 /* Tile assignment, ordering and blending (Sec. 3.1, blend kernel).  Orders the visible

@@ -16,7 +16,8 @@ struct GsContext {
   int device;
   int num_sms;
   unsigned long long *d_counter;      // device: [0] instance counter of the last gs_preprocess, [1] second word of
-                                      // gs_profile_blend_counts, [2] set when a device-counted view overflowed its capacity
+                                      // gs_profile_blend_counts, [2] set when a device-counted view overflowed its capacity,
+                                      // [3] set when a bounded device-side wait ran out
   unsigned long long *h_counter;      // pinned host mirror
   float *d_w_partials;                // device: per-CTA partial sums of the decoder gradient ([kWgradBlocks, 816];
                                       // sized for the decoder variants' largest case as well)
@@ -104,9 +105,10 @@ bool default_decoder(const GsScene *s) {
 // The rendering step with the appearance as passes of its own (asked for, or the only way for a decoder variant).
 bool unfused(const GsScene *s) { return s->separate_pass != 0 || !default_decoder(s); }
 
-AppearanceArgs appearance_args(const GsScene *scene) {
+AppearanceArgs appearance_args(GsContext *ctx, const GsScene *scene) {
   AppearanceArgs a;
   memset(&a, 0, sizeof(a));
+  a.timeout = ctx->d_counter + 3;
   a.n = scene->n; a.deg = scene->active_degree; a.act = scene->color_activation;
   a.base_color = scene->base_color; a.sh_rest = scene->app == GS_APP_SV ? scene->sv_sites : scene->sh_rest;
   a.features = reinterpret_cast<const __half *>(scene->features);
@@ -291,7 +293,7 @@ GsStatus preprocess_impl(GsContext *ctx, const GsScene *scene, const GsCamera *c
     t.done(launch_preprocess_fwd(unfused(scene) ? kAppExternal : scene->app, a, make_cam(cam), s));
   }
   if (unfused(scene)) {   // directions sit in out->color: decode them in place, visible Gaussians only
-    AppearanceArgs ap = appearance_args(scene);
+    AppearanceArgs ap = appearance_args(ctx, scene);
     ap.dirs = out->color; ap.color = out->color; ap.mask = out->tiles_touched;
     StageTimer t(ctx, GS_STAGE_APPEARANCE_FWD, s);
     t.done(run_appearance_fwd(scene, ap, s));
@@ -324,10 +326,12 @@ GsStatus gs_async_status(GsContext *ctx, void *stream) {
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   cudaSetDevice(ctx->device);
   GsStatus st;
-  if ((st = check_cuda(ctx, cudaMemcpyAsync(ctx->h_counter + 2, ctx->d_counter + 2, sizeof(unsigned long long),
+  if ((st = check_cuda(ctx, cudaMemcpyAsync(ctx->h_counter + 2, ctx->d_counter + 2, 2 * sizeof(unsigned long long),
                                             cudaMemcpyDeviceToHost, s), "status copy")) != GS_OK) return st;
-  if ((st = check_cuda(ctx, cudaMemsetAsync(ctx->d_counter + 2, 0, sizeof(unsigned long long), s), "status reset")) != GS_OK) return st;
+  if ((st = check_cuda(ctx, cudaMemsetAsync(ctx->d_counter + 2, 0, 2 * sizeof(unsigned long long), s), "status reset")) != GS_OK) return st;
   if ((st = check_cuda(ctx, cudaStreamSynchronize(s), "status")) != GS_OK) return st;
+  if (ctx->h_counter[3] != 0)
+    return fail(ctx, GS_ERR_INTERNAL, "a bounded wait on a bulk copy ran out in an appearance kernel: its results are incomplete");
   if (ctx->h_counter[2] != 0)
     return fail(ctx, GS_ERR_CAPACITY, "a device-counted gs_render_forward had more instances than pair_capacity: that view's lists were cut off");
   return GS_OK;
@@ -458,7 +462,7 @@ GsStatus gs_render_backward(GsContext *ctx, const GsScene *scene, const GsCamera
     return check_cuda(ctx, cudaMemsetAsync(grads->mlp_weights, 0, sizeof(float) * variant_num_weights(d.hidden, d.layers), s), "memset");
   }
   if (ext && n > 0) {   // the appearance backward as a pass of its own, through dense arrays in the workspace
-    AppearanceArgs ap = appearance_args(scene);
+    AppearanceArgs ap = appearance_args(ctx, scene);
     ap.dirs = bw.dirs; ap.g_color = bw.g_color; ap.mask = proj->tiles_touched;
     ap.g_base = grads->base_color; ap.g_sh_rest = scene->app == GS_APP_SV ? grads->sv_sites : grads->sh_rest;
     ap.g_features = grads->features; ap.g_dirs = bw.g_dirs;
@@ -482,12 +486,8 @@ GsStatus gs_appearance_forward(GsContext *ctx, const GsScene *scene, const float
   if (scene->n == 0) return GS_OK;
   if (bad_ptr(dirs) || bad_ptr(color)) return fail(ctx, GS_ERR_INVALID_ARG, "dirs / color is NULL or misaligned");
   cudaSetDevice(ctx->device);
-  AppearanceArgs a;
-  memset(&a, 0, sizeof(a));
-  a.n = scene->n; a.deg = scene->active_degree; a.act = scene->color_activation;
-  a.base_color = scene->base_color; a.sh_rest = scene->app == GS_APP_SV ? scene->sv_sites : scene->sh_rest; a.dirs = dirs;
-  a.features = reinterpret_cast<const __half *>(scene->features);
-  a.weights = reinterpret_cast<const __half *>(scene->mlp_weights);
+  AppearanceArgs a = appearance_args(ctx, scene);
+  a.dirs = dirs;
   a.color = color;
   {
     StageTimer t(ctx, GS_STAGE_APPEARANCE_FWD, static_cast<cudaStream_t>(stream));
@@ -518,12 +518,8 @@ GsStatus gs_appearance_backward(GsContext *ctx, const GsScene *scene, const floa
   if (scene->app == GS_APP_SH && bad_ptr(grads->sh_rest)) return fail(ctx, GS_ERR_INVALID_ARG, "grads->sh_rest is NULL or misaligned");
   if (scene->app == GS_APP_SV && bad_ptr(grads->sv_sites)) return fail(ctx, GS_ERR_INVALID_ARG, "grads->sv_sites is NULL or misaligned");
   if (scene->app == GS_APP_NEURAL && bad_ptr(grads->features)) return fail(ctx, GS_ERR_INVALID_ARG, "grads->features is NULL or misaligned");
-  AppearanceArgs a;
-  memset(&a, 0, sizeof(a));
-  a.n = scene->n; a.deg = scene->active_degree; a.act = scene->color_activation;
-  a.base_color = scene->base_color; a.sh_rest = scene->app == GS_APP_SV ? scene->sv_sites : scene->sh_rest; a.dirs = dirs;
-  a.features = reinterpret_cast<const __half *>(scene->features);
-  a.weights = reinterpret_cast<const __half *>(scene->mlp_weights);
+  AppearanceArgs a = appearance_args(ctx, scene);
+  a.dirs = dirs;
   a.g_color = dL_dcolor;
   a.g_base = grads->base_color; a.g_sh_rest = scene->app == GS_APP_SV ? grads->sv_sites : grads->sh_rest;
   a.g_features = grads->features; a.g_dirs = dL_ddirs;

@@ -864,6 +864,141 @@ __global__ void __launch_bounds__(kBlock) k_appearance_bwd(AppearanceArgs a) {
   }
 }
 
+// ---- separate-pass kernels of the explicit models with bulk copies ---------------------------------------------
+// The parameter rows of a warp's 32 Gaussians are one contiguous piece of global memory (5760 B for SH, 6272 B
+// for Spherical Voronoi, a multiple of 16 either way).  One lane moves it with a single 1D bulk copy of the
+// tensor memory accelerator into the warp's shared-memory slab and the warp sleeps on an mbarrier until the
+// bytes have landed; the gradient slab of the backward goes back the same way.  Each warp owns two slabs and is
+// persistent, so the copy of its next 32 rows is in flight while it works on the current ones, with no
+// registers or store instructions spent on staging.  Every wait is bounded: if a barrier does not flip within
+// the limit the warp records it in *timeout and leaves, draining its own copies first.
+namespace bulk {
+__device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void barrier_init(uint32_t bar) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity) {
+  for (int it = 0; it < (1 << 20); ++it) {   // each try sleeps at most about a microsecond: the wait ends within a second
+    uint32_t done;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(done) : "r"(bar), "r"(parity), "r"(1000u) : "memory");
+    if (done) return true;
+  }
+  return false;
+}
+__device__ __forceinline__ void store(void *dst, uint32_t src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes) : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void wait_stores_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void wait_stores_done() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_generic_writes() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+}  // namespace bulk
+
+template <int APP> constexpr size_t bulk_smem_bytes() {
+  return sizeof(float) * kWarps * 2 * SlabOf<APP>::value + sizeof(unsigned long long) * kWarps * 2;
+}
+
+// BWD = false: colours.  BWD = true: gradient rows (written in place over the parameter rows), dL/dc0, dL/dd.
+template <int APP, bool BWD>
+__global__ void __launch_bounds__(kBlock) k_appearance_bulk(AppearanceArgs a) {
+  static_assert(Explicit<APP>::value, "the explicit models only");
+  constexpr int kRow = RowOf<APP>::value, kSlab = SlabOf<APP>::value;
+  constexpr uint32_t kBytes = kSlab * sizeof(float);
+  static_assert(kBytes % 16 == 0, "a bulk copy moves multiples of 16 bytes");
+  extern __shared__ __align__(128) unsigned char bulk_smem[];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  float *const buf0 = reinterpret_cast<float *>(bulk_smem) + (warp * 2) * kSlab, *const buf1 = buf0 + kSlab;
+  unsigned long long *bars = reinterpret_cast<unsigned long long *>(bulk_smem + sizeof(float) * kWarps * 2 * kSlab);
+  const uint32_t bar0 = bulk::smem_addr(bars + warp * 2), bar1 = bar0 + 8;
+  if (lane == 0) {
+    bulk::barrier_init(bar0); bulk::barrier_init(bar1);
+    bulk::fence_barrier_init();
+  }
+  __syncwarp();
+  const bool rows_needed = a.deg > 0;
+  const int64_t nchunks = (a.n + kBlock - 1) / kBlock;
+  uint32_t parity0 = 0u, parity1 = 0u;   // phase each barrier completes next
+  int s = 0;
+  // the first copy
+  {
+    const int64_t row0 = (int64_t)blockIdx.x * kBlock + warp * 32;
+    if (rows_needed && lane == 0 && row0 + 32 <= a.n) bulk::load(bulk::smem_addr(buf0), a.sh_rest + row0 * kRow, kBytes, bar0);
+  }
+  bool ok = true;
+  for (int64_t chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x, s ^= 1) {
+    const int64_t row0 = chunk * kBlock + warp * 32, i = row0 + lane;
+    const int rows = row0 < a.n ? (int)min((int64_t)32, a.n - row0) : 0;
+    __syncwarp();                      // every lane is done with the other slab
+    if (lane == 0) {
+      if (BWD) bulk::wait_stores_read();   // ... and so is the copy that carried its gradients away
+      const int64_t nrow0 = row0 + (int64_t)gridDim.x * kBlock;
+      if (rows_needed && nrow0 + 32 <= a.n) bulk::load(bulk::smem_addr(s ? buf0 : buf1), a.sh_rest + nrow0 * kRow, kBytes, s ? bar0 : bar1);
+    }
+    if (rows == 0) continue;
+    const bool exists = lane < rows;
+    const bool in = exists && (!a.mask || __ldg(a.mask + i) != 0u);
+    float d[3] = {0.f, 0.f, 1.f}, base[3] = {0.f, 0.f, 0.f}, gcol[3] = {0.f, 0.f, 0.f};
+    if (in) {
+      load3(a.dirs, i, d); load3(a.base_color, i, base);
+      if (BWD) load3(a.g_color, i, gcol);
+    }
+    float *slab = s ? buf1 : buf0, *row = slab + lane * kRow;
+    if (rows_needed) {
+      if (rows == 32) {
+        ok = bulk::wait(s ? bar1 : bar0, s ? parity1 : parity0);
+        if (s) parity1 ^= 1u; else parity0 ^= 1u;
+        if (!__all_sync(kFull, ok)) { ok = false; break; }
+      } else {
+        __syncwarp();
+        warp_load_rows<kRow>(a.sh_rest, row0, a.n, slab, lane);   // the ragged last rows: plain loads
+      }
+    }
+    float pre[3] = {base[0] + 0.5f, base[1] + 0.5f, base[2] + 0.5f};
+    SvCarry cy;
+    if (in && rows_needed) explicit_pre<APP>(row, base, d[0], d[1], d[2], a.deg, pre, cy);
+    if (!BWD) {
+      if (in) store3(a.color, i, color_act_z(a.act, pre[0]), color_act_z(a.act, pre[1]), color_act_z(a.act, pre[2]));
+    } else {
+      float gp[3] = {0.f, 0.f, 0.f}, gd[3] = {0.f, 0.f, 0.f};
+      if (in) {
+#pragma unroll
+        for (int c = 0; c < 3; ++c) gp[c] = color_act_grad_z(a.act, pre[c]) * gcol[c];
+        explicit_bwd<APP>(row, gp, d[0], d[1], d[2], a.deg, cy, gd);
+      } else if (exists) {
+#pragma unroll
+        for (int k = 0; k < kRow; ++k) row[k] = 0.f;
+      }
+      if (exists) {
+        store3(a.g_base, i, gp[0], gp[1], gp[2]);
+        store3(a.g_dirs, i, gd[0], gd[1], gd[2]);
+      }
+      if (rows == 32) {
+        bulk::fence_generic_writes();      // the lanes' rows become visible to the copy engine
+        __syncwarp();
+        if (lane == 0) bulk::store(a.g_sh_rest + row0 * kRow, bulk::smem_addr(slab), kBytes);
+      } else {
+        warp_store_rows<kRow>(a.g_sh_rest, row0, a.n, slab, lane);
+      }
+    }
+  }
+  if (lane == 0) {
+    if (BWD) bulk::wait_stores_done();
+    if (!ok && a.timeout) atomicExch(a.timeout, 1ull);
+  }
+  if (!ok && rows_needed) {
+    // a copy may still be in flight into this warp's slabs: give it the same bounded time before the CTA ends
+    bulk::wait(bar0, parity0);
+    bulk::wait(bar1, parity1);
+  }
+}
+
 // Unfused step, backward: what the separate appearance backward reads, as dense arrays.
 __global__ void __launch_bounds__(kBlock) k_unfused_prepare(int64_t n, const float *__restrict__ means, CamDev cam,
                                                             const float *__restrict__ g2d, const uint32_t *__restrict__ mask,
@@ -893,8 +1028,8 @@ void opt_in_smem(K kernel, size_t bytes) {
 
 // Grid of a persistent kernel: as many CTAs as fit on the device at once (a second, thinner wave of a
 // grid-stride loop would run at a fraction of the occupancy), at most kWgradBlocks (rows of the partial buffer).
-template <class K>
-int resident_blocks(K kernel, size_t smem_bytes) {
+template <auto kernel>      // one cache per kernel, not per signature
+int resident_blocks(size_t smem_bytes) {
   static int cached[64] = {};
   int dev = 0;
   cudaGetDevice(&dev);
@@ -944,35 +1079,40 @@ int launch_preprocess_bwd(int app, const PreprocessBwdArgs &a, const CamDev &cam
     return 1;
   } else {
     opt_in_smem(k_preprocess_bwd<GS_APP_NEURAL>, kBwdSmemNN);
-    const int blocks = resident_blocks(k_preprocess_bwd<GS_APP_NEURAL>, kBwdSmemNN);
+    const int blocks = resident_blocks<k_preprocess_bwd<GS_APP_NEURAL>>(kBwdSmemNN);
     k_preprocess_bwd<GS_APP_NEURAL><<<blocks, kBlock, kBwdSmemNN, st>>>(a, cam);
     launch_wgrad_reduce(a.w_partials, blocks, a.g_weights, st);
     return 2;
   }
 }
 
+template <int APP, bool BWD>
+int launch_bulk(const AppearanceArgs &a, cudaStream_t st) {
+  constexpr size_t smem = bulk_smem_bytes<APP>();
+  opt_in_smem(k_appearance_bulk<APP, BWD>, smem);
+  const int wave = resident_blocks<k_appearance_bulk<APP, BWD>>(smem), chunks = grid_for(a.n);
+  k_appearance_bulk<APP, BWD><<<chunks < wave ? chunks : wave, kBlock, smem, st>>>(a);
+  return 1;
+}
+
 int launch_appearance_fwd(int app, const AppearanceArgs &a, cudaStream_t st) {
   if (a.n == 0) return 0;
-  if (app == GS_APP_SH) k_appearance_fwd<GS_APP_SH><<<grid_for(a.n), kBlock, 0, st>>>(a);
-  else if (app == GS_APP_SV) k_appearance_fwd<GS_APP_SV><<<grid_for(a.n), kBlock, 0, st>>>(a);
-  else k_appearance_fwd<GS_APP_NEURAL><<<grid_for(a.n), kBlock, 0, st>>>(a);
+  if (app == GS_APP_SH) return launch_bulk<GS_APP_SH, false>(a, st);
+  if (app == GS_APP_SV) return launch_bulk<GS_APP_SV, false>(a, st);
+  k_appearance_fwd<GS_APP_NEURAL><<<grid_for(a.n), kBlock, 0, st>>>(a);
   return 1;
 }
 
 int launch_appearance_bwd(int app, const AppearanceArgs &a, cudaStream_t st) {
   if (app == GS_APP_SH) {
     if (a.n == 0) return 0;
-    opt_in_smem(k_appearance_bwd<GS_APP_SH>, kBwdSmemSH);
-    k_appearance_bwd<GS_APP_SH><<<grid_for(a.n), kBlock, kBwdSmemSH, st>>>(a);
-    return 1;
+    return launch_bulk<GS_APP_SH, true>(a, st);
   } else if (app == GS_APP_SV) {
     if (a.n == 0) return 0;
-    opt_in_smem(k_appearance_bwd<GS_APP_SV>, kBwdSmemSV);
-    k_appearance_bwd<GS_APP_SV><<<grid_for(a.n), kBlock, kBwdSmemSV, st>>>(a);
-    return 1;
+    return launch_bulk<GS_APP_SV, true>(a, st);
   } else {
     opt_in_smem(k_appearance_bwd<GS_APP_NEURAL>, kBwdSmemNN);
-    const int blocks = resident_blocks(k_appearance_bwd<GS_APP_NEURAL>, kBwdSmemNN);
+    const int blocks = resident_blocks<k_appearance_bwd<GS_APP_NEURAL>>(kBwdSmemNN);
     k_appearance_bwd<GS_APP_NEURAL><<<blocks, kBlock, kBwdSmemNN, st>>>(a);
     launch_wgrad_reduce(a.w_partials, blocks, a.g_weights, st);
     return 2;
