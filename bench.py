@@ -251,7 +251,16 @@ def run_ours(args):
                 except Exception as e:                      # capture is an optimisation of the launching only
                     graph_note = {"captured": False, "why": str(e)[:200]}
                     torch.cuda.synchronize()
+            half_streams = None
+            if tag == "neural" and args.config == 3 and not args.skip_decode:
+                ds.decoder_precision = 1                    # plain fp16 operands, the paper's precision
+                half_streams = timed(lambda: step_two_streams(ds, rs), args.steps, args.warmup)
+                for c, s_ in zip(lane_ctx, lanes):
+                    api.gs_async_status(c, s_)
+                ds.decoder_precision = 0
             del rs
+        else:
+            half_streams = None
         stage_ms, stage_launches = profile(lambda: step(ds, r), max(1, min(args.steps, 3)))
         if tag == head:
             # keep the GPU under the same load until the sampler has a few readings (100 ms apart)
@@ -281,7 +290,18 @@ def run_ours(args):
             ds.separate_pass = 0
             unfused = {"ms_per_step_single_stream": u_one, "fused_ms_per_step_single_stream": ms_one,
                        "stages_ms_per_step": {k: round(v, 4) for k, v in u_stage.items() if v > 0}}
-        results[tag] = dict(ms=ms, ms_one=ms_one, ms_streams=ms_streams, graph=graph_note, unfused=unfused,
+        half = None
+        if tag == "neural" and args.config == 3 and not args.skip_decode:
+            ds.decoder_precision = 1
+            h_one = timed(lambda: step(ds, r), args.steps, args.warmup)
+            h_stage, _ = profile(lambda: step(ds, r), max(1, min(args.steps, 3)))
+            ds.decoder_precision = 0
+            half = {"ms_per_step": half_streams, "ms_per_step_single_stream": h_one,
+                    "split_ms_per_step": ms_streams, "split_ms_per_step_single_stream": ms_one,
+                    "stages_ms_per_step": {k: round(v, 4) for k, v in h_stage.items() if v > 0},
+                    "what": "the decoder's products on plain fp16 operands (GS_DECODER_HALF, the paper's precision) instead of "
+                            "split ones; colours within 2e-3 of the oracle instead of 2e-5 (tests/test_gpu_half_precision.py)"}
+        results[tag] = dict(ms=ms, ms_one=ms_one, ms_streams=ms_streams, graph=graph_note, unfused=unfused, half=half,
                             stage_ms=stage_ms, stage_launches=stage_launches, pairs=pairs,
                             entries=entries, visible=visible, evaluated=evaluated, composited=composited,
                             host=host, ds=ds, r=r, app=tag)
@@ -334,6 +354,7 @@ def run_ours(args):
         "sv": None if "sv" not in results or head == "sv" else {
             "ms_per_step": results["sv"]["ms"], "ms_per_step_single_stream": results["sv"]["ms_one"],
             "stages_ms_per_step": {k: round(v, 4) for k, v in results["sv"]["stage_ms"].items() if v > 0}},
+        "neural_half_precision": results[head].get("half") if head == "neural" else None,
         "separate_pass_step": {t: results[t]["unfused"] for t in results if results[t].get("unfused")} or None,
         "appearance_decode": decode,
         "adam_update": adam,
@@ -706,10 +727,13 @@ def decode_sweep(api, torch, ctx, dev, peaks, args):
                         ts.append(e0.elapsed_time(e1))
                 ts.sort()
                 return ts[len(ts) // 2]
-            f_ms = run(lambda: api.gs_appearance_forward(ctx, sc, dirs, color))
-            b_ms = run(lambda: api.gs_appearance_backward(ctx, sc, dirs, gcol, grads, gd))
-            gbs = (bytes_fwd + bytes_bwd) * n / ((f_ms + b_ms) * 1e-3) / 1e9
-            out[f"{tag}_{n // 1_000_000}M"] = {
+            for precision in ((0, 1) if app == 1 else (0,)):
+              sc.decoder_precision = precision
+              row = f"{tag}{'_half' if precision else ''}_{n // 1_000_000}M"
+              f_ms = run(lambda: api.gs_appearance_forward(ctx, sc, dirs, color))
+              b_ms = run(lambda: api.gs_appearance_backward(ctx, sc, dirs, gcol, grads, gd))
+              gbs = (bytes_fwd + bytes_bwd) * n / ((f_ms + b_ms) * 1e-3) / 1e9
+              out[row] = {
                 "fwd_ms": round(f_ms, 4), "bwd_ms": round(b_ms, 4), "bytes_per_primitive": bytes_fwd + bytes_bwd,
                 "GBps": round(gbs, 1), "frac_of_hbm_peak": round(gbs / peaks["hbm_gbs"], 4),
                 "fwd_GBps": round(bytes_fwd * n / (f_ms * 1e-3) / 1e9, 1),

@@ -68,6 +68,8 @@ typedef enum {
   GS_ACT_HARD_SIGMOID = 3  /* clamp(x + 0.5, 0, 1)                                              */
 } GsColorActivation;
 
+typedef enum { GS_DECODER_SPLIT = 0, GS_DECODER_HALF = 1 } GsDecoderPrecision;
+
 /* Pinhole camera (host struct). */
 typedef struct {
   int32_t width, height;        /* pixels; at most 65535 tiles of 16 pixels per axis and 2^24
@@ -119,6 +121,13 @@ typedef struct {
                                     backward as a pass of its own between the blend backward and the
                                     projection backward, exchanging directions, dL/dcolor and dL/dd
                                     through the workspace.  Same results up to rounding             */
+  int32_t decoder_precision;     /* neural, default decoder only.  GS_DECODER_SPLIT (0): every product of
+                                    the decoder takes its fp32 activation or gradient as two fp16 halves
+                                    (fp32 accumulation), which keeps the results as accurate as fp32 FMAs:
+                                    the mode every stated tolerance refers to.  GS_DECODER_HALF (1): plain
+                                    fp16 operands with fp32 accumulation, the precision the paper runs its
+                                    decoder in (Sec. 4 "CUDA Implementation"): about half the tensor-core
+                                    work; colours then carry errors of the order of 1e-3                  */
 } GsScene;
 
 /* Per-Gaussian results of gs_preprocess (caller-allocated device buffers). */

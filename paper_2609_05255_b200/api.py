@@ -24,6 +24,7 @@ _lib = C.CDLL(LIB_PATH)
 
 GS_OK, GS_ERR_INVALID_ARG, GS_ERR_CAPACITY, GS_ERR_CUDA, GS_ERR_UNSUPPORTED, GS_ERR_INTERNAL = 0, -1, -2, -3, -4, -6
 GS_APP_SH, GS_APP_NEURAL, GS_APP_SV = 0, 1, 2
+GS_DECODER_SPLIT, GS_DECODER_HALF = 0, 1
 TILE = 16
 MLP_WEIGHTS = 816
 
@@ -41,7 +42,7 @@ class GsScene(C.Structure):
                 ("base_color", _vp), ("app", C.c_int32), ("active_degree", C.c_int32), ("sh_rest", _vp),
                 ("features", _vp), ("mlp_weights", _vp), ("color_activation", C.c_int32), ("sv_sites", _vp),
                 ("mlp_hidden", C.c_int32), ("mlp_layers", C.c_int32), ("num_features", C.c_int32),
-                ("separate_pass", C.c_int32)]
+                ("separate_pass", C.c_int32), ("decoder_precision", C.c_int32)]
 
 
 class GsProjected(C.Structure):
@@ -166,6 +167,7 @@ class DeviceScene:
     mlp_layers: int = 2              # gs_appearance_forward / backward only
     num_features: int = 8
     separate_pass: int = 0           # 1: the unfused reference path (appearance as passes of its own)
+    decoder_precision: int = 0       # 0: split fp16 operands (fp32-accurate); 1: plain fp16 operands (the paper's)
 
     @property
     def n(self) -> int:
@@ -182,6 +184,7 @@ class DeviceScene:
         s.sv_sites = _ptr(self.sv_sites)
         s.mlp_hidden, s.mlp_layers, s.num_features = int(self.mlp_hidden), int(self.mlp_layers), int(self.num_features)
         s.separate_pass = int(self.separate_pass)
+        s.decoder_precision = int(self.decoder_precision)
         return s
 
 
@@ -197,7 +200,7 @@ def upload_scene(scene, device="cuda") -> DeviceScene:
                        up(getattr(scene, "sv_sites", None), torch.float32),
                        int(getattr(scene, "mlp_hidden", 0)) or 16, int(getattr(scene, "mlp_layers", 0)) or 2,
                        int(scene.features.shape[1]) if scene.features is not None else 8,
-                       int(getattr(scene, "separate_pass", 0)))
+                       int(getattr(scene, "separate_pass", 0)), int(getattr(scene, "decoder_precision", 0)))
 
 
 @dataclass

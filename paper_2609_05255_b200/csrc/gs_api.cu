@@ -102,6 +102,10 @@ bool default_decoder(const GsScene *s) {
   const DecoderArch d = decoder_arch(s);
   return s->app != GS_APP_NEURAL || (d.hidden == 16 && d.layers == 2 && d.nfeat == 8);
 }
+// The template instance a scene's appearance kernels run as.
+int kernel_app(const GsScene *s) {
+  return s->app == GS_APP_NEURAL && s->decoder_precision == GS_DECODER_HALF ? kAppNeuralHalf : s->app;
+}
 // The rendering step with the appearance as passes of its own (asked for, or the only way for a decoder variant).
 bool unfused(const GsScene *s) { return s->separate_pass != 0 || !default_decoder(s); }
 
@@ -117,11 +121,11 @@ AppearanceArgs appearance_args(GsContext *ctx, const GsScene *scene) {
 }
 int run_appearance_fwd(const GsScene *scene, const AppearanceArgs &a, cudaStream_t s) {
   const DecoderArch d = decoder_arch(scene);
-  return default_decoder(scene) ? launch_appearance_fwd(scene->app, a, s) : launch_variant_fwd(d.hidden, d.layers, d.nfeat, a, s);
+  return default_decoder(scene) ? launch_appearance_fwd(kernel_app(scene), a, s) : launch_variant_fwd(d.hidden, d.layers, d.nfeat, a, s);
 }
 int run_appearance_bwd(const GsScene *scene, const AppearanceArgs &a, cudaStream_t s) {
   const DecoderArch d = decoder_arch(scene);
-  return default_decoder(scene) ? launch_appearance_bwd(scene->app, a, s) : launch_variant_bwd(d.hidden, d.layers, d.nfeat, a, s);
+  return default_decoder(scene) ? launch_appearance_bwd(kernel_app(scene), a, s) : launch_variant_bwd(d.hidden, d.layers, d.nfeat, a, s);
 }
 
 GsStatus scene_appearance_ok(GsContext *ctx, const GsScene *s) {
@@ -129,6 +133,8 @@ GsStatus scene_appearance_ok(GsContext *ctx, const GsScene *s) {
   if (s->active_degree < 0 || s->active_degree > 3) return fail(ctx, GS_ERR_INVALID_ARG, "active_degree must be 0..3");
   if (s->color_activation < GS_ACT_RELU || s->color_activation > GS_ACT_HARD_SIGMOID)
     return fail(ctx, GS_ERR_INVALID_ARG, "unknown colour activation");
+  if (s->decoder_precision != GS_DECODER_SPLIT && s->decoder_precision != GS_DECODER_HALF)
+    return fail(ctx, GS_ERR_INVALID_ARG, "unknown decoder precision");
   if (s->n < 0) return fail(ctx, GS_ERR_INVALID_ARG, "n < 0");
   if (s->n >= ((int64_t)1 << 31)) return fail(ctx, GS_ERR_CAPACITY, "n must stay below 2^31 (32-bit Gaussian ids and grids)");
   if (s->app == GS_APP_NEURAL) {
@@ -290,7 +296,7 @@ GsStatus preprocess_impl(GsContext *ctx, const GsScene *scene, const GsCamera *c
   a.pair_counter = ctx->d_counter;
   {
     StageTimer t(ctx, GS_STAGE_PREPROCESS_FWD, s);
-    t.done(launch_preprocess_fwd(unfused(scene) ? kAppExternal : scene->app, a, make_cam(cam), s));
+    t.done(launch_preprocess_fwd(unfused(scene) ? kAppExternal : kernel_app(scene), a, make_cam(cam), s));
   }
   if (unfused(scene)) {   // directions sit in out->color: decode them in place, visible Gaussians only
     AppearanceArgs ap = appearance_args(ctx, scene);
@@ -473,7 +479,7 @@ GsStatus gs_render_backward(GsContext *ctx, const GsScene *scene, const GsCamera
   }
   {
     StageTimer t(ctx, GS_STAGE_PREPROCESS_BWD, s);
-    t.done(launch_preprocess_bwd(ext ? kAppExternal : scene->app, a, cd, s));
+    t.done(launch_preprocess_bwd(ext ? kAppExternal : kernel_app(scene), a, cd, s));
   }
   return check_cuda(ctx, cudaGetLastError(), "render_backward launch");
 }

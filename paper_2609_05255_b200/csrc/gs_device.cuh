@@ -34,6 +34,9 @@ struct CamDev {
 // forward leaves the view directions of the visible Gaussians where the colours go, the backward takes dL/dd
 // from a buffer.  The appearance kernels run as launches of their own around them.
 constexpr int kAppExternal = 3;
+// The neural model with the decoder's products taken on plain fp16 operands (the paper's precision) instead of
+// split ones: GsScene.decoder_precision = GS_DECODER_HALF.  Same kernels, same weights, same layout.
+constexpr int kAppNeuralHalf = 4;
 
 struct PreprocessArgs {
   int64_t n;

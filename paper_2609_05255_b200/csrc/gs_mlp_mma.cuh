@@ -63,13 +63,23 @@ __device__ __forceinline__ uint32_t movm_trans(uint32_t a) {
   return d;
 }
 
+// Transpose of a low half: nothing to do when operands are not split.
+template <bool kSplit>
+__device__ __forceinline__ uint32_t movm_lo(uint32_t a) { return kSplit ? movm_trans(a) : 0u; }
+
 // (a, b) -> packed fp16 pairs hi and lo with a = hi.x + lo.x, b = hi.y + lo.y up to ~2^-22.
+// kSplit = false is the paper's own precision (Sec. 4: the decoder in half precision): the operand is the
+// rounded value alone, lo stays zero and every product that would take it is left out.
+template <bool kSplit = true>
 __device__ __forceinline__ void split2(float a, float b, uint32_t &hi, uint32_t &lo) {
   const __half2 h = __floats2half2_rn(a, b);
-  const float2 f = __half22float2(h);
-  const __half2 l = __floats2half2_rn(a - f.x, b - f.y);
   hi = *reinterpret_cast<const uint32_t *>(&h);
-  lo = *reinterpret_cast<const uint32_t *>(&l);
+  lo = 0u;
+  if (kSplit) {
+    const float2 f = __half22float2(h);
+    const __half2 l = __floats2half2_rn(a - f.x, b - f.y);
+    lo = *reinterpret_cast<const uint32_t *>(&l);
+  }
 }
 
 __device__ __forceinline__ float2 unsplit(uint32_t hi, uint32_t lo) {
@@ -80,25 +90,26 @@ __device__ __forceinline__ float2 unsplit(uint32_t hi, uint32_t lo) {
 
 // The owner lane (lane = Gaussian row) parks its 32 inputs.  `Stage` is WarpStage or any struct
 // that starts with the same xhi / xlo / y members.
-template <class Stage>
+template <bool kSplit, class Stage>
 __device__ __forceinline__ void stage_inputs(const float x[32], Stage &S, int lane) {
   uint32_t hi[16], lo[16];
 #pragma unroll
-  for (int p = 0; p < 16; ++p) split2(x[2 * p], x[2 * p + 1], hi[p], lo[p]);
+  for (int p = 0; p < 16; ++p) split2<kSplit>(x[2 * p], x[2 * p + 1], hi[p], lo[p]);
   uint4 *dh = reinterpret_cast<uint4 *>(S.xhi + lane * kXStride), *dl = reinterpret_cast<uint4 *>(S.xlo + lane * kXStride);
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
     dh[q] = make_uint4(hi[4 * q], hi[4 * q + 1], hi[4 * q + 2], hi[4 * q + 3]);
-    dl[q] = make_uint4(lo[4 * q], lo[4 * q + 1], lo[4 * q + 2], lo[4 * q + 3]);
+    if (kSplit) dl[q] = make_uint4(lo[4 * q], lo[4 * q + 1], lo[4 * q + 2], lo[4 * q + 3]);
   }
 }
 
 // A operand (hi and lo) out of two neighbouring C tiles of one 16-row block.
+template <bool kSplit>
 __device__ __forceinline__ void a_from_c(const float c_lo[4], const float c_hi[4], uint32_t ahi[4], uint32_t alo[4]) {
-  split2(c_lo[0], c_lo[1], ahi[0], alo[0]);
-  split2(c_lo[2], c_lo[3], ahi[1], alo[1]);
-  split2(c_hi[0], c_hi[1], ahi[2], alo[2]);
-  split2(c_hi[2], c_hi[3], ahi[3], alo[3]);
+  split2<kSplit>(c_lo[0], c_lo[1], ahi[0], alo[0]);
+  split2<kSplit>(c_lo[2], c_lo[3], ahi[1], alo[1]);
+  split2<kSplit>(c_hi[0], c_hi[1], ahi[2], alo[2]);
+  split2<kSplit>(c_hi[2], c_hi[3], ahi[3], alo[3]);
 }
 
 struct Activations {
@@ -108,7 +119,7 @@ struct Activations {
 
 // Forward of the three layers for the warp's 32 staged rows.  Leaves y (3 values per row) in
 // S.y for the owner lanes; returns the hidden activations for the backward.
-template <class Stage>
+template <bool kSplit, class Stage>
 __device__ __forceinline__ void forward_warp(const Weights &W, Stage &S, int lane, Activations &act) {
   const int g = lane >> 2, t = lane & 3;
   const uint32_t *w32 = reinterpret_cast<const uint32_t *>(W.w);
@@ -132,11 +143,12 @@ __device__ __forceinline__ void forward_warp(const Weights &W, Stage &S, int lan
     for (int mt = 0; mt < 2; ++mt) {
       const int r0 = (16 * mt + g) * kXStride + 8 * ks + t, r1 = r0 + 8 * kXStride;
       const uint32_t ahi[4] = {S.xhi[r0], S.xhi[r1], S.xhi[r0 + 4], S.xhi[r1 + 4]};
-      const uint32_t alo[4] = {S.xlo[r0], S.xlo[r1], S.xlo[r0 + 4], S.xlo[r1 + 4]};
+      uint32_t alo[4] = {0u, 0u, 0u, 0u};
+      if (kSplit) { alo[0] = S.xlo[r0]; alo[1] = S.xlo[r1]; alo[2] = S.xlo[r0 + 4]; alo[3] = S.xlo[r1 + 4]; }
 #pragma unroll
       for (int nt = 0; nt < 2; ++nt) {
         mma16816(act.h1[mt][nt], ahi, b0[nt], b1[nt]);
-        mma16816(act.h1[mt][nt], alo, b0[nt], b1[nt]);
+        if (kSplit) mma16816(act.h1[mt][nt], alo, b0[nt], b1[nt]);
       }
     }
   }
@@ -157,13 +169,13 @@ __device__ __forceinline__ void forward_warp(const Weights &W, Stage &S, int lan
 #pragma unroll
     for (int mt = 0; mt < 2; ++mt) {
       uint32_t ahi[4], alo[4];
-      a_from_c(act.h1[mt][0], act.h1[mt][1], ahi, alo);
+      a_from_c<kSplit>(act.h1[mt][0], act.h1[mt][1], ahi, alo);
 #pragma unroll
       for (int nt = 0; nt < 2; ++nt) {
 #pragma unroll
         for (int k = 0; k < 4; ++k) act.h2[mt][nt][k] = 0.f;
         mma16816(act.h2[mt][nt], ahi, b0[nt], b1[nt]);
-        mma16816(act.h2[mt][nt], alo, b0[nt], b1[nt]);
+        if (kSplit) mma16816(act.h2[mt][nt], alo, b0[nt], b1[nt]);
       }
     }
   }
@@ -180,10 +192,10 @@ __device__ __forceinline__ void forward_warp(const Weights &W, Stage &S, int lan
 #pragma unroll
     for (int mt = 0; mt < 2; ++mt) {
       uint32_t ahi[4], alo[4];
-      a_from_c(act.h2[mt][0], act.h2[mt][1], ahi, alo);
+      a_from_c<kSplit>(act.h2[mt][0], act.h2[mt][1], ahi, alo);
       float c[4] = {0.f, 0.f, 0.f, 0.f};
       mma16816(c, ahi, b0, b1);
-      mma16816(c, alo, b0, b1);
+      if (kSplit) mma16816(c, alo, b0, b1);
       const int r0 = (16 * mt + g) * 4, r1 = r0 + 32;
       if (t == 0) { S.y[r0] = c[0]; S.y[r0 + 1] = c[1]; S.y[r1] = c[2]; S.y[r1 + 1] = c[3]; }
       if (t == 1) { S.y[r0 + 2] = c[0]; S.y[r1 + 2] = c[2]; }
@@ -209,16 +221,20 @@ struct WeightGrad {
 };
 
 // c += A^T-style product with both operands split: (Ahi + Alo)(Bhi + Blo) without the lo*lo term.
+template <bool kSplit>
 __device__ __forceinline__ void mma3(float c[4], const uint32_t ahi[4], const uint32_t alo[4], uint32_t b0h, uint32_t b1h,
                                      uint32_t b0l, uint32_t b1l) {
   mma16816(c, ahi, b0h, b1h);
-  mma16816(c, ahi, b0l, b1l);
-  mma16816(c, alo, b0h, b1h);
+  if (kSplit) {
+    mma16816(c, ahi, b0l, b1l);
+    mma16816(c, alo, b0h, b1h);
+  }
 }
 
 // Backward of the three layers.  On entry the owner lanes have written dL/dy (3 values per row,
 // 4th = 0) into S.y.  On exit S.gx holds dL/dx of the 16 direction inputs and S.gf holds dL/df per
 // row, and the warp's weight-gradient fragments have been advanced.
+template <bool kSplit>
 __device__ __forceinline__ void backward_warp(const Weights &W, WarpStage &S, int lane, const Activations &act,
                                               WeightGrad &dW) {
   const int g = lane >> 2, t = lane & 3;
@@ -236,15 +252,15 @@ __device__ __forceinline__ void backward_warp(const Weights &W, WarpStage &S, in
       if (t < 2) {
         const float2 u0 = *reinterpret_cast<const float2 *>(S.y + (16 * mt + g) * 4 + 2 * t);
         const float2 u1 = *reinterpret_cast<const float2 *>(S.y + (16 * mt + g + 8) * 4 + 2 * t);
-        split2(u0.x, u0.y, ahi[0], alo[0]);
-        split2(u1.x, u1.y, ahi[1], alo[1]);
+        split2<kSplit>(u0.x, u0.y, ahi[0], alo[0]);
+        split2<kSplit>(u1.x, u1.y, ahi[1], alo[1]);
       }
 #pragma unroll
       for (int nt = 0; nt < 2; ++nt) {
 #pragma unroll
         for (int k = 0; k < 4; ++k) d2[mt][nt][k] = 0.f;
         mma16816(d2[mt][nt], ahi, b0[nt], 0u);
-        mma16816(d2[mt][nt], alo, b0[nt], 0u);
+        if (kSplit) mma16816(d2[mt][nt], alo, b0[nt], 0u);
 #pragma unroll
         for (int k = 0; k < 4; ++k) d2[mt][nt][k] = act.h2[mt][nt][k] > 0.f ? d2[mt][nt][k] : 0.f;
       }
@@ -262,13 +278,13 @@ __device__ __forceinline__ void backward_warp(const Weights &W, WarpStage &S, in
 #pragma unroll
     for (int mt = 0; mt < 2; ++mt) {
       uint32_t ahi[4], alo[4];
-      a_from_c(d2[mt][0], d2[mt][1], ahi, alo);
+      a_from_c<kSplit>(d2[mt][0], d2[mt][1], ahi, alo);
 #pragma unroll
       for (int nt = 0; nt < 2; ++nt) {
 #pragma unroll
         for (int k = 0; k < 4; ++k) d1[mt][nt][k] = 0.f;
         mma16816(d1[mt][nt], ahi, b0[nt], b1[nt]);
-        mma16816(d1[mt][nt], alo, b0[nt], b1[nt]);
+        if (kSplit) mma16816(d1[mt][nt], alo, b0[nt], b1[nt]);
 #pragma unroll
         for (int k = 0; k < 4; ++k) d1[mt][nt][k] = act.h1[mt][nt][k] > 0.f ? d1[mt][nt][k] : 0.f;
       }
@@ -280,7 +296,7 @@ __device__ __forceinline__ void backward_warp(const Weights &W, WarpStage &S, in
 #pragma unroll
     for (int mt = 0; mt < 2; ++mt) {
       uint32_t ahi[4], alo[4];
-      a_from_c(d1[mt][0], d1[mt][1], ahi, alo);
+      a_from_c<kSplit>(d1[mt][0], d1[mt][1], ahi, alo);
       const int r0 = 16 * mt + g, r1 = r0 + 8;
 #pragma unroll
       for (int nt = 0; nt < 4; ++nt) {
@@ -288,15 +304,15 @@ __device__ __forceinline__ void backward_warp(const Weights &W, WarpStage &S, in
         const uint32_t b0 = w1t[word], b1 = w1t[word + 4];
         float c[4] = {0.f, 0.f, 0.f, 0.f};
         mma16816(c, ahi, b0, b1);
-        mma16816(c, alo, b0, b1);
+        if (kSplit) mma16816(c, alo, b0, b1);
         if (nt < 2) {
           *reinterpret_cast<float2 *>(S.gx + r0 * kGxStride + 8 * nt + 2 * t) = make_float2(c[0], c[1]);
           *reinterpret_cast<float2 *>(S.gx + r1 * kGxStride + 8 * nt + 2 * t) = make_float2(c[2], c[3]);
         } else {
           // columns 16 + 2j, 17 + 2j are (sin f_j, cos f_j) with j = 4 (nt - 2) + t
           const int j = 4 * (nt - 2) + t;
-          const float2 sc0 = unsplit(S.xhi[r0 * kXStride + 8 + j], S.xlo[r0 * kXStride + 8 + j]);
-          const float2 sc1 = unsplit(S.xhi[r1 * kXStride + 8 + j], S.xlo[r1 * kXStride + 8 + j]);
+          const float2 sc0 = unsplit(S.xhi[r0 * kXStride + 8 + j], kSplit ? S.xlo[r0 * kXStride + 8 + j] : 0u);
+          const float2 sc1 = unsplit(S.xhi[r1 * kXStride + 8 + j], kSplit ? S.xlo[r1 * kXStride + 8 + j] : 0u);
           S.gf[r0 * 8 + j] = c[0] * sc0.y - c[1] * sc0.x;
           S.gf[r1 * 8 + j] = c[2] * sc1.y - c[3] * sc1.x;
         }
@@ -311,15 +327,15 @@ __device__ __forceinline__ void backward_warp(const Weights &W, WarpStage &S, in
       uint32_t ahi[4] = {0u, 0u, 0u, 0u}, alo[4] = {0u, 0u, 0u, 0u};
       if (g < 3) {
         const int ra = (16 * ks + 2 * t) * 4 + g;
-        split2(S.y[ra], S.y[ra + 4], ahi[0], alo[0]);
-        split2(S.y[ra + 32], S.y[ra + 36], ahi[2], alo[2]);
+        split2<kSplit>(S.y[ra], S.y[ra + 4], ahi[0], alo[0]);
+        split2<kSplit>(S.y[ra + 32], S.y[ra + 36], ahi[2], alo[2]);
       }
 #pragma unroll
       for (int nt = 0; nt < 2; ++nt) {
         uint32_t th, tl, bh, bl;
-        split2(act.h2[ks][nt][0], act.h2[ks][nt][1], th, tl);
-        split2(act.h2[ks][nt][2], act.h2[ks][nt][3], bh, bl);
-        mma3(dW.w3[nt], ahi, alo, movm_trans(th), movm_trans(bh), movm_trans(tl), movm_trans(bl));
+        split2<kSplit>(act.h2[ks][nt][0], act.h2[ks][nt][1], th, tl);
+        split2<kSplit>(act.h2[ks][nt][2], act.h2[ks][nt][3], bh, bl);
+        mma3<kSplit>(dW.w3[nt], ahi, alo, movm_trans(th), movm_trans(bh), movm_lo<kSplit>(tl), movm_lo<kSplit>(bl));
       }
     }
     // dW2 += d2^T H1
@@ -327,17 +343,17 @@ __device__ __forceinline__ void backward_warp(const Weights &W, WarpStage &S, in
       uint32_t ahi[4], alo[4];
       {
         uint32_t h, l;
-        split2(d2[ks][0][0], d2[ks][0][1], h, l); ahi[0] = movm_trans(h); alo[0] = movm_trans(l);
-        split2(d2[ks][1][0], d2[ks][1][1], h, l); ahi[1] = movm_trans(h); alo[1] = movm_trans(l);
-        split2(d2[ks][0][2], d2[ks][0][3], h, l); ahi[2] = movm_trans(h); alo[2] = movm_trans(l);
-        split2(d2[ks][1][2], d2[ks][1][3], h, l); ahi[3] = movm_trans(h); alo[3] = movm_trans(l);
+        split2<kSplit>(d2[ks][0][0], d2[ks][0][1], h, l); ahi[0] = movm_trans(h); alo[0] = movm_lo<kSplit>(l);
+        split2<kSplit>(d2[ks][1][0], d2[ks][1][1], h, l); ahi[1] = movm_trans(h); alo[1] = movm_lo<kSplit>(l);
+        split2<kSplit>(d2[ks][0][2], d2[ks][0][3], h, l); ahi[2] = movm_trans(h); alo[2] = movm_lo<kSplit>(l);
+        split2<kSplit>(d2[ks][1][2], d2[ks][1][3], h, l); ahi[3] = movm_trans(h); alo[3] = movm_lo<kSplit>(l);
       }
 #pragma unroll
       for (int nt = 0; nt < 2; ++nt) {
         uint32_t th, tl, bh, bl;
-        split2(act.h1[ks][nt][0], act.h1[ks][nt][1], th, tl);
-        split2(act.h1[ks][nt][2], act.h1[ks][nt][3], bh, bl);
-        mma3(dW.w2[nt], ahi, alo, movm_trans(th), movm_trans(bh), movm_trans(tl), movm_trans(bl));
+        split2<kSplit>(act.h1[ks][nt][0], act.h1[ks][nt][1], th, tl);
+        split2<kSplit>(act.h1[ks][nt][2], act.h1[ks][nt][3], bh, bl);
+        mma3<kSplit>(dW.w2[nt], ahi, alo, movm_trans(th), movm_trans(bh), movm_lo<kSplit>(tl), movm_lo<kSplit>(bl));
       }
     }
     // dW1 += d1^T X
@@ -345,17 +361,17 @@ __device__ __forceinline__ void backward_warp(const Weights &W, WarpStage &S, in
       uint32_t ahi[4], alo[4];
       {
         uint32_t h, l;
-        split2(d1[ks][0][0], d1[ks][0][1], h, l); ahi[0] = movm_trans(h); alo[0] = movm_trans(l);
-        split2(d1[ks][1][0], d1[ks][1][1], h, l); ahi[1] = movm_trans(h); alo[1] = movm_trans(l);
-        split2(d1[ks][0][2], d1[ks][0][3], h, l); ahi[2] = movm_trans(h); alo[2] = movm_trans(l);
-        split2(d1[ks][1][2], d1[ks][1][3], h, l); ahi[3] = movm_trans(h); alo[3] = movm_trans(l);
+        split2<kSplit>(d1[ks][0][0], d1[ks][0][1], h, l); ahi[0] = movm_trans(h); alo[0] = movm_lo<kSplit>(l);
+        split2<kSplit>(d1[ks][1][0], d1[ks][1][1], h, l); ahi[1] = movm_trans(h); alo[1] = movm_lo<kSplit>(l);
+        split2<kSplit>(d1[ks][0][2], d1[ks][0][3], h, l); ahi[2] = movm_trans(h); alo[2] = movm_lo<kSplit>(l);
+        split2<kSplit>(d1[ks][1][2], d1[ks][1][3], h, l); ahi[3] = movm_trans(h); alo[3] = movm_lo<kSplit>(l);
       }
 #pragma unroll
       for (int nt = 0; nt < 4; ++nt) {
         // the 8 x 8 tile X[rows 16ks + (0..7 | 8..15)][cols 8nt .. 8nt+7] as packed pairs, then transposed
         const int r0 = (16 * ks + g) * kXStride + 4 * nt + t, r1 = r0 + 8 * kXStride;
-        mma3(dW.w1[nt], ahi, alo, movm_trans(S.xhi[r0]), movm_trans(S.xhi[r1]), movm_trans(S.xlo[r0]),
-             movm_trans(S.xlo[r1]));
+        mma3<kSplit>(dW.w1[nt], ahi, alo, movm_trans(S.xhi[r0]), movm_trans(S.xhi[r1]), movm_lo<kSplit>(kSplit ? S.xlo[r0] : 0u),
+                     movm_lo<kSplit>(kSplit ? S.xlo[r1] : 0u));
       }
     }
   }

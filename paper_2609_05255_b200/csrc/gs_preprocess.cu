@@ -21,6 +21,10 @@ constexpr int kWarps = kBlock / 32;
 template <int APP> struct RowOf { static constexpr int value = APP == GS_APP_SV ? GS_SV_ROW : GS_SH_REST; };
 template <int APP> struct SlabOf { static constexpr int value = 32 * RowOf<APP>::value; };
 template <int APP> struct Explicit { static constexpr bool value = APP == GS_APP_SH || APP == GS_APP_SV; };
+// The neural model in either precision of its decoder's products: fp16 operands split into two halves (results as
+// accurate as fp32 FMAs, the default), or plain fp16 operands as the paper runs it (kAppNeuralHalf).
+template <int APP> struct IsNeural { static constexpr bool value = APP == GS_APP_NEURAL || APP == kAppNeuralHalf; };
+template <int APP> struct Split { static constexpr bool value = APP != kAppNeuralHalf; };
 constexpr unsigned kFull = 0xffffffffu;
 
 __device__ __forceinline__ bool finite_f(float x) { return fabsf(x) <= FLT_MAX; }
@@ -212,11 +216,11 @@ struct __align__(16) StageFwd {
 
 // Whole-warp decode: every lane passes its Gaussian's inputs (zeros if it has none) and gets the
 // tanh-bounded residual A back.  All 32 lanes must call it.
-template <class Stage>
+template <bool kSplit, class Stage>
 __device__ __forceinline__ void decode_warp(const mlp::Weights &W, Stage &S, int lane, const float x[32],
                                             mlp::Activations &act, float A[3]) {
-  mlp::stage_inputs(x, S, lane);
-  mlp::forward_warp(W, S, lane, act);
+  mlp::stage_inputs<kSplit>(x, S, lane);
+  mlp::forward_warp<kSplit>(W, S, lane, act);
 #pragma unroll
   for (int c = 0; c < 3; ++c) A[c] = tanhf(S.y[lane * 4 + c]);
 }
@@ -224,13 +228,14 @@ __device__ __forceinline__ void decode_warp(const mlp::Weights &W, Stage &S, int
 // Whole-warp backward of the decoder.  `has`: this lane owns a Gaussian (inputs x, direction d, base
 // colour, dL/dcolour gcol); lanes without one pass zeros.  Returns the colour gradient through the activation
 // gp, dL/df and dL/dd of the lane's Gaussian and advances the warp's weight-gradient fragments.
+template <bool kSplit>
 __device__ __forceinline__ void decode_backward_warp(const mlp::Weights &W, mlp::WarpStage &S, int lane, bool has,
                                                      const float x[32], float dx, float dy, float dz, int deg, int cact,
                                                      const float base[3], const float gcol[3], mlp::WeightGrad &dW,
                                                      float gp[3], float gf[8], float gd[3]) {
   mlp::Activations act;
   float A[3];
-  decode_warp(W, S, lane, x, act, A);
+  decode_warp<kSplit>(W, S, lane, x, act, A);
   float gy[3];
 #pragma unroll
   for (int c = 0; c < 3; ++c) {
@@ -238,7 +243,7 @@ __device__ __forceinline__ void decode_backward_warp(const mlp::Weights &W, mlp:
     gy[c] = gp[c] * (1.f - A[c] * A[c]);
   }
   *reinterpret_cast<float4 *>(S.y + lane * 4) = make_float4(gy[0], gy[1], gy[2], 0.f);
-  mlp::backward_warp(W, S, lane, act, dW);
+  mlp::backward_warp<kSplit>(W, S, lane, act, dW);
   const float4 f0 = *reinterpret_cast<const float4 *>(S.gf + lane * 8), f1 = *reinterpret_cast<const float4 *>(S.gf + lane * 8 + 4);
   gf[0] = f0.x; gf[1] = f0.y; gf[2] = f0.z; gf[3] = f0.w; gf[4] = f1.x; gf[5] = f1.y; gf[6] = f1.z; gf[7] = f1.w;
   float gx[16];
@@ -409,12 +414,12 @@ __device__ __forceinline__ void load3(const float *p, int64_t i, float v[3]) {
 template <int APP>
 __global__ void __launch_bounds__(kBlock) k_preprocess_fwd(PreprocessArgs a, CamDev cam) {
   __shared__ __align__(16) float sData[Explicit<APP>::value ? kWarps * SlabOf<APP>::value : 4];
-  __shared__ __align__(16) unsigned char sNN[APP == GS_APP_NEURAL ? sizeof(mlp::Weights) + kWarps * sizeof(StageFwd) : 16];
+  __shared__ __align__(16) unsigned char sNN[IsNeural<APP>::value ? sizeof(mlp::Weights) + kWarps * sizeof(StageFwd) : 16];
   mlp::Weights *sWt = reinterpret_cast<mlp::Weights *>(sNN);
-  StageFwd *sStage = reinterpret_cast<StageFwd *>(sNN + (APP == GS_APP_NEURAL ? sizeof(mlp::Weights) : 0));   // unused for SH
+  StageFwd *sStage = reinterpret_cast<StageFwd *>(sNN + (IsNeural<APP>::value ? sizeof(mlp::Weights) : 0));   // unused for SH
   __shared__ unsigned int sPairs[kWarps];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (APP == GS_APP_NEURAL) {
+  if (IsNeural<APP>::value) {
     mlp::load_weights(a.weights, sWt[0], tid, kBlock);
     __syncthreads();
   }
@@ -453,7 +458,7 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_fwd(PreprocessArgs a, Cam
       SvCarry cy;
       explicit_pre<APP>(slab + lane * RowOf<APP>::value, base, g.dirx, g.diry, g.dirz, a.deg, pre, cy);
     }
-  } else if (APP == GS_APP_NEURAL) {
+  } else if (IsNeural<APP>::value) {
     float A[3] = {0.f, 0.f, 0.f};
     if (a.deg > 0 && __any_sync(kFull, vis)) {   // the whole warp decodes; culled lanes feed zeros
       float x[32];
@@ -466,7 +471,7 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_fwd(PreprocessArgs a, Cam
         for (int k = 0; k < 32; ++k) x[k] = 0.f;
       }
       mlp::Activations act;
-      decode_warp(sWt[0], sStage[warp], lane, x, act, A);
+      decode_warp<Split<APP>::value>(sWt[0], sStage[warp], lane, x, act, A);
     }
     if (vis) {
       float base[3];
@@ -631,7 +636,7 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_bwd(PreprocessBwdArgs a, 
   mlp::Weights &sWt = *reinterpret_cast<mlp::Weights *>(smem);
   mlp::WarpStage *sStage = reinterpret_cast<mlp::WarpStage *>(reinterpret_cast<unsigned char *>(smem) + sizeof(mlp::Weights));
   mlp::WeightGrad dW;
-  if (APP == GS_APP_NEURAL) {
+  if (IsNeural<APP>::value) {
     mlp::load_weights(a.weights, sWt, tid, kBlock);
     dW.clear();
     __syncthreads();
@@ -662,7 +667,7 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_bwd(PreprocessBwdArgs a, 
       ga = g2[0]; gb = g2[1]; gc = g2[2];   // (gr, gg, gb, go) (gA, gB, gC, gu) (gv, -, -, -)
       if (APP != kAppExternal) load3(a.base_color, i, base_in);
       else load3(a.gd_in, i, gd);
-      if (APP == GS_APP_NEURAL) feat_raw = __ldg(reinterpret_cast<const uint4 *>(a.features) + i);
+      if (IsNeural<APP>::value) feat_raw = __ldg(reinterpret_cast<const uint4 *>(a.features) + i);
       q[0] = q4.x; q[1] = q4.y; q[2] = q4.z; q[3] = q4.w;
       vis = rc.z > rc.x && rc.w > rc.y;
     }
@@ -712,7 +717,7 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_bwd(PreprocessBwdArgs a, 
 #pragma unroll
           for (int k = 0; k < 32; ++k) x[k] = 0.f;
         }
-        decode_backward_warp(sWt, sStage[warp], lane, vis, x, dx, dy, dz, a.deg, a.act, base, gcol, dW, gp, gf, gd);
+        decode_backward_warp<Split<APP>::value>(sWt, sStage[warp], lane, vis, x, dx, dy, dz, a.deg, a.act, base, gcol, dW, gp, gf, gd);
       } else if (vis) {
 #pragma unroll
         for (int c = 0; c < 3; ++c) gp[c] = color_act_grad_z(a.act, base[c] + 0.5f) * gcol[c];
@@ -742,7 +747,7 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_bwd(PreprocessBwdArgs a, 
       if (APP != kAppExternal) store3(a.g_base, i, gp[0], gp[1], gp[2]);
     }
   }
-  if (APP == GS_APP_NEURAL) {
+  if (IsNeural<APP>::value) {
     weight_grad_flush(dW, reinterpret_cast<float *>(sStage), a.w_partials + (size_t)blockIdx.x * GS_MLP_WEIGHTS, tid);
   }
 }
@@ -750,12 +755,12 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_bwd(PreprocessBwdArgs a, 
 // ---- separate-pass appearance kernels ---------------------------------------------------------
 template <int APP>
 __global__ void __launch_bounds__(kBlock) k_appearance_fwd(AppearanceArgs a) {
-  __shared__ __align__(16) float sData[APP != GS_APP_NEURAL ? kWarps * SlabOf<APP>::value : 4];
-  __shared__ __align__(16) unsigned char sNN[APP == GS_APP_NEURAL ? sizeof(mlp::Weights) + kWarps * sizeof(StageFwd) : 16];
+  __shared__ __align__(16) float sData[!IsNeural<APP>::value ? kWarps * SlabOf<APP>::value : 4];
+  __shared__ __align__(16) unsigned char sNN[IsNeural<APP>::value ? sizeof(mlp::Weights) + kWarps * sizeof(StageFwd) : 16];
   mlp::Weights *sWt = reinterpret_cast<mlp::Weights *>(sNN);
-  StageFwd *sStage = reinterpret_cast<StageFwd *>(sNN + (APP == GS_APP_NEURAL ? sizeof(mlp::Weights) : 0));   // unused for SH
+  StageFwd *sStage = reinterpret_cast<StageFwd *>(sNN + (IsNeural<APP>::value ? sizeof(mlp::Weights) : 0));   // unused for SH
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (APP == GS_APP_NEURAL) {
+  if (IsNeural<APP>::value) {
     mlp::load_weights(a.weights, sWt[0], tid, kBlock);
     __syncthreads();
   }
@@ -764,7 +769,7 @@ __global__ void __launch_bounds__(kBlock) k_appearance_fwd(AppearanceArgs a) {
   const bool in = i < a.n && (!a.mask || __ldg(a.mask + i) != 0u);   // masked-out Gaussians are skipped
   float d[3] = {0.f, 0.f, 1.f}, base[3] = {0.f, 0.f, 0.f}, pre[3];
   if (in) { load3(a.dirs, i, d); load3(a.base_color, i, base); }
-  if (APP != GS_APP_NEURAL) {
+  if (!IsNeural<APP>::value) {
     float *slab = sData + warp * SlabOf<APP>::value;
     if (a.deg > 0 && row0 < a.n) warp_load_rows<RowOf<APP>::value>(a.sh_rest, row0, a.n, slab, lane);
     SvCarry cy;
@@ -782,7 +787,7 @@ __global__ void __launch_bounds__(kBlock) k_appearance_fwd(AppearanceArgs a) {
         for (int k = 0; k < 32; ++k) x[k] = 0.f;
       }
       mlp::Activations act;
-      decode_warp(sWt[0], sStage[warp], lane, x, act, A);
+      decode_warp<Split<APP>::value>(sWt[0], sStage[warp], lane, x, act, A);
     }
 #pragma unroll
     for (int c = 0; c < 3; ++c) pre[c] = base[c] + 0.5f + A[c];
@@ -798,7 +803,7 @@ __global__ void __launch_bounds__(kBlock) k_appearance_bwd(AppearanceArgs a) {
   mlp::Weights &sWt = *reinterpret_cast<mlp::Weights *>(smem);
   mlp::WarpStage *sStage = reinterpret_cast<mlp::WarpStage *>(reinterpret_cast<unsigned char *>(smem) + sizeof(mlp::Weights));
   mlp::WeightGrad dW;
-  if (APP == GS_APP_NEURAL) {
+  if (IsNeural<APP>::value) {
     mlp::load_weights(a.weights, sWt, tid, kBlock);
     dW.clear();
     __syncthreads();
@@ -813,7 +818,7 @@ __global__ void __launch_bounds__(kBlock) k_appearance_bwd(AppearanceArgs a) {
     float d[3] = {0.f, 0.f, 1.f}, base[3] = {0.f, 0.f, 0.f}, gcol[3] = {0.f, 0.f, 0.f};
     if (in) { load3(a.dirs, i, d); load3(a.base_color, i, base); load3(a.g_color, i, gcol); }
     float gp[3] = {0.f, 0.f, 0.f}, gd[3] = {0.f, 0.f, 0.f};
-    if (APP != GS_APP_NEURAL) {
+    if (!IsNeural<APP>::value) {
       if (row0 < a.n) {
         if (a.deg > 0) warp_load_rows<RowOf<APP>::value>(a.sh_rest, row0, a.n, slab, lane);
         float *row = slab + lane * RowOf<APP>::value;
@@ -843,7 +848,7 @@ __global__ void __launch_bounds__(kBlock) k_appearance_bwd(AppearanceArgs a) {
 #pragma unroll
           for (int k = 0; k < 32; ++k) x[k] = 0.f;
         }
-        decode_backward_warp(sWt, sStage[warp], lane, in, x, d[0], d[1], d[2], a.deg, a.act, base, gcol, dW, gp, gf, gd);
+        decode_backward_warp<Split<APP>::value>(sWt, sStage[warp], lane, in, x, d[0], d[1], d[2], a.deg, a.act, base, gcol, dW, gp, gf, gd);
       } else if (in) {
 #pragma unroll
         for (int c = 0; c < 3; ++c) gp[c] = color_act_grad_z(a.act, base[c] + 0.5f) * gcol[c];
@@ -859,7 +864,7 @@ __global__ void __launch_bounds__(kBlock) k_appearance_bwd(AppearanceArgs a) {
       store3(a.g_dirs, i, gd[0], gd[1], gd[2]);
     }
   }
-  if (APP == GS_APP_NEURAL) {
+  if (IsNeural<APP>::value) {
     weight_grad_flush(dW, reinterpret_cast<float *>(sStage), a.w_partials + (size_t)blockIdx.x * GS_MLP_WEIGHTS, tid);
   }
 }
@@ -1051,6 +1056,7 @@ int launch_preprocess_fwd(int app, const PreprocessArgs &a, const CamDev &cam, c
   if (app == GS_APP_SH) k_preprocess_fwd<GS_APP_SH><<<grid_for(a.n), kBlock, 0, st>>>(a, cam);
   else if (app == GS_APP_SV) k_preprocess_fwd<GS_APP_SV><<<grid_for(a.n), kBlock, 0, st>>>(a, cam);
   else if (app == kAppExternal) k_preprocess_fwd<kAppExternal><<<grid_for(a.n), kBlock, 0, st>>>(a, cam);
+  else if (app == kAppNeuralHalf) k_preprocess_fwd<kAppNeuralHalf><<<grid_for(a.n), kBlock, 0, st>>>(a, cam);
   else k_preprocess_fwd<GS_APP_NEURAL><<<grid_for(a.n), kBlock, 0, st>>>(a, cam);
   return 1;
 }
@@ -1078,6 +1084,13 @@ int launch_preprocess_bwd(int app, const PreprocessBwdArgs &a, const CamDev &cam
     k_preprocess_bwd<kAppExternal><<<grid_for(a.n), kBlock, 16, st>>>(a, cam);
     return 1;
   } else {
+    if (app == kAppNeuralHalf) {
+      opt_in_smem(k_preprocess_bwd<kAppNeuralHalf>, kBwdSmemNN);
+      const int blocks = resident_blocks<k_preprocess_bwd<kAppNeuralHalf>>(kBwdSmemNN);
+      k_preprocess_bwd<kAppNeuralHalf><<<blocks, kBlock, kBwdSmemNN, st>>>(a, cam);
+      launch_wgrad_reduce(a.w_partials, blocks, a.g_weights, st);
+      return 2;
+    }
     opt_in_smem(k_preprocess_bwd<GS_APP_NEURAL>, kBwdSmemNN);
     const int blocks = resident_blocks<k_preprocess_bwd<GS_APP_NEURAL>>(kBwdSmemNN);
     k_preprocess_bwd<GS_APP_NEURAL><<<blocks, kBlock, kBwdSmemNN, st>>>(a, cam);
@@ -1099,7 +1112,8 @@ int launch_appearance_fwd(int app, const AppearanceArgs &a, cudaStream_t st) {
   if (a.n == 0) return 0;
   if (app == GS_APP_SH) return launch_bulk<GS_APP_SH, false>(a, st);
   if (app == GS_APP_SV) return launch_bulk<GS_APP_SV, false>(a, st);
-  k_appearance_fwd<GS_APP_NEURAL><<<grid_for(a.n), kBlock, 0, st>>>(a);
+  if (app == kAppNeuralHalf) k_appearance_fwd<kAppNeuralHalf><<<grid_for(a.n), kBlock, 0, st>>>(a);
+  else k_appearance_fwd<GS_APP_NEURAL><<<grid_for(a.n), kBlock, 0, st>>>(a);
   return 1;
 }
 
@@ -1111,6 +1125,13 @@ int launch_appearance_bwd(int app, const AppearanceArgs &a, cudaStream_t st) {
     if (a.n == 0) return 0;
     return launch_bulk<GS_APP_SV, true>(a, st);
   } else {
+    if (app == kAppNeuralHalf) {
+      opt_in_smem(k_appearance_bwd<kAppNeuralHalf>, kBwdSmemNN);
+      const int blocks = resident_blocks<k_appearance_bwd<kAppNeuralHalf>>(kBwdSmemNN);
+      k_appearance_bwd<kAppNeuralHalf><<<blocks, kBlock, kBwdSmemNN, st>>>(a);
+      launch_wgrad_reduce(a.w_partials, blocks, a.g_weights, st);
+      return 2;
+    }
     opt_in_smem(k_appearance_bwd<GS_APP_NEURAL>, kBwdSmemNN);
     const int blocks = resident_blocks<k_appearance_bwd<GS_APP_NEURAL>>(kBwdSmemNN);
     k_appearance_bwd<GS_APP_NEURAL><<<blocks, kBlock, kBwdSmemNN, st>>>(a);

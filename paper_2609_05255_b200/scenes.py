@@ -62,6 +62,7 @@ class Scene:
     mlp_hidden: int = 0                       # decoder variant: neurons per hidden layer (0 = the default 16)
     mlp_layers: int = 0                       # decoder variant: hidden layers (0 = the default 2)
     separate_pass: int = 0                    # 1: ask the library for its unfused reference path (same results)
+    decoder_precision: int = 0                # 1: the decoder's products on plain fp16 operands (the paper's precision)
 
     @property
     def n(self) -> int:
