@@ -104,6 +104,28 @@ def test_decoder_variant_through_the_whole_step(oracle, arch):
             assert np.all(got[~gpu.visible] == 0)
 
 
+@pytest.mark.parametrize("app", [scenes.APP_SH, scenes.APP_NEURAL, scenes.APP_SV], ids=["sh", "neural", "sv"])
+@pytest.mark.parametrize("n", [0, 1, 33, 130])
+def test_unfused_step_on_tiny_scenes(oracle, app, n):
+    w = scenes.config2(n=max(n, 1), app=app)
+    sc, cam = w.scene, w.cameras[0]
+    if n == 0:
+        for f in ("means", "log_scales", "quats", "opacity_logits", "base_color", "sh_rest", "features", "sv_sites"):
+            if getattr(sc, f) is not None:
+                setattr(sc, f, getattr(sc, f)[:0])
+    sc.separate_pass = 1
+    sc.color_activation = 1                      # softplus, to go through the activation argument too
+    G = scenes.upstream_gradient(cam, 12)
+    gpu = run_gpu(sc, cam, G)
+    fwd, grads = oracle.render(sc, cam, G)
+    assert image_mismatch(gpu.image, fwd.image, fwd.fragile).sum() == 0
+    if n == 0:
+        return
+    for nm in grad_names(app):
+        got, want = getattr(gpu.grads, nm), getattr(grads, nm)
+        assert np.abs(got - want).max() <= max(2e-3 * np.abs(want).max(), GRAD_ATOL), nm
+
+
 def test_workspace_covers_the_separate_passes():
     from paper_2609_05255_b200 import api
     n = 100_000
