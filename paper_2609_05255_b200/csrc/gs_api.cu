@@ -463,6 +463,7 @@ GsStatus gs_render_backward(GsContext *ctx, const GsScene *scene, const GsCamera
   a.g_sh_rest = scene->app == GS_APP_SV ? grads->sv_sites : grads->sh_rest;
   a.g_features = grads->features; a.w_partials = ctx->d_w_partials; a.g_weights = grads->mlp_weights;
   a.gd_in = bw.g_dirs;
+  a.timeout = ctx->d_counter + 3;
   if (n == 0 && scene->app == GS_APP_NEURAL) {
     const DecoderArch d = decoder_arch(scene);
     return check_cuda(ctx, cudaMemsetAsync(grads->mlp_weights, 0, sizeof(float) * variant_num_weights(d.hidden, d.layers), s), "memset");

@@ -55,6 +55,38 @@ __device__ __forceinline__ void warp_store_rows(float *g, int64_t row0, int64_t 
   __syncwarp();
 }
 
+// ---- 1D bulk copies (tensor memory accelerator) with bounded waits ------------------------------------------
+// load(): one lane arms the warp's mbarrier with the byte count and starts the copy; wait(): every lane polls the
+// barrier's phase, at most about a second in all; store(): shared -> global as a bulk group of the issuing lane.
+namespace bulk {
+__device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void barrier_init(uint32_t bar) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity) {
+  for (int it = 0; it < (1 << 20); ++it) {   // each try sleeps at most about a microsecond: the wait ends within a second
+    uint32_t done;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(done) : "r"(bar), "r"(parity), "r"(1000u) : "memory");
+    if (done) return true;
+  }
+  return false;
+}
+__device__ __forceinline__ void store(void *dst, uint32_t src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes) : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void wait_stores_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void wait_stores_done() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_generic_writes() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+}  // namespace bulk
+
 // ---- appearance: SH -------------------------------------------------------------------------
 // colour = max(0, c0 + 0.5 + sum_k Y_k(d) c_k); row = this Gaussian's 45 coefficients in smem.
 __device__ __forceinline__ void sh_decode(const float *row, const float base[3], float dx, float dy,
@@ -418,6 +450,7 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_fwd(PreprocessArgs a, Cam
   mlp::Weights *sWt = reinterpret_cast<mlp::Weights *>(sNN);
   StageFwd *sStage = reinterpret_cast<StageFwd *>(sNN + (IsNeural<APP>::value ? sizeof(mlp::Weights) : 0));   // unused for SH
   __shared__ unsigned int sPairs[kWarps];
+  __shared__ unsigned long long sBar[kWarps];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (IsNeural<APP>::value) {
     mlp::load_weights(a.weights, sWt[0], tid, kBlock);
@@ -430,13 +463,31 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_fwd(PreprocessArgs a, Cam
   g.valid = false;
   int rect[4] = {0, 0, 0, 0};
   bool vis = false;
+  float mu[3] = {0.f, 0.f, 0.f}, ls[3] = {0.f, 0.f, 0.f}, q[4] = {1.f, 0.f, 0.f, 0.f}, logit = 0.f;
   if (in) {
-    float mu[3], ls[3];
     load3(a.means, i, mu);
     load3(a.log_scales, i, ls);
     const float4 q4 = __ldg(reinterpret_cast<const float4 *>(a.quats) + i);
-    const float q[4] = {q4.x, q4.y, q4.z, q4.w};
-    g = project(mu, ls, q, __ldg(a.logits + i), cam);
+    q[0] = q4.x; q[1] = q4.y; q[2] = q4.z; q[3] = q4.w;
+    logit = __ldg(a.logits + i);
+  }
+  // SH / Spherical Voronoi: the warp's slab of parameter rows is one contiguous piece of memory.  Unless the depth
+  // test already culls the whole warp, a bulk copy brings it in while the projection below runs (a ragged last
+  // warp uses plain loads further down).
+  bool slab_by_copy = false;
+  if (Explicit<APP>::value && a.deg > 0 && row0 + 32 <= a.n) {
+    const float z = __fmaf_rn(cam.R[8], mu[2], __fmaf_rn(cam.R[7], mu[1], __fmaf_rn(cam.R[6], mu[0], cam.t[2])));
+    slab_by_copy = __any_sync(kFull, z >= cam.near_plane && z <= cam.far_plane);
+    if (slab_by_copy && lane == 0) {
+      const uint32_t bar = bulk::smem_addr(sBar + warp);
+      bulk::barrier_init(bar);
+      bulk::fence_barrier_init();
+      bulk::load(bulk::smem_addr(sData + warp * SlabOf<APP>::value), a.sh_rest + row0 * RowOf<APP>::value,
+                 SlabOf<APP>::value * sizeof(float), bar);
+    }
+  }
+  if (in) {
+    g = project(mu, ls, q, logit, cam);
     if (g.valid) vis = tile_rect(g.u, g.v, g.ex, g.ey, cam, rect);
   }
   // tiles the ellipse really meets inside its bounding rectangle
@@ -451,8 +502,15 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_fwd(PreprocessArgs a, Cam
   float pre[3] = {0.f, 0.f, 0.f};
   if (Explicit<APP>::value) {   // SH or Spherical Voronoi: parameter rows through the warp's slab
     float *slab = sData + warp * SlabOf<APP>::value;
-    if (__any_sync(kFull, vis) && a.deg > 0 && row0 < a.n) warp_load_rows<RowOf<APP>::value>(a.sh_rest, row0, a.n, slab, lane);
-    if (vis) {
+    bool arrived = true;
+    if (slab_by_copy) {
+      __syncwarp();                         // lane 0 has initialised the barrier
+      arrived = __all_sync(kFull, bulk::wait(bulk::smem_addr(sBar + warp), 0u));
+      if (!arrived && lane == 0) atomicExch(a.pair_counter + 3, 1ull);   // reported by gs_async_status
+    } else if (__any_sync(kFull, vis) && a.deg > 0 && row0 + 32 > a.n) {   // the ragged last warp
+      warp_load_rows<RowOf<APP>::value>(a.sh_rest, row0, a.n, slab, lane);
+    }
+    if (vis && arrived) {
       float base[3];
       load3(a.base_color, i, base);
       SvCarry cy;
@@ -641,6 +699,15 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_bwd(PreprocessBwdArgs a, 
     dW.clear();
     __syncthreads();
   }
+  // SH / Spherical Voronoi: the warp's slab of parameter rows comes in by one bulk copy and its slab of gradient
+  // rows leaves by one (a ragged last warp uses plain loads and stores)
+  __shared__ unsigned long long sBar[kWarps];
+  uint32_t slab_parity = 0u;
+  if (Explicit<APP>::value && lane == 0) {
+    bulk::barrier_init(bulk::smem_addr(sBar + warp));
+    bulk::fence_barrier_init();
+  }
+  __syncwarp();
   const int64_t nchunks = (a.n + kBlock - 1) / kBlock;
   for (int64_t chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x) {
     reload_fence();
@@ -672,6 +739,15 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_bwd(PreprocessBwdArgs a, 
       vis = rc.z > rc.x && rc.w > rc.y;
     }
     const bool warp_vis = __any_sync(kFull, vis);
+    const bool full_warp = row0 + 32 <= a.n;
+    const bool slab_by_copy = Explicit<APP>::value && warp_vis && a.deg > 0 && full_warp;
+    if (Explicit<APP>::value && lane == 0) {
+      bulk::wait_stores_read();          // an earlier trip's gradient slab has left shared memory
+      if (slab_by_copy)
+        bulk::load(bulk::smem_addr(slab), a.sh_rest + row0 * RowOf<APP>::value, SlabOf<APP>::value * sizeof(float),
+                   bulk::smem_addr(sBar + warp));
+    }
+    if (Explicit<APP>::value) __syncwarp();
     if (vis) {
       const float vx = mu[0] - cam.oc[0], vy = mu[1] - cam.oc[1], vz = mu[2] - cam.oc[2];
       const float vi = rsqrtf(vx * vx + vy * vy + vz * vz);
@@ -683,11 +759,16 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_bwd(PreprocessBwdArgs a, 
       // dL/dd came from the separate appearance backward (zero rows for culled Gaussians)
     } else if (Explicit<APP>::value) {
       if (row0 < a.n) {
-        if (warp_vis && a.deg > 0) {
+        bool arrived = true;
+        if (slab_by_copy) {
+          arrived = __all_sync(kFull, bulk::wait(bulk::smem_addr(sBar + warp), slab_parity));
+          slab_parity ^= 1u;
+          if (!arrived && lane == 0 && a.timeout) atomicExch(a.timeout, 1ull);   // reported by gs_async_status
+        } else if (warp_vis && a.deg > 0) {
           warp_load_rows<RowOf<APP>::value>(a.sh_rest, row0, a.n, slab, lane);
         }
         float *row = slab + lane * RowOf<APP>::value;
-        if (vis) {
+        if (vis && arrived) {
           float pre[3];
           const float (&base)[3] = base_in;
           SvCarry cy;
@@ -700,7 +781,13 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_bwd(PreprocessBwdArgs a, 
 #pragma unroll
           for (int k = 0; k < RowOf<APP>::value; ++k) row[k] = 0.f;
         }
-        warp_store_rows<RowOf<APP>::value>(a.g_sh_rest, row0, a.n, slab, lane);
+        if (full_warp) {
+          bulk::fence_generic_writes();     // the lanes' rows become visible to the copy engine
+          __syncwarp();
+          if (lane == 0) bulk::store(a.g_sh_rest + row0 * RowOf<APP>::value, bulk::smem_addr(slab), SlabOf<APP>::value * sizeof(float));
+        } else {
+          warp_store_rows<RowOf<APP>::value>(a.g_sh_rest, row0, a.n, slab, lane);
+        }
       }
     } else {
       float gf[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
@@ -750,6 +837,7 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_bwd(PreprocessBwdArgs a, 
   if (IsNeural<APP>::value) {
     weight_grad_flush(dW, reinterpret_cast<float *>(sStage), a.w_partials + (size_t)blockIdx.x * GS_MLP_WEIGHTS, tid);
   }
+  if (Explicit<APP>::value && lane == 0) bulk::wait_stores_done();
 }
 
 // ---- separate-pass appearance kernels ---------------------------------------------------------
@@ -877,34 +965,6 @@ __global__ void __launch_bounds__(kBlock) k_appearance_bwd(AppearanceArgs a) {
 // persistent, so the copy of its next 32 rows is in flight while it works on the current ones, with no
 // registers or store instructions spent on staging.  Every wait is bounded: if a barrier does not flip within
 // the limit the warp records it in *timeout and leaves, draining its own copies first.
-namespace bulk {
-__device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void barrier_init(uint32_t bar) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
-__device__ __forceinline__ void load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-__device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity) {
-  for (int it = 0; it < (1 << 20); ++it) {   // each try sleeps at most about a microsecond: the wait ends within a second
-    uint32_t done;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(done) : "r"(bar), "r"(parity), "r"(1000u) : "memory");
-    if (done) return true;
-  }
-  return false;
-}
-__device__ __forceinline__ void store(void *dst, uint32_t src, uint32_t bytes) {
-  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes) : "memory");
-  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-}
-__device__ __forceinline__ void wait_stores_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-__device__ __forceinline__ void wait_stores_done() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void fence_generic_writes() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-}  // namespace bulk
 
 template <int APP> constexpr size_t bulk_smem_bytes() {
   return sizeof(float) * kWarps * 2 * SlabOf<APP>::value + sizeof(unsigned long long) * kWarps * 2;
