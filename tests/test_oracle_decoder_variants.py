@@ -90,3 +90,28 @@ def test_gradients_by_finite_differences(oracle, hidden, layers, nfeat):
             vals.append(float((oracle.decoder_forward(sc, d) * gcol).sum()))
         fd = (vals[0] - vals[1]) / (2 * h)
         assert abs(fd - out.dirs[i, c]) < 2e-6 * max(1.0, abs(fd))
+
+
+@pytest.mark.parametrize("arch", [(32, 1, 16), (16, 3, 8)], ids=lambda a: "h%d_l%d_f%d" % a)
+def test_whole_step_with_a_variant_against_finite_differences(oracle, arch):
+    """The oracle's rendering step composes projection, appearance and blend; with a decoder of another size the
+    composition calls the generic decoder.  Central differences of the image loss pin that composition: features,
+    decoder weights and means (whose gradient carries the direction term of the decoder)."""
+    import test_oracle_gradients as og
+    hidden, layers, nfeat = arch
+    sc = og.tiny_scene(1, seed=31)
+    rng = np.random.default_rng(77)
+    sc.features = rng.normal(0, 0.7, (sc.means.shape[0], nfeat))
+    sc.mlp_weights = rng.uniform(-0.6, 0.6, oracle.decoder_num_weights(hidden, layers))
+    sc.mlp_hidden, sc.mlp_layers = hidden, layers
+    cam = og.tiny_cam(None)
+    G = np.random.default_rng(98).standard_normal((3, cam.height, cam.width))
+    fwd, grads = oracle.render(sc, cam, G)
+    assert fwd.pre.visible.sum() >= 10
+    assert grads.features.shape == (sc.means.shape[0], nfeat)
+    assert grads.mlp_weights.shape == (oracle.decoder_num_weights(hidden, layers),)
+    for name, stride in (("features", 1), ("mlp_weights", 7), ("means", 1), ("base_color", 1)):
+        checked, skipped, bad, worst, gmax = og.fd_check(oracle, sc, cam, G, [name], stride=stride)[name]
+        assert gmax > 1e-3, (name, gmax)
+        assert bad == 0, (name, checked, skipped, bad, worst)
+        assert skipped <= 0.1 * (checked + skipped), (name, checked, skipped)
