@@ -840,62 +840,50 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_bwd(PreprocessBwdArgs a, 
   if (Explicit<APP>::value && lane == 0) bulk::wait_stores_done();
 }
 
-// ---- separate-pass appearance kernels ---------------------------------------------------------
+// ---- separate-pass appearance kernels of the neural model (the explicit models follow, with bulk copies) ------
 template <int APP>
 __global__ void __launch_bounds__(kBlock) k_appearance_fwd(AppearanceArgs a) {
-  __shared__ __align__(16) float sData[!IsNeural<APP>::value ? kWarps * SlabOf<APP>::value : 4];
-  __shared__ __align__(16) unsigned char sNN[IsNeural<APP>::value ? sizeof(mlp::Weights) + kWarps * sizeof(StageFwd) : 16];
+  static_assert(IsNeural<APP>::value, "the neural model in either decoder precision");
+  __shared__ __align__(16) unsigned char sNN[sizeof(mlp::Weights) + kWarps * sizeof(StageFwd)];
   mlp::Weights *sWt = reinterpret_cast<mlp::Weights *>(sNN);
-  StageFwd *sStage = reinterpret_cast<StageFwd *>(sNN + (IsNeural<APP>::value ? sizeof(mlp::Weights) : 0));   // unused for SH
+  StageFwd *sStage = reinterpret_cast<StageFwd *>(sNN + sizeof(mlp::Weights));
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (IsNeural<APP>::value) {
-    mlp::load_weights(a.weights, sWt[0], tid, kBlock);
-    __syncthreads();
-  }
+  mlp::load_weights(a.weights, sWt[0], tid, kBlock);
+  __syncthreads();
   const int64_t i = (int64_t)blockIdx.x * kBlock + tid;
   const int64_t row0 = (int64_t)blockIdx.x * kBlock + warp * 32;
   const bool in = i < a.n && (!a.mask || __ldg(a.mask + i) != 0u);   // masked-out Gaussians are skipped
-  float d[3] = {0.f, 0.f, 1.f}, base[3] = {0.f, 0.f, 0.f}, pre[3];
+  float d[3] = {0.f, 0.f, 1.f}, base[3] = {0.f, 0.f, 0.f}, A[3] = {0.f, 0.f, 0.f};
   if (in) { load3(a.dirs, i, d); load3(a.base_color, i, base); }
-  if (!IsNeural<APP>::value) {
-    float *slab = sData + warp * SlabOf<APP>::value;
-    if (a.deg > 0 && row0 < a.n) warp_load_rows<RowOf<APP>::value>(a.sh_rest, row0, a.n, slab, lane);
-    SvCarry cy;
-    if (in) explicit_pre<APP>(slab + lane * RowOf<APP>::value, base, d[0], d[1], d[2], a.deg, pre, cy);
-  } else {
-    float A[3] = {0.f, 0.f, 0.f};
-    if (a.deg > 0 && row0 < a.n) {
-      float x[32];
-      if (in) {
-        float f[8];
-        load_features(a.features, i, f);
-        decoder_inputs(d[0], d[1], d[2], f, a.deg, x);
-      } else {
+  if (a.deg > 0 && row0 < a.n) {   // the whole warp decodes; lanes without a Gaussian feed zeros
+    float x[32];
+    if (in) {
+      float f[8];
+      load_features(a.features, i, f);
+      decoder_inputs(d[0], d[1], d[2], f, a.deg, x);
+    } else {
 #pragma unroll
-        for (int k = 0; k < 32; ++k) x[k] = 0.f;
-      }
-      mlp::Activations act;
-      decode_warp<Split<APP>::value>(sWt[0], sStage[warp], lane, x, act, A);
+      for (int k = 0; k < 32; ++k) x[k] = 0.f;
     }
-#pragma unroll
-    for (int c = 0; c < 3; ++c) pre[c] = base[c] + 0.5f + A[c];
+    mlp::Activations act;
+    decode_warp<Split<APP>::value>(sWt[0], sStage[warp], lane, x, act, A);
   }
-  if (in) store3(a.color, i, color_act_z(a.act, pre[0]), color_act_z(a.act, pre[1]), color_act_z(a.act, pre[2]));
+  if (in)
+    store3(a.color, i, color_act_z(a.act, base[0] + 0.5f + A[0]), color_act_z(a.act, base[1] + 0.5f + A[1]),
+           color_act_z(a.act, base[2] + 0.5f + A[2]));
 }
 
 template <int APP>
 __global__ void __launch_bounds__(kBlock) k_appearance_bwd(AppearanceArgs a) {
+  static_assert(IsNeural<APP>::value, "the neural model in either decoder precision");
   extern __shared__ __align__(16) float smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  float *slab = smem + warp * SlabOf<APP>::value;   // SH / SV: this warp's slab of parameter rows
   mlp::Weights &sWt = *reinterpret_cast<mlp::Weights *>(smem);
   mlp::WarpStage *sStage = reinterpret_cast<mlp::WarpStage *>(reinterpret_cast<unsigned char *>(smem) + sizeof(mlp::Weights));
   mlp::WeightGrad dW;
-  if (IsNeural<APP>::value) {
-    mlp::load_weights(a.weights, sWt, tid, kBlock);
-    dW.clear();
-    __syncthreads();
-  }
+  mlp::load_weights(a.weights, sWt, tid, kBlock);
+  dW.clear();
+  __syncthreads();
   const int64_t nchunks = (a.n + kBlock - 1) / kBlock;
   for (int64_t chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x) {
     reload_fence();
@@ -906,55 +894,31 @@ __global__ void __launch_bounds__(kBlock) k_appearance_bwd(AppearanceArgs a) {
     float d[3] = {0.f, 0.f, 1.f}, base[3] = {0.f, 0.f, 0.f}, gcol[3] = {0.f, 0.f, 0.f};
     if (in) { load3(a.dirs, i, d); load3(a.base_color, i, base); load3(a.g_color, i, gcol); }
     float gp[3] = {0.f, 0.f, 0.f}, gd[3] = {0.f, 0.f, 0.f};
-    if (!IsNeural<APP>::value) {
-      if (row0 < a.n) {
-        if (a.deg > 0) warp_load_rows<RowOf<APP>::value>(a.sh_rest, row0, a.n, slab, lane);
-        float *row = slab + lane * RowOf<APP>::value;
-        if (in) {
-          float pre[3];
-          SvCarry cy;
-          if (a.deg > 0) explicit_pre<APP>(row, base, d[0], d[1], d[2], a.deg, pre, cy);
-          else { pre[0] = base[0] + 0.5f; pre[1] = base[1] + 0.5f; pre[2] = base[2] + 0.5f; }
+    float gf[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    if (a.deg > 0 && row0 < a.n) {
+      float x[32];
+      if (in) {
+        float f[8];
+        load_features(a.features, i, f);
+        decoder_inputs(d[0], d[1], d[2], f, a.deg, x);
+      } else {
 #pragma unroll
-          for (int c = 0; c < 3; ++c) gp[c] = color_act_grad_z(a.act, pre[c]) * gcol[c];
-          explicit_bwd<APP>(row, gp, d[0], d[1], d[2], a.deg, cy, gd);
-        } else if (exists) {
-#pragma unroll
-          for (int k = 0; k < RowOf<APP>::value; ++k) row[k] = 0.f;
-        }
-        warp_store_rows<RowOf<APP>::value>(a.g_sh_rest, row0, a.n, slab, lane);
+        for (int k = 0; k < 32; ++k) x[k] = 0.f;
       }
-    } else {
-      float gf[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-      if (a.deg > 0 && row0 < a.n) {
-        float x[32];
-        if (in) {
-          float f[8];
-          load_features(a.features, i, f);
-          decoder_inputs(d[0], d[1], d[2], f, a.deg, x);
-        } else {
+      decode_backward_warp<Split<APP>::value>(sWt, sStage[warp], lane, in, x, d[0], d[1], d[2], a.deg, a.act, base, gcol, dW, gp, gf, gd);
+    } else if (in) {
 #pragma unroll
-          for (int k = 0; k < 32; ++k) x[k] = 0.f;
-        }
-        decode_backward_warp<Split<APP>::value>(sWt, sStage[warp], lane, in, x, d[0], d[1], d[2], a.deg, a.act, base, gcol, dW, gp, gf, gd);
-      } else if (in) {
-#pragma unroll
-        for (int c = 0; c < 3; ++c) gp[c] = color_act_grad_z(a.act, base[c] + 0.5f) * gcol[c];
-      }
-      if (exists) {
-        float4 *gfp = reinterpret_cast<float4 *>(a.g_features) + 2 * i;
-        gfp[0] = make_float4(gf[0], gf[1], gf[2], gf[3]);
-        gfp[1] = make_float4(gf[4], gf[5], gf[6], gf[7]);
-      }
+      for (int c = 0; c < 3; ++c) gp[c] = color_act_grad_z(a.act, base[c] + 0.5f) * gcol[c];
     }
     if (exists) {
+      float4 *gfp = reinterpret_cast<float4 *>(a.g_features) + 2 * i;
+      gfp[0] = make_float4(gf[0], gf[1], gf[2], gf[3]);
+      gfp[1] = make_float4(gf[4], gf[5], gf[6], gf[7]);
       store3(a.g_base, i, gp[0], gp[1], gp[2]);
       store3(a.g_dirs, i, gd[0], gd[1], gd[2]);
     }
   }
-  if (IsNeural<APP>::value) {
-    weight_grad_flush(dW, reinterpret_cast<float *>(sStage), a.w_partials + (size_t)blockIdx.x * GS_MLP_WEIGHTS, tid);
-  }
+  weight_grad_flush(dW, reinterpret_cast<float *>(sStage), a.w_partials + (size_t)blockIdx.x * GS_MLP_WEIGHTS, tid);
 }
 
 // ---- separate-pass kernels of the explicit models with bulk copies ---------------------------------------------
