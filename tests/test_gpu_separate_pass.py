@@ -131,3 +131,33 @@ def test_workspace_covers_the_separate_passes():
     n = 100_000
     # backward scratch: [n,12] + three [n,3] arrays, each rounded up to 256 bytes
     assert api.gs_workspace_bytes(n, 64, 64, 0) >= n * (12 + 9) * 4
+
+
+@pytest.mark.parametrize("app", [scenes.APP_SH, scenes.APP_SV], ids=["sh", "sv"])
+@pytest.mark.parametrize("n", [32, 128, 160, 4096, 4128, 75_776, 75_777])
+def test_bulk_copy_decode_at_warp_and_block_boundaries(oracle, app, n):
+    """The separate-pass kernels of the explicit models move whole 32-row slabs by bulk copies and a ragged last
+    warp by plain loads: sizes that end exactly on a warp, on a block, one warp past a block, and (75 776 = 592 x
+    128) exactly one block per persistent CTA and one Gaussian more."""
+    import torch
+    from paper_2609_05255_b200 import api
+    sc, dirs, gcol = scenes.config5(n, app)
+    ctx = api.Context(0)
+    ds = api.upload_scene(sc, ctx.device)
+    d = torch.from_numpy(dirs).to(ctx.device); gc = torch.from_numpy(gcol).to(ctx.device)
+    color = torch.full((n, 3), float("nan"), device=ctx.device)
+    api.gs_appearance_forward(ctx, ds, d, color)
+    grads = api.alloc_grads_for(ds, ctx.device)
+    rows = grads.sh_rest if app == scenes.APP_SH else grads.sv_sites
+    rows.fill_(float("nan")); grads.base_color.fill_(float("nan"))
+    gd = torch.full((n, 3), float("nan"), device=ctx.device)
+    api.gs_appearance_backward(ctx, ds, d, gc, grads, gd)
+    torch.cuda.synchronize()
+    api.gs_async_status(ctx)
+    ref_c, _ = oracle.appearance_forward(sc, dirs)
+    ref = oracle.appearance_backward(sc, dirs, gcol)
+    assert np.abs(color.cpu().numpy() - ref_c).max() < 2e-5
+    assert grad_mismatch(grads.base_color.cpu().numpy(), ref.base_color).sum() == 0
+    assert grad_mismatch(gd.cpu().numpy(), ref.dirs).sum() == 0
+    assert grad_mismatch(rows.cpu().numpy(), ref.sh_rest if app == scenes.APP_SH else ref.sv_sites).sum() == 0
+    ctx.close()
