@@ -334,7 +334,8 @@ GsStatus gs_neural_prepass(GsContext *ctx, const GsScene *scene, const uint16_t 
 
 /* Per-stage device timing, for benchmarks (the paper gives wall-clock protocols only, App. C; this
  * is the measurement hook of this library).  While enabled, every stage the library launches is
- * bracketed by CUDA events on the caller's stream.  gs_profile_collect synchronises those events,
+ * bracketed by CUDA events on the caller's stream and by an NVTX range named after the stage (for a tracing
+ * tool; a no-op without one).  gs_profile_collect synchronises those events,
  * ADDS the elapsed milliseconds and the kernel-launch counts since the last collect into
  * ms[GS_NUM_STAGES] / launches[GS_NUM_STAGES] (host arrays, either may be NULL) and forgets them.
  * At most 4096 stage records are kept between two collects; further ones are dropped. */

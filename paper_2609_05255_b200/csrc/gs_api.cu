@@ -8,6 +8,8 @@
 #include <new>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "gs_device.cuh"
 
 struct StageRecord { int stage; int launches; cudaEvent_t begin, end; };
@@ -45,7 +47,12 @@ GsStatus check_cuda(GsContext *ctx, cudaError_t e, const char *what) {
   return GS_ERR_CUDA;
 }
 
-// Brackets one stage with events when profiling is on.
+const char *const kStageNames[] = {"preprocess_fwd", "depth_sort", "tile_offsets", "keygen", "tile_sort", "tile_ranges",
+                                   "blend_fwd", "blend_bwd", "preprocess_bwd", "appearance_fwd", "appearance_bwd",
+                                   "adam", "prepass"};
+static_assert(sizeof(kStageNames) / sizeof(kStageNames[0]) == GS_NUM_STAGES, "one name per stage");
+
+// Brackets one stage with events, and with an NVTX range for a tracing tool, when profiling is on.
 struct StageTimer {
   GsContext *ctx; cudaStream_t st; StageRecord rec; bool active;
   static cudaEvent_t get_event(GsContext *ctx) {
@@ -58,12 +65,15 @@ struct StageTimer {
     if (!active) return;
     rec.stage = stage; rec.launches = 0;
     rec.begin = get_event(ctx); rec.end = get_event(ctx);
+    if (stage >= 0 && stage < (int)(sizeof(kStageNames) / sizeof(kStageNames[0]))) nvtxRangePushA(kStageNames[stage]);
+    else nvtxRangePushA("gs");
     cudaEventRecord(rec.begin, st);
   }
   void done(int launches) {
     if (!active) return;
     rec.launches = launches;
     cudaEventRecord(rec.end, st);
+    nvtxRangePop();
     ctx->records.push_back(rec);
   }
 };
