@@ -797,6 +797,23 @@ static void blend_pixel(double px, double py, const uint32_t* list, int64_t len,
   if (fragile_pos) *fragile_pos = fpos;
 }
 
+// One pixel's records, for the tests that pin the allowance logic: every entry the pixel composited and
+// every ghost, in list order.  Returns the number of records (at most `cap` are written).
+int64_t gso_blend_pixel_records(double px, double py, const uint32_t* list, int64_t len, const double* mean2d,
+                                const double* conic, const double* opacity, const double* color, int64_t cap,
+                                uint32_t* g, int32_t* pos, double* alpha, double* T, uint8_t* clamped,
+                                uint8_t* ghost) {
+  std::vector<Composited> rec;
+  const double bg[3] = {0, 0, 0};
+  double out[3], fT; uint32_t nc; uint8_t frag; int32_t fpos;
+  blend_pixel(px, py, list, len, mean2d, conic, opacity, color, bg, out, &fT, &nc, &frag, &fpos, &rec);
+  for (int64_t k = 0; k < (int64_t)rec.size() && k < cap; ++k) {
+    g[k] = rec[k].g; pos[k] = rec[k].pos; alpha[k] = rec[k].alpha; T[k] = rec[k].T;
+    clamped[k] = rec[k].clamped ? 1 : 0; ghost[k] = rec[k].ghost ? 1 : 0;
+  }
+  return (int64_t)rec.size();
+}
+
 // Tiled forward: image[3,H,W], final_T[H,W], n_contrib[H,W], fragile[H,W] (u8), fragile_pos[H,W].
 void gso_blend_forward(int W, int H, const double* bg, const uint32_t* vals, const uint32_t* ranges,
                        const double* mean2d, const double* conic, const double* opacity,

@@ -352,6 +352,24 @@ def blend_forward(cam, vals, ranges, mean2d, conic, opacity, color):
     return o
 
 
+def blend_pixel_records(px, py, vals, mean2d, conic, opacity, color):
+    """What one pixel (centre px, py) records from the ordered list `vals`: the entries it composites and the
+    ghosts (pairs it leaves out although they sit within tolerance of a blend threshold), in list order."""
+    vals = np.ascontiguousarray(vals, np.uint32)
+    cap = 2 * len(vals) + 4
+    o = SimpleNamespace(g=np.zeros(cap, np.uint32), pos=np.zeros(cap, np.int32), alpha=np.zeros(cap), T=np.zeros(cap),
+                        clamped=np.zeros(cap, np.uint8), ghost=np.zeros(cap, np.uint8))
+    f = lib().gso_blend_pixel_records
+    f.restype = C.c_int64
+    k = int(f(C.c_double(px), C.c_double(py), _p(vals, C.c_uint32), C.c_int64(len(vals)), _dp(_f64(mean2d)),
+              _dp(_f64(conic)), _dp(_f64(opacity)), _dp(_f64(color)), C.c_int64(cap), _p(o.g, C.c_uint32),
+              _p(o.pos, C.c_int32), _dp(o.alpha), _dp(o.T), _p(o.clamped, C.c_uint8), _p(o.ghost, C.c_uint8)))
+    assert k <= cap
+    for nm in ("g", "pos", "alpha", "T", "clamped", "ghost"):
+        setattr(o, nm, getattr(o, nm)[:k])
+    return o
+
+
 def blend_brute(cam, visible, depth_bits, mean2d, conic, opacity, color):
     W, H = cam.width, cam.height
     bg = _f64(cam.background)
