@@ -732,6 +732,11 @@ void gso_tile_ranges(int64_t P, const uint64_t* keys, int num_tiles, uint32_t* r
 // fp32 evaluation might; it only feeds the flip allowance of the backward.
 struct Composited { uint32_t g; int pos; double alpha, T, power; bool clamped; bool ghost; };
 
+// Half-width of the window around T (1 - alpha) = 1e-4 inside which a stop counts as one that an fp32 evaluation
+// may take the other way.  A test may narrow it to measure how many pixels need the default.
+static double g_stop_window = 1e-7;
+void gso_set_stop_window(double w) { g_stop_window = w; }
+
 static void blend_pixel(double px, double py, const uint32_t* list, int64_t len, const double* mean2d,
                         const double* conic, const double* opacity, const double* color,
                         const double bg[3], double out[3], double* final_T, uint32_t* n_contrib,
@@ -761,8 +766,8 @@ static void blend_pixel(double px, double py, const uint32_t* list, int64_t len,
       continue;
     }
     const double Tn = T * (1.0 - alpha);
-    if (std::fabs(Tn - kTmin) < 1e-7) frag = true;
-    const bool near_stop = std::fabs(Tn - kTmin) < 1e-7;
+    if (std::fabs(Tn - kTmin) < g_stop_window) frag = true;
+    const bool near_stop = std::fabs(Tn - kTmin) < g_stop_window;
     if (near_stop && fpos < 0) fpos = (int32_t)k;
     if (Tn < kTmin) {
       if (near_stop && rec) {
@@ -778,7 +783,7 @@ static void blend_pixel(double px, double py, const uint32_t* list, int64_t len,
           const double rw = opacity[gg] * std::exp(pw), al = std::min(kAlphaMax, rw);
           if (al < kAlphaMin) continue;
           const double Tgn = Tg * (1.0 - al);
-          if (kk > k && Tgn < kTmin - 1e-7) break;
+          if (kk > k && Tgn < kTmin - g_stop_window) break;
           rec->push_back({gg, (int)kk, al, Tg, pw, rw > kAlphaMax, true});
           Tg = Tgn;
         }

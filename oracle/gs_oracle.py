@@ -352,6 +352,11 @@ def blend_forward(cam, vals, ranges, mean2d, conic, opacity, color):
     return o
 
 
+def set_stop_window(width=1e-7):
+    """Half-width of the window around T (1 - alpha) = 1e-4 in which a stop is flagged fragile (default 1e-7)."""
+    lib().gso_set_stop_window(C.c_double(width))
+
+
 def blend_pixel_records(px, py, vals, mean2d, conic, opacity, color):
     """What one pixel (centre px, py) records from the ordered list `vals`: the entries it composites and the
     ghosts (pairs it leaves out although they sit within tolerance of a blend threshold), in list order."""

@@ -76,10 +76,10 @@ def fused(request, oracle):
     return {request.param: r}, request.param
 
 
-def test_fused_step_floats_and_image(fused):
+def test_fused_step_floats_and_image(fused, oracle):
     results, name = fused
     small.test_per_gaussian_floats(results, name)
-    small.test_image(results, name)
+    small.test_image(results, oracle, name)
 
 
 def test_fused_step_gradients(fused, oracle):
