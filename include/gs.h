@@ -257,12 +257,14 @@ GsStatus gs_appearance_backward(GsContext *ctx, const GsScene *scene, const floa
  *
  * The scratch the kernel needs - one row of 816 fp32 partial sums of the decoder-weight gradient per
  * CTA - is a static device array compiled into the library: 1024 rows = 3,342,336 bytes, held by
- * every GPU that loads the library until the process exits.  Each CTA covers at most 32 x 128
- * Gaussians, so n may be at most 4,194,304; a larger n is rejected with GS_ERR_CAPACITY and a
- * message, nothing launched.  Arguments and results are those of gs_appearance_backward (device
- * pointers on the CURRENT device, 16-byte aligned); per-Gaussian results are bit-identical to it,
- * grads->mlp_weights is the same sum taken in a different order.  error_text (host, may be NULL)
- * receives a description when the status is not GS_OK.
+ * every GPU that loads the library until the process exits.  A launch has at most 1024 CTAs, each
+ * covering at most 32 x 128 Gaussians, so n may be at most 4,194,304; a larger n is rejected with
+ * GS_ERR_CAPACITY and a message, nothing launched.  Arguments and results are those of
+ * gs_appearance_backward (device pointers on the CURRENT device, 16-byte aligned), including
+ * scene->color_activation and scene->decoder_precision (GS_DECODER_HALF runs the same unsplit kernel
+ * as there; an unknown value of either is GS_ERR_INVALID_ARG); per-Gaussian results are
+ * bit-identical to it, grads->mlp_weights is the same sum taken in a different order.  error_text
+ * (host, may be NULL) receives a description when the status is not GS_OK.
  *
  * The first call on each device looks up the device address of the array; make that call before any
  * stream capture begins.  All calls share the one array, which keeps the previous call's values:

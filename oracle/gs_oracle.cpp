@@ -125,6 +125,7 @@ constexpr int kNumW = kIn * kHid + kHid * kHid + kHid * kOut;
 
 struct MlpState {
   double x[kIn], h1[kHid], h2[kHid], y[kOut], A[kOut];
+  double kink;   // smallest |pre-activation| of the 32 hidden units: how far the nearest ReLU decision is from flipping
 };
 
 // Colour activations of Sec. 3.1, as functions of x = c0 + A(d).  All map 0 to (about) 0.5 with slope
@@ -207,15 +208,18 @@ void mlp_forward(const double* W, const double d[3], const double* f, int deg, M
     s.x[16 + 2 * j] = std::sin(f[j]);
     s.x[17 + 2 * j] = std::cos(f[j]);
   }
+  s.kink = 1e300;
   for (int o = 0; o < kHid; ++o) {
     double a = 0;
     for (int i = 0; i < kIn; ++i) a += W[kW1 + o * kIn + i] * s.x[i];
     s.h1[o] = a > 0 ? a : 0;
+    s.kink = std::min(s.kink, std::fabs(a));
   }
   for (int o = 0; o < kHid; ++o) {
     double a = 0;
     for (int i = 0; i < kHid; ++i) a += W[kW2 + o * kHid + i] * s.h1[i];
     s.h2[o] = a > 0 ? a : 0;
+    s.kink = std::min(s.kink, std::fabs(a));
   }
   for (int o = 0; o < kOut; ++o) {
     double a = 0;
@@ -477,6 +481,21 @@ void gso_appearance_forward(int64_t n, int app, int deg, int act, const double* 
 // Backward of the decode.  g_color = dL/dc.  Outputs: g_base[n,3], g_sh_rest[n,15,3] or
 // g_features[n,8], g_weights[816] (sum over Gaussians in index order), g_dirs[n,3] (gradient
 // with respect to the direction as a free R^3 vector).
+// Per Gaussian, the smallest |pre-activation| among the decoder's 32 hidden units (infinite where the residual is
+// disabled): a row whose margin is within fp32 rounding of zero is one where a single-precision evaluation may take
+// the other branch of a ReLU.  The parity tests use it to say WHICH rows may differ, instead of only how many.
+void gso_mlp_kink_margin(int64_t n, int deg, const double* features, const double* weights, const double* dirs,
+                         double* margin) {
+#pragma omp parallel for schedule(static)
+  for (int64_t i = 0; i < n; ++i) {
+    margin[i] = INFINITY;
+    if (deg <= 0) continue;
+    MlpState s;
+    mlp_forward(weights, dirs + 3 * i, features + kFeat * i, deg, s);
+    margin[i] = s.kink;
+  }
+}
+
 void gso_appearance_backward(int64_t n, int app, int deg, int act, const double* base_color,
                              const double* sh_rest, const double* features, const double* weights,
                              const double* dirs, const uint8_t* mask, const double* g_color,
@@ -733,8 +752,9 @@ void gso_tile_ranges(int64_t P, const uint64_t* keys, int num_tiles, uint32_t* r
 struct Composited { uint32_t g; int pos; double alpha, T, power; bool clamped; bool ghost; };
 
 // Half-width of the window around T (1 - alpha) = 1e-4 inside which a stop counts as one that an fp32 evaluation
-// may take the other way.  A test may narrow it to measure how many pixels need the default.
-static double g_stop_window = 1e-7;
+// may take the other way: 1e-8 (a product of a few hundred fp32 factors, each carrying alpha's few ulp, is good to
+// about 1e-4 relative, i.e. 1e-8 at the threshold).  A test may change it to measure what another width would flag.
+static double g_stop_window = 1e-8;
 void gso_set_stop_window(double w) { g_stop_window = w; }
 
 static void blend_pixel(double px, double py, const uint32_t* list, int64_t len, const double* mean2d,

@@ -281,6 +281,15 @@ def appearance_backward(scene, dirs, g_color, mask=None, deg=None):
     return o
 
 
+def mlp_kink_margin(scene, dirs, deg=None):
+    """[n]: smallest |pre-activation| among the 32 hidden units of the default decoder, per Gaussian."""
+    dirs = _f64(dirs); n = dirs.shape[0]
+    out = np.zeros(n)
+    lib().gso_mlp_kink_margin(C.c_int64(n), C.c_int(scene.active_degree if deg is None else deg),
+                              _dp(_f64(scene.features)), _dp(_f64(scene.mlp_weights)), _dp(dirs), _dp(out))
+    return out
+
+
 def _tile_spans(suffix, dtype, ctype, valid, mean2d, chol, ext, width, height):
     valid = np.ascontiguousarray(valid, np.uint8)
     m = np.ascontiguousarray(mean2d, dtype); c = np.ascontiguousarray(chol, dtype)
@@ -352,8 +361,8 @@ def blend_forward(cam, vals, ranges, mean2d, conic, opacity, color):
     return o
 
 
-def set_stop_window(width=1e-7):
-    """Half-width of the window around T (1 - alpha) = 1e-4 in which a stop is flagged fragile (default 1e-7)."""
+def set_stop_window(width=1e-8):
+    """Half-width of the window around T (1 - alpha) = 1e-4 in which a stop is flagged fragile (default 1e-8)."""
     lib().gso_set_stop_window(C.c_double(width))
 
 

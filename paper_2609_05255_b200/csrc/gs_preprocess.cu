@@ -1196,6 +1196,10 @@ extern "C" GsStatus gs_appearance_backward_noalloc(const GsScene *scene, const f
   if (scene->app != GS_APP_NEURAL)
     return fail(GS_ERR_UNSUPPORTED, "only the neural appearance backward uses scratch memory; call gs_appearance_backward for SH");
   if (scene->active_degree < 0 || scene->active_degree > 3) return fail(GS_ERR_INVALID_ARG, "active_degree must be 0..3");
+  if (scene->color_activation < GS_ACT_RELU || scene->color_activation > GS_ACT_HARD_SIGMOID)
+    return fail(GS_ERR_INVALID_ARG, "unknown colour activation");
+  if (scene->decoder_precision != GS_DECODER_SPLIT && scene->decoder_precision != GS_DECODER_HALF)
+    return fail(GS_ERR_INVALID_ARG, "unknown decoder precision");
   if ((scene->mlp_hidden != 0 && scene->mlp_hidden != 16) || (scene->mlp_layers != 0 && scene->mlp_layers != 2) ||
       (scene->num_features != 0 && scene->num_features != 8))
     return fail(GS_ERR_UNSUPPORTED, "this entry point serves the 16 / 2 / 8 decoder only");
@@ -1239,10 +1243,17 @@ extern "C" GsStatus gs_appearance_backward_noalloc(const GsScene *scene, const f
   a.g_color = dL_dcolor;
   a.g_base = grads->base_color; a.g_features = grads->features; a.g_dirs = dL_ddirs;
   a.w_partials = scratch; a.g_weights = grads->mlp_weights;
+  // one CTA per chunk of 128 Gaussians until the scratch's rows run out; from there on the CTAs walk the chunks with
+  // the grid as their stride (at the largest n each covers 32 of them)
   const int64_t chunks = (a.n + kBlock - 1) / kBlock;
-  const int blocks = (int)((chunks + kNoAllocChunksPerBlock - 1) / kNoAllocChunksPerBlock);   // <= 1024
-  opt_in_smem(k_appearance_bwd<GS_APP_NEURAL>, kBwdSmemNN);
-  k_appearance_bwd<GS_APP_NEURAL><<<blocks, kBlock, kBwdSmemNN, st>>>(a);
+  const int blocks = (int)(chunks < kNoAllocMaxBlocks ? chunks : kNoAllocMaxBlocks);
+  if (scene->decoder_precision == GS_DECODER_HALF) {   // same dispatch as gs_appearance_backward
+    opt_in_smem(k_appearance_bwd<kAppNeuralHalf>, kBwdSmemNN);
+    k_appearance_bwd<kAppNeuralHalf><<<blocks, kBlock, kBwdSmemNN, st>>>(a);
+  } else {
+    opt_in_smem(k_appearance_bwd<GS_APP_NEURAL>, kBwdSmemNN);
+    k_appearance_bwd<GS_APP_NEURAL><<<blocks, kBlock, kBwdSmemNN, st>>>(a);
+  }
   launch_wgrad_reduce(scratch, blocks, a.g_weights, st);
   const cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return fail(GS_ERR_CUDA, cudaGetErrorString(e));

@@ -18,7 +18,8 @@ def oracle():
 
 
 # Measured counts behind the parity tolerances (fragile pixels, values outside the literal gradient rule, values that
-# need an allowance): tests append rows here, the summary prints them, and GS_PARITY_REPORT=<file> also stores them.
+# need an allowance): tests/gpu_helpers.check_bound appends rows here, the summary prints them, and
+# GS_PARITY_REPORT=<file> also stores them (tests/make_parity_bounds.py turns that file into tests/parity_bounds.json).
 PARITY_ROWS = []
 
 

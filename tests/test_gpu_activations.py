@@ -79,7 +79,7 @@ def fused(request, oracle):
 def test_fused_step_floats_and_image(fused, oracle):
     results, name = fused
     small.test_per_gaussian_floats(results, name)
-    small.test_image(results, oracle, name)
+    small.test_image(results, name)
 
 
 def test_fused_step_gradients(fused, oracle):

@@ -4,12 +4,14 @@ Gaussians - for degree-3 SH, Spherical Voronoi, the neural decoder with split op
 operands; and at sizes that make every CTA of the persistent grids take a second and a third full trip (and one
 Gaussian more), so that the later bulk loads of both slabs, both barrier phases and the accumulation of the
 decoder-weight gradient across trips are all checked against the oracle, not only against themselves."""
+import os
+
 import numpy as np
 import pytest
 
 from paper_2609_05255_b200 import scenes
 from conftest import record_parity
-from gpu_helpers import grad_mismatch
+from gpu_helpers import MEASURE, check_bound, grad_mismatch
 from test_gpu_half_precision import COLOR_ATOL as HALF_COLOR_ATOL, check_gradient as check_half_gradient
 
 pytestmark = pytest.mark.gpu
@@ -17,23 +19,23 @@ pytestmark = pytest.mark.gpu
 MODELS = {"sh": (scenes.APP_SH, 0), "sv": (scenes.APP_SV, 0), "neural_split": (scenes.APP_NEURAL, 0),
           "neural_half": (scenes.APP_NEURAL, 1)}
 
-# Colours: 2e-5 absolute (split / explicit models).  Per-Gaussian gradients: the literal rule, 1e-3 relative or 1e-5
-# absolute, no exceptions for the explicit models; for the neural decoder a Gaussian whose hidden pre-activation sits
-# within fp32 rounding of the ReLU kink may take the other branch - measured at most 3 rows in 10M, bounded at 1e-6
-# of the rows.  Decoder-weight gradients (each the sum of n signed terms, accumulated in fp32 per CTA): the literal
-# rule for all but a few of the 816 (bounded per size below, from the measured counts) and no element off by more
-# than 1e-5 of the largest one.
-KINK_ROW_FRACTION = 1e-6
-WEIGHTS_OFF = {1_000_000: 8, 3_000_000: 8, 10_000_000: 8}
-WEIGHTS_OFF_DEFAULT = 8
-WEIGHT_MAX_REL = 1e-5
+# Colours: 2e-5 absolute (explicit models and split operands).  Per-Gaussian gradients: the literal rule, 1e-3
+# relative or 1e-5 absolute.  Neural decoder: a ReLU decision is taken on a pre-activation that the kernel holds in
+# fp32; where the oracle's double-precision value lies within KINK_MARGIN of zero the two sides may take different
+# branches, and that Gaussian's gradients then differ as a whole.  The oracle names those rows (its smallest hidden
+# |pre-activation| per Gaussian): every row outside the literal rule must be one of them, and the decoder-weight
+# gradient is compared in a second run in which those rows receive a zero upstream gradient on both sides, so that
+# it is a sum over rows whose decisions agree.
+KINK_MARGIN = 2.5e-7      # twice the largest margin measured on a row that did differ (1.2e-7, at 10M Gaussians)
 
 
-def _decode(app, precision, n):
+def _decode(app, precision, n, zero_rows=None):
     import torch
     from paper_2609_05255_b200 import api
     sc, dirs, gcol = scenes.config5(n, app)
     sc.decoder_precision = precision
+    if zero_rows is not None:
+        gcol[zero_rows] = 0
     ctx = api.Context(0)
     ds = api.upload_scene(sc, ctx.device)
     d = torch.from_numpy(dirs).to(ctx.device); gc = torch.from_numpy(gcol).to(ctx.device)
@@ -56,6 +58,13 @@ def _decode(app, precision, n):
     return sc, dirs, gcol, out
 
 
+# What cannot be exact is counted and held to the recorded measurement (gpu_helpers.check_bound): rows of an explicit
+# model outside the literal rule (measured: none, except one Spherical Voronoi site gradient in 490 million at 10M
+# Gaussians - a tangential projection that cancels to 1e-4 of its terms - 1.5e-3 relative and 1.2e-5 absolute off);
+# decoder-weight gradients (816 sums of n signed terms, fp32 partial sums per CTA) outside the literal rule once the
+# kink rows are taken out, and their largest error relative to the largest weight gradient.
+
+
 def _check(oracle, model, n):
     app, precision = MODELS[model]
     sc, dirs, gcol, got = _decode(app, precision, n)
@@ -72,21 +81,32 @@ def _check(oracle, model, n):
         return
     assert err_c < 2e-5, err_c
     rows = {"sh": ["sh_rest"], "sv": ["sv_sites"], "neural_split": ["features"]}[model]
-    counts = {}
+    off = np.zeros(n, bool)
     for nm in ["base_color", "dirs"] + rows:
-        bad = grad_mismatch(got[nm], getattr(ref, nm))
-        bad_rows = int(bad.reshape(n, -1).any(1).sum())
-        counts[nm + "_rows_off"] = bad_rows
-        limit = int(KINK_ROW_FRACTION * n) + (3 if app == scenes.APP_NEURAL else 0)
-        assert bad_rows <= (limit if app == scenes.APP_NEURAL else 0), f"{nm}: {bad_rows} of {n} rows off"
-    if app == scenes.APP_NEURAL:
-        w_got, w_ref = got["mlp_weights"].astype(np.float64), ref.mlp_weights
-        off = int(grad_mismatch(w_got, w_ref).sum())
-        rel = float(np.abs(w_got - w_ref).max() / np.abs(w_ref).max())
-        counts.update(weights_off=off, weights_max_rel_to_largest=rel)
-        assert off <= WEIGHTS_OFF.get(n, WEIGHTS_OFF_DEFAULT), f"{off} of 816 weight gradients outside the literal rule"
-        assert rel <= WEIGHT_MAX_REL, rel
-    record_parity(case, "decode vs oracle", color_max_err=err_c, **counts)
+        off |= grad_mismatch(got[nm], getattr(ref, nm)).reshape(n, -1).any(1)
+    if app != scenes.APP_NEURAL:
+        record_parity(case, "decode vs oracle", color_max_err=err_c)
+        check_bound(case, "decode vs oracle", "rows_outside_literal_rule", int(off.sum()))
+        return
+    margin = oracle.mlp_kink_margin(sc, dirs)
+    kink = margin < KINK_MARGIN
+    worst = float(margin[off].max()) if off.any() else 0.0
+    assert MEASURE or not (off & ~kink).any(), f"{(off & ~kink).sum()} rows off whose ReLU decisions are clear (margin up to {worst:.2e})"
+    # the weight gradient over the rows whose decisions agree
+    sc2, dirs2, gcol2, got2 = _decode(app, precision, n, zero_rows=kink)
+    ref2 = oracle.appearance_backward(sc2, dirs2, gcol2)
+    w_got, w_ref = got2["mlp_weights"].astype(np.float64), ref2.mlp_weights
+    w_off = int(grad_mismatch(w_got, w_ref).sum())
+    rel = float(np.abs(w_got - w_ref).max() / np.abs(w_ref).max())
+    w_off_all = int(grad_mismatch(got["mlp_weights"], ref.mlp_weights).sum())
+    record_parity(case, "decode vs oracle", color_max_err=err_c, rows_off=int(off.sum()), kink_rows=int(kink.sum()),
+                  largest_margin_of_a_row_off=worst, weights_off_with_kink_rows=w_off_all)
+    check_bound(case, "decode vs oracle", "weights_outside_literal_rule", w_off)
+    check_bound(case, "decode vs oracle", "largest_weight_error_over_largest_weight_gradient", rel)
+    # and every other row still agrees in the second run
+    for nm in ("base_color", "dirs", "features"):
+        bad = grad_mismatch(got2[nm], getattr(ref2, nm)).reshape(n, -1).any(1)
+        assert MEASURE or not (bad & ~kink).any(), nm
 
 
 @pytest.mark.parametrize("n", [1_000_000, 3_000_000, 10_000_000])

@@ -49,9 +49,9 @@ def test_full_size_integer_stage_bit_exact(full, oracle):
     small.test_integer_stage_bit_exact(results, oracle, name)
 
 
-def test_full_size_image(full, oracle):
+def test_full_size_image(full):
     results, name = full
-    small.test_image(results, oracle, name)
+    small.test_image(results, name)
 
 
 def test_full_size_blend_backward(full):

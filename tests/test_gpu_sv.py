@@ -61,7 +61,7 @@ def test_fused_step_floats_integers_and_image(fused, oracle):
     results, name = fused
     small.test_per_gaussian_floats(results, name)
     small.test_integer_stage_bit_exact(results, oracle, name)
-    small.test_image(results, oracle, name)
+    small.test_image(results, name)
 
 
 def test_fused_step_gradients(fused, oracle):

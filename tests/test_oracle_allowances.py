@@ -5,7 +5,7 @@ rule (alpha = 1/255, T (1 - alpha) = 1e-4, raw alpha = 0.99) is placed there on 
 and which are ghosts is written down as literals, and the sums of |terms| are formed by the few lines of numpy
 below from the definition of the blend backward.
 
-Windows under test: |255 alpha - 1| < 1e-4, |T (1 - alpha) - 1e-4| < 1e-7, |raw - 0.99| < 0.99e-4.
+Windows under test: |255 alpha - 1| < 1e-4, |T (1 - alpha) - 1e-4| < 1e-8, |raw - 0.99| < 0.99e-4.
 """
 import numpy as np
 import pytest
@@ -49,7 +49,7 @@ def test_fragile_window_at_the_alpha_threshold(oracle, delta, fragile, composite
     assert fwd.n_contrib[0, 0] == 4
 
 
-@pytest.mark.parametrize("delta,fragile", [(+5e-8, True), (-5e-8, True), (+5e-7, False), (-5e-7, False)])
+@pytest.mark.parametrize("delta,fragile", [(+5e-9, True), (-5e-9, True), (+5e-8, False), (-5e-8, False)])
 def test_fragile_window_at_the_transmittance_stop(oracle, delta, fragile):
     T3 = (1.0 * (1.0 - 0.9)) * (1.0 - 0.9) * (1.0 - 0.9)      # after three entries of alpha 0.9
     a4 = 1.0 - (1e-4 + delta) / T3
@@ -106,21 +106,21 @@ def test_ghost_of_a_pair_just_below_the_alpha_threshold(oracle):
 
 def test_ghosts_of_a_stop_within_the_window(oracle):
     T3 = (1.0 * (1.0 - 0.9)) * (1.0 - 0.9) * (1.0 - 0.9)
-    a4 = 1.0 - (1e-4 - 5e-8) / T3
+    a4 = 1.0 - (1e-4 - 5e-9) / T3
     m, q, o, c = _centred([0.9, 0.9, 0.9, a4, 0.5, 0.5])
     r = oracle.blend_pixel_records(0.5, 0.5, np.arange(6), m, q, o, c)
     # the stopping pair is the one ghost: behind it 0.5 takes the transmittance to 5e-5, clearly below the window
     assert r.pos.tolist() == [0, 1, 2, 3] and r.ghost.tolist() == [0, 0, 0, 1]
     assert r.alpha[3] == a4 and r.T[3] == pytest.approx(T3, rel=1e-15)
     # a pair behind it that keeps the transmittance inside the window is walked over as a ghost too
-    a4 = 1.0 - (1e-4 - 1e-9) / T3
+    a4 = 1.0 - (1e-4 - 1e-10) / T3
     tiny = 4e-3                                                # >= 1/255, so it is evaluated ...
     m, q, o, c = _centred([0.9, 0.9, 0.9, a4, tiny, 0.5])
     r = oracle.blend_pixel_records(0.5, 0.5, np.arange(6), m, q, o, c)
-    assert (1e-4 - 1e-9) * (1 - tiny) < 1e-4 - 1e-7          # ... it leaves the window, so the chain ends at once
+    assert (1e-4 - 1e-10) * (1 - tiny) < 1e-4 - 1e-8          # ... it leaves the window, so the chain ends at once
     assert r.pos.tolist() == [0, 1, 2, 3] and r.ghost.tolist() == [0, 0, 0, 1]
-    # 5e-7 below the threshold: a plain stop, no ghost
-    a4 = 1.0 - (1e-4 - 5e-7) / T3
+    # 5e-8 below the threshold: a plain stop, no ghost
+    a4 = 1.0 - (1e-4 - 5e-8) / T3
     m, q, o, c = _centred([0.9, 0.9, 0.9, a4, 0.5])
     r = oracle.blend_pixel_records(0.5, 0.5, np.arange(5), m, q, o, c)
     assert r.pos.tolist() == [0, 1, 2] and r.ghost.tolist() == [0, 0, 0]
@@ -253,7 +253,7 @@ def test_flip_sum_counts_the_flagged_pair_and_everything_behind_it_in_that_pixel
 def test_flip_sum_of_a_stop_within_the_window(oracle):
     cam = _cam()
     T3 = (1.0 * (1.0 - 0.9)) * (1.0 - 0.9) * (1.0 - 0.9)
-    a4 = 1.0 - (1e-4 - 5e-8) / T3
+    a4 = 1.0 - (1e-4 - 5e-9) / T3
     alphas = [0.9, 0.9, 0.9, a4, 0.5]
     cols = [(0.9, 0.1, 0.3), (0.2, 0.7, 0.4), (0.5, 0.5, 0.1), (0.3, 0.3, 0.9), (0.6, 0.2, 0.2)]
     rows = [((0.5, 0.5), (1.0, 0.0, 1.0), a, c) for a, c in zip(alphas, cols)]
@@ -271,3 +271,30 @@ def test_flip_sum_of_a_stop_within_the_window(oracle):
     want[0:3] = np.abs(a4 * T3 * G[:, 0, 0])
     want[3] = abs(float(G[:, 0, 0] @ (T3 * np.asarray(cols[3]) - S / (1 - a4))))
     assert np.allclose(flip_sum[3], want, rtol=1e-12, atol=1e-18)
+
+
+# ---------------------------------------------------------------------------------------- ReLU margin of the decoder
+
+def test_kink_margin_is_the_smallest_hidden_pre_activation(oracle):
+    """Hand-set weights: with f = 0 the input cos f_0 is exactly 1, W1 routes it to hidden unit o with gain
+    0.1 (o + 1), W2 is diagonal with one negative and one small entry.  The 32 pre-activations are then known in
+    closed form; the margin is the smallest of their absolute values.  Degree 0 disables the residual: no decision."""
+    n = 3
+    w = np.zeros(816)
+    for o in range(16):
+        w[o * 32 + 17] = 0.1 * (o + 1)                  # W1[o][cos f_0]
+        w[512 + o * 16 + o] = 1.0                       # W2 diagonal
+    w[512 + 3 * 16 + 3] = -0.5                          # unit 3 of layer 2: pre-activation -0.5 * 0.4 = -0.2
+    w[512 + 5 * 16 + 5] = 0.01                          # unit 5 of layer 2: 0.01 * 0.6 = 0.006, the smallest
+    sc = scenes.Scene(np.zeros((n, 3), np.float32), np.zeros((n, 3), np.float32), np.zeros((n, 4), np.float32),
+                      np.zeros(n, np.float32), np.zeros((n, 3), np.float32), app=scenes.APP_NEURAL, active_degree=3,
+                      features=np.zeros((n, 8)), mlp_weights=w)
+    d = np.array([[0.0, 0.0, 1.0], [1.0, 0.0, 0.0], [0.6, 0.0, 0.8]])
+    m = oracle.mlp_kink_margin(sc, d)
+    assert np.allclose(m, 0.006, rtol=1e-13)
+    w[512 + 5 * 16 + 5] = 1.0
+    assert np.allclose(oracle.mlp_kink_margin(sc, d), 0.1, rtol=1e-13)       # now the first unit of layer 1
+    w[7 * 32 + 17] = -3e-7                                                    # a unit just below its kink
+    m = oracle.mlp_kink_margin(sc, d)
+    assert np.allclose(m, 0.0, atol=3.1e-7) and np.all(m <= 3e-7)           # layer 2 sees relu(-3e-7) = 0 there
+    assert np.all(np.isinf(oracle.mlp_kink_margin(sc, d, deg=0)))
