@@ -272,13 +272,13 @@ def run_ours(args):
         # units of the blend kernels: list entries up to each pixel's last composited one, over the views
         entries = 0
         visible = 0
-        evaluated = composited = 0
+        evaluated = composited = warp_steps = warp_steps_idle = 0
         for v in range(views):
             r.forward(ds, cams[v])
             torch.cuda.synchronize()
             entries += int(r.n_contrib.sum(dtype=torch.int64).item())
-            ev, co = api.gs_profile_blend_counts(ctx, r.proj, r.binning, cams[v])
-            evaluated += ev; composited += co
+            ev, co, ws_, wi = api.gs_profile_blend_counts(ctx, r.proj, r.binning, cams[v])
+            evaluated += ev; composited += co; warp_steps += ws_; warp_steps_idle += wi
             rect = r.proj.rect.to(torch.int32) & 0xFFFF
             visible += int(((rect[:, 2] > rect[:, 0]) & (rect[:, 3] > rect[:, 1])).sum().item())
         # the same step through the unfused reference path (App. D "Fusion"): appearance as passes of its own
@@ -304,6 +304,7 @@ def run_ours(args):
         results[tag] = dict(ms=ms, ms_one=ms_one, ms_streams=ms_streams, graph=graph_note, unfused=unfused, half=half,
                             stage_ms=stage_ms, stage_launches=stage_launches, pairs=pairs,
                             entries=entries, visible=visible, evaluated=evaluated, composited=composited,
+                            warp_steps=warp_steps, warp_steps_idle=warp_steps_idle,
                             host=host, ds=ds, r=r, app=tag)
 
     # ---- end to end through the public API with host buffers (neural arm)
@@ -348,6 +349,8 @@ def run_ours(args):
         "stages_ms_per_step": {k: round(v, 4) for k, v in stage_ms.items() if v > 0},
         "stage_share": {k: round(v / total_stage, 4) for k, v in stage_ms.items() if v > 0},
         "pairs_per_view": neural["pairs"], "visible_per_view": neural["visible"] / views,
+        "blend_warp_steps_per_view": neural["warp_steps"] / views,
+        "blend_warp_steps_without_a_taker_per_view": neural["warp_steps_idle"] / views,
         "sh": None if "sh" not in results or head == "sh" else {
             "ms_per_step": results["sh"]["ms"], "ms_per_step_single_stream": results["sh"]["ms_one"],
             "stages_ms_per_step": {k: round(v, 4) for k, v in results["sh"]["stage_ms"].items() if v > 0}},

@@ -360,7 +360,9 @@ typedef enum {
 GsStatus gs_profile_enable(GsContext *ctx, int enable);
 /* Measurement only: for the view last rendered into (proj, bin), count over all pixels the list
  * entries the blend evaluates (until each pixel stops) and the pairs it composites; these are the
- * work units of the blend kernels' roofline.  counts_host[2] is a host array; synchronises. */
+ * work units of the blend kernels' roofline.  counts_host is a host array of FOUR values: entries
+ * evaluated, pairs composited, (warp, entry) steps the forward walks (a warp covers 16 x 8 pixels)
+ * and the steps among them in which no pixel of the warp accepts the entry.  Synchronises. */
 GsStatus gs_profile_blend_counts(GsContext *ctx, const GsProjected *proj, const GsBinning *bin, const GsCamera *cam,
                                  int64_t *counts_host, void *stream);
 GsStatus gs_profile_collect(GsContext *ctx, double *ms, int64_t *launches);

@@ -339,12 +339,13 @@ def gs_profile_collect(ctx: Context):
 
 
 def gs_profile_blend_counts(ctx: Context, proj: "Projected", binning: "Binning", cam: GsCamera, stream=None):
-    """(list entries evaluated, pairs composited) over all pixels of the view held in proj / binning."""
-    out = (C.c_int64 * 2)()
+    """(list entries evaluated, pairs composited, warp steps, warp steps without a taker) over all pixels of the view
+    held in proj / binning."""
+    out = (C.c_int64 * 4)()
     pp, bb = proj.c_struct(), binning.c_struct()
     ctx._check(_lib.gs_profile_blend_counts(ctx._h, C.byref(pp), C.byref(bb), C.byref(cam), out,
                                             _stream_handle(stream)))
-    return int(out[0]), int(out[1])
+    return int(out[0]), int(out[1]), int(out[2]), int(out[3])
 
 
 def gs_workspace_bytes(n: int, width: int, height: int, pair_capacity: int) -> int:

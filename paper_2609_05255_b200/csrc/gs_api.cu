@@ -17,9 +17,9 @@ struct StageRecord { int stage; int launches; cudaEvent_t begin, end; };
 struct GsContext {
   int device;
   int num_sms;
-  unsigned long long *d_counter;      // device: [0] instance counter of the last gs_preprocess, [1] second word of
-                                      // gs_profile_blend_counts, [2] set when a device-counted view overflowed its capacity,
-                                      // [3] set when a bounded device-side wait ran out
+  unsigned long long *d_counter;      // device: [0] instance counter of the last gs_preprocess, [2] set when a device-counted
+                                      // view overflowed its capacity, [3] set when a bounded device-side wait ran out,
+                                      // [4..7] the four words of gs_profile_blend_counts
   unsigned long long *h_counter;      // pinned host mirror
   float *d_w_partials;                // device: per-CTA partial sums of the decoder gradient ([kWgradBlocks, 816];
                                       // sized for the decoder variants' largest case as well)
@@ -249,9 +249,9 @@ GsStatus gs_create(int device, GsContext **out) {
   ctx->error[0] = 0;
   ctx->d_counter = nullptr; ctx->h_counter = nullptr; ctx->d_w_partials = nullptr;
   ctx->profiling = false;
-  if (cudaMalloc(&ctx->d_counter, 4 * sizeof(unsigned long long)) != cudaSuccess ||
-      cudaMemset(ctx->d_counter, 0, 4 * sizeof(unsigned long long)) != cudaSuccess ||
-      cudaMallocHost(&ctx->h_counter, 4 * sizeof(unsigned long long)) != cudaSuccess ||
+  if (cudaMalloc(&ctx->d_counter, 8 * sizeof(unsigned long long)) != cudaSuccess ||
+      cudaMemset(ctx->d_counter, 0, 8 * sizeof(unsigned long long)) != cudaSuccess ||
+      cudaMallocHost(&ctx->h_counter, 8 * sizeof(unsigned long long)) != cudaSuccess ||
       cudaMalloc(&ctx->d_w_partials, sizeof(float) * std::max((size_t)kWgradBlocks * GS_MLP_WEIGHTS, variant_partials_floats())) != cudaSuccess) {
     gs_destroy(ctx);
     return GS_ERR_CUDA;
@@ -555,14 +555,13 @@ GsStatus gs_profile_blend_counts(GsContext *ctx, const GsProjected *proj, const 
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   cudaSetDevice(ctx->device);
   GsStatus st;
-  if ((st = check_cuda(ctx, cudaMemsetAsync(ctx->d_counter, 0, 2 * sizeof(unsigned long long), s), "memset")) != GS_OK) return st;
+  if ((st = check_cuda(ctx, cudaMemsetAsync(ctx->d_counter + 4, 0, 4 * sizeof(unsigned long long), s), "memset")) != GS_OK) return st;
   launch_blend_count(make_cam(cam), bin->tile_ranges, bin->sorted_vals, proj->mean2d, proj->conic_opacity, proj->color,
-                     ctx->d_counter, s);
-  if ((st = check_cuda(ctx, cudaMemcpyAsync(ctx->h_counter, ctx->d_counter, 2 * sizeof(unsigned long long),
+                     ctx->d_counter + 4, s);
+  if ((st = check_cuda(ctx, cudaMemcpyAsync(ctx->h_counter + 4, ctx->d_counter + 4, 4 * sizeof(unsigned long long),
                                             cudaMemcpyDeviceToHost, s), "count copy")) != GS_OK) return st;
   if ((st = check_cuda(ctx, cudaStreamSynchronize(s), "blend counts")) != GS_OK) return st;
-  counts_host[0] = (int64_t)ctx->h_counter[0];
-  counts_host[1] = (int64_t)ctx->h_counter[1];
+  for (int k = 0; k < 4; ++k) counts_host[k] = (int64_t)ctx->h_counter[4 + k];
   return GS_OK;
 }
 

@@ -69,6 +69,24 @@ __device__ __forceinline__ bool alpha_of(float p, float o, float pmin, float &e2
   return true;
 }
 
+// 1.0f where a >= b or either is NaN, else 0.0f; 1.0f where a < b, else 0.0f: masks as numbers, so that what
+// depends on them runs as packed multiplies on the FMA pipe instead of selects on the ALU pipe.
+__device__ __forceinline__ float set_geu(float a, float b) {
+  float d;
+  asm("set.geu.f32.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+  return d;
+}
+__device__ __forceinline__ float set_lt(float a, float b) {
+  float d;
+  asm("set.lt.f32.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+  return d;
+}
+__device__ __forceinline__ float2 sub2(float2 a, float2 b) { return __ffma2_rn(b, make_float2(-1.f, -1.f), a); }   // a - b, exact products
+
+// Forward.  The four pixels of a quad travel as two packed pairs, (0, 1) and (2, 3), and the composite of an entry is
+// branch-free: "this pixel still composites" (live), "it accepts this entry" (q: alpha >= 1/255, decided on the
+// exponent) and "it stops here" (s: T - alpha T < 1e-4) are 0/1 numbers.  A pixel that skips the entry, has stopped
+// or stops here enters with weight exactly 0, which leaves its transmittance and colour sums unchanged bit for bit.
 __global__ void __launch_bounds__(kThreads) k_blend_fwd(CamDev cam, const uint32_t *__restrict__ ranges,
                                                         const uint32_t *__restrict__ order,
                                                         const uint32_t *__restrict__ vals,
@@ -84,16 +102,16 @@ __global__ void __launch_bounds__(kThreads) k_blend_fwd(CamDev cam, const uint32
   quad_of(tile, cam.gx, tid, px, py);
   const float fx = (float)px + 0.5f, fy = (float)py + 0.5f;
   const uint32_t start = __ldg(ranges + 2 * tile), end = __ldg(ranges + 2 * tile + 1);
-  float T[4], Cr[4], Cg[4], Cb[4];
-  uint32_t last[4];
-  unsigned live = 0;   // bit k set while pixel k still composites
-#pragma unroll
-  for (int k = 0; k < 4; ++k) {
-    T[k] = 1.f; Cr[k] = Cg[k] = Cb[k] = 0.f; last[k] = 0;
-    if (px + (k & 1) < cam.W && py + (k >> 1) < cam.H) live |= 1u << k;
-  }
+  const float in_x1 = px + 1 < cam.W ? 1.f : 0.f, in_y1 = py + 1 < cam.H ? 1.f : 0.f, in_0 = (px < cam.W && py < cam.H) ? 1.f : 0.f;
+  // T is the transmittance while the pixel composites and 0 once it has stopped (then every later weight alpha T is
+  // 0 by itself); the value it stopped with is kept in F.  Pixels outside the image start stopped.
+  float2 T01 = make_float2(in_0, in_0 * in_x1), T23 = make_float2(in_0 * in_y1, in_0 * in_x1 * in_y1);
+  const float2 zero = make_float2(0.f, 0.f), one = make_float2(1.f, 1.f);
+  float2 F01 = zero, F23 = zero;
+  float2 R01 = zero, R23 = zero, G01 = zero, G23 = zero, B01 = zero, B23 = zero;
+  uint32_t last[4] = {0u, 0u, 0u, 0u};      // position + 1 of the last composited entry
   for (uint32_t base = start; base < end; base += kBatch) {
-    if (__syncthreads_and(live == 0)) break;
+    if (__syncthreads_and((T01.x + T01.y) + (T23.x + T23.y) == 0.f)) break;
 #pragma unroll
     for (int h = 0; h < kBatch / kThreads; ++h) {
       const int slot = tid + h * kThreads;
@@ -102,26 +120,56 @@ __global__ void __launch_bounds__(kThreads) k_blend_fwd(CamDev cam, const uint32
     }
     __syncthreads();
     const int cnt = (int)min((uint32_t)kBatch, end - base);
+    float posf = 0.f;                         // position + 1 inside the batch, as a number (exact)
+    float2 last01 = zero, last23 = zero;      // the same of the last entry composited in this batch; 0 = none
+    for (int j0 = 0; j0 < cnt; j0 += 8) {
+      if (!__any_sync(kFull, (T01.x + T01.y) + (T23.x + T23.y) != 0.f)) break;   // every pixel of the warp has stopped
+      const int j1 = min(j0 + 8, cnt);
 #pragma unroll 2
-    for (int j = 0; j < cnt && live; ++j) {
-      const float4 a = s_xyab[j];
-      const float2 c = s_co[j];
-      float p[4], t1[4], t2[2];
-      quad_power(fx - a.x, fy - a.y, a.z, a.w, c.x, p, t1, t2);
-      const float4 col = s_rgb[j];
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        float e2, raw, alpha;
-        if (!((live >> k) & 1u) || !alpha_of(p[k], c.y, col.w, e2, raw, alpha)) continue;
-        const float Tn = __fmul_rn(T[k], 1.f - alpha);
-        if (Tn < kTmin) { live &= ~(1u << k); continue; }
-        const float w = __fmul_rn(alpha, T[k]);
-        Cr[k] = fmaf(col.x, w, Cr[k]); Cg[k] = fmaf(col.y, w, Cg[k]); Cb[k] = fmaf(col.z, w, Cb[k]);
-        T[k] = Tn;
-        last[k] = base - start + (uint32_t)j + 1u;
+      for (int j = j0; j < j1; ++j) {
+        const float4 a = s_xyab[j];
+        const float2 c = s_co[j];
+        float p[4], t1[4], t2[2];
+        quad_power(fx - a.x, fy - a.y, a.z, a.w, c.x, p, t1, t2);
+        const float4 col = s_rgb[j];
+        posf += 1.f;
+        const float2 q01 = make_float2(set_geu(p[0], col.w), set_geu(p[1], col.w));
+        const float2 q23 = make_float2(set_geu(p[2], col.w), set_geu(p[3], col.w));
+        if (!__any_sync(kFull, (q01.x + q01.y) + (q23.x + q23.y) != 0.f)) continue;   // no pixel of the warp takes it
+        const float2 o2 = make_float2(c.y, c.y);
+        const float2 raw01 = __fmul2_rn(o2, make_float2(ex2_approx(p[0]), ex2_approx(p[1])));
+        const float2 raw23 = __fmul2_rn(o2, make_float2(ex2_approx(p[2]), ex2_approx(p[3])));
+        const float2 al01 = __fmul2_rn(q01, make_float2(fminf(kAlphaMax, raw01.x), fminf(kAlphaMax, raw01.y)));
+        const float2 al23 = __fmul2_rn(q23, make_float2(fminf(kAlphaMax, raw23.x), fminf(kAlphaMax, raw23.y)));
+        float2 w01 = __fmul2_rn(al01, T01), w23 = __fmul2_rn(al23, T23);
+        // transmittance behind this entry, T - alpha T; below 1e-4 the pixel stops and the entry is not composited.
+        // A live pixel that skips the entry keeps T >= 1e-4 and cannot stop here; a stopped one has T = 0 and
+        // "stops" again with nothing to lose.
+        const float2 n01 = sub2(T01, w01), n23 = sub2(T23, w23);
+        const float2 s01 = make_float2(set_lt(n01.x, kTmin), set_lt(n01.y, kTmin));
+        const float2 s23 = make_float2(set_lt(n23.x, kTmin), set_lt(n23.y, kTmin));
+        const float2 k01 = sub2(one, s01), k23 = sub2(one, s23);
+        F01 = __ffma2_rn(s01, T01, F01); F23 = __ffma2_rn(s23, T23, F23);
+        w01 = __fmul2_rn(w01, k01); w23 = __fmul2_rn(w23, k23);
+        T01 = __fmul2_rn(n01, k01); T23 = __fmul2_rn(n23, k23);
+        R01 = __ffma2_rn(make_float2(col.x, col.x), w01, R01); R23 = __ffma2_rn(make_float2(col.x, col.x), w23, R23);
+        G01 = __ffma2_rn(make_float2(col.y, col.y), w01, G01); G23 = __ffma2_rn(make_float2(col.y, col.y), w23, G23);
+        B01 = __ffma2_rn(make_float2(col.z, col.z), w01, B01); B23 = __ffma2_rn(make_float2(col.z, col.z), w23, B23);
+        // last += composited * (position - last)
+        const float2 pos2 = make_float2(posf, posf);
+        last01 = __ffma2_rn(__fmul2_rn(q01, k01), sub2(pos2, last01), last01);
+        last23 = __ffma2_rn(__fmul2_rn(q23, k23), sub2(pos2, last23), last23);
       }
     }
+    const uint32_t off = base - start;
+    if (last01.x != 0.f) last[0] = off + (uint32_t)last01.x;
+    if (last01.y != 0.f) last[1] = off + (uint32_t)last01.y;
+    if (last23.x != 0.f) last[2] = off + (uint32_t)last23.x;
+    if (last23.y != 0.f) last[3] = off + (uint32_t)last23.y;
   }
+  T01 = __fadd2_rn(T01, F01); T23 = __fadd2_rn(T23, F23);    // one of the two is 0
+  const float T[4] = {T01.x, T01.y, T23.x, T23.y};
+  const float Cr[4] = {R01.x, R01.y, R23.x, R23.y}, Cg[4] = {G01.x, G01.y, G23.x, G23.y}, Cb[4] = {B01.x, B01.y, B23.x, B23.y};
   const size_t plane = (size_t)cam.W * cam.H;
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
@@ -241,6 +289,12 @@ __global__ void __launch_bounds__(kThreads, 16) k_blend_bwd(CamDev cam, const ui
   // value that this lane holds after the reduction (lanes 0, 4, .., 28: one of 0..7; lane 1 stores value 8)
   const int my_value = ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1);
   const int nbatches = (int)((maxc + kBatchBwd - 1) / kBatchBwd);
+  // pixels (0, 1) and (2, 3) as packed pairs; nGS carries minus G . (light from behind)
+  float2 T01 = make_float2(T[0], T[1]), T23 = make_float2(T[2], T[3]);
+  float2 nGS01 = make_float2(-GS[0], -GS[1]), nGS23 = make_float2(-GS[2], -GS[3]);
+  const float2 Gr01 = make_float2(Gr[0], Gr[1]), Gr23 = make_float2(Gr[2], Gr[3]);
+  const float2 Gg01 = make_float2(Gg[0], Gg[1]), Gg23 = make_float2(Gg[2], Gg[3]);
+  const float2 Gb01 = make_float2(Gb[0], Gb[1]), Gb23 = make_float2(Gb[2], Gb[3]);
   for (int b = nbatches - 1; b >= 0; --b) {
     __syncthreads();
     const uint32_t first = (uint32_t)b * kBatchBwd;
@@ -258,40 +312,55 @@ __global__ void __launch_bounds__(kThreads, 16) k_blend_bwd(CamDev cam, const ui
     }
     __syncthreads();
     const int jtop = (int)min((uint32_t)cnt, wmax > first ? wmax - first : 0u);
+    // positions of this batch that each pixel composited: j < lim[k]
+    int lim[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) lim[k] = nc[k] > first ? (int)(nc[k] - first) : 0;
     for (int j = jtop - 1; j >= 0; --j) {
-      const uint32_t pos = first + (uint32_t)j;
       const float4 a = s_xyab[j];
       const float2 c = s_co[j];
       float p[4], t1[4], t2[2];
       quad_power(fx - a.x, fy - a.y, a.z, a.w, c.x, p, t1, t2);
       const float4 col = s_rgb[j];
-      float dp[4] = {0.f, 0.f, 0.f, 0.f};
+      const bool q0 = j < lim[0] && !(p[0] < col.w), q1 = j < lim[1] && !(p[1] < col.w);
+      const bool q2 = j < lim[2] && !(p[2] < col.w), q3 = j < lim[3] && !(p[3] < col.w);
+      if (!__any_sync(kFull, q0 | q1 | q2 | q3)) continue;
+      // Branch-free from here, two packed pixel pairs: a pixel that did not composite this entry enters with
+      // alpha = 0, for which the reciprocal is 1, every product below is 0 and its carried state is unchanged.
+      const float2 o2 = make_float2(c.y, c.y), one = make_float2(1.f, 1.f), mone = make_float2(-1.f, -1.f);
+      const float2 raw01 = __fmul2_rn(o2, make_float2(ex2_approx(p[0]), ex2_approx(p[1])));
+      const float2 raw23 = __fmul2_rn(o2, make_float2(ex2_approx(p[2]), ex2_approx(p[3])));
+      const float2 al01 = make_float2(q0 ? fminf(kAlphaMax, raw01.x) : 0.f, q1 ? fminf(kAlphaMax, raw01.y) : 0.f);
+      const float2 al23 = make_float2(q2 ? fminf(kAlphaMax, raw23.x) : 0.f, q3 ? fminf(kAlphaMax, raw23.y) : 0.f);
+      const float2 d01 = __ffma2_rn(al01, mone, one), d23 = __ffma2_rn(al23, mone, one);
+      const float2 inv01 = make_float2(rcp_approx(d01.x), rcp_approx(d01.y)), inv23 = make_float2(rcp_approx(d23.x), rcp_approx(d23.y));
+      const float2 Tb01 = __fmul2_rn(T01, inv01), Tb23 = __fmul2_rn(T23, inv23);     // transmittance in front of this entry
+      const float2 w01 = __fmul2_rn(al01, Tb01), w23 = __fmul2_rn(al23, Tb23);
       float v[9];
-      v[6] = v[7] = v[8] = 0.f;
-      bool any = false;
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        float e2, raw, alpha;
-        if (pos >= nc[k] || !alpha_of(p[k], c.y, col.w, e2, raw, alpha)) continue;
-        any = true;
-        const float inv = rcp_approx(1.f - alpha);
-        const float Tb = T[k] * inv;              // transmittance in front of this entry
-        const float w = alpha * Tb;
-        v[6] = fmaf(w, Gr[k], v[6]); v[7] = fmaf(w, Gg[k], v[7]); v[8] = fmaf(w, Gb[k], v[8]);
-        // d pixel / d alpha = T c - S / (1 - alpha), S = everything composited behind this entry
-        const float gc = fmaf(Gb[k], col.z, fmaf(Gg[k], col.y, Gr[k] * col.x));
-        const float dalpha = fmaf(T[k], gc, -GS[k]) * inv;
-        if (raw <= kAlphaMax) dp[k] = alpha * dalpha;   // not clamped: alpha depends on o and power
-        GS[k] = fmaf(w, gc, GS[k]);
-        T[k] = Tb;
+      {
+        const float2 r = __ffma2_rn(w01, Gr01, __fmul2_rn(w23, Gr23)), g = __ffma2_rn(w01, Gg01, __fmul2_rn(w23, Gg23));
+        const float2 bl = __ffma2_rn(w01, Gb01, __fmul2_rn(w23, Gb23));
+        v[6] = r.x + r.y; v[7] = g.x + g.y; v[8] = bl.x + bl.y;
       }
-      if (__any_sync(kFull, any)) {
-        const float sL = dp[0] + dp[2], sR = dp[1] + dp[3], sT = dp[0] + dp[1], sB = dp[2] + dp[3];
+      // d pixel / d alpha = T c - S / (1 - alpha), S = everything composited behind this entry
+      const float2 cx = make_float2(col.x, col.x), cy = make_float2(col.y, col.y), cz = make_float2(col.z, col.z);
+      const float2 gc01 = __ffma2_rn(Gb01, cz, __ffma2_rn(Gg01, cy, __fmul2_rn(Gr01, cx)));
+      const float2 gc23 = __ffma2_rn(Gb23, cz, __ffma2_rn(Gg23, cy, __fmul2_rn(Gr23, cx)));
+      const float2 da01 = __fmul2_rn(__ffma2_rn(T01, gc01, nGS01), inv01), da23 = __fmul2_rn(__ffma2_rn(T23, gc23, nGS23), inv23);
+      const float2 e01 = __fmul2_rn(al01, da01), e23 = __fmul2_rn(al23, da23);
+      // clamped at 0.99: alpha does not depend on opacity and power there
+      const float dp0 = raw01.x <= kAlphaMax ? e01.x : 0.f, dp1 = raw01.y <= kAlphaMax ? e01.y : 0.f;
+      const float dp2 = raw23.x <= kAlphaMax ? e23.x : 0.f, dp3 = raw23.y <= kAlphaMax ? e23.y : 0.f;
+      nGS01 = __ffma2_rn(make_float2(-w01.x, -w01.y), gc01, nGS01);
+      nGS23 = __ffma2_rn(make_float2(-w23.x, -w23.y), gc23, nGS23);
+      T01 = Tb01; T23 = Tb23;
+      {
+        const float sL = dp0 + dp2, sR = dp1 + dp3, sT = dp0 + dp1, sB = dp2 + dp3;
         v[0] = sL + sR;
         v[1] = fmaf(X0, sL, X1 * sR);
         v[2] = fmaf(Y0, sT, Y1 * sB);
         v[3] = fmaf(XX0, sL, XX1 * sR);
-        v[4] = fmaf(X0, fmaf(Y0, dp[0], Y1 * dp[2]), X1 * fmaf(Y0, dp[1], Y1 * dp[3]));
+        v[4] = fmaf(X0, fmaf(Y0, dp0, Y1 * dp2), X1 * fmaf(Y0, dp1, Y1 * dp3));
         v[5] = fmaf(YY0, sT, YY1 * sB);
         float mine, ninth;
         warp_reduce9(v, lane, mine, ninth);
@@ -333,8 +402,9 @@ __global__ void __launch_bounds__(kThreads, 16) k_blend_bwd(CamDev cam, const ui
 }
 
 // Measurement only: replay the forward's decisions and count, over all pixels, the list entries
-// evaluated (until each pixel stopped) and the pairs composited.  counts[0] += evaluated,
-// counts[1] += composited.
+// evaluated (until each pixel stopped) and the pairs composited; and per warp (16 x 8 pixels) the
+// entries it walked and those among them that none of its live pixels accepted.
+// counts[0] += evaluated, counts[1] += composited, counts[2] += (warp, entry) steps, counts[3] += steps without a taker.
 __global__ void __launch_bounds__(kThreads) k_blend_count(CamDev cam, const uint32_t *__restrict__ ranges,
                                                           const uint32_t *__restrict__ vals,
                                                           const float *__restrict__ mean2d,
@@ -351,7 +421,7 @@ __global__ void __launch_bounds__(kThreads) k_blend_count(CamDev cam, const uint
   const uint32_t start = __ldg(ranges + 2 * tile), end = __ldg(ranges + 2 * tile + 1);
   float T[4] = {1.f, 1.f, 1.f, 1.f};
   unsigned live = 0;
-  unsigned long long evaluated = 0, composited = 0;
+  unsigned long long evaluated = 0, composited = 0, steps = 0, idle = 0;
 #pragma unroll
   for (int k = 0; k < 4; ++k)
     if (px + (k & 1) < cam.W && py + (k >> 1) < cam.H) live |= 1u << k;
@@ -365,22 +435,27 @@ __global__ void __launch_bounds__(kThreads) k_blend_count(CamDev cam, const uint
     }
     __syncthreads();
     const int cnt = (int)min((uint32_t)kBatch, end - base);
-    for (int j = 0; j < cnt && live; ++j) {
+    for (int j = 0; j < cnt; ++j) {
+      if (!__any_sync(kFull, live != 0)) break;
       const float4 a = s_xyab[j];
       const float2 c = s_co[j];
       float p[4], t1[4], t2[2];
       quad_power(fx - a.x, fy - a.y, a.z, a.w, c.x, p, t1, t2);
       const float4 col = s_rgb[j];
       evaluated += __popc(live);
+      bool taken = false;
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
         float e2, raw, alpha;
         if (!((live >> k) & 1u) || !alpha_of(p[k], c.y, col.w, e2, raw, alpha)) continue;
-        const float Tn = __fmul_rn(T[k], 1.f - alpha);
+        taken = true;
+        const float Tn = __fadd_rn(T[k], -__fmul_rn(alpha, T[k]));
         if (Tn < kTmin) { live &= ~(1u << k); continue; }
         T[k] = Tn;
         ++composited;
       }
+      ++steps;
+      if (!__any_sync(kFull, taken)) ++idle;
     }
   }
 #pragma unroll
@@ -388,7 +463,10 @@ __global__ void __launch_bounds__(kThreads) k_blend_count(CamDev cam, const uint
     evaluated += __shfl_xor_sync(kFull, evaluated, s);
     composited += __shfl_xor_sync(kFull, composited, s);
   }
-  if ((tid & 31) == 0) { atomicAdd(counts, evaluated); atomicAdd(counts + 1, composited); }
+  if ((tid & 31) == 0) {
+    atomicAdd(counts, evaluated); atomicAdd(counts + 1, composited);
+    atomicAdd(counts + 2, steps); atomicAdd(counts + 3, idle);     // warp-uniform: one lane speaks for the warp
+  }
 }
 
 }  // namespace
