@@ -344,7 +344,7 @@ GsStatus gs_neural_prepass(GsContext *ctx, const GsScene *scene, const uint16_t 
 typedef enum {
   GS_STAGE_PREPROCESS_FWD = 0, /* projection + fused colour decode                              */
   GS_STAGE_DEPTH_SORT,         /* radix sort of the Gaussians by depth key                      */
-  GS_STAGE_TILE_OFFSETS,       /* prefix sum of tiles touched, in depth order                   */
+  GS_STAGE_TILE_OFFSETS,       /* (the sums of tiles touched are taken by the depth sort's last pass: no time of its own) */
   GS_STAGE_KEYGEN,             /* instance emission                                             */
   GS_STAGE_TILE_SORT,          /* radix sort of the instances by tile id                        */
   GS_STAGE_TILE_RANGES,

@@ -381,18 +381,17 @@ GsStatus gs_render_forward(GsContext *ctx, int64_t n, const GsProjected *proj, c
   const CamDev cd = make_cam(cam);
   const int num_tiles = cd.gx * cd.gy;
   const FwdWorkspace w = carve_fwd(workspace, n, pair_capacity);
-  if (n > 0 && num_pairs > 0) {
-    // stage 1: Gaussians by depth key (stable => ties keep the index order)
+  const bool sorted = n > 0 && num_pairs > 0;
+  if (sorted) {
+    // stage 1: Gaussians by depth key (stable => ties keep the index order); the last pass also leaves the tiles
+    // touched per 256 sorted Gaussians, from which the instance emission takes its offsets
     {
       StageTimer t(ctx, GS_STAGE_DEPTH_SORT, s);
+      const SortEpilogue ep = {proj->tiles_touched, w.block_offsets, num_scan_blocks(n), nullptr, 0, nullptr};
       t.done(launch_radix_sort(proj->depth_key, nullptr, w.sorted_depth, bin->depth_order, w.tmp_keys, w.tmp_vals,
-                               n, nullptr, 32, w.sort_table, s));
+                               n, nullptr, 32, w.sort_table, &ep, s));
     }
-    // stage 2: instances in depth order, then a stable sort by tile id alone
-    {
-      StageTimer t(ctx, GS_STAGE_TILE_OFFSETS, s);
-      t.done(launch_tile_offsets(bin->depth_order, proj->tiles_touched, w.block_offsets, n, nullptr, s));
-    }
+    // stage 2: instances in depth order, then a stable sort by tile id alone, whose last pass finds the tile ranges
     {
       StageTimer t(ctx, GS_STAGE_KEYGEN, s);
       t.done(launch_keygen(bin->depth_order, proj->rect, proj->mean2d, proj->conic_opacity, proj->tiles_touched,
@@ -400,14 +399,14 @@ GsStatus gs_render_forward(GsContext *ctx, int64_t n, const GsProjected *proj, c
     }
     {
       StageTimer t(ctx, GS_STAGE_TILE_SORT, s);
+      const SortEpilogue ep = {nullptr, nullptr, 0, bin->tile_ranges, num_tiles, reinterpret_cast<uint32_t *>(ctx->d_counter + 2)};
       t.done(launch_radix_sort(w.inst_tiles, w.inst_vals, bin->sorted_tiles, bin->sorted_vals, w.tmp_tiles,
-                               w.tmp_ivals, num_pairs, count_dev, tile_bits(num_tiles), w.sort_table, s));
+                               w.tmp_ivals, num_pairs, count_dev, tile_bits(num_tiles), w.sort_table, &ep, s));
     }
   }
   {
     StageTimer t(ctx, GS_STAGE_TILE_RANGES, s);
-    t.done(launch_tile_ranges(bin->sorted_tiles, num_pairs, count_dev, reinterpret_cast<uint32_t *>(ctx->d_counter + 2),
-                              bin->tile_ranges, bin->tile_order, num_tiles, s));
+    t.done(launch_tile_order(bin->tile_ranges, bin->tile_order, num_tiles, !sorted, s));
   }
   {
     StageTimer t(ctx, GS_STAGE_BLEND_FWD, s);

@@ -95,20 +95,32 @@ int launch_unfused_prepare(int64_t n, const float *means, const CamDev &cam, con
 constexpr int kWgradBlocks = 592;   // persistent blocks of the decoder-gradient kernels (4 x 148)
 
 // Sorting / binning.
+// What the scatter of the last pass of a sort adds on its way out (nothing where the pointers are null).
+struct SortEpilogue {
+  // depth sort: sums of tiles touched per 256 consecutive Gaussians of the sorted order (the instance emission turns
+  // them into its offsets); cleared by the same pass
+  const uint32_t *tiles_touched;
+  uint32_t *block_sums;
+  int num_block_sums;
+  // tile sort: [start, end) of every tile in the sorted instance list (an empty tile is left at (0xffffffff, 0) for
+  // launch_tile_order to settle), and the flag raised when a device-side instance count exceeded the capacity
+  uint32_t *ranges;
+  int num_tiles;
+  uint32_t *overflow;
+};
 size_t sort_scratch_bytes(int64_t count);
 // LSD radix sort of (key, val) pairs on bits [0, num_bits).  If vals_in == nullptr the values are
 // the element indices.  Result lands in keys_out / vals_out; tmp_* are same-sized alternates.
 int launch_radix_sort(const uint32_t *keys_in, const uint32_t *vals_in, uint32_t *keys_out,
                        uint32_t *vals_out, uint32_t *tmp_keys, uint32_t *tmp_vals, int64_t count,
-                       const unsigned long long *count_dev, int num_bits, void *scratch, cudaStream_t st);
+                       const unsigned long long *count_dev, int num_bits, void *scratch, const SortEpilogue *epilogue,
+                       cudaStream_t st);
 size_t scan_scratch_bytes(int64_t n);
-int launch_tile_offsets(const uint32_t *depth_order, const uint32_t *tiles_touched, uint32_t *offsets,
-                        int64_t n, void *scratch, cudaStream_t st);
+int num_scan_blocks(int64_t n);   // entries of the block sums that launch_keygen reads
 int launch_keygen(const uint32_t *depth_order, const uint16_t *rect, const float *mean2d, const float *conic_opacity,
-                  const uint32_t *tiles_touched, const uint32_t *offsets, uint32_t *inst_tiles, uint32_t *inst_vals,
+                  const uint32_t *tiles_touched, const uint32_t *block_sums, uint32_t *inst_tiles, uint32_t *inst_vals,
                   int64_t n, int gx, int W, int H, int64_t capacity, cudaStream_t st);
-int launch_tile_ranges(const uint32_t *sorted_tiles, int64_t P, const unsigned long long *count_dev, uint32_t *overflow,
-                       uint32_t *ranges, uint32_t *order, int num_tiles, cudaStream_t st);
+int launch_tile_order(uint32_t *ranges, uint32_t *order, int num_tiles, bool clear, cudaStream_t st);
 
 // Blend.
 int launch_blend_fwd(const CamDev &cam, const uint32_t *ranges, const uint32_t *order, const uint32_t *vals,

@@ -16,6 +16,7 @@ constexpr int kItems = 16;
 constexpr int kSortTile = kSortThreads * kItems;   // 4096 elements per block iteration
 constexpr int kMaxSortBlocks = 444;                // 3 resident CTAs x 148 SMs: one full wave
 constexpr unsigned kFull = 0xffffffffu;
+constexpr int kScanBlock = 256;   // Gaussians per block of the tiles-touched prefix sum and per CTA of the instance emission
 
 // Block b sorts tiles_per_block (+ 1 if b < extra) consecutive tiles of kSortTile elements: the tiles are dealt
 // out as evenly as whole tiles allow over one full wave of CTAs.
@@ -42,8 +43,18 @@ __device__ __forceinline__ void block_tiles(int tiles_per_block, int extra, int6
 __global__ void __launch_bounds__(kSortThreads) k_radix_hist(const uint32_t *__restrict__ keys, int64_t count,
                                                              const unsigned long long *__restrict__ count_dev,
                                                              int shift, uint32_t mask, int tiles_per_block, int extra,
-                                                             uint32_t *__restrict__ table) {
-  if (count_dev) count = min(count, (int64_t)__ldg(count_dev));   // the true length lives on the device
+                                                             uint32_t *__restrict__ table, SortEpilogue ep) {
+  // the arrays the scatter of this pass accumulates into start from their neutral values
+  if (ep.block_sums)
+    for (int i = blockIdx.x * kSortThreads + threadIdx.x; i < ep.num_block_sums; i += gridDim.x * kSortThreads) ep.block_sums[i] = 0u;
+  if (ep.ranges)
+    for (int i = blockIdx.x * kSortThreads + threadIdx.x; i < 2 * ep.num_tiles; i += gridDim.x * kSortThreads)
+      ep.ranges[i] = (i & 1) ? 0u : 0xffffffffu;
+  if (count_dev) {
+    const int64_t c = (int64_t)__ldg(count_dev);                    // the true length lives on the device
+    if (ep.overflow && c > count && blockIdx.x == 0 && threadIdx.x == 0) *ep.overflow = 1u;   // lists were cut off: tell the host
+    count = min(count, c);
+  }
   __shared__ uint32_t s_hist[kSortWarps][256];
   const int tid = threadIdx.x, warp = tid >> 5;
   for (int k = tid; k < kSortWarps * 256; k += kSortThreads) (&s_hist[0][0])[k] = 0;
@@ -118,12 +129,16 @@ __device__ __forceinline__ uint32_t block_exclusive_scan_256(uint32_t v, uint32_
 // One pass: stable scatter of this block's range by the BITS-wide digit at `shift`.  Slots past the
 // end of the input carry the largest digit and sit at the end of the last tile, so they rank after
 // every real key and are never written.
-template <int BITS>
+// EP selects the epilogue: 0 none, 1 block sums of tiles touched (last pass of the depth sort), 2 tile ranges (last
+// pass of the tile sort: inside a block's run of one digit the keys are non-decreasing, because the earlier passes
+// ordered the lower bits, so a change of key between neighbours of a run is a tile boundary; the two ends of a run
+// may continue in another block and enter with an atomic min / max).
+template <int BITS, int EP>
 __global__ void __launch_bounds__(kSortThreads, 3) k_radix_scatter(
     const uint32_t *__restrict__ keys_in, const uint32_t *__restrict__ vals_in, uint32_t *__restrict__ keys_out,
     uint32_t *__restrict__ vals_out, int64_t count, const unsigned long long *__restrict__ count_dev, int shift,
     int tiles_per_block, int extra,
-    const uint32_t *__restrict__ table, const uint32_t *__restrict__ totals, int nblocks) {
+    const uint32_t *__restrict__ table, const uint32_t *__restrict__ totals, int nblocks, SortEpilogue ep) {
   __shared__ uint32_t s_keys[kSortTile];
   __shared__ uint32_t s_vals[kSortTile];
   __shared__ uint32_t s_warp_cnt[kSortWarps][256];
@@ -207,12 +222,39 @@ __global__ void __launch_bounds__(kSortThreads, 3) k_radix_scatter(
       s_vals[pos] = val[it];
     }
     __syncthreads();
-    for (int j = tid; j < valid_count; j += kSortThreads) {
-      const uint32_t k = s_keys[j];
-      const uint32_t d = (k >> shift) & kDigitMask;
-      const uint32_t gpos = s_base[d] + ((uint32_t)j - s_digit_start[d]);
-      keys_out[gpos] = k;
-      vals_out[gpos] = s_vals[j];
+    for (int j0 = 0; j0 < valid_count; j0 += kSortThreads) {
+      const int j = j0 + tid;
+      const bool ok = j < valid_count;
+      uint32_t k = 0, d = 0, gpos = 0, v = 0;
+      if (ok) {
+        k = s_keys[j];
+        d = (k >> shift) & kDigitMask;
+        gpos = s_base[d] + ((uint32_t)j - s_digit_start[d]);
+        v = s_vals[j];
+        keys_out[gpos] = k;
+        vals_out[gpos] = v;
+      }
+      if (EP == 1) {
+        // tiles touched by this Gaussian, added to the sum of its block of kScanBlock sorted positions; a warp whose
+        // lanes all fall into one block (the usual case: a run is contiguous) adds once
+        uint32_t tt = ok ? __ldg(ep.tiles_touched + v) : 0u;
+        const uint32_t blk = gpos / kScanBlock, blk0 = __shfl_sync(kFull, blk, 0);
+        if (__all_sync(kFull, !ok || blk == blk0)) {
+#pragma unroll
+          for (int sft = 16; sft > 0; sft >>= 1) tt += __shfl_xor_sync(kFull, tt, sft);
+          if (lane == 0 && tt) atomicAdd(ep.block_sums + blk0, tt);
+        } else if (tt) {
+          atomicAdd(ep.block_sums + blk, tt);
+        }
+      }
+      if (EP == 2 && ok) {
+        const uint32_t run_first = s_digit_start[d];
+        const uint32_t run_end = d == kDigitMask ? (uint32_t)valid_count : s_digit_start[d + 1];   // slots past the input hold no run
+        if ((uint32_t)j == run_first) atomicMin(ep.ranges + 2 * k, gpos);
+        else if (s_keys[j - 1] != k) ep.ranges[2 * k] = gpos;
+        if ((uint32_t)j + 1 == run_end) atomicMax(ep.ranges + 2 * k + 1, gpos + 1);
+        else if (s_keys[j + 1] != k) ep.ranges[2 * k + 1] = gpos + 1;
+      }
     }
     __syncthreads();
     s_base[tid] += cnt;
@@ -221,61 +263,6 @@ __global__ void __launch_bounds__(kSortThreads, 3) k_radix_scatter(
 }
 
 // ---- tiles touched in depth order -----------------------------------------------------------
-constexpr int kScanBlock = 256;
-
-__global__ void __launch_bounds__(kScanBlock) k_tiles_block_sums(const uint32_t *__restrict__ order,
-                                                                 const uint32_t *__restrict__ tiles_touched, int64_t n,
-                                                                 uint32_t *__restrict__ block_sums) {
-  __shared__ uint32_t s_w[kScanBlock / 32];
-  const int64_t i = (int64_t)blockIdx.x * kScanBlock + threadIdx.x;
-  uint32_t v = i < n ? __ldg(tiles_touched + __ldg(order + i)) : 0u;
-#pragma unroll
-  for (int s = 16; s > 0; s >>= 1) v += __shfl_xor_sync(kFull, v, s);
-  if ((threadIdx.x & 31) == 0) s_w[threadIdx.x >> 5] = v;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    uint32_t t = 0;
-#pragma unroll
-    for (int w = 0; w < kScanBlock / 32; ++w) t += s_w[w];
-    block_sums[blockIdx.x] = t;
-  }
-}
-
-// In-place exclusive scan of `count` values by one block.
-__global__ void __launch_bounds__(1024) k_scan_single_block(uint32_t *__restrict__ data, int count) {
-  __shared__ uint32_t s_w[32];
-  __shared__ uint32_t s_carry;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (tid == 0) s_carry = 0;
-  __syncthreads();
-  for (int base = 0; base < count; base += 1024) {
-    const int i = base + tid;
-    const uint32_t v = i < count ? data[i] : 0u;
-    uint32_t inc = v;
-#pragma unroll
-    for (int s = 1; s < 32; s <<= 1) {
-      const uint32_t t = __shfl_up_sync(kFull, inc, s);
-      if (lane >= s) inc += t;
-    }
-    if (lane == 31) s_w[warp] = inc;
-    __syncthreads();
-    if (warp == 0) {
-      uint32_t w = s_w[lane], winc = w;
-#pragma unroll
-      for (int s = 1; s < 32; s <<= 1) {
-        const uint32_t t = __shfl_up_sync(kFull, winc, s);
-        if (lane >= s) winc += t;
-      }
-      s_w[lane] = winc - w;
-    }
-    __syncthreads();
-    const uint32_t carry = s_carry;
-    if (i < count) data[i] = carry + s_w[warp] + inc - v;
-    __syncthreads();
-    if (tid == 1023) s_carry = carry + s_w[warp] + inc;
-    __syncthreads();
-  }
-}
 
 // Emit the instances of each Gaussian, in depth order: the tiles its alpha >= 1/255 ellipse meets
 // (TileSpans, the same function the preprocess counted with), tile rows top to bottom, tiles left
@@ -286,11 +273,11 @@ __global__ void __launch_bounds__(kScanBlock) k_keygen(const uint32_t *__restric
                                                        const float *__restrict__ mean2d,
                                                        const float *__restrict__ conic_opacity,
                                                        const uint32_t *__restrict__ tiles_touched,
-                                                       const uint32_t *__restrict__ block_offsets, int64_t n, int gx,
+                                                       const uint32_t *__restrict__ block_sums, int64_t n, int gx,
                                                        int W, int H, uint32_t capacity,
                                                        uint32_t *__restrict__ inst_tiles,
                                                        uint32_t *__restrict__ inst_vals) {
-  __shared__ uint32_t s_w[kScanBlock / 32];
+  __shared__ uint32_t s_w[kScanBlock / 32], s_before[kScanBlock / 32];
   __shared__ uint32_t s_stage[kScanBlock / 32][2 * kKeygenStage];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int64_t i = (int64_t)blockIdx.x * kScanBlock + tid;
@@ -318,10 +305,17 @@ __global__ void __launch_bounds__(kScanBlock) k_keygen(const uint32_t *__restric
     if (lane >= s) inc += t;
   }
   if (lane == 31) s_w[warp] = inc;
-  __syncthreads();
-  uint32_t off = __ldg(block_offsets + blockIdx.x);
+  // instances of all CTAs before this one: the sums per kScanBlock Gaussians come from the last pass of the depth
+  // sort; every CTA adds up its own prefix (a few loads per thread) instead of a scan kernel doing it for all
+  uint32_t before = 0;
+  for (int k = tid; k < (int)blockIdx.x; k += kScanBlock) before += __ldg(block_sums + k);
 #pragma unroll
-  for (int k = 0; k < kScanBlock / 32; ++k) off += (k < warp) ? s_w[k] : 0u;
+  for (int sft = 16; sft > 0; sft >>= 1) before += __shfl_xor_sync(kFull, before, sft);
+  if (lane == 0) s_before[warp] = before;
+  __syncthreads();
+  uint32_t off = 0;
+#pragma unroll
+  for (int k = 0; k < kScanBlock / 32; ++k) off += s_before[k] + ((k < warp) ? s_w[k] : 0u);
   off += inc - tiles;
   constexpr uint32_t kSmall = 32;
   // A warp whose footprints add up to at most kKeygenStage instances writes them to shared memory first and
@@ -400,46 +394,18 @@ __global__ void __launch_bounds__(kScanBlock) k_keygen(const uint32_t *__restric
   }
 }
 
-// Four consecutive entries per thread (one 16-byte load plus the two neighbours).
-__global__ void __launch_bounds__(256) k_tile_ranges(const uint32_t *__restrict__ sorted_tiles, int64_t P,
-                                                     const unsigned long long *__restrict__ count_dev,
-                                                     uint32_t *__restrict__ overflow, uint32_t *__restrict__ ranges) {
-  const int64_t p0 = 4 * ((int64_t)blockIdx.x * blockDim.x + threadIdx.x);
-  if (count_dev) {   // P is the capacity here; more instances than that were cut off: tell the host
-    const int64_t c = (int64_t)__ldg(count_dev);
-    if (p0 == 0 && c > P) *overflow = 1u;
-    P = min(P, c);
-  }
-  if (p0 >= P) return;
-  uint32_t t[6];   // entries p0 - 1 .. p0 + 4
-  if (p0 + 4 <= P) {
-    const uint4 v = __ldg(reinterpret_cast<const uint4 *>(sorted_tiles + p0));
-    t[1] = v.x; t[2] = v.y; t[3] = v.z; t[4] = v.w;
-  } else {
-#pragma unroll
-    for (int k = 0; k < 4; ++k) t[1 + k] = p0 + k < P ? __ldg(sorted_tiles + p0 + k) : 0u;
-  }
-  t[0] = p0 > 0 ? __ldg(sorted_tiles + p0 - 1) : 0u;
-  t[5] = p0 + 4 < P ? __ldg(sorted_tiles + p0 + 4) : 0u;
-#pragma unroll
-  for (int k = 0; k < 4; ++k) {
-    const int64_t p = p0 + k;
-    if (p >= P) break;
-    if (p == 0 || t[1 + k] != t[k]) ranges[2 * t[1 + k]] = (uint32_t)p;
-    if (p == P - 1 || t[1 + k] != t[2 + k]) ranges[2 * t[1 + k] + 1] = (uint32_t)(p + 1);
-  }
-}
-
 // Launch order of the blend CTAs: tiles by decreasing list length (log2 buckets), so that the long
 // tiles start first and the short ones fill the tail.  The order inside a bucket is whatever the
 // atomics give; it affects scheduling only, never a result.
-__global__ void __launch_bounds__(1024) k_tile_order(const uint32_t *__restrict__ ranges, int num_tiles,
+// A tile without instances comes in as (0xffffffff, 0), the neutral values of the range epilogue, and leaves as (0, 0).
+__global__ void __launch_bounds__(1024) k_tile_order(uint32_t *__restrict__ ranges, int num_tiles,
                                                      uint32_t *__restrict__ order) {
   __shared__ uint32_t s_cnt[33], s_off[33];
   const int tid = threadIdx.x;
   if (tid < 33) s_cnt[tid] = 0;
   __syncthreads();
   for (int t = tid; t < num_tiles; t += 1024) {
+    if (ranges[2 * t + 1] == 0u) ranges[2 * t] = 0u;
     const uint32_t len = ranges[2 * t + 1] - ranges[2 * t];
     atomicAdd(&s_cnt[len ? 32 - __clz(len) : 0], 1u);
   }
@@ -461,7 +427,7 @@ size_t sort_scratch_bytes(int64_t count) { return ((size_t)plan_for(count).block
 
 int launch_radix_sort(const uint32_t *keys_in, const uint32_t *vals_in, uint32_t *keys_out, uint32_t *vals_out,
                        uint32_t *tmp_keys, uint32_t *tmp_vals, int64_t count, const unsigned long long *count_dev,
-                       int num_bits, void *scratch, cudaStream_t st) {
+                       int num_bits, void *scratch, const SortEpilogue *epilogue, cudaStream_t st) {
   if (count <= 0) return 0;
   const SortPlan plan = plan_for(count);
   int passes = (num_bits + 7) / 8;
@@ -470,24 +436,32 @@ int launch_radix_sort(const uint32_t *keys_in, const uint32_t *vals_in, uint32_t
   uint32_t *table = static_cast<uint32_t *>(scratch);
   uint32_t *totals = table + (size_t)plan.blocks * 256;
   const uint32_t *src_k = keys_in, *src_v = vals_in;
+  const SortEpilogue none = {nullptr, nullptr, 0, nullptr, 0, nullptr};
   for (int p = 0; p < passes; ++p) {
     const bool to_out = ((passes - 1 - p) % 2) == 0;
     uint32_t *dst_k = to_out ? keys_out : tmp_keys, *dst_v = to_out ? vals_out : tmp_vals;
+    const SortEpilogue ep = (p == passes - 1 && epilogue) ? *epilogue : none;
+    const int mode = ep.block_sums ? 1 : ep.ranges ? 2 : 0;
     k_radix_hist<<<plan.blocks, kSortThreads, 0, st>>>(src_k, count, count_dev, bits * p, (1u << bits) - 1u,
-                                                        plan.tiles_per_block, plan.extra, table);
+                                                        plan.tiles_per_block, plan.extra, table, ep);
     k_radix_scan_rows<<<256, 256, 0, st>>>(table, plan.blocks, totals);
-#define GS_SCATTER(B)                                                                                              \
-  case B:                                                                                                          \
-    k_radix_scatter<B><<<plan.blocks, kSortThreads, 0, st>>>(src_k, src_v, dst_k, dst_v, count, count_dev, bits * p, \
-                                                              plan.tiles_per_block, plan.extra, table, totals, plan.blocks);   \
+#define GS_SCATTER_ARGS                                                                                              \
+  <<<plan.blocks, kSortThreads, 0, st>>>(src_k, src_v, dst_k, dst_v, count, count_dev, bits * p, plan.tiles_per_block, \
+                                         plan.extra, table, totals, plan.blocks, ep)
+#define GS_SCATTER(B)                                              \
+  case B:                                                          \
+    if (mode == 2) k_radix_scatter<B, 2> GS_SCATTER_ARGS;          \
+    else k_radix_scatter<B, 0> GS_SCATTER_ARGS;                    \
     break;
     switch (bits) {
       GS_SCATTER(1) GS_SCATTER(2) GS_SCATTER(3) GS_SCATTER(4) GS_SCATTER(5) GS_SCATTER(6) GS_SCATTER(7)
       default:
-        k_radix_scatter<8><<<plan.blocks, kSortThreads, 0, st>>>(src_k, src_v, dst_k, dst_v, count, count_dev, bits * p,
-                                                                  plan.tiles_per_block, plan.extra, table, totals, plan.blocks);
+        if (mode == 1) k_radix_scatter<8, 1> GS_SCATTER_ARGS;
+        else if (mode == 2) k_radix_scatter<8, 2> GS_SCATTER_ARGS;
+        else k_radix_scatter<8, 0> GS_SCATTER_ARGS;
     }
 #undef GS_SCATTER
+#undef GS_SCATTER_ARGS
     src_k = dst_k;
     src_v = dst_v;
   }
@@ -495,33 +469,25 @@ int launch_radix_sort(const uint32_t *keys_in, const uint32_t *vals_in, uint32_t
 }
 
 size_t scan_scratch_bytes(int64_t n) { return (size_t)((n + kScanBlock - 1) / kScanBlock + 1) * sizeof(uint32_t); }
-
-int launch_tile_offsets(const uint32_t *depth_order, const uint32_t *tiles_touched, uint32_t *block_offsets, int64_t n,
-                        void *, cudaStream_t st) {
-  if (n <= 0) return 0;
-  const int blocks = (int)((n + kScanBlock - 1) / kScanBlock);
-  k_tiles_block_sums<<<blocks, kScanBlock, 0, st>>>(depth_order, tiles_touched, n, block_offsets);
-  k_scan_single_block<<<1, 1024, 0, st>>>(block_offsets, blocks);
-  return 2;
-}
+int num_scan_blocks(int64_t n) { return (int)((n + kScanBlock - 1) / kScanBlock); }
 
 int launch_keygen(const uint32_t *depth_order, const uint16_t *rect, const float *mean2d, const float *conic_opacity,
-                  const uint32_t *tiles_touched, const uint32_t *block_offsets, uint32_t *inst_tiles, uint32_t *inst_vals,
+                  const uint32_t *tiles_touched, const uint32_t *block_sums, uint32_t *inst_tiles, uint32_t *inst_vals,
                   int64_t n, int gx, int W, int H, int64_t capacity, cudaStream_t st) {
   if (n <= 0) return 0;
-  const int blocks = (int)((n + kScanBlock - 1) / kScanBlock);
+  const int blocks = num_scan_blocks(n);
   const uint32_t cap = capacity > 0xffffffffll ? 0xffffffffu : (uint32_t)capacity;
-  k_keygen<<<blocks, kScanBlock, 0, st>>>(depth_order, rect, mean2d, conic_opacity, tiles_touched, block_offsets, n, gx, W, H,
+  k_keygen<<<blocks, kScanBlock, 0, st>>>(depth_order, rect, mean2d, conic_opacity, tiles_touched, block_sums, n, gx, W, H,
                                           cap, inst_tiles, inst_vals);
   return 1;
 }
 
-int launch_tile_ranges(const uint32_t *sorted_tiles, int64_t P, const unsigned long long *count_dev, uint32_t *overflow,
-                       uint32_t *ranges, uint32_t *order, int num_tiles, cudaStream_t st) {
-  cudaMemsetAsync(ranges, 0, (size_t)num_tiles * 2 * sizeof(uint32_t), st);
-  if (P > 0) k_tile_ranges<<<(int)((P + 1023) / 1024), 256, 0, st>>>(sorted_tiles, P, count_dev, overflow, ranges);
+// Settles the ranges of the empty tiles and orders the tiles for the blend launches.  With `clear` (no instance was
+// sorted, so no range epilogue ran) every range is zeroed first.
+int launch_tile_order(uint32_t *ranges, uint32_t *order, int num_tiles, bool clear, cudaStream_t st) {
+  if (clear) cudaMemsetAsync(ranges, 0, (size_t)num_tiles * 2 * sizeof(uint32_t), st);
   k_tile_order<<<1, 1024, 0, st>>>(ranges, num_tiles, order);
-  return P > 0 ? 2 : 1;
+  return 1;
 }
 
 }  // namespace gs
