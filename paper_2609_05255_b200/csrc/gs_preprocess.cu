@@ -230,13 +230,29 @@ __device__ __forceinline__ void load_features(const __half *features, int64_t i,
 __device__ __forceinline__ void decoder_inputs(float dx, float dy, float dz, const float f[8], int deg, float x[32]) {
   sh_basis(dx, dy, dz, x);
   const int na = (deg + 1) * (deg + 1);
+  if (na < 16) {
 #pragma unroll
-  for (int k = 0; k < 16; ++k) x[k] = k < na ? x[k] : 0.f;
-#pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    if (fabsf(f[j]) <= 3.14159265f) __sincosf(f[j], &x[16 + 2 * j], &x[17 + 2 * j]);
-    else sincosf(f[j], &x[16 + 2 * j], &x[17 + 2 * j]);
+    for (int k = 0; k < 16; ++k) x[k] = k < na ? x[k] : 0.f;
   }
+  float big = 0.f;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) big = fmaxf(big, fabsf(f[j]));
+  if (big <= 3.14159265f) {   // one decision for the eight of them: features are O(0.1 .. 1)
+#pragma unroll
+    for (int j = 0; j < 8; ++j) __sincosf(f[j], &x[16 + 2 * j], &x[17 + 2 * j]);
+  } else {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) sincosf(f[j], &x[16 + 2 * j], &x[17 + 2 * j]);
+  }
+}
+
+// tanh(y) = 1 - 2 / (e^{2y} + 1) on the exponential and reciprocal units: absolute error of a few 1e-7 over the
+// whole range (the residual is an absolute colour offset, so that is the error that counts), saturating to +-1.
+__device__ __forceinline__ float tanh_fast(float y) {
+  const float e = ex2_approx(y * 2.885390081777927f);    // 2 log2(e)
+  float r;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(e + 1.f));
+  return fmaf(-2.f, r, 1.f);
 }
 
 // Forward-only staging of the tensor-core decoder: the leading members of mlp::WarpStage.
@@ -249,12 +265,12 @@ struct __align__(16) StageFwd {
 // Whole-warp decode: every lane passes its Gaussian's inputs (zeros if it has none) and gets the
 // tanh-bounded residual A back.  All 32 lanes must call it.
 template <bool kSplit, class Stage>
-__device__ __forceinline__ void decode_warp(const mlp::Weights &W, Stage &S, int lane, const float x[32],
+__device__ __forceinline__ void decode_warp(const mlp::FwdFrags &F, Stage &S, int lane, const float x[32],
                                             mlp::Activations &act, float A[3]) {
   mlp::stage_inputs<kSplit>(x, S, lane);
-  mlp::forward_warp<kSplit>(W, S, lane, act);
-#pragma unroll
-  for (int c = 0; c < 3; ++c) A[c] = tanhf(S.y[lane * 4 + c]);
+  mlp::forward_warp<kSplit>(F, S, lane, act);
+  const float4 y = *reinterpret_cast<const float4 *>(S.y + lane * 4);
+  A[0] = tanh_fast(y.x); A[1] = tanh_fast(y.y); A[2] = tanh_fast(y.z);
 }
 
 // Whole-warp backward of the decoder.  `has`: this lane owns a Gaussian (inputs x, direction d, base
@@ -267,7 +283,10 @@ __device__ __forceinline__ void decode_backward_warp(const mlp::Weights &W, mlp:
                                                      float gp[3], float gf[8], float gd[3]) {
   mlp::Activations act;
   float A[3];
-  decode_warp<kSplit>(W, S, lane, x, act, A);
+  {
+    const mlp::FwdFrags F = mlp::load_fwd_frags(W.w, lane);   // out of shared memory, every trip: the registers are needed elsewhere
+    decode_warp<kSplit>(F, S, lane, x, act, A);
+  }
   float gy[3];
 #pragma unroll
   for (int c = 0; c < 3; ++c) {
@@ -446,16 +465,11 @@ __device__ __forceinline__ void load3(const float *p, int64_t i, float v[3]) {
 template <int APP>
 __global__ void __launch_bounds__(kBlock) k_preprocess_fwd(PreprocessArgs a, CamDev cam) {
   __shared__ __align__(16) float sData[Explicit<APP>::value ? kWarps * SlabOf<APP>::value : 4];
-  __shared__ __align__(16) unsigned char sNN[IsNeural<APP>::value ? sizeof(mlp::Weights) + kWarps * sizeof(StageFwd) : 16];
-  mlp::Weights *sWt = reinterpret_cast<mlp::Weights *>(sNN);
-  StageFwd *sStage = reinterpret_cast<StageFwd *>(sNN + (IsNeural<APP>::value ? sizeof(mlp::Weights) : 0));   // unused for SH
+  __shared__ __align__(16) unsigned char sNN[IsNeural<APP>::value ? kWarps * sizeof(StageFwd) : 16];
+  StageFwd *sStage = reinterpret_cast<StageFwd *>(sNN);   // unused for SH
   __shared__ unsigned int sPairs[kWarps];
   __shared__ unsigned long long sBar[kWarps];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (IsNeural<APP>::value) {
-    mlp::load_weights(a.weights, sWt[0], tid, kBlock);
-    __syncthreads();
-  }
   const int64_t i = (int64_t)blockIdx.x * kBlock + tid;
   const int64_t row0 = (int64_t)blockIdx.x * kBlock + warp * 32;
   const bool in = i < a.n;
@@ -529,7 +543,9 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_fwd(PreprocessArgs a, Cam
         for (int k = 0; k < 32; ++k) x[k] = 0.f;
       }
       mlp::Activations act;
-      decode_warp<Split<APP>::value>(sWt[0], sStage[warp], lane, x, act, A);
+      // the lane's 14 words of the forward's weight operands come straight from global memory (1.6 KB that stay in L1)
+      const mlp::FwdFrags F = mlp::load_fwd_frags(a.weights, lane);
+      decode_warp<Split<APP>::value>(F, sStage[warp], lane, x, act, A);
     }
     if (vis) {
       float base[3];
@@ -844,33 +860,35 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_bwd(PreprocessBwdArgs a, 
 template <int APP>
 __global__ void __launch_bounds__(kBlock) k_appearance_fwd(AppearanceArgs a) {
   static_assert(IsNeural<APP>::value, "the neural model in either decoder precision");
-  __shared__ __align__(16) unsigned char sNN[sizeof(mlp::Weights) + kWarps * sizeof(StageFwd)];
-  mlp::Weights *sWt = reinterpret_cast<mlp::Weights *>(sNN);
-  StageFwd *sStage = reinterpret_cast<StageFwd *>(sNN + sizeof(mlp::Weights));
+  __shared__ __align__(16) StageFwd sStage[kWarps];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  mlp::load_weights(a.weights, sWt[0], tid, kBlock);
-  __syncthreads();
-  const int64_t i = (int64_t)blockIdx.x * kBlock + tid;
-  const int64_t row0 = (int64_t)blockIdx.x * kBlock + warp * 32;
-  const bool in = i < a.n && (!a.mask || __ldg(a.mask + i) != 0u);   // masked-out Gaussians are skipped
-  float d[3] = {0.f, 0.f, 1.f}, base[3] = {0.f, 0.f, 0.f}, A[3] = {0.f, 0.f, 0.f};
-  if (in) { load3(a.dirs, i, d); load3(a.base_color, i, base); }
-  if (a.deg > 0 && row0 < a.n) {   // the whole warp decodes; lanes without a Gaussian feed zeros
-    float x[32];
-    if (in) {
-      float f[8];
-      load_features(a.features, i, f);
-      decoder_inputs(d[0], d[1], d[2], f, a.deg, x);
-    } else {
+  // persistent: the forward's weight operands are read once into 14 registers per lane and serve every trip
+  const mlp::FwdFrags F = mlp::load_fwd_frags(a.weights, lane);
+  const int64_t nchunks = (a.n + kBlock - 1) / kBlock;
+  for (int64_t chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x) {
+    const int64_t i = chunk * kBlock + tid;
+    const int64_t row0 = chunk * kBlock + warp * 32;
+    const bool in = i < a.n && (!a.mask || __ldg(a.mask + i) != 0u);   // masked-out Gaussians are skipped
+    float d[3] = {0.f, 0.f, 1.f}, base[3] = {0.f, 0.f, 0.f}, A[3] = {0.f, 0.f, 0.f};
+    if (in) { load3(a.dirs, i, d); load3(a.base_color, i, base); }
+    if (a.deg > 0 && row0 < a.n) {   // the whole warp decodes; lanes without a Gaussian feed zeros
+      float x[32];
+      if (in) {
+        float f[8];
+        load_features(a.features, i, f);
+        decoder_inputs(d[0], d[1], d[2], f, a.deg, x);
+      } else {
 #pragma unroll
-      for (int k = 0; k < 32; ++k) x[k] = 0.f;
+        for (int k = 0; k < 32; ++k) x[k] = 0.f;
+      }
+      mlp::Activations act;
+      decode_warp<Split<APP>::value>(F, sStage[warp], lane, x, act, A);
+      __syncwarp();   // the staging area is free for the next trip
     }
-    mlp::Activations act;
-    decode_warp<Split<APP>::value>(sWt[0], sStage[warp], lane, x, act, A);
+    if (in)
+      store3(a.color, i, color_act_z(a.act, base[0] + 0.5f + A[0]), color_act_z(a.act, base[1] + 0.5f + A[1]),
+             color_act_z(a.act, base[2] + 0.5f + A[2]));
   }
-  if (in)
-    store3(a.color, i, color_act_z(a.act, base[0] + 0.5f + A[0]), color_act_z(a.act, base[1] + 0.5f + A[1]),
-           color_act_z(a.act, base[2] + 0.5f + A[2]));
 }
 
 template <int APP>
@@ -1058,7 +1076,7 @@ void opt_in_smem(K kernel, size_t bytes) {
 // Grid of a persistent kernel: as many CTAs as fit on the device at once (a second, thinner wave of a
 // grid-stride loop would run at a fraction of the occupancy), at most kWgradBlocks (rows of the partial buffer).
 template <auto kernel>      // one cache per kernel, not per signature
-int resident_blocks(size_t smem_bytes) {
+int resident_blocks(size_t smem_bytes, int cap = kWgradBlocks) {
   static int cached[64] = {};
   int dev = 0;
   cudaGetDevice(&dev);
@@ -1068,7 +1086,7 @@ int resident_blocks(size_t smem_bytes) {
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kBlock, smem_bytes) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || per_sm <= 0 || sms <= 0)
       return kWgradBlocks;
-    cached[dev] = per_sm * sms < kWgradBlocks ? per_sm * sms : kWgradBlocks;
+    cached[dev] = per_sm * sms < cap ? per_sm * sms : cap;
   }
   return cached[dev];
 }
@@ -1136,8 +1154,14 @@ int launch_appearance_fwd(int app, const AppearanceArgs &a, cudaStream_t st) {
   if (a.n == 0) return 0;
   if (app == GS_APP_SH) return launch_bulk<GS_APP_SH, false>(a, st);
   if (app == GS_APP_SV) return launch_bulk<GS_APP_SV, false>(a, st);
-  if (app == kAppNeuralHalf) k_appearance_fwd<kAppNeuralHalf><<<grid_for(a.n), kBlock, 0, st>>>(a);
-  else k_appearance_fwd<GS_APP_NEURAL><<<grid_for(a.n), kBlock, 0, st>>>(a);
+  const int chunks = grid_for(a.n);
+  if (app == kAppNeuralHalf) {
+    const int wave = resident_blocks<k_appearance_fwd<kAppNeuralHalf>>(0, 1 << 20);
+    k_appearance_fwd<kAppNeuralHalf><<<chunks < wave ? chunks : wave, kBlock, 0, st>>>(a);
+  } else {
+    const int wave = resident_blocks<k_appearance_fwd<GS_APP_NEURAL>>(0, 1 << 20);
+    k_appearance_fwd<GS_APP_NEURAL><<<chunks < wave ? chunks : wave, kBlock, 0, st>>>(a);
+  }
   return 1;
 }
 
