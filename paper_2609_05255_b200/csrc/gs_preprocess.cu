@@ -367,6 +367,12 @@ __device__ __forceinline__ void quat_rot(float r, float x, float y, float z, flo
   R[6] = 2.f * (x * z - r * y); R[7] = 2.f * (y * z + r * x); R[8] = 1.f - 2.f * (x * x + y * y);
 }
 
+__device__ __forceinline__ float sqrt_approx(float x) {
+  float y;
+  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 // det(N N^T + 0.3 I) without the cancellation of a*c - b*b for elongated splats: by Lagrange's
 // identity |N0|^2 |N1|^2 - (N0.N1)^2 = |N0 x N1|^2, so det = |N0 x N1|^2 + 0.3 (|N0|^2 + |N1|^2) + 0.09.
 __device__ __forceinline__ float cov_det(const float N[6], float a, float c) {
@@ -389,21 +395,24 @@ __device__ __forceinline__ Geo project(const float mu[3], const float ls[3], con
   // the depth key: one fp32 FMA chain, identical bits on any IEEE machine
   const float z32 = __fmaf_rn(cam.R[8], mu[2], __fmaf_rn(cam.R[7], mu[1], __fmaf_rn(cam.R[6], mu[0], cam.t[2])));
   if (!(z32 >= cam.near_plane) || !(z32 <= cam.far_plane)) return g;
-  const float o = 1.f / (1.f + expf(-logit));
+  // The values that leave this function are compared with the oracle's within 1e-5-ish relative bounds; the
+  // integers of the tile stage are derived from the STORED values by operations that are rounded correctly
+  // (tile_rect, TileSpans).  So here the fast forms of division, square root and exponential do (a few ulp).
+  const float o = 1.f / (1.f + expf(-logit));   // accurate: tau = 2 ln(255 o) magnifies its error where o is near 1/255
   if (o < kAlphaMin) return g;
   const float qn2 = q[0] * q[0] + q[1] * q[1] + q[2] * q[2] + q[3] * q[3];
   if (!(qn2 > 0.f)) return g;
   const float qi = rsqrtf(qn2);
   float R[9];
   quat_rot(q[0] * qi, q[1] * qi, q[2] * qi, q[3] * qi, R);
-  const float s0 = expf(ls[0]), s1 = expf(ls[1]), s2 = expf(ls[2]);
+  const float s0 = __expf(ls[0]), s1 = __expf(ls[1]), s2 = __expf(ls[2]);
   float M[9];
 #pragma unroll
   for (int r = 0; r < 3; ++r) { M[3 * r] = R[3 * r] * s0; M[3 * r + 1] = R[3 * r + 1] * s1; M[3 * r + 2] = R[3 * r + 2] * s2; }
   const float tx = cam.R[0] * mu[0] + cam.R[1] * mu[1] + cam.R[2] * mu[2] + cam.t[0];
   const float ty = cam.R[3] * mu[0] + cam.R[4] * mu[1] + cam.R[5] * mu[2] + cam.t[1];
   const float tz = cam.R[6] * mu[0] + cam.R[7] * mu[1] + cam.R[8] * mu[2] + cam.t[2];
-  const float iz = 1.f / tz;
+  const float iz = __fdividef(1.f, tz);
   const float rx = tx * iz, ry = ty * iz;
   const float txc = tz * fminf(cam.limx, fmaxf(-cam.limx, rx));
   const float tyc = tz * fminf(cam.limy, fmaxf(-cam.limy, ry));
@@ -426,18 +435,16 @@ __device__ __forceinline__ Geo project(const float mu[3], const float ls[3], con
   const float c = N[3] * N[3] + N[4] * N[4] + N[5] * N[5] + kDilation;
   const float det = cov_det(N, a, c);
   if (!(det > 0.f) || !finite_f(det)) return g;
-  const float idet = 1.f / det;
   const float tau = footprint_tau(o);
-  const float ex = __fmul_rn(sqrtf(tau * a), kExtentPad), ey = __fmul_rn(sqrtf(tau * c), kExtentPad);
+  const float ex = __fmul_rn(sqrt_approx(tau * a), kExtentPad), ey = __fmul_rn(sqrt_approx(tau * c), kExtentPad);
   const float u = fmaf(cam.fx, rx, cam.cx), v = fmaf(cam.fy, ry, cam.cy);
   if (!finite_f(u) || !finite_f(v) || !finite_f(ex) || !finite_f(ey)) return g;
   g.valid = true;
   g.zbits = __float_as_uint(z32);
   // Cholesky factor of the conic Q = cov^-1 = L L^T, straight from the covariance entries (no
   // cancellation even for needle-like splats): l22 = 1/sqrt(c), l11 = sqrt(c/det), l21 = -b/sqrt(c det)
-  const float isd = 1.f / sqrtf(det), l22 = 1.f / sqrtf(c);
-  (void)idet;
-  g.u = u; g.v = v; g.A = sqrtf(c) * isd; g.B = -b * l22 * isd; g.C = l22; g.o = o; g.ex = ex; g.ey = ey; g.tau = tau;
+  const float isd = rsqrtf(det), l22 = rsqrtf(c);
+  g.u = u; g.v = v; g.A = c * l22 * isd; g.B = -b * l22 * isd; g.C = l22; g.o = o; g.ex = ex; g.ey = ey; g.tau = tau;
   const float vx = mu[0] - cam.oc[0], vy = mu[1] - cam.oc[1], vz = mu[2] - cam.oc[2];
   const float vi = rsqrtf(vx * vx + vy * vy + vz * vz);
   g.dirx = vx * vi; g.diry = vy * vi; g.dirz = vz * vi;
@@ -592,12 +599,12 @@ __device__ __forceinline__ GeoGrads project_backward(const float mu[3], const fl
                                                      float logit, const CamDev &cam, float gA, float gB,
                                                      float gC, float gu, float gv, float go, const float gd[3]) {
   GeoGrads out;
-  const float qn = sqrtf(q[0] * q[0] + q[1] * q[1] + q[2] * q[2] + q[3] * q[3]);
-  const float qi = 1.f / qn;
+  // the same fast forms as the forward: gradients are held to 1e-3, these are good to a few ulp
+  const float qi = rsqrtf(q[0] * q[0] + q[1] * q[1] + q[2] * q[2] + q[3] * q[3]);
   const float r = q[0] * qi, x = q[1] * qi, y = q[2] * qi, z = q[3] * qi;
   float R[9];
   quat_rot(r, x, y, z, R);
-  const float s[3] = {expf(ls[0]), expf(ls[1]), expf(ls[2])};
+  const float s[3] = {__expf(ls[0]), __expf(ls[1]), __expf(ls[2])};
   float M[9];
 #pragma unroll
   for (int i = 0; i < 3; ++i)
@@ -606,7 +613,7 @@ __device__ __forceinline__ GeoGrads project_backward(const float mu[3], const fl
   const float tx = cam.R[0] * mu[0] + cam.R[1] * mu[1] + cam.R[2] * mu[2] + cam.t[0];
   const float ty = cam.R[3] * mu[0] + cam.R[4] * mu[1] + cam.R[5] * mu[2] + cam.t[1];
   const float tz = cam.R[6] * mu[0] + cam.R[7] * mu[1] + cam.R[8] * mu[2] + cam.t[2];
-  const float iz = 1.f / tz, iz2 = iz * iz;
+  const float iz = __fdividef(1.f, tz), iz2 = iz * iz;
   const float rx = tx * iz, ry = ty * iz;
   const bool clx = rx < -cam.limx || rx > cam.limx, cly = ry < -cam.limy || ry > cam.limy;
   const float txc = tz * fminf(cam.limx, fmaxf(-cam.limx, rx));
@@ -627,7 +634,7 @@ __device__ __forceinline__ GeoGrads project_backward(const float mu[3], const fl
   const float a = N[0] * N[0] + N[1] * N[1] + N[2] * N[2] + kDilation;
   const float b = N[0] * N[3] + N[1] * N[4] + N[2] * N[5];
   const float c = N[3] * N[3] + N[4] * N[4] + N[5] * N[5] + kDilation;
-  const float idet = 1.f / cov_det(N, a, c);
+  const float idet = __fdividef(1.f, cov_det(N, a, c));
   const float A = c * idet, B = -b * idet, C = a * idet;
   // conic -> covariance: G_cov = -Q G_Q Q, G_Q = [[gA, gB/2], [gB/2, gC]]
   const float h = 0.5f * gB;
@@ -685,7 +692,7 @@ __device__ __forceinline__ GeoGrads project_backward(const float mu[3], const fl
   const float qd = r * gq[0] + x * gq[1] + y * gq[2] + z * gq[3];
   out.q[0] = (gq[0] - r * qd) * qi; out.q[1] = (gq[1] - x * qd) * qi;
   out.q[2] = (gq[2] - y * qd) * qi; out.q[3] = (gq[3] - z * qd) * qi;
-  const float o = 1.f / (1.f + expf(-logit));
+  const float o = __fdividef(1.f, 1.f + __expf(-logit));
   out.logit = go * o * (1.f - o);
   return out;
 }
