@@ -145,6 +145,13 @@ typedef struct {
   float *extent;         /* [n,4]  optional (may be NULL): (ex, ey, tau, 0): half-size in pixels of the
                                    box that bounds alpha >= 1/255 and tau = 2 ln(255 opacity);
                                    ex = ey = -1 if culled before the box test                  */
+  /* The same footprint by cells of 4 x 4 tiles (64 x 64 pixels), for the binning of gs_render_forward: one
+   * record per cell the footprint reaches, (cell id << 16) | 16-bit mask of the tiles it meets inside the
+   * cell (bit 4 (ty % 4) + tx % 4; cell id = (ty / 4) * ceil(tiles_x / 4) + tx / 4), cells in row-major
+   * order.  Opaque to the caller: allocate and pass on. */
+  uint32_t *cell_count;    /* [n]    number of records; bit 31 set: more cells than 3 x 3, records not stored
+                                     (gs_render_forward derives them again); 0 if the Gaussian touches no tile */
+  uint32_t *cell_records;  /* [n,9]  the records of a Gaussian whose rectangle spans at most 3 x 3 cells      */
 } GsProjected;
 
 /* Tile binning produced by gs_render_forward (caller-allocated device buffers). */

@@ -47,7 +47,7 @@ class GsScene(C.Structure):
 
 class GsProjected(C.Structure):
     _fields_ = [("mean2d", _vp), ("conic_opacity", _vp), ("color", _vp), ("depth_key", _vp), ("rect", _vp),
-                ("tiles_touched", _vp), ("extent", _vp)]
+                ("tiles_touched", _vp), ("extent", _vp), ("cell_count", _vp), ("cell_records", _vp)]
 
 
 class GsBinning(C.Structure):
@@ -212,12 +212,15 @@ class Projected:
     rect: torch.Tensor         # int16 storage holding uint16 tile coordinates, [n,4]
     tiles_touched: torch.Tensor
     extent: Optional[torch.Tensor]
+    cell_count: torch.Tensor = None      # [n]   footprint by cells of 4 x 4 tiles: opaque, for gs_render_forward
+    cell_records: torch.Tensor = None    # [n,9]
 
     def c_struct(self) -> GsProjected:
         p = GsProjected()
         p.mean2d, p.conic_opacity, p.color = _ptr(self.mean2d), _ptr(self.conic_opacity), _ptr(self.color)
         p.depth_key, p.rect, p.extent = _ptr(self.depth_key), _ptr(self.rect), _ptr(self.extent)
         p.tiles_touched = _ptr(self.tiles_touched)
+        p.cell_count, p.cell_records = _ptr(self.cell_count), _ptr(self.cell_records)
         return p
 
 
@@ -228,7 +231,9 @@ def alloc_projected(n: int, device, with_extent: bool = True) -> Projected:
                      torch.empty((m,), device=device, dtype=torch.int32),
                      torch.empty((m, 4), device=device, dtype=torch.int16),
                      torch.empty((m,), device=device, dtype=torch.int32),
-                     torch.empty((m, 4), **f) if with_extent else None)
+                     torch.empty((m, 4), **f) if with_extent else None,
+                     torch.empty((m,), device=device, dtype=torch.int32),
+                     torch.empty((m, 9), device=device, dtype=torch.int32))
 
 
 @dataclass

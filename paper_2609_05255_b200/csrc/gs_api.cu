@@ -82,7 +82,7 @@ bool camera_ok(const GsCamera *c) {
   if (!c || c->width <= 0 || c->height <= 0) return false;
   if (!(c->fx > 0.f) || !(c->fy > 0.f)) return false;
   const int64_t gx = (c->width + GS_TILE - 1) / GS_TILE, gy = (c->height + GS_TILE - 1) / GS_TILE;
-  if (gx > 65535 || gy > 65535 || gx * gy > ((int64_t)1 << 24)) return false;   // rect is u16; tile ids and grids stay small
+  if (gx > 65535 || gy > 65535 || ((gx + 3) / 4) * ((gy + 3) / 4) > 65536) return false;   // rect is u16; a cell id takes 16 bits
   return true;
 }
 
@@ -90,6 +90,7 @@ CamDev make_cam(const GsCamera *c) {
   CamDev d;
   d.W = c->width; d.H = c->height;
   d.gx = (c->width + GS_TILE - 1) / GS_TILE; d.gy = (c->height + GS_TILE - 1) / GS_TILE;
+  d.cgx = (d.gx + 3) / 4; d.cgy = (d.gy + 3) / 4;
   d.fx = c->fx; d.fy = c->fy; d.cx = c->cx; d.cy = c->cy;
   for (int r = 0; r < 3; ++r) {
     for (int k = 0; k < 3; ++k) d.R[3 * r + k] = c->w2c[4 * r + k];
@@ -186,24 +187,38 @@ struct Carver {
 
 struct FwdWorkspace {
   uint32_t *sorted_depth, *tmp_keys, *tmp_vals;          // [n]
-  uint32_t *block_offsets;                               // scan of tiles touched
-  uint32_t *inst_tiles, *inst_vals, *tmp_tiles, *tmp_ivals;  // [pair_capacity]
+  uint32_t *block_sums;                                  // cell records per 256 depth-sorted Gaussians
+  uint32_t *rec_keys, *rec_vals, *tmp_rkeys, *tmp_rvals; // [pair_capacity]: cell records (never more than instances, save for
+                                                         // slivers that reach a cell's rows but none of its tiles)
+  uint32_t *cell_ranges;                                 // [cells, 2]
+  CellScratch cells;
+  unsigned long long *rec_total;                         // number of records, written by the emission
   void *sort_table;
   size_t bytes;
 };
 
-FwdWorkspace carve_fwd(void *ws, int64_t n, int64_t cap) {
+FwdWorkspace carve_fwd(void *ws, int64_t n, int64_t cap, int width, int height) {
   Carver c{static_cast<char *>(ws), 0};
   FwdWorkspace w;
   const size_t nn = (size_t)(n > 0 ? n : 1), cc = (size_t)(cap > 0 ? cap : 1);
+  const int gx = (width + GS_TILE - 1) / GS_TILE, gy = (height + GS_TILE - 1) / GS_TILE;
+  const int cells = ((gx + 3) / 4) * ((gy + 3) / 4);
+  const size_t chunks = (size_t)max_chunks((int64_t)cc, cells);
   w.sorted_depth = c.take<uint32_t>(nn);
   w.tmp_keys = c.take<uint32_t>(nn);
   w.tmp_vals = c.take<uint32_t>(nn);
-  w.block_offsets = reinterpret_cast<uint32_t *>(c.take<char>(scan_scratch_bytes((int64_t)nn)));
-  w.inst_tiles = c.take<uint32_t>(cc);
-  w.inst_vals = c.take<uint32_t>(cc);
-  w.tmp_tiles = c.take<uint32_t>(cc);
-  w.tmp_ivals = c.take<uint32_t>(cc);
+  w.block_sums = reinterpret_cast<uint32_t *>(c.take<char>(scan_scratch_bytes((int64_t)nn)));
+  w.rec_keys = c.take<uint32_t>(cc);
+  w.rec_vals = c.take<uint32_t>(cc);
+  w.tmp_rkeys = c.take<uint32_t>(cc);
+  w.tmp_rvals = c.take<uint32_t>(cc);
+  w.cell_ranges = c.take<uint32_t>((size_t)cells * 2);
+  w.cells.chunk_first = c.take<uint32_t>((size_t)cells + 1);
+  w.cells.chunk_counts = c.take<uint32_t>(chunks * 16);
+  w.cells.chunk_bases = c.take<uint32_t>(chunks * 16);
+  w.cells.tile_counts = c.take<uint32_t>((size_t)gx * gy);
+  w.cells.tile_starts = c.take<uint32_t>((size_t)gx * gy);
+  w.rec_total = c.take<unsigned long long>(1);
   w.sort_table = c.take<char>(sort_scratch_bytes((int64_t)(nn > cc ? nn : cc)));
   w.bytes = c.used;
   return w;
@@ -225,9 +240,9 @@ BwdWorkspace carve_bwd(void *ws, int64_t n) {
 }
 size_t bwd_bytes(int64_t n) { return carve_bwd(nullptr, n).bytes; }
 
-int tile_bits(int num_tiles) {
+int id_bits(int count) {
   int bits = 1;
-  while ((1 << bits) < num_tiles) ++bits;
+  while ((1 << bits) < count) ++bits;
   return bits;
 }
 
@@ -275,7 +290,7 @@ const char *gs_last_error(const GsContext *ctx) { return ctx ? ctx->error : "no 
 
 size_t gs_workspace_bytes(int64_t n, int32_t width, int32_t height, int64_t pair_capacity) {
   if (n < 0 || width <= 0 || height <= 0 || pair_capacity < 0) return 0;
-  const size_t f = carve_fwd(nullptr, n, pair_capacity).bytes, b = bwd_bytes(n);
+  const size_t f = carve_fwd(nullptr, n, pair_capacity, width, height).bytes, b = bwd_bytes(n);
   return f > b ? f : b;
 }
 
@@ -284,7 +299,7 @@ GsStatus preprocess_impl(GsContext *ctx, const GsScene *scene, const GsCamera *c
                          int64_t *num_pairs_host, void *stream) {
   GsStatus st = scene_ok(ctx, scene);
   if (st != GS_OK) return st;
-  if (!camera_ok(cam)) return fail(ctx, GS_ERR_INVALID_ARG, "bad camera (size, focal length, more than 65535 tiles per axis or more than 2^24 tiles)");
+  if (!camera_ok(cam)) return fail(ctx, GS_ERR_INVALID_ARG, "bad camera (size, focal length, or more than 65536 cells of 64 x 64 pixels, e.g. beyond 16384 x 16384)");
   if (!out) return fail(ctx, GS_ERR_INVALID_ARG, "out is NULL");
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   cudaSetDevice(ctx->device);
@@ -292,7 +307,8 @@ GsStatus preprocess_impl(GsContext *ctx, const GsScene *scene, const GsCamera *c
   if ((st = check_cuda(ctx, cudaMemsetAsync(ctx->d_counter, 0, sizeof(unsigned long long), s), "memset")) != GS_OK) return st;
   if (scene->n == 0) return GS_OK;
   if (bad_ptr(out->mean2d) || bad_ptr(out->conic_opacity) || bad_ptr(out->color) || bad_ptr(out->depth_key) ||
-      bad_ptr(out->rect) || bad_ptr(out->tiles_touched) || (out->extent && !aligned16(out->extent)))
+      bad_ptr(out->rect) || bad_ptr(out->tiles_touched) || bad_ptr(out->cell_count) || bad_ptr(out->cell_records) ||
+      (out->extent && !aligned16(out->extent)))
     return fail(ctx, GS_ERR_INVALID_ARG, "a GsProjected buffer is NULL or misaligned");
   PreprocessArgs a;
   a.n = scene->n;
@@ -303,6 +319,7 @@ GsStatus preprocess_impl(GsContext *ctx, const GsScene *scene, const GsCamera *c
   a.deg = scene->active_degree; a.act = scene->color_activation;
   a.mean2d = out->mean2d; a.conic_opacity = out->conic_opacity; a.color = out->color; a.extent = out->extent;
   a.depth_key = out->depth_key; a.rect = out->rect; a.tiles_touched = out->tiles_touched;
+  a.cell_count = out->cell_count; a.cell_records = out->cell_records;
   a.pair_counter = ctx->d_counter;
   {
     StageTimer t(ctx, GS_STAGE_PREPROCESS_FWD, s);
@@ -380,33 +397,50 @@ GsStatus gs_render_forward(GsContext *ctx, int64_t n, const GsProjected *proj, c
   cudaSetDevice(ctx->device);
   const CamDev cd = make_cam(cam);
   const int num_tiles = cd.gx * cd.gy;
-  const FwdWorkspace w = carve_fwd(workspace, n, pair_capacity);
+  const FwdWorkspace w = carve_fwd(workspace, n, pair_capacity, cam->width, cam->height);
   const bool sorted = n > 0 && num_pairs > 0;
   if (sorted) {
-    // stage 1: Gaussians by depth key (stable => ties keep the index order); the last pass also leaves the tiles
-    // touched per 256 sorted Gaussians, from which the instance emission takes its offsets
+    uint32_t *overflow = reinterpret_cast<uint32_t *>(ctx->d_counter + 2);
+    // stage 1: Gaussians by depth key (stable => ties keep the index order); the last pass also leaves the cell records
+    // per 256 sorted Gaussians, from which their emission takes its offsets
     {
       StageTimer t(ctx, GS_STAGE_DEPTH_SORT, s);
-      const SortEpilogue ep = {proj->tiles_touched, w.block_offsets, num_scan_blocks(n), nullptr, 0, nullptr};
+      const SortEpilogue ep = {proj->cell_count, ~kCellBig, w.block_sums, num_scan_blocks(n), nullptr, 0, 0, nullptr};
       t.done(launch_radix_sort(proj->depth_key, nullptr, w.sorted_depth, bin->depth_order, w.tmp_keys, w.tmp_vals,
-                               n, nullptr, 32, w.sort_table, &ep, s));
+                               n, nullptr, 0, 32, 8, w.sort_table, &ep, s));
     }
-    // stage 2: instances in depth order, then a stable sort by tile id alone, whose last pass finds the tile ranges
+    // stage 2: one record per (Gaussian, cell of 4 x 4 tiles) in depth order, then a stable sort by cell id alone,
+    // whose last pass finds where every cell's records begin and end
     {
       StageTimer t(ctx, GS_STAGE_KEYGEN, s);
-      t.done(launch_keygen(bin->depth_order, proj->rect, proj->mean2d, proj->conic_opacity, proj->tiles_touched,
-                           w.block_offsets, w.inst_tiles, w.inst_vals, n, cd.gx, cd.W, cd.H, pair_capacity, s));
+      t.done(launch_emit_records(bin->depth_order, proj->cell_count, proj->cell_records, proj->rect, proj->mean2d,
+                                 proj->conic_opacity, w.block_sums, w.rec_keys, w.rec_vals, w.rec_total, overflow, n, cd.cgx,
+                                 cd.W, cd.H, pair_capacity, s));
     }
+    const int num_cells = cd.cgx * cd.cgy;
+    // two buffers serve the passes: an odd number of passes ends in the other one, an even number back in the first
+    const int cell_bits = id_bits(num_cells);
+    constexpr int kCellDigit = 9;   // up to 512 cells (2048 x 1024 pixels) sort in one pass
+    const bool odd = (radix_passes(cell_bits, kCellDigit) & 1) != 0;
+    uint32_t *sorted_rkeys = odd ? w.tmp_rkeys : w.rec_keys, *sorted_rvals = odd ? w.tmp_rvals : w.rec_vals;
     {
       StageTimer t(ctx, GS_STAGE_TILE_SORT, s);
-      const SortEpilogue ep = {nullptr, nullptr, 0, bin->tile_ranges, num_tiles, reinterpret_cast<uint32_t *>(ctx->d_counter + 2)};
-      t.done(launch_radix_sort(w.inst_tiles, w.inst_vals, bin->sorted_tiles, bin->sorted_vals, w.tmp_tiles,
-                               w.tmp_ivals, num_pairs, count_dev, tile_bits(num_tiles), w.sort_table, &ep, s));
+      const SortEpilogue ep = {nullptr, 0u, nullptr, 0, w.cell_ranges, num_cells, 16, nullptr};
+      // the count lives on the device; its host-side bound: a record holds at least one instance
+      t.done(launch_radix_sort(w.rec_keys, w.rec_vals, sorted_rkeys, sorted_rvals, odd ? w.rec_keys : w.tmp_rkeys,
+                               odd ? w.rec_vals : w.tmp_rvals, num_pairs, w.rec_total, 16, cell_bits, kCellDigit, w.sort_table, &ep, s));
     }
-  }
-  {
+    // stage 3: the records of every cell, still in depth order, expanded into the lists of its 16 tiles
+    {
+      StageTimer t(ctx, GS_STAGE_TILE_RANGES, s);
+      if (on_device)   // more instances than the capacity: the lists are cut off, the host is told
+        launch_flag_if_greater(count_dev, (unsigned long long)pair_capacity, overflow, s);
+      t.done(launch_expand(sorted_rkeys, sorted_rvals, w.cell_ranges, w.cells, num_pairs, pair_capacity, cd.gx, cd.gy, cd.cgx,
+                           cd.cgy, bin->sorted_tiles, bin->sorted_vals, bin->tile_ranges, bin->tile_order, s));
+    }
+  } else {
     StageTimer t(ctx, GS_STAGE_TILE_RANGES, s);
-    t.done(launch_tile_order(bin->tile_ranges, bin->tile_order, num_tiles, !sorted, s));
+    t.done(launch_empty_binning(bin->tile_ranges, bin->tile_order, num_tiles, s));
   }
   {
     StageTimer t(ctx, GS_STAGE_BLEND_FWD, s);

@@ -18,8 +18,14 @@ constexpr float kLog2e = 1.4426950408889634f;
 constexpr int kMlpW1 = 0, kMlpW2 = 512, kMlpW3 = 768;
 
 // Camera as the kernels see it (passed by value).
+// Cells: 4 x 4 tiles.  The binning sorts one record per (Gaussian, cell) instead of one per (Gaussian, tile).
+constexpr int kCellSlots = 9;                 // records kept per Gaussian by the preprocess (3 x 3 cells)
+constexpr uint32_t kCellBig = 0x80000000u;    // flag in cell_count: records not stored, derive them again
+constexpr int kCellChunk = 2048;              // records of one cell that one CTA expands
+
 struct CamDev {
   int W, H, gx, gy;
+  int cgx, cgy;         // cells per row / column: ceil(gx / 4), ceil(gy / 4)
   float fx, fy, cx, cy;
   float R[9], t[3];
   float oc[3];          // camera centre in world space
@@ -44,7 +50,7 @@ struct PreprocessArgs {
   const __half *features, *weights;
   int deg, act;
   float *mean2d, *conic_opacity, *color, *extent;
-  uint32_t *depth_key, *tiles_touched;
+  uint32_t *depth_key, *tiles_touched, *cell_count, *cell_records;
   uint16_t *rect;
   unsigned long long *pair_counter;
 };
@@ -97,30 +103,44 @@ constexpr int kWgradBlocks = 592;   // persistent blocks of the decoder-gradient
 // Sorting / binning.
 // What the scatter of the last pass of a sort adds on its way out (nothing where the pointers are null).
 struct SortEpilogue {
-  // depth sort: sums of tiles touched per 256 consecutive Gaussians of the sorted order (the instance emission turns
-  // them into its offsets); cleared by the same pass
-  const uint32_t *tiles_touched;
+  // depth sort: sums of a per-Gaussian count (counts[id] & count_mask) per 256 consecutive Gaussians of the sorted
+  // order, from which the record emission takes its offsets; cleared by the same pass
+  const uint32_t *counts;
+  uint32_t count_mask;
   uint32_t *block_sums;
   int num_block_sums;
-  // tile sort: [start, end) of every tile in the sorted instance list (an empty tile is left at (0xffffffff, 0) for
-  // launch_tile_order to settle), and the flag raised when a device-side instance count exceeded the capacity
+  // record sort: [start, end) of every id = key >> key_shift in the sorted list (an id that does not occur is left at
+  // (0xffffffff, 0)), and the flag raised when the device-side count exceeded the capacity
   uint32_t *ranges;
-  int num_tiles;
+  int num_ranges;
+  int key_shift;
   uint32_t *overflow;
 };
 size_t sort_scratch_bytes(int64_t count);
-// LSD radix sort of (key, val) pairs on bits [0, num_bits).  If vals_in == nullptr the values are
-// the element indices.  Result lands in keys_out / vals_out; tmp_* are same-sized alternates.
+// LSD radix sort of (key, val) pairs on bits [first_bit, first_bit + num_bits), in digits of at most max_digit_bits
+// (4 .. 11; wide digits save passes but take registers and shared memory: they pay for short keys only).  If vals_in == nullptr the values are
+// the element indices.  Result lands in keys_out / vals_out; tmp_* are same-sized alternates.  `count` bounds the
+// number of elements (and sizes the grid); with count_dev the true number is read on the device.
 int launch_radix_sort(const uint32_t *keys_in, const uint32_t *vals_in, uint32_t *keys_out,
                        uint32_t *vals_out, uint32_t *tmp_keys, uint32_t *tmp_vals, int64_t count,
-                       const unsigned long long *count_dev, int num_bits, void *scratch, const SortEpilogue *epilogue,
-                       cudaStream_t st);
+                       const unsigned long long *count_dev, int first_bit, int num_bits, int max_digit_bits, void *scratch,
+                       const SortEpilogue *epilogue, cudaStream_t st);
+int radix_passes(int num_bits, int max_digit_bits);   // passes launch_radix_sort makes over num_bits key bits
 size_t scan_scratch_bytes(int64_t n);
-int num_scan_blocks(int64_t n);   // entries of the block sums that launch_keygen reads
-int launch_keygen(const uint32_t *depth_order, const uint16_t *rect, const float *mean2d, const float *conic_opacity,
-                  const uint32_t *tiles_touched, const uint32_t *block_sums, uint32_t *inst_tiles, uint32_t *inst_vals,
-                  int64_t n, int gx, int W, int H, int64_t capacity, cudaStream_t st);
-int launch_tile_order(uint32_t *ranges, uint32_t *order, int num_tiles, bool clear, cudaStream_t st);
+int num_scan_blocks(int64_t n);   // entries of the block sums that launch_emit_records reads
+int launch_emit_records(const uint32_t *depth_order, const uint32_t *cell_count, const uint32_t *cell_records,
+                        const uint16_t *rect, const float *mean2d, const float *conic_opacity, const uint32_t *block_sums,
+                        uint32_t *rec_keys, uint32_t *rec_vals, unsigned long long *rec_total, uint32_t *overflow, int64_t n,
+                        int cgx, int W, int H, int64_t capacity, cudaStream_t st);
+// Scratch of the expansion: chunk_first [cells + 1], chunk_counts and chunk_bases [max_chunks, 16], tile_counts and
+// tile_starts [tiles].
+struct CellScratch { uint32_t *chunk_first, *chunk_counts, *chunk_bases, *tile_counts, *tile_starts; };
+int max_chunks(int64_t record_capacity, int num_cells);
+int launch_expand(const uint32_t *rec_keys, const uint32_t *rec_vals, const uint32_t *cell_ranges, const CellScratch &cs,
+                  int64_t record_capacity, int64_t pair_capacity, int gx, int gy, int cgx, int cgy, uint32_t *sorted_tiles,
+                  uint32_t *sorted_vals, uint32_t *tile_ranges, uint32_t *tile_order, cudaStream_t st);
+int launch_empty_binning(uint32_t *tile_ranges, uint32_t *tile_order, int num_tiles, cudaStream_t st);
+void launch_flag_if_greater(const unsigned long long *value, unsigned long long bound, uint32_t *flag, cudaStream_t st);
 
 // Blend.
 int launch_blend_fwd(const CamDev &cam, const uint32_t *ranges, const uint32_t *order, const uint32_t *vals,

@@ -469,8 +469,19 @@ __device__ __forceinline__ void load3(const float *p, int64_t i, float v[3]) {
   v[0] = __ldg(p + 3 * i); v[1] = __ldg(p + 3 * i + 1); v[2] = __ldg(p + 3 * i + 2);
 }
 
+// Per-warp shared memory of the cooperative tile-row evaluation: span parameters, rectangle and cell masks of the 32
+// owners, and the list of (owner << 8 | row) pairs.
+struct RowStage {
+  float par[32][8];
+  int4 geo[32];
+  uint32_t mask[32][9];
+  uint32_t tiles[32];
+  unsigned short list[32 * 12];
+};
+
 template <int APP>
 __global__ void __launch_bounds__(kBlock) k_preprocess_fwd(PreprocessArgs a, CamDev cam) {
+  __shared__ __align__(16) RowStage sRows[kWarps];
   __shared__ __align__(16) float sData[Explicit<APP>::value ? kWarps * SlabOf<APP>::value : 4];
   __shared__ __align__(16) unsigned char sNN[IsNeural<APP>::value ? kWarps * sizeof(StageFwd) : 16];
   StageFwd *sStage = reinterpret_cast<StageFwd *>(sNN);   // unused for SH
@@ -511,13 +522,88 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_fwd(PreprocessArgs a, Cam
     g = project(mu, ls, q, logit, cam);
     if (g.valid) vis = tile_rect(g.u, g.v, g.ex, g.ey, cam, rect);
   }
-  // tiles the ellipse really meets inside its bounding rectangle
-  unsigned int tiles = 0;
-  if (vis) {
+  // tiles the ellipse really meets inside its bounding rectangle, and the same by cells of 4 x 4 tiles: one
+  // record (cell id, mask of the tiles met) per cell, which is what the binning sorts.
+  unsigned int tiles = 0, nrec = 0;
+  bool stored = false;
+  {
     TileSpans sp;
-    sp.setup(g.u, g.v, g.A, g.B, g.C, g.tau, cam.W, cam.H);
-    tiles = sp.count(rect[0], rect[1], rect[2], rect[3]);
-    if (tiles == 0) { vis = false; rect[0] = rect[1] = rect[2] = rect[3] = 0; }
+    if (vis) sp.setup(g.u, g.v, g.A, g.B, g.C, g.tau, cam.W, cam.H);
+    const int cx0 = rect[0] >> 2, cx1 = (rect[2] - 1) >> 2, cy0 = rect[1] >> 2, cy1 = (rect[3] - 1) >> 2;
+    stored = vis && cx1 - cx0 <= 2 && cy1 - cy0 <= 2;          // at most 3 x 3 cells: the records fit the Gaussian's slots
+    if (vis && !stored) {
+      // a large footprint is only counted here (the record emission works its cells out again): a row of cells
+      // contributes the cells from the leftmost to the rightmost tile met in its tile rows
+      for (int cy = cy0; cy <= cy1; ++cy) {
+        int lo = 1 << 30, hi = -1;
+        const int ta = max(rect[1], 4 * cy), tb = min(rect[3], 4 * cy + 4);
+        for (int ty = ta; ty < tb; ++ty) {
+          int xa, xb;
+          if (!sp.row(ty, rect[0], rect[2], xa, xb)) continue;
+          tiles += (unsigned)(xb - xa);
+          lo = min(lo, xa >> 2); hi = max(hi, (xb - 1) >> 2);
+        }
+        if (hi >= lo) nrec += (unsigned)(hi - lo + 1);
+      }
+    }
+    // The tile rows of the other footprints are evaluated by the warp together, one (Gaussian, tile row) per lane
+    // and round: lanes own very different numbers of rows (1 to 12), and a loop per lane would idle most of them.
+    // Each owner parks its span parameters and the list of its rows in shared memory; a row's tiles go into the
+    // owner's cell masks with shared-memory atomics (integer OR / add: any order gives the same bits).
+    RowStage &rs = sRows[warp];
+    const int rows = stored ? rect[3] - rect[1] : 0;
+    int incl = rows;
+#pragma unroll
+    for (int sft = 1; sft < 32; sft <<= 1) {
+      const int t = __shfl_up_sync(kFull, incl, sft);
+      if (lane >= sft) incl += t;
+    }
+    const int total = __shfl_sync(kFull, incl, 31);
+    if (stored) {
+      float *par = rs.par[lane];
+      par[0] = sp.u; par[1] = sp.v; par[2] = sp.ila; par[3] = sp.lb; par[4] = sp.lc; par[5] = sp.taup; par[6] = sp.dys; par[7] = sp.eyp;
+      rs.geo[lane] = make_int4(rect[0], rect[2], rect[1], cx0);
+#pragma unroll
+      for (int j = 0; j < 9; ++j) rs.mask[lane][j] = 0u;
+      rs.tiles[lane] = 0u;
+      for (int k = 0; k < rows; ++k) rs.list[incl - rows + k] = (unsigned short)((lane << 8) | k);
+    }
+    __syncwarp();
+    for (int base = 0; base < total; base += 32) {
+      if (base + lane < total) {
+        const unsigned e = rs.list[base + lane];
+        const int o = (int)(e >> 8), k = (int)(e & 255u);
+        const float *par = rs.par[o];
+        TileSpans so;
+        so.u = par[0]; so.v = par[1]; so.ila = par[2]; so.lb = par[3]; so.lc = par[4]; so.taup = par[5]; so.dys = par[6]; so.eyp = par[7];
+        so.W = cam.W; so.H = cam.H;
+        const int4 ge = rs.geo[o];      // (tx0, tx1, ty0, first cell column)
+        const int ty = ge.z + k;
+        int xa, xb;
+        if (so.row(ty, ge.x, ge.y, xa, xb)) {
+          atomicAdd(&rs.tiles[o], (unsigned)(xb - xa));
+          // the row's tiles as bits counted from the first column of the first cell (at most 12), a nibble per cell
+          const uint32_t bits = ((1u << (xb - xa)) - 1u) << (xa - 4 * ge.w);
+          const int cyi = (ty >> 2) - (ge.z >> 2), sh = 4 * (ty & 3);
+#pragma unroll
+          for (int c = 0; c < 3; ++c) {
+            const uint32_t nib = (bits >> (4 * c)) & 15u;
+            if (nib) atomicOr(&rs.mask[o][3 * cyi + c], nib << sh);
+          }
+        }
+      }
+    }
+    __syncwarp();
+    if (stored) {
+      tiles = rs.tiles[lane];
+      uint32_t *slot = a.cell_records + (size_t)i * kCellSlots;
+#pragma unroll
+      for (int j = 0; j < 9; ++j) {
+        const uint32_t m = rs.mask[lane][j];
+        if (m) slot[nrec++] = ((uint32_t)((cy0 + j / 3) * cam.cgx + cx0 + j % 3) << 16) | m;
+      }
+    }
+    if (vis && tiles == 0) { vis = false; nrec = 0; rect[0] = rect[1] = rect[2] = rect[3] = 0; }
   }
   // ---- fused colour decode for the Gaussians that survived culling
   float pre[3] = {0.f, 0.f, 0.f};
@@ -575,6 +661,7 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_fwd(PreprocessArgs a, Cam
     }
     a.depth_key[i] = vis ? g.zbits : 0xffffffffu;
     a.tiles_touched[i] = tiles;
+    a.cell_count[i] = nrec | ((nrec && !stored) ? kCellBig : 0u);   // (vis was cleared if no tile is met: nrec = 0)
     reinterpret_cast<ushort4 *>(a.rect)[i] = make_ushort4((unsigned short)rect[0], (unsigned short)rect[1],
                                                           (unsigned short)rect[2], (unsigned short)rect[3]);
     if (a.extent) reinterpret_cast<float4 *>(a.extent)[i] = g.valid ? make_float4(g.ex, g.ey, g.tau, 0.f) : make_float4(-1.f, -1.f, 0.f, 0.f);

@@ -1,10 +1,14 @@
 // Ordering and binning: a stable LSD radix sort (digits of up to 8 bits, keys staged and ranked in shared
-// memory, no inter-block waiting), the prefix sum of tiles touched in depth order, instance
-// generation and per-tile ranges.
+// memory, no inter-block waiting) and the kernels that turn its output into per-tile lists.
 //
-// Two-stage ordering: (1) the Gaussians are sorted once by their 32-bit depth key (ties keep the
-// index order because the sort is stable); (2) instances are emitted in that order and sorted by
-// tile id only (ceil(log2(tiles)) bits).  The result is the order by (tile, depth key, index).
+// (1) The Gaussians are sorted once by their 32-bit depth key (ties keep the index order: the sort is stable).
+// (2) In that order every Gaussian emits one record per CELL of 4 x 4 tiles that its footprint reaches - the cell id
+//     and a 16-bit mask of the tiles met inside the cell, as the preprocess left them - and the records are sorted by
+//     cell id alone (a quarter of the elements and fewer bits than a sort of the (Gaussian, tile) instances).
+// (3) A cell's records, still in depth order, are expanded into the lists of its 16 tiles: counts per chunk of 2048
+//     records, one scan for the start of every tile and of every chunk inside it, then each chunk writes its
+//     instances, the lanes that share a tile finding their slots with one ballot.
+// The result is the instance list ordered by (tile, depth key, index), with its per-tile ranges.
 #include "gs_device.cuh"
 
 namespace gs {
@@ -16,64 +20,63 @@ constexpr int kItems = 16;
 constexpr int kSortTile = kSortThreads * kItems;   // 4096 elements per block iteration
 constexpr int kMaxSortBlocks = 444;                // 3 resident CTAs x 148 SMs: one full wave
 constexpr unsigned kFull = 0xffffffffu;
+constexpr int kMaxDigitBits = 11;  // widest radix digit: 2048 bins
 constexpr int kScanBlock = 256;   // Gaussians per block of the tiles-touched prefix sum and per CTA of the instance emission
 
-// Block b sorts tiles_per_block (+ 1 if b < extra) consecutive tiles of kSortTile elements: the tiles are dealt
-// out as evenly as whole tiles allow over one full wave of CTAs.
-struct SortPlan { int blocks; int tiles_per_block; int extra; };
-
-SortPlan plan_for(int64_t count) {
+// Block b sorts consecutive tiles of kSortTile elements: the tiles are dealt out as evenly as whole tiles allow over
+// the grid, which is one full wave of CTAs at most.  The grid is sized by the host's bound on the count; the ranges
+// follow the count the kernels see (which may live on the device), so the work stays balanced either way.
+int sort_blocks(int64_t count) {
   const int64_t tiles = (count + kSortTile - 1) / kSortTile;
-  SortPlan p;
-  p.blocks = (int)(tiles < kMaxSortBlocks ? tiles : kMaxSortBlocks);
-  if (p.blocks < 1) p.blocks = 1;
-  p.tiles_per_block = (int)(tiles / p.blocks);
-  p.extra = (int)(tiles - (int64_t)p.tiles_per_block * p.blocks);
-  return p;
+  return (int)(tiles < 1 ? 1 : tiles < kMaxSortBlocks ? tiles : kMaxSortBlocks);
 }
 
-// First tile and number of tiles of a block under the plan.
-__device__ __forceinline__ void block_tiles(int tiles_per_block, int extra, int64_t &first, int &num) {
-  const int b = (int)blockIdx.x;
+// First tile and number of tiles of this block.
+__device__ __forceinline__ void block_tiles(int64_t count, int64_t &first, int &num) {
+  const int64_t tiles = (count + kSortTile - 1) / kSortTile;
+  const int b = (int)blockIdx.x, nb = (int)gridDim.x;
+  const int tiles_per_block = (int)(tiles / nb), extra = (int)(tiles - (int64_t)tiles_per_block * nb);
   first = (int64_t)b * tiles_per_block + min(b, extra);
   num = tiles_per_block + (b < extra ? 1 : 0);
 }
 
-// Digit histogram of each block's contiguous range: table[block][digit].
+// Digit histogram of each block's contiguous range: table[digit][block] (digits of up to kMaxDigitBits bits).
 __global__ void __launch_bounds__(kSortThreads) k_radix_hist(const uint32_t *__restrict__ keys, int64_t count,
                                                              const unsigned long long *__restrict__ count_dev,
-                                                             int shift, uint32_t mask, int tiles_per_block, int extra,
+                                                             int shift, int bits,
                                                              uint32_t *__restrict__ table, SortEpilogue ep) {
   // the arrays the scatter of this pass accumulates into start from their neutral values
   if (ep.block_sums)
     for (int i = blockIdx.x * kSortThreads + threadIdx.x; i < ep.num_block_sums; i += gridDim.x * kSortThreads) ep.block_sums[i] = 0u;
   if (ep.ranges)
-    for (int i = blockIdx.x * kSortThreads + threadIdx.x; i < 2 * ep.num_tiles; i += gridDim.x * kSortThreads)
+    for (int i = blockIdx.x * kSortThreads + threadIdx.x; i < 2 * ep.num_ranges; i += gridDim.x * kSortThreads)
       ep.ranges[i] = (i & 1) ? 0u : 0xffffffffu;
   if (count_dev) {
     const int64_t c = (int64_t)__ldg(count_dev);                    // the true length lives on the device
     if (ep.overflow && c > count && blockIdx.x == 0 && threadIdx.x == 0) *ep.overflow = 1u;   // lists were cut off: tell the host
     count = min(count, c);
   }
-  __shared__ uint32_t s_hist[kSortWarps][256];
+  // up to 256 digits: one histogram per warp (fewer collisions); more: two shared by the warps
+  __shared__ uint32_t s_hist[2 << kMaxDigitBits];
   const int tid = threadIdx.x, warp = tid >> 5;
-  for (int k = tid; k < kSortWarps * 256; k += kSortThreads) (&s_hist[0][0])[k] = 0;
+  const int nb = 1 << bits, copies = nb <= 256 ? kSortWarps : 2;
+  const uint32_t mask = (uint32_t)nb - 1u;
+  for (int k = tid; k < copies * nb; k += kSortThreads) s_hist[k] = 0;
   __syncthreads();
   int64_t first_tile;
   int my_tiles;
-  block_tiles(tiles_per_block, extra, first_tile, my_tiles);
+  block_tiles(count, first_tile, my_tiles);
   const int64_t begin = first_tile * kSortTile;
   int64_t end = begin + (int64_t)my_tiles * kSortTile;
   if (end > count) end = count;
-  for (int64_t i = begin + tid; i < end; i += kSortThreads) {
-    const uint32_t d = (__ldg(keys + i) >> shift) & mask;
-    atomicAdd(&s_hist[warp][d], 1u);
-  }
+  uint32_t *mine = s_hist + (warp % copies) * nb;
+  for (int64_t i = begin + tid; i < end; i += kSortThreads) atomicAdd(mine + ((__ldg(keys + i) >> shift) & mask), 1u);
   __syncthreads();
-  uint32_t s = 0;
-#pragma unroll
-  for (int w = 0; w < kSortWarps; ++w) s += s_hist[w][tid];
-  table[(size_t)tid * gridDim.x + blockIdx.x] = s;   // digit-major: one contiguous row per digit
+  for (int d = tid; d < nb; d += kSortThreads) {
+    uint32_t t = 0;
+    for (int w = 0; w < copies; ++w) t += s_hist[w * nb + d];
+    table[(size_t)d * gridDim.x + blockIdx.x] = t;   // digit-major: one contiguous row per digit
+  }
 }
 
 // Per digit (one CTA each): exclusive scan of the row of per-block counts, in place, and the row
@@ -109,9 +112,15 @@ __global__ void __launch_bounds__(256) k_radix_scan_rows(uint32_t *__restrict__ 
   if (tid == 0) totals[blockIdx.x] = s_carry;
 }
 
-__device__ __forceinline__ uint32_t block_exclusive_scan_256(uint32_t v, uint32_t *s_warp_tot, int tid) {
+// Exclusive prefix sums over kSortThreads * DPT values in thread-major order (thread t holds values t * DPT ..): each
+// thread scans its own values, the thread totals are scanned across the block.
+template <int DPT>
+__device__ __forceinline__ void block_exclusive_scan(const uint32_t v[DPT], uint32_t out[DPT], uint32_t *s_warp_tot, int tid) {
   const int lane = tid & 31, warp = tid >> 5;
-  uint32_t inc = v;
+  uint32_t sum = 0;
+#pragma unroll
+  for (int j = 0; j < DPT; ++j) { out[j] = sum; sum += v[j]; }
+  uint32_t inc = sum;
 #pragma unroll
   for (int s = 1; s < 32; s <<= 1) {
     const uint32_t t = __shfl_up_sync(kFull, inc, s);
@@ -119,32 +128,37 @@ __device__ __forceinline__ uint32_t block_exclusive_scan_256(uint32_t v, uint32_
   }
   if (lane == 31) s_warp_tot[warp] = inc;
   __syncthreads();
-  uint32_t off = 0;
+  uint32_t off = inc - sum;
 #pragma unroll
   for (int w = 0; w < kSortWarps; ++w) off += (w < warp) ? s_warp_tot[w] : 0u;
   __syncthreads();
-  return off + inc - v;
+#pragma unroll
+  for (int j = 0; j < DPT; ++j) out[j] += off;
 }
 
-// One pass: stable scatter of this block's range by the BITS-wide digit at `shift`.  Slots past the
+template <int BITS> constexpr size_t scatter_smem_bytes() {
+  return sizeof(uint32_t) * (2 * kSortTile + (size_t)(kSortWarps + 2) * (BITS <= 8 ? 256 : (1 << BITS)) + kSortWarps);
+}
+
+// One pass: stable scatter of this block's range by the BITS-wide digit at `shift` (BITS up to kMaxDigitBits; the
+// digit arrays hold max(256, 2^BITS) entries, thread t looking after digits t * DPT ..).  Slots past the
 // end of the input carry the largest digit and sit at the end of the last tile, so they rank after
 // every real key and are never written.
-// EP selects the epilogue: 0 none, 1 block sums of tiles touched (last pass of the depth sort), 2 tile ranges (last
-// pass of the tile sort: inside a block's run of one digit the keys are non-decreasing, because the earlier passes
-// ordered the lower bits, so a change of key between neighbours of a run is a tile boundary; the two ends of a run
-// may continue in another block and enter with an atomic min / max).
+// EP selects the epilogue: 0 none, 1 block sums of a per-Gaussian count (last pass of the depth sort), 2 ranges of
+// equal ids = key >> key_shift (last pass of the record sort: inside a block's run of one digit the keys are
+// non-decreasing, because the earlier passes ordered the lower bits, so a change of id between neighbours of a run
+// is a boundary; the two ends of a run may continue in another block and enter with an atomic min / max).
 template <int BITS, int EP>
-__global__ void __launch_bounds__(kSortThreads, 3) k_radix_scatter(
+__global__ void __launch_bounds__(kSortThreads, BITS <= 9 ? 3 : 2) k_radix_scatter(
     const uint32_t *__restrict__ keys_in, const uint32_t *__restrict__ vals_in, uint32_t *__restrict__ keys_out,
     uint32_t *__restrict__ vals_out, int64_t count, const unsigned long long *__restrict__ count_dev, int shift,
-    int tiles_per_block, int extra,
     const uint32_t *__restrict__ table, const uint32_t *__restrict__ totals, int nblocks, SortEpilogue ep) {
-  __shared__ uint32_t s_keys[kSortTile];
-  __shared__ uint32_t s_vals[kSortTile];
-  __shared__ uint32_t s_warp_cnt[kSortWarps][256];
-  __shared__ uint32_t s_digit_start[256];
-  __shared__ uint32_t s_base[256];
-  __shared__ uint32_t s_warp_tot[kSortWarps];
+  constexpr int NB = BITS <= 8 ? 256 : (1 << BITS);   // entries of the digit arrays
+  constexpr int DPT = NB / kSortThreads;              // digits per thread
+  extern __shared__ __align__(16) uint32_t s_dyn[];
+  uint32_t *s_keys = s_dyn, *s_vals = s_keys + kSortTile;
+  uint32_t *s_warp_cnt = s_vals + kSortTile;          // [kSortWarps][NB]
+  uint32_t *s_digit_start = s_warp_cnt + kSortWarps * NB, *s_base = s_digit_start + NB, *s_warp_tot = s_base + NB;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t lt_mask = (1u << lane) - 1u;
   if (count_dev) count = min(count, (int64_t)__ldg(count_dev));
@@ -153,19 +167,26 @@ __global__ void __launch_bounds__(kSortThreads, 3) k_radix_scatter(
   // global base of every digit for this block: all smaller digits everywhere (scan of the row
   // totals) + the same digit in the blocks before this one (the row prefix from k_radix_scan_rows)
   {
-    const uint32_t start = block_exclusive_scan_256(__ldg(totals + tid), s_warp_tot, tid);
-    s_base[tid] = start + __ldg(table + (size_t)tid * nblocks + blockIdx.x);
+    uint32_t tot[DPT], start[DPT];
+#pragma unroll
+    for (int j = 0; j < DPT; ++j) { const int d = tid * DPT + j; tot[j] = d <= (int)kDigitMask ? __ldg(totals + d) : 0u; }
+    block_exclusive_scan<DPT>(tot, start, s_warp_tot, tid);
+#pragma unroll
+    for (int j = 0; j < DPT; ++j) {
+      const int d = tid * DPT + j;
+      s_base[d] = start[j] + (d <= (int)kDigitMask ? __ldg(table + (size_t)d * nblocks + blockIdx.x) : 0u);
+    }
   }
 
   int64_t first_tile;
   int my_tiles;
-  block_tiles(tiles_per_block, extra, first_tile, my_tiles);
+  block_tiles(count, first_tile, my_tiles);
   const int64_t begin = first_tile * kSortTile;
   for (int t = 0; t < my_tiles; ++t) {
     const int64_t tile_begin = begin + (int64_t)t * kSortTile;
     if (tile_begin >= count) break;
     const int valid_count = (int)min((int64_t)kSortTile, count - tile_begin);
-    for (int k = tid; k < kSortWarps * 256; k += kSortThreads) (&s_warp_cnt[0][0])[k] = 0;
+    for (int k = tid; k < kSortWarps * NB; k += kSortThreads) s_warp_cnt[k] = 0;
     __syncthreads();
     uint32_t key[kItems], val[kItems];
     unsigned short rank[kItems];
@@ -197,27 +218,34 @@ __global__ void __launch_bounds__(kSortThreads, 3) k_radix_scatter(
       }
       const int leader = __ffs(peers) - 1;
       uint32_t prior = 0;
-      if (lane == leader) prior = atomicAdd(&s_warp_cnt[warp][d], (uint32_t)__popc(peers));
+      if (lane == leader) prior = atomicAdd(&s_warp_cnt[warp * NB + d], (uint32_t)__popc(peers));
       prior = __shfl_sync(kFull, prior, leader);
       rank[it] = (unsigned short)(prior + __popc(peers & lt_mask));
     }
     __syncthreads();
     // per digit: exclusive scan over warps, then over digits
-    uint32_t cnt = 0;
+    uint32_t cnt[DPT], dstart[DPT];
 #pragma unroll
-    for (int w = 0; w < kSortWarps; ++w) {
-      const uint32_t c = s_warp_cnt[w][tid];
-      s_warp_cnt[w][tid] = cnt;
-      cnt += c;
+    for (int j = 0; j < DPT; ++j) {
+      const int d = tid * DPT + j;
+      uint32_t c = 0;
+#pragma unroll
+      for (int w = 0; w < kSortWarps; ++w) {
+        const uint32_t x = s_warp_cnt[w * NB + d];
+        s_warp_cnt[w * NB + d] = c;
+        c += x;
+      }
+      cnt[j] = c;
     }
-    const uint32_t dstart = block_exclusive_scan_256(cnt, s_warp_tot, tid);
-    s_digit_start[tid] = dstart;
+    block_exclusive_scan<DPT>(cnt, dstart, s_warp_tot, tid);
+#pragma unroll
+    for (int j = 0; j < DPT; ++j) s_digit_start[tid * DPT + j] = dstart[j];
     __syncthreads();
 #pragma unroll
     for (int it = 0; it < kItems; ++it) {
       const int local = warp * (32 * kItems) + it * 32 + lane;
       const uint32_t d = (local < valid_count) ? ((key[it] >> shift) & kDigitMask) : kDigitMask;
-      const uint32_t pos = s_digit_start[d] + s_warp_cnt[warp][d] + rank[it];
+      const uint32_t pos = s_digit_start[d] + s_warp_cnt[warp * NB + d] + rank[it];
       s_keys[pos] = key[it];
       s_vals[pos] = val[it];
     }
@@ -235,9 +263,9 @@ __global__ void __launch_bounds__(kSortThreads, 3) k_radix_scatter(
         vals_out[gpos] = v;
       }
       if (EP == 1) {
-        // tiles touched by this Gaussian, added to the sum of its block of kScanBlock sorted positions; a warp whose
+        // the Gaussian's count, added to the sum of its block of kScanBlock sorted positions; a warp whose
         // lanes all fall into one block (the usual case: a run is contiguous) adds once
-        uint32_t tt = ok ? __ldg(ep.tiles_touched + v) : 0u;
+        uint32_t tt = ok ? (__ldg(ep.counts + v) & ep.count_mask) : 0u;
         const uint32_t blk = gpos / kScanBlock, blk0 = __shfl_sync(kFull, blk, 0);
         if (__all_sync(kFull, !ok || blk == blk0)) {
 #pragma unroll
@@ -250,62 +278,56 @@ __global__ void __launch_bounds__(kSortThreads, 3) k_radix_scatter(
       if (EP == 2 && ok) {
         const uint32_t run_first = s_digit_start[d];
         const uint32_t run_end = d == kDigitMask ? (uint32_t)valid_count : s_digit_start[d + 1];   // slots past the input hold no run
-        if ((uint32_t)j == run_first) atomicMin(ep.ranges + 2 * k, gpos);
-        else if (s_keys[j - 1] != k) ep.ranges[2 * k] = gpos;
-        if ((uint32_t)j + 1 == run_end) atomicMax(ep.ranges + 2 * k + 1, gpos + 1);
-        else if (s_keys[j + 1] != k) ep.ranges[2 * k + 1] = gpos + 1;
+        const uint32_t id = k >> ep.key_shift;
+        if ((uint32_t)j == run_first) atomicMin(ep.ranges + 2 * id, gpos);
+        else if ((s_keys[j - 1] >> ep.key_shift) != id) ep.ranges[2 * id] = gpos;
+        if ((uint32_t)j + 1 == run_end) atomicMax(ep.ranges + 2 * id + 1, gpos + 1);
+        else if ((s_keys[j + 1] >> ep.key_shift) != id) ep.ranges[2 * id + 1] = gpos + 1;
       }
     }
     __syncthreads();
-    s_base[tid] += cnt;
+#pragma unroll
+    for (int j = 0; j < DPT; ++j) s_base[tid * DPT + j] += cnt[j];
     __syncthreads();
   }
 }
 
-// ---- tiles touched in depth order -----------------------------------------------------------
+__global__ void k_flag_if_greater(const unsigned long long *__restrict__ value, unsigned long long bound, uint32_t *__restrict__ flag) {
+  if (*value > bound) *flag = 1u;
+}
 
-// Emit the instances of each Gaussian, in depth order: the tiles its alpha >= 1/255 ellipse meets
-// (TileSpans, the same function the preprocess counted with), tile rows top to bottom, tiles left
-// to right.  Small footprints are written by their own thread; large ones by the whole warp.
-constexpr uint32_t kKeygenStage = 512;   // instances a warp stages in shared memory (4 KB per warp)
+__global__ void k_iota(uint32_t *__restrict__ out, int n) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) out[i] = (uint32_t)i;
+}
 
-__global__ void __launch_bounds__(kScanBlock) k_keygen(const uint32_t *__restrict__ order, const uint16_t *__restrict__ rect,
-                                                       const float *__restrict__ mean2d,
-                                                       const float *__restrict__ conic_opacity,
-                                                       const uint32_t *__restrict__ tiles_touched,
-                                                       const uint32_t *__restrict__ block_sums, int64_t n, int gx,
-                                                       int W, int H, uint32_t capacity,
-                                                       uint32_t *__restrict__ inst_tiles,
-                                                       uint32_t *__restrict__ inst_vals) {
+// ---- cell records in depth order ---------------------------------------------------------------
+// Every Gaussian, in depth order, writes its records (cell id << 16 | tile mask) and its id.  A Gaussian of at most
+// 3 x 3 cells copies what the preprocess stored; a larger one is worked out again by its whole warp: per row of cells
+// four lanes take the four tile rows, then the lanes take one cell each.
+__global__ void __launch_bounds__(kScanBlock) k_emit_records(
+    const uint32_t *__restrict__ order, const uint32_t *__restrict__ cell_count, const uint32_t *__restrict__ cell_records,
+    const uint16_t *__restrict__ rect, const float *__restrict__ mean2d, const float *__restrict__ conic_opacity,
+    const uint32_t *__restrict__ block_sums, int64_t n, int cgx, int W, int H, uint32_t capacity,
+    uint32_t *__restrict__ rec_keys, uint32_t *__restrict__ rec_vals, unsigned long long *__restrict__ rec_total,
+    uint32_t *__restrict__ overflow) {
   __shared__ uint32_t s_w[kScanBlock / 32], s_before[kScanBlock / 32];
-  __shared__ uint32_t s_stage[kScanBlock / 32][2 * kKeygenStage];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int64_t i = (int64_t)blockIdx.x * kScanBlock + tid;
-  uint32_t g = 0, tiles = 0;
-  ushort4 r = make_ushort4(0, 0, 0, 0);
-  float4 sp0 = make_float4(0.f, 0.f, 1.f, 0.f);   // u, v, la, lb
-  float2 sp1 = make_float2(1.f, 0.f);             // lc, tau
+  uint32_t g = 0, cc = 0;
   if (i < n) {
     g = __ldg(order + i);
-    // the four gathers go out together (also for Gaussians without tiles, whose rows are then ignored)
-    tiles = __ldg(tiles_touched + g);
-    const ushort4 rr = __ldg(reinterpret_cast<const ushort4 *>(rect) + g);
-    const float2 m = __ldg(reinterpret_cast<const float2 *>(mean2d) + g);
-    const float4 q = __ldg(reinterpret_cast<const float4 *>(conic_opacity) + g);
-    if (tiles) {
-      r = rr;
-      sp0 = make_float4(m.x, m.y, q.x, q.y);
-      sp1 = make_float2(q.z, footprint_tau(q.w));
-    }
+    cc = __ldg(cell_count + g);
   }
-  uint32_t inc = tiles;
+  const uint32_t cnt = cc & ~kCellBig;
+  uint32_t inc = cnt;
 #pragma unroll
   for (int s = 1; s < 32; s <<= 1) {
     const uint32_t t = __shfl_up_sync(kFull, inc, s);
     if (lane >= s) inc += t;
   }
   if (lane == 31) s_w[warp] = inc;
-  // instances of all CTAs before this one: the sums per kScanBlock Gaussians come from the last pass of the depth
+  // records of all CTAs before this one: the sums per kScanBlock Gaussians come from the last pass of the depth
   // sort; every CTA adds up its own prefix (a few loads per thread) instead of a scan kernel doing it for all
   uint32_t before = 0;
   for (int k = tid; k < (int)blockIdx.x; k += kScanBlock) before += __ldg(block_sums + k);
@@ -316,177 +338,475 @@ __global__ void __launch_bounds__(kScanBlock) k_keygen(const uint32_t *__restric
   uint32_t off = 0;
 #pragma unroll
   for (int k = 0; k < kScanBlock / 32; ++k) off += s_before[k] + ((k < warp) ? s_w[k] : 0u);
-  off += inc - tiles;
-  constexpr uint32_t kSmall = 32;
-  // A warp whose footprints add up to at most kKeygenStage instances writes them to shared memory first and
-  // copies the block out with coalesced stores; lanes writing their own short runs directly would touch a
-  // different sector with every store.  Staged or not, the emission below is the same: only the destination
-  // and the origin of the positions differ.
-  const uint32_t warp_total = __shfl_sync(kFull, inc, 31);
-  const uint32_t warp_base = __shfl_sync(kFull, off, 0);
-  const bool staged = warp_total <= kKeygenStage;
-  uint32_t *dst_tiles = staged ? s_stage[warp] : inst_tiles;
-  uint32_t *dst_vals = staged ? s_stage[warp] + kKeygenStage : inst_vals;
-  const uint32_t limit = staged ? kKeygenStage : capacity;   // never past the buffers, even if the count was taken on the device
-  if (staged) off -= warp_base;
-  if (tiles > 0 && tiles <= kSmall) {
-    TileSpans sp;
-    sp.setup(sp0.x, sp0.y, sp0.z, sp0.w, sp1.x, sp1.y, W, H);
-    uint32_t p = off;
-    for (int ty = r.y; ty < (int)r.w; ++ty) {
-      int xa, xb;
-      if (!sp.row(ty, r.x, r.z, xa, xb)) continue;
-      for (int tx = xa; tx < xb; ++tx) {
-        if (p < limit) {
-          dst_tiles[p] = (uint32_t)(ty * gx + tx);
-          dst_vals[p] = g;
-        }
-        ++p;
+  off += inc - cnt;
+  if (blockIdx.x == gridDim.x - 1 && tid == kScanBlock - 1) {   // the last thread of all: its end is the number of records
+    *rec_total = (unsigned long long)off + cnt;
+    if (off + cnt > capacity) *overflow = 1u;                    // more records than the buffers hold: tell the host
+  }
+  if (cnt && !(cc & kCellBig)) {
+    const uint32_t *src = cell_records + (size_t)g * kCellSlots;
+    for (uint32_t k = 0; k < cnt; ++k) {
+      if (off + k < capacity) {   // never past the buffers, even if the count was taken on the device
+        rec_keys[off + k] = __ldg(src + k);
+        rec_vals[off + k] = g;
       }
     }
   }
-  // a large footprint is shared by the warp: one tile row per lane, then the tiles of each row
-  uint32_t big = __ballot_sync(kFull, tiles > kSmall);
+  uint32_t big = __ballot_sync(kFull, (cc & kCellBig) != 0u);
   while (big) {
     const int src = __ffs(big) - 1;
     big &= big - 1;
-    TileSpans sp;
-    sp.setup(__shfl_sync(kFull, sp0.x, src), __shfl_sync(kFull, sp0.y, src), __shfl_sync(kFull, sp0.z, src),
-             __shfl_sync(kFull, sp0.w, src), __shfl_sync(kFull, sp1.x, src), __shfl_sync(kFull, sp1.y, src), W, H);
-    uint32_t p = __shfl_sync(kFull, off, src);
     const uint32_t s_g = __shfl_sync(kFull, g, src);
-    const int x0 = (int)__shfl_sync(kFull, (uint32_t)r.x, src), x1 = (int)__shfl_sync(kFull, (uint32_t)r.z, src);
-    const int y0 = (int)__shfl_sync(kFull, (uint32_t)r.y, src), y1 = (int)__shfl_sync(kFull, (uint32_t)r.w, src);
-    for (int tyb = y0; tyb < y1; tyb += 32) {
+    uint32_t p = __shfl_sync(kFull, off, src);
+    // the owner's projected values reach every lane by a broadcast load
+    const ushort4 r = __ldg(reinterpret_cast<const ushort4 *>(rect) + s_g);
+    const float2 m = __ldg(reinterpret_cast<const float2 *>(mean2d) + s_g);
+    const float4 q = __ldg(reinterpret_cast<const float4 *>(conic_opacity) + s_g);
+    TileSpans sp;
+    sp.setup(m.x, m.y, q.x, q.y, q.z, footprint_tau(q.w), W, H);
+    const int cy0 = r.y >> 2, cy1 = ((int)r.w - 1) >> 2;
+    for (int cy = cy0; cy <= cy1; ++cy) {
+      // lanes 0..3: the tile rows of this row of cells
       int xa = 0, xb = 0;
-      if (tyb + lane < y1 && !sp.row(tyb + lane, x0, x1, xa, xb)) xa = xb = 0;
-      uint32_t incl = (uint32_t)(xb - xa);
+      const int ty = 4 * cy + lane;
+      const bool has = lane < 4 && ty >= (int)r.y && ty < (int)r.w && sp.row(ty, r.x, r.z, xa, xb);
+      int lo = has ? (xa >> 2) : (1 << 30), hi = has ? ((xb - 1) >> 2) : -1;
+      lo = min(lo, __shfl_xor_sync(kFull, lo, 1)); hi = max(hi, __shfl_xor_sync(kFull, hi, 1));
+      lo = min(lo, __shfl_xor_sync(kFull, lo, 2)); hi = max(hi, __shfl_xor_sync(kFull, hi, 2));
+      lo = __shfl_sync(kFull, lo, 0); hi = __shfl_sync(kFull, hi, 0);
+      if (hi < lo) continue;
+      int ra[4], rb[4];
 #pragma unroll
-      for (int s = 1; s < 32; s <<= 1) {
-        const uint32_t t = __shfl_up_sync(kFull, incl, s);
-        if (lane >= s) incl += t;
+      for (int k = 0; k < 4; ++k) {
+        ra[k] = __shfl_sync(kFull, has ? xa : 0, k);
+        rb[k] = __shfl_sync(kFull, has ? xb : 0, k);
       }
-      const uint32_t excl = incl - (uint32_t)(xb - xa);
-      const int rows = min(32, y1 - tyb);
-      for (int rr = 0; rr < rows; ++rr) {
-        const int a = __shfl_sync(kFull, xa, rr), b = __shfl_sync(kFull, xb, rr);
-        const uint32_t o = p + __shfl_sync(kFull, excl, rr);
-        for (int tx = a + lane; tx < b; tx += 32) {
-          const uint32_t q = o + (uint32_t)(tx - a);
-          if (q < limit) {
-            dst_tiles[q] = (uint32_t)((tyb + rr) * gx + tx);
-            dst_vals[q] = s_g;
+      for (int cb = lo; cb <= hi; cb += 32) {
+        const int cx = cb + lane;
+        if (cx <= hi) {
+          uint32_t mask = 0u;
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const int a0 = max(ra[k], 4 * cx) - 4 * cx, b0 = min(rb[k], 4 * cx + 4) - 4 * cx;
+            if (b0 > a0) mask |= (((1u << (b0 - a0)) - 1u) << a0) << (4 * k);
+          }
+          const uint32_t dst = p + (uint32_t)(cx - lo);
+          if (dst < capacity) {
+            rec_keys[dst] = ((uint32_t)(cy * cgx + cx) << 16) | mask;
+            rec_vals[dst] = s_g;
           }
         }
       }
-      p += __shfl_sync(kFull, incl, 31);
-    }
-  }
-  if (staged) {
-    __syncwarp();
-    const uint32_t *st = s_stage[warp], *sv = st + kKeygenStage;
-    for (uint32_t q = lane; q < warp_total; q += 32) {
-      if (warp_base + q < capacity) {
-        inst_tiles[warp_base + q] = st[q];
-        inst_vals[warp_base + q] = sv[q];
-      }
+      p += (uint32_t)(hi - lo + 1);
     }
   }
 }
 
-// Launch order of the blend CTAs: tiles by decreasing list length (log2 buckets), so that the long
-// tiles start first and the short ones fill the tail.  The order inside a bucket is whatever the
-// atomics give; it affects scheduling only, never a result.
-// A tile without instances comes in as (0xffffffff, 0), the neutral values of the range epilogue, and leaves as (0, 0).
-__global__ void __launch_bounds__(1024) k_tile_order(uint32_t *__restrict__ ranges, int num_tiles,
-                                                     uint32_t *__restrict__ order) {
+// ---- from the sorted records of a cell to the lists of its tiles ----------------------------------
+// Chunks: the records of cell c, [range_c.start, range_c.end), in pieces of kCellChunk; chunk_first[c] = number of
+// chunks of the cells before c.  A cell without records comes in as (0xffffffff, 0), the neutral values of the
+// range epilogue.
+__global__ void __launch_bounds__(1024) k_cell_chunks(const uint32_t *__restrict__ cell_ranges, int num_cells,
+                                                      uint32_t *__restrict__ chunk_first) {
+  __shared__ uint32_t s_w[32];
+  __shared__ uint32_t s_carry;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) s_carry = 0;
+  __syncthreads();
+  for (int base = 0; base < num_cells; base += 1024) {
+    const int c = base + tid;
+    uint32_t v = 0;
+    if (c < num_cells) {
+      const uint32_t s0 = cell_ranges[2 * c], e0 = cell_ranges[2 * c + 1];
+      v = e0 > s0 ? (e0 - s0 + kCellChunk - 1) / kCellChunk : 0u;
+    }
+    uint32_t inc = v;
+#pragma unroll
+    for (int s = 1; s < 32; s <<= 1) {
+      const uint32_t t = __shfl_up_sync(kFull, inc, s);
+      if (lane >= s) inc += t;
+    }
+    if (lane == 31) s_w[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+      uint32_t w = s_w[lane], winc = w;
+#pragma unroll
+      for (int s = 1; s < 32; s <<= 1) {
+        const uint32_t t = __shfl_up_sync(kFull, winc, s);
+        if (lane >= s) winc += t;
+      }
+      s_w[lane] = winc - w;
+    }
+    __syncthreads();
+    const uint32_t carry = s_carry;
+    if (c < num_cells) chunk_first[c] = carry + s_w[warp] + inc - v;
+    __syncthreads();
+    if (tid == 1023) s_carry = carry + s_w[warp] + inc;
+    __syncthreads();
+  }
+  if (tid == 0) chunk_first[num_cells] = s_carry;
+}
+
+// The cell and the record range of chunk q, or false if there is no such chunk.
+__device__ __forceinline__ bool chunk_of(uint32_t q, const uint32_t *__restrict__ chunk_first, const uint32_t *__restrict__ cell_ranges,
+                                         int num_cells, int &cell, uint32_t &begin, uint32_t &end) {
+  if (q >= __ldg(chunk_first + num_cells)) return false;
+  int lo = 0, hi = num_cells - 1;     // largest c with chunk_first[c] <= q (cells without records share a value: take the last)
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (__ldg(chunk_first + mid) <= q) lo = mid; else hi = mid - 1;
+  }
+  cell = lo;
+  const uint32_t s0 = __ldg(cell_ranges + 2 * lo), e0 = __ldg(cell_ranges + 2 * lo + 1);
+  begin = s0 + (q - __ldg(chunk_first + lo)) * kCellChunk;
+  end = min(begin + (uint32_t)kCellChunk, e0);
+  return true;
+}
+
+// The 16 tile counts of the records a lane holds (masks of up to 8 records), as four words of four byte counters:
+// one multiplication spreads the four bits of a tile row of the cell over the four bytes of a word.
+__device__ __forceinline__ void count_masks(const uint32_t mask[8], int have, uint32_t acc[4]) {
+  acc[0] = acc[1] = acc[2] = acc[3] = 0u;
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const uint32_t m = k < have ? mask[k] : 0u;
+#pragma unroll
+    for (int r = 0; r < 4; ++r) acc[r] += (((m >> (4 * r)) & 15u) * 0x00204081u) & 0x01010101u;
+  }
+}
+
+// Sum over the warp of the byte counters, widened to 16 bits on the way (8 records x 32 lanes = 256 at most): tile
+// 4 r + b of the cell ends in bits [16 (b & 1), +16) of word r * 2 + (b >> 1), in every lane.
+__device__ __forceinline__ void warp_sum_counts(const uint32_t acc[4], uint32_t out[8]) {
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    out[2 * r] = (acc[r] & 0xffu) | ((acc[r] & 0xff00u) << 8);
+    out[2 * r + 1] = ((acc[r] >> 16) & 0xffu) | ((acc[r] >> 8) & 0xff0000u);
+  }
+#pragma unroll
+  for (int w = 0; w < 8; ++w)
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) out[w] += __shfl_xor_sync(kFull, out[w], s);
+}
+__device__ __forceinline__ uint32_t tile_count_of(const uint32_t sums[8], int t) {   // t = 4 r + b
+  return (sums[2 * (t >> 2) + ((t & 3) >> 1)] >> (16 * (t & 1))) & 0xffffu;
+}
+
+constexpr int kExpandThreads = 256;
+constexpr int kExpandWarps = kExpandThreads / 32;
+
+// Per chunk: how many instances it holds for each of the 16 tiles of its cell.
+__global__ void __launch_bounds__(kExpandThreads) k_chunk_counts(const uint32_t *__restrict__ rec_keys,
+                                                                 const uint32_t *__restrict__ cell_ranges,
+                                                                 const uint32_t *__restrict__ chunk_first, int num_cells,
+                                                                 uint32_t *__restrict__ chunk_counts) {
+  __shared__ uint32_t s_cnt[kExpandWarps][16];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  int cell;
+  uint32_t begin, end;
+  if (!chunk_of(blockIdx.x, chunk_first, cell_ranges, num_cells, cell, begin, end)) return;
+  // warp w holds records [begin + 256 w, + 256): lane l the records 256 w + 32 k + l, k = 0..7
+  uint32_t mask[8];
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const uint32_t idx = begin + (uint32_t)(256 * warp + 32 * k + lane);
+    mask[k] = idx < end ? (__ldg(rec_keys + idx) & 0xffffu) : 0u;
+  }
+  uint32_t acc[4], sums[8];
+  count_masks(mask, 8, acc);
+  warp_sum_counts(acc, sums);
+  if (lane < 16) s_cnt[warp][lane] = tile_count_of(sums, lane);
+  __syncthreads();
+  if (tid < 16) {
+    uint32_t t = 0;
+#pragma unroll
+    for (int w = 0; w < kExpandWarps; ++w) t += s_cnt[w][tid];
+    chunk_counts[(size_t)blockIdx.x * 16 + tid] = t;
+  }
+}
+
+// Per cell (one warp each, lanes 0..15 = its tiles): where each chunk's instances of a tile begin inside the tile's
+// list (the running sum of the chunks' counts, in chunk order) and the length of that list.
+__global__ void __launch_bounds__(256) k_cell_prefix(const uint32_t *__restrict__ chunk_first, const uint32_t *__restrict__ chunk_counts,
+                                                     int gx, int gy, int cgx, int num_cells, uint32_t *__restrict__ chunk_bases,
+                                                     uint32_t *__restrict__ tile_counts) {
+  const int lane = threadIdx.x & 31, cell = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (cell >= num_cells || lane >= 16) return;
+  const uint32_t q0 = __ldg(chunk_first + cell), q1 = __ldg(chunk_first + cell + 1);
+  uint32_t run = 0;
+  uint32_t q = q0;
+  for (; q + 4 <= q1; q += 4) {   // four independent loads in flight
+    const uint32_t v0 = __ldg(chunk_counts + (size_t)q * 16 + lane), v1 = __ldg(chunk_counts + (size_t)(q + 1) * 16 + lane);
+    const uint32_t v2 = __ldg(chunk_counts + (size_t)(q + 2) * 16 + lane), v3 = __ldg(chunk_counts + (size_t)(q + 3) * 16 + lane);
+    chunk_bases[(size_t)q * 16 + lane] = run; run += v0;
+    chunk_bases[(size_t)(q + 1) * 16 + lane] = run; run += v1;
+    chunk_bases[(size_t)(q + 2) * 16 + lane] = run; run += v2;
+    chunk_bases[(size_t)(q + 3) * 16 + lane] = run; run += v3;
+  }
+  for (; q < q1; ++q) {
+    chunk_bases[(size_t)q * 16 + lane] = run;
+    run += __ldg(chunk_counts + (size_t)q * 16 + lane);
+  }
+  const int tx = 4 * (cell % cgx) + (lane & 3), ty = 4 * (cell / cgx) + (lane >> 2);
+  if (tx < gx && ty < gy) tile_counts[ty * gx + tx] = run;
+}
+
+// One CTA: the exclusive scan of the tile counts in tile order = the tile ranges, and the launch order of the blend
+// CTAs (tiles by decreasing list length in log2 buckets: the long tiles start first and the short ones fill the tail;
+// the order inside a bucket is whatever the atomics give, it affects scheduling only, never a result).
+__global__ void __launch_bounds__(1024) k_tile_scan(const uint32_t *__restrict__ tile_counts, int num_tiles, uint32_t capacity,
+                                                    uint32_t *__restrict__ tile_starts, uint32_t *__restrict__ ranges,
+                                                    uint32_t *__restrict__ order) {
+  __shared__ uint32_t s_w[32];
+  __shared__ uint32_t s_carry;
   __shared__ uint32_t s_cnt[33], s_off[33];
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) s_carry = 0;
   if (tid < 33) s_cnt[tid] = 0;
   __syncthreads();
-  for (int t = tid; t < num_tiles; t += 1024) {
-    if (ranges[2 * t + 1] == 0u) ranges[2 * t] = 0u;
-    const uint32_t len = ranges[2 * t + 1] - ranges[2 * t];
-    atomicAdd(&s_cnt[len ? 32 - __clz(len) : 0], 1u);
+  for (int base = 0; base < num_tiles; base += 1024) {
+    const int t = base + tid;
+    const uint32_t v = t < num_tiles ? tile_counts[t] : 0u;
+    if (t < num_tiles) atomicAdd(&s_cnt[v ? 32 - __clz(v) : 0], 1u);
+    uint32_t inc = v;
+#pragma unroll
+    for (int s = 1; s < 32; s <<= 1) {
+      const uint32_t u = __shfl_up_sync(kFull, inc, s);
+      if (lane >= s) inc += u;
+    }
+    if (lane == 31) s_w[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+      uint32_t w = s_w[lane], winc = w;
+#pragma unroll
+      for (int s = 1; s < 32; s <<= 1) {
+        const uint32_t u = __shfl_up_sync(kFull, winc, s);
+        if (lane >= s) winc += u;
+      }
+      s_w[lane] = winc - w;
+    }
+    __syncthreads();
+    const uint32_t carry = s_carry;
+    if (t < num_tiles) {
+      const uint32_t start = carry + s_w[warp] + inc - v;
+      tile_starts[t] = start;
+      // a tile without instances: (0, 0); never past the capacity of the instance buffers (a device-side count may
+      // exceed it: the lists are then cut off and the host is told)
+      const uint32_t s0 = min(start, capacity), e0 = start + v < start ? capacity : min(start + v, capacity);
+      ranges[2 * t] = e0 > s0 ? s0 : 0u;
+      ranges[2 * t + 1] = e0 > s0 ? e0 : 0u;
+    }
+    __syncthreads();
+    if (tid == 1023) s_carry = carry + s_w[warp] + inc;
+    __syncthreads();
   }
-  __syncthreads();
   if (tid == 0) {
     uint32_t off = 0;
     for (int b = 32; b >= 0; --b) { s_off[b] = off; off += s_cnt[b]; }
   }
   __syncthreads();
   for (int t = tid; t < num_tiles; t += 1024) {
-    const uint32_t len = ranges[2 * t + 1] - ranges[2 * t];
+    const uint32_t len = tile_counts[t];
     order[atomicAdd(&s_off[len ? 32 - __clz(len) : 0], 1u)] = (uint32_t)t;
+  }
+}
+
+__device__ __forceinline__ void store_if(bool p, uint32_t *addr, uint32_t v) {
+  asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %0, 0;\n\t@q st.global.u32 [%1], %2;\n\t}" :: "r"((uint32_t)p), "l"(addr), "r"(v) : "memory");
+}
+
+// The tile id of every instance, from the ranges: one CTA per tile fills its stretch of the sorted list.
+__global__ void __launch_bounds__(128) k_fill_tile_ids(const uint32_t *__restrict__ ranges, uint32_t *__restrict__ out_tiles) {
+  const uint32_t t = blockIdx.x, b = __ldg(ranges + 2 * t), e = __ldg(ranges + 2 * t + 1);
+  for (uint32_t p = b + threadIdx.x; p < e; p += 128) out_tiles[p] = t;
+}
+
+// Per chunk: write its instances.  A warp's records are consecutive in depth order, 32 at a time.  A record's slot
+// in the list of tile t is the tile's running position plus the number of lower lanes that also list t: the 16
+// indicator bits of a lane's mask are spread over four words of byte counters and one warp-wide prefix sum of those
+// four words ranks all 16 tiles at once (at most 32 per byte).  The running positions start from the tile's range,
+// the chunk's offset inside it and what the warps before this one hold; every lane keeps all 16 of them.
+__global__ void __launch_bounds__(kExpandThreads) k_expand(const uint32_t *__restrict__ rec_keys, const uint32_t *__restrict__ rec_vals,
+                                                           const uint32_t *__restrict__ cell_ranges,
+                                                           const uint32_t *__restrict__ chunk_first, int num_cells,
+                                                           const uint32_t *__restrict__ chunk_bases,
+                                                           const uint32_t *__restrict__ tile_starts, int gx, int gy, int cgx,
+                                                           uint32_t capacity, uint32_t *__restrict__ out_vals) {
+  __shared__ uint32_t s_cnt[kExpandWarps][16];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  int cell;
+  uint32_t begin, end;
+  if (!chunk_of(blockIdx.x, chunk_first, cell_ranges, num_cells, cell, begin, end)) return;
+  uint32_t mask[8], gid[8];
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const uint32_t idx = begin + (uint32_t)(256 * warp + 32 * k + lane);
+    const bool ok = idx < end;
+    mask[k] = ok ? (__ldg(rec_keys + idx) & 0xffffu) : 0u;
+    gid[k] = ok ? __ldg(rec_vals + idx) : 0u;
+  }
+  uint32_t acc[4], sums[8];
+  count_masks(mask, 8, acc);
+  warp_sum_counts(acc, sums);
+  if (lane < 16) s_cnt[warp][lane] = tile_count_of(sums, lane);
+  __syncthreads();
+  // lane t < 16 works out where tile t of the cell continues, then every lane takes a copy of all 16
+  const int tx0 = 4 * (cell % cgx), ty0 = 4 * (cell / cgx);
+  uint32_t mine = 0;
+  if (lane < 16) {
+    const int tx = tx0 + (lane & 3), ty = ty0 + (lane >> 2);
+    if (tx < gx && ty < gy) {   // (a tile of the cell outside the image has no instances)
+      mine = __ldg(tile_starts + ty * gx + tx) + __ldg(chunk_bases + (size_t)blockIdx.x * 16 + lane);
+      for (int w = 0; w < warp; ++w) mine += s_cnt[w][lane];
+    }
+  }
+  uint32_t cur[16];
+#pragma unroll
+  for (int t = 0; t < 16; ++t) cur[t] = __shfl_sync(kFull, mine, t);
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const uint32_t m = mask[k];
+    if (__ballot_sync(kFull, m != 0u) == 0u) continue;
+    uint32_t incl[4], own[4], tot[4];
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      own[r] = (((m >> (4 * r)) & 15u) * 0x00204081u) & 0x01010101u;
+      incl[r] = own[r];
+    }
+#pragma unroll
+    for (int sft = 1; sft < 32; sft <<= 1) {
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        const uint32_t u = __shfl_up_sync(kFull, incl[r], sft);
+        if (lane >= sft) incl[r] += u;
+      }
+    }
+#pragma unroll
+    for (int r = 0; r < 4; ++r) tot[r] = __shfl_sync(kFull, incl[r], 31);
+#pragma unroll
+    for (int t = 0; t < 16; ++t) {
+      const int r = t >> 2, sh = 8 * (t & 3);
+      // one predicated store (no branch): the lane lists tile t and the slot lies inside the buffer
+      const uint32_t pos = cur[t] + (((incl[r] - own[r]) >> sh) & 0xffu);
+      store_if(((m >> t) & 1u) != 0u && pos < capacity, out_vals + pos, gid[k]);
+      cur[t] += (tot[r] >> sh) & 0xffu;
+    }
   }
 }
 
 }  // namespace
 
-size_t sort_scratch_bytes(int64_t count) { return ((size_t)plan_for(count).blocks + 1) * 256 * sizeof(uint32_t); }
+size_t sort_scratch_bytes(int64_t count) { return ((size_t)sort_blocks(count) + 1) * (1 << kMaxDigitBits) * sizeof(uint32_t); }
+
+namespace {
+template <int BITS, int EP>
+void launch_scatter(int blocks, const uint32_t *src_k, const uint32_t *src_v, uint32_t *dst_k, uint32_t *dst_v, int64_t count,
+                    const unsigned long long *count_dev, int shift, const uint32_t *table, const uint32_t *totals,
+                    const SortEpilogue &ep, cudaStream_t st) {
+  constexpr size_t smem = scatter_smem_bytes<BITS>();
+  static bool opted[64] = {};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (smem > 48 * 1024 && dev >= 0 && dev < 64 && !opted[dev]) {
+    cudaFuncSetAttribute(k_radix_scatter<BITS, EP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    opted[dev] = true;
+  }
+  k_radix_scatter<BITS, EP><<<blocks, kSortThreads, smem, st>>>(src_k, src_v, dst_k, dst_v, count, count_dev, shift, table, totals,
+                                                                 blocks, ep);
+}
+}  // namespace
 
 int launch_radix_sort(const uint32_t *keys_in, const uint32_t *vals_in, uint32_t *keys_out, uint32_t *vals_out,
                        uint32_t *tmp_keys, uint32_t *tmp_vals, int64_t count, const unsigned long long *count_dev,
-                       int num_bits, void *scratch, const SortEpilogue *epilogue, cudaStream_t st) {
+                       int first_bit, int num_bits, int max_digit_bits, void *scratch, const SortEpilogue *epilogue,
+                       cudaStream_t st) {
   if (count <= 0) return 0;
-  const SortPlan plan = plan_for(count);
-  int passes = (num_bits + 7) / 8;
-  if (passes < 1) passes = 1;
-  const int bits = (num_bits + passes - 1) / passes;     // digits of equal width: 13 bits sort as 7 + 6
+  const int blocks = sort_blocks(count);
+  const int passes = radix_passes(num_bits, max_digit_bits);
+  int bits = (num_bits + passes - 1) / passes;     // digits of equal width: 13 bits sort as 7 + 6 under a limit of 8
+  if (bits < 4) bits = 4;                          // (bits above the keys' range are zero: sorting on them changes nothing)
   uint32_t *table = static_cast<uint32_t *>(scratch);
-  uint32_t *totals = table + (size_t)plan.blocks * 256;
+  uint32_t *totals = table + ((size_t)blocks << bits);
   const uint32_t *src_k = keys_in, *src_v = vals_in;
-  const SortEpilogue none = {nullptr, nullptr, 0, nullptr, 0, nullptr};
+  const SortEpilogue none = {nullptr, 0u, nullptr, 0, nullptr, 0, 0, nullptr};
   for (int p = 0; p < passes; ++p) {
     const bool to_out = ((passes - 1 - p) % 2) == 0;
     uint32_t *dst_k = to_out ? keys_out : tmp_keys, *dst_v = to_out ? vals_out : tmp_vals;
     const SortEpilogue ep = (p == passes - 1 && epilogue) ? *epilogue : none;
     const int mode = ep.block_sums ? 1 : ep.ranges ? 2 : 0;
-    k_radix_hist<<<plan.blocks, kSortThreads, 0, st>>>(src_k, count, count_dev, bits * p, (1u << bits) - 1u,
-                                                        plan.tiles_per_block, plan.extra, table, ep);
-    k_radix_scan_rows<<<256, 256, 0, st>>>(table, plan.blocks, totals);
-#define GS_SCATTER_ARGS                                                                                              \
-  <<<plan.blocks, kSortThreads, 0, st>>>(src_k, src_v, dst_k, dst_v, count, count_dev, bits * p, plan.tiles_per_block, \
-                                         plan.extra, table, totals, plan.blocks, ep)
-#define GS_SCATTER(B)                                              \
-  case B:                                                          \
-    if (mode == 2) k_radix_scatter<B, 2> GS_SCATTER_ARGS;          \
-    else k_radix_scatter<B, 0> GS_SCATTER_ARGS;                    \
+    const int shift = first_bit + bits * p;
+    k_radix_hist<<<blocks, kSortThreads, 0, st>>>(src_k, count, count_dev, shift, bits, table, ep);
+    k_radix_scan_rows<<<1 << bits, 256, 0, st>>>(table, blocks, totals);
+#define GS_ARGS blocks, src_k, src_v, dst_k, dst_v, count, count_dev, shift, table, totals, ep, st
+#define GS_SCATTER(B)                                             \
+  case B:                                                         \
+    if (mode == 2) launch_scatter<B, 2>(GS_ARGS);                 \
+    else launch_scatter<B, 0>(GS_ARGS);                           \
     break;
     switch (bits) {
-      GS_SCATTER(1) GS_SCATTER(2) GS_SCATTER(3) GS_SCATTER(4) GS_SCATTER(5) GS_SCATTER(6) GS_SCATTER(7)
+      GS_SCATTER(4) GS_SCATTER(5) GS_SCATTER(6) GS_SCATTER(7) GS_SCATTER(9) GS_SCATTER(10)
+      case 8:
+        if (mode == 1) launch_scatter<8, 1>(GS_ARGS);
+        else if (mode == 2) launch_scatter<8, 2>(GS_ARGS);
+        else launch_scatter<8, 0>(GS_ARGS);
+        break;
       default:
-        if (mode == 1) k_radix_scatter<8, 1> GS_SCATTER_ARGS;
-        else if (mode == 2) k_radix_scatter<8, 2> GS_SCATTER_ARGS;
-        else k_radix_scatter<8, 0> GS_SCATTER_ARGS;
+        if (mode == 2) launch_scatter<11, 2>(GS_ARGS);
+        else launch_scatter<11, 0>(GS_ARGS);
     }
 #undef GS_SCATTER
-#undef GS_SCATTER_ARGS
+#undef GS_ARGS
     src_k = dst_k;
     src_v = dst_v;
   }
   return 3 * passes;
 }
 
+int radix_passes(int num_bits, int max_digit_bits) {
+  const int m = max_digit_bits < 4 ? 4 : max_digit_bits > kMaxDigitBits ? kMaxDigitBits : max_digit_bits;
+  const int p = (num_bits + m - 1) / m;
+  return p < 1 ? 1 : p;
+}
+
 size_t scan_scratch_bytes(int64_t n) { return (size_t)((n + kScanBlock - 1) / kScanBlock + 1) * sizeof(uint32_t); }
 int num_scan_blocks(int64_t n) { return (int)((n + kScanBlock - 1) / kScanBlock); }
 
-int launch_keygen(const uint32_t *depth_order, const uint16_t *rect, const float *mean2d, const float *conic_opacity,
-                  const uint32_t *tiles_touched, const uint32_t *block_sums, uint32_t *inst_tiles, uint32_t *inst_vals,
-                  int64_t n, int gx, int W, int H, int64_t capacity, cudaStream_t st) {
+int launch_emit_records(const uint32_t *depth_order, const uint32_t *cell_count, const uint32_t *cell_records,
+                        const uint16_t *rect, const float *mean2d, const float *conic_opacity, const uint32_t *block_sums,
+                        uint32_t *rec_keys, uint32_t *rec_vals, unsigned long long *rec_total, uint32_t *overflow, int64_t n,
+                        int cgx, int W, int H, int64_t capacity, cudaStream_t st) {
   if (n <= 0) return 0;
-  const int blocks = num_scan_blocks(n);
   const uint32_t cap = capacity > 0xffffffffll ? 0xffffffffu : (uint32_t)capacity;
-  k_keygen<<<blocks, kScanBlock, 0, st>>>(depth_order, rect, mean2d, conic_opacity, tiles_touched, block_sums, n, gx, W, H,
-                                          cap, inst_tiles, inst_vals);
+  k_emit_records<<<num_scan_blocks(n), kScanBlock, 0, st>>>(depth_order, cell_count, cell_records, rect, mean2d, conic_opacity,
+                                                           block_sums, n, cgx, W, H, cap, rec_keys, rec_vals, rec_total, overflow);
   return 1;
 }
 
-// Settles the ranges of the empty tiles and orders the tiles for the blend launches.  With `clear` (no instance was
-// sorted, so no range epilogue ran) every range is zeroed first.
-int launch_tile_order(uint32_t *ranges, uint32_t *order, int num_tiles, bool clear, cudaStream_t st) {
-  if (clear) cudaMemsetAsync(ranges, 0, (size_t)num_tiles * 2 * sizeof(uint32_t), st);
-  k_tile_order<<<1, 1024, 0, st>>>(ranges, num_tiles, order);
+int max_chunks(int64_t record_capacity, int num_cells) { return (int)((record_capacity + kCellChunk - 1) / kCellChunk) + num_cells; }
+
+int launch_expand(const uint32_t *rec_keys, const uint32_t *rec_vals, const uint32_t *cell_ranges, const CellScratch &cs,
+                  int64_t record_capacity, int64_t pair_capacity, int gx, int gy, int cgx, int cgy, uint32_t *sorted_tiles,
+                  uint32_t *sorted_vals, uint32_t *tile_ranges, uint32_t *tile_order, cudaStream_t st) {
+  const int num_cells = cgx * cgy, chunks = max_chunks(record_capacity, num_cells);
+  const uint32_t cap = pair_capacity > 0xffffffffll ? 0xffffffffu : (uint32_t)pair_capacity;
+  k_cell_chunks<<<1, 1024, 0, st>>>(cell_ranges, num_cells, cs.chunk_first);
+  k_chunk_counts<<<chunks, kExpandThreads, 0, st>>>(rec_keys, cell_ranges, cs.chunk_first, num_cells, cs.chunk_counts);
+  k_cell_prefix<<<(num_cells + 7) / 8, 256, 0, st>>>(cs.chunk_first, cs.chunk_counts, gx, gy, cgx, num_cells, cs.chunk_bases, cs.tile_counts);
+  k_tile_scan<<<1, 1024, 0, st>>>(cs.tile_counts, gx * gy, cap, cs.tile_starts, tile_ranges, tile_order);
+  k_expand<<<chunks, kExpandThreads, 0, st>>>(rec_keys, rec_vals, cell_ranges, cs.chunk_first, num_cells, cs.chunk_bases, cs.tile_starts,
+                                              gx, gy, cgx, cap, sorted_vals);
+  k_fill_tile_ids<<<gx * gy, 128, 0, st>>>(tile_ranges, sorted_tiles);
+  return 6;
+}
+
+void launch_flag_if_greater(const unsigned long long *value, unsigned long long bound, uint32_t *flag, cudaStream_t st) {
+  k_flag_if_greater<<<1, 1, 0, st>>>(value, bound, flag);
+}
+
+// No record was sorted (no Gaussian, or none that reaches a tile): every tile is empty.
+int launch_empty_binning(uint32_t *tile_ranges, uint32_t *tile_order, int num_tiles, cudaStream_t st) {
+  cudaMemsetAsync(tile_ranges, 0, (size_t)num_tiles * 2 * sizeof(uint32_t), st);
+  k_iota<<<(num_tiles + 255) / 256, 256, 0, st>>>(tile_order, num_tiles);
   return 1;
 }
 

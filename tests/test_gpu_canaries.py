@@ -44,7 +44,7 @@ def step(api, torch, sc, cam, device_count):
     g = Guarded(torch, dev)
     f32, i32, i16 = torch.float32, torch.int32, torch.int16
     proj = api.Projected(g((n, 2), f32), g((n, 4), f32), g((n, 3), f32), g((n,), i32), g((n, 4), i16), g((n,), i32),
-                         g((n, 4), f32))
+                         g((n, 4), f32), g((n,), i32), g((n, 9), i32))
     P = api.gs_preprocess(ctx, ds, ccam, proj)           # sizes the instance buffers exactly
     assert P > 0
     binning = api.Binning(g((n,), i32), g((P,), i32), g((P,), i32), g((tiles, 2), i32), g((tiles,), i32))
