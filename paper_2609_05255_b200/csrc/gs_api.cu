@@ -436,7 +436,7 @@ GsStatus gs_render_forward(GsContext *ctx, int64_t n, const GsProjected *proj, c
       if (on_device)   // more instances than the capacity: the lists are cut off, the host is told
         launch_flag_if_greater(count_dev, (unsigned long long)pair_capacity, overflow, s);
       t.done(launch_expand(sorted_rkeys, sorted_rvals, w.cell_ranges, w.cells, num_pairs, pair_capacity, cd.gx, cd.gy, cd.cgx,
-                           cd.cgy, bin->sorted_tiles, bin->sorted_vals, bin->tile_ranges, bin->tile_order, s));
+                           cd.cgy, bin->sorted_vals, bin->tile_ranges, bin->tile_order, s));
     }
   } else {
     StageTimer t(ctx, GS_STAGE_TILE_RANGES, s);
@@ -445,7 +445,7 @@ GsStatus gs_render_forward(GsContext *ctx, int64_t n, const GsProjected *proj, c
   {
     StageTimer t(ctx, GS_STAGE_BLEND_FWD, s);
     t.done(launch_blend_fwd(cd, bin->tile_ranges, bin->tile_order, bin->sorted_vals, proj->mean2d, proj->conic_opacity, proj->color,
-                            image, final_T, n_contrib, s));
+                            num_pairs > 0 ? bin->sorted_tiles : nullptr, image, final_T, n_contrib, s));
   }
   return check_cuda(ctx, cudaGetLastError(), "render_forward launch");
 }

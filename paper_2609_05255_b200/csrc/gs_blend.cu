@@ -92,7 +92,8 @@ __global__ void __launch_bounds__(kThreads) k_blend_fwd(CamDev cam, const uint32
                                                         const uint32_t *__restrict__ vals,
                                                         const float *__restrict__ mean2d,
                                                         const float *__restrict__ conic_opacity,
-                                                        const float *__restrict__ color, float *__restrict__ image,
+                                                        const float *__restrict__ color, uint32_t *__restrict__ sorted_tiles,
+                                                        float *__restrict__ image,
                                                         float *__restrict__ final_T, uint32_t *__restrict__ n_contrib) {
   __shared__ float4 s_xyab[kBatch];
   __shared__ float2 s_co[kBatch];
@@ -102,6 +103,9 @@ __global__ void __launch_bounds__(kThreads) k_blend_fwd(CamDev cam, const uint32
   quad_of(tile, cam.gx, tid, px, py);
   const float fx = (float)px + 0.5f, fy = (float)py + 0.5f;
   const uint32_t start = __ldg(ranges + 2 * tile), end = __ldg(ranges + 2 * tile + 1);
+  // the key of every instance of this tile's stretch of the sorted list is the tile id: stores that nothing here waits for
+  if (sorted_tiles)
+    for (uint32_t p = start + tid; p < end; p += kThreads) sorted_tiles[p] = (uint32_t)tile;
   const float in_x1 = px + 1 < cam.W ? 1.f : 0.f, in_y1 = py + 1 < cam.H ? 1.f : 0.f, in_0 = (px < cam.W && py < cam.H) ? 1.f : 0.f;
   // T is the transmittance while the pixel composites and 0 once it has stopped (then every later weight alpha T is
   // 0 by itself); the value it stopped with is kept in F.  Pixels outside the image start stopped.
@@ -479,9 +483,9 @@ int launch_blend_count(const CamDev &cam, const uint32_t *ranges, const uint32_t
 
 int launch_blend_fwd(const CamDev &cam, const uint32_t *ranges, const uint32_t *order, const uint32_t *vals,
                      const float *mean2d,
-                     const float *conic_opacity, const float *color, float *image, float *final_T,
+                     const float *conic_opacity, const float *color, uint32_t *sorted_tiles, float *image, float *final_T,
                      uint32_t *n_contrib, cudaStream_t st) {
-  k_blend_fwd<<<cam.gx * cam.gy, kThreads, 0, st>>>(cam, ranges, order, vals, mean2d, conic_opacity, color, image,
+  k_blend_fwd<<<cam.gx * cam.gy, kThreads, 0, st>>>(cam, ranges, order, vals, mean2d, conic_opacity, color, sorted_tiles, image,
                                                     final_T, n_contrib);
   return 1;
 }

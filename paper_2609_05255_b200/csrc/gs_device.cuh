@@ -137,14 +137,15 @@ int launch_emit_records(const uint32_t *depth_order, const uint32_t *cell_count,
 struct CellScratch { uint32_t *chunk_first, *chunk_counts, *chunk_bases, *tile_counts, *tile_starts; };
 int max_chunks(int64_t record_capacity, int num_cells);
 int launch_expand(const uint32_t *rec_keys, const uint32_t *rec_vals, const uint32_t *cell_ranges, const CellScratch &cs,
-                  int64_t record_capacity, int64_t pair_capacity, int gx, int gy, int cgx, int cgy, uint32_t *sorted_tiles,
+                  int64_t record_capacity, int64_t pair_capacity, int gx, int gy, int cgx, int cgy,
                   uint32_t *sorted_vals, uint32_t *tile_ranges, uint32_t *tile_order, cudaStream_t st);
 int launch_empty_binning(uint32_t *tile_ranges, uint32_t *tile_order, int num_tiles, cudaStream_t st);
 void launch_flag_if_greater(const unsigned long long *value, unsigned long long bound, uint32_t *flag, cudaStream_t st);
 
 // Blend.
+// (sorted_tiles: the tile id of every instance of the sorted list, written by the tile's CTA on its way in)
 int launch_blend_fwd(const CamDev &cam, const uint32_t *ranges, const uint32_t *order, const uint32_t *vals,
-                      const float *mean2d, const float *conic_opacity, const float *color,
+                      const float *mean2d, const float *conic_opacity, const float *color, uint32_t *sorted_tiles,
                       float *image, float *final_T, uint32_t *n_contrib, cudaStream_t st);
 int launch_blend_bwd(const CamDev &cam, const uint32_t *ranges, const uint32_t *order, const uint32_t *vals,
                       const float *mean2d, const float *conic_opacity, const float *color,

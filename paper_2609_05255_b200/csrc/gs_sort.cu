@@ -558,67 +558,56 @@ __global__ void __launch_bounds__(1024) k_tile_scan(const uint32_t *__restrict__
                                                     uint32_t *__restrict__ tile_starts, uint32_t *__restrict__ ranges,
                                                     uint32_t *__restrict__ order) {
   __shared__ uint32_t s_w[32];
-  __shared__ uint32_t s_carry;
   __shared__ uint32_t s_cnt[33], s_off[33];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (tid == 0) s_carry = 0;
   if (tid < 33) s_cnt[tid] = 0;
   __syncthreads();
-  for (int base = 0; base < num_tiles; base += 1024) {
-    const int t = base + tid;
-    const uint32_t v = t < num_tiles ? tile_counts[t] : 0u;
-    if (t < num_tiles) atomicAdd(&s_cnt[v ? 32 - __clz(v) : 0], 1u);
-    uint32_t inc = v;
+  // thread t takes the tiles [t per, (t + 1) per): one pass over its counts, one scan of the thread sums
+  const int per = (num_tiles + 1023) / 1024, first = tid * per, last = min(first + per, num_tiles);
+  uint32_t sum = 0;
+  for (int t = first; t < last; ++t) {
+    const uint32_t v = tile_counts[t];
+    sum += v;
+    atomicAdd(&s_cnt[v ? 32 - __clz(v) : 0], 1u);
+  }
+  uint32_t inc = sum;
+#pragma unroll
+  for (int s = 1; s < 32; s <<= 1) {
+    const uint32_t u = __shfl_up_sync(kFull, inc, s);
+    if (lane >= s) inc += u;
+  }
+  if (lane == 31) s_w[warp] = inc;
+  __syncthreads();
+  if (warp == 0) {
+    uint32_t w = s_w[lane], winc = w;
 #pragma unroll
     for (int s = 1; s < 32; s <<= 1) {
-      const uint32_t u = __shfl_up_sync(kFull, inc, s);
-      if (lane >= s) inc += u;
+      const uint32_t u = __shfl_up_sync(kFull, winc, s);
+      if (lane >= s) winc += u;
     }
-    if (lane == 31) s_w[warp] = inc;
-    __syncthreads();
-    if (warp == 0) {
-      uint32_t w = s_w[lane], winc = w;
-#pragma unroll
-      for (int s = 1; s < 32; s <<= 1) {
-        const uint32_t u = __shfl_up_sync(kFull, winc, s);
-        if (lane >= s) winc += u;
-      }
-      s_w[lane] = winc - w;
-    }
-    __syncthreads();
-    const uint32_t carry = s_carry;
-    if (t < num_tiles) {
-      const uint32_t start = carry + s_w[warp] + inc - v;
-      tile_starts[t] = start;
-      // a tile without instances: (0, 0); never past the capacity of the instance buffers (a device-side count may
-      // exceed it: the lists are then cut off and the host is told)
-      const uint32_t s0 = min(start, capacity), e0 = start + v < start ? capacity : min(start + v, capacity);
-      ranges[2 * t] = e0 > s0 ? s0 : 0u;
-      ranges[2 * t + 1] = e0 > s0 ? e0 : 0u;
-    }
-    __syncthreads();
-    if (tid == 1023) s_carry = carry + s_w[warp] + inc;
-    __syncthreads();
+    s_w[lane] = winc - w;
   }
   if (tid == 0) {
     uint32_t off = 0;
     for (int b = 32; b >= 0; --b) { s_off[b] = off; off += s_cnt[b]; }
   }
   __syncthreads();
-  for (int t = tid; t < num_tiles; t += 1024) {
-    const uint32_t len = tile_counts[t];
-    order[atomicAdd(&s_off[len ? 32 - __clz(len) : 0], 1u)] = (uint32_t)t;
+  uint32_t start = s_w[warp] + inc - sum;
+  for (int t = first; t < last; ++t) {
+    const uint32_t v = tile_counts[t];
+    tile_starts[t] = start;
+    // a tile without instances: (0, 0); never past the capacity of the instance buffers (a device-side count may
+    // exceed it: the lists are then cut off and the host is told)
+    const uint32_t s0 = min(start, capacity), e0 = start + v < start ? capacity : min(start + v, capacity);
+    ranges[2 * t] = e0 > s0 ? s0 : 0u;
+    ranges[2 * t + 1] = e0 > s0 ? e0 : 0u;
+    order[atomicAdd(&s_off[v ? 32 - __clz(v) : 0], 1u)] = (uint32_t)t;
+    start += v;
   }
 }
 
 __device__ __forceinline__ void store_if(bool p, uint32_t *addr, uint32_t v) {
   asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %0, 0;\n\t@q st.global.u32 [%1], %2;\n\t}" :: "r"((uint32_t)p), "l"(addr), "r"(v) : "memory");
-}
-
-// The tile id of every instance, from the ranges: one CTA per tile fills its stretch of the sorted list.
-__global__ void __launch_bounds__(128) k_fill_tile_ids(const uint32_t *__restrict__ ranges, uint32_t *__restrict__ out_tiles) {
-  const uint32_t t = blockIdx.x, b = __ldg(ranges + 2 * t), e = __ldg(ranges + 2 * t + 1);
-  for (uint32_t p = b + threadIdx.x; p < e; p += 128) out_tiles[p] = t;
 }
 
 // Per chunk: write its instances.  A warp's records are consecutive in depth order, 32 at a time.  A record's slot
@@ -785,7 +774,7 @@ int launch_emit_records(const uint32_t *depth_order, const uint32_t *cell_count,
 int max_chunks(int64_t record_capacity, int num_cells) { return (int)((record_capacity + kCellChunk - 1) / kCellChunk) + num_cells; }
 
 int launch_expand(const uint32_t *rec_keys, const uint32_t *rec_vals, const uint32_t *cell_ranges, const CellScratch &cs,
-                  int64_t record_capacity, int64_t pair_capacity, int gx, int gy, int cgx, int cgy, uint32_t *sorted_tiles,
+                  int64_t record_capacity, int64_t pair_capacity, int gx, int gy, int cgx, int cgy,
                   uint32_t *sorted_vals, uint32_t *tile_ranges, uint32_t *tile_order, cudaStream_t st) {
   const int num_cells = cgx * cgy, chunks = max_chunks(record_capacity, num_cells);
   const uint32_t cap = pair_capacity > 0xffffffffll ? 0xffffffffu : (uint32_t)pair_capacity;
@@ -795,8 +784,7 @@ int launch_expand(const uint32_t *rec_keys, const uint32_t *rec_vals, const uint
   k_tile_scan<<<1, 1024, 0, st>>>(cs.tile_counts, gx * gy, cap, cs.tile_starts, tile_ranges, tile_order);
   k_expand<<<chunks, kExpandThreads, 0, st>>>(rec_keys, rec_vals, cell_ranges, cs.chunk_first, num_cells, cs.chunk_bases, cs.tile_starts,
                                               gx, gy, cgx, cap, sorted_vals);
-  k_fill_tile_ids<<<gx * gy, 128, 0, st>>>(tile_ranges, sorted_tiles);
-  return 6;
+  return 5;
 }
 
 void launch_flag_if_greater(const unsigned long long *value, unsigned long long bound, uint32_t *flag, cudaStream_t st) {

@@ -36,8 +36,9 @@ def test_device_counted_view_equals_host_counted_view():
     assert torch.equal(a.binning.sorted_vals[:P], b.binning.sorted_vals[:P])
     for k in ("means", "log_scales", "quats", "opacity_logits", "base_color", "features"):
         x, y = getattr(a.grads, k), getattr(b.grads, k)
-        # the blend backward sums with atomics: equal up to the order of those sums
-        assert torch.allclose(x, y, rtol=1e-4, atol=1e-6), k
+        # the blend backward sums with atomics: equal up to the order of those sums.  Two runs of the SAME path differ
+        # by up to 3e-7 of the largest gradient of the kind (measured: 2.3e-5 on gradients of up to 87)
+        assert (x - y).abs().max().item() <= 2e-6 * x.abs().max().item(), k
     ctx.close()
 
 
