@@ -81,6 +81,11 @@ __device__ __forceinline__ float set_lt(float a, float b) {
   asm("set.lt.f32.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
   return d;
 }
+__device__ __forceinline__ float set_le(float a, float b) {
+  float d;
+  asm("set.le.f32.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+  return d;
+}
 __device__ __forceinline__ float2 sub2(float2 a, float2 b) { return __ffma2_rn(b, make_float2(-1.f, -1.f), a); }   // a - b, exact products
 
 // Forward.  The four pixels of a quad travel as two packed pairs, (0, 1) and (2, 3), and the composite of an entry is
@@ -316,26 +321,29 @@ __global__ void __launch_bounds__(kThreads, 16) k_blend_bwd(CamDev cam, const ui
     }
     __syncthreads();
     const int jtop = (int)min((uint32_t)cnt, wmax > first ? wmax - first : 0u);
-    // positions of this batch that each pixel composited: j < lim[k]
-    int lim[4];
+    // positions of this batch that each pixel composited: j < lim[k] (as numbers: the comparisons below make 0 / 1 masks)
+    float limf[4];
 #pragma unroll
-    for (int k = 0; k < 4; ++k) lim[k] = nc[k] > first ? (int)(nc[k] - first) : 0;
+    for (int k = 0; k < 4; ++k) limf[k] = nc[k] > first ? (float)min(nc[k] - first, (uint32_t)kBatchBwd) : 0.f;
+    float jf = (float)jtop;
     for (int j = jtop - 1; j >= 0; --j) {
       const float4 a = s_xyab[j];
       const float2 c = s_co[j];
       float p[4], t1[4], t2[2];
       quad_power(fx - a.x, fy - a.y, a.z, a.w, c.x, p, t1, t2);
       const float4 col = s_rgb[j];
-      const bool q0 = j < lim[0] && !(p[0] < col.w), q1 = j < lim[1] && !(p[1] < col.w);
-      const bool q2 = j < lim[2] && !(p[2] < col.w), q3 = j < lim[3] && !(p[3] < col.w);
-      if (!__any_sync(kFull, q0 | q1 | q2 | q3)) continue;
+      jf -= 1.f;
+      // q: the pixel composited this entry (it lies inside the pixel's walk and alpha >= 1/255), as 0 / 1
+      const float2 q01 = __fmul2_rn(make_float2(set_geu(p[0], col.w), set_geu(p[1], col.w)), make_float2(set_lt(jf, limf[0]), set_lt(jf, limf[1])));
+      const float2 q23 = __fmul2_rn(make_float2(set_geu(p[2], col.w), set_geu(p[3], col.w)), make_float2(set_lt(jf, limf[2]), set_lt(jf, limf[3])));
+      if (!__any_sync(kFull, (q01.x + q01.y) + (q23.x + q23.y) != 0.f)) continue;
       // Branch-free from here, two packed pixel pairs: a pixel that did not composite this entry enters with
       // alpha = 0, for which the reciprocal is 1, every product below is 0 and its carried state is unchanged.
       const float2 o2 = make_float2(c.y, c.y), one = make_float2(1.f, 1.f), mone = make_float2(-1.f, -1.f);
       const float2 raw01 = __fmul2_rn(o2, make_float2(ex2_approx(p[0]), ex2_approx(p[1])));
       const float2 raw23 = __fmul2_rn(o2, make_float2(ex2_approx(p[2]), ex2_approx(p[3])));
-      const float2 al01 = make_float2(q0 ? fminf(kAlphaMax, raw01.x) : 0.f, q1 ? fminf(kAlphaMax, raw01.y) : 0.f);
-      const float2 al23 = make_float2(q2 ? fminf(kAlphaMax, raw23.x) : 0.f, q3 ? fminf(kAlphaMax, raw23.y) : 0.f);
+      const float2 al01 = __fmul2_rn(q01, make_float2(fminf(kAlphaMax, raw01.x), fminf(kAlphaMax, raw01.y)));
+      const float2 al23 = __fmul2_rn(q23, make_float2(fminf(kAlphaMax, raw23.x), fminf(kAlphaMax, raw23.y)));
       const float2 d01 = __ffma2_rn(al01, mone, one), d23 = __ffma2_rn(al23, mone, one);
       const float2 inv01 = make_float2(rcp_approx(d01.x), rcp_approx(d01.y)), inv23 = make_float2(rcp_approx(d23.x), rcp_approx(d23.y));
       const float2 Tb01 = __fmul2_rn(T01, inv01), Tb23 = __fmul2_rn(T23, inv23);     // transmittance in front of this entry
@@ -351,10 +359,10 @@ __global__ void __launch_bounds__(kThreads, 16) k_blend_bwd(CamDev cam, const ui
       const float2 gc01 = __ffma2_rn(Gb01, cz, __ffma2_rn(Gg01, cy, __fmul2_rn(Gr01, cx)));
       const float2 gc23 = __ffma2_rn(Gb23, cz, __ffma2_rn(Gg23, cy, __fmul2_rn(Gr23, cx)));
       const float2 da01 = __fmul2_rn(__ffma2_rn(T01, gc01, nGS01), inv01), da23 = __fmul2_rn(__ffma2_rn(T23, gc23, nGS23), inv23);
-      const float2 e01 = __fmul2_rn(al01, da01), e23 = __fmul2_rn(al23, da23);
-      // clamped at 0.99: alpha does not depend on opacity and power there
-      const float dp0 = raw01.x <= kAlphaMax ? e01.x : 0.f, dp1 = raw01.y <= kAlphaMax ? e01.y : 0.f;
-      const float dp2 = raw23.x <= kAlphaMax ? e23.x : 0.f, dp3 = raw23.y <= kAlphaMax ? e23.y : 0.f;
+      // clamped at 0.99: alpha does not depend on opacity and power there (mask 0)
+      const float2 e01 = __fmul2_rn(__fmul2_rn(al01, da01), make_float2(set_le(raw01.x, kAlphaMax), set_le(raw01.y, kAlphaMax)));
+      const float2 e23 = __fmul2_rn(__fmul2_rn(al23, da23), make_float2(set_le(raw23.x, kAlphaMax), set_le(raw23.y, kAlphaMax)));
+      const float dp0 = e01.x, dp1 = e01.y, dp2 = e23.x, dp3 = e23.y;
       nGS01 = __ffma2_rn(make_float2(-w01.x, -w01.y), gc01, nGS01);
       nGS23 = __ffma2_rn(make_float2(-w23.x, -w23.y), gc23, nGS23);
       T01 = Tb01; T23 = Tb23;
