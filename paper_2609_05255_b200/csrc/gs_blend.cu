@@ -151,10 +151,13 @@ __global__ void __launch_bounds__(kThreads) k_blend_fwd(CamDev cam, const uint32
         const float2 al01 = __fmul2_rn(q01, make_float2(fminf(kAlphaMax, raw01.x), fminf(kAlphaMax, raw01.y)));
         const float2 al23 = __fmul2_rn(q23, make_float2(fminf(kAlphaMax, raw23.x), fminf(kAlphaMax, raw23.y)));
         float2 w01 = __fmul2_rn(al01, T01), w23 = __fmul2_rn(al23, T23);
-        // transmittance behind this entry, T - alpha T; below 1e-4 the pixel stops and the entry is not composited.
+        // transmittance behind this entry, T (1 - alpha) - in this form, because the backward recovers the
+        // transmittances by dividing (1 - alpha) out again and drifts if the forward rounds another expression (ten
+        // 2D-gradient values of a 1M-Gaussian view were then off by more than 1e-3 of the sum of their terms); below
+        // 1e-4 the pixel stops and the entry is not composited.
         // A live pixel that skips the entry keeps T >= 1e-4 and cannot stop here; a stopped one has T = 0 and
         // "stops" again with nothing to lose.
-        const float2 n01 = sub2(T01, w01), n23 = sub2(T23, w23);
+        const float2 n01 = __fmul2_rn(T01, sub2(one, al01)), n23 = __fmul2_rn(T23, sub2(one, al23));
         const float2 s01 = make_float2(set_lt(n01.x, kTmin), set_lt(n01.y, kTmin));
         const float2 s23 = make_float2(set_lt(n23.x, kTmin), set_lt(n23.y, kTmin));
         const float2 k01 = sub2(one, s01), k23 = sub2(one, s23);
