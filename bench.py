@@ -271,7 +271,7 @@ def run_ours(args):
             clocks = sampler.stop()
         # units of the blend kernels: list entries up to each pixel's last composited one, over the views
         entries = 0
-        visible = 0
+        visible = records = 0
         evaluated = composited = warp_steps = warp_steps_idle = 0
         for v in range(views):
             r.forward(ds, cams[v])
@@ -281,6 +281,7 @@ def run_ours(args):
             evaluated += ev; composited += co; warp_steps += ws_; warp_steps_idle += wi
             rect = r.proj.rect.to(torch.int32) & 0xFFFF
             visible += int(((rect[:, 2] > rect[:, 0]) & (rect[:, 3] > rect[:, 1])).sum().item())
+            records += int((r.proj.cell_count.to(torch.int64) & 0x7FFFFFFF).sum().item())
         # the same step through the unfused reference path (App. D "Fusion"): appearance as passes of its own
         unfused = None
         if args.config == 3 and not args.skip_decode:
@@ -303,7 +304,7 @@ def run_ours(args):
                             "split ones; colours within 2e-3 of the oracle instead of 2e-5 (tests/test_gpu_half_precision.py)"}
         results[tag] = dict(ms=ms, ms_one=ms_one, ms_streams=ms_streams, graph=graph_note, unfused=unfused, half=half,
                             stage_ms=stage_ms, stage_launches=stage_launches, pairs=pairs,
-                            entries=entries, visible=visible, evaluated=evaluated, composited=composited,
+                            entries=entries, visible=visible, records=records, evaluated=evaluated, composited=composited,
                             warp_steps=warp_steps, warp_steps_idle=warp_steps_idle,
                             host=host, ds=ds, r=r, app=tag)
 
@@ -329,6 +330,21 @@ def run_ours(args):
     clock_mhz = peaks["sm_max_mhz"]
     alu_peak = NUM_SMS * FP32_LANES_PER_SM * 2 * clock_mhz * 1e6 / 1e12   # TFLOP/s
     roof = stage_roofline(dominant, neural, views, n, peaks, alu_peak)
+    # which run the fraction refers to: the stage times come from the single-stream pass, not from `value`
+    roof["ms_per_step_single_stream"] = neural["ms_one"]
+    roof["stage_sum_ms_per_step_single_stream"] = total_stage
+    roof["stage_ms_per_step_single_stream"] = stage_ms[dominant]
+    roof["launches_of_the_stage_per_step"] = views
+    roof["note"] = ("achieved = algorithmic work of one launch / (stage_ms_per_step_single_stream / launches); `value` is the "
+                    "same step with several views in flight on streams of their own, where stages overlap")
+    if e2e is not None:
+        e2e["what"] = ("e2e = a training iteration: " + e2e["what"] + ".  e2e_gradients_to_host = the other reading, every "
+                       "input from the host and every output to it: scene parameters and upstream gradients start in pinned host "
+                       "memory each step, the image and all per-Gaussian gradients of every view end there")
+    if e2e_host is not None:
+        e2e_host["what"] = ("scene parameters and upstream gradients start in pinned host memory each step; the image and all "
+                            "per-Gaussian gradient buffers of every view end there (no optimiser step); the other reading of "
+                            "'end to end' beside `e2e`")
     out = {
         "metric": METRIC, "value": replicas.job_ms_per_iteration(ms, 1, world), "unit": f"ms/iter ({views} views, fwd+bwd)", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": False,
@@ -344,8 +360,8 @@ def run_ours(args):
         "clocks": clocks, "e2e": e2e, "e2e_gradients_to_host": e2e_host, "gpu_launches": launches_per_step,
         "roofline": roof,
         "rooflines": {k: stage_roofline(k, neural, views, n, peaks, alu_peak)
-                      for k in ("preprocess_fwd", "depth_sort", "keygen", "tile_sort", "blend_fwd", "blend_bwd",
-                                "preprocess_bwd") if stage_ms.get(k, 0) > 0},
+                      for k in ("preprocess_fwd", "depth_sort", "keygen", "tile_sort", "tile_ranges", "blend_fwd",
+                                "blend_bwd", "preprocess_bwd") if stage_ms.get(k, 0) > 0},
         "stages_ms_per_step": {k: round(v, 4) for k, v in stage_ms.items() if v > 0},
         "stage_share": {k: round(v / total_stage, 4) for k, v in stage_ms.items() if v > 0},
         "pairs_per_view": neural["pairs"], "visible_per_view": neural["visible"] / views,
@@ -370,25 +386,45 @@ def run_ours(args):
     print(json.dumps(out))
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of ONE launch (orbit view 0 of the default workload), from the
-# ncu --set full captures summarised under profiles/.  Bytes.
-NCU_TRAFFIC_1M_NEURAL = {"blend_bwd": 47.37e6, "blend_fwd": 25.73e6, "preprocess_bwd": 180.64e6,
-                         "preprocess_fwd": 89.63e6}
+# Figures read from ncu captures of single launches (orbit view 0 of the default workload) live in
+# profiles/ncu_constants.json, each with the command that produced it and the commit it was taken at:
+#   dram_bytes    dram__bytes_read.sum + dram__bytes_write.sum of the launch
+#   issue_active  smsp__issue_active.avg.pct_of_peak_sustained_active / 100: the share of issue slots the kernel
+#                 fills while it runs.  For the ALU-bound blend kernels this, not the flop rate, says how close to
+#                 the machine they are: the flop count is the method's minimum arithmetic, the issue slots also
+#                 carry loads, predicates, shuffles and loop control.
+def ncu_constants():
+    path = os.path.join(ROOT, "profiles", "ncu_constants.json")
+    if not os.path.exists(path):
+        return None
+    return json.load(open(path))
 
 
-# smsp__issue_active.avg.pct_of_peak_sustained_active of the same captures: the share of issue slots the kernel
-# fills while it runs.  For the ALU-bound blend kernels this, not the flop rate, says how close to the machine they
-# are: the flop count above is the method's minimum arithmetic, the issue slots also carry loads, predicates,
-# shuffles and loop control.
-NCU_ISSUE_ACTIVE_1M_NEURAL = {"blend_bwd": 0.81, "blend_fwd": 0.70, "preprocess_bwd": 0.53, "preprocess_fwd": 0.72,
-                              "keygen": 0.57}
+# Names of the timed stages (the C ABI's stage enumeration) and the kernels behind them.
+STAGE_KERNELS = {
+    "preprocess_fwd": "k_preprocess_fwd (projection, fused appearance, cell records of 4x4 tiles)",
+    "depth_sort": "4 x (k_radix_hist, k_radix_scan_rows, k_radix_scatter<8>) on the 32-bit depth keys of all Gaussians",
+    "keygen": "k_emit_records: (cell id, 16-bit tile mask) records in depth order",
+    "tile_sort": "k_radix_hist, k_radix_scan_rows, k_radix_scatter<9>: one stable pass on the cell id",
+    "tile_ranges": "k_cell_chunks, k_chunk_counts, k_cell_prefix, k_tile_scan, k_expand: records -> per-tile lists",
+    "blend_fwd": "k_blend_fwd", "blend_bwd": "k_blend_bwd",
+    "preprocess_bwd": "k_preprocess_bwd (+ k_wgrad_reduce for the decoder weights)"}
 
 
 def stage_roofline(stage, arm, views, n, peaks, alu_peak):
     out = _stage_roofline(stage, arm, views, n, peaks, alu_peak)
-    if n == 1_000_000 and arm.get("app") == "neural":
-        out["traffic"] = NCU_TRAFFIC_1M_NEURAL.get(stage)
-        out["issue_active_frac_ncu"] = NCU_ISSUE_ACTIVE_1M_NEURAL.get(stage)
+    out["kernels"] = STAGE_KERNELS.get(stage)
+    out["ms_per_launch"] = arm["stage_ms"][stage] / views
+    out["timed_as"] = "single stream, views one after another (CUDA events around the stage's launches)"
+    out["traffic_source"] = None
+    consts = ncu_constants()
+    if consts and n == consts.get("n") and arm.get("app") == consts.get("appearance"):
+        e = consts["entries"].get(stage)
+        if e:
+            out["traffic"] = e.get("dram_bytes")
+            out["issue_active_frac_ncu"] = e.get("issue_active")
+            out["traffic_source"] = (f"profiles/ncu_constants.json: {e.get('kernel')} ({e.get('launch')}), "
+                                     f"captured at commit {consts.get('commit')}")
     return out
 
 
@@ -407,15 +443,19 @@ def _stage_roofline(stage, arm, views, n, peaks, alu_peak):
                 "evaluated_per_launch": ev, "composited_per_launch": co,
                 "flops_per_evaluated": BLEND_FLOPS_PER_EVALUATED, "flops_per_composited": per_c}
     vis = arm["visible"] / views
+    P = sum(arm["pairs"]) / views                # (Gaussian, tile) instances of a view
+    R = arm["records"] / views                   # (Gaussian, cell of 4 x 4 tiles) records of a view
     app_bytes = 28.0
-    per_launch = {"preprocess_fwd": 44.0 * n + 12.0 * n + (app_bytes + 48.0) * vis,
+    per_launch = {"preprocess_fwd": 44.0 * n + 12.0 * n + (app_bytes + 48.0) * vis + 4.0 * R,
                   "preprocess_bwd": 8.0 * n + (44.0 + 48.0 + app_bytes) * vis + 88.0 * n,
-                  "depth_sort": (4 * 20.0 - 4.0) * n,
-                  "tile_sort": 2 * 20.0 * (sum(arm["pairs"]) / views),
-                  "keygen": 12.0 * n + 8.0 * (sum(arm["pairs"]) / views)}.get(stage, 0.0)
+                  "depth_sort": (4 * 20.0 - 4.0) * n,     # per pass: keys read twice, values once, both written
+                  "keygen": 8.0 * n + 12.0 * R,           # id + count per Gaussian; record read, key + value written
+                  "tile_sort": 20.0 * R,                  # one pass: keys read twice, values once, both written
+                  "tile_ranges": 12.0 * R + 4.0 * P}.get(stage, 0.0)   # keys twice + values read, ids written
     achieved = per_launch / (ms * 1e-3) / 1e9
     return {"kernel": stage, "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-            "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"]}
+            "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+            "algorithmic_bytes_per_launch": per_launch, "visible": vis, "instances": P, "records": R}
 
 
 def measure_e2e(api, torch, ctx, arm, cams, G, views, args, timed, dev):
@@ -580,7 +620,8 @@ def measure_e2e_training(api, torch, lane_ctx, lanes, arm, cams, G, views, args,
 def sort_reference(torch, arm, cams, views, dev):
     """Context for the ordering stages: the library's stable sort of one view's instance list as 64-bit
     (tile, depth bits) keys with the Gaussian ids as values - the one-key formulation - timed as a library
-    call beside this library's two-stage ordering (depth sort of the Gaussians + tile sort of the instances)."""
+    call beside this library's ordering (depth sort of the Gaussians, then records per cell of 4 x 4 tiles sorted by
+    cell and expanded into the per-tile lists)."""
     r = arm["r"]
     r.forward(arm["ds"], cams[0])      # view 0's lists, with the host-side count
     torch.cuda.synchronize()
@@ -603,10 +644,12 @@ def sort_reference(torch, arm, cams, views, dev):
         if i >= 3:
             ts.append(e0.elapsed_time(e1))
     ts.sort()
-    ours = (arm["stage_ms"]["depth_sort"] + arm["stage_ms"]["tile_sort"]) / views
+    ours = sum(arm["stage_ms"][k] for k in ("depth_sort", "keygen", "tile_sort", "tile_ranges")) / views
     return {"instances": P, "library_sort_64bit_keys_ms": round(ts[len(ts) // 2], 4),
-            "two_stage_ordering_ms_per_view": round(ours, 4),
-            "what": "torch.sort(stable) of (tile << 32 | depth bits) keys + gather of the ids, against depth_sort + tile_sort of one view"}
+            "this_library_ordering_ms_per_view": round(ours, 4),
+            "what": "torch.sort(stable) of (tile << 32 | depth bits) keys + gather of the ids (the one-key formulation, keys already "
+                    "emitted), against this library's whole ordering of one view: depth sort of the Gaussians, record emission, "
+                    "record sort by cell and expansion into the per-tile lists"}
 
 
 def adam_sweep(api, torch, ctx, dev, peaks, n):

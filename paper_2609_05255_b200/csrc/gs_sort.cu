@@ -1,4 +1,4 @@
-// Ordering and binning: a stable LSD radix sort (digits of up to 8 bits, keys staged and ranked in shared
+// Ordering and binning: a stable LSD radix sort (digits of 4 to 11 bits, keys staged and ranked in shared
 // memory, no inter-block waiting) and the kernels that turn its output into per-tile lists.
 //
 // (1) The Gaussians are sorted once by their 32-bit depth key (ties keep the index order: the sort is stable).
@@ -23,21 +23,34 @@ constexpr unsigned kFull = 0xffffffffu;
 constexpr int kMaxDigitBits = 11;  // widest radix digit: 2048 bins
 constexpr int kScanBlock = 256;   // Gaussians per block of the tiles-touched prefix sum and per CTA of the instance emission
 
-// Block b sorts consecutive tiles of kSortTile elements: the tiles are dealt out as evenly as whole tiles allow over
-// the grid, which is one full wave of CTAs at most.  The grid is sized by the host's bound on the count; the ranges
-// follow the count the kernels see (which may live on the device), so the work stays balanced either way.
+// Block b sorts one contiguous range of the input; the ranges are equal (rounded up to a multiple of the block size),
+// so a full wave of CTAs shares the work evenly whatever the count.  A range is worked through in tiles of at most
+// kSortTile elements, all of one length (a multiple of the block size again: every warp of the CTA then ranks the
+// same number of items).  The grid is sized by the host's bound on the count; the ranges follow the count the
+// kernels see (which may live on the device), so the work stays balanced either way.
+constexpr int kMinPerBlock = 2048;
 int sort_blocks(int64_t count) {
-  const int64_t tiles = (count + kSortTile - 1) / kSortTile;
-  return (int)(tiles < 1 ? 1 : tiles < kMaxSortBlocks ? tiles : kMaxSortBlocks);
+  const int64_t b = (count + kMinPerBlock - 1) / kMinPerBlock;
+  return (int)(b < 1 ? 1 : b < kMaxSortBlocks ? b : kMaxSortBlocks);
 }
 
-// First tile and number of tiles of this block.
-__device__ __forceinline__ void block_tiles(int64_t count, int64_t &first, int &num) {
-  const int64_t tiles = (count + kSortTile - 1) / kSortTile;
-  const int b = (int)blockIdx.x, nb = (int)gridDim.x;
-  const int tiles_per_block = (int)(tiles / nb), extra = (int)(tiles - (int64_t)tiles_per_block * nb);
-  first = (int64_t)b * tiles_per_block + min(b, extra);
-  num = tiles_per_block + (b < extra ? 1 : 0);
+struct BlockRange {
+  int64_t begin, end;   // this block's elements
+  int tiles, tile_len;  // worked through as `tiles` pieces of `tile_len` (the last one may be short)
+};
+
+__device__ __forceinline__ BlockRange block_range(int64_t count) {
+  const int64_t nb = (int64_t)gridDim.x;
+  int64_t per = (count + nb - 1) / nb;
+  per = (per + kSortThreads - 1) / kSortThreads * kSortThreads;
+  BlockRange r;
+  r.begin = min(count, (int64_t)blockIdx.x * per);
+  r.end = min(count, r.begin + per);
+  const int len = (int)(r.end - r.begin);
+  r.tiles = (len + kSortTile - 1) / kSortTile;
+  const int t = r.tiles > 0 ? (len + r.tiles - 1) / r.tiles : 0;
+  r.tile_len = (t + kSortThreads - 1) / kSortThreads * kSortThreads;
+  return r;
 }
 
 // Digit histogram of each block's contiguous range: table[digit][block] (digits of up to kMaxDigitBits bits).
@@ -63,14 +76,9 @@ __global__ void __launch_bounds__(kSortThreads) k_radix_hist(const uint32_t *__r
   const uint32_t mask = (uint32_t)nb - 1u;
   for (int k = tid; k < copies * nb; k += kSortThreads) s_hist[k] = 0;
   __syncthreads();
-  int64_t first_tile;
-  int my_tiles;
-  block_tiles(count, first_tile, my_tiles);
-  const int64_t begin = first_tile * kSortTile;
-  int64_t end = begin + (int64_t)my_tiles * kSortTile;
-  if (end > count) end = count;
+  const BlockRange r = block_range(count);
   uint32_t *mine = s_hist + (warp % copies) * nb;
-  for (int64_t i = begin + tid; i < end; i += kSortThreads) atomicAdd(mine + ((__ldg(keys + i) >> shift) & mask), 1u);
+  for (int64_t i = r.begin + tid; i < r.end; i += kSortThreads) atomicAdd(mine + ((__ldg(keys + i) >> shift) & mask), 1u);
   __syncthreads();
   for (int d = tid; d < nb; d += kSortThreads) {
     uint32_t t = 0;
@@ -178,14 +186,13 @@ __global__ void __launch_bounds__(kSortThreads, BITS <= 9 ? 3 : 2) k_radix_scatt
     }
   }
 
-  int64_t first_tile;
-  int my_tiles;
-  block_tiles(count, first_tile, my_tiles);
-  const int64_t begin = first_tile * kSortTile;
-  for (int t = 0; t < my_tiles; ++t) {
-    const int64_t tile_begin = begin + (int64_t)t * kSortTile;
-    if (tile_begin >= count) break;
-    const int valid_count = (int)min((int64_t)kSortTile, count - tile_begin);
+  const BlockRange r = block_range(count);
+  const int span = r.tile_len / kSortWarps;           // consecutive elements of a tile that one warp ranks
+  const int items = span / 32;                        // ... as this many rows of 32 (at most kItems)
+  for (int t = 0; t < r.tiles; ++t) {
+    const int64_t tile_begin = r.begin + (int64_t)t * r.tile_len;
+    if (tile_begin >= r.end) break;
+    const int valid_count = (int)min((int64_t)r.tile_len, r.end - tile_begin);
     for (int k = tid; k < kSortWarps * NB; k += kSortThreads) s_warp_cnt[k] = 0;
     __syncthreads();
     uint32_t key[kItems], val[kItems];
@@ -193,15 +200,16 @@ __global__ void __launch_bounds__(kSortThreads, BITS <= 9 ? 3 : 2) k_radix_scatt
     // all loads first (independent, in flight together), then the serial ranking chain
 #pragma unroll
     for (int it = 0; it < kItems; ++it) {
-      const int local = warp * (32 * kItems) + it * 32 + lane;
-      const bool ok = local < valid_count;
+      const int local = warp * span + it * 32 + lane;
+      const bool ok = it < items && local < valid_count;
       const int64_t idx = tile_begin + local;
       key[it] = ok ? __ldg(keys_in + idx) : 0xffffffffu;
       val[it] = ok ? (vals_in ? __ldg(vals_in + idx) : (uint32_t)idx) : 0u;
     }
 #pragma unroll
     for (int it = 0; it < kItems; ++it) {
-      const int local = warp * (32 * kItems) + it * 32 + lane;
+      if (it >= items) break;                         // the same for every thread of the CTA
+      const int local = warp * span + it * 32 + lane;
       const bool ok = local < valid_count;
       const uint32_t d = ok ? ((key[it] >> shift) & kDigitMask) : kDigitMask;
       // lanes with the same digit form a group; its first lane bumps the warp's counter once and
@@ -243,7 +251,8 @@ __global__ void __launch_bounds__(kSortThreads, BITS <= 9 ? 3 : 2) k_radix_scatt
     __syncthreads();
 #pragma unroll
     for (int it = 0; it < kItems; ++it) {
-      const int local = warp * (32 * kItems) + it * 32 + lane;
+      if (it >= items) break;
+      const int local = warp * span + it * 32 + lane;
       const uint32_t d = (local < valid_count) ? ((key[it] >> shift) & kDigitMask) : kDigitMask;
       const uint32_t pos = s_digit_start[d] + s_warp_cnt[warp * NB + d] + rank[it];
       s_keys[pos] = key[it];

@@ -26,7 +26,7 @@ MODELS = {"sh": (scenes.APP_SH, 0), "sv": (scenes.APP_SV, 0), "neural_split": (s
 # |pre-activation| per Gaussian): every row outside the literal rule must be one of them, and the decoder-weight
 # gradient is compared in a second run in which those rows receive a zero upstream gradient on both sides, so that
 # it is a sum over rows whose decisions agree.
-KINK_MARGIN = 2.5e-7      # twice the largest margin measured on a row that did differ (1.2e-7, at 10M Gaussians)
+KINK_MARGIN = 2.5e-7      # 1.5 times the largest margin measured on a row that did differ (1.7e-7, at 1M Gaussians)
 
 
 def _decode(app, precision, n, zero_rows=None):
