@@ -23,11 +23,13 @@ constexpr unsigned kFull = 0xffffffffu;
 constexpr int kMaxDigitBits = 11;  // widest radix digit: 2048 bins
 constexpr int kScanBlock = 256;   // Gaussians per block of the tiles-touched prefix sum and per CTA of the instance emission
 
-// Block b sorts one contiguous range of the input; the ranges are equal (rounded up to a multiple of the block size),
-// so a full wave of CTAs shares the work evenly whatever the count.  A range is worked through in tiles of at most
-// kSortTile elements, all of one length (a multiple of the block size again: every warp of the CTA then ranks the
-// same number of items).  The grid is sized by the host's bound on the count; the ranges follow the count the
-// kernels see (which may live on the device), so the work stays balanced either way.
+// Block b sorts one contiguous range of the input, worked through in tiles of at most kSortTile elements.  While one
+// tile per block is enough (count <= blocks x kSortTile) the ranges are equal, rounded up to a multiple of the block
+// size, so that a full wave of CTAs shares the work evenly and every warp of a CTA ranks the same number of items.
+// Beyond that, whole tiles are dealt out as evenly as they go: a pass costs a fixed latency per tile, and two full
+// tiles in a few blocks measured faster than two half tiles in every block (0.40 against 0.45 ms per 8 views on
+// 2 M records).  The grid is sized by the host's bound on the count; the ranges follow the count the kernels see
+// (which may live on the device), so the work stays balanced either way.
 constexpr int kMinPerBlock = 2048;
 int sort_blocks(int64_t count) {
   const int64_t b = (count + kMinPerBlock - 1) / kMinPerBlock;
@@ -41,15 +43,23 @@ struct BlockRange {
 
 __device__ __forceinline__ BlockRange block_range(int64_t count) {
   const int64_t nb = (int64_t)gridDim.x;
-  int64_t per = (count + nb - 1) / nb;
-  per = (per + kSortThreads - 1) / kSortThreads * kSortThreads;
   BlockRange r;
-  r.begin = min(count, (int64_t)blockIdx.x * per);
-  r.end = min(count, r.begin + per);
-  const int len = (int)(r.end - r.begin);
-  r.tiles = (len + kSortTile - 1) / kSortTile;
-  const int t = r.tiles > 0 ? (len + r.tiles - 1) / r.tiles : 0;
-  r.tile_len = (t + kSortThreads - 1) / kSortThreads * kSortThreads;
+  if (count <= nb * kSortTile) {
+    int64_t per = (count + nb - 1) / nb;
+    per = (per + kSortThreads - 1) / kSortThreads * kSortThreads;
+    r.begin = min(count, (int64_t)blockIdx.x * per);
+    r.end = min(count, r.begin + per);
+    r.tiles = r.end > r.begin ? 1 : 0;
+    r.tile_len = (int)per;
+  } else {
+    const int64_t tiles = (count + kSortTile - 1) / kSortTile;
+    const int b = (int)blockIdx.x;
+    const int each = (int)(tiles / nb), extra = (int)(tiles - (int64_t)each * nb);
+    r.tiles = each + (b < extra ? 1 : 0);
+    r.begin = ((int64_t)b * each + min(b, extra)) * kSortTile;
+    r.end = min(count, r.begin + (int64_t)r.tiles * kSortTile);
+    r.tile_len = kSortTile;
+  }
   return r;
 }
 
