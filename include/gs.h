@@ -365,6 +365,16 @@ typedef enum {
   GS_NUM_STAGES
 } GsStage;
 GsStatus gs_profile_enable(GsContext *ctx, int enable);
+/* Which kernel evaluates the default decoder (Eq. 5-7) in the separate-pass forward of this context
+ * (gs_appearance_forward, and the appearance pass of gs_preprocess when GsScene.separate_pass is set).
+ * GS_ENGINE_WARP_MMA (the default): warp-level mma.sync tiles, 32 Gaussians per warp.
+ * GS_ENGINE_TCGEN05: tcgen05.mma with the accumulators in tensor memory, 128 Gaussians per CTA, one
+ * operand row and one lane of tensor memory per thread.  Same arithmetic (fp16 operands, split or plain,
+ * fp32 accumulation) and the same tolerances; the two were measured within a few percent of each other,
+ * which is why this is a switch and not a replacement.  The paper has no counterpart of this call.
+ * Returns GS_ERR_INVALID_ARG for any other value.  Takes effect for the calls issued after it. */
+typedef enum GsDecoderEngine { GS_ENGINE_WARP_MMA = 0, GS_ENGINE_TCGEN05 = 1 } GsDecoderEngine;
+GsStatus gs_set_decoder_engine(GsContext *ctx, int engine);
 /* Measurement only: for the view last rendered into (proj, bin), count over all pixels the list
  * entries the blend evaluates (until each pixel stops) and the pairs it composites; these are the
  * work units of the blend kernels' roofline.  counts_host is a host array of FOUR values: entries

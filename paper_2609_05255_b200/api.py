@@ -97,6 +97,8 @@ _lib.gs_profile_collect.argtypes = [_vp, C.POINTER(C.c_double), C.POINTER(C.c_in
 _lib.gs_profile_collect.restype = C.c_int
 
 
+_lib.gs_set_decoder_engine.argtypes = [_vp, C.c_int]
+_lib.gs_set_decoder_engine.restype = C.c_int
 _lib.gs_profile_blend_counts.argtypes = [_vp, C.POINTER(GsProjected), C.POINTER(GsBinning), C.POINTER(GsCamera),
                                          C.POINTER(C.c_int64), _vp]
 _lib.gs_profile_blend_counts.restype = C.c_int
@@ -341,6 +343,13 @@ def gs_profile_collect(ctx: Context):
     launches = (C.c_int64 * len(STAGES))()
     ctx._check(_lib.gs_profile_collect(ctx._h, ms, launches))
     return dict(zip(STAGES, list(ms))), dict(zip(STAGES, list(launches)))
+
+
+GS_ENGINE_WARP_MMA, GS_ENGINE_TCGEN05 = 0, 1
+
+
+def gs_set_decoder_engine(ctx: Context, engine: int):
+    ctx._check(_lib.gs_set_decoder_engine(ctx._h, int(engine)))
 
 
 def gs_profile_blend_counts(ctx: Context, proj: "Projected", binning: "Binning", cam: GsCamera, stream=None):

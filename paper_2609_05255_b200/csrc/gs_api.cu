@@ -24,6 +24,7 @@ struct GsContext {
   float *d_w_partials;                // device: per-CTA partial sums of the decoder gradient ([kWgradBlocks, 816];
                                       // sized for the decoder variants' largest case as well)
   char error[256];
+  int decoder_engine;                 // GsDecoderEngine of the separate-pass forward
   bool profiling;
   std::vector<StageRecord> records;   // stage timings since the last collect
   std::vector<cudaEvent_t> free_events;
@@ -124,6 +125,7 @@ AppearanceArgs appearance_args(GsContext *ctx, const GsScene *scene) {
   AppearanceArgs a;
   memset(&a, 0, sizeof(a));
   a.timeout = ctx->d_counter + 3;
+  a.engine = ctx->decoder_engine;
   a.n = scene->n; a.deg = scene->active_degree; a.act = scene->color_activation;
   a.base_color = scene->base_color; a.sh_rest = scene->app == GS_APP_SV ? scene->sv_sites : scene->sh_rest;
   a.features = reinterpret_cast<const __half *>(scene->features);
@@ -264,6 +266,7 @@ GsStatus gs_create(int device, GsContext **out) {
   ctx->error[0] = 0;
   ctx->d_counter = nullptr; ctx->h_counter = nullptr; ctx->d_w_partials = nullptr;
   ctx->profiling = false;
+  ctx->decoder_engine = GS_ENGINE_WARP_MMA;
   if (cudaMalloc(&ctx->d_counter, 8 * sizeof(unsigned long long)) != cudaSuccess ||
       cudaMemset(ctx->d_counter, 0, 8 * sizeof(unsigned long long)) != cudaSuccess ||
       cudaMallocHost(&ctx->h_counter, 8 * sizeof(unsigned long long)) != cudaSuccess ||
@@ -674,6 +677,13 @@ GsStatus gs_neural_prepass(GsContext *ctx, const GsScene *scene, const uint16_t 
 GsStatus gs_profile_enable(GsContext *ctx, int enable) {
   if (!ctx) return GS_ERR_INVALID_ARG;
   ctx->profiling = enable != 0;
+  return GS_OK;
+}
+
+GsStatus gs_set_decoder_engine(GsContext *ctx, int engine) {
+  if (!ctx) return GS_ERR_INVALID_ARG;
+  if (engine != GS_ENGINE_WARP_MMA && engine != GS_ENGINE_TCGEN05) return fail(ctx, GS_ERR_INVALID_ARG, "unknown decoder engine");
+  ctx->decoder_engine = engine;
   return GS_OK;
 }
 

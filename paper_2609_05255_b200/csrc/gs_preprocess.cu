@@ -951,6 +951,8 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_bwd(PreprocessBwdArgs a, 
 }
 
 // ---- separate-pass appearance kernels of the neural model (the explicit models follow, with bulk copies) ------
+#include "gs_decoder_tc.cuh"
+
 template <int APP>
 __global__ void __launch_bounds__(kBlock) k_appearance_fwd(AppearanceArgs a) {
   static_assert(IsNeural<APP>::value, "the neural model in either decoder precision");
@@ -1244,11 +1246,31 @@ int launch_bulk(const AppearanceArgs &a, cudaStream_t st) {
   return 1;
 }
 
+// Grid of the tcgen05 kernel: tc::kCtasPerSm CTAs per SM.  The occupancy query answers 1 for this kernel, so the
+// count is set here.
+static int tc_wave() {
+  int dev = 0, sms = 0;
+  cudaGetDevice(&dev);
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
+  return tc::kCtasPerSm * sms;
+}
+
 int launch_appearance_fwd(int app, const AppearanceArgs &a, cudaStream_t st) {
   if (a.n == 0) return 0;
   if (app == GS_APP_SH) return launch_bulk<GS_APP_SH, false>(a, st);
   if (app == GS_APP_SV) return launch_bulk<GS_APP_SV, false>(a, st);
   const int chunks = grid_for(a.n);
+  if (a.deg > 0 && a.engine == GS_ENGINE_TCGEN05) {   // the tensor-memory path (tiles of 128 Gaussians = kBlock)
+    constexpr size_t smem = sizeof(tc::Smem);
+    if (app == kAppNeuralHalf) {
+      const int wave = tc_wave();
+      tc::k_appearance_fwd_tc<false><<<chunks < wave ? chunks : wave, kBlock, smem, st>>>(a);
+    } else {
+      const int wave = tc_wave();
+      tc::k_appearance_fwd_tc<true><<<chunks < wave ? chunks : wave, kBlock, smem, st>>>(a);
+    }
+    return 1;
+  }
   if (app == kAppNeuralHalf) {
     const int wave = resident_blocks<k_appearance_fwd<kAppNeuralHalf>>(0, 1 << 20);
     k_appearance_fwd<kAppNeuralHalf><<<chunks < wave ? chunks : wave, kBlock, 0, st>>>(a);

@@ -75,11 +75,13 @@ def _conic_from_cholesky(lo):
     return np.stack([lo[:, 0] ** 2, lo[:, 0] * lo[:, 1], lo[:, 1] ** 2 + lo[:, 2] ** 2, lo[:, 3]], 1)
 
 
-def run_gpu(scene, cam, G=None, pair_capacity=None, with_extent=True, device=0):
+def run_gpu(scene, cam, G=None, pair_capacity=None, with_extent=True, device=0, decoder_engine=None):
     """One view through gs_preprocess / gs_render_forward / gs_render_backward.  Returns numpy copies."""
     import torch
     from paper_2609_05255_b200 import api
     ctx = api.Context(device)
+    if decoder_engine is not None:
+        api.gs_set_decoder_engine(ctx, decoder_engine)
     dev = ctx.device
     ds = api.upload_scene(scene, dev)
     ccam = api.make_camera(cam)
