@@ -269,8 +269,9 @@ GsStatus gs_appearance_backward(GsContext *ctx, const GsScene *scene, const floa
  * GS_ERR_CAPACITY and a message, nothing launched.  Arguments and results are those of
  * gs_appearance_backward (device pointers on the CURRENT device, 16-byte aligned), including
  * scene->color_activation and scene->decoder_precision (GS_DECODER_HALF runs the same unsplit kernel
- * as there; an unknown value of either is GS_ERR_INVALID_ARG); per-Gaussian results are
- * bit-identical to it, grads->mlp_weights is the same sum taken in a different order.  error_text
+ * as there; an unknown value of either is GS_ERR_INVALID_ARG); it always runs the warp-level MMA
+ * kernel: per-Gaussian results are bit-identical to gs_appearance_backward under
+ * GS_ENGINE_WARP_MMA, grads->mlp_weights is the same sum taken in a different order.  error_text
  * (host, may be NULL) receives a description when the status is not GS_OK.
  *
  * The first call on each device looks up the device address of the array; make that call before any
@@ -365,15 +366,20 @@ typedef enum {
   GS_NUM_STAGES
 } GsStage;
 GsStatus gs_profile_enable(GsContext *ctx, int enable);
-/* Which kernel evaluates the default decoder (Eq. 5-7) in the separate-pass forward of this context
- * (gs_appearance_forward, and the appearance pass of gs_preprocess when GsScene.separate_pass is set).
- * GS_ENGINE_WARP_MMA (the default): warp-level mma.sync tiles, 32 Gaussians per warp.
+/* Which kernels evaluate the default decoder (Eq. 5-7) in the separate pass of this context
+ * (gs_appearance_forward / gs_appearance_backward, and the appearance passes of gs_preprocess and
+ * gs_render_backward when GsScene.separate_pass is set).
+ * GS_ENGINE_WARP_MMA: warp-level mma.sync tiles, 32 Gaussians per warp.
  * GS_ENGINE_TCGEN05: tcgen05.mma with the accumulators in tensor memory, 128 Gaussians per CTA, one
- * operand row and one lane of tensor memory per thread.  Same arithmetic (fp16 operands, split or plain,
- * fp32 accumulation) and the same tolerances; the two were measured within a few percent of each other,
- * which is why this is a switch and not a replacement.  The paper has no counterpart of this call.
- * Returns GS_ERR_INVALID_ARG for any other value.  Takes effect for the calls issued after it. */
-typedef enum GsDecoderEngine { GS_ENGINE_WARP_MMA = 0, GS_ENGINE_TCGEN05 = 1 } GsDecoderEngine;
+ * operand row and one lane of tensor memory per thread; in the backward the weight gradients are
+ * products over the 128 Gaussians of a tile, accumulated in tensor memory across the CTA's tiles.
+ * GS_ENGINE_AUTO (the default): per kernel, whichever measured faster on a B200 - the backward with
+ * split operands on tcgen05, the forward and the plain-fp16 backward on warp-level MMA.
+ * Same arithmetic (fp16 operands, split or plain, fp32 accumulation) and the same tolerances either
+ * way; per-Gaussian results differ only by the order of the fp32 sums.  The paper has no counterpart
+ * of this call.  Returns GS_ERR_INVALID_ARG for any other value.  Takes effect for the calls issued
+ * after it. */
+typedef enum GsDecoderEngine { GS_ENGINE_WARP_MMA = 0, GS_ENGINE_TCGEN05 = 1, GS_ENGINE_AUTO = 2 } GsDecoderEngine;
 GsStatus gs_set_decoder_engine(GsContext *ctx, int engine);
 /* Measurement only: for the view last rendered into (proj, bin), count over all pixels the list
  * entries the blend evaluates (until each pixel stops) and the pairs it composites; these are the

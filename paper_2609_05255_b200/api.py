@@ -345,7 +345,7 @@ def gs_profile_collect(ctx: Context):
     return dict(zip(STAGES, list(ms))), dict(zip(STAGES, list(launches)))
 
 
-GS_ENGINE_WARP_MMA, GS_ENGINE_TCGEN05 = 0, 1
+GS_ENGINE_WARP_MMA, GS_ENGINE_TCGEN05, GS_ENGINE_AUTO = 0, 1, 2
 
 
 def gs_set_decoder_engine(ctx: Context, engine: int):

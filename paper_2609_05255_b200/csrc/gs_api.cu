@@ -266,7 +266,7 @@ GsStatus gs_create(int device, GsContext **out) {
   ctx->error[0] = 0;
   ctx->d_counter = nullptr; ctx->h_counter = nullptr; ctx->d_w_partials = nullptr;
   ctx->profiling = false;
-  ctx->decoder_engine = GS_ENGINE_WARP_MMA;
+  ctx->decoder_engine = GS_ENGINE_AUTO;
   if (cudaMalloc(&ctx->d_counter, 8 * sizeof(unsigned long long)) != cudaSuccess ||
       cudaMemset(ctx->d_counter, 0, 8 * sizeof(unsigned long long)) != cudaSuccess ||
       cudaMallocHost(&ctx->h_counter, 8 * sizeof(unsigned long long)) != cudaSuccess ||
@@ -682,7 +682,7 @@ GsStatus gs_profile_enable(GsContext *ctx, int enable) {
 
 GsStatus gs_set_decoder_engine(GsContext *ctx, int engine) {
   if (!ctx) return GS_ERR_INVALID_ARG;
-  if (engine != GS_ENGINE_WARP_MMA && engine != GS_ENGINE_TCGEN05) return fail(ctx, GS_ERR_INVALID_ARG, "unknown decoder engine");
+  if (engine != GS_ENGINE_WARP_MMA && engine != GS_ENGINE_TCGEN05 && engine != GS_ENGINE_AUTO) return fail(ctx, GS_ERR_INVALID_ARG, "unknown decoder engine");
   ctx->decoder_engine = engine;
   return GS_OK;
 }

@@ -81,7 +81,7 @@ struct AppearanceArgs {
   float *g_base, *g_sh_rest, *g_features, *g_dirs;
   float *w_partials, *g_weights;
   unsigned long long *timeout; // optional: set to 1 if a bounded wait on a bulk copy ran out (never expected)
-  int engine;                  // forward of the default neural decoder: 0 warp-level MMA, 1 tcgen05 (tensor memory)
+  int engine;                  // GsDecoderEngine for the default neural decoder: warp-level MMA, tcgen05, or per kernel the faster
   const uint32_t *mask;        // optional [n]: Gaussians with a zero here are skipped (no colour written; zero
                                // gradient rows written); the tiles-touched array in the unfused step
 };

@@ -29,7 +29,7 @@ MODELS = {"sh": (scenes.APP_SH, 0), "sv": (scenes.APP_SV, 0), "neural_split": (s
 KINK_MARGIN = 2.5e-7      # 1.5 times the largest margin measured on a row that did differ (1.7e-7, at 1M Gaussians)
 
 
-def _decode(app, precision, n, zero_rows=None):
+def _decode(app, precision, n, zero_rows=None, engine=None):
     import torch
     from paper_2609_05255_b200 import api
     sc, dirs, gcol = scenes.config5(n, app)
@@ -37,6 +37,8 @@ def _decode(app, precision, n, zero_rows=None):
     if zero_rows is not None:
         gcol[zero_rows] = 0
     ctx = api.Context(0)
+    if engine is not None:                    # None: the library's default, which picks per kernel
+        api.gs_set_decoder_engine(ctx, engine)
     ds = api.upload_scene(sc, ctx.device)
     d = torch.from_numpy(dirs).to(ctx.device); gc = torch.from_numpy(gcol).to(ctx.device)
     color = torch.full((n, 3), float("nan"), device=ctx.device)
@@ -65,12 +67,12 @@ def _decode(app, precision, n, zero_rows=None):
 # kink rows are taken out, and their largest error relative to the largest weight gradient.
 
 
-def _check(oracle, model, n):
+def _check(oracle, model, n, engine=None):
     app, precision = MODELS[model]
-    sc, dirs, gcol, got = _decode(app, precision, n)
+    sc, dirs, gcol, got = _decode(app, precision, n, engine=engine)
     ref_c, _ = oracle.appearance_forward(sc, dirs)
     ref = oracle.appearance_backward(sc, dirs, gcol)
-    case = f"decode_{model}_{n}"
+    case = f"decode_{model}_{n}" + {None: "", 0: "_warp_mma", 1: "_tcgen05"}[engine]
     err_c = float(np.abs(got["color"] - ref_c).max())
     assert np.all(np.isfinite(got["color"]))
     if precision == 1:
@@ -93,7 +95,7 @@ def _check(oracle, model, n):
     worst = float(margin[off].max()) if off.any() else 0.0
     assert MEASURE or not (off & ~kink).any(), f"{(off & ~kink).sum()} rows off whose ReLU decisions are clear (margin up to {worst:.2e})"
     # the weight gradient over the rows whose decisions agree
-    sc2, dirs2, gcol2, got2 = _decode(app, precision, n, zero_rows=kink)
+    sc2, dirs2, gcol2, got2 = _decode(app, precision, n, zero_rows=kink, engine=engine)
     ref2 = oracle.appearance_backward(sc2, dirs2, gcol2)
     w_got, w_ref = got2["mlp_weights"].astype(np.float64), ref2.mlp_weights
     w_off = int(grad_mismatch(w_got, w_ref).sum())
@@ -113,6 +115,13 @@ def _check(oracle, model, n):
 @pytest.mark.parametrize("model", list(MODELS))
 def test_decode_at_the_sweep_sizes(oracle, model, n):
     _check(oracle, model, n)
+
+
+# The default engine runs the split-operand backward on tcgen05; the warp-level kernel (the one the fused preprocess
+# backward shares its decoder code with) stays checked at size too.
+@pytest.mark.parametrize("n", [444 * 128 * 2 + 1, 1_000_000, 10_000_000])
+def test_decode_at_size_on_the_warp_level_kernels(oracle, n):
+    _check(oracle, "neural_split", n, engine=0)
 
 
 # 592 and 444 CTAs are the persistent grids of these kernels on a 148-SM part (4 and 3 resident CTAs per SM), 128

@@ -1,4 +1,4 @@
-"""The separate-pass forward of the default decoder (Eq. 5-7) on tcgen05.mma with the accumulators in tensor memory
+"""The separate-pass forward and backward of the default decoder (Eq. 5-7) on tcgen05.mma with the accumulators in tensor memory
 (gs_set_decoder_engine(ctx, GS_ENGINE_TCGEN05)) against the oracle, element by element: split operands within the
 2e-5 of the default kernel, plain fp16 operands within their own stated bound; sizes that give every persistent CTA
 (8 per SM on 148 SMs, 128 Gaussians per tile) a second and a third tile and a ragged last one, the sweep's sizes up
@@ -12,6 +12,7 @@ from paper_2609_05255_b200 import scenes
 from conftest import record_parity
 from gpu_helpers import run_gpu
 from test_gpu_half_precision import COLOR_ATOL as HALF_COLOR_ATOL
+from test_gpu_decode_at_size import _check as check_decode
 
 pytestmark = pytest.mark.gpu
 
@@ -107,3 +108,20 @@ def test_tcgen05_engine_in_the_unfused_step(oracle):
     assert np.abs(got.image - fused.image).max() < 1e-5
     both = vis & (ref.tiles_touched > 0)
     assert np.abs(got.color[both] - ref.color[both]).max() < 2e-5
+
+
+# The backward on the same engine (recompute, data gradients, and the weight gradients as products over the 128
+# Gaussians of a tile accumulated in tensor memory), held to the rules of the warp-level kernel's test: per-Gaussian
+# gradients by the literal rule except rows at a ReLU kink that the oracle names, weight gradients over the other rows.
+# 3 CTAs per SM x 148 SMs x 128 Gaussians = one trip of the backward's persistent grid.
+WAVE_BWD = 3 * 148 * 128
+
+
+@pytest.mark.parametrize("n", [1, 129, 4_099, WAVE_BWD + 1, 2 * WAVE_BWD + 127, 1_000_000, 3_000_000, 10_000_000])
+def test_tcgen05_backward_split_operands(oracle, n):
+    check_decode(oracle, "neural_split", n, engine=1)
+
+
+@pytest.mark.parametrize("n", [4_099, 2 * WAVE_BWD + 127, 1_000_000])
+def test_tcgen05_backward_plain_fp16_operands(oracle, n):
+    check_decode(oracle, "neural_half", n, engine=1)

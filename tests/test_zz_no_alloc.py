@@ -33,6 +33,7 @@ def test_noalloc_matches_the_allocating_entry_point_twice_in_a_row():
     import torch
     from paper_2609_05255_b200 import api
     ctx = api.Context(0)                       # only the existing entry point needs a context
+    api.gs_set_decoder_engine(ctx, api.GS_ENGINE_WARP_MMA)   # the kernel the allocation-free entry point runs
     dev = ctx.device
     # second call smaller than the first: rows of the shared scratch left over from call 1 must not leak
     for n, seed in ((70_001, 1), (9_000, 2)):
@@ -104,6 +105,7 @@ def test_noalloc_honours_the_decoder_precision_and_the_colour_activation():
     import torch
     from paper_2609_05255_b200 import api
     ctx = api.Context(0)
+    api.gs_set_decoder_engine(ctx, api.GS_ENGINE_WARP_MMA)
     dev = ctx.device
     n = 33_333
     ds, dirs, gcol = _inputs(n, 4, dev)
