@@ -787,10 +787,12 @@ def decode_sweep(api, torch, ctx, dev, peaks, args):
                 "fwd_GBps": round(bytes_fwd * n / (f_ms * 1e-3) / 1e9, 1),
                 "bwd_GBps": round(bytes_bwd * n / (b_ms * 1e-3) / 1e9, 1),
                 "Gprimitives_per_s": round(n / ((f_ms + b_ms) * 1e-3) / 1e9, 3)}
-              if app == 1:      # the same forward on tcgen05.mma with the accumulators in tensor memory
-                api.gs_set_decoder_engine(ctx, api.GS_ENGINE_TCGEN05)
-                out[row]["fwd_ms_tcgen05"] = round(run(lambda: api.gs_appearance_forward(ctx, sc, dirs, color)), 4)
-                api.gs_set_decoder_engine(ctx, api.GS_ENGINE_WARP_MMA)
+              if app == 1:      # the row above is the default engine (per kernel the faster); both engines on their own
+                for eng, name in ((api.GS_ENGINE_WARP_MMA, "warp_mma"), (api.GS_ENGINE_TCGEN05, "tcgen05")):
+                    api.gs_set_decoder_engine(ctx, eng)
+                    out[row]["fwd_ms_" + name] = round(run(lambda: api.gs_appearance_forward(ctx, sc, dirs, color)), 4)
+                    out[row]["bwd_ms_" + name] = round(run(lambda: api.gs_appearance_backward(ctx, sc, dirs, gcol, grads, gd)), 4)
+                api.gs_set_decoder_engine(ctx, api.GS_ENGINE_AUTO)
             del sc, color, grads, gd, flush
         # the decoder variants of the architecture table (App. D), fp32 CUDA-core kernels: 1M only
         for hidden, layers, nfeat in (((16, 1, 8), (16, 3, 8), (32, 2, 8), (16, 2, 16)) if n == 1_000_000 else ()):
