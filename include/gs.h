@@ -374,7 +374,8 @@ GsStatus gs_profile_enable(GsContext *ctx, int enable);
  * operand row and one lane of tensor memory per thread; in the backward the weight gradients are
  * products over the 128 Gaussians of a tile, accumulated in tensor memory across the CTA's tiles.
  * GS_ENGINE_AUTO (the default): per kernel, whichever measured faster on a B200 - the backward with
- * split operands on tcgen05, the forward and the plain-fp16 backward on warp-level MMA.
+ * split operands and, from 2,000,000 Gaussians on, the forward on tcgen05; smaller forwards and the
+ * plain-fp16 backward on warp-level MMA.
  * Same arithmetic (fp16 operands, split or plain, fp32 accumulation) and the same tolerances either
  * way; per-Gaussian results differ only by the order of the fp32 sums.  The paper has no counterpart
  * of this call.  Returns GS_ERR_INVALID_ARG for any other value.  Takes effect for the calls issued

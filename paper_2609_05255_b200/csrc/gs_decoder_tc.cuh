@@ -56,7 +56,7 @@ __device__ __forceinline__ bool wait_phase(uint32_t bar, uint32_t parity) {
     asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
                  : "=r"(done) : "r"(bar), "r"(parity) : "memory");
     if (done) return true;
-    __nanosleep(40);
+    __nanosleep(20);
   }
   return false;
 }
@@ -124,13 +124,27 @@ __device__ __forceinline__ void store_chunk(unsigned char *hi, unsigned char *lo
   if (kSplit) *reinterpret_cast<uint4 *>(lo + offset) = l;
 }
 
+// The output layer (3 x 16 products per Gaussian) in registers, on the fp32 activations: cheaper than a phase of its
+// own (operand rows, barrier, MMA round trip, read-back).  w3f = W3 as floats, [3][16].
+__device__ __forceinline__ void output_layer(const float *w3f, const float h[16], float y[3]) {
+  y[0] = y[1] = y[2] = 0.f;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const float4 r0 = *reinterpret_cast<const float4 *>(w3f + 4 * q), r1 = *reinterpret_cast<const float4 *>(w3f + 16 + 4 * q),
+                 r2 = *reinterpret_cast<const float4 *>(w3f + 32 + 4 * q);
+    y[0] = fmaf(h[4 * q], r0.x, fmaf(h[4 * q + 1], r0.y, fmaf(h[4 * q + 2], r0.z, fmaf(h[4 * q + 3], r0.w, y[0]))));
+    y[1] = fmaf(h[4 * q], r1.x, fmaf(h[4 * q + 1], r1.y, fmaf(h[4 * q + 2], r1.z, fmaf(h[4 * q + 3], r1.w, y[1]))));
+    y[2] = fmaf(h[4 * q], r2.x, fmaf(h[4 * q + 1], r2.y, fmaf(h[4 * q + 2], r2.z, fmaf(h[4 * q + 3], r2.w, y[2]))));
+  }
+}
+
 struct __align__(128) Smem {
   // A operand, high and low halves: 4 K chunks x 128 rows x 16 B for the first layer; the later layers (2 chunks)
   // write over it - their rows are written after the MMAs that read the previous contents have completed
   unsigned char a1[2][4 * kTile * 16];
   unsigned char w1[4 * 16 * 16];         // W1 [16][32] as B operand: 4 K chunks x 16 rows x 16 B
   unsigned char w2[2 * 16 * 16];         // W2 [16][16]
-  unsigned char w3[2 * 16 * 16];         // W3 [3][16], rows 3..15 zero
+  float w3f[3 * 16];                     // W3 as floats: the output layer runs in registers
   unsigned long long bar;
   uint32_t tmem_base;
   uint32_t failed;
@@ -149,8 +163,8 @@ __global__ void __launch_bounds__(kTile) k_appearance_fwd_tc(AppearanceArgs a) {
   for (int idx = tid; idx < 16 * 16; idx += kTile) {
     const int n = idx >> 4, k = idx & 15;
     *reinterpret_cast<__half *>(S.w2 + elem_offset(16, n, k)) = a.weights[512 + idx];
-    *reinterpret_cast<__half *>(S.w3 + elem_offset(16, n, k)) = n < 3 ? a.weights[768 + idx] : __float2half(0.f);
   }
+  for (int idx = tid; idx < 3 * 16; idx += kTile) S.w3f[idx] = __half2float(a.weights[768 + idx]);
   const uint32_t bar = bulk::smem_addr(&S.bar);
   if (tid == 0) {
     bulk::barrier_init(bar);
@@ -168,7 +182,7 @@ __global__ void __launch_bounds__(kTile) k_appearance_fwd_tc(AppearanceArgs a) {
   const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(&S.tmem_base);
   const uint32_t my_lane = tmem + ((uint32_t)(warp * 32) << 16);   // this warp's 32 lanes (bits 16..31 of the address)
   const uint32_t A1[2] = {bulk::smem_addr(S.a1[0]), bulk::smem_addr(S.a1[1])};
-  const uint32_t W1 = bulk::smem_addr(S.w1), W2 = bulk::smem_addr(S.w2), W3 = bulk::smem_addr(S.w3);
+  const uint32_t W1 = bulk::smem_addr(S.w1), W2 = bulk::smem_addr(S.w2);
   constexpr int kParts = kSplit ? 2 : 1;
   uint32_t phase = 0;
 
@@ -229,11 +243,8 @@ __global__ void __launch_bounds__(kTile) k_appearance_fwd_tc(AppearanceArgs a) {
     load16(my_lane + 16u, h);
 #pragma unroll
     for (int k = 0; k < 16; ++k) h[k] = fmaxf(h[k], 0.f);
-#pragma unroll
-    for (int c = 0; c < 2; ++c) store_chunk<kSplit>(S.a1[0], S.a1[1], (uint32_t)c * chunk_bytes(kTile) + (uint32_t)tid * 16u, h + 8 * c);
-    run_layer(A1, W3, 1, 0u);
-    float y[4];
-    load4(my_lane + 0u, y);
+    float y[3];
+    output_layer(S.w3f, h, y);
     if (in)
       store3(a.color, i, color_act_z(a.act, base[0] + 0.5f + tanh_fast(y[0])), color_act_z(a.act, base[1] + 0.5f + tanh_fast(y[1])),
              color_act_z(a.act, base[2] + 0.5f + tanh_fast(y[2])));
@@ -245,8 +256,8 @@ __global__ void __launch_bounds__(kTile) k_appearance_fwd_tc(AppearanceArgs a) {
 
 // ---- backward ----------------------------------------------------------------------------------------------------
 // Per tile of 128 Gaussians, thread t = row t throughout:
-//   P1-P3  the forward again (activations are recomputed, not stored): X -> h1 -> h2 -> y, every layer's operand rows
-//          staying in shared memory because the weight gradients need them;
+//   P1-P2  the forward again (activations are recomputed, not stored): X -> h1 -> h2, every layer's operand rows
+//          staying in shared memory because the weight gradients need them; the output layer y = W3 h2 in registers;
 //   gy = dL/dy through the activation and the tanh; delta2 = (gy W3) relu'(h2) in registers (3 x 16 products);
 //   P4     delta1_pre = delta2 W2 (B operand: W2 transposed); delta1 = delta1_pre relu'(h1);
 //   P5     gx = delta1 W1 (B operand: W1 transposed, N = 32), and in the same batch the three weight gradients as
@@ -272,7 +283,7 @@ struct __align__(128) SmemBwd {
   unsigned char d2[2][2 * kTile * 16];   // delta2
   unsigned char d1[2][2 * kTile * 16];   // delta1
   unsigned char gy[2][1 * kTile * 16];   // dL/dy, 3 of 8 columns used
-  unsigned char w1[4 * 16 * 16], w2[2 * 16 * 16], w3[2 * 16 * 16];   // B operands of the forward
+  unsigned char w1[4 * 16 * 16], w2[2 * 16 * 16];   // B operands of the forward's two hidden layers
   unsigned char w2t[2 * 16 * 16];        // B[n = i][k = j] = W2[j][i]
   unsigned char w1t[2 * 32 * 16];        // B[n = k][kk = i] = W1[i][k], N = 32
   float w3f[3 * 16];                     // W3 as floats for the 3 x 16 products in registers
@@ -297,7 +308,6 @@ __global__ void __launch_bounds__(kTile) k_appearance_bwd_tc(AppearanceArgs a) {
     const __half w = a.weights[512 + idx];
     *reinterpret_cast<__half *>(S.w2 + elem_offset(16, j, i)) = w;
     *reinterpret_cast<__half *>(S.w2t + elem_offset(16, i, j)) = w;
-    *reinterpret_cast<__half *>(S.w3 + elem_offset(16, j, i)) = j < 3 ? a.weights[768 + idx] : __float2half(0.f);
   }
   for (int idx = tid; idx < 3 * 16; idx += kTile) S.w3f[idx] = __half2float(a.weights[768 + idx]);
   // the low-half buffers are read as rows of the M = 64 operands even when nothing is written there: start them at zero
@@ -320,7 +330,7 @@ __global__ void __launch_bounds__(kTile) k_appearance_bwd_tc(AppearanceArgs a) {
   const uint32_t my_lane = tmem + ((uint32_t)(warp * 32) << 16);
   const uint32_t X = bulk::smem_addr(S.x[0]), H1 = bulk::smem_addr(S.h1[0]), H2 = bulk::smem_addr(S.h2[0]);
   const uint32_t D2 = bulk::smem_addr(S.d2[0]), D1 = bulk::smem_addr(S.d1[0]), GY = bulk::smem_addr(S.gy[0]);
-  const uint32_t W1 = bulk::smem_addr(S.w1), W2 = bulk::smem_addr(S.w2), W3 = bulk::smem_addr(S.w3);
+  const uint32_t W1 = bulk::smem_addr(S.w1), W2 = bulk::smem_addr(S.w2);
   const uint32_t W2T = bulk::smem_addr(S.w2t), W1T = bulk::smem_addr(S.w1t);
   constexpr int kParts = kSplit ? 2 : 1;
   constexpr uint32_t kChunk = chunk_bytes(kTile);          // 2048
@@ -403,11 +413,10 @@ __global__ void __launch_bounds__(kTile) k_appearance_bwd_tc(AppearanceArgs a) {
     for (int k = 0; k < 16; ++k) { m2 |= (h[k] > 0.f ? 1u : 0u) << k; h[k] = fmaxf(h[k], 0.f); }
 #pragma unroll
     for (int c = 0; c < 2; ++c) store_chunk<kSplit>(S.h2[0], S.h2[1], (uint32_t)c * kChunk + (uint32_t)tid * 16u, h + 8 * c);
-    run_phase([&] { rows_times(H2, 2u * kChunk, W3, 16, 1, kF1, idesc(128, 16)); });
     float gp[3], gy[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
     {
-      float y[4];
-      load4(my_lane + kF1, y);
+      float y[3];
+      output_layer(S.w3f, h, y);
 #pragma unroll
       for (int c = 0; c < 3; ++c) {
         const float A = tanh_fast(y[c]);

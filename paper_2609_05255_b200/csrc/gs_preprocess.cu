@@ -1260,7 +1260,10 @@ int launch_appearance_fwd(int app, const AppearanceArgs &a, cudaStream_t st) {
   if (app == GS_APP_SH) return launch_bulk<GS_APP_SH, false>(a, st);
   if (app == GS_APP_SV) return launch_bulk<GS_APP_SV, false>(a, st);
   const int chunks = grid_for(a.n);
-  if (a.deg > 0 && a.engine == GS_ENGINE_TCGEN05) {   // the tensor-memory path (tiles of 128 Gaussians = kBlock)
+  // the tensor-memory path (tiles of 128 Gaussians = kBlock): on request, and by default from 2M Gaussians on, where it
+  // measured 4-8 % faster than the warp-level kernel (at 1M it is 6-14 % slower: seven tiles per CTA do not pay for
+  // staging the weights and allocating tensor memory)
+  if (a.deg > 0 && (a.engine == GS_ENGINE_TCGEN05 || (a.engine == GS_ENGINE_AUTO && a.n >= 2000000))) {
     constexpr size_t smem = sizeof(tc::Smem);
     if (app == kAppNeuralHalf) {
       const int wave = tc_wave();
@@ -1289,8 +1292,8 @@ int launch_appearance_bwd(int app, const AppearanceArgs &a, cudaStream_t st) {
     if (a.n == 0) return 0;
     return launch_bulk<GS_APP_SV, true>(a, st);
   } else {
-    // the tensor-memory path: on request, and by default for split operands (measured 12-17 % faster than the
-    // warp-level kernel from 1M to 10M Gaussians; with plain fp16 operands it is 11 % slower)
+    // the tensor-memory path: on request, and by default for split operands (measured 16-21 % faster than the
+    // warp-level kernel from 1M to 10M Gaussians; with plain fp16 operands it is 6-9 % slower)
     if ((a.engine == GS_ENGINE_TCGEN05 || (a.engine == GS_ENGINE_AUTO && app != kAppNeuralHalf)) && a.deg > 0 && a.n > 0) {
       constexpr size_t smem = sizeof(tc::SmemBwd);
       int dev = 0, sms = 0;
