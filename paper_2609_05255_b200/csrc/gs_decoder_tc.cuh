@@ -1,13 +1,15 @@
-// The decoder (Eq. 5-7) of the separate-pass forward on the 5th-generation tensor cores: tcgen05.mma with the
-// accumulators in tensor memory.  Included by gs_preprocess.cu after the helpers it uses (decoder_inputs,
-// load_features, tanh_fast, the bounded mbarrier wait of namespace bulk).
+// The decoder (Eq. 5-7) of the separate pass, forward and backward, on the 5th-generation tensor cores: tcgen05.mma
+// with the accumulators in tensor memory.  Included by gs_preprocess.cu after the helpers it uses (decoder_inputs,
+// load_features, tanh_fast, the mbarrier helpers of namespace bulk).
 //
 // One CTA of 128 threads works on tiles of 128 Gaussians: thread t owns row t of every operand and lane t of the
-// tensor memory.  Per tile and layer the threads write their rows of the A operand (activations, fp16, a high and
-// - with split operands - a low half) into shared memory in the canonical K-major layout without swizzle, one
+// tensor memory.  Per tile and hidden layer the threads write their rows of the A operand (activations, fp16, a high
+// and - with split operands - a low half) into shared memory in the canonical K-major layout without swizzle, one
 // thread issues the MMAs against the layer's weights (B operand, staged once per CTA) into a 128 x 16 fp32
 // accumulator, commits them to an mbarrier, and every thread reads its accumulator row back with tcgen05.ld for
-// the ReLU and the next layer.  A thread never needs another thread's values: no fragment shuffling at all.
+// the ReLU and the next layer; the 3 x 16 output layer runs in registers.  A thread never needs another thread's
+// values: no fragment shuffling at all.  The backward (further down) adds the transposed products and takes the
+// weight gradients as products over the tile's rows, accumulated in tensor memory.
 //
 // Single-GPU code: no cluster, no multicast of any kind.  Every wait on the mbarrier is bounded; a wait that runs
 // out sets *timeout (read by gs_async_status), the CTA stops issuing MMAs, runs its loops to the end without
@@ -79,7 +81,7 @@ __device__ __forceinline__ void mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b
 __device__ __forceinline__ void commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-// This thread's lane of the accumulator: 16 (or 4) consecutive fp32 columns, complete when the call returns.
+// This thread's lane of the accumulator: 16 consecutive fp32 columns, complete when the call returns.
 __device__ __forceinline__ void load16(uint32_t taddr, float v[16]) {
   uint32_t r[16];
   asm volatile(
@@ -92,18 +94,6 @@ __device__ __forceinline__ void load16(uint32_t taddr, float v[16]) {
 #pragma unroll
   for (int k = 0; k < 16; ++k) v[k] = __uint_as_float(r[k]);
 }
-__device__ __forceinline__ void load4(uint32_t taddr, float v[4]) {
-  uint32_t r[4];
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0, %1, %2, %3}, [%4];\n\t"
-      "tcgen05.wait::ld.sync.aligned;"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-      : "r"(taddr)
-      : "memory");
-#pragma unroll
-  for (int k = 0; k < 4; ++k) v[k] = __uint_as_float(r[k]);
-}
-
 // Eight consecutive values of this thread's operand row as one 16-byte chunk of halves: the high halves, and the
 // halves of what the rounding left (the products then carry about 22 bits).
 template <bool kSplit>
