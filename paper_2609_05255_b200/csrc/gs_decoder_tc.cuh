@@ -26,7 +26,6 @@ constexpr int kCtasPerSm = 8;   // what 63 registers x 128 threads allow; 8 x 32
 __host__ __device__ constexpr uint32_t idesc(int m, int n, bool a_mn = false, bool b_mn = false) {
   return (1u << 4) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
-constexpr uint32_t kIdesc = idesc(128, 16);
 
 // Canonical K-major operand without swizzle: core matrices of 8 rows x 16 bytes (8 halves), stored as 128
 // contiguous bytes; the core matrices of consecutive 8-row groups lie 128 B apart (stride byte offset), those of
@@ -35,20 +34,12 @@ __device__ __forceinline__ constexpr uint32_t chunk_bytes(int rows) { return (ui
 __device__ __forceinline__ constexpr uint32_t elem_offset(int rows, int r, int k) {
   return (uint32_t)(k >> 3) * chunk_bytes(rows) + (uint32_t)r * 16u + (uint32_t)(k & 7) * 2u;
 }
-// Shared-memory matrix descriptor: start address, leading and stride byte offsets in units of 16 B, descriptor
-// version 1 (bits 46-47), base offset 0, no swizzle (bits 61-63 = 0).
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, int rows) {
-  return (uint64_t)((addr >> 4) & 0x3fffu) | ((uint64_t)((chunk_bytes(rows) >> 4) & 0x3fffu) << 16) |
-         ((uint64_t)(128u >> 4) << 32) | (1ull << 46);
-}
-
-// The same buffer read the other way round (MN-major): the 128 rows are the K dimension (8 rows of 16 B form a
-// core matrix, consecutive groups of 8 rows 128 B apart: leading byte offset) and the 16-byte chunks of a row are 8
-// consecutive elements of M or N, further chunks `chunk_stride` bytes apart (stride byte offset).
-__device__ __forceinline__ uint64_t smem_desc_mn(uint32_t addr, uint32_t chunk_stride) {
-  return (uint64_t)((addr >> 4) & 0x3fffu) | ((uint64_t)(128u >> 4) << 16) | ((uint64_t)((chunk_stride >> 4) & 0x3fffu) << 32) | (1ull << 46);
-}
-
+// Shared-memory matrix descriptor (64 bits): start address (bits 0-13), leading byte offset (16-29) and stride byte
+// offset (32-45), all in units of 16 B; descriptor version 1 (bits 46-47); base offset 0; no swizzle (bits 61-63 = 0).
+// K-major operand of R rows: leading byte offset = R * 16 (next 8-element K chunk), stride byte offset = 128 (next
+// group of 8 rows).  The same buffer read MN-major (the rows are the K dimension, the 16-byte chunks of a row are 8
+// consecutive elements of M or N): leading byte offset = 128 (next group of 8 rows of K), stride byte offset = the
+// distance of the chunks (next 8 elements of M or N).
 // Bounded wait for a phase of the MMAs' mbarrier: the MMAs of a phase complete within a microsecond, so the threads
 // poll, with a short pause between polls that leaves the issue slots to the CTAs that have work; 2^22 polls (about a
 // second) is the bound after which the caller gives up and reports.
@@ -66,11 +57,34 @@ __device__ __forceinline__ bool wait_phase(uint32_t bar, uint32_t parity) {
 // The inputs of this thread's row in the tile after the next barrier-bound stretch: asked into L2 ahead of time.
 __device__ __forceinline__ void prefetch_l2(const void *p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
+__device__ __forceinline__ void mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t accumulate, uint32_t desc);
+
+// The issuing thread's fast path: with the buffer's address field (address >> 4) computed once, a descriptor `off`
+// bytes into the buffer is one add (the low word) and an immediate (the high word).  Shared-memory addresses stay
+// below 2^18, so the address field never carries into the offset fields.
+template <uint32_t kLboBytes, uint32_t kSboBytes>
+__device__ __forceinline__ uint64_t desc_at(uint32_t base4, uint32_t off_bytes) {
+  const uint32_t lo = base4 + ((off_bytes >> 4) | ((kLboBytes >> 4) << 16));
+  constexpr uint32_t hi = (kSboBytes >> 4) | (1u << 14);
+  return ((uint64_t)hi << 32) | lo;
+}
+// D (128 x n) = or += A * B^T for a K-major A of the tile's rows (kSteps x 16 columns per part, kParts parts
+// kPartStride bytes apart) and a K-major B of kBRows rows; a4 / b4 are the buffers' address fields.
+template <int kParts, int kSteps, int kBRows, uint32_t kPartStride>
+__device__ __forceinline__ void rows_times(uint32_t d_tmem, uint32_t a4, uint32_t b4, uint32_t desc) {
+#pragma unroll
+  for (int p = 0; p < kParts; ++p)
+#pragma unroll
+    for (int ks = 0; ks < kSteps; ++ks)
+      mma(d_tmem, desc_at<chunk_bytes(kTile), 128u>(a4, (uint32_t)p * kPartStride + (uint32_t)ks * 2u * chunk_bytes(kTile)),
+          desc_at<chunk_bytes(kBRows), 128u>(b4, (uint32_t)ks * 2u * chunk_bytes(kBRows)), (p | ks) ? 1u : 0u, desc);
+}
+
 __device__ __forceinline__ void fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
 // D (tensor memory, 128 lanes x 16 columns) = or += A (128 x 16, shared) * B^T (16 x 16, shared); one thread issues.
-__device__ __forceinline__ void mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t accumulate, uint32_t desc = kIdesc) {
+__device__ __forceinline__ void mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t accumulate, uint32_t desc) {
   asm volatile(
       "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}"
@@ -171,25 +185,19 @@ __global__ void __launch_bounds__(kTile) k_appearance_fwd_tc(AppearanceArgs a) {
   fence_after_sync();
   const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(&S.tmem_base);
   const uint32_t my_lane = tmem + ((uint32_t)(warp * 32) << 16);   // this warp's 32 lanes (bits 16..31 of the address)
-  const uint32_t A1[2] = {bulk::smem_addr(S.a1[0]), bulk::smem_addr(S.a1[1])};
-  const uint32_t W1 = bulk::smem_addr(S.w1), W2 = bulk::smem_addr(S.w2);
+  const uint32_t A4 = bulk::smem_addr(S.a1[0]) >> 4, W14 = bulk::smem_addr(S.w1) >> 4, W24 = bulk::smem_addr(S.w2) >> 4;
   constexpr int kParts = kSplit ? 2 : 1;
+  constexpr uint32_t kPartStride = 4u * chunk_bytes(kTile);      // the low halves' buffer follows the high halves'
   uint32_t phase = 0;
 
-  // one layer: the operands are in shared memory; issue, commit, wait (bounded)
-  auto run_layer = [&](const uint32_t A[2], uint32_t W, int ksteps, uint32_t d_cols) {
+  // one layer: the operands are in shared memory; issue (one thread), commit, wait (bounded)
+  auto run_layer = [&](auto issue) {
     bulk::fence_generic_writes();     // the rows just written with ordinary stores, for the tensor core's reads
     fence_before_sync();
     __syncthreads();
     if (tid == 0 && !*reinterpret_cast<volatile uint32_t *>(&S.failed)) {
       fence_after_sync();
-      uint32_t acc = 0u;
-      for (int p = 0; p < kParts; ++p)
-        for (int ks = 0; ks < ksteps; ++ks) {   // 16 columns of K per MMA = two chunks
-          mma(tmem + d_cols, smem_desc(A[p] + (uint32_t)ks * 2u * chunk_bytes(kTile), kTile),
-              smem_desc(W + (uint32_t)ks * 2u * chunk_bytes(16), 16), acc);
-          acc = 1u;
-        }
+      issue();
       commit(bar);
     }
     if (!*reinterpret_cast<volatile uint32_t *>(&S.failed)) {
@@ -222,14 +230,14 @@ __global__ void __launch_bounds__(kTile) k_appearance_fwd_tc(AppearanceArgs a) {
 #pragma unroll
       for (int c = 0; c < 4; ++c) store_chunk<kSplit>(S.a1[0], S.a1[1], (uint32_t)c * chunk_bytes(kTile) + (uint32_t)tid * 16u, x + 8 * c);
     }
-    run_layer(A1, W1, 2, 0u);
+    run_layer([&] { rows_times<kParts, 2, 16, kPartStride>(tmem + 0u, A4, W14, idesc(128, 16)); });
     float h[16];
     load16(my_lane + 0u, h);
 #pragma unroll
     for (int k = 0; k < 16; ++k) h[k] = fmaxf(h[k], 0.f);
 #pragma unroll
     for (int c = 0; c < 2; ++c) store_chunk<kSplit>(S.a1[0], S.a1[1], (uint32_t)c * chunk_bytes(kTile) + (uint32_t)tid * 16u, h + 8 * c);
-    run_layer(A1, W2, 1, 16u);
+    run_layer([&] { rows_times<kParts, 1, 16, kPartStride>(tmem + 16u, A4, W24, idesc(128, 16)); });
     load16(my_lane + 16u, h);
 #pragma unroll
     for (int k = 0; k < 16; ++k) h[k] = fmaxf(h[k], 0.f);
@@ -318,10 +326,11 @@ __global__ void __launch_bounds__(kTile) k_appearance_bwd_tc(AppearanceArgs a) {
   fence_after_sync();
   const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(&S.tmem_base);
   const uint32_t my_lane = tmem + ((uint32_t)(warp * 32) << 16);
-  const uint32_t X = bulk::smem_addr(S.x[0]), H1 = bulk::smem_addr(S.h1[0]), H2 = bulk::smem_addr(S.h2[0]);
-  const uint32_t D2 = bulk::smem_addr(S.d2[0]), D1 = bulk::smem_addr(S.d1[0]), GY = bulk::smem_addr(S.gy[0]);
-  const uint32_t W1 = bulk::smem_addr(S.w1), W2 = bulk::smem_addr(S.w2);
-  const uint32_t W2T = bulk::smem_addr(S.w2t), W1T = bulk::smem_addr(S.w1t);
+  // address fields (address >> 4) of the operand buffers
+  const uint32_t X4 = bulk::smem_addr(S.x[0]) >> 4, H14 = bulk::smem_addr(S.h1[0]) >> 4, H24 = bulk::smem_addr(S.h2[0]) >> 4;
+  const uint32_t D24 = bulk::smem_addr(S.d2[0]) >> 4, D14 = bulk::smem_addr(S.d1[0]) >> 4;
+  const uint32_t W14 = bulk::smem_addr(S.w1) >> 4, W24 = bulk::smem_addr(S.w2) >> 4;
+  const uint32_t W2T4 = bulk::smem_addr(S.w2t) >> 4, W1T4 = bulk::smem_addr(S.w1t) >> 4;
   constexpr int kParts = kSplit ? 2 : 1;
   constexpr uint32_t kChunk = chunk_bytes(kTile);          // 2048
   uint32_t phase = 0;
@@ -346,17 +355,6 @@ __global__ void __launch_bounds__(kTile) k_appearance_bwd_tc(AppearanceArgs a) {
     ++phase;
     fence_after_sync();
   };
-  // D (128 x n) = A (this tile's rows, `ksteps` x 16 columns, high and low halves `part_stride` bytes apart) * B^T
-  auto rows_times = [&](uint32_t A, uint32_t part_stride, uint32_t B, int brows, int ksteps, uint32_t d_cols, uint32_t desc) {
-    uint32_t acc = 0u;
-    for (int p = 0; p < kParts; ++p)
-      for (int ks = 0; ks < ksteps; ++ks) {
-        mma(tmem + d_cols, smem_desc(A + (uint32_t)p * part_stride + (uint32_t)ks * 2u * kChunk, kTile),
-            smem_desc(B + (uint32_t)ks * 2u * chunk_bytes(brows), brows), acc, desc);
-        acc = 1u;
-      }
-  };
-
   const int64_t ntiles = (a.n + kTile - 1) / kTile;
   for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
     const int64_t i = tile * kTile + tid;
@@ -389,7 +387,7 @@ __global__ void __launch_bounds__(kTile) k_appearance_bwd_tc(AppearanceArgs a) {
 #pragma unroll
       for (int c = 0; c < 4; ++c) store_chunk<kSplit>(S.x[0], S.x[1], (uint32_t)c * kChunk + (uint32_t)tid * 16u, x + 8 * c);
     }
-    run_phase([&] { rows_times(X, 4u * kChunk, W1, 16, 2, kF1, idesc(128, 16)); });
+    run_phase([&] { rows_times<kParts, 2, 16, 4u * kChunk>(tmem + kF1, X4, W14, idesc(128, 16)); });
     float h[16];
     uint32_t m1 = 0u, m2 = 0u;           // relu'(h1), relu'(h2) as bit masks
     load16(my_lane + kF1, h);
@@ -397,7 +395,7 @@ __global__ void __launch_bounds__(kTile) k_appearance_bwd_tc(AppearanceArgs a) {
     for (int k = 0; k < 16; ++k) { m1 |= (h[k] > 0.f ? 1u : 0u) << k; h[k] = fmaxf(h[k], 0.f); }
 #pragma unroll
     for (int c = 0; c < 2; ++c) store_chunk<kSplit>(S.h1[0], S.h1[1], (uint32_t)c * kChunk + (uint32_t)tid * 16u, h + 8 * c);
-    run_phase([&] { rows_times(H1, 2u * kChunk, W2, 16, 1, kF2, idesc(128, 16)); });
+    run_phase([&] { rows_times<kParts, 1, 16, 2u * kChunk>(tmem + kF2, H14, W24, idesc(128, 16)); });
     load16(my_lane + kF2, h);
 #pragma unroll
     for (int k = 0; k < 16; ++k) { m2 |= (h[k] > 0.f ? 1u : 0u) << k; h[k] = fmaxf(h[k], 0.f); }
@@ -429,7 +427,7 @@ __global__ void __launch_bounds__(kTile) k_appearance_bwd_tc(AppearanceArgs a) {
     for (int k = 0; k < 16; ++k) h[k] = (m2 >> k) & 1u ? h[k] : 0.f;
 #pragma unroll
     for (int c = 0; c < 2; ++c) store_chunk<kSplit>(S.d2[0], S.d2[1], (uint32_t)c * kChunk + (uint32_t)tid * 16u, h + 8 * c);
-    run_phase([&] { rows_times(D2, 2u * kChunk, W2T, 16, 1, kE, idesc(128, 16)); });
+    run_phase([&] { rows_times<kParts, 1, 16, 2u * kChunk>(tmem + kE, D24, W2T4, idesc(128, 16)); });
     load16(my_lane + kE, h);
 #pragma unroll
     for (int k = 0; k < 16; ++k) h[k] = (m1 >> k) & 1u ? h[k] : 0.f;
@@ -437,12 +435,12 @@ __global__ void __launch_bounds__(kTile) k_appearance_bwd_tc(AppearanceArgs a) {
     for (int c = 0; c < 2; ++c) store_chunk<kSplit>(S.d1[0], S.d1[1], (uint32_t)c * kChunk + (uint32_t)tid * 16u, h + 8 * c);
     const bool fresh = first_tile;
     run_phase([&] {
-      rows_times(D1, 2u * kChunk, W1T, 32, 1, kGX, idesc(128, 32));
+      rows_times<kParts, 1, 32, 2u * kChunk>(tmem + kGX, D14, W1T4, idesc(128, 32));
       // weight gradients: K runs over the tile's rows, 16 per MMA; A = [X | h1 | h2] (16 chunks), B = [delta2 | delta1 | gy] (10)
-      for (int ks = 0; ks < kTile / 16; ++ks) {
-        const uint32_t off = (uint32_t)ks * 256u;
-        mma(tmem + kDW, smem_desc_mn(X + off, kChunk), smem_desc_mn(D2 + off, kChunk), (fresh && ks == 0) ? 0u : 1u, idesc(128, 80, true, true));
-      }
+#pragma unroll
+      for (int ks = 0; ks < kTile / 16; ++ks)
+        mma(tmem + kDW, desc_at<128u, kChunk>(X4, (uint32_t)ks * 256u), desc_at<128u, kChunk>(D24, (uint32_t)ks * 256u),
+            (fresh && ks == 0) ? 0u : 1u, idesc(128, 80, true, true));
     });
     first_tile = false;
     float gx[32];
