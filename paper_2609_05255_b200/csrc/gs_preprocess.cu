@@ -950,6 +950,167 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_bwd(PreprocessBwdArgs a, 
   if (Explicit<APP>::value && lane == 0) bulk::wait_stores_done();
 }
 
+// ---- preprocess backward over the Gaussians that received a gradient -------------------------------------------
+// A Gaussian whose nine 2D gradients are all zero - culled, or listed in tiles but composited by no pixel of this view
+// because the pixels it covers saturated in front of it - gets zero gradients whatever its parameters are.  In a
+// scene with occlusion that is most of them (config 3: 94 % of the visible Gaussians of a view).  This kernel writes
+// their zero rows straight away and queues the others; whenever kBlock of them are queued, the CTA runs them through
+// the decoder and projection backward, one per thread, with every lane busy.  The queue is filled in thread order and
+// a CTA's chunks are fixed by the grid, so the order of all sums is the same from run to run.
+template <int APP>
+__global__ void __launch_bounds__(kBlock) k_preprocess_bwd_sparse(PreprocessBwdArgs a, CamDev cam) {
+  static_assert(IsNeural<APP>::value || APP == kAppExternal, "the neural model, or the projection alone");
+  extern __shared__ __align__(16) float smem[];
+  constexpr int kScan = 4;                               // chunks looked at per round
+  __shared__ uint32_t s_queue[2 * kScan * kBlock];       // a power of two above kScan * kBlock + kBlock - 1
+  __shared__ int s_warp_count[kScan][kWarps];
+  constexpr int kMask = 2 * kScan * kBlock - 1;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  mlp::Weights &sWt = *reinterpret_cast<mlp::Weights *>(smem);
+  mlp::WarpStage *sStage = reinterpret_cast<mlp::WarpStage *>(reinterpret_cast<unsigned char *>(smem) + sizeof(mlp::Weights));
+  mlp::WeightGrad dW;
+  if (IsNeural<APP>::value) {
+    mlp::load_weights(a.weights, sWt, tid, kBlock);
+    dW.clear();
+    __syncthreads();
+  }
+  int q_head = 0, q_count = 0;      // the same in every thread
+
+  // the first `count` queued Gaussians, one per thread
+  auto process = [&](int count) {
+    const bool has = tid < count;
+    const int64_t i = has ? (int64_t)s_queue[(q_head + tid) & kMask] : 0;
+    float gd[3] = {0.f, 0.f, 0.f};
+    float mu[3] = {0.f, 0.f, 0.f}, ls[3] = {0.f, 0.f, 0.f}, q[4] = {1.f, 0.f, 0.f, 0.f}, logit = 0.f;
+    float4 ga = make_float4(0.f, 0.f, 0.f, 0.f), gb = ga, gc = ga;
+    float base[3] = {0.f, 0.f, 0.f};
+    uint4 feat_raw = make_uint4(0u, 0u, 0u, 0u);
+    float dx = 0.f, dy = 0.f, dz = 1.f;
+    if (has) {
+      load3(a.means, i, mu);
+      load3(a.log_scales, i, ls);
+      const float4 q4 = __ldg(reinterpret_cast<const float4 *>(a.quats) + i);
+      logit = __ldg(a.logits + i);
+      const float4 *g2 = reinterpret_cast<const float4 *>(a.g2d) + 3 * i;
+      ga = g2[0]; gb = g2[1]; gc = g2[2];
+      if (APP != kAppExternal) load3(a.base_color, i, base);
+      else load3(a.gd_in, i, gd);
+      if (IsNeural<APP>::value) feat_raw = __ldg(reinterpret_cast<const uint4 *>(a.features) + i);
+      q[0] = q4.x; q[1] = q4.y; q[2] = q4.z; q[3] = q4.w;
+      const float vx = mu[0] - cam.oc[0], vy = mu[1] - cam.oc[1], vz = mu[2] - cam.oc[2];
+      const float vi = rsqrtf(vx * vx + vy * vy + vz * vz);
+      dx = vx * vi; dy = vy * vi; dz = vz * vi;
+    }
+    float gp[3] = {0.f, 0.f, 0.f};
+    if (IsNeural<APP>::value) {
+      float gf[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+      const float gcol[3] = {ga.x, ga.y, ga.z};
+      if (warp * 32 < count && a.deg > 0) {     // the whole warp goes through the decoder; lanes past the count feed zeros
+        float x[32];
+        if (has) {
+          float f[8];
+          unpack_features(feat_raw, f);
+          decoder_inputs(dx, dy, dz, f, a.deg, x);
+        } else {
+#pragma unroll
+          for (int k = 0; k < 32; ++k) x[k] = 0.f;
+        }
+        decode_backward_warp<Split<APP>::value>(sWt, sStage[warp], lane, has, x, dx, dy, dz, a.deg, a.act, base, gcol, dW, gp, gf, gd);
+      } else if (has) {
+#pragma unroll
+        for (int c = 0; c < 3; ++c) gp[c] = color_act_grad_z(a.act, base[c] + 0.5f) * gcol[c];
+      }
+      if (has) {
+        float4 *gfp = reinterpret_cast<float4 *>(a.g_features) + 2 * i;
+        gfp[0] = make_float4(gf[0], gf[1], gf[2], gf[3]);
+        gfp[1] = make_float4(gf[4], gf[5], gf[6], gf[7]);
+      }
+    }
+    if (has) {
+      const GeoGrads gg = project_backward(mu, ls, q, logit, cam, gb.x, gb.y, gb.z, gb.w, gc.x, ga.w, gd);
+      store3(a.g_means, i, gg.mu[0], gg.mu[1], gg.mu[2]);
+      store3(a.g_log_scales, i, gg.ls[0], gg.ls[1], gg.ls[2]);
+      reinterpret_cast<float4 *>(a.g_quats)[i] = make_float4(gg.q[0], gg.q[1], gg.q[2], gg.q[3]);
+      a.g_logits[i] = gg.logit;
+      if (APP != kAppExternal) store3(a.g_base, i, gp[0], gp[1], gp[2]);
+    }
+  };
+
+  // The scan: kScan chunks of kBlock Gaussians per round, all their loads in flight together.
+  const int64_t nrounds = (a.n + kScan * kBlock - 1) / (kScan * kBlock);
+  for (int64_t round = blockIdx.x; round < nrounds; round += gridDim.x) {
+    reload_fence();
+    bool active[kScan];
+    ushort4 rc[kScan];
+#pragma unroll
+    for (int k = 0; k < kScan; ++k) {
+      const int64_t i = (round * kScan + k) * kBlock + tid;
+      rc[k] = i < a.n ? __ldg(reinterpret_cast<const ushort4 *>(a.rect) + i) : make_ushort4(0, 0, 0, 0);
+    }
+    float4 ga[kScan], gb[kScan];
+    float gv[kScan];
+#pragma unroll
+    for (int k = 0; k < kScan; ++k) {
+      const int64_t i = (round * kScan + k) * kBlock + tid;
+      active[k] = rc[k].z > rc[k].x && rc[k].w > rc[k].y;     // (false past the end: an empty rectangle)
+      ga[k] = gb[k] = make_float4(0.f, 0.f, 0.f, 0.f); gv[k] = 0.f;
+      if (active[k]) {
+        const float4 *g2 = reinterpret_cast<const float4 *>(a.g2d) + 3 * i;
+        ga[k] = g2[0]; gb[k] = g2[1]; gv[k] = a.g2d[12 * i + 8];
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < kScan; ++k) {
+      const int64_t i = (round * kScan + k) * kBlock + tid;
+      active[k] = active[k] && (ga[k].x != 0.f || ga[k].y != 0.f || ga[k].z != 0.f || ga[k].w != 0.f || gb[k].x != 0.f ||
+                                gb[k].y != 0.f || gb[k].z != 0.f || gb[k].w != 0.f || gv[k] != 0.f);
+      if (i < a.n && !active[k]) {
+        store3(a.g_means, i, 0.f, 0.f, 0.f);
+        store3(a.g_log_scales, i, 0.f, 0.f, 0.f);
+        reinterpret_cast<float4 *>(a.g_quats)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        a.g_logits[i] = 0.f;
+        if (APP != kAppExternal) store3(a.g_base, i, 0.f, 0.f, 0.f);
+        if (IsNeural<APP>::value) {
+          float4 *gfp = reinterpret_cast<float4 *>(a.g_features) + 2 * i;
+          gfp[0] = make_float4(0.f, 0.f, 0.f, 0.f);
+          gfp[1] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+      }
+    }
+    // queue the active ones in index order: chunk by chunk, thread by thread
+    unsigned ballot[kScan];
+#pragma unroll
+    for (int k = 0; k < kScan; ++k) {
+      ballot[k] = __ballot_sync(kFull, active[k]);
+      if (lane == 0) s_warp_count[k][warp] = __popc(ballot[k]);
+    }
+    __syncthreads();
+    int before = 0;
+#pragma unroll
+    for (int k = 0; k < kScan; ++k) {
+      int offset = 0, total = 0;
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) { const int c = s_warp_count[k][w]; offset += w < warp ? c : 0; total += c; }
+      if (active[k])
+        s_queue[(q_head + q_count + before + offset + __popc(ballot[k] & ((1u << lane) - 1u))) & kMask] =
+            (uint32_t)((round * kScan + k) * kBlock + tid);
+      before += total;
+    }
+    __syncthreads();
+    q_count += before;
+    while (q_count >= kBlock) {
+      process(kBlock);
+      q_head = (q_head + kBlock) & kMask;
+      q_count -= kBlock;
+      __syncthreads();
+    }
+  }
+  if (q_count > 0) process(q_count);
+  if (IsNeural<APP>::value) {
+    weight_grad_flush(dW, reinterpret_cast<float *>(sStage), a.w_partials + (size_t)blockIdx.x * GS_MLP_WEIGHTS, tid);
+  }
+}
+
 // ---- separate-pass appearance kernels of the neural model (the explicit models follow, with bulk copies) ------
 #include "gs_decoder_tc.cuh"
 
@@ -1219,19 +1380,20 @@ int launch_preprocess_bwd(int app, const PreprocessBwdArgs &a, const CamDev &cam
     return 1;
   } else if (app == kAppExternal) {
     if (a.n == 0) return 0;
-    k_preprocess_bwd<kAppExternal><<<grid_for(a.n), kBlock, 16, st>>>(a, cam);
+    const int wave = resident_blocks<k_preprocess_bwd_sparse<kAppExternal>>(sizeof(mlp::Weights), 1 << 20), chunks = grid_for(a.n);
+    k_preprocess_bwd_sparse<kAppExternal><<<chunks < wave ? chunks : wave, kBlock, sizeof(mlp::Weights), st>>>(a, cam);
     return 1;
   } else {
     if (app == kAppNeuralHalf) {
-      opt_in_smem(k_preprocess_bwd<kAppNeuralHalf>, kBwdSmemNN);
-      const int blocks = resident_blocks<k_preprocess_bwd<kAppNeuralHalf>>(kBwdSmemNN);
-      k_preprocess_bwd<kAppNeuralHalf><<<blocks, kBlock, kBwdSmemNN, st>>>(a, cam);
+      opt_in_smem(k_preprocess_bwd_sparse<kAppNeuralHalf>, kBwdSmemNN);
+      const int blocks = resident_blocks<k_preprocess_bwd_sparse<kAppNeuralHalf>>(kBwdSmemNN);
+      k_preprocess_bwd_sparse<kAppNeuralHalf><<<blocks, kBlock, kBwdSmemNN, st>>>(a, cam);
       launch_wgrad_reduce(a.w_partials, blocks, a.g_weights, st);
       return 2;
     }
-    opt_in_smem(k_preprocess_bwd<GS_APP_NEURAL>, kBwdSmemNN);
-    const int blocks = resident_blocks<k_preprocess_bwd<GS_APP_NEURAL>>(kBwdSmemNN);
-    k_preprocess_bwd<GS_APP_NEURAL><<<blocks, kBlock, kBwdSmemNN, st>>>(a, cam);
+    opt_in_smem(k_preprocess_bwd_sparse<GS_APP_NEURAL>, kBwdSmemNN);
+    const int blocks = resident_blocks<k_preprocess_bwd_sparse<GS_APP_NEURAL>>(kBwdSmemNN);
+    k_preprocess_bwd_sparse<GS_APP_NEURAL><<<blocks, kBlock, kBwdSmemNN, st>>>(a, cam);
     launch_wgrad_reduce(a.w_partials, blocks, a.g_weights, st);
     return 2;
   }
