@@ -277,7 +277,7 @@ def run_ours(args):
             clocks = sampler.stop()
         # units of the blend kernels: list entries up to each pixel's last composited one, over the views
         entries = 0
-        visible = records = 0
+        visible = records = with_gradient = 0
         evaluated = composited = warp_steps = warp_steps_idle = 0
         for v in range(views):
             r.forward(ds, cams[v])
@@ -286,7 +286,14 @@ def run_ours(args):
             ev, co, ws_, wi = api.gs_profile_blend_counts(ctx, r.proj, r.binning, cams[v])
             evaluated += ev; composited += co; warp_steps += ws_; warp_steps_idle += wi
             rect = r.proj.rect.to(torch.int32) & 0xFFFF
-            visible += int(((rect[:, 2] > rect[:, 0]) & (rect[:, 3] > rect[:, 1])).sum().item())
+            vis_rows = (rect[:, 2] > rect[:, 0]) & (rect[:, 3] > rect[:, 1])
+            visible += int(vis_rows.sum().item())
+            # Gaussians that receive a gradient in this view (the backward leaves the 2D gradients [n,12] at the start of
+            # the workspace): the others are hidden behind saturated pixels and the preprocess backward skips them
+            r.backward(ds, cams[v], G[v])
+            torch.cuda.synchronize()
+            g2d = r.workspace[: ds.n * 48].view(torch.float32).reshape(ds.n, 12)
+            with_gradient += int(((g2d[:, :9] != 0).any(1) & vis_rows).sum().item())
             records += int((r.proj.cell_count.to(torch.int64) & 0x7FFFFFFF).sum().item())
         # the same step through the unfused reference path (App. D "Fusion"): appearance as passes of its own
         unfused = None
@@ -310,7 +317,7 @@ def run_ours(args):
                             "split ones; colours within 2e-3 of the oracle instead of 2e-5 (tests/test_gpu_half_precision.py)"}
         results[tag] = dict(ms=ms, ms_one=ms_one, ms_streams=ms_streams, graph=graph_note, unfused=unfused, half=half,
                             stage_ms=stage_ms, stage_launches=stage_launches, pairs=pairs,
-                            entries=entries, visible=visible, records=records, evaluated=evaluated, composited=composited,
+                            entries=entries, visible=visible, records=records, with_gradient=with_gradient, evaluated=evaluated, composited=composited,
                             warp_steps=warp_steps, warp_steps_idle=warp_steps_idle,
                             host=host, ds=ds, r=r, app=tag)
 
@@ -371,6 +378,7 @@ def run_ours(args):
         "stages_ms_per_step": {k: round(v, 4) for k, v in stage_ms.items() if v > 0},
         "stage_share": {k: round(v / total_stage, 4) for k, v in stage_ms.items() if v > 0},
         "pairs_per_view": neural["pairs"], "visible_per_view": neural["visible"] / views,
+        "with_gradient_per_view": neural["with_gradient"] / views,
         "blend_warp_steps_per_view": neural["warp_steps"] / views,
         "blend_warp_steps_without_a_taker_per_view": neural["warp_steps_idle"] / views,
         "sh": None if "sh" not in results or head == "sh" else {
@@ -414,7 +422,7 @@ STAGE_KERNELS = {
     "tile_sort": "k_radix_hist, k_radix_scan_rows, k_radix_scatter<9>: one stable pass on the cell id",
     "tile_ranges": "k_cell_chunks, k_chunk_counts, k_cell_prefix, k_tile_scan, k_expand: records -> per-tile lists",
     "blend_fwd": "k_blend_fwd", "blend_bwd": "k_blend_bwd",
-    "preprocess_bwd": "k_preprocess_bwd (+ k_wgrad_reduce for the decoder weights)"}
+    "preprocess_bwd": "k_preprocess_bwd_sparse (zero rows at once, the Gaussians with a gradient in full batches) + k_wgrad_reduce"}
 
 
 def stage_roofline(stage, arm, views, n, peaks, alu_peak):
@@ -455,7 +463,9 @@ def _stage_roofline(stage, arm, views, n, peaks, alu_peak):
     R = arm["records"] / views                   # (Gaussian, cell of 4 x 4 tiles) records of a view
     app_bytes = 28.0
     per_launch = {"preprocess_fwd": 44.0 * n + 12.0 * n + (app_bytes + 48.0) * vis + 4.0 * R,
-                  "preprocess_bwd": 8.0 * n + (44.0 + 48.0 + app_bytes) * vis + 88.0 * n,
+                  # rectangle of every Gaussian, 2D gradients of the visible ones, a gradient row for every Gaussian;
+                  # parameters and 2D gradients again for the ones that received a gradient
+                  "preprocess_bwd": 8.0 * n + 48.0 * vis + 88.0 * n + (44.0 + 48.0 + app_bytes) * (arm["with_gradient"] / views),
                   "depth_sort": (4 * 20.0 - 4.0) * n,     # per pass: keys read twice, values once, both written
                   "keygen": 8.0 * n + 12.0 * R,           # id + count per Gaussian; record read, key + value written
                   "tile_sort": 20.0 * R,                  # one pass: keys read twice, values once, both written

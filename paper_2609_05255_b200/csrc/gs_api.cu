@@ -227,8 +227,8 @@ FwdWorkspace carve_fwd(void *ws, int64_t n, int64_t cap, int width, int height) 
 }
 
 // Backward scratch: the 2D gradients [n,12], then (used by the separate-pass path only) directions, dL/dcolor and
-// dL/dd as [n,3] each.
-struct BwdWorkspace { float *g2d, *dirs, *g_color, *g_dirs; size_t bytes; };
+// dL/dd as [n,3] each, then the flags of the Gaussians that received a gradient.
+struct BwdWorkspace { float *g2d, *dirs, *g_color, *g_dirs; uint32_t *flags; size_t bytes; };
 BwdWorkspace carve_bwd(void *ws, int64_t n) {
   Carver c{static_cast<char *>(ws), 0};
   const size_t nn = (size_t)(n > 0 ? n : 1);
@@ -237,6 +237,7 @@ BwdWorkspace carve_bwd(void *ws, int64_t n) {
   w.dirs = c.take<float>(nn * 3);
   w.g_color = c.take<float>(nn * 3);
   w.g_dirs = c.take<float>(nn * 3);
+  w.flags = c.take<uint32_t>((nn + 31) / 32);     // one bit per Gaussian: it received a gradient
   w.bytes = c.used;
   return w;
 }
@@ -509,6 +510,7 @@ GsStatus gs_render_backward(GsContext *ctx, const GsScene *scene, const GsCamera
   a.g_sh_rest = scene->app == GS_APP_SV ? grads->sv_sites : grads->sh_rest;
   a.g_features = grads->features; a.w_partials = ctx->d_w_partials; a.g_weights = grads->mlp_weights;
   a.gd_in = bw.g_dirs;
+  a.flags = bw.flags;
   a.timeout = ctx->d_counter + 3;
   if (n == 0 && scene->app == GS_APP_NEURAL) {
     const DecoderArch d = decoder_arch(scene);

@@ -65,6 +65,7 @@ struct PreprocessBwdArgs {
   const float *g2d;            // [n,12]: dL/dcolor(3), dL/dopacity, dL/dconic(3), dL/dmean2d(2), pad
   unsigned long long *timeout; // set to 1 if a bounded wait on a bulk copy ran out (never expected)
   const float *gd_in;          // kAppExternal only: [n,3] dL/dd from the separate appearance backward
+  uint32_t *flags;             // scratch, one bit per Gaussian: it received a gradient in this view
   float *g_means, *g_log_scales, *g_quats, *g_logits, *g_base, *g_sh_rest, *g_features;
   float *w_partials;           // [kWgradBlocks, 816]
   float *g_weights;            // [816]

@@ -953,18 +953,51 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_bwd(PreprocessBwdArgs a, 
 // ---- preprocess backward over the Gaussians that received a gradient -------------------------------------------
 // A Gaussian whose nine 2D gradients are all zero - culled, or listed in tiles but composited by no pixel of this view
 // because the pixels it covers saturated in front of it - gets zero gradients whatever its parameters are.  In a
-// scene with occlusion that is most of them (config 3: 94 % of the visible Gaussians of a view).  This kernel writes
-// their zero rows straight away and queues the others; whenever kBlock of them are queued, the CTA runs them through
-// the decoder and projection backward, one per thread, with every lane busy.  The queue is filled in thread order and
-// a CTA's chunks are fixed by the grid, so the order of all sums is the same from run to run.
+// scene with occlusion that is most of them (config 3: 94 % of the visible Gaussians of a view).  Two kernels:
+// k_bwd_flags streams over all Gaussians at full occupancy, writes the zero rows and leaves one bit per Gaussian
+// (set = it received a gradient); k_preprocess_bwd_sparse, persistent, gathers the flagged ones in index order and,
+// whenever kBlock of them are queued, runs them through the decoder and projection backward, one per thread, with
+// every lane busy.  A CTA's run of flag words is fixed by the grid, so the order of all sums is the same from run to
+// run.
+constexpr int kFlagThreads = 256;
+template <bool kBase, bool kFeatures>
+__global__ void __launch_bounds__(kFlagThreads) k_bwd_flags(PreprocessBwdArgs a) {
+  const int64_t i = (int64_t)blockIdx.x * kFlagThreads + threadIdx.x;
+  bool active = false;
+  if (i < a.n) {
+    const ushort4 rc = __ldg(reinterpret_cast<const ushort4 *>(a.rect) + i);
+    if (rc.z > rc.x && rc.w > rc.y) {
+      const float4 *g2 = reinterpret_cast<const float4 *>(a.g2d) + 3 * i;
+      const float4 ga = g2[0], gb = g2[1];
+      const float gv = a.g2d[12 * i + 8];
+      active = ga.x != 0.f || ga.y != 0.f || ga.z != 0.f || ga.w != 0.f || gb.x != 0.f || gb.y != 0.f || gb.z != 0.f ||
+               gb.w != 0.f || gv != 0.f;
+    }
+    if (!active) {
+      store3(a.g_means, i, 0.f, 0.f, 0.f);
+      store3(a.g_log_scales, i, 0.f, 0.f, 0.f);
+      reinterpret_cast<float4 *>(a.g_quats)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+      a.g_logits[i] = 0.f;
+      if (kBase) store3(a.g_base, i, 0.f, 0.f, 0.f);
+      if (kFeatures) {
+        float4 *gfp = reinterpret_cast<float4 *>(a.g_features) + 2 * i;
+        gfp[0] = make_float4(0.f, 0.f, 0.f, 0.f);
+        gfp[1] = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    }
+  }
+  const unsigned ballot = __ballot_sync(kFull, active);
+  if ((threadIdx.x & 31) == 0 && i < a.n) a.flags[i >> 5] = ballot;    // (i is a multiple of 32 here)
+}
+
 template <int APP>
 __global__ void __launch_bounds__(kBlock) k_preprocess_bwd_sparse(PreprocessBwdArgs a, CamDev cam) {
   static_assert(IsNeural<APP>::value || APP == kAppExternal, "the neural model, or the projection alone");
   extern __shared__ __align__(16) float smem[];
-  constexpr int kScan = 4;                               // chunks looked at per round
-  __shared__ uint32_t s_queue[2 * kScan * kBlock];       // a power of two above kScan * kBlock + kBlock - 1
-  __shared__ int s_warp_count[kScan][kWarps];
-  constexpr int kMask = 2 * kScan * kBlock - 1;
+  constexpr int kWordsPerRound = kBlock / 4;             // flag words (of 32 Gaussians) looked at per round
+  __shared__ uint32_t s_queue[2 * 32 * kWordsPerRound];  // a power of two above 32 * kWordsPerRound + kBlock - 1
+  __shared__ int s_warp_count[kWarps];
+  constexpr int kMask = 2 * 32 * kWordsPerRound - 1;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   mlp::Weights &sWt = *reinterpret_cast<mlp::Weights *>(smem);
   mlp::WarpStage *sStage = reinterpret_cast<mlp::WarpStage *>(reinterpret_cast<unsigned char *>(smem) + sizeof(mlp::Weights));
@@ -1036,68 +1069,37 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_bwd_sparse(PreprocessBwdA
     }
   };
 
-  // The scan: kScan chunks of kBlock Gaussians per round, all their loads in flight together.
-  const int64_t nrounds = (a.n + kScan * kBlock - 1) / (kScan * kBlock);
-  for (int64_t round = blockIdx.x; round < nrounds; round += gridDim.x) {
+  // The flags of k_bwd_flags, one bit per Gaussian, say who is left.  Every CTA takes one contiguous run of flag words
+  // (equal to within a word whatever the grid) and reads it kWordsPerRound words at a time: thread t looks at byte
+  // t % 4 of word t / 4, an exclusive scan over the CTA gives its place in the queue, and it writes the indices of its
+  // set bits there - index order, the same from run to run.
+  const int64_t nwords = (a.n + 31) / 32, per_cta = (nwords + gridDim.x - 1) / gridDim.x;
+  const int64_t w_begin = min(nwords, (int64_t)blockIdx.x * per_cta), w_end = min(nwords, w_begin + per_cta);
+  for (int64_t w0 = w_begin; w0 < w_end; w0 += kWordsPerRound) {
     reload_fence();
-    bool active[kScan];
-    ushort4 rc[kScan];
+    const int64_t w = w0 + (tid >> 2);
+    const uint32_t byte = w < w_end ? (__ldg(a.flags + w) >> (8 * (tid & 3))) & 255u : 0u;
+    const int cnt = __popc(byte);
+    int incl = cnt;
 #pragma unroll
-    for (int k = 0; k < kScan; ++k) {
-      const int64_t i = (round * kScan + k) * kBlock + tid;
-      rc[k] = i < a.n ? __ldg(reinterpret_cast<const ushort4 *>(a.rect) + i) : make_ushort4(0, 0, 0, 0);
+    for (int sft = 1; sft < 32; sft <<= 1) {
+      const int t = __shfl_up_sync(kFull, incl, sft);
+      if (lane >= sft) incl += t;
     }
-    float4 ga[kScan], gb[kScan];
-    float gv[kScan];
+    if (lane == 31) s_warp_count[warp] = incl;
+    __syncthreads();
+    int offset = incl - cnt, total = 0;
 #pragma unroll
-    for (int k = 0; k < kScan; ++k) {
-      const int64_t i = (round * kScan + k) * kBlock + tid;
-      active[k] = rc[k].z > rc[k].x && rc[k].w > rc[k].y;     // (false past the end: an empty rectangle)
-      ga[k] = gb[k] = make_float4(0.f, 0.f, 0.f, 0.f); gv[k] = 0.f;
-      if (active[k]) {
-        const float4 *g2 = reinterpret_cast<const float4 *>(a.g2d) + 3 * i;
-        ga[k] = g2[0]; gb[k] = g2[1]; gv[k] = a.g2d[12 * i + 8];
-      }
-    }
-#pragma unroll
-    for (int k = 0; k < kScan; ++k) {
-      const int64_t i = (round * kScan + k) * kBlock + tid;
-      active[k] = active[k] && (ga[k].x != 0.f || ga[k].y != 0.f || ga[k].z != 0.f || ga[k].w != 0.f || gb[k].x != 0.f ||
-                                gb[k].y != 0.f || gb[k].z != 0.f || gb[k].w != 0.f || gv[k] != 0.f);
-      if (i < a.n && !active[k]) {
-        store3(a.g_means, i, 0.f, 0.f, 0.f);
-        store3(a.g_log_scales, i, 0.f, 0.f, 0.f);
-        reinterpret_cast<float4 *>(a.g_quats)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-        a.g_logits[i] = 0.f;
-        if (APP != kAppExternal) store3(a.g_base, i, 0.f, 0.f, 0.f);
-        if (IsNeural<APP>::value) {
-          float4 *gfp = reinterpret_cast<float4 *>(a.g_features) + 2 * i;
-          gfp[0] = make_float4(0.f, 0.f, 0.f, 0.f);
-          gfp[1] = make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-      }
-    }
-    // queue the active ones in index order: chunk by chunk, thread by thread
-    unsigned ballot[kScan];
-#pragma unroll
-    for (int k = 0; k < kScan; ++k) {
-      ballot[k] = __ballot_sync(kFull, active[k]);
-      if (lane == 0) s_warp_count[k][warp] = __popc(ballot[k]);
+    for (int ww = 0; ww < kWarps; ++ww) { const int c = s_warp_count[ww]; offset += ww < warp ? c : 0; total += c; }
+    uint32_t bits = byte;
+    const uint32_t row0 = (uint32_t)(w * 32 + 8 * (tid & 3));
+    for (int slot = q_head + q_count + offset; bits; ++slot) {
+      const int b = __ffs(bits) - 1;
+      bits &= bits - 1u;
+      s_queue[slot & kMask] = row0 + (uint32_t)b;
     }
     __syncthreads();
-    int before = 0;
-#pragma unroll
-    for (int k = 0; k < kScan; ++k) {
-      int offset = 0, total = 0;
-#pragma unroll
-      for (int w = 0; w < kWarps; ++w) { const int c = s_warp_count[k][w]; offset += w < warp ? c : 0; total += c; }
-      if (active[k])
-        s_queue[(q_head + q_count + before + offset + __popc(ballot[k] & ((1u << lane) - 1u))) & kMask] =
-            (uint32_t)((round * kScan + k) * kBlock + tid);
-      before += total;
-    }
-    __syncthreads();
-    q_count += before;
+    q_count += total;
     while (q_count >= kBlock) {
       process(kBlock);
       q_head = (q_head + kBlock) & kMask;
@@ -1380,22 +1382,25 @@ int launch_preprocess_bwd(int app, const PreprocessBwdArgs &a, const CamDev &cam
     return 1;
   } else if (app == kAppExternal) {
     if (a.n == 0) return 0;
+    k_bwd_flags<false, false><<<(int)((a.n + kFlagThreads - 1) / kFlagThreads), kFlagThreads, 0, st>>>(a);
     const int wave = resident_blocks<k_preprocess_bwd_sparse<kAppExternal>>(sizeof(mlp::Weights), 1 << 20), chunks = grid_for(a.n);
     k_preprocess_bwd_sparse<kAppExternal><<<chunks < wave ? chunks : wave, kBlock, sizeof(mlp::Weights), st>>>(a, cam);
-    return 1;
+    return 2;
   } else {
     if (app == kAppNeuralHalf) {
       opt_in_smem(k_preprocess_bwd_sparse<kAppNeuralHalf>, kBwdSmemNN);
       const int blocks = resident_blocks<k_preprocess_bwd_sparse<kAppNeuralHalf>>(kBwdSmemNN);
+      if (a.n > 0) k_bwd_flags<true, true><<<(int)((a.n + kFlagThreads - 1) / kFlagThreads), kFlagThreads, 0, st>>>(a);
       k_preprocess_bwd_sparse<kAppNeuralHalf><<<blocks, kBlock, kBwdSmemNN, st>>>(a, cam);
       launch_wgrad_reduce(a.w_partials, blocks, a.g_weights, st);
-      return 2;
+      return 3;
     }
     opt_in_smem(k_preprocess_bwd_sparse<GS_APP_NEURAL>, kBwdSmemNN);
     const int blocks = resident_blocks<k_preprocess_bwd_sparse<GS_APP_NEURAL>>(kBwdSmemNN);
+    if (a.n > 0) k_bwd_flags<true, true><<<(int)((a.n + kFlagThreads - 1) / kFlagThreads), kFlagThreads, 0, st>>>(a);
     k_preprocess_bwd_sparse<GS_APP_NEURAL><<<blocks, kBlock, kBwdSmemNN, st>>>(a, cam);
     launch_wgrad_reduce(a.w_partials, blocks, a.g_weights, st);
-    return 2;
+    return 3;
   }
 }
 
