@@ -440,7 +440,7 @@ def stage_roofline(stage, arm, views, n, peaks, alu_peak):
             out["fma_pipe_active_frac_ncu"] = e.get("fma_pipe_cycles_active")
             out["alu_pipe_active_frac_ncu"] = e.get("alu_pipe_cycles_active")
             out["traffic_source"] = (f"profiles/ncu_constants.json: {e.get('kernel')} ({e.get('launch')}), "
-                                     f"captured at commit {consts.get('commit')}")
+                                     f"captured at commit {e.get('commit') or consts.get('commit')}")
     return out
 
 
