@@ -810,7 +810,8 @@ def decode_sweep(api, torch, ctx, dev, peaks, args):
                     out[row]["bwd_ms_" + name] = round(run(lambda: api.gs_appearance_backward(ctx, sc, dirs, gcol, grads, gd)), 4)
                 api.gs_set_decoder_engine(ctx, api.GS_ENGINE_AUTO)
             del sc, color, grads, gd, flush
-        # the decoder variants of the architecture table (App. D), fp32 CUDA-core kernels: 1M only
+        # the decoder variants of the architecture table (App. D): 1M only; the default engine runs them on tcgen05,
+        # GS_ENGINE_WARP_MMA selects the fp32 CUDA-core kernels they were first built on
         for hidden, layers, nfeat in (((16, 1, 8), (16, 3, 8), (32, 2, 8), (16, 2, 16)) if n == 1_000_000 else ()):
             nw = api.decoder_num_weights(hidden, layers)
             w = ((torch.rand((nw,), device=dev, generator=gen) - 0.5) * (16.0 / hidden) ** 0.5).half()
@@ -837,15 +838,24 @@ def decode_sweep(api, torch, ctx, dev, peaks, args):
                 return ts[len(ts) // 2]
             f_ms = run_v(lambda: api.gs_appearance_forward(ctx, sc, dirs, color))
             b_ms = run_v(lambda: api.gs_appearance_backward(ctx, sc, dirs, gcol, grads, gd))
+            api.gs_set_decoder_engine(ctx, api.GS_ENGINE_WARP_MMA)
+            f_fma = run_v(lambda: api.gs_appearance_forward(ctx, sc, dirs, color))
+            b_fma = run_v(lambda: api.gs_appearance_backward(ctx, sc, dirs, gcol, grads, gd))
+            api.gs_set_decoder_engine(ctx, api.GS_ENGINE_AUTO)
             # forward: one pass over the weights; backward: the forward again, the transposed pass and the weight gradient
             flop_fwd, flop_bwd = 2 * nw * n, 6 * nw * n
+            gbs = (bytes_fwd + bytes_bwd) * n / ((f_ms + b_ms) * 1e-3) / 1e9
+            dflt = out[f"neural_{n // 1_000_000}M"]          # the default decoder (816 weights) on the same Gaussians
             out[f"neural_h{hidden}_l{layers}_f{nfeat}_{n // 1_000_000}M"] = {
-                "weights": nw, "fwd_ms": round(f_ms, 4), "bwd_ms": round(b_ms, 4),
+                "weights": nw, "engine": "tcgen05", "fwd_ms": round(f_ms, 4), "bwd_ms": round(b_ms, 4),
+                "fwd_ms_fp32_fma": round(f_fma, 4), "bwd_ms_fp32_fma": round(b_fma, 4),
                 "bytes_per_primitive": bytes_fwd + bytes_bwd,
-                "GBps": round((bytes_fwd + bytes_bwd) * n / ((f_ms + b_ms) * 1e-3) / 1e9, 1),
-                "fwd_fp32_TFLOPs": round(flop_fwd / (f_ms * 1e-3) / 1e12, 2),
-                "bwd_fp32_TFLOPs": round(flop_bwd / (b_ms * 1e-3) / 1e12, 2),
-                "frac_of_fp32_alu_peak": round((flop_fwd + flop_bwd) / ((f_ms + b_ms) * 1e-3) / 1e12 / FP32_ALU_PEAK_TFLOPS, 4),
+                "GBps": round(gbs, 1), "frac_of_hbm_peak": round(gbs / peaks["hbm_gbs"], 4),
+                "fwd_TFLOPs": round(flop_fwd / (f_ms * 1e-3) / 1e12, 2),
+                "bwd_TFLOPs": round(flop_bwd / (b_ms * 1e-3) / 1e12, 2),
+                "fp32_fma_frac_of_fp32_alu_peak": round((flop_fwd + flop_bwd) / ((f_fma + b_fma) * 1e-3) / 1e12 / FP32_ALU_PEAK_TFLOPS, 4),
+                "time_per_weight_over_default_decoder": {
+                    "fwd": round((f_ms / nw) / (dflt["fwd_ms"] / 816), 3), "bwd": round((b_ms / nw) / (dflt["bwd_ms"] / 816), 3)},
                 "Gprimitives_per_s": round(n / ((f_ms + b_ms) * 1e-3) / 1e9, 3)}
             del sc, color, grads, gd, flush
         del dirs, gcol, base

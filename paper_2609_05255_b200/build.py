@@ -11,7 +11,7 @@ CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libgs_b200.so")
 SOURCES = ["gs_api.cu", "gs_preprocess.cu", "gs_sort.cu", "gs_blend.cu", "gs_adam.cu", "gs_prepass.cu",
            "gs_decoder_variants.cu"]
-HEADERS = [os.path.join(CSRC, h) for h in ("gs_device.cuh", "gs_mlp_mma.cuh", "gs_decoder_tc.cuh")] + [os.path.join(_ROOT, "include", "gs.h")]
+HEADERS = [os.path.join(CSRC, h) for h in ("gs_device.cuh", "gs_mlp_mma.cuh", "gs_decoder_tc.cuh", "gs_tcgen05.cuh", "gs_variants_tc.cuh")] + [os.path.join(_ROOT, "include", "gs.h")]
 
 
 def _stale() -> bool:

@@ -48,6 +48,8 @@ __device__ __forceinline__ void variant_inputs(const AppearanceArgs &a, int64_t 
   }
 }
 
+#include "gs_variants_tc.cuh"
+
 // y[o] = sum_i W[o][i] in[i]; the weights are read as shared-memory broadcasts.
 template <int NOUT, int NIN>
 __device__ __forceinline__ void matvec(const float *W, const float in[NIN], float out[NOUT]) {
@@ -309,6 +311,43 @@ int run_bwd(const AppearanceArgs &a, int nfeat, cudaStream_t st) {
   return 2;
 }
 
+int sm_count() {
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
+  return sms;
+}
+
+// The tcgen05 kernels: persistent grids of one full wave.  The occupancy query does not see tensor memory, so the
+// resident CTAs per SM are taken from the three budgets directly: 512 columns of tensor memory, 228 KB of shared
+// memory (1 KB per CTA is the system's), 64 K registers.
+template <int H, int L>
+int run_fwd_tc(const AppearanceArgs &a, int nfeat, cudaStream_t st) {
+  const size_t smem = sizeof(vtc::SmemFwd<H, L>);
+  opt_in(vtc::k_variant_fwd_tc<H, L>, smem);
+  const int64_t tiles = (a.n + tc::kTile - 1) / tc::kTile;
+  const int64_t wave = (int64_t)(H == 16 ? 8 : 4) * sm_count();
+  vtc::k_variant_fwd_tc<H, L><<<(unsigned)(tiles < wave ? tiles : wave), tc::kTile, smem, st>>>(a, nfeat);
+  return 1;
+}
+template <int H, int L>
+int run_bwd_tc(const AppearanceArgs &a, int nfeat, cudaStream_t st) {
+  using D = VarDims<H, L>;
+  const size_t smem = sizeof(vtc::SmemBwd<H, L>);
+  opt_in(vtc::k_variant_bwd_tc<H, L>, smem);
+  int per_sm = 512 / vtc::Shape<H, L>::kColsAlloc;
+  const int by_smem = (int)((228 * 1024) / (smem + 1024));
+  if (by_smem < per_sm) per_sm = by_smem;
+  if (per_sm > (H == 16 ? 4 : 2)) per_sm = H == 16 ? 4 : 2;   // registers: the launch bounds of the kernel
+  if (per_sm < 1) per_sm = 1;
+  const int64_t tiles = (a.n + tc::kTile - 1) / tc::kTile;
+  int64_t wave = (int64_t)per_sm * sm_count();
+  if (wave > kVarPartialBlocks) wave = kVarPartialBlocks;
+  const int blocks = (int)(tiles < wave ? tiles : wave);
+  vtc::k_variant_bwd_tc<H, L><<<blocks, tc::kTile, smem, st>>>(a, nfeat);
+  k_variant_wreduce<<<(D::kNumW + 127) / 128, 128, 0, st>>>(a.w_partials, blocks, D::kNumW, a.g_weights);
+  return 2;
+}
+
 }  // namespace
 
 int variant_num_weights(int hidden, int layers) { return 32 * hidden + (layers - 1) * hidden * hidden + 3 * hidden; }
@@ -325,6 +364,7 @@ size_t variant_partials_floats() { return (size_t)kVarPartialBlocks * VarDims<32
 
 int launch_variant_fwd(int hidden, int layers, int nfeat, const AppearanceArgs &a, cudaStream_t st) {
   if (a.n == 0) return 0;
+  if (a.engine != GS_ENGINE_WARP_MMA && a.deg > 0) { GS_VARIANT_DISPATCH(run_fwd_tc) }
   GS_VARIANT_DISPATCH(run_fwd)
 }
 int launch_variant_bwd(int hidden, int layers, int nfeat, const AppearanceArgs &a, cudaStream_t st) {
@@ -332,6 +372,7 @@ int launch_variant_bwd(int hidden, int layers, int nfeat, const AppearanceArgs &
     cudaMemsetAsync(a.g_weights, 0, sizeof(float) * variant_num_weights(hidden, layers), st);
     return 0;
   }
+  if (a.engine != GS_ENGINE_WARP_MMA && a.deg > 0) { GS_VARIANT_DISPATCH(run_bwd_tc) }
   GS_VARIANT_DISPATCH(run_bwd)
 }
 

@@ -289,6 +289,50 @@ __device__ __forceinline__ float ex2_approx(float x) {
   return y;
 }
 
+// ---- the neural decoder's inputs and residual squashing, shared by every kernel that evaluates it
+__device__ __forceinline__ void unpack_features(const uint4 &raw, float f[8]) {
+  const __half2 *h = reinterpret_cast<const __half2 *>(&raw);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const float2 v = __half22float2(h[j]);
+    f[2 * j] = v.x; f[2 * j + 1] = v.y;
+  }
+}
+__device__ __forceinline__ void load_features(const __half *features, int64_t i, float f[8]) {
+  unpack_features(__ldg(reinterpret_cast<const uint4 *>(features) + i), f);
+}
+
+// Decoder inputs of one Gaussian (Eq. 5, Eq. 6 with k = 1): SH basis of the direction masked by the
+// active degree, then (sin f_j, cos f_j).  The fast sincos is used inside [-pi, pi] (absolute error
+// below 4e-7 there), the accurate one outside.
+__device__ __forceinline__ void decoder_inputs(float dx, float dy, float dz, const float f[8], int deg, float x[32]) {
+  sh_basis(dx, dy, dz, x);
+  const int na = (deg + 1) * (deg + 1);
+  if (na < 16) {
+#pragma unroll
+    for (int k = 0; k < 16; ++k) x[k] = k < na ? x[k] : 0.f;
+  }
+  float big = 0.f;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) big = fmaxf(big, fabsf(f[j]));
+  if (big <= 3.14159265f) {   // one decision for the eight of them: features are O(0.1 .. 1)
+#pragma unroll
+    for (int j = 0; j < 8; ++j) __sincosf(f[j], &x[16 + 2 * j], &x[17 + 2 * j]);
+  } else {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) sincosf(f[j], &x[16 + 2 * j], &x[17 + 2 * j]);
+  }
+}
+
+// tanh(y) = 1 - 2 / (e^{2y} + 1) on the exponential and reciprocal units: absolute error of a few 1e-7 over the
+// whole range (the residual is an absolute colour offset, so that is the error that counts), saturating to +-1.
+__device__ __forceinline__ float tanh_fast(float y) {
+  const float e = ex2_approx(y * 2.885390081777927f);    // 2 log2(e)
+  float r;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(e + 1.f));
+  return fmaf(-2.f, r, 1.f);
+}
+
 #endif  // __CUDACC__
 
 }  // namespace gs
