@@ -315,7 +315,26 @@ def run_ours(args):
                     "stages_ms_per_step": {k: round(v, 4) for k, v in h_stage.items() if v > 0},
                     "what": "the decoder's products on plain fp16 operands (GS_DECODER_HALF, the paper's precision) instead of "
                             "split ones; colours within 2e-3 of the oracle instead of 2e-5 (tests/test_gpu_half_precision.py)"}
-        results[tag] = dict(ms=ms, ms_one=ms_one, ms_streams=ms_streams, graph=graph_note, unfused=unfused, half=half,
+        # the architecture table's other decoders (App. D) through the same step: they run unfused, their appearance
+        # passes on the tcgen05 kernels, the backward on the Gaussians that received a gradient only
+        variants_step = None
+        if tag == "neural" and args.config == 3 and not args.skip_decode:
+            variants_step = {"default_decoder_fused_ms_per_step_single_stream": ms_one}
+            keep = (ds.features, ds.mlp_weights, ds.mlp_hidden, ds.mlp_layers, ds.num_features, r.grads)
+            gen_v = torch.Generator(device=dev); gen_v.manual_seed(909)
+            for hidden, layers, nfeat in ((16, 1, 8), (16, 3, 8), (32, 2, 8), (16, 2, 16)):
+                nw = api.decoder_num_weights(hidden, layers)
+                ds.features = (0.5 * torch.randn((ds.n, nfeat), device=dev, generator=gen_v)).half()
+                ds.mlp_weights = ((torch.rand((nw,), device=dev, generator=gen_v) - 0.5) * (16.0 / hidden) ** 0.5).half()
+                ds.mlp_hidden, ds.mlp_layers, ds.num_features = hidden, layers, nfeat
+                r.grads = api.alloc_grads(ds.n, 1, dev, nfeat, nw)
+                v_one = timed(lambda: step(ds, r), args.steps, args.warmup)
+                v_stage, _ = profile(lambda: step(ds, r), max(1, min(args.steps, 3)))
+                variants_step[f"h{hidden}_l{layers}_f{nfeat}"] = {
+                    "weights": nw, "ms_per_step_single_stream": v_one,
+                    "stages_ms_per_step": {k: round(v, 4) for k, v in v_stage.items() if v > 0}}
+            ds.features, ds.mlp_weights, ds.mlp_hidden, ds.mlp_layers, ds.num_features, r.grads = keep
+        results[tag] = dict(ms=ms, ms_one=ms_one, ms_streams=ms_streams, graph=graph_note, unfused=unfused, half=half, variants_step=variants_step,
                             stage_ms=stage_ms, stage_launches=stage_launches, pairs=pairs,
                             entries=entries, visible=visible, records=records, with_gradient=with_gradient, evaluated=evaluated, composited=composited,
                             warp_steps=warp_steps, warp_steps_idle=warp_steps_idle,
@@ -389,6 +408,7 @@ def run_ours(args):
             "stages_ms_per_step": {k: round(v, 4) for k, v in results["sv"]["stage_ms"].items() if v > 0}},
         "neural_half_precision": results[head].get("half") if head == "neural" else None,
         "separate_pass_step": {t: results[t]["unfused"] for t in results if results[t].get("unfused")} or None,
+        "decoder_variants_step": results[head].get("variants_step") if head == "neural" else None,
         "appearance_decode": decode,
         "adam_update": adam,
         "viewer_prepass": prepass,

@@ -511,24 +511,37 @@ GsStatus gs_render_backward(GsContext *ctx, const GsScene *scene, const GsCamera
   a.g_features = grads->features; a.w_partials = ctx->d_w_partials; a.g_weights = grads->mlp_weights;
   a.gd_in = bw.g_dirs;
   a.flags = bw.flags;
+  a.nfeat = scene->app == GS_APP_NEURAL ? decoder_arch(scene).nfeat : 8;
   a.timeout = ctx->d_counter + 3;
   if (n == 0 && scene->app == GS_APP_NEURAL) {
     const DecoderArch d = decoder_arch(scene);
     return check_cuda(ctx, cudaMemsetAsync(grads->mlp_weights, 0, sizeof(float) * variant_num_weights(d.hidden, d.layers), s), "memset");
   }
+  bool flags_ready = false;
   if (ext && n > 0) {   // the appearance backward as a pass of its own, through dense arrays in the workspace
     AppearanceArgs ap = appearance_args(ctx, scene);
     ap.dirs = bw.dirs; ap.g_color = bw.g_color; ap.mask = proj->tiles_touched;
     ap.g_base = grads->base_color; ap.g_sh_rest = scene->app == GS_APP_SV ? grads->sv_sites : grads->sh_rest;
     ap.g_features = grads->features; ap.g_dirs = bw.g_dirs;
     ap.w_partials = ctx->d_w_partials; ap.g_weights = grads->mlp_weights;
+    // A decoder variant on the tcgen05 kernels works on the Gaussians that received a gradient only: the flag bits
+    // (and the zero rows of everyone else) are taken first, and serve the projection backward below as well.
+    flags_ready = scene->app == GS_APP_NEURAL && !default_decoder(scene) && ctx->decoder_engine != GS_ENGINE_WARP_MMA && scene->active_degree > 0;
     StageTimer t(ctx, GS_STAGE_APPEARANCE_BWD, s);
-    t.done(launch_unfused_prepare(n, scene->means, cd, g2d, proj->tiles_touched, bw.dirs, bw.g_color, s) +
-           run_appearance_bwd(scene, ap, s));
+    int launches = 0;
+    if (flags_ready) {   // directions and dL/dcolor are taken from the means and the 2D gradient rows in the kernel itself
+      launches = launch_bwd_flags(a, true, s);
+      ap.flags = bw.flags;
+      ap.means = scene->means; ap.g2d = g2d;
+      ap.oc[0] = cd.oc[0]; ap.oc[1] = cd.oc[1]; ap.oc[2] = cd.oc[2];
+    } else {
+      launches = launch_unfused_prepare(n, scene->means, cd, g2d, proj->tiles_touched, bw.dirs, bw.g_color, s);
+    }
+    t.done(launches + run_appearance_bwd(scene, ap, s));
   }
   {
     StageTimer t(ctx, GS_STAGE_PREPROCESS_BWD, s);
-    t.done(launch_preprocess_bwd(ext ? kAppExternal : kernel_app(scene), a, cd, s));
+    t.done(launch_preprocess_bwd(ext ? kAppExternal : kernel_app(scene), a, cd, s, flags_ready));
   }
   return check_cuda(ctx, cudaGetLastError(), "render_backward launch");
 }

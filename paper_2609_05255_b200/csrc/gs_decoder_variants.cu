@@ -275,12 +275,34 @@ __global__ void __launch_bounds__(kVarBlock) k_variant_bwd(AppearanceArgs a, int
   }
 }
 
-__global__ void k_variant_wreduce(const float *__restrict__ partials, int nblocks, int nw, float *__restrict__ out) {
-  const int k = blockIdx.x * blockDim.x + threadIdx.x;
-  if (k >= nw) return;
+// Deterministic sum of the per-block partials: 32 weights per CTA, the rows shared out over sixteen groups of threads
+// (each sums every sixteenth row, in order, four loads in flight), the sixteen sums added in a fixed order.
+constexpr int kVarReduceGroups = 16;
+__global__ void __launch_bounds__(32 * kVarReduceGroups) k_variant_wreduce(const float *__restrict__ partials, int nblocks, int nw,
+                                                                           float *__restrict__ out) {
+  __shared__ float s_part[kVarReduceGroups][32];
+  const int k = blockIdx.x * 32 + threadIdx.x, grp = threadIdx.y;
   float s = 0.f;
-  for (int b = 0; b < nblocks; ++b) s += partials[(size_t)b * nw + k];
-  out[k] = s;
+  if (k < nw) {
+    int b = grp;
+    for (; b + 3 * kVarReduceGroups < nblocks; b += 4 * kVarReduceGroups) {
+      const float p0 = partials[(size_t)b * nw + k], p1 = partials[(size_t)(b + kVarReduceGroups) * nw + k],
+                  p2 = partials[(size_t)(b + 2 * kVarReduceGroups) * nw + k], p3 = partials[(size_t)(b + 3 * kVarReduceGroups) * nw + k];
+      s += p0; s += p1; s += p2; s += p3;
+    }
+    for (; b < nblocks; b += kVarReduceGroups) s += partials[(size_t)b * nw + k];
+  }
+  s_part[grp][threadIdx.x] = s;
+  __syncthreads();
+  if (grp == 0 && k < nw) {
+    float t = 0.f;
+#pragma unroll
+    for (int q = 0; q < kVarReduceGroups; ++q) t += s_part[q][threadIdx.x];
+    out[k] = t;
+  }
+}
+inline void launch_variant_wreduce(const float *partials, int nblocks, int nw, float *out, cudaStream_t st) {
+  k_variant_wreduce<<<(nw + 31) / 32, dim3(32, kVarReduceGroups), 0, st>>>(partials, nblocks, nw, out);
 }
 
 template <class K>
@@ -307,7 +329,7 @@ int run_bwd(const AppearanceArgs &a, int nfeat, cudaStream_t st) {
     wave = per_sm * sms < kVarPartialBlocks ? per_sm * sms : kVarPartialBlocks;
   const int blocks = (int)(chunks < wave ? chunks : wave);
   k_variant_bwd<H, L><<<blocks, kVarBlock, smem, st>>>(a, nfeat);
-  k_variant_wreduce<<<(D::kNumW + 127) / 128, 128, 0, st>>>(a.w_partials, blocks, D::kNumW, a.g_weights);
+  launch_variant_wreduce(a.w_partials, blocks, D::kNumW, a.g_weights, st);
   return 2;
 }
 
@@ -333,9 +355,11 @@ template <int H, int L>
 int run_bwd_tc(const AppearanceArgs &a, int nfeat, cudaStream_t st) {
   using D = VarDims<H, L>;
   const size_t smem = sizeof(vtc::SmemBwd<H, L>);
-  opt_in(vtc::k_variant_bwd_tc<H, L>, smem);
+  const bool gather = a.flags != nullptr;
+  opt_in(vtc::k_variant_bwd_tc<H, L, false>, smem);
+  opt_in(vtc::k_variant_bwd_tc<H, L, true>, smem);
   int per_sm = 512 / vtc::Shape<H, L>::kColsAlloc;
-  const int by_smem = (int)((228 * 1024) / (smem + 1024));
+  const int by_smem = (int)((228 * 1024) / (smem + 1024 + (gather ? sizeof(uint32_t) * vtc::kGatherQueue + 64 : 0)));
   if (by_smem < per_sm) per_sm = by_smem;
   if (per_sm > (H == 16 ? 4 : 2)) per_sm = H == 16 ? 4 : 2;   // registers: the launch bounds of the kernel
   if (per_sm < 1) per_sm = 1;
@@ -343,8 +367,9 @@ int run_bwd_tc(const AppearanceArgs &a, int nfeat, cudaStream_t st) {
   int64_t wave = (int64_t)per_sm * sm_count();
   if (wave > kVarPartialBlocks) wave = kVarPartialBlocks;
   const int blocks = (int)(tiles < wave ? tiles : wave);
-  vtc::k_variant_bwd_tc<H, L><<<blocks, tc::kTile, smem, st>>>(a, nfeat);
-  k_variant_wreduce<<<(D::kNumW + 127) / 128, 128, 0, st>>>(a.w_partials, blocks, D::kNumW, a.g_weights);
+  if (gather) vtc::k_variant_bwd_tc<H, L, true><<<blocks, tc::kTile, smem, st>>>(a, nfeat);
+  else vtc::k_variant_bwd_tc<H, L, false><<<blocks, tc::kTile, smem, st>>>(a, nfeat);
+  launch_variant_wreduce(a.w_partials, blocks, D::kNumW, a.g_weights, st);
   return 2;
 }
 

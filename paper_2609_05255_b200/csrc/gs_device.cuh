@@ -66,11 +66,16 @@ struct PreprocessBwdArgs {
   unsigned long long *timeout; // set to 1 if a bounded wait on a bulk copy ran out (never expected)
   const float *gd_in;          // kAppExternal only: [n,3] dL/dd from the separate appearance backward
   uint32_t *flags;             // scratch, one bit per Gaussian: it received a gradient in this view
+  int nfeat;                   // features per Gaussian of g_features (8, or 16 for the raw-feature decoder variants)
   float *g_means, *g_log_scales, *g_quats, *g_logits, *g_base, *g_sh_rest, *g_features;
   float *w_partials;           // [kWgradBlocks, 816]
   float *g_weights;            // [816]
 };
-int launch_preprocess_bwd(int app, const PreprocessBwdArgs &a, const CamDev &cam, cudaStream_t st);
+// flags_ready (kAppExternal): launch_bwd_flags has run on these arguments already.
+int launch_preprocess_bwd(int app, const PreprocessBwdArgs &a, const CamDev &cam, cudaStream_t st, bool flags_ready = false);
+// The flag bits (who received a gradient) and the zero rows of everyone else: projection gradients, and with
+// appearance_rows also base colour and features.
+int launch_bwd_flags(const PreprocessBwdArgs &a, bool appearance_rows, cudaStream_t st);
 
 struct AppearanceArgs {
   int64_t n;
@@ -85,6 +90,10 @@ struct AppearanceArgs {
   int engine;                  // GsDecoderEngine for the default neural decoder: warp-level MMA, tcgen05, or per kernel the faster
   const uint32_t *mask;        // optional [n]: Gaussians with a zero here are skipped (no colour written; zero
                                // gradient rows written); the tiles-touched array in the unfused step
+  const uint32_t *flags;       // optional, backward of the decoder variants on tcgen05: one bit per Gaussian; only the
+                               // flagged ones are worked on (gathered into full tiles) and written
+  const float *means, *g2d;    // optional, with flags (the unfused step): view directions from the means and the camera
+  float oc[3];                 // centre oc, dL/dcolor from columns 0..2 of the [n,12] rows g2d, instead of dirs / g_color
 };
 int launch_appearance_fwd(int app, const AppearanceArgs &a, cudaStream_t st);
 int launch_appearance_bwd(int app, const AppearanceArgs &a, cudaStream_t st);

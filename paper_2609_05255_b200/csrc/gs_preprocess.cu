@@ -937,9 +937,9 @@ __global__ void __launch_bounds__(kFlagThreads) k_bwd_flags(PreprocessBwdArgs a)
       a.g_logits[i] = 0.f;
       if (kBase) store3(a.g_base, i, 0.f, 0.f, 0.f);
       if (kFeatures) {
-        float4 *gfp = reinterpret_cast<float4 *>(a.g_features) + 2 * i;
-        gfp[0] = make_float4(0.f, 0.f, 0.f, 0.f);
-        gfp[1] = make_float4(0.f, 0.f, 0.f, 0.f);
+        const int quads = a.nfeat == 16 ? 4 : 2;
+        float4 *gfp = reinterpret_cast<float4 *>(a.g_features) + quads * i;
+        for (int q = 0; q < quads; ++q) gfp[q] = make_float4(0.f, 0.f, 0.f, 0.f);
       }
     }
   }
@@ -1326,7 +1326,15 @@ int launch_unfused_prepare(int64_t n, const float *means, const CamDev &cam, con
   return 1;
 }
 
-int launch_preprocess_bwd(int app, const PreprocessBwdArgs &a, const CamDev &cam, cudaStream_t st) {
+int launch_bwd_flags(const PreprocessBwdArgs &a, bool appearance_rows, cudaStream_t st) {
+  if (a.n == 0) return 0;
+  const int blocks = (int)((a.n + kFlagThreads - 1) / kFlagThreads);
+  if (appearance_rows) k_bwd_flags<true, true><<<blocks, kFlagThreads, 0, st>>>(a);
+  else k_bwd_flags<false, false><<<blocks, kFlagThreads, 0, st>>>(a);
+  return 1;
+}
+
+int launch_preprocess_bwd(int app, const PreprocessBwdArgs &a, const CamDev &cam, cudaStream_t st, bool flags_ready) {
   if (app == GS_APP_SH) {
     if (a.n == 0) return 0;
     opt_in_smem(k_preprocess_bwd<GS_APP_SH>, kBwdSmemSH);
@@ -1339,10 +1347,10 @@ int launch_preprocess_bwd(int app, const PreprocessBwdArgs &a, const CamDev &cam
     return 1;
   } else if (app == kAppExternal) {
     if (a.n == 0) return 0;
-    k_bwd_flags<false, false><<<(int)((a.n + kFlagThreads - 1) / kFlagThreads), kFlagThreads, 0, st>>>(a);
+    if (!flags_ready) launch_bwd_flags(a, false, st);
     const int wave = resident_blocks<k_preprocess_bwd_sparse<kAppExternal>>(sizeof(mlp::Weights), 1 << 20), chunks = grid_for(a.n);
     k_preprocess_bwd_sparse<kAppExternal><<<chunks < wave ? chunks : wave, kBlock, sizeof(mlp::Weights), st>>>(a, cam);
-    return 2;
+    return flags_ready ? 1 : 2;
   } else {
     if (app == kAppNeuralHalf) {
       opt_in_smem(k_preprocess_bwd_sparse<kAppNeuralHalf>, kBwdSmemNN);

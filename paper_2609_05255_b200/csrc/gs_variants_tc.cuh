@@ -233,7 +233,14 @@ struct __align__(128) SmemBwd {
   uint32_t failed;
 };
 
-template <int H, int L>
+// kGather: only the Gaussians whose bit is set in a.flags are worked on and written.  Every CTA takes one contiguous
+// run of flag words, reads it 32 words at a time (thread t looks at byte t % 4 of word t / 4, an exclusive scan over the
+// CTA gives its place in a queue in shared memory, it writes the indices of its set bits there: index order, the same
+// from run to run) and runs a tile whenever 128 indices are queued, and once more for what is left.
+constexpr int kGatherWords = tc::kTile / 4;               // flag words per round
+constexpr int kGatherQueue = 2 * 32 * kGatherWords;       // a power of two above 32 kGatherWords + 127
+
+template <int H, int L, bool kGather>
 __global__ void __launch_bounds__(tc::kTile, H == 16 ? 4 : 2) k_variant_bwd_tc(AppearanceArgs a, int nfeat) {
   using S_t = SmemBwd<H, L>;
   using Sh = Shape<H, L>;
@@ -278,10 +285,8 @@ __global__ void __launch_bounds__(tc::kTile, H == 16 ? 4 : 2) k_variant_bwd_tc(A
     ++phase;
     tc::fence_after_sync();
   };
-  const int64_t ntiles = (a.n + tc::kTile - 1) / tc::kTile;
-  for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
-    const int64_t i = tile * tc::kTile + tid;
-    const bool exists = i < a.n;
+  // one tile: thread t works on Gaussian i (exists: it has one)
+  auto do_tile = [&](const int64_t i, const bool exists) {
     const bool in = exists && (!a.mask || __ldg(a.mask + i) != 0u);
     float d[3] = {0.f, 0.f, 1.f}, base[3] = {0.f, 0.f, 0.f}, gcol[3] = {0.f, 0.f, 0.f};
     float xs[16];                        // inputs 16..31 ((sin, cos) pairs or raw features), needed again for dL/df
@@ -289,7 +294,17 @@ __global__ void __launch_bounds__(tc::kTile, H == 16 ? 4 : 2) k_variant_bwd_tc(A
       float x[32];
       if (in) {
 #pragma unroll
-        for (int c = 0; c < 3; ++c) { d[c] = __ldg(a.dirs + 3 * i + c); base[c] = __ldg(a.base_color + 3 * i + c); gcol[c] = __ldg(a.g_color + 3 * i + c); }
+        for (int c = 0; c < 3; ++c) base[c] = __ldg(a.base_color + 3 * i + c);
+        if (kGather && a.g2d) {          // inside the step: the direction as the forward took it, dL/dcolor where the blend left it
+          const float vx = __ldg(a.means + 3 * i) - a.oc[0], vy = __ldg(a.means + 3 * i + 1) - a.oc[1], vz = __ldg(a.means + 3 * i + 2) - a.oc[2];
+          const float vi = rsqrtf(vx * vx + vy * vy + vz * vz);
+          d[0] = vx * vi; d[1] = vy * vi; d[2] = vz * vi;
+          const float4 ga = __ldg(reinterpret_cast<const float4 *>(a.g2d) + 3 * i);
+          gcol[0] = ga.x; gcol[1] = ga.y; gcol[2] = ga.z;
+        } else {
+#pragma unroll
+          for (int c = 0; c < 3; ++c) { d[c] = __ldg(a.dirs + 3 * i + c); gcol[c] = __ldg(a.g_color + 3 * i + c); }
+        }
         inputs(a, i, nfeat, d, x);
       } else {
 #pragma unroll
@@ -391,6 +406,53 @@ __global__ void __launch_bounds__(tc::kTile, H == 16 ? 4 : 2) k_variant_bwd_tc(A
         if (k < na) sh_grad_acc(k, d[0], d[1], d[2], gx[k], ax, ay, az);
       a.g_dirs[3 * i] = ax; a.g_dirs[3 * i + 1] = ay; a.g_dirs[3 * i + 2] = az;
     }
+  };
+  if constexpr (!kGather) {
+    const int64_t ntiles = (a.n + tc::kTile - 1) / tc::kTile;
+    for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+      const int64_t i = tile * tc::kTile + tid;
+      do_tile(i, i < a.n);
+    }
+  } else {
+    __shared__ uint32_t s_queue[kGatherQueue];
+    __shared__ int s_warp_count[tc::kTile / 32];
+    constexpr int kMask = kGatherQueue - 1;
+    const int lane = tid & 31;
+    int q_head = 0, q_count = 0;         // the same in every thread
+    const int64_t nwords = (a.n + 31) / 32, per_cta = (nwords + gridDim.x - 1) / gridDim.x;
+    const int64_t w_begin = min(nwords, (int64_t)blockIdx.x * per_cta), w_end = min(nwords, w_begin + per_cta);
+    for (int64_t w0 = w_begin; w0 < w_end; w0 += kGatherWords) {
+      const int64_t w = w0 + (tid >> 2);
+      const uint32_t byte = w < w_end ? (__ldg(a.flags + w) >> (8 * (tid & 3))) & 255u : 0u;
+      const int cnt = __popc(byte);
+      int incl = cnt;
+#pragma unroll
+      for (int sft = 1; sft < 32; sft <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, sft);
+        if (lane >= sft) incl += t;
+      }
+      if (lane == 31) s_warp_count[warp] = incl;
+      __syncthreads();
+      int offset = incl - cnt, total = 0;
+#pragma unroll
+      for (int ww = 0; ww < tc::kTile / 32; ++ww) { const int c = s_warp_count[ww]; offset += ww < warp ? c : 0; total += c; }
+      uint32_t bits = byte;
+      const uint32_t row0 = (uint32_t)(w * 32 + 8 * (tid & 3));
+      for (int slot = q_head + q_count + offset; bits; ++slot) {
+        const int b = __ffs(bits) - 1;
+        bits &= bits - 1u;
+        s_queue[slot & kMask] = row0 + (uint32_t)b;
+      }
+      __syncthreads();
+      q_count += total;
+      while (q_count >= tc::kTile) {
+        do_tile((int64_t)s_queue[(q_head + tid) & kMask], true);
+        q_head = (q_head + tc::kTile) & kMask;
+        q_count -= tc::kTile;
+        __syncthreads();
+      }
+    }
+    if (q_count > 0) do_tile(tid < q_count ? (int64_t)s_queue[(q_head + tid) & kMask] : 0, tid < q_count);
   }
   // ---- this CTA's partial of the weight gradient.  In block b, thread t holds the row of column 128 b + t of
   // [X | h_1 | ...]; of that row it reads its partner's columns and adds the high- and low-half columns.

@@ -84,3 +84,33 @@ def test_unfused_path_uses_the_same_kernels(oracle):
     sc = copy.copy(w.scene)
     sc.separate_pass = 1
     _check(oracle, sc, cam, _window_gradient(cam, 7, 100, 60, 40))
+
+
+@pytest.mark.parametrize("arch", [(16, 1, 8), (16, 3, 8), (32, 2, 8), (16, 2, 16), (32, 3, 16)], ids=lambda a: "h%d_l%d_f%d" % a)
+@pytest.mark.parametrize("n", [129, 30_000])
+def test_decoder_variants_work_on_the_flagged_gaussians_only(oracle, arch, n):
+    """A decoder of another size runs through the step unfused, and its backward (the tcgen05 kernels) gathers the
+    Gaussians that received a gradient into tiles of 128: same check, gradient in a small window, rows of 8 and of 16
+    features."""
+    hidden, layers, nfeat = arch
+    w = scenes.config3(scenes.APP_NEURAL, n=n, width=320, height=208, views=1)
+    cam = w.cameras[0]
+    sc = w.scene
+    rng = np.random.default_rng(np.random.PCG64(777))
+    _, sc.features, sc.mlp_weights = scenes.draw_neural_appearance(rng, sc.n, hidden, layers, nfeat)
+    sc.mlp_hidden, sc.mlp_layers = hidden, layers
+    gpu, skipped = _check(oracle, sc, cam, _window_gradient(cam, 3, 150, 90, 24))
+    assert skipped > 0.5 * n
+    assert gpu.grads.features.shape == (n, nfeat)
+
+
+def test_decoder_variant_with_a_zero_upstream_gradient(oracle):
+    w = scenes.config3(scenes.APP_NEURAL, n=5_003, width=320, height=208, views=1)
+    cam = w.cameras[0]
+    sc = w.scene
+    rng = np.random.default_rng(np.random.PCG64(778))
+    _, sc.features, sc.mlp_weights = scenes.draw_neural_appearance(rng, sc.n, 32, 2, 16)
+    sc.mlp_hidden, sc.mlp_layers = 32, 2
+    gpu = run_gpu(sc, cam, np.zeros((3, cam.height, cam.width), np.float32))
+    for nm in grad_names(sc.app):
+        assert np.all(getattr(gpu.grads, nm) == 0), nm
