@@ -330,8 +330,11 @@ def run_ours(args):
                 r.grads = api.alloc_grads(ds.n, 1, dev, nfeat, nw)
                 v_one = timed(lambda: step(ds, r), args.steps, args.warmup)
                 v_stage, _ = profile(lambda: step(ds, r), max(1, min(args.steps, 3)))
+                api.gs_set_decoder_engine(ctx, api.GS_ENGINE_WARP_MMA)   # the fp32 kernels, dense over all Gaussians
+                v_fma = timed(lambda: step(ds, r), args.steps, args.warmup)
+                api.gs_set_decoder_engine(ctx, api.GS_ENGINE_AUTO)
                 variants_step[f"h{hidden}_l{layers}_f{nfeat}"] = {
-                    "weights": nw, "ms_per_step_single_stream": v_one,
+                    "weights": nw, "ms_per_step_single_stream": v_one, "ms_per_step_single_stream_fp32_fma_dense": v_fma,
                     "stages_ms_per_step": {k: round(v, 4) for k, v in v_stage.items() if v > 0}}
             ds.features, ds.mlp_weights, ds.mlp_hidden, ds.mlp_layers, ds.num_features, r.grads = keep
         results[tag] = dict(ms=ms, ms_one=ms_one, ms_streams=ms_streams, graph=graph_note, unfused=unfused, half=half, variants_step=variants_step,
