@@ -377,8 +377,12 @@ GsStatus gs_profile_enable(GsContext *ctx, int enable);
  * split operands and, from 2,000,000 Gaussians on, the forward on tcgen05; smaller forwards and the
  * plain-fp16 backward on warp-level MMA.
  * Same arithmetic (fp16 operands, split or plain, fp32 accumulation) and the same tolerances either
- * way; per-Gaussian results differ only by the order of the fp32 sums.  The paper has no counterpart
- * of this call.  Returns GS_ERR_INVALID_ARG for any other value.  Takes effect for the calls issued
+ * way; per-Gaussian results differ only by the order of the fp32 sums.
+ * A decoder of another size (GsScene.mlp_hidden / mlp_layers / num_features, App. D's architecture
+ * table) runs on tcgen05 kernels of the same construction under GS_ENGINE_TCGEN05 and GS_ENGINE_AUTO -
+ * inside gs_render_backward they work on the Gaussians that received a gradient only - and on fp32
+ * FMA kernels (dense over all Gaussians) under GS_ENGINE_WARP_MMA; same tolerances.  The paper has
+ * no counterpart of this call.  Returns GS_ERR_INVALID_ARG for any other value.  Takes effect for the calls issued
  * after it. */
 typedef enum GsDecoderEngine { GS_ENGINE_WARP_MMA = 0, GS_ENGINE_TCGEN05 = 1, GS_ENGINE_AUTO = 2 } GsDecoderEngine;
 GsStatus gs_set_decoder_engine(GsContext *ctx, int engine);

@@ -1,9 +1,9 @@
 // The decoder variants of the paper's architecture table (App. D): 1 to 3 hidden layers of 16 or 32
 // neurons, 8 frequency-encoded or 16 raw features, evaluated in the separate-pass path (the path the paper
-// calls "without fusion").  Plain fp32 FMAs with the weights in shared memory: these are the ablation
-// configurations, not the hot path - the default decoder (16 / 2 / 8) runs on the tensor-core kernels of
-// gs_preprocess.cu.  One thread per Gaussian.  The weight gradient is a contraction over Gaussians: each warp
-// stages the inputs and output gradients of its 32 Gaussians in shared memory, every lane owns every 32nd
+// calls "without fusion").  Two engines: the tcgen05 kernels of gs_variants_tc.cuh (the default), and the
+// kernels of this file, plain fp32 FMAs with the weights in shared memory, one thread per Gaussian (the second
+// engine, and the path of degree 0, where nothing is decoded).  In the fp32 backward the weight gradient - a
+// contraction over Gaussians - is taken per warp: it stages the inputs and output gradients of its 32 Gaussians in shared memory, every lane owns every 32nd
 // weight of the layer and sums its 32 products, and the per-warp sums (kept in shared memory, one owner per
 // element, so no atomics) leave as per-block partials that a last kernel adds up in a fixed order.
 #include <cuda_fp16.h>
@@ -347,7 +347,7 @@ int run_fwd_tc(const AppearanceArgs &a, int nfeat, cudaStream_t st) {
   const size_t smem = sizeof(vtc::SmemFwd<H, L>);
   opt_in(vtc::k_variant_fwd_tc<H, L>, smem);
   const int64_t tiles = (a.n + tc::kTile - 1) / tc::kTile;
-  const int64_t wave = (int64_t)(H == 16 ? 8 : 4) * sm_count();
+  const int64_t wave = (int64_t)(H == 16 ? 8 : 7) * sm_count();   // 59 and 71 registers per thread
   vtc::k_variant_fwd_tc<H, L><<<(unsigned)(tiles < wave ? tiles : wave), tc::kTile, smem, st>>>(a, nfeat);
   return 1;
 }

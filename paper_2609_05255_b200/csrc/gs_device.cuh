@@ -98,7 +98,8 @@ struct AppearanceArgs {
 int launch_appearance_fwd(int app, const AppearanceArgs &a, cudaStream_t st);
 int launch_appearance_bwd(int app, const AppearanceArgs &a, cudaStream_t st);
 
-// Decoder variants (1-3 hidden layers of 16 or 32 neurons, 8 encoded or 16 raw features): fp32 kernels.
+// Decoder variants (1-3 hidden layers of 16 or 32 neurons, 8 encoded or 16 raw features): tcgen05 kernels unless
+// a.engine is GS_ENGINE_WARP_MMA or the active degree is 0, fp32 FMA kernels then.
 int variant_num_weights(int hidden, int layers);
 size_t variant_partials_floats();   // floats of per-block weight-gradient partials the backward needs
 int launch_variant_fwd(int hidden, int layers, int nfeat, const AppearanceArgs &a, cudaStream_t st);
