@@ -288,15 +288,23 @@ __device__ __forceinline__ void weight_grad_flush(const mlp::WeightGrad &dW, flo
 __device__ __forceinline__ void reload_fence() { asm volatile("" ::: "memory"); }
 
 // Deterministic final reduction of the per-block partials: 32 weights per CTA, the rows shared out over
-// eight groups of threads (each sums every eighth row, in order), the eight sums added in a fixed order.
-constexpr int kReduceGroups = 8;
+// sixteen groups of threads (each sums every sixteenth row, in order, four loads in flight), the sixteen sums added
+// in a fixed order.
+constexpr int kReduceGroups = 16;
 __global__ void __launch_bounds__(32 * kReduceGroups) k_wgrad_reduce(const float *__restrict__ partials, int nblocks,
                                                                     float *__restrict__ out) {
   __shared__ float s_part[kReduceGroups][32];
   const int k = blockIdx.x * 32 + threadIdx.x, grp = threadIdx.y;
   float s = 0.f;
-  if (k < GS_MLP_WEIGHTS)
-    for (int b = grp; b < nblocks; b += kReduceGroups) s += partials[(size_t)b * GS_MLP_WEIGHTS + k];
+  if (k < GS_MLP_WEIGHTS) {
+    int b = grp;
+    for (; b + 3 * kReduceGroups < nblocks; b += 4 * kReduceGroups) {
+      const float p0 = partials[(size_t)b * GS_MLP_WEIGHTS + k], p1 = partials[(size_t)(b + kReduceGroups) * GS_MLP_WEIGHTS + k],
+                  p2 = partials[(size_t)(b + 2 * kReduceGroups) * GS_MLP_WEIGHTS + k], p3 = partials[(size_t)(b + 3 * kReduceGroups) * GS_MLP_WEIGHTS + k];
+      s += p0; s += p1; s += p2; s += p3;
+    }
+    for (; b < nblocks; b += kReduceGroups) s += partials[(size_t)b * GS_MLP_WEIGHTS + k];
+  }
   s_part[grp][threadIdx.x] = s;
   __syncthreads();
   if (grp == 0 && k < GS_MLP_WEIGHTS) {
