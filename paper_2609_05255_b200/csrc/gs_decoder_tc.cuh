@@ -11,8 +11,8 @@
 // values: no fragment shuffling at all.  The backward (further down) adds the transposed products and takes the
 // weight gradients as products over the tile's rows, accumulated in tensor memory.
 //
-// Single-GPU code: no cluster, no multicast of any kind.  Every wait on the mbarrier is bounded; a wait that runs
-// out sets *timeout (read by gs_async_status), the CTA stops issuing MMAs, runs its loops to the end without
+// Single-GPU code: every CTA works alone (no cluster, no copy or commit addressed to more than one CTA).  Every wait
+// on the mbarrier is bounded; a wait that runs out sets *timeout (read by gs_async_status), the CTA stops issuing MMAs, runs its loops to the end without
 // waiting, frees its tensor memory and returns.
 #pragma once
 

@@ -1,8 +1,8 @@
 // tcgen05 building blocks shared by the decoder kernels on the 5th-generation tensor cores: instruction and
 // shared-memory descriptors for operands in the canonical layouts without swizzle, the MMA / commit / tensor-memory
 // load wrappers, the bounded mbarrier wait and the operand-row writer with high / low fp16 halves.  Included inside
-// namespace gs's unnamed namespace by the translation units that hold such kernels.  Single-GPU code: no cluster
-// and no multicast of any kind.
+// namespace gs's unnamed namespace by the translation units that hold such kernels.  Single-GPU code: every CTA
+// works alone (no cluster, no copy or commit addressed to more than one CTA).
 #pragma once
 #include <cuda_fp16.h>
 #include <stdint.h>

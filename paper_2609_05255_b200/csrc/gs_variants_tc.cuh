@@ -16,7 +16,7 @@
 // same whatever its N, so one or two wide products per 16 Gaussians replace a dozen small ones; the blocks that pair
 // non-partners are computed and ignored.  The accumulators stay in tensor memory across all tiles of the CTA.
 //
-// Single-GPU code: no cluster, no multicast.  Every wait is bounded; one that runs out sets *timeout (read by
+// Single-GPU code: every CTA works alone (no cluster).  Every wait is bounded; one that runs out sets *timeout (read by
 // gs_async_status), the CTA stops issuing MMAs, runs its loops to the end without waiting, frees its tensor memory
 // and returns.
 #pragma once
