@@ -319,9 +319,11 @@ def run_ours(args):
         # passes on the tcgen05 kernels, the backward on the Gaussians that received a gradient only
         variants_step = None
         if tag == "neural" and args.config == 3 and not args.skip_decode:
-            variants_step = {"default_decoder_fused_ms_per_step_single_stream": ms_one}
+            variants_step = {"default_decoder_fused_ms_per_step": ms_streams, "default_decoder_fused_ms_per_step_single_stream": ms_one}
             keep = (ds.features, ds.mlp_weights, ds.mlp_hidden, ds.mlp_layers, ds.num_features, r.grads)
             gen_v = torch.Generator(device=dev); gen_v.manual_seed(909)
+            rs_v = ([r] + [api.Renderer(c, ds.n, WIDTH, HEIGHT, app, pair_capacity=r.pair_capacity) for c in lane_ctx[1:]]
+                    if views > 1 and n_lanes > 1 else None)
             for hidden, layers, nfeat in ((16, 1, 8), (16, 3, 8), (32, 2, 8), (16, 2, 16)):
                 nw = api.decoder_num_weights(hidden, layers)
                 ds.features = (0.5 * torch.randn((ds.n, nfeat), device=dev, generator=gen_v)).half()
@@ -330,13 +332,22 @@ def run_ours(args):
                 r.grads = api.alloc_grads(ds.n, 1, dev, nfeat, nw)
                 v_one = timed(lambda: step(ds, r), args.steps, args.warmup)
                 v_stage, _ = profile(lambda: step(ds, r), max(1, min(args.steps, 3)))
+                v_streams = None
+                if rs_v:                                               # the views on the lanes' streams, as the headline runs
+                    for rr in rs_v[1:]:
+                        rr.grads = api.alloc_grads(ds.n, 1, dev, nfeat, nw)
+                    v_streams = timed(lambda: step_two_streams(ds, rs_v), args.steps, args.warmup)
+                    for c, s_ in zip(lane_ctx, lanes):
+                        api.gs_async_status(c, s_)
                 api.gs_set_decoder_engine(ctx, api.GS_ENGINE_WARP_MMA)   # the fp32 kernels, dense over all Gaussians
                 v_fma = timed(lambda: step(ds, r), args.steps, args.warmup)
                 api.gs_set_decoder_engine(ctx, api.GS_ENGINE_AUTO)
                 variants_step[f"h{hidden}_l{layers}_f{nfeat}"] = {
-                    "weights": nw, "ms_per_step_single_stream": v_one, "ms_per_step_single_stream_fp32_fma_dense": v_fma,
+                    "weights": nw, "ms_per_step": v_streams, "ms_per_step_single_stream": v_one,
+                    "ms_per_step_single_stream_fp32_fma_dense": v_fma,
                     "stages_ms_per_step": {k: round(v, 4) for k, v in v_stage.items() if v > 0}}
             ds.features, ds.mlp_weights, ds.mlp_hidden, ds.mlp_layers, ds.num_features, r.grads = keep
+            del rs_v
         results[tag] = dict(ms=ms, ms_one=ms_one, ms_streams=ms_streams, graph=graph_note, unfused=unfused, half=half, variants_step=variants_step,
                             stage_ms=stage_ms, stage_launches=stage_launches, pairs=pairs,
                             entries=entries, visible=visible, records=records, with_gradient=with_gradient, evaluated=evaluated, composited=composited,
