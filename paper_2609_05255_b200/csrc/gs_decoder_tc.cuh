@@ -111,6 +111,13 @@ __global__ void __launch_bounds__(kTile) k_appearance_fwd_tc(AppearanceArgs a) {
     const bool in = i < a.n && (!a.mask || __ldg(a.mask + i) != 0u);
     float base[3] = {0.f, 0.f, 0.f};
     {
+      const int64_t nx = i + (int64_t)gridDim.x * kTile;     // this thread's row of the CTA's next tile
+      if (nx < a.n) {
+        prefetch_l2(a.dirs + 3 * nx); prefetch_l2(a.base_color + 3 * nx);
+        prefetch_l2(reinterpret_cast<const uint4 *>(a.features) + nx);
+      }
+    }
+    {
       float x[32];
       if (in) {
         float d[3], f[8];
