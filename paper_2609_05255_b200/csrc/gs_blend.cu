@@ -100,6 +100,7 @@ __global__ void __launch_bounds__(kThreads) k_blend_fwd(CamDev cam, const uint32
                                                         const float *__restrict__ color, uint32_t *__restrict__ sorted_tiles,
                                                         float *__restrict__ image,
                                                         float *__restrict__ final_T, uint32_t *__restrict__ n_contrib) {
+  dependency_wait();
   __shared__ float4 s_xyab[kBatch];
   __shared__ float2 s_co[kBatch];
   __shared__ float4 s_rgb[kBatch];
@@ -496,8 +497,8 @@ int launch_blend_fwd(const CamDev &cam, const uint32_t *ranges, const uint32_t *
                      const float *mean2d,
                      const float *conic_opacity, const float *color, uint32_t *sorted_tiles, float *image, float *final_T,
                      uint32_t *n_contrib, cudaStream_t st) {
-  k_blend_fwd<<<cam.gx * cam.gy, kThreads, 0, st>>>(cam, ranges, order, vals, mean2d, conic_opacity, color, sorted_tiles, image,
-                                                    final_T, n_contrib);
+  launch_chained(k_blend_fwd, cam.gx * cam.gy, kThreads, 0, st, cam, ranges, order, vals, mean2d, conic_opacity, color, sorted_tiles, image,
+                 final_T, n_contrib);
   return 1;
 }
 

@@ -446,6 +446,7 @@ struct RowStage {
 
 template <int APP>
 __global__ void __launch_bounds__(kBlock) k_preprocess_fwd(PreprocessArgs a, CamDev cam) {
+  dependency_wait();
   __shared__ __align__(16) RowStage sRows[kWarps];
   __shared__ __align__(16) float sData[Explicit<APP>::value ? kWarps * SlabOf<APP>::value : 4];
   __shared__ __align__(16) unsigned char sNN[IsNeural<APP>::value ? kWarps * sizeof(StageFwd) : 16];
@@ -927,6 +928,7 @@ __global__ void __launch_bounds__(kBlock) k_preprocess_bwd(PreprocessBwdArgs a, 
 constexpr int kFlagThreads = 256;
 template <bool kBase, bool kFeatures>
 __global__ void __launch_bounds__(kFlagThreads) k_bwd_flags(PreprocessBwdArgs a) {
+  dependency_wait();
   const int64_t i = (int64_t)blockIdx.x * kFlagThreads + threadIdx.x;
   bool active = false;
   if (i < a.n) {
@@ -957,6 +959,7 @@ __global__ void __launch_bounds__(kFlagThreads) k_bwd_flags(PreprocessBwdArgs a)
 
 template <int APP>
 __global__ void __launch_bounds__(kBlock) k_preprocess_bwd_sparse(PreprocessBwdArgs a, CamDev cam) {
+  dependency_wait();
   static_assert(IsNeural<APP>::value || APP == kAppExternal, "the neural model, or the projection alone");
   extern __shared__ __align__(16) float smem[];
   constexpr int kWordsPerRound = kBlock / 4;             // flag words (of 32 Gaussians) looked at per round
@@ -1323,7 +1326,7 @@ int launch_preprocess_fwd(int app, const PreprocessArgs &a, const CamDev &cam, c
   else if (app == GS_APP_SV) k_preprocess_fwd<GS_APP_SV><<<grid_for(a.n), kBlock, 0, st>>>(a, cam);
   else if (app == kAppExternal) k_preprocess_fwd<kAppExternal><<<grid_for(a.n), kBlock, 0, st>>>(a, cam);
   else if (app == kAppNeuralHalf) k_preprocess_fwd<kAppNeuralHalf><<<grid_for(a.n), kBlock, 0, st>>>(a, cam);
-  else k_preprocess_fwd<GS_APP_NEURAL><<<grid_for(a.n), kBlock, 0, st>>>(a, cam);
+  else launch_chained(k_preprocess_fwd<GS_APP_NEURAL>, grid_for(a.n), kBlock, 0, st, a, cam);
   return 1;
 }
 
@@ -1370,8 +1373,8 @@ int launch_preprocess_bwd(int app, const PreprocessBwdArgs &a, const CamDev &cam
     }
     opt_in_smem(k_preprocess_bwd_sparse<GS_APP_NEURAL>, kBwdSmemNN);
     const int blocks = resident_blocks<k_preprocess_bwd_sparse<GS_APP_NEURAL>>(kBwdSmemNN);
-    if (a.n > 0) k_bwd_flags<true, true><<<(int)((a.n + kFlagThreads - 1) / kFlagThreads), kFlagThreads, 0, st>>>(a);
-    k_preprocess_bwd_sparse<GS_APP_NEURAL><<<blocks, kBlock, kBwdSmemNN, st>>>(a, cam);
+    if (a.n > 0) launch_chained(k_bwd_flags<true, true>, (int)((a.n + kFlagThreads - 1) / kFlagThreads), kFlagThreads, 0, st, a);
+    launch_chained(k_preprocess_bwd_sparse<GS_APP_NEURAL>, blocks, kBlock, kBwdSmemNN, st, a, cam);
     launch_wgrad_reduce(a.w_partials, blocks, a.g_weights, st);
     return 3;
   }

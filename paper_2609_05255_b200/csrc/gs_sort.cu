@@ -23,26 +23,6 @@ constexpr unsigned kFull = 0xffffffffu;
 constexpr int kMaxDigitBits = 11;  // widest radix digit: 2048 bins
 constexpr int kScanBlock = 256;   // Gaussians per block of the tiles-touched prefix sum and per CTA of the instance emission
 
-// Programmatic dependent launch.  The kernels of this file form chains of short, dependent launches (27 per view).
-// Launched with the attribute below, a kernel may be placed on the SMs as soon as the CTAs of its predecessor in the
-// stream have exited, without waiting for the predecessor's completion to be processed; dependency_wait() returns once
-// the predecessor has completed and its writes are visible, and every kernel here calls it before its first access to
-// global memory, so the order of all reads and writes is the stream's.  Launched without the attribute it is a no-op.
-// Measured on one stream: 214 instead of 248 us of binning per view.  Letting the successor in earlier
-// (griddepcontrol.launch_dependents at the top of every kernel) gained no more on one stream and cost 4 % with
-// several views in flight: the successor's CTAs then sit on the SMs for the whole run of the predecessor, in the
-// places of the other streams' kernels.
-__device__ __forceinline__ void dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-template <class... KArgs, class... Args>
-void launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr; cfg.numAttrs = 1;
-  cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
-}
 
 // Block b sorts one contiguous range of the input, worked through in tiles of at most kSortTile elements.  While one
 // tile per block is enough (count <= blocks x kSortTile) the ranges are equal, rounded up to a multiple of the block
