@@ -764,6 +764,7 @@ static_assert(sizeof(mlp::Weights) % 16 == 0, "staging areas must stay 16-byte a
 
 template <int APP>
 __global__ void __launch_bounds__(kBlock) k_preprocess_bwd(PreprocessBwdArgs a, CamDev cam) {
+  dependency_wait();
   extern __shared__ __align__(16) float smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   float *slab = smem + warp * SlabOf<APP>::value;   // SH / SV: this warp's slab of parameter rows
@@ -1322,10 +1323,10 @@ int resident_blocks(size_t smem_bytes, int cap = kWgradBlocks) {
 
 int launch_preprocess_fwd(int app, const PreprocessArgs &a, const CamDev &cam, cudaStream_t st) {
   if (a.n == 0) return 0;
-  if (app == GS_APP_SH) k_preprocess_fwd<GS_APP_SH><<<grid_for(a.n), kBlock, 0, st>>>(a, cam);
-  else if (app == GS_APP_SV) k_preprocess_fwd<GS_APP_SV><<<grid_for(a.n), kBlock, 0, st>>>(a, cam);
-  else if (app == kAppExternal) k_preprocess_fwd<kAppExternal><<<grid_for(a.n), kBlock, 0, st>>>(a, cam);
-  else if (app == kAppNeuralHalf) k_preprocess_fwd<kAppNeuralHalf><<<grid_for(a.n), kBlock, 0, st>>>(a, cam);
+  if (app == GS_APP_SH) launch_chained(k_preprocess_fwd<GS_APP_SH>, grid_for(a.n), kBlock, 0, st, a, cam);
+  else if (app == GS_APP_SV) launch_chained(k_preprocess_fwd<GS_APP_SV>, grid_for(a.n), kBlock, 0, st, a, cam);
+  else if (app == kAppExternal) launch_chained(k_preprocess_fwd<kAppExternal>, grid_for(a.n), kBlock, 0, st, a, cam);
+  else if (app == kAppNeuralHalf) launch_chained(k_preprocess_fwd<kAppNeuralHalf>, grid_for(a.n), kBlock, 0, st, a, cam);
   else launch_chained(k_preprocess_fwd<GS_APP_NEURAL>, grid_for(a.n), kBlock, 0, st, a, cam);
   return 1;
 }
@@ -1340,8 +1341,8 @@ int launch_unfused_prepare(int64_t n, const float *means, const CamDev &cam, con
 int launch_bwd_flags(const PreprocessBwdArgs &a, bool appearance_rows, cudaStream_t st) {
   if (a.n == 0) return 0;
   const int blocks = (int)((a.n + kFlagThreads - 1) / kFlagThreads);
-  if (appearance_rows) k_bwd_flags<true, true><<<blocks, kFlagThreads, 0, st>>>(a);
-  else k_bwd_flags<false, false><<<blocks, kFlagThreads, 0, st>>>(a);
+  if (appearance_rows) launch_chained(k_bwd_flags<true, true>, blocks, kFlagThreads, 0, st, a);
+  else launch_chained(k_bwd_flags<false, false>, blocks, kFlagThreads, 0, st, a);
   return 1;
 }
 
@@ -1349,25 +1350,25 @@ int launch_preprocess_bwd(int app, const PreprocessBwdArgs &a, const CamDev &cam
   if (app == GS_APP_SH) {
     if (a.n == 0) return 0;
     opt_in_smem(k_preprocess_bwd<GS_APP_SH>, kBwdSmemSH);
-    k_preprocess_bwd<GS_APP_SH><<<grid_for(a.n), kBlock, kBwdSmemSH, st>>>(a, cam);
+    launch_chained(k_preprocess_bwd<GS_APP_SH>, grid_for(a.n), kBlock, kBwdSmemSH, st, a, cam);
     return 1;
   } else if (app == GS_APP_SV) {
     if (a.n == 0) return 0;
     opt_in_smem(k_preprocess_bwd<GS_APP_SV>, kBwdSmemSV);
-    k_preprocess_bwd<GS_APP_SV><<<grid_for(a.n), kBlock, kBwdSmemSV, st>>>(a, cam);
+    launch_chained(k_preprocess_bwd<GS_APP_SV>, grid_for(a.n), kBlock, kBwdSmemSV, st, a, cam);
     return 1;
   } else if (app == kAppExternal) {
     if (a.n == 0) return 0;
     if (!flags_ready) launch_bwd_flags(a, false, st);
     const int wave = resident_blocks<k_preprocess_bwd_sparse<kAppExternal>>(sizeof(mlp::Weights), 1 << 20), chunks = grid_for(a.n);
-    k_preprocess_bwd_sparse<kAppExternal><<<chunks < wave ? chunks : wave, kBlock, sizeof(mlp::Weights), st>>>(a, cam);
+    launch_chained(k_preprocess_bwd_sparse<kAppExternal>, chunks < wave ? chunks : wave, kBlock, sizeof(mlp::Weights), st, a, cam);
     return flags_ready ? 1 : 2;
   } else {
     if (app == kAppNeuralHalf) {
       opt_in_smem(k_preprocess_bwd_sparse<kAppNeuralHalf>, kBwdSmemNN);
       const int blocks = resident_blocks<k_preprocess_bwd_sparse<kAppNeuralHalf>>(kBwdSmemNN);
-      if (a.n > 0) k_bwd_flags<true, true><<<(int)((a.n + kFlagThreads - 1) / kFlagThreads), kFlagThreads, 0, st>>>(a);
-      k_preprocess_bwd_sparse<kAppNeuralHalf><<<blocks, kBlock, kBwdSmemNN, st>>>(a, cam);
+      if (a.n > 0) launch_chained(k_bwd_flags<true, true>, (int)((a.n + kFlagThreads - 1) / kFlagThreads), kFlagThreads, 0, st, a);
+      launch_chained(k_preprocess_bwd_sparse<kAppNeuralHalf>, blocks, kBlock, kBwdSmemNN, st, a, cam);
       launch_wgrad_reduce(a.w_partials, blocks, a.g_weights, st);
       return 3;
     }
